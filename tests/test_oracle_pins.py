@@ -1,0 +1,208 @@
+"""Pins for the CPU oracle: each test ties oracle/rrf_oracle.py to something
+other than itself (LAPACK's dense Householder QR, an SVD, closed forms and the
+invariants the paper states), so that a dropped term, a wrong sign, index or
+transpose in the oracle fails at least one of them."""
+import numpy as np
+import pytest
+import scipy.linalg as sla
+
+from oracle import rrf_oracle as orc
+from paper_2608_28941_b200 import workloads as wl
+
+
+def _case(m=96, n=80, b=8, max_rank=48, seed=3, decay=3.0):
+    rng = np.random.default_rng(seed)
+    p = min(m, n)
+    u, _ = np.linalg.qr(rng.standard_normal((m, p)))
+    v, _ = np.linalg.qr(rng.standard_normal((n, p)))
+    s = np.exp(-np.arange(p) / decay)
+    A = (u * s) @ v.T
+    Om = rng.standard_normal((n, max_rank))
+    return A, Om, s, b, max_rank
+
+
+def _lapack_vtau(Y):
+    (h, tau), _ = sla.qr(Y, mode="raw")
+    V = np.tril(h, -1)[:, :Y.shape[1]]
+    V[np.arange(Y.shape[1]), np.arange(Y.shape[1])] = 1.0
+    return V, tau, np.triu(h[:Y.shape[1], :])
+
+
+# ---- P2 / Theorem 3.1: concatenated reflectors == dense Householder QR of A*Omega
+
+
+@pytest.mark.parametrize("b", [1, 4, 8])
+def test_reflectors_equal_dense_householder_qr(b):
+    A, Om, _, _, max_rank = _case(b=b, max_rank=48)
+    r = orc.rrf(A, Om, b, 0.0, max_rank)            # tol 0: runs to the cap
+    assert r.k == max_rank and r.status == orc.RRF_MAX_RANK_REACHED
+    V_ref, tau_ref, _ = _lapack_vtau(A @ Om[:, :r.k])
+    tau = np.concatenate([np.diag(r.T[:, i * b:(i + 1) * b]) for i in range(r.k // b)])
+    # block 0 agrees to round-off; block i is sampled from a residual of relative size
+    # sqrt(E_{i-1}/E_0) and loses digits in that proportion, hence the graded tolerance
+    prev = [r.normA2] + r.E_dir[:-1]
+    for i in range(r.k // b):
+        amp = np.sqrt(r.normA2 / prev[i])
+        blk = slice(i * b, (i + 1) * b)
+        assert np.max(np.abs(r.V[:, blk] - V_ref[:, blk])) < 2e-13 * amp, i
+        assert np.max(np.abs(tau[blk] - tau_ref[blk])) < 2e-13 * amp, i
+
+
+def test_panel_qr_matches_lapack():
+    rng = np.random.default_rng(0)
+    Y = rng.standard_normal((50, 7))
+    V, tau, T, R = orc.panel_qr(Y)
+    V_ref, tau_ref, R_ref = _lapack_vtau(Y)
+    assert np.allclose(V, V_ref, atol=1e-14)
+    assert np.allclose(tau, tau_ref, atol=1e-14)
+    assert np.allclose(R, R_ref, atol=1e-13)          # sign convention: R_jj = beta
+
+
+def test_house_closed_form():
+    v, tau, beta = orc.house(np.array([3.0, 4.0]))
+    assert beta == -5.0 and np.isclose(tau, 1.6) and np.allclose(v, [1.0, 0.5])
+    v, tau, beta = orc.house(np.array([-3.0, 4.0]))
+    assert beta == 5.0 and np.isclose(tau, 1.6) and np.allclose(v, [1.0, -0.5])
+    v, tau, beta = orc.house(np.array([2.0, 0.0, 0.0]))   # nothing to annihilate: H = I
+    assert tau == 0.0 and beta == 2.0 and np.allclose(v, [1, 0, 0])
+
+
+# ---- P5: compact WY factor
+
+
+def test_compact_wy_identities():
+    rng = np.random.default_rng(1)
+    Y = rng.standard_normal((40, 6))
+    V, tau, T, R = orc.panel_qr(Y)
+    H = np.eye(40)
+    for j in range(6):
+        H = H @ (np.eye(40) - tau[j] * np.outer(V[:, j], V[:, j]))
+    Q = np.eye(40) - V @ T @ V.T
+    assert np.allclose(Q, H, atol=1e-14)
+    assert np.allclose(np.diag(T), tau)
+    assert np.allclose(np.tril(T, -1), 0.0)
+    Tinv = np.linalg.inv(T)
+    assert np.allclose(Tinv + Tinv.T, V.T @ V, atol=1e-12)
+    assert np.allclose((Q.T @ Y)[:6], R, atol=1e-13)
+    assert np.allclose((Q.T @ Y)[6:], 0.0, atol=1e-13)
+
+
+# ---- P1, P3, P4: triangularity, orthogonality, Frobenius identity, B = Q^T A
+
+
+def test_invariants_of_a_run():
+    A, Om, s, b, max_rank = _case()
+    r = orc.rrf(A, Om, b, 1e-3, max_rank, keep_w=True)
+    assert r.status == orc.RRF_OK and 0 < r.k < max_rank
+    Q = orc.form_q(r.V, r.T, b)
+    k = r.k
+    assert np.linalg.norm(Q.T @ Q - np.eye(k)) < 1e-13
+    R = Q.T @ (A @ Om[:, :k])
+    assert np.max(np.abs(np.tril(R, -1))) < 1e-13 * np.linalg.norm(R)
+    assert np.allclose(r.B, Q.T @ A, atol=1e-14)
+    res2 = np.linalg.norm(A - Q @ r.B) ** 2
+    assert np.isclose(res2, r.normA2 - np.linalg.norm(r.B) ** 2, rtol=1e-9)
+    assert np.isclose(res2, r.E_dir[-1], rtol=1e-10)
+    assert np.isclose(r.E_sub[-1], r.E_dir[-1], rtol=1e-6)
+    assert np.sqrt(res2) <= 1e-3 * np.sqrt(r.normA2)
+    # apply_qt reproduces the working matrix; its top k rows are B
+    assert np.allclose(orc.apply_qt(r.V, r.T, b, A), r.W, atol=1e-14)
+
+
+# ---- brute force on tiny inputs: k is the first multiple of b meeting the tolerance
+
+
+@pytest.mark.parametrize("tol", [3e-1, 1e-2, 1e-4])
+def test_k_is_first_block_count_meeting_tolerance(tol):
+    A, Om, s, b, max_rank = _case(m=60, n=50, b=5, max_rank=40, seed=11, decay=3.0)
+    r = orc.rrf(A, Om, b, tol, max_rank)
+    nrm = np.linalg.norm(A)
+    expected = None
+    for k in range(0, max_rank + 1, b):
+        if k == 0:
+            err = nrm
+        else:
+            Qk, _ = np.linalg.qr(A @ Om[:, :k])
+            err = np.linalg.norm(A - Qk @ (Qk.T @ A))
+        if err <= tol * nrm:
+            expected = k
+            break
+    assert expected is not None
+    assert r.k == expected and r.status == orc.RRF_OK
+
+
+# ---- P6: Eckart-Young lower bound with the known singular values
+
+
+def test_eckart_young_bound():
+    A, Om, s, b, max_rank = _case()
+    for tol in (1e-1, 1e-2, 1e-4):
+        r = orc.rrf(A, Om, b, tol, max_rank)
+        tail = np.sqrt(np.sum(s[r.k:] ** 2))
+        err = np.sqrt(r.E_dir[-1])
+        assert err >= tail * (1 - 1e-10)
+        assert err <= tol * np.sqrt(r.normA2)
+        if r.k > b:   # and the block before did not meet it
+            assert np.sqrt(r.E_dir[-2]) > tol * np.sqrt(r.normA2)
+
+
+# ---- P7: run to completion
+
+
+def test_run_to_completion_tall():
+    A, Om, s, b, _ = _case(m=72, n=40, b=8, max_rank=40)
+    r = orc.rrf(A, Om, b, 0.0, 40, keep_w=True)
+    assert r.k == 40
+    Q = orc.form_q(r.V, r.T, b)
+    assert np.linalg.norm(A - Q @ r.B) < 1e-13 * np.linalg.norm(A)
+    assert np.linalg.norm(r.W[40:, :]) < 1e-13 * np.linalg.norm(A)
+
+
+# ---- P8: exact rank, zero matrix, b = 1
+
+
+def test_exact_rank_stops_at_rank():
+    rng = np.random.default_rng(5)
+    A = rng.standard_normal((64, 12)) @ rng.standard_normal((12, 48))
+    Om = rng.standard_normal((48, 32))
+    r = orc.rrf(A, Om, 4, 1e-10, 32)
+    assert r.k == 12 and r.status == orc.RRF_OK
+    assert r.E_dir[-1] <= 1e-24 * r.normA2
+
+
+def test_zero_matrix_gives_rank_zero():
+    Om = np.random.default_rng(0).standard_normal((10, 8))
+    r = orc.rrf(np.zeros((12, 10)), Om, 4, 1e-3, 8)
+    assert r.k == 0 and r.steps == 0 and r.status == orc.RRF_OK and r.B.shape == (0, 10)
+
+
+def test_absolute_tolerance_and_subtractive_estimator():
+    A, Om, s, b, max_rank = _case()
+    nrm = np.linalg.norm(A)
+    r_rel = orc.rrf(A, Om, b, 1e-2, max_rank)
+    r_abs = orc.rrf(A, Om, b, 1e-2 * nrm, max_rank, relative=False)
+    r_sub = orc.rrf(A, Om, b, 1e-2, max_rank, estimator="subtractive")
+    assert r_rel.k == r_abs.k == r_sub.k
+    assert np.array_equal(r_rel.B, r_sub.B)
+
+
+def test_permuted_rerun_is_the_same_problem():
+    A, Om, s, b, max_rank = _case()
+    r = orc.rrf(A, Om, b, 1e-3, max_rank)
+    rp = orc.permuted_rerun(A, Om, b, 1e-3, max_rank, seed=1)
+    assert r.k == rp.k
+    assert np.max(np.abs(r.B - rp.B)) < 1e-12 * np.max(np.abs(r.B))
+    assert np.max(np.abs(r.V - rp.V)) < 1e-8
+
+
+# ---- P9: the law of k does not depend on the singular vectors (diag stand-in)
+
+
+def test_diag_standin_predicts_same_rank():
+    w = wl.CONFIGS["cfg1"].scaled(256, 192, max_rank=128)
+    A, s = wl.make_matrix(w)
+    Om = wl.make_omega(w)
+    r = orc.rrf(A, Om, w.b, 1e-4, w.max_rank)
+    rd = orc.rrf(wl.diag_matrix(s, w.m, w.n), Om, w.b, 1e-4, w.max_rank)
+    assert abs(r.k - rd.k) <= w.b
+    assert np.isclose(np.linalg.svd(A, compute_uv=False)[:20], s[:20], rtol=1e-10).all()
