@@ -1,0 +1,176 @@
+/*
+ * rrf.h - C ABI of the B200 (sm_100a) blocked adaptive randomized range finder.
+ *
+ * The library computes, entirely on one GPU, the factorisation A ~= Q B of the
+ * paper's problem statement (Eqs. "A ~= Q Q^T A, Q^T Q = I_k" and "B = Q^T A"):
+ * an orthonormal basis Q (m x k) kept as Householder block reflectors
+ * Q = Q_0 Q_1 ... Q_{i-1}, Q_l = I - V_l T_l V_l^T (Eq. "Q_i = I_m - V_i T_i V_i^T"),
+ * the projected matrix B (k x n), and the rank k found from a Frobenius
+ * tolerance (Algorithm 2, "Householder Blocked Adaptive Randomized Range Finder").
+ *
+ * Conventions shared by every call
+ *   - Every matrix pointer is DEVICE memory, row-major (C order): element (i, j) of a
+ *     matrix with leading dimension ld is p[i*ld + j].  Leading dimensions are in
+ *     elements.  Pointers must be 16-byte aligned and ld*sizeof(element) must be a
+ *     multiple of 16 bytes (the tiles are fetched by TMA).
+ *   - The caller owns every buffer and the CUDA stream.  The library allocates device
+ *     memory only in rrf_create (a few hundred bytes of status words).
+ *   - Scalars and result structs are HOST memory.
+ *   - Every call returns an rrf_status_t; nothing throws, nothing exits.  Arguments are
+ *     validated before anything is launched.  Device-side waits are bounded: a wait
+ *     that gives up reports RRF_ERR_TIMEOUT and leaves the context usable.
+ *   - Block size b must be one of 8, 16, 32, 64, 128; max_rank must be a multiple of b
+ *     and at most min(m, n)  (the paper assumes all dimensions divisible by b; here
+ *     only max_rank has to be).
+ */
+#ifndef RRF_H_
+#define RRF_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct rrf_ctx* rrf_handle_t;
+
+typedef enum { RRF_F64 = 0, RRF_F32 = 1 } rrf_dtype_t;
+
+typedef enum {
+  RRF_OK = 0,
+  RRF_MAX_RANK_REACHED = 1,   /* success with information: rank cap hit before the tolerance */
+  RRF_ERR_INVALID_ARG = -1,
+  RRF_ERR_WORKSPACE = -2,     /* workspace too small, or a panel too tall for on-chip storage */
+  RRF_ERR_CUDA = -3,          /* a CUDA call failed; the raw code is in rrf_result_t.cuda_error */
+  RRF_ERR_TIMEOUT = -4,       /* a bounded device-side wait gave up */
+  RRF_ERR_NONFINITE = -5      /* A contains NaN or Inf */
+} rrf_status_t;
+
+/* Flags for rrf_params_t.flags */
+#define RRF_FLAG_INPLACE 1u     /* A itself is the working matrix (it is overwritten) */
+#define RRF_FLAG_FIXED_RANK 2u  /* ignore the tolerance, always run to max_rank (fixed-rank mode) */
+
+typedef struct {
+  int32_t dtype;            /* rrf_dtype_t: element type of A, Omega, V, T, B, Q */
+  int32_t b;                /* block size */
+  int32_t max_rank;         /* rank cap, multiple of b, <= min(m, n) */
+  int32_t estimator;        /* 0: stop on the residual norm ||W[r0+b:, :]||_F^2 (default);
+                               1: stop on the paper's E <- E - ||B_i||_F^2 (Algorithm 2, line 9) */
+  int64_t m, n;             /* A is m x n */
+  double tol;               /* the tolerance sigma of Algorithm 2 ... */
+  int32_t tol_is_relative;  /* ... taken as tol*||A||_F if non-zero */
+  uint32_t flags;
+  uint64_t seed;            /* seed of the built-in Gaussian generator (used when dOmegaT == NULL) */
+} rrf_params_t;
+
+typedef struct {
+  int32_t status;           /* rrf_status_t of the run */
+  int32_t k;                /* rank found: steps * b */
+  int32_t steps;            /* block steps executed */
+  int32_t cuda_error;       /* raw cudaError_t when status == RRF_ERR_CUDA */
+  double normA2;            /* ||A||_F^2 */
+  double sigma2;            /* squared absolute tolerance the loop compared against */
+  double E_sub;             /* final value of Algorithm 2's E = ||A||_F^2 - sum ||B_i||_F^2 */
+  double E_dir;             /* final ||W[k:, :]||_F^2 = ||A - Q B||_F^2 */
+} rrf_result_t;
+
+/* Create / destroy a context bound to one CUDA device.  rrf_create makes `device`
+ * current, queries its limits and allocates the context's status words. */
+rrf_status_t rrf_create(rrf_handle_t* out, int device);
+rrf_status_t rrf_destroy(rrf_handle_t h);
+
+/* Bytes of device workspace rrf_run needs for these parameters (Algorithm 2 keeps B in
+ * place of A; unless RRF_FLAG_INPLACE is set the working copy lives in the workspace). */
+rrf_status_t rrf_workspace_bytes(const rrf_params_t* p, size_t* bytes);
+
+/*
+ * rrf_run - Algorithm 2, every step on the device.
+ *
+ *   dA       m x n input (lda >= n).  Read-only unless RRF_FLAG_INPLACE.
+ *   dOmegaT  max_rank x n (ldo >= n): row j is the j-th Gaussian sample vector, i.e. the
+ *            transpose of the n x max_rank matrix whose column block i is Omega_i of
+ *            Algorithm 2 line 6.  NULL: drawn on the device from p->seed.
+ *   dV       m x max_rank (ldv >= max_rank): Householder vectors, unit lower trapezoidal,
+ *            block column i holds V_i in rows i*b.. and zeros above.  Columns >= k are
+ *            unspecified on return.
+ *   dT       b x max_rank, leading dimension max_rank: T_i (upper triangular) in columns i*b...
+ *   dB       max_rank x n (ldb >= n): rows 0..k-1 are B = Q^T A.  With RRF_FLAG_INPLACE,
+ *            dB may alias dA (ldb == lda).
+ *   d_workspace / workspace_bytes   at least rrf_workspace_bytes(), 256-byte aligned.
+ *   cuda_stream   a cudaStream_t (NULL: the default stream).  All work is enqueued on it;
+ *            the call synchronises it once, at the end, to read back the result.
+ *   h_E_sub_trace, h_E_dir_trace   optional HOST arrays of max_rank/b doubles receiving
+ *            both stopping quantities after every block step.
+ *
+ * The loop `while E > sigma^2` runs on the device: each kernel of a block step first
+ * reads a device flag and returns at once when the stop rule has fired, so there is no
+ * host round-trip per block.  Returns RRF_OK / RRF_MAX_RANK_REACHED, or an error (out->status
+ * is the same value).
+ */
+rrf_status_t rrf_run(rrf_handle_t h, const rrf_params_t* p,
+                     void* dA, int64_t lda,
+                     const void* dOmegaT, int64_t ldo,
+                     void* dV, int64_t ldv,
+                     void* dT,
+                     void* dB, int64_t ldb,
+                     void* d_workspace, size_t workspace_bytes,
+                     void* cuda_stream, rrf_result_t* out,
+                     double* h_E_sub_trace, double* h_E_dir_trace);
+
+/*
+ * rrf_panel_qr - Algorithm 2 line 7 on its own (LAPACK geqrt semantics): Householder QR of a
+ * tall device panel Y (rows x b, ldy >= b) into V (rows x b, ldv >= b, unit lower trapezoidal,
+ * explicit ones and zeros) and the compact-WY factor T (b x b, ldt >= b, upper triangular) with
+ * H_0 ... H_{b-1} = I - V T V^T.  Reflector convention: beta = -sign(alpha) ||x||, v_0 = 1,
+ * tau = (beta - alpha)/beta.  R is not returned.  Workspace: rrf_panel_workspace_bytes().
+ * Does not synchronise the stream; a timeout of the in-kernel grid barrier is reported by
+ * the next rrf_last_status() call.
+ */
+rrf_status_t rrf_panel_workspace_bytes(int32_t dtype, int64_t rows, int32_t b, size_t* bytes);
+rrf_status_t rrf_panel_qr(rrf_handle_t h, int32_t dtype, int64_t rows, int32_t b,
+                          const void* dY, int64_t ldy, void* dV, int64_t ldv,
+                          void* dT, int64_t ldt,
+                          void* d_workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
+ * rrf_apply_qt / rrf_apply_q - C <- Q^T C or C <- Q C for a device matrix C (m x ncols,
+ * ldc >= ncols) with Q = Q_0 ... Q_{k/b-1} given by V (m x k) and T (b x k, leading dimension
+ * ldt) as rrf_run returns them (Algorithm 2 line 8 applied block by block; "Applying Q resolves
+ * into a series of matrix-matrix products").  Workspace: rrf_apply_workspace_bytes().
+ * rrf_form_q writes the explicit basis Q = Q I[:, 0:k] (m x k, ldq >= k).  None of the three
+ * synchronises the stream.
+ */
+rrf_status_t rrf_apply_workspace_bytes(int32_t dtype, int64_t m, int64_t ncols, int32_t b, size_t* bytes);
+rrf_status_t rrf_apply_qt(rrf_handle_t h, int32_t dtype, int64_t m, int32_t b, int32_t k,
+                          const void* dV, int64_t ldv, const void* dT, int64_t ldt,
+                          void* dC, int64_t ldc, int64_t ncols,
+                          void* d_workspace, size_t workspace_bytes, void* cuda_stream);
+rrf_status_t rrf_apply_q(rrf_handle_t h, int32_t dtype, int64_t m, int32_t b, int32_t k,
+                         const void* dV, int64_t ldv, const void* dT, int64_t ldt,
+                         void* dC, int64_t ldc, int64_t ncols,
+                         void* d_workspace, size_t workspace_bytes, void* cuda_stream);
+rrf_status_t rrf_form_q(rrf_handle_t h, int32_t dtype, int64_t m, int32_t b, int32_t k,
+                        const void* dV, int64_t ldv, const void* dT, int64_t ldt,
+                        void* dQ, int64_t ldq,
+                        void* d_workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
+ * rrf_fill_omega - Algorithm 2 line 6: fill dOmegaT (nvec x n, ldo >= n) with i.i.d. standard
+ * Gaussians.  Counter-based: element (j, c) depends only on (seed, j, c) - Philox-4x32-10 keyed
+ * by the seed with counter (c/2, j), Box-Muller in double precision, rounded to dtype - so any
+ * block of vectors can be regenerated independently.  Does not synchronise the stream.
+ */
+rrf_status_t rrf_fill_omega(rrf_handle_t h, int32_t dtype, uint64_t seed, int64_t n, int32_t nvec,
+                            int32_t first_vec, void* dOmegaT, int64_t ldo, void* cuda_stream);
+
+/* Status word of the handle's device side (set by bounded waits), read with one small
+ * device-to-host copy after synchronising `cuda_stream`; clears it. */
+rrf_status_t rrf_last_status(rrf_handle_t h, void* cuda_stream);
+
+const char* rrf_status_string(rrf_status_t s);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* RRF_H_ */

@@ -44,17 +44,18 @@ RRF_MAX_RANK_REACHED = 1
 def house(x: np.ndarray):
     """Householder reflector of a vector (section 3, "factored form ... geqrf").
 
-    Returns (v, tau, beta) with v[0] = 1 and (I - tau v v^T) x = beta e_1.
+    Returns (v, tau, beta) with v[0] = 1 and (I - tau v v^T) x = beta e_1, in x's precision.
     """
-    x = np.asarray(x, dtype=np.float64)
+    x = np.asarray(x)
+    dt = x.dtype.type
     alpha = x[0]
     tail = x[1:]
     xnorm = np.sqrt(np.dot(tail, tail))
     v = np.zeros_like(x)
     v[0] = 1.0
     if xnorm == 0.0:
-        return v, 0.0, alpha
-    sign = 1.0 if alpha >= 0.0 else -1.0
+        return v, dt(0.0), alpha
+    sign = dt(1.0) if alpha >= 0.0 else dt(-1.0)
     beta = -sign * np.sqrt(alpha * alpha + xnorm * xnorm)
     tau = (beta - alpha) / beta
     v[1:] = tail / (alpha - beta)
@@ -69,11 +70,13 @@ def panel_qr(Y: np.ndarray):
     T is b x b upper triangular with H_0 H_1 ... H_{b-1} = I - V T V^T
     (Eq. "Q_i = I_m - V_i T_i V_i^T"), R is the b x b triangular factor.
     """
-    Y = np.array(Y, dtype=np.float64, copy=True)
+    Y = np.array(Y, copy=True)
+    if Y.dtype not in (np.float32, np.float64):
+        Y = Y.astype(np.float64)
     rows, b = Y.shape
-    V = np.zeros((rows, b))
-    tau = np.zeros(b)
-    T = np.zeros((b, b))
+    V = np.zeros((rows, b), dtype=Y.dtype)
+    tau = np.zeros(b, dtype=Y.dtype)
+    T = np.zeros((b, b), dtype=Y.dtype)
     for j in range(b):
         if j < rows:
             v, tau[j], beta = house(Y[j:, j])
@@ -105,23 +108,32 @@ class OracleResult:
     W: np.ndarray | None = None                 # final working matrix (m x n)
 
 
+def _sumsq(X: np.ndarray) -> float:
+    """Squared Frobenius norm, accumulated in float64 whatever X's precision."""
+    X64 = X.astype(np.float64, copy=False)
+    return float(np.sum(X64 * X64))
+
+
 def rrf(A: np.ndarray, Omega: np.ndarray, b: int, tol: float, max_rank: int,
-        relative: bool = True, estimator: str = "direct", keep_w: bool = False) -> OracleResult:
+        relative: bool = True, estimator: str = "direct", keep_w: bool = False,
+        dtype=np.float64) -> OracleResult:
     """Algorithm 2, in the paper's order.
 
     A: m x n; Omega: n x max_rank (block i uses columns i*b:(i+1)*b, i.e. the
     "fresh Gaussian" of line 6 is passed in); tol: sigma (relative to ||A||_F
-    if `relative`).
+    if `relative`).  `dtype` is the working precision: float64 is the oracle
+    proper; float32 reruns the same steps in single precision (the paper's
+    experiments are in single precision) and serves as the plain-fp32 yardstick.
     """
-    W = np.array(A, dtype=np.float64, copy=True)           # line 2: B <- A
-    Omega = np.asarray(Omega, dtype=np.float64)
+    W = np.array(A, dtype=dtype, copy=True)                 # line 2: B <- A
+    Omega = np.asarray(Omega, dtype=dtype)
     m, n = W.shape
     assert b >= 1 and max_rank % b == 0 and max_rank <= min(m, n)
     assert Omega.shape[0] == n and Omega.shape[1] >= max_rank
-    normA2 = float(np.sum(W * W))                           # line 1: E <- ||A||_F^2
+    normA2 = _sumsq(W)                                      # line 1: E <- ||A||_F^2
     sigma2 = (tol * tol * normA2) if relative else tol * tol
-    V = np.zeros((m, max_rank))                             # line 3
-    T = np.zeros((b, max_rank))
+    V = np.zeros((m, max_rank), dtype=dtype)                # line 3
+    T = np.zeros((b, max_rank), dtype=dtype)
     res = OracleResult(0, RRF_OK, 0, normA2, sigma2, V, T, W)
     E_sub = normA2
     E = normA2
@@ -137,9 +149,9 @@ def rrf(A: np.ndarray, Omega: np.ndarray, b: int, tol: float, max_rank: int,
         Z = Ti.T @ Z
         W[r0:, :] -= Vi @ Z
         Bi = W[r0:r0 + b, :]
-        E_sub = E_sub - float(np.sum(Bi * Bi))              # line 9
+        E_sub = E_sub - _sumsq(Bi)                          # line 9
         trail = W[r0 + b:, :]
-        E_dir = float(np.sum(trail * trail))
+        E_dir = _sumsq(trail)
         res.E_sub.append(E_sub)
         res.E_dir.append(E_dir)
         E = E_dir if estimator == "direct" else E_sub

@@ -1,0 +1,652 @@
+// C ABI of the range finder: argument checks, workspace carving, tensor maps and the
+// enqueue of Algorithm 2's block loop.  See include/rrf.h for the contract of every call.
+#include <algorithm>
+#include <cstdio>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+
+#include "gemm.cuh"
+#include "panel.cuh"
+
+namespace rrf {
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+constexpr int kMaxSmem = 232448;   // 227 KB opt-in dynamic shared memory per CTA on sm_100
+constexpr int kTargetCtas = 296;   // split-K until about two CTAs per SM exist
+
+}  // namespace rrf
+
+struct rrf_ctx {
+  int device;
+  int sms;
+  int smem_optin;
+  rrf::EncodeTiledFn encode;
+  rrf::Ctrl* d_ctrl;     // status words for the calls that do not run Algorithm 2's loop
+  int last_cuda;
+  int panel_smem_max;    // dynamic shared memory the panel kernel may use (opt-in limit minus its static part)
+};
+
+namespace rrf {
+
+static inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+static inline int ceil_div(long long a, long long b) { return (int)((a + b - 1) / b); }
+
+// ------------------------------------------------------------------ tile configuration
+constexpr int kSampleBM = 128, kSampleStages = 4;
+constexpr int kVtwBN = 128, kVtwBK = 16, kVtwStages = 4;
+constexpr int kUpdBM = 64, kUpdBN = 64;
+
+struct SamplePlan { int nslabs, nseg, kt_per_seg; };
+struct VtwPlan { int ntiles, nseg, kt_per_seg, npad; };
+
+static SamplePlan plan_sample(long long rows, long long n, int esize) {
+  SamplePlan p;
+  const int KE = 128 / esize;
+  p.nslabs = ceil_div(rows, kSampleBM);
+  const int KT = ceil_div(n, KE);
+  int nseg = std::max(1, std::min(std::min(KT, 16), ceil_div(kTargetCtas, p.nslabs)));
+  p.kt_per_seg = ceil_div(KT, nseg);
+  p.nseg = ceil_div(KT, p.kt_per_seg);
+  return p;
+}
+static VtwPlan plan_vtw(long long rows, long long ncols) {
+  VtwPlan p;
+  p.ntiles = ceil_div(ncols, kVtwBN);
+  p.npad = p.ntiles * kVtwBN;
+  const int KT = ceil_div(rows, kVtwBK);
+  int nseg = std::max(1, std::min(std::min(KT, 32), ceil_div(kTargetCtas, p.ntiles)));
+  p.kt_per_seg = ceil_div(KT, nseg);
+  p.nseg = ceil_div(KT, p.kt_per_seg);
+  return p;
+}
+struct PanelPlan { int G, R, Rp; size_t smem; };
+static bool plan_panel(const rrf_ctx* h, long long rows, int b, PanelPlan* p) {
+  int R = std::max(32, ceil_div(rows, h->sms));
+  p->R = R;
+  p->G = ceil_div(rows, R);
+  // odd pitch keeps the transposing load/store phases bank-conflict free; the tallest panels
+  // (config 5: 222 rows x 128 columns per CTA) only fit without the padding
+  for (int Rp : {R | 1, R}) {
+    p->Rp = Rp;
+    p->smem = ((size_t)b * Rp + panel_extra_doubles(b)) * sizeof(double);
+    if (p->smem <= (size_t)h->panel_smem_max) return p->G <= h->sms;
+  }
+  return false;
+}
+static size_t panel_scratch_bytes(int sms, int b) {
+  // P[2][sms][b] + piv[2][b] + gram[b][b] + tau[b] (+ barrier word, padded)
+  return align_up(((size_t)2 * sms * b + 2 * (size_t)b + (size_t)b * b + b) * sizeof(double) + 256, 256);
+}
+struct PanelScratch { double *P, *piv, *gram, *tau; unsigned* bar; };
+static PanelScratch carve_panel(unsigned char* base, int sms, int b) {
+  PanelScratch s;
+  s.P = reinterpret_cast<double*>(base);
+  s.piv = s.P + (size_t)2 * sms * b;
+  s.gram = s.piv + 2 * (size_t)b;
+  s.tau = s.gram + (size_t)b * b;
+  s.bar = reinterpret_cast<unsigned*>(s.tau + b);
+  return s;
+}
+
+// ------------------------------------------------------------------ tensor maps
+static bool make_map(const rrf_ctx* h, CUtensorMap* map, int dtype, const void* base, unsigned long long rows,
+                     unsigned long long cols, unsigned long long ld, unsigned box_rows) {
+  const int esize = dtype == RRF_F64 ? 8 : 4;
+  cuuint64_t gdim[2] = {cols, rows};
+  cuuint64_t gstr[1] = {ld * (unsigned long long)esize};
+  cuuint32_t box[2] = {(cuuint32_t)(128 / esize), box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  const CUresult r = h->encode(map, dtype == RRF_F64 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT64 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32,
+                               2, const_cast<void*>(base), gdim, gstr, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                               CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS;
+}
+
+static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+static bool ld_ok(long long ld, long long mincols, int esize) { return ld >= mincols && (ld * esize) % 16 == 0; }
+static bool b_ok(int dtype, int b) {
+  if (dtype == RRF_F64) return b == 16 || b == 32 || b == 64 || b == 128;
+  if (dtype == RRF_F32) return b == 32 || b == 64 || b == 128;
+  return false;
+}
+
+// ------------------------------------------------------------------ typed launchers
+template <typename T, int B>
+struct Ops {
+  // sample
+  static constexpr int S_WM = (B == 16) ? 8 : 4, S_WN = (B == 16) ? 1 : 2;
+  static constexpr int S_SMEM = kSampleStages * (kSampleBM + B) * 128 + 1024;
+  // vtw: M = B
+  static constexpr int V_WM = (B == 16) ? 1 : (B == 128 ? 4 : 2), V_WN = 8 / V_WM;
+  static constexpr int V_SMEM = kVtwStages * kVtwBK * (B + kVtwBN) * (int)sizeof(T) + 1024;
+  // update
+  static constexpr int U_SMEM = B * (int)sizeof(T) * (kUpdBM + kUpdBN) + 1024;
+
+  static cudaError_t setup() {
+    cudaError_t e;
+    e = cudaFuncSetAttribute(sample_kernel<T, B, kSampleBM, S_WM, S_WN, kSampleStages>,
+                             cudaFuncAttributeMaxDynamicSharedMemorySize, S_SMEM);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(vtw_kernel<T, B, kVtwBN, kVtwBK, V_WM, V_WN, kVtwStages>,
+                             cudaFuncAttributeMaxDynamicSharedMemorySize, V_SMEM);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(update_kernel<T, B, kUpdBM, kUpdBN, 2, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             U_SMEM);
+    return e;
+  }
+  static void sample(const CUtensorMap& tmW, const CUtensorMap& tmO, void* Ypart, int r0, int rows, int n, int j0,
+                     const SamplePlan& p, Ctrl* ctrl, cudaStream_t st) {
+    sample_kernel<T, B, kSampleBM, S_WM, S_WN, kSampleStages>
+        <<<dim3(p.nslabs, p.nseg), S_WM * S_WN * 32, S_SMEM, st>>>(tmW, tmO, (T*)Ypart, r0, rows, n, j0, p.kt_per_seg,
+                                                                     ctrl);
+  }
+  static void vtw(const CUtensorMap& tmV, const CUtensorMap& tmC, void* Zpart, int r0, int rows, int cv0,
+                  const VtwPlan& p, Ctrl* ctrl, cudaStream_t st) {
+    vtw_kernel<T, B, kVtwBN, kVtwBK, V_WM, V_WN, kVtwStages>
+        <<<dim3(p.ntiles, p.nseg), 256, V_SMEM, st>>>(tmV, tmC, (T*)Zpart, r0, rows, cv0, p.npad, p.kt_per_seg, ctrl);
+  }
+  static void update(const CUtensorMap& tmV, const CUtensorMap& tmZ, void* C, long long ldc, void* top,
+                     long long ldtop, int r0, int rows, int ncols, int cv0, int top_rows, double* norm_part,
+                     Ctrl* ctrl, cudaStream_t st) {
+    dim3 grid(ceil_div(ncols, kUpdBN), ceil_div(rows, kUpdBM));
+    update_kernel<T, B, kUpdBM, kUpdBN, 2, 2><<<grid, 128, U_SMEM, st>>>(
+        tmV, tmZ, (T*)C, ldc, (T*)top, ldtop, r0, rows, ncols, cv0, top_rows, norm_part, ctrl);
+  }
+};
+
+struct OpTable {
+  cudaError_t (*setup)();
+  void (*sample)(const CUtensorMap&, const CUtensorMap&, void*, int, int, int, int, const SamplePlan&, Ctrl*,
+                 cudaStream_t);
+  void (*vtw)(const CUtensorMap&, const CUtensorMap&, void*, int, int, int, const VtwPlan&, Ctrl*, cudaStream_t);
+  void (*update)(const CUtensorMap&, const CUtensorMap&, void*, long long, void*, long long, int, int, int, int, int,
+                 double*, Ctrl*, cudaStream_t);
+};
+template <typename T, int B>
+static OpTable make_ops() {
+  return OpTable{&Ops<T, B>::setup, &Ops<T, B>::sample, &Ops<T, B>::vtw, &Ops<T, B>::update};
+}
+static const OpTable* get_ops(int dtype, int b) {
+  static const OpTable d16 = make_ops<double, 16>(), d32 = make_ops<double, 32>(), d64 = make_ops<double, 64>(),
+                       d128 = make_ops<double, 128>(), f32 = make_ops<float, 32>(), f64 = make_ops<float, 64>(),
+                       f128 = make_ops<float, 128>();
+  if (dtype == RRF_F64) {
+    switch (b) {
+      case 16: return &d16;
+      case 32: return &d32;
+      case 64: return &d64;
+      case 128: return &d128;
+    }
+  } else if (dtype == RRF_F32) {
+    switch (b) {
+      case 32: return &f32;
+      case 64: return &f64;
+      case 128: return &f128;
+    }
+  }
+  return nullptr;
+}
+
+// panel QR + T factor, enqueued on `st`
+static rrf_status_t launch_panel(rrf_ctx* h, int dtype, const void* Y, int nseg, long long seg_stride, int ldy,
+                                 long long rows, int b, void* V, long long ldv, void* Tout, long long ldt,
+                                 const PanelScratch& ps, Ctrl* ctrl, const int* done_flag, cudaStream_t st) {
+  PanelPlan pp;
+  if (!plan_panel(h, rows, b, &pp)) return RRF_ERR_WORKSPACE;
+  int rows_i = (int)rows, R = pp.R, Rp = pp.Rp;
+  double *P = ps.P, *piv = ps.piv, *gram = ps.gram, *tau = ps.tau;
+  unsigned* bar = ps.bar;
+  void* args[] = {&Y, &nseg, &seg_stride, &ldy, &rows_i, &b, &R, &Rp, &V, &ldv, &P, &piv, &gram, &tau, &bar, &ctrl,
+                  &done_flag};
+  cudaError_t e;
+  const size_t tsmem = ((size_t)b * (b + 1) + b) * sizeof(double);
+  if (dtype == RRF_F64) {
+    e = cudaLaunchCooperativeKernel((void*)panel_kernel<double>, dim3(pp.G), dim3(kPanelThreads), args, pp.smem, st);
+    if (e == cudaSuccess) {
+      tfactor_kernel<double><<<1, 128, tsmem, st>>>(gram, tau, b, (double*)Tout, ldt, done_flag);
+      e = cudaGetLastError();
+    }
+  } else {
+    e = cudaLaunchCooperativeKernel((void*)panel_kernel<float>, dim3(pp.G), dim3(kPanelThreads), args, pp.smem, st);
+    if (e == cudaSuccess) {
+      tfactor_kernel<float><<<1, 128, tsmem, st>>>(gram, tau, b, (float*)Tout, ldt, done_flag);
+      e = cudaGetLastError();
+    }
+  }
+  if (e != cudaSuccess) {
+    h->last_cuda = (int)e;
+    return RRF_ERR_CUDA;
+  }
+  return RRF_OK;
+}
+
+static void launch_tz(int dtype, const void* Zpart, int nseg, int npad, int b, const void* Tm, long long ldt,
+                      int transpose_t, void* Zt, const int* done_flag, cudaStream_t st) {
+  const size_t smem = ((size_t)b * (b + 1) + (size_t)kTzCols * (b + 1)) * sizeof(double);
+  if (dtype == RRF_F64)
+    tz_kernel<double><<<npad / kTzCols, 256, smem, st>>>((const double*)Zpart, nseg, npad, b, (const double*)Tm, ldt,
+                                                          transpose_t, (double*)Zt, done_flag);
+  else
+    tz_kernel<float><<<npad / kTzCols, 256, smem, st>>>((const float*)Zpart, nseg, npad, b, (const float*)Tm, ldt,
+                                                         transpose_t, (float*)Zt, done_flag);
+}
+
+static cudaError_t setup_all(int smem_optin, int* panel_smem_max) {
+  cudaError_t e;
+  for (int b : {16, 32, 64, 128}) {
+    e = get_ops(RRF_F64, b)->setup();
+    if (e != cudaSuccess) return e;
+  }
+  for (int b : {32, 64, 128}) {
+    e = get_ops(RRF_F32, b)->setup();
+    if (e != cudaSuccess) return e;
+  }
+  cudaFuncAttributes fa, fb;
+  e = cudaFuncGetAttributes(&fa, panel_kernel<double>);
+  if (e != cudaSuccess) return e;
+  e = cudaFuncGetAttributes(&fb, panel_kernel<float>);
+  if (e != cudaSuccess) return e;
+  *panel_smem_max = std::min(smem_optin, kMaxSmem) - (int)std::max(fa.sharedSizeBytes, fb.sharedSizeBytes);
+  e = cudaFuncSetAttribute(panel_kernel<double>, cudaFuncAttributeMaxDynamicSharedMemorySize, *panel_smem_max);
+  if (e != cudaSuccess) return e;
+  e = cudaFuncSetAttribute(panel_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, *panel_smem_max);
+  if (e != cudaSuccess) return e;
+  const int tmax = (128 * 129 + 128) * 8;
+  e = cudaFuncSetAttribute(tfactor_kernel<double>, cudaFuncAttributeMaxDynamicSharedMemorySize, tmax);
+  if (e != cudaSuccess) return e;
+  e = cudaFuncSetAttribute(tfactor_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, tmax);
+  if (e != cudaSuccess) return e;
+  const int zmax = (128 * 129 + kTzCols * 129) * 8;
+  e = cudaFuncSetAttribute(tz_kernel<double>, cudaFuncAttributeMaxDynamicSharedMemorySize, zmax);
+  if (e != cudaSuccess) return e;
+  e = cudaFuncSetAttribute(tz_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, zmax);
+  return e;
+}
+
+// ------------------------------------------------------------------ workspace of rrf_run
+struct RunLayout {
+  size_t ctrl, traces, norm_part, init_part, ypart, zpart, zt, panel, w, omega, total;
+  int init_ctas, max_norm_parts;
+  long long ldw;
+};
+constexpr int kInitCtas = 148 * 8;
+
+static bool run_layout(const rrf_params_t* p, bool need_omega, RunLayout* L) {
+  const int esize = p->dtype == RRF_F64 ? 8 : 4;
+  const int b = p->b, steps = p->max_rank / b;
+  size_t ymax = 0, zmax = 0;
+  int npad = 0, normmax = 0;
+  for (int i = 0; i < steps; ++i) {
+    const long long rows = p->m - (long long)i * b;
+    const SamplePlan sp = plan_sample(rows, p->n, esize);
+    ymax = std::max(ymax, (size_t)sp.nseg * (size_t)rows * b);
+    const VtwPlan vp = plan_vtw(rows, p->n);
+    zmax = std::max(zmax, (size_t)vp.nseg * b * (size_t)vp.npad);
+    npad = vp.npad;
+    normmax = std::max(normmax, ceil_div(p->n, kUpdBN) * ceil_div(rows, kUpdBM));
+  }
+  size_t off = 0;
+  L->ctrl = off; off += 256;
+  L->traces = off; off += align_up((size_t)2 * steps * sizeof(double), 256);
+  L->init_ctas = kInitCtas;
+  L->init_part = off; off += align_up((size_t)kInitCtas * sizeof(double), 256);
+  L->max_norm_parts = normmax;
+  L->norm_part = off; off += align_up((size_t)2 * normmax * sizeof(double), 256);
+  L->ypart = off; off += align_up(ymax * esize, 256);
+  L->zpart = off; off += align_up(zmax * esize, 256);
+  L->zt = off; off += align_up((size_t)npad * b * esize, 256);
+  L->panel = off; off += panel_scratch_bytes(148 * 2, b);
+  L->w = off;
+  L->ldw = (long long)align_up((size_t)p->n, 16);   // rows of the working copy start on 128-byte lines
+  if (!(p->flags & RRF_FLAG_INPLACE)) off += align_up((size_t)p->m * (size_t)L->ldw * esize, 256);
+  L->omega = off;
+  if (need_omega) off += align_up((size_t)p->max_rank * (size_t)p->n * esize, 256);
+  L->total = off;
+  return true;
+}
+
+static rrf_status_t check_params(const rrf_params_t* p) {
+  if (p == nullptr) return RRF_ERR_INVALID_ARG;
+  if (p->dtype != RRF_F64 && p->dtype != RRF_F32) return RRF_ERR_INVALID_ARG;
+  if (!b_ok(p->dtype, p->b)) return RRF_ERR_INVALID_ARG;
+  if (p->m < 1 || p->n < 1 || p->m > 0x7fffffffLL || p->n > 0x7fffffffLL) return RRF_ERR_INVALID_ARG;
+  if (p->max_rank < p->b || p->max_rank % p->b != 0) return RRF_ERR_INVALID_ARG;
+  if (p->max_rank > p->m || p->max_rank > p->n) return RRF_ERR_INVALID_ARG;
+  if (!(p->tol >= 0.0)) return RRF_ERR_INVALID_ARG;
+  if (p->estimator != 0 && p->estimator != 1) return RRF_ERR_INVALID_ARG;
+  return RRF_OK;
+}
+
+}  // namespace rrf
+
+using namespace rrf;
+
+extern "C" {
+
+const char* rrf_status_string(rrf_status_t s) {
+  switch (s) {
+    case RRF_OK: return "ok";
+    case RRF_MAX_RANK_REACHED: return "rank cap reached before the tolerance";
+    case RRF_ERR_INVALID_ARG: return "invalid argument";
+    case RRF_ERR_WORKSPACE: return "workspace too small or panel too tall";
+    case RRF_ERR_CUDA: return "CUDA error";
+    case RRF_ERR_TIMEOUT: return "bounded device-side wait gave up";
+    case RRF_ERR_NONFINITE: return "input contains NaN or Inf";
+  }
+  return "unknown status";
+}
+
+rrf_status_t rrf_create(rrf_handle_t* out, int device) {
+  if (out == nullptr) return RRF_ERR_INVALID_ARG;
+  *out = nullptr;
+  if (cudaSetDevice(device) != cudaSuccess) return RRF_ERR_CUDA;
+  rrf_ctx* h = new (std::nothrow) rrf_ctx();
+  if (h == nullptr) return RRF_ERR_CUDA;
+  h->device = device;
+  h->last_cuda = 0;
+  cudaError_t e = cudaDeviceGetAttribute(&h->sms, cudaDevAttrMultiProcessorCount, device);
+  if (e == cudaSuccess) e = cudaDeviceGetAttribute(&h->smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, device);
+  void* fn = nullptr;
+  cudaDriverEntryPointQueryResult q;
+  if (e == cudaSuccess) e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q);
+  if (e == cudaSuccess && (fn == nullptr || q != cudaDriverEntryPointSuccess)) e = cudaErrorUnknown;
+  h->encode = reinterpret_cast<EncodeTiledFn>(fn);
+  if (e == cudaSuccess) e = setup_all(h->smem_optin, &h->panel_smem_max);
+  if (e == cudaSuccess) e = cudaMalloc(&h->d_ctrl, sizeof(Ctrl));
+  if (e == cudaSuccess) e = cudaMemset(h->d_ctrl, 0, sizeof(Ctrl));
+  if (e != cudaSuccess) {
+    if (std::getenv("RRF_VERBOSE")) std::fprintf(stderr, "rrf_create: %s\n", cudaGetErrorString(e));
+    delete h;
+    return RRF_ERR_CUDA;
+  }
+  if (h->smem_optin > kMaxSmem) h->smem_optin = kMaxSmem;
+  *out = h;
+  return RRF_OK;
+}
+
+rrf_status_t rrf_destroy(rrf_handle_t h) {
+  if (h == nullptr) return RRF_ERR_INVALID_ARG;
+  cudaSetDevice(h->device);
+  cudaFree(h->d_ctrl);
+  delete h;
+  return RRF_OK;
+}
+
+rrf_status_t rrf_last_status(rrf_handle_t h, void* cuda_stream) {
+  if (h == nullptr) return RRF_ERR_INVALID_ARG;
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  Ctrl c;
+  if (cudaMemcpyAsync(&c, h->d_ctrl, sizeof(Ctrl), cudaMemcpyDeviceToHost, st) != cudaSuccess) return RRF_ERR_CUDA;
+  if (cudaStreamSynchronize(st) != cudaSuccess) return RRF_ERR_CUDA;
+  if (c.status != 0) cudaMemsetAsync(h->d_ctrl, 0, sizeof(Ctrl), st);
+  return (rrf_status_t)c.status;
+}
+
+rrf_status_t rrf_workspace_bytes(const rrf_params_t* p, size_t* bytes) {
+  if (bytes == nullptr) return RRF_ERR_INVALID_ARG;
+  const rrf_status_t s = check_params(p);
+  if (s != RRF_OK) return s;
+  RunLayout L;
+  run_layout(p, true, &L);
+  *bytes = L.total;
+  return RRF_OK;
+}
+
+rrf_status_t rrf_fill_omega(rrf_handle_t h, int32_t dtype, uint64_t seed, int64_t n, int32_t nvec, int32_t first_vec,
+                            void* dOmegaT, int64_t ldo, void* cuda_stream) {
+  if (h == nullptr || dOmegaT == nullptr || n < 1 || nvec < 1 || first_vec < 0 || ldo < n) return RRF_ERR_INVALID_ARG;
+  if (dtype != RRF_F64 && dtype != RRF_F32) return RRF_ERR_INVALID_ARG;
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  const long long total = ((n + 1) / 2) * nvec;
+  const int grid = (int)std::min<long long>((total + 255) / 256, (long long)h->sms * 16);
+  if (dtype == RRF_F64)
+    omega_kernel<double><<<grid, 256, 0, st>>>((double*)dOmegaT, ldo, n, nvec, first_vec, seed);
+  else
+    omega_kernel<float><<<grid, 256, 0, st>>>((float*)dOmegaT, ldo, n, nvec, first_vec, seed);
+  const cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) {
+    h->last_cuda = (int)e;
+    return RRF_ERR_CUDA;
+  }
+  return RRF_OK;
+}
+
+rrf_status_t rrf_panel_workspace_bytes(int32_t dtype, int64_t rows, int32_t b, size_t* bytes) {
+  if (bytes == nullptr || !b_ok(dtype, b) || rows < b) return RRF_ERR_INVALID_ARG;
+  *bytes = panel_scratch_bytes(148 * 2, b);
+  return RRF_OK;
+}
+
+rrf_status_t rrf_panel_qr(rrf_handle_t h, int32_t dtype, int64_t rows, int32_t b, const void* dY, int64_t ldy,
+                          void* dV, int64_t ldv, void* dT, int64_t ldt, void* d_workspace, size_t workspace_bytes,
+                          void* cuda_stream) {
+  if (h == nullptr || dY == nullptr || dV == nullptr || dT == nullptr || d_workspace == nullptr)
+    return RRF_ERR_INVALID_ARG;
+  if (!b_ok(dtype, b) || rows < b || rows > 0x7fffffffLL || ldy < b || ldv < b || ldt < b || ldy > 0x7fffffffLL)
+    return RRF_ERR_INVALID_ARG;
+  if (workspace_bytes < panel_scratch_bytes(148 * 2, b) || h->sms > 148 * 2) return RRF_ERR_WORKSPACE;
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  PanelScratch ps = carve_panel((unsigned char*)d_workspace, h->sms, b);
+  if (cudaMemsetAsync(ps.bar, 0, sizeof(unsigned), st) != cudaSuccess) return RRF_ERR_CUDA;
+  return launch_panel(h, dtype, dY, 1, 0, (int)ldy, rows, b, dV, ldv, dT, ldt, ps, h->d_ctrl, &h->d_ctrl->done, st);
+}
+
+rrf_status_t rrf_apply_workspace_bytes(int32_t dtype, int64_t m, int64_t ncols, int32_t b, size_t* bytes) {
+  if (bytes == nullptr || !b_ok(dtype, b) || m < b || ncols < 1) return RRF_ERR_INVALID_ARG;
+  const int esize = dtype == RRF_F64 ? 8 : 4;
+  const VtwPlan vp = plan_vtw(m, ncols);   // the first block has the most rows and segments are capped
+  size_t zmax = 0;
+  for (long long r0 = 0; r0 + b <= m; r0 += b) {
+    const VtwPlan q = plan_vtw(m - r0, ncols);
+    zmax = std::max(zmax, (size_t)q.nseg * b * (size_t)q.npad);
+  }
+  *bytes = align_up(zmax * esize, 256) + align_up((size_t)vp.npad * b * esize, 256);
+  return RRF_OK;
+}
+
+}  // extern "C"
+
+namespace rrf {
+
+// C <- Q^T C (forward over the blocks, T^T) or C <- Q C (backward, T).
+static rrf_status_t apply_blocks(rrf_handle_t h, int dtype, long long m, int b, int k, const void* dV, long long ldv,
+                                 const void* dT, long long ldt, void* dC, long long ldc, long long ncols,
+                                 void* d_workspace, size_t workspace_bytes, cudaStream_t st, bool transpose) {
+  if (h == nullptr || dV == nullptr || dT == nullptr || dC == nullptr || d_workspace == nullptr)
+    return RRF_ERR_INVALID_ARG;
+  const int esize = dtype == RRF_F64 ? 8 : 4;
+  if (!b_ok(dtype, b) || k < 0 || k % b != 0 || k > m || m > 0x7fffffffLL || ncols < 1 || ncols > 0x7fffffffLL)
+    return RRF_ERR_INVALID_ARG;
+  if (!ld_ok(ldv, k, esize) || !ld_ok(ldc, ncols, esize) || ldt < k || !aligned16(dV) || !aligned16(dC))
+    return RRF_ERR_INVALID_ARG;
+  size_t need = 0;
+  if (rrf_apply_workspace_bytes(dtype, m, ncols, b, &need) != RRF_OK) return RRF_ERR_INVALID_ARG;
+  if (workspace_bytes < need || (reinterpret_cast<uintptr_t>(d_workspace) & 255u)) return RRF_ERR_WORKSPACE;
+  if (k == 0) return RRF_OK;
+  const OpTable* ops = get_ops(dtype, b);
+  const VtwPlan vp0 = plan_vtw(m, ncols);
+  unsigned char* ws = (unsigned char*)d_workspace;
+  void* Zt = ws;
+  void* Zpart = ws + align_up((size_t)vp0.npad * b * esize, 256);
+  CUtensorMap tmV_k, tmC_k, tmV_u, tmZ;
+  if (!make_map(h, &tmV_k, dtype, dV, m, k, ldv, kVtwBK) || !make_map(h, &tmC_k, dtype, dC, m, ncols, ldc, kVtwBK) ||
+      !make_map(h, &tmV_u, dtype, dV, m, k, ldv, kUpdBM) || !make_map(h, &tmZ, dtype, Zt, vp0.npad, b, b, kUpdBN))
+    return RRF_ERR_INVALID_ARG;
+  const int nblk = k / b;
+  for (int q = 0; q < nblk; ++q) {
+    const int l = transpose ? q : nblk - 1 - q;
+    const int r0 = l * b, rows = (int)(m - r0);
+    const VtwPlan vp = plan_vtw(rows, ncols);
+    ops->vtw(tmV_k, tmC_k, Zpart, r0, rows, r0, vp, h->d_ctrl, st);
+    launch_tz(dtype, Zpart, vp.nseg, vp.npad, b, (const char*)dT + (size_t)r0 * esize, ldt, transpose ? 1 : 0, Zt,
+              &h->d_ctrl->done, st);
+    ops->update(tmV_u, tmZ, dC, ldc, (char*)dC + (size_t)r0 * ldc * esize, ldc, r0, rows, (int)ncols, r0, 0, nullptr,
+                h->d_ctrl, st);
+  }
+  const cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) {
+    h->last_cuda = (int)e;
+    return RRF_ERR_CUDA;
+  }
+  return RRF_OK;
+}
+
+}  // namespace rrf
+
+extern "C" {
+
+rrf_status_t rrf_apply_qt(rrf_handle_t h, int32_t dtype, int64_t m, int32_t b, int32_t k, const void* dV, int64_t ldv,
+                          const void* dT, int64_t ldt, void* dC, int64_t ldc, int64_t ncols, void* d_workspace,
+                          size_t workspace_bytes, void* cuda_stream) {
+  return apply_blocks(h, dtype, m, b, k, dV, ldv, dT, ldt, dC, ldc, ncols, d_workspace, workspace_bytes,
+                      (cudaStream_t)cuda_stream, true);
+}
+
+rrf_status_t rrf_apply_q(rrf_handle_t h, int32_t dtype, int64_t m, int32_t b, int32_t k, const void* dV, int64_t ldv,
+                         const void* dT, int64_t ldt, void* dC, int64_t ldc, int64_t ncols, void* d_workspace,
+                         size_t workspace_bytes, void* cuda_stream) {
+  return apply_blocks(h, dtype, m, b, k, dV, ldv, dT, ldt, dC, ldc, ncols, d_workspace, workspace_bytes,
+                      (cudaStream_t)cuda_stream, false);
+}
+
+rrf_status_t rrf_form_q(rrf_handle_t h, int32_t dtype, int64_t m, int32_t b, int32_t k, const void* dV, int64_t ldv,
+                        const void* dT, int64_t ldt, void* dQ, int64_t ldq, void* d_workspace, size_t workspace_bytes,
+                        void* cuda_stream) {
+  if (h == nullptr || dQ == nullptr || k < 1 || m < k || ldq < k) return RRF_ERR_INVALID_ARG;
+  if (dtype != RRF_F64 && dtype != RRF_F32) return RRF_ERR_INVALID_ARG;
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  const int grid = (int)std::min<long long>(((long long)m * k + 255) / 256, (long long)h->sms * 16);
+  if (dtype == RRF_F64)
+    eye_kernel<double><<<grid, 256, 0, st>>>((double*)dQ, ldq, m, k);
+  else
+    eye_kernel<float><<<grid, 256, 0, st>>>((float*)dQ, ldq, m, k);
+  return apply_blocks(h, dtype, m, b, k, dV, ldv, dT, ldt, dQ, ldq, k, d_workspace, workspace_bytes, st, false);
+}
+
+rrf_status_t rrf_run(rrf_handle_t h, const rrf_params_t* p, void* dA, int64_t lda, const void* dOmegaT, int64_t ldo,
+                     void* dV, int64_t ldv, void* dT, void* dB, int64_t ldb, void* d_workspace, size_t workspace_bytes,
+                     void* cuda_stream, rrf_result_t* out, double* h_E_sub_trace, double* h_E_dir_trace) {
+  if (out == nullptr) return RRF_ERR_INVALID_ARG;
+  std::memset(out, 0, sizeof(*out));
+  auto fail = [&](rrf_status_t s) {
+    out->status = s;
+    return s;
+  };
+  if (h == nullptr) return fail(RRF_ERR_INVALID_ARG);
+  rrf_status_t s = check_params(p);
+  if (s != RRF_OK) return fail(s);
+  const int esize = p->dtype == RRF_F64 ? 8 : 4;
+  const int b = p->b;
+  const long long m = p->m, n = p->n;
+  if (dA == nullptr || dV == nullptr || dT == nullptr || dB == nullptr || d_workspace == nullptr)
+    return fail(RRF_ERR_INVALID_ARG);
+  if (!ld_ok(lda, n, esize) || !ld_ok(ldv, p->max_rank, esize) || !ld_ok(ldb, n, esize))
+    return fail(RRF_ERR_INVALID_ARG);
+  if (dOmegaT != nullptr && (!ld_ok(ldo, n, esize) || !aligned16(dOmegaT))) return fail(RRF_ERR_INVALID_ARG);
+  if (!aligned16(dA) || !aligned16(dV) || !aligned16(dB) || (reinterpret_cast<uintptr_t>(d_workspace) & 255u))
+    return fail(RRF_ERR_INVALID_ARG);
+  RunLayout L;
+  run_layout(p, dOmegaT == nullptr, &L);
+  if (workspace_bytes < L.total) return fail(RRF_ERR_WORKSPACE);
+  if (h->sms > 148 * 2) return fail(RRF_ERR_WORKSPACE);
+  PanelPlan pp0;
+  if (!plan_panel(h, m, b, &pp0)) return fail(RRF_ERR_WORKSPACE);   // first (tallest) panel must fit on chip
+
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  if (cudaSetDevice(h->device) != cudaSuccess) return fail(RRF_ERR_CUDA);
+  unsigned char* ws = (unsigned char*)d_workspace;
+  Ctrl* ctrl = reinterpret_cast<Ctrl*>(ws + L.ctrl);
+  const int steps = p->max_rank / b;
+  double* tr_sub = reinterpret_cast<double*>(ws + L.traces);
+  double* tr_dir = tr_sub + steps;
+  double* init_part = reinterpret_cast<double*>(ws + L.init_part);
+  double* norm_part = reinterpret_cast<double*>(ws + L.norm_part);
+  void* Ypart = ws + L.ypart;
+  void* Zpart = ws + L.zpart;
+  void* Zt = ws + L.zt;
+  PanelScratch ps = carve_panel(ws + L.panel, h->sms, b);
+  ps.bar = &ctrl->bar;
+  const bool inplace = (p->flags & RRF_FLAG_INPLACE) != 0;
+  const bool fixed = (p->flags & RRF_FLAG_FIXED_RANK) != 0;
+  void* W = inplace ? dA : (void*)(ws + L.w);
+  const long long ldw = inplace ? lda : L.ldw;
+  const void* Om = dOmegaT;
+  long long ldom = ldo;
+  if (Om == nullptr) {
+    Om = ws + L.omega;
+    ldom = n;
+    s = rrf_fill_omega(h, p->dtype, p->seed, n, p->max_rank, 0, ws + L.omega, n, st);
+    if (s != RRF_OK) return fail(s);
+  }
+  const OpTable* ops = get_ops(p->dtype, b);
+  const int npad = plan_vtw(m, n).npad;
+  CUtensorMap tmW_s, tmO, tmV_k, tmW_k, tmV_u, tmZ;
+  if (!make_map(h, &tmW_s, p->dtype, W, m, n, ldw, kSampleBM) ||
+      !make_map(h, &tmO, p->dtype, Om, p->max_rank, n, ldom, b) ||
+      !make_map(h, &tmV_k, p->dtype, dV, m, p->max_rank, ldv, kVtwBK) ||
+      !make_map(h, &tmW_k, p->dtype, W, m, n, ldw, kVtwBK) ||
+      !make_map(h, &tmV_u, p->dtype, dV, m, p->max_rank, ldv, kUpdBM) ||
+      !make_map(h, &tmZ, p->dtype, Zt, npad, b, b, kUpdBN))
+    return fail(RRF_ERR_INVALID_ARG);
+
+  // Algorithm 2 lines 1-4
+  if (p->dtype == RRF_F64)
+    init_kernel<double><<<L.init_ctas, 256, 0, st>>>((const double*)dA, lda, inplace ? nullptr : (double*)W, ldw, m, n,
+                                                     (double*)dV, ldv, p->max_rank, init_part);
+  else
+    init_kernel<float><<<L.init_ctas, 256, 0, st>>>((const float*)dA, lda, inplace ? nullptr : (float*)W, ldw, m, n,
+                                                    (float*)dV, ldv, p->max_rank, init_part);
+  init_ctrl_kernel<<<1, 256, 0, st>>>(init_part, L.init_ctas, p->tol, p->tol_is_relative, fixed ? 1 : 0, b, p->max_rank,
+                                      ctrl);
+
+  // Algorithm 2 lines 5-11: every pass is enqueued; passes after the stop return at once
+  for (int i = 0; i < steps; ++i) {
+    const int r0 = i * b, rows = (int)(m - r0);
+    const SamplePlan sp = plan_sample(rows, n, esize);
+    ops->sample(tmW_s, tmO, Ypart, r0, rows, (int)n, r0, sp, ctrl, st);
+    s = launch_panel(h, p->dtype, Ypart, sp.nseg, (long long)rows * b, b, rows, b,
+                     (char*)dV + ((size_t)r0 * ldv + r0) * esize, ldv, (char*)dT + (size_t)r0 * esize, p->max_rank, ps,
+                     ctrl, &ctrl->done, st);
+    if (s != RRF_OK) {
+      out->cuda_error = h->last_cuda;
+      cudaStreamSynchronize(st);
+      return fail(s);
+    }
+    const VtwPlan vp = plan_vtw(rows, n);
+    ops->vtw(tmV_k, tmW_k, Zpart, r0, rows, r0, vp, ctrl, st);
+    launch_tz(p->dtype, Zpart, vp.nseg, vp.npad, b, (const char*)dT + (size_t)r0 * esize, p->max_rank, 1, Zt,
+              &ctrl->done, st);
+    ops->update(tmV_u, tmZ, W, ldw, (char*)dB + (size_t)r0 * ldb * esize, ldb, r0, rows, (int)n, r0, b, norm_part, ctrl,
+                st);
+    const int nparts = ceil_div(n, kUpdBN) * ceil_div(rows, kUpdBM);
+    stop_kernel<<<1, 256, 0, st>>>(norm_part, nparts, b, p->max_rank, p->estimator, fixed ? 1 : 0, tr_sub, tr_dir, ctrl);
+  }
+  cudaError_t e = cudaGetLastError();
+  Ctrl hc;
+  if (e == cudaSuccess) e = cudaMemcpyAsync(&hc, ctrl, sizeof(Ctrl), cudaMemcpyDeviceToHost, st);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+  if (e != cudaSuccess) {
+    h->last_cuda = (int)e;
+    out->cuda_error = (int)e;
+    return fail(RRF_ERR_CUDA);
+  }
+  out->status = hc.status;
+  out->k = hc.k;
+  out->steps = hc.steps;
+  out->normA2 = hc.normA2;
+  out->sigma2 = hc.sigma2;
+  out->E_sub = hc.E_sub;
+  out->E_dir = hc.E_dir;
+  if (hc.steps > 0) {
+    if (h_E_sub_trace != nullptr) cudaMemcpy(h_E_sub_trace, tr_sub, sizeof(double) * hc.steps, cudaMemcpyDeviceToHost);
+    if (h_E_dir_trace != nullptr) cudaMemcpy(h_E_dir_trace, tr_dir, sizeof(double) * hc.steps, cudaMemcpyDeviceToHost);
+  }
+  return (rrf_status_t)hc.status;
+}
+
+}  // extern "C"

@@ -1,0 +1,389 @@
+// Panel Householder QR (Algorithm 2 line 7, geqrt semantics) on the GPU, plus the small
+// kernels around it: compact-WY T factor, Z <- op(T) Z, norms, stop rule, Gaussian fill.
+#pragma once
+
+#include "common.cuh"
+
+namespace rrf {
+
+constexpr int kPanelThreads = 256;
+// doubles of shared memory the panel kernel needs besides the slab: w[b] and a region that holds
+// p[b], pivot_row[b] and, at another time, one partial per thread
+__host__ __device__ constexpr int panel_extra_doubles(int b) { return b + (2 * b > kPanelThreads ? 2 * b : kPanelThreads); }
+
+// Grid-wide barrier over a monotonically increasing arrival counter.  Needs all CTAs
+// co-resident (cooperative launch).  Bounded: gives up after kWaitLimitClocks.
+__device__ __forceinline__ bool grid_barrier(unsigned* ctr, unsigned target, Ctrl* ctrl) {
+  __shared__ int ok_s;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    __threadfence();
+    atomicAdd(ctr, 1u);
+    int ok = 1;
+    const long long t0 = clock64();
+    while (true) {
+      unsigned v;
+      asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(ctr) : "memory");
+      if (v >= target) break;
+      if (clock64() - t0 > kWaitLimitClocks) {
+        atomicExch(&ctrl->status, (int)RRF_ERR_TIMEOUT);
+        ok = 0;
+        break;
+      }
+    }
+    ok_s = ok;
+  }
+  __syncthreads();
+  return ok_s != 0;
+}
+
+// ------------------------------------------------------------------------------------------
+// Householder QR of a rows x b panel.  Each CTA keeps a slab of R consecutive rows in shared
+// memory (column-major, double precision, pitch Rp odd) for the whole factorisation.  Column j
+// costs one pass over the slab and ONE grid barrier: the pass applies the pending reflector
+// H_{j-1} and accumulates p[c] = sum_{row > j} Y[row, j] * X[row, c] for every column c, where
+// X[:, c] is the finished vector v_c for c < j and the current Y[:, c] for c >= j.  After the
+// barrier every CTA sums the per-CTA partials in CTA order and derives, with alpha = Y[j, j]:
+//   beta = -sign(alpha) sqrt(alpha^2 + p[j]),  tau = (beta - alpha)/beta,  v = Y[j+1:, j]/(alpha - beta)
+//   w[c] = v^T Y[:, c]   = Y[j, c] + p[c]/(alpha - beta)           (c > j: needed by H_j)
+//   g[c] = v_c^T v_j     = v_c[j] + p[c]/(alpha - beta)           (c < j: row j of V^T V, for T)
+// so norms, reflector application and the Gram matrix for T share one reduction.
+// ------------------------------------------------------------------------------------------
+template <typename T>
+__global__ void __launch_bounds__(kPanelThreads)
+    panel_kernel(const T* __restrict__ Y, int nseg, long long seg_stride, int ldy,  // sum of nseg partial panels
+                 int rows, int b, int R, int Rp,
+                 T* __restrict__ V, long long ldv,   // rows x b block of the V array
+                 double* __restrict__ P,             // [2][gridDim.x][b] per-CTA partial dots
+                 double* __restrict__ piv,           // [2][b] broadcast pivot row
+                 double* __restrict__ gram,          // [b][b] strictly-lower part: v_c^T v_j (c < j)
+                 double* __restrict__ tau_out,       // [b]
+                 unsigned* bar, Ctrl* ctrl, const int* done_flag) {
+  if (*reinterpret_cast<const volatile int*>(done_flag)) return;
+  extern __shared__ double psm[];
+  double* S = psm;                        // [b][Rp]
+  double* w_s = S + (size_t)b * Rp;       // [b]
+  double* p_s = w_s + b;                  // [b]
+  double* pr_s = p_s + b;                 // [b]
+  double* part_s = p_s;                   // [kPanelThreads], aliases p_s/pr_s (see panel_extra_doubles)
+
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  constexpr int NW = kPanelThreads / 32;
+  const int G = gridDim.x, cta = blockIdx.x;
+  const int gr0 = cta * R;
+  const int nloc = max(0, min(R, rows - gr0));
+
+  // load the slab: sum the partial panels in segment order
+  for (int idx = tid; idx < nloc * b; idx += kPanelThreads) {
+    const int r = idx / b, c = idx - r * b;
+    const T* src = Y + (size_t)(gr0 + r) * ldy + c;
+    double s = 0.0;
+    for (int sg = 0; sg < nseg; ++sg) s += (double)src[(size_t)sg * seg_stride];
+    S[(size_t)c * Rp + r] = s;
+  }
+  __syncthreads();
+
+  double tau_prev = 0.0;
+  for (int j = 0; j < b; ++j) {
+    double* Sj = S + (size_t)j * Rp;
+    const double* Sjm1 = S + (size_t)(j > 0 ? j - 1 : 0) * Rp;
+    // finish column j: pending reflector H_{j-1}
+    if (j > 0 && tau_prev != 0.0) {
+      const double f = tau_prev * w_s[j];
+      for (int r = tid; r < nloc; r += kPanelThreads)
+        if (gr0 + r >= j) Sj[r] -= f * Sjm1[r];
+    }
+    __syncthreads();
+    // one pass: update trailing columns and take all dot products with column j
+    for (int c = warp; c < b; c += NW) {
+      double* Sc = S + (size_t)c * Rp;
+      const bool upd = (j > 0) && (c > j) && (tau_prev != 0.0);
+      const double f = upd ? tau_prev * w_s[c] : 0.0;
+      double acc = 0.0;
+      for (int r = lane; r < nloc; r += 32) {
+        const int grow = gr0 + r;
+        double x = Sc[r];
+        if (upd && grow >= j) {
+          x -= f * Sjm1[r];
+          Sc[r] = x;
+        }
+        if (grow > j) acc += Sj[r] * x;
+      }
+      acc = warp_sum(acc);
+      if (lane == 0) p_s[c] = acc;
+    }
+    __syncthreads();
+    double* Pj = P + (size_t)(j & 1) * G * b;
+    for (int c = tid; c < b; c += kPanelThreads) Pj[(size_t)cta * b + c] = p_s[c];
+    if (j >= gr0 && j < gr0 + nloc)
+      for (int c = tid; c < b; c += kPanelThreads) piv[(j & 1) * b + c] = S[(size_t)c * Rp + (j - gr0)];
+    if (!grid_barrier(bar, (unsigned)(j + 1) * (unsigned)G, ctrl)) return;
+
+    // every CTA: fixed-order sum of the partials (kPanelThreads/b threads per column)
+    {
+      const int per = kPanelThreads / b;          // b in {16,...,128} divides 256
+      const int c = tid % b, q = tid / b;
+      double s = 0.0;
+      for (int x = q; x < G; x += per) s += __ldcg(Pj + (size_t)x * b + c);
+      part_s[tid] = s;
+      __syncthreads();
+      double tot = 0.0, prv = 0.0;
+      if (tid < b) {
+        for (int qq = 0; qq < per; ++qq) tot += part_s[qq * b + tid];
+        prv = __ldcg(piv + (j & 1) * b + tid);
+      }
+      __syncthreads();
+      if (tid < b) {
+        p_s[tid] = tot;
+        pr_s[tid] = prv;
+      }
+      __syncthreads();
+    }
+    const double alpha = pr_s[j], s2 = p_s[j];
+    double tau = 0.0, denom = 1.0;
+    if (s2 != 0.0) {
+      const double beta = -copysign(sqrt(alpha * alpha + s2), alpha);
+      tau = (beta - alpha) / beta;
+      denom = alpha - beta;
+    }
+    if (tid < b && tid != j) {
+      const double wv = (s2 != 0.0) ? pr_s[tid] + p_s[tid] / denom : pr_s[tid];
+      w_s[tid] = wv;
+      if (cta == 0 && tid < j) gram[(size_t)j * b + tid] = wv;
+    }
+    if (cta == 0 && tid == 0) tau_out[j] = tau;
+    // column j becomes v_j (unit lower trapezoidal, explicit ones and zeros)
+    for (int r = tid; r < nloc; r += kPanelThreads) {
+      const int grow = gr0 + r;
+      Sj[r] = grow > j ? (s2 != 0.0 ? Sj[r] / denom : 0.0) : (grow == j ? 1.0 : 0.0);
+    }
+    tau_prev = tau;
+    __syncthreads();
+  }
+
+  for (int idx = tid; idx < nloc * b; idx += kPanelThreads) {
+    const int r = idx / b, c = idx - r * b;
+    V[(size_t)(gr0 + r) * ldv + c] = (T)S[(size_t)c * Rp + r];
+  }
+}
+
+// ------------------------------------------------------------------------------------------
+// Compact-WY factor from the Gram rows:  T[j][j] = tau_j,
+// T[0:j, j] = -tau_j * T[0:j, 0:j] * (V[:, 0:j]^T v_j)   (Eq. "Q_i = I_m - V_i T_i V_i^T").
+// One CTA; T is built in shared memory in double and written as T (b x b, leading dim ldt).
+// ------------------------------------------------------------------------------------------
+template <typename T>
+__global__ void __launch_bounds__(128)
+    tfactor_kernel(const double* __restrict__ gram, const double* __restrict__ tau, int b,
+                   T* __restrict__ Tout, long long ldt, const int* done_flag) {
+  if (*reinterpret_cast<const volatile int*>(done_flag)) return;
+  extern __shared__ double tsm[];
+  const int pitch = b + 1;
+  double* Ts = tsm;                        // [b][pitch]
+  double* gj = Ts + (size_t)b * pitch;     // [b]: gj[l] = v_l^T v_j, l < j
+  const int tid = threadIdx.x;
+  for (int idx = tid; idx < b * pitch; idx += blockDim.x) Ts[idx] = 0.0;
+  __syncthreads();
+  for (int j = 0; j < b; ++j) {
+    const double tj = tau[j];
+    if (tid < j) gj[tid] = gram[(size_t)j * b + tid];
+    __syncthreads();
+    if (tid < j) {
+      double s = 0.0;
+      for (int l = tid; l < j; ++l) s += Ts[tid * pitch + l] * gj[l];
+      Ts[tid * pitch + j] = -tj * s;
+    } else if (tid == j) {
+      Ts[j * pitch + j] = tj;
+    }
+    __syncthreads();
+  }
+  for (int idx = tid; idx < b * b; idx += blockDim.x) {
+    const int i = idx / b, j = idx - i * b;
+    Tout[(size_t)i * ldt + j] = (T)Ts[i * pitch + j];
+  }
+}
+
+// ------------------------------------------------------------------------------------------
+// Zt[col][0:b] = (op(T) * sum_seg Zpart[seg][:, col])   with op(T) = T^T (apply Q^T) or T (apply Q).
+// Each CTA owns kTzCols columns.  Output is the transposed (K-contiguous) operand of update_kernel.
+// ------------------------------------------------------------------------------------------
+constexpr int kTzCols = 32;
+template <typename T>
+__global__ void __launch_bounds__(256)
+    tz_kernel(const T* __restrict__ Zpart, int nseg, int npad, int b, const T* __restrict__ Tm, long long ldt,
+              int transpose_t, T* __restrict__ Zt, const int* done_flag) {
+  if (*reinterpret_cast<const volatile int*>(done_flag)) return;
+  extern __shared__ double zsm[];
+  const int pitch = b + 1;
+  double* Ts = zsm;                         // [b][pitch]
+  double* Zs = Ts + (size_t)b * pitch;      // [kTzCols][pitch]
+  const int tid = threadIdx.x;
+  const int col0 = blockIdx.x * kTzCols;
+  for (int idx = tid; idx < b * b; idx += 256) {
+    const int i = idx / b, j = idx - i * b;
+    Ts[i * pitch + j] = (double)Tm[(size_t)i * ldt + j];
+  }
+  for (int idx = tid; idx < b * kTzCols; idx += 256) {
+    const int l = idx / kTzCols, cl = idx - l * kTzCols;
+    double s = 0.0;
+    for (int sg = 0; sg < nseg; ++sg) s += (double)Zpart[((size_t)sg * b + l) * npad + col0 + cl];
+    Zs[cl * pitch + l] = s;
+  }
+  __syncthreads();
+  const int j = tid % b, cq = tid / b, ncq = 256 / b;
+  for (int cl = cq; cl < kTzCols; cl += ncq) {
+    const double* z = Zs + cl * pitch;
+    double s = 0.0;
+    if (transpose_t) {
+      for (int l = 0; l <= j; ++l) s += Ts[l * pitch + j] * z[l];
+    } else {
+      for (int l = j; l < b; ++l) s += Ts[j * pitch + l] * z[l];
+    }
+    Zt[(size_t)(col0 + cl) * b + j] = (T)s;
+  }
+}
+
+// ------------------------------------------------------------------------------------------
+// Algorithm 2 lines 1-3: W <- A (unless in place), partial sums of ||A||_F^2, V <- 0.
+// Fixed chunking and fixed-order reductions: the result does not depend on scheduling.
+// ------------------------------------------------------------------------------------------
+template <typename T>
+__global__ void __launch_bounds__(256)
+    init_kernel(const T* __restrict__ A, long long lda, T* __restrict__ W, long long ldw, long long m, long long n,
+                T* __restrict__ V, long long ldv, int vcols, double* __restrict__ part) {
+  __shared__ double red[32];
+  const long long total = m * n;
+  const long long chunk = (total + gridDim.x - 1) / gridDim.x;
+  const long long lo = (long long)blockIdx.x * chunk, hi = min(total, lo + chunk);
+  double s = 0.0;
+  for (long long idx = lo + threadIdx.x; idx < hi; idx += 256) {
+    const long long r = idx / n, c = idx - r * n;
+    const T x = A[r * lda + c];
+    if (W != nullptr) W[r * ldw + c] = x;
+    s += (double)x * (double)x;
+  }
+  const double tot = block_sum(s, red);
+  if (threadIdx.x == 0) part[blockIdx.x] = tot;
+  const long long vtotal = m * vcols;
+  const long long vchunk = (vtotal + gridDim.x - 1) / gridDim.x;
+  const long long vlo = (long long)blockIdx.x * vchunk, vhi = min(vtotal, vlo + vchunk);
+  for (long long idx = vlo + threadIdx.x; idx < vhi; idx += 256) {
+    const long long r = idx / vcols, c = idx - r * vcols;
+    V[r * ldv + c] = T(0);
+  }
+}
+
+__global__ void __launch_bounds__(256)
+    init_ctrl_kernel(const double* __restrict__ part, int npart, double tol, int relative, int fixed_rank,
+                     int b, int max_rank, Ctrl* ctrl) {
+  __shared__ double red[32];
+  double s = 0.0;
+  for (int i = threadIdx.x; i < npart; i += 256) s += part[i];
+  const double tot = block_sum(s, red);
+  if (threadIdx.x == 0) {
+    ctrl->normA2 = tot;
+    ctrl->sigma2 = relative ? tol * tol * tot : tol * tol;
+    ctrl->E_sub = tot;
+    ctrl->E_dir = tot;
+    ctrl->steps = 0;
+    ctrl->k = 0;
+    ctrl->bar = 0;
+    int status = RRF_OK, done = 0;
+    if (!(tot == tot) || tot > 1.7e308) {
+      status = RRF_ERR_NONFINITE;
+      done = 1;
+    } else if (!fixed_rank && !(tot > ctrl->sigma2)) {
+      done = 1;
+    } else if (b > max_rank) {
+      done = 1;
+      status = RRF_MAX_RANK_REACHED;
+    }
+    ctrl->status = status;
+    ctrl->done = done;
+  }
+}
+
+// Algorithm 2 lines 9-10 and the test of line 5 for the next pass, on the device.
+__global__ void __launch_bounds__(256)
+    stop_kernel(const double* __restrict__ norm_part, int npart, int b, int max_rank, int estimator,
+                int fixed_rank, double* __restrict__ tr_sub, double* __restrict__ tr_dir, Ctrl* ctrl) {
+  if (*reinterpret_cast<volatile int*>(&ctrl->done)) return;
+  __shared__ double red[64];
+  double st = 0.0, sr = 0.0;
+  for (int i = threadIdx.x; i < npart; i += 256) {
+    st += norm_part[2 * i];
+    sr += norm_part[2 * i + 1];
+  }
+  const double top = block_sum(st, red);
+  const double trail = block_sum(sr, red + 32);
+  if (threadIdx.x == 0) {
+    const double e_sub = ctrl->E_sub - top;
+    ctrl->E_sub = e_sub;
+    ctrl->E_dir = trail;
+    const int i = ctrl->steps;
+    tr_sub[i] = e_sub;
+    tr_dir[i] = trail;
+    ctrl->steps = i + 1;
+    ctrl->k = (i + 1) * b;
+    ctrl->bar = 0;
+    const double E = estimator == 0 ? trail : e_sub;
+    const bool below = !(E > ctrl->sigma2);
+    const bool met = !fixed_rank && below;
+    const bool cap = (i + 2) * b > max_rank;
+    if (ctrl->status == RRF_OK && !below && cap) ctrl->status = RRF_MAX_RANK_REACHED;
+    if (met || cap) ctrl->done = 1;
+  }
+}
+
+// ------------------------------------------------------------------------------------------
+// Algorithm 2 line 6: standard Gaussians from a counter-based generator (Philox-4x32, 10
+// rounds, Salmon et al. 2011; Box-Muller in double).  Counter = (pair index, 0, vector index,
+// 0), key = seed: one call yields elements (j, 2q) and (j, 2q+1) of OmegaT.
+// ------------------------------------------------------------------------------------------
+__device__ __forceinline__ void philox4x32_10(uint32_t (&c)[4], uint32_t k0, uint32_t k1) {
+#pragma unroll
+  for (int r = 0; r < 10; ++r) {
+    const uint64_t p0 = (uint64_t)0xD2511F53u * c[0];
+    const uint64_t p1 = (uint64_t)0xCD9E8D57u * c[2];
+    const uint32_t n0 = (uint32_t)(p1 >> 32) ^ c[1] ^ k0;
+    const uint32_t n1 = (uint32_t)p1;
+    const uint32_t n2 = (uint32_t)(p0 >> 32) ^ c[3] ^ k1;
+    const uint32_t n3 = (uint32_t)p0;
+    c[0] = n0; c[1] = n1; c[2] = n2; c[3] = n3;
+    k0 += 0x9E3779B9u;
+    k1 += 0xBB67AE85u;
+  }
+}
+
+template <typename T>
+__global__ void __launch_bounds__(256)
+    omega_kernel(T* __restrict__ O, long long ldo, long long n, int nvec, int first_vec, uint64_t seed) {
+  const long long npairs = (n + 1) / 2;
+  const long long total = npairs * nvec;
+  for (long long idx = (long long)blockIdx.x * 256 + threadIdx.x; idx < total; idx += (long long)gridDim.x * 256) {
+    const long long jv = idx / npairs, q = idx - jv * npairs;
+    const uint64_t vec = (uint64_t)(first_vec + jv);
+    uint32_t c[4] = {(uint32_t)q, (uint32_t)((uint64_t)q >> 32), (uint32_t)vec, (uint32_t)(vec >> 32)};
+    philox4x32_10(c, (uint32_t)seed, (uint32_t)(seed >> 32));
+    const uint64_t a = ((uint64_t)c[1] << 32) | c[0], bb = ((uint64_t)c[3] << 32) | c[2];
+    const double u1 = ((double)(a >> 12) + 0.5) * (1.0 / 4503599627370496.0);   // (0, 1), exact
+    const double u2 = ((double)(bb >> 12) + 0.5) * (1.0 / 4503599627370496.0);
+    const double rad = sqrt(-2.0 * log(u1));
+    double sn, cs;
+    sincospi(2.0 * u2, &sn, &cs);
+    T* row = O + jv * ldo;
+    row[2 * q] = (T)(rad * cs);
+    if (2 * q + 1 < n) row[2 * q + 1] = (T)(rad * sn);
+  }
+}
+
+template <typename T>
+__global__ void __launch_bounds__(256) eye_kernel(T* __restrict__ Q, long long ldq, long long m, int k) {
+  const long long total = m * k;
+  for (long long idx = (long long)blockIdx.x * 256 + threadIdx.x; idx < total; idx += (long long)gridDim.x * 256) {
+    const long long r = idx / k, c = idx - r * k;
+    Q[r * ldq + c] = r == c ? T(1) : T(0);
+  }
+}
+
+}  // namespace rrf

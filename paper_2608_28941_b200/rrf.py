@@ -1,0 +1,274 @@
+"""ctypes binding of librrf.so: same names as include/rrf.h, argument marshalling only.
+
+Every function takes torch CUDA tensors (device memory and streams are PyTorch's),
+passes raw pointers, sizes and the current CUDA stream to the C ABI and returns
+what the library wrote.  Nothing is computed here, and there is no fallback: a
+missing or unloadable library raises.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from dataclasses import dataclass
+
+import torch
+
+RRF_F64, RRF_F32 = 0, 1
+RRF_OK, RRF_MAX_RANK_REACHED = 0, 1
+RRF_ERR_INVALID_ARG, RRF_ERR_WORKSPACE, RRF_ERR_CUDA, RRF_ERR_TIMEOUT, RRF_ERR_NONFINITE = -1, -2, -3, -4, -5
+RRF_FLAG_INPLACE, RRF_FLAG_FIXED_RANK = 1, 2
+
+_LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "librrf.so")
+_lib = None
+
+
+class rrf_params_t(C.Structure):
+    _fields_ = [("dtype", C.c_int32), ("b", C.c_int32), ("max_rank", C.c_int32), ("estimator", C.c_int32),
+                ("m", C.c_int64), ("n", C.c_int64), ("tol", C.c_double), ("tol_is_relative", C.c_int32),
+                ("flags", C.c_uint32), ("seed", C.c_uint64)]
+
+
+class rrf_result_t(C.Structure):
+    _fields_ = [("status", C.c_int32), ("k", C.c_int32), ("steps", C.c_int32), ("cuda_error", C.c_int32),
+                ("normA2", C.c_double), ("sigma2", C.c_double), ("E_sub", C.c_double), ("E_dir", C.c_double)]
+
+
+EXPORTS = ["rrf_create", "rrf_destroy", "rrf_workspace_bytes", "rrf_run", "rrf_panel_workspace_bytes",
+           "rrf_panel_qr", "rrf_apply_workspace_bytes", "rrf_apply_qt", "rrf_apply_q", "rrf_form_q",
+           "rrf_fill_omega", "rrf_last_status", "rrf_status_string"]
+
+
+def load():
+    """Open librrf.so (once).  Raises if it has not been built."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(_LIB_PATH):
+        raise RuntimeError(f"{_LIB_PATH} is missing: build it with `python -m paper_2608_28941_b200.build` "
+                           "(there is no CPU fallback)")
+    lib = C.CDLL(_LIB_PATH)
+    vp, i32, i64, u64, sz = C.c_void_p, C.c_int32, C.c_int64, C.c_uint64, C.c_size_t
+    lib.rrf_create.argtypes = [C.POINTER(vp), C.c_int]
+    lib.rrf_destroy.argtypes = [vp]
+    lib.rrf_workspace_bytes.argtypes = [C.POINTER(rrf_params_t), C.POINTER(sz)]
+    lib.rrf_run.argtypes = [vp, C.POINTER(rrf_params_t), vp, i64, vp, i64, vp, i64, vp, vp, i64, vp, sz, vp,
+                            C.POINTER(rrf_result_t), C.POINTER(C.c_double), C.POINTER(C.c_double)]
+    lib.rrf_panel_workspace_bytes.argtypes = [i32, i64, i32, C.POINTER(sz)]
+    lib.rrf_panel_qr.argtypes = [vp, i32, i64, i32, vp, i64, vp, i64, vp, i64, vp, sz, vp]
+    lib.rrf_apply_workspace_bytes.argtypes = [i32, i64, i64, i32, C.POINTER(sz)]
+    for f in (lib.rrf_apply_qt, lib.rrf_apply_q):
+        f.argtypes = [vp, i32, i64, i32, i32, vp, i64, vp, i64, vp, i64, i64, vp, sz, vp]
+    lib.rrf_form_q.argtypes = [vp, i32, i64, i32, i32, vp, i64, vp, i64, vp, i64, vp, sz, vp]
+    lib.rrf_fill_omega.argtypes = [vp, i32, u64, i64, i32, i32, vp, i64, vp]
+    lib.rrf_last_status.argtypes = [vp, vp]
+    lib.rrf_status_string.argtypes = [C.c_int]
+    lib.rrf_status_string.restype = C.c_char_p
+    for name in EXPORTS:
+        if name != "rrf_status_string":
+            getattr(lib, name).restype = C.c_int
+    _lib = lib
+    return lib
+
+
+class RrfError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {rrf_status_string(status)} ({status})")
+
+
+def rrf_status_string(status: int) -> str:
+    return load().rrf_status_string(int(status)).decode()
+
+
+def _dtype_code(t: torch.Tensor) -> int:
+    if t.dtype == torch.float64:
+        return RRF_F64
+    if t.dtype == torch.float32:
+        return RRF_F32
+    raise TypeError(f"unsupported dtype {t.dtype}")
+
+
+def _stream() -> C.c_void_p:
+    return C.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def _rowmajor(t: torch.Tensor, name: str) -> int:
+    """Leading dimension of a 2-D row-major tensor (last stride 1)."""
+    if t.dim() != 2 or t.stride(1) != 1 or not t.is_cuda:
+        raise ValueError(f"{name} must be a 2-D CUDA tensor with unit inner stride")
+    return t.stride(0) if t.shape[0] > 1 else max(t.shape[1], t.stride(0))
+
+
+def _empty(rows: int, cols: int, dtype, device) -> torch.Tensor:
+    """rows x cols view whose leading dimension keeps every row 16-byte aligned."""
+    pad = 2 if dtype == torch.float64 else 4
+    ld = (cols + pad - 1) // pad * pad
+    return torch.empty((rows, ld), dtype=dtype, device=device)[:, :cols]
+
+
+def rrf_create(device: int = 0) -> C.c_void_p:
+    h = C.c_void_p()
+    s = load().rrf_create(C.byref(h), int(device))
+    if s != RRF_OK:
+        raise RrfError(s, "rrf_create")
+    return h
+
+
+def rrf_destroy(h) -> None:
+    load().rrf_destroy(h)
+
+
+def make_params(dtype: int, m: int, n: int, b: int, tol: float, max_rank: int, relative: bool = True,
+                estimator: int = 0, flags: int = 0, seed: int = 0) -> rrf_params_t:
+    return rrf_params_t(dtype=dtype, b=b, max_rank=max_rank, estimator=estimator, m=m, n=n, tol=tol,
+                        tol_is_relative=1 if relative else 0, flags=flags, seed=seed)
+
+
+def rrf_workspace_bytes(p: rrf_params_t) -> int:
+    out = C.c_size_t()
+    s = load().rrf_workspace_bytes(C.byref(p), C.byref(out))
+    if s != RRF_OK:
+        raise RrfError(s, "rrf_workspace_bytes")
+    return out.value
+
+
+@dataclass
+class RunResult:
+    status: int
+    k: int
+    steps: int
+    normA2: float
+    sigma2: float
+    E_sub: float
+    E_dir: float
+    E_sub_trace: list
+    E_dir_trace: list
+    V: torch.Tensor   # m x max_rank buffer; columns [:k] are defined
+    T: torch.Tensor   # b x max_rank
+    B: torch.Tensor   # max_rank x n buffer; rows [:k] are defined
+
+
+def rrf_run(h, A: torch.Tensor, b: int, tol: float, max_rank: int, omegaT: torch.Tensor | None = None,
+            relative: bool = True, estimator: int = 0, flags: int = 0, seed: int = 0,
+            V: torch.Tensor | None = None, T: torch.Tensor | None = None, B: torch.Tensor | None = None,
+            workspace: torch.Tensor | None = None, check: bool = True) -> RunResult:
+    """Algorithm 2 on the device.  `omegaT` is max_rank x n (row j = j-th Gaussian vector) or None."""
+    lib = load()
+    m, n = A.shape
+    dt = _dtype_code(A)
+    p = make_params(dt, m, n, b, tol, max_rank, relative, estimator, flags, seed)
+    need = C.c_size_t()
+    s = lib.rrf_workspace_bytes(C.byref(p), C.byref(need))
+    if s != RRF_OK:
+        raise RrfError(s, "rrf_workspace_bytes")
+    dev = A.device
+    if V is None:
+        V = _empty(m, max_rank, A.dtype, dev)
+    if T is None:
+        T = torch.empty((b, max_rank), dtype=A.dtype, device=dev)   # leading dimension max_rank
+    if B is None:
+        B = _empty(max_rank, n, A.dtype, dev)
+    if workspace is None:
+        workspace = torch.empty(need.value, dtype=torch.uint8, device=dev)
+    res = rrf_result_t()
+    steps = max_rank // b
+    tr_sub = (C.c_double * steps)()
+    tr_dir = (C.c_double * steps)()
+    om_ptr, ldo = (None, 0) if omegaT is None else (C.c_void_p(omegaT.data_ptr()), _rowmajor(omegaT, "omegaT"))
+    s = lib.rrf_run(h, C.byref(p), C.c_void_p(A.data_ptr()), _rowmajor(A, "A"), om_ptr, ldo,
+                    C.c_void_p(V.data_ptr()), _rowmajor(V, "V"), C.c_void_p(T.data_ptr()),
+                    C.c_void_p(B.data_ptr()), _rowmajor(B, "B"), C.c_void_p(workspace.data_ptr()),
+                    workspace.numel(), _stream(), C.byref(res), tr_sub, tr_dir)
+    if check and s < 0:
+        raise RrfError(s, "rrf_run")
+    return RunResult(res.status, res.k, res.steps, res.normA2, res.sigma2, res.E_sub, res.E_dir,
+                     list(tr_sub)[:res.steps], list(tr_dir)[:res.steps], V, T, B)
+
+
+def rrf_panel_qr(h, Y: torch.Tensor):
+    """Householder QR of a tall panel: returns (V, T) as the library writes them."""
+    lib = load()
+    rows, b = Y.shape
+    dt = _dtype_code(Y)
+    need = C.c_size_t()
+    s = lib.rrf_panel_workspace_bytes(dt, rows, b, C.byref(need))
+    if s != RRF_OK:
+        raise RrfError(s, "rrf_panel_workspace_bytes")
+    ws = torch.empty(need.value, dtype=torch.uint8, device=Y.device)
+    V = torch.empty_like(Y)
+    T = torch.empty((b, b), dtype=Y.dtype, device=Y.device)
+    s = lib.rrf_panel_qr(h, dt, rows, b, C.c_void_p(Y.data_ptr()), _rowmajor(Y, "Y"), C.c_void_p(V.data_ptr()),
+                         _rowmajor(V, "V"), C.c_void_p(T.data_ptr()), b, C.c_void_p(ws.data_ptr()), ws.numel(),
+                         _stream())
+    if s != RRF_OK:
+        raise RrfError(s, "rrf_panel_qr")
+    s = lib.rrf_last_status(h, _stream())
+    if s != RRF_OK:
+        raise RrfError(s, "rrf_panel_qr (device)")
+    return V, T
+
+
+def _apply(fn_name: str, h, V: torch.Tensor, T: torch.Tensor, b: int, k: int, Cm: torch.Tensor) -> torch.Tensor:
+    lib = load()
+    m, ncols = Cm.shape
+    dt = _dtype_code(Cm)
+    need = C.c_size_t()
+    s = lib.rrf_apply_workspace_bytes(dt, m, ncols, b, C.byref(need))
+    if s != RRF_OK:
+        raise RrfError(s, "rrf_apply_workspace_bytes")
+    ws = torch.empty(need.value, dtype=torch.uint8, device=Cm.device)
+    s = getattr(lib, fn_name)(h, dt, m, b, k, C.c_void_p(V.data_ptr()), _rowmajor(V, "V"), C.c_void_p(T.data_ptr()),
+                              _rowmajor(T, "T"), C.c_void_p(Cm.data_ptr()), _rowmajor(Cm, "C"), ncols,
+                              C.c_void_p(ws.data_ptr()), ws.numel(), _stream())
+    if s != RRF_OK:
+        raise RrfError(s, fn_name)
+    torch.cuda.current_stream().synchronize()   # the workspace is freed on return
+    return Cm
+
+
+def rrf_apply_qt(h, V, T, b: int, k: int, Cm: torch.Tensor) -> torch.Tensor:
+    """C <- Q^T C in place."""
+    return _apply("rrf_apply_qt", h, V, T, b, k, Cm)
+
+
+def rrf_apply_q(h, V, T, b: int, k: int, Cm: torch.Tensor) -> torch.Tensor:
+    """C <- Q C in place."""
+    return _apply("rrf_apply_q", h, V, T, b, k, Cm)
+
+
+def rrf_form_q(h, V: torch.Tensor, T: torch.Tensor, b: int, k: int) -> torch.Tensor:
+    """Explicit m x k orthonormal basis."""
+    lib = load()
+    m = V.shape[0]
+    dt = _dtype_code(V)
+    Q = _empty(m, k, V.dtype, V.device)
+    need = C.c_size_t()
+    s = lib.rrf_apply_workspace_bytes(dt, m, k, b, C.byref(need))
+    if s != RRF_OK:
+        raise RrfError(s, "rrf_apply_workspace_bytes")
+    ws = torch.empty(need.value, dtype=torch.uint8, device=V.device)
+    s = lib.rrf_form_q(h, dt, m, b, k, C.c_void_p(V.data_ptr()), _rowmajor(V, "V"), C.c_void_p(T.data_ptr()),
+                       _rowmajor(T, "T"), C.c_void_p(Q.data_ptr()), _rowmajor(Q, "Q"), C.c_void_p(ws.data_ptr()),
+                       ws.numel(), _stream())
+    if s != RRF_OK:
+        raise RrfError(s, "rrf_form_q")
+    torch.cuda.current_stream().synchronize()
+    return Q
+
+
+def rrf_fill_omega(h, n: int, nvec: int, seed: int, dtype=torch.float64, first_vec: int = 0,
+                   device="cuda") -> torch.Tensor:
+    """nvec x n Gaussian matrix (OmegaT layout) from the library's counter-based generator."""
+    lib = load()
+    pad = 2 if dtype == torch.float64 else 4
+    ldo = (n + pad - 1) // pad * pad
+    buf = torch.empty((nvec, ldo), dtype=dtype, device=device)
+    O = buf[:, :n]
+    s = lib.rrf_fill_omega(h, _dtype_code(O), seed, n, nvec, first_vec, C.c_void_p(O.data_ptr()), ldo, _stream())
+    if s != RRF_OK:
+        raise RrfError(s, "rrf_fill_omega")
+    return O
+
+
+def rrf_last_status(h) -> int:
+    return load().rrf_last_status(h, _stream())

@@ -206,3 +206,27 @@ def test_diag_standin_predicts_same_rank():
     rd = orc.rrf(wl.diag_matrix(s, w.m, w.n), Om, w.b, 1e-4, w.max_rank)
     assert abs(r.k - rd.k) <= w.b
     assert np.isclose(np.linalg.svd(A, compute_uv=False)[:20], s[:20], rtol=1e-10).all()
+
+
+# ---- P10: the one numerical behaviour the paper prints (section "Numerical Stability and
+# Performance"): single precision, 1024 x 1024, singular values log-spaced from 1 to 1e-14,
+# b = 64: the subtractive stopping quantity stops tracking the residual near k = 384 through
+# cancellation, while orthogonality and the residual stay at single-precision round-off.
+
+
+def test_fp32_subtractive_estimator_stops_tracking_near_384():
+    rng = np.random.default_rng(10)
+    n, b = 1024, 64
+    U, _ = np.linalg.qr(rng.standard_normal((n, n)))
+    Vv, _ = np.linalg.qr(rng.standard_normal((n, n)))
+    s = 10.0 ** (-14 * np.arange(n) / (n - 1))
+    A = ((U * s) @ Vv.T).astype(np.float32)
+    Om = rng.standard_normal((n, 640)).astype(np.float32)
+    r = orc.rrf(A, Om, b, 0.0, 640, dtype=np.float32)
+    e_sub, e_dir = np.array(r.E_sub), np.array(r.E_dir)
+    assert np.all(np.abs(e_sub[:3] - e_dir[:3]) <= 1e-2 * e_dir[:3])        # k <= 192: tracks
+    assert e_sub[5] > 10 * e_dir[5] or e_sub[5] <= 0                        # k = 384: lost
+    assert np.all(np.abs(e_sub[6:]) > 100 * e_dir[6:])                      # and never recovers
+    Q = orc.form_q(r.V.astype(np.float64), r.T.astype(np.float64), b)
+    assert np.linalg.norm(Q.T @ Q - np.eye(640), 2) < 5e-6
+    assert np.linalg.norm(A - Q @ (Q.T @ A), 2) < 2e-6
