@@ -1,0 +1,361 @@
+#!/usr/bin/env python
+"""Benchmark of the blocked adaptive randomized range finder on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload cfg2]
+
+One "step" is one complete run of the hot path (Algorithm 2: norm, sample, panel QR, WY
+update, norms, stop rule, for every block until the tolerance is met) on one seeded synthetic
+matrix.  The default workload is the 8192 x 8192 float64 configuration (polynomial spectrum,
+b = 64, relative tolerance 1e-4, rank cap 1024).  The metric is the method's own arithmetic,
+sum_i (6 m_i n b + 3 m_i b^2) over the executed blocks, per second.  With N > 1 every rank runs
+an independent replica (the path has no exchange step): value = N runs' flops / slowest rank.
+Rank 0 prints one JSON line.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu
+# capture summarised under profiles/ (None until a capture of the current kernel exists).
+NCU_TRAFFIC_BYTES = {}
+
+NOMINAL_FP64_OVER_BF16 = 37.0 / 2250.0   # HGX B200 dense figures: FP64 tensor 37 TF, bf16 2250 TF
+
+
+def method_flops(m: int, n: int, b: int, steps: int) -> float:
+    return float(sum(6.0 * (m - i * b) * n * b + 3.0 * (m - i * b) * b * b for i in range(steps)))
+
+
+def measured_peaks() -> dict:
+    try:
+        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
+            return json.load(f)
+    except Exception:
+        return {}
+
+
+class ClockSampler:
+    """nvidia-smi clock / throttle samples while the timed region runs."""
+
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.rows, self.proc = index, [], None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append(line.strip())
+
+    def stop(self) -> dict:
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], None, set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            f = [x.strip() for x in r.split(",")]
+            if len(f) < 7:
+                continue
+            try:
+                sm.append(float(f[0]))
+                mx = float(f[1])
+            except ValueError:
+                continue
+            for nm, v in zip(names, f[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(nm)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": mx, "reasons": sorted(reasons),
+                "samples": len(sm)}
+
+
+def oracle_run(A, Om, w, blocks=None):
+    from oracle import rrf_oracle as orc
+    max_rank = w.max_rank if blocks is None else min(w.max_rank, blocks * w.b)
+    t0 = time.perf_counter()
+    r = orc.rrf(A, Om, w.b, w.tol, max_rank)
+    dt = time.perf_counter() - t0
+    return r, dt
+
+
+def host_threads() -> int:
+    try:
+        from threadpoolctl import threadpool_info
+        n = [p.get("num_threads", 0) for p in threadpool_info() if p.get("user_api") == "blas"]
+        if n:
+            return int(max(n))
+    except Exception:
+        pass
+    return os.cpu_count() or 1
+
+
+def generate(w, device):
+    """A on the device (or host when device is None) and Omega^T, both in the path's dtype."""
+    import torch
+    from paper_2608_28941_b200 import workloads as wl
+    A, _ = wl.make_matrix(w, device=device)
+    Om = wl.make_omega(w).astype(w.np_dtype)
+    OmT = np.ascontiguousarray(Om.T)
+    if device is not None:
+        OmT = torch.from_numpy(OmT).to(device)
+    return A, Om, OmT
+
+
+def run_reference(args, w, rank, world):
+    """The oracle, as it stands, timed on the host cores (rank 0 only)."""
+    if rank != 0:
+        return
+    import torch
+    dev = "cuda:0" if torch.cuda.is_available() else None
+    A, Om, _ = generate(w, dev)
+    A = A.cpu().numpy().astype(np.float64) if dev else A.astype(np.float64)
+    Om = Om.astype(np.float64)
+    # bound the sample: a full run if K+W of them fit in about three minutes, else a prefix of blocks
+    _, t_full = oracle_run(A, Om, w, blocks=2)
+    est_full = t_full / 2 * (w.max_rank // w.b) * 0.7
+    blocks = None
+    budget = 180.0 / max(1, args.steps + args.warmup)
+    if est_full > budget:
+        blocks = max(1, int(budget / (t_full / 2)))
+    for _ in range(args.warmup):
+        oracle_run(A, Om, w, blocks)
+    times, steps_done = [], 0
+    for _ in range(args.steps):
+        r, dt = oracle_run(A, Om, w, blocks)
+        times.append(dt)
+        steps_done = r.steps
+    sec = float(np.mean(times))
+    tf = method_flops(w.m, w.n, w.b, steps_done) / sec / 1e12
+    sample = "full workload" if blocks is None else f"first {steps_done} block steps of the workload"
+    line = {"impl": "reference", "metric": "rangefinder_tflops", "value": tf, "unit": "TFLOP/s", "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": sec * 1e3, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": w.dtype, "data": "synthetic",
+            "config": {"workload": w.name, "m": w.m, "n": w.n, "b": w.b, "tol": w.tol, "max_rank": w.max_rank,
+                       "sample": sample},
+            "cpu_baseline": {"value": tf, "unit": "TFLOP/s", "cores": host_threads(), "kind": "oracle",
+                             "sample": sample},
+            "e2e": {"value": tf, "unit": "TFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=30)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="cfg2")
+    ap.add_argument("--m", type=int, default=0, help="override the workload's rows (profiling captures)")
+    ap.add_argument("--n", type=int, default=0, help="override the workload's columns")
+    ap.add_argument("--max-rank", type=int, default=0, help="override the workload's rank cap")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 0)
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+
+    from paper_2608_28941_b200 import workloads as wl
+    w = wl.CONFIGS[args.workload]
+    if args.m or args.n or args.max_rank:
+        w = w.scaled(args.m or w.m, args.n or w.n, max_rank=args.max_rank or w.max_rank)
+
+    if args.impl == "reference":
+        run_reference(args, w, rank, world)
+        return
+
+    import torch
+    import torch.distributed as dist
+    from paper_2608_28941_b200 import build as _build, rrf
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the product path has no CPU fallback")
+    torch.cuda.set_device(local)
+    dev = f"cuda:{local}"
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device(dev))
+    if rank == 0:
+        _build.build()
+    if world > 1:
+        dist.barrier()
+    h = rrf.rrf_create(local)
+
+    A, Om, OmT = generate(w, dev)
+    tdt = A.dtype
+    esize = A.element_size()
+    p = rrf.make_params(rrf.RRF_F64 if w.dtype == "f64" else rrf.RRF_F32, w.m, w.n, w.b, w.tol, w.max_rank)
+    ws = torch.empty(rrf.rrf_workspace_bytes(p), dtype=torch.uint8, device=dev)
+    V = torch.empty((w.m, w.max_rank), dtype=tdt, device=dev)
+    T = torch.empty((w.b, w.max_rank), dtype=tdt, device=dev)
+    B = torch.empty((w.max_rank, w.n), dtype=tdt, device=dev)
+
+    def step():
+        return rrf.rrf_run(h, A, w.b, w.tol, w.max_rank, omegaT=OmT, V=V, T=T, B=B, workspace=ws)
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    rrf.rrf_set_profiling(h, True)
+    for _ in range(max(args.warmup, 1)):
+        res = step()
+    sampler = ClockSampler(local)
+    barrier()
+    sampler.start()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    prof = {}
+    e0.record()
+    for _ in range(args.steps):
+        res = step()
+        for name, (ms, cnt) in rrf.rrf_get_profile(h).items():
+            a = prof.setdefault(name, [0.0, 0])
+            a[0] += ms
+            a[1] += cnt
+    e1.record()
+    barrier()
+    clocks = sampler.stop()
+    ms_total = e0.elapsed_time(e1)
+    t = torch.tensor([ms_total], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    ms_step = float(t.item()) / args.steps
+    flops = method_flops(w.m, w.n, w.b, res.steps)
+    value = world * flops / (ms_step * 1e-3) / 1e12
+    launches_per_run = 2 + 7 * (w.max_rank // w.b)
+
+    # ---- end to end through the C ABI with host buffers
+    e2e = None
+    if not args.no_e2e:
+        A_h = A.cpu().pin_memory()
+        O_h = OmT.cpu().pin_memory()
+        k = res.k
+        B_h = torch.empty((w.max_rank, w.n), dtype=tdt).pin_memory()
+        V_h = torch.empty((w.m, w.max_rank), dtype=tdt).pin_memory()
+        T_h = torch.empty((w.b, w.max_rank), dtype=tdt).pin_memory()
+        A_d = torch.empty_like(A)
+        O_d = torch.empty_like(OmT)
+
+        def e2e_step():
+            A_d.copy_(A_h, non_blocking=True)
+            O_d.copy_(O_h, non_blocking=True)
+            r = rrf.rrf_run(h, A_d, w.b, w.tol, w.max_rank, omegaT=O_d, V=V, T=T, B=B, workspace=ws)
+            B_h[:r.k].copy_(B[:r.k], non_blocking=True)
+            V_h[:, :r.k].copy_(V[:, :r.k], non_blocking=True)
+            T_h[:, :r.k].copy_(T[:, :r.k], non_blocking=True)
+            torch.cuda.current_stream().synchronize()
+            return r
+        e2e_step()
+        barrier()
+        n_e2e = max(2, min(args.steps, 5))
+        e0.record()
+        for _ in range(n_e2e):
+            e2e_step()
+        e1.record()
+        barrier()
+        t = torch.tensor([e0.elapsed_time(e1)], dtype=torch.float64, device=dev)
+        if world > 1:
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_e2e = float(t.item()) / n_e2e
+        e2e = {"value": world * flops / (ms_e2e * 1e-3) / 1e12, "unit": "TFLOP/s", "ms_per_step": ms_e2e,
+               "h2d_bytes_per_step": int((A_h.numel() + O_h.numel()) * esize),
+               "d2h_bytes_per_step": int((k * w.n + w.m * k + w.b * k) * esize)}
+
+    # ---- roofline of the dominant kernel, from the event profile of the timed region
+    roofline = None
+    if rank == 0:
+        peaks = measured_peaks()
+        gemm = {"sample", "vtw", "update"}
+        top = max((nm for nm in prof if nm not in ("skipped",)), key=lambda nm: prof[nm][0])
+        ms, cnt = prof[top]
+        per_run_steps = res.steps
+        mi = [w.m - i * w.b for i in range(per_run_steps)]
+        if top in gemm:
+            kind = 0 if w.dtype == "f64" else 3
+            peak = rrf.rrf_measure_peak(h, kind, 200.0)
+            if w.dtype == "f32":
+                peak /= 3.0                       # three TF32 products per fp32 product
+            work = args.steps * sum(2.0 * r * w.n * w.b for r in mi)
+            achieved = work / (ms * 1e-3) / 1e12
+            recipe = peaks.get("bf16_tflops", 1590.0) * NOMINAL_FP64_OVER_BF16 if w.dtype == "f64" else None
+            roofline = {"kernel": top, "bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
+                        "frac": achieved / peak, "traffic": NCU_TRAFFIC_BYTES.get(top),
+                        "peak_source": "FP64 mma.sync rate measured live by rrf_measure_peak" if w.dtype == "f64"
+                        else "TF32 mma.sync rate / 3 measured live by rrf_measure_peak",
+                        "peak_recipe": recipe,
+                        "frac_recipe": achieved / recipe if recipe else None,
+                        "peak_recipe_source": ("MEASURED_PEAKS.json bf16 x nominal FP64/bf16 ratio (of measured)"
+                                               if "bf16_tflops" in peaks else "fallback bf16 x nominal ratio (of fallback)"),
+                        "avg_launch_ms": ms / max(cnt, 1), "launches": cnt}
+        else:
+            hbm = peaks.get("hbm_gbs", 6650.0)
+            byts = args.steps * sum(2.0 * r * w.b * esize for r in mi)
+            achieved = byts / (ms * 1e-3) / 1e9
+            roofline = {"kernel": top, "bound": "hbm", "achieved": achieved, "peak": hbm, "unit": "GB/s",
+                        "frac": achieved / hbm, "traffic": NCU_TRAFFIC_BYTES.get(top),
+                        "peak_source": "MEASURED_PEAKS.json (of measured)" if "hbm_gbs" in peaks else "of fallback",
+                        "avg_launch_ms": ms / max(cnt, 1), "launches": cnt}
+        roofline["phases_ms_per_step"] = {nm: prof[nm][0] / args.steps for nm in prof}
+
+    # ---- CPU baseline: the oracle on the host cores (rank 0, single-GPU runs only)
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        A64 = A.cpu().numpy().astype(np.float64)
+        Om64 = Om.astype(np.float64)
+        _, t2 = oracle_run(A64, Om64, w, blocks=2)
+        est = t2 / 2 * (w.max_rank // w.b)
+        blocks = None if est < 40 else max(1, int(25.0 / (t2 / 2)))
+        r, dt = oracle_run(A64, Om64, w, blocks)
+        cpu = {"value": method_flops(w.m, w.n, w.b, r.steps) / dt / 1e12, "unit": "TFLOP/s", "cores": host_threads(),
+               "kind": "oracle", "seconds": dt, "k": r.k,
+               "sample": "full workload, one run" if blocks is None else f"first {r.steps} block steps, one run"}
+
+    if rank == 0:
+        line = {"metric": "rangefinder_tflops", "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps,
+                "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+                "vs_baseline": None, "dtype": w.dtype, "data": "synthetic",
+                "config": {"workload": w.name, "m": w.m, "n": w.n, "b": w.b, "tol": w.tol, "max_rank": w.max_rank,
+                           "k": res.k, "block_steps": res.steps, "status": res.status,
+                           "l2": "inputs larger than L2 (A is %.0f MB)" % (w.m * w.n * esize / 1e6),
+                           "parallelism": "replicas only" if world > 1 else "single GPU"},
+                "clocks": clocks, "e2e": e2e, "gpu_launches": args.steps * launches_per_run,
+                "roofline": roofline, "cpu_baseline": cpu}
+        print(json.dumps(line))
+    rrf.rrf_destroy(h)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

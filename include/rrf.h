@@ -14,14 +14,15 @@
  *     elements.  Pointers must be 16-byte aligned and ld*sizeof(element) must be a
  *     multiple of 16 bytes (the tiles are fetched by TMA).
  *   - The caller owns every buffer and the CUDA stream.  The library allocates device
- *     memory only in rrf_create (a few hundred bytes of status words).
+ *     memory only in rrf_create (a few hundred bytes of status words) and, temporarily,
+ *     in the measurement aid rrf_measure_peak.
  *   - Scalars and result structs are HOST memory.
  *   - Every call returns an rrf_status_t; nothing throws, nothing exits.  Arguments are
  *     validated before anything is launched.  Device-side waits are bounded: a wait
  *     that gives up reports RRF_ERR_TIMEOUT and leaves the context usable.
- *   - Block size b must be one of 8, 16, 32, 64, 128; max_rank must be a multiple of b
- *     and at most min(m, n)  (the paper assumes all dimensions divisible by b; here
- *     only max_rank has to be).
+ *   - Block size b must be one of 16, 32, 64, 128 (32, 64, 128 in single precision);
+ *     max_rank must be a multiple of b and at most min(m, n)  (the paper assumes all
+ *     dimensions divisible by b; here only max_rank has to be).  m and n are arbitrary.
  */
 #ifndef RRF_H_
 #define RRF_H_
@@ -163,6 +164,38 @@ rrf_status_t rrf_form_q(rrf_handle_t h, int32_t dtype, int64_t m, int32_t b, int
  */
 rrf_status_t rrf_fill_omega(rrf_handle_t h, int32_t dtype, uint64_t seed, int64_t n, int32_t nvec,
                             int32_t first_vec, void* dOmegaT, int64_t ldo, void* cuda_stream);
+
+/*
+ * Measurement aids (the paper reports wall times only; these have no counterpart in it).
+ *
+ * rrf_set_profiling(h, 1) makes every following rrf_run record a CUDA event on its stream
+ * before each kernel it enqueues; rrf_get_profile then returns, for the last run, the device
+ * time and the number of launches of each phase over the block steps that actually executed
+ * (passes skipped by the device-side stop flag are reported under RRF_PHASE_SKIPPED).
+ * rrf_measure_peak runs a register-resident arithmetic loop on all SMs for about `ms`
+ * milliseconds and reports the achieved rate: kind 0 = FP64 tensor-core mma (m16n8k8),
+ * 1 = FP64 FMA, 2 = FP32 FMA, 3 = TF32 tensor-core mma (m16n8k8).  It synchronises the device.
+ */
+enum {
+  RRF_PHASE_INIT = 0,     /* Algorithm 2 lines 1-4 (and the Gaussian fill when Omega is generated) */
+  RRF_PHASE_SAMPLE = 1,   /* line 7: Y = W[r0:, :] Omega_i */
+  RRF_PHASE_PANEL = 2,    /* line 7: panel Householder QR */
+  RRF_PHASE_TFACTOR = 3,  /* line 7: compact-WY T_i */
+  RRF_PHASE_VTW = 4,      /* line 8: Z = V_i^T W */
+  RRF_PHASE_TZ = 5,       /* line 8: Z <- T_i^T Z */
+  RRF_PHASE_UPDATE = 6,   /* line 8: W -= V_i Z, with the norms of line 9 */
+  RRF_PHASE_STOP = 7,     /* lines 9, 10 and the test of line 5 */
+  RRF_PHASE_SKIPPED = 8,  /* launches of passes after the stop, which return at once */
+  RRF_NPHASES = 9
+};
+typedef struct {
+  double ms[RRF_NPHASES];
+  int32_t launches[RRF_NPHASES];
+  int32_t pad;
+} rrf_profile_t;
+rrf_status_t rrf_set_profiling(rrf_handle_t h, int32_t enable);
+rrf_status_t rrf_get_profile(rrf_handle_t h, rrf_profile_t* out);
+rrf_status_t rrf_measure_peak(rrf_handle_t h, int32_t kind, double ms, double* tflops);
 
 /* Status word of the handle's device side (set by bounded waits), read with one small
  * device-to-host copy after synchronising `cuda_stream`; clears it. */

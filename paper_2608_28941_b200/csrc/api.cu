@@ -5,6 +5,7 @@
 #include <cstdlib>
 #include <cstring>
 #include <new>
+#include <vector>
 
 #include "gemm.cuh"
 #include "panel.cuh"
@@ -28,6 +29,9 @@ struct rrf_ctx {
   rrf::Ctrl* d_ctrl;     // status words for the calls that do not run Algorithm 2's loop
   int last_cuda;
   int panel_smem_max;    // dynamic shared memory the panel kernel may use (opt-in limit minus its static part)
+  int profiling;
+  std::vector<cudaEvent_t> events;
+  rrf_profile_t profile;
 };
 
 namespace rrf {
@@ -193,9 +197,14 @@ static const OpTable* get_ops(int dtype, int b) {
 }
 
 // panel QR + T factor, enqueued on `st`
+struct NoMark {
+  void operator()(int, int) const {}
+};
+template <typename Mark = NoMark>
 static rrf_status_t launch_panel(rrf_ctx* h, int dtype, const void* Y, int nseg, long long seg_stride, int ldy,
                                  long long rows, int b, void* V, long long ldv, void* Tout, long long ldt,
-                                 const PanelScratch& ps, Ctrl* ctrl, const int* done_flag, cudaStream_t st) {
+                                 const PanelScratch& ps, Ctrl* ctrl, const int* done_flag, cudaStream_t st,
+                                 Mark mark = Mark(), int step = 0) {
   PanelPlan pp;
   if (!plan_panel(h, rows, b, &pp)) return RRF_ERR_WORKSPACE;
   int rows_i = (int)rows, R = pp.R, Rp = pp.Rp;
@@ -205,15 +214,18 @@ static rrf_status_t launch_panel(rrf_ctx* h, int dtype, const void* Y, int nseg,
                   &done_flag};
   cudaError_t e;
   const size_t tsmem = ((size_t)b * (b + 1) + b) * sizeof(double);
+  mark(RRF_PHASE_PANEL, step);
   if (dtype == RRF_F64) {
     e = cudaLaunchCooperativeKernel((void*)panel_kernel<double>, dim3(pp.G), dim3(kPanelThreads), args, pp.smem, st);
     if (e == cudaSuccess) {
+      mark(RRF_PHASE_TFACTOR, step);
       tfactor_kernel<double><<<1, 128, tsmem, st>>>(gram, tau, b, (double*)Tout, ldt, done_flag);
       e = cudaGetLastError();
     }
   } else {
     e = cudaLaunchCooperativeKernel((void*)panel_kernel<float>, dim3(pp.G), dim3(kPanelThreads), args, pp.smem, st);
     if (e == cudaSuccess) {
+      mark(RRF_PHASE_TFACTOR, step);
       tfactor_kernel<float><<<1, 128, tsmem, st>>>(gram, tau, b, (float*)Tout, ldt, done_flag);
       e = cudaGetLastError();
     }
@@ -349,6 +361,8 @@ rrf_status_t rrf_create(rrf_handle_t* out, int device) {
   if (h == nullptr) return RRF_ERR_CUDA;
   h->device = device;
   h->last_cuda = 0;
+  h->profiling = 0;
+  std::memset(&h->profile, 0, sizeof(h->profile));
   cudaError_t e = cudaDeviceGetAttribute(&h->sms, cudaDevAttrMultiProcessorCount, device);
   if (e == cudaSuccess) e = cudaDeviceGetAttribute(&h->smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, device);
   void* fn = nullptr;
@@ -373,6 +387,7 @@ rrf_status_t rrf_destroy(rrf_handle_t h) {
   if (h == nullptr) return RRF_ERR_INVALID_ARG;
   cudaSetDevice(h->device);
   cudaFree(h->d_ctrl);
+  for (cudaEvent_t ev : h->events) cudaEventDestroy(ev);
   delete h;
   return RRF_OK;
 }
@@ -385,6 +400,49 @@ rrf_status_t rrf_last_status(rrf_handle_t h, void* cuda_stream) {
   if (cudaStreamSynchronize(st) != cudaSuccess) return RRF_ERR_CUDA;
   if (c.status != 0) cudaMemsetAsync(h->d_ctrl, 0, sizeof(Ctrl), st);
   return (rrf_status_t)c.status;
+}
+
+rrf_status_t rrf_set_profiling(rrf_handle_t h, int32_t enable) {
+  if (h == nullptr) return RRF_ERR_INVALID_ARG;
+  h->profiling = enable ? 1 : 0;
+  return RRF_OK;
+}
+
+rrf_status_t rrf_get_profile(rrf_handle_t h, rrf_profile_t* out) {
+  if (h == nullptr || out == nullptr) return RRF_ERR_INVALID_ARG;
+  *out = h->profile;
+  return RRF_OK;
+}
+
+rrf_status_t rrf_measure_peak(rrf_handle_t h, int32_t kind, double ms, double* tflops) {
+  if (h == nullptr || tflops == nullptr || kind < 0 || kind > 3 || !(ms > 0.0)) return RRF_ERR_INVALID_ARG;
+  if (cudaSetDevice(h->device) != cudaSuccess) return RRF_ERR_CUDA;
+  double* sink = nullptr;
+  const int blocks = h->sms * 2, threads = 256;
+  if (cudaMalloc(&sink, sizeof(double) * blocks * threads) != cudaSuccess) return RRF_ERR_CUDA;
+  cudaEvent_t e0, e1;
+  cudaEventCreate(&e0);
+  cudaEventCreate(&e1);
+  // flops of one loop iteration of one warp
+  const double per_iter = (kind == 0 || kind == 3) ? 8.0 * 2.0 * 16 * 8 * 8 : 32.0 * 16 * 2.0;
+  auto run = [&](int iters) {
+    cudaEventRecord(e0);
+    peak_kernel<<<blocks, threads>>>(sink, iters, kind);
+    cudaEventRecord(e1);
+    cudaEventSynchronize(e1);
+    float t = 0.f;
+    cudaEventElapsedTime(&t, e0, e1);
+    return (double)t;
+  };
+  run(1000);
+  const double t1 = run(20000);
+  const int iters = (int)std::min(2.0e8, std::max(20000.0, 20000.0 * ms / std::max(t1, 1e-3)));
+  const double t = run(iters);
+  *tflops = (double)blocks * (threads / 32) * (double)iters * per_iter / (t * 1e-3) / 1e12;
+  cudaEventDestroy(e0);
+  cudaEventDestroy(e1);
+  cudaFree(sink);
+  return cudaGetLastError() == cudaSuccess ? RRF_OK : RRF_ERR_CUDA;
 }
 
 rrf_status_t rrf_workspace_bytes(const rrf_params_t* p, size_t* bytes) {
@@ -594,7 +652,22 @@ rrf_status_t rrf_run(rrf_handle_t h, const rrf_params_t* p, void* dA, int64_t ld
       !make_map(h, &tmZ, p->dtype, Zt, npad, b, b, kUpdBN))
     return fail(RRF_ERR_INVALID_ARG);
 
+  // profiling: one event before every kernel, tagged with (phase, block step)
+  std::vector<std::pair<int, int>> marks;
+  size_t nev = 0;
+  auto mark = [&](int phase, int step) {
+    if (!h->profiling) return;
+    if (nev == h->events.size()) {
+      cudaEvent_t ev;
+      if (cudaEventCreate(&ev) != cudaSuccess) return;
+      h->events.push_back(ev);
+    }
+    cudaEventRecord(h->events[nev++], st);
+    marks.emplace_back(phase, step);
+  };
+
   // Algorithm 2 lines 1-4
+  mark(RRF_PHASE_INIT, -1);
   if (p->dtype == RRF_F64)
     init_kernel<double><<<L.init_ctas, 256, 0, st>>>((const double*)dA, lda, inplace ? nullptr : (double*)W, ldw, m, n,
                                                      (double*)dV, ldv, p->max_rank, init_part);
@@ -608,24 +681,30 @@ rrf_status_t rrf_run(rrf_handle_t h, const rrf_params_t* p, void* dA, int64_t ld
   for (int i = 0; i < steps; ++i) {
     const int r0 = i * b, rows = (int)(m - r0);
     const SamplePlan sp = plan_sample(rows, n, esize);
+    mark(RRF_PHASE_SAMPLE, i);
     ops->sample(tmW_s, tmO, Ypart, r0, rows, (int)n, r0, sp, ctrl, st);
     s = launch_panel(h, p->dtype, Ypart, sp.nseg, (long long)rows * b, b, rows, b,
                      (char*)dV + ((size_t)r0 * ldv + r0) * esize, ldv, (char*)dT + (size_t)r0 * esize, p->max_rank, ps,
-                     ctrl, &ctrl->done, st);
+                     ctrl, &ctrl->done, st, mark, i);
     if (s != RRF_OK) {
       out->cuda_error = h->last_cuda;
       cudaStreamSynchronize(st);
       return fail(s);
     }
     const VtwPlan vp = plan_vtw(rows, n);
+    mark(RRF_PHASE_VTW, i);
     ops->vtw(tmV_k, tmW_k, Zpart, r0, rows, r0, vp, ctrl, st);
+    mark(RRF_PHASE_TZ, i);
     launch_tz(p->dtype, Zpart, vp.nseg, vp.npad, b, (const char*)dT + (size_t)r0 * esize, p->max_rank, 1, Zt,
               &ctrl->done, st);
+    mark(RRF_PHASE_UPDATE, i);
     ops->update(tmV_u, tmZ, W, ldw, (char*)dB + (size_t)r0 * ldb * esize, ldb, r0, rows, (int)n, r0, b, norm_part, ctrl,
                 st);
     const int nparts = ceil_div(n, kUpdBN) * ceil_div(rows, kUpdBM);
+    mark(RRF_PHASE_STOP, i);
     stop_kernel<<<1, 256, 0, st>>>(norm_part, nparts, b, p->max_rank, p->estimator, fixed ? 1 : 0, tr_sub, tr_dir, ctrl);
   }
+  mark(RRF_PHASE_SKIPPED, steps);   // closing event
   cudaError_t e = cudaGetLastError();
   Ctrl hc;
   if (e == cudaSuccess) e = cudaMemcpyAsync(&hc, ctrl, sizeof(Ctrl), cudaMemcpyDeviceToHost, st);
@@ -634,6 +713,16 @@ rrf_status_t rrf_run(rrf_handle_t h, const rrf_params_t* p, void* dA, int64_t ld
     h->last_cuda = (int)e;
     out->cuda_error = (int)e;
     return fail(RRF_ERR_CUDA);
+  }
+  if (h->profiling && nev > 1) {
+    std::memset(&h->profile, 0, sizeof(h->profile));
+    for (size_t q = 0; q + 1 < nev; ++q) {
+      float ms = 0.f;
+      if (cudaEventElapsedTime(&ms, h->events[q], h->events[q + 1]) != cudaSuccess) continue;
+      const int phase = marks[q].second >= hc.steps ? (int)RRF_PHASE_SKIPPED : marks[q].first;
+      h->profile.ms[phase] += ms;
+      h->profile.launches[phase] += 1;
+    }
   }
   out->status = hc.status;
   out->k = hc.k;

@@ -377,6 +377,54 @@ __global__ void __launch_bounds__(256)
   }
 }
 
+// Register-resident arithmetic loop used to measure the attainable rate of one pipe:
+// kind 0 = f64 mma m16n8k8, 1 = f64 FMA, 2 = f32 FMA, 3 = tf32 mma m16n8k8.
+__global__ void __launch_bounds__(256) peak_kernel(double* __restrict__ sink, int iters, int kind) {
+  double out = 0.0;
+  if (kind == 0) {
+    double c[8][4];
+    for (int i = 0; i < 8; ++i)
+      for (int j = 0; j < 4; ++j) c[i][j] = 0.0;
+    const double a[4] = {threadIdx.x * 1e-9 + 1.0, 2.0, 3.0, 4.0}, b[2] = {threadIdx.x * 1e-9 - 1.0, 0.5};
+    for (int it = 0; it < iters; ++it) {
+#pragma unroll
+      for (int i = 0; i < 8; ++i) mma16x8x8(c[i], a, b);
+    }
+    for (int i = 0; i < 8; ++i)
+      for (int j = 0; j < 4; ++j) out += c[i][j];
+  } else if (kind == 3) {
+    float c[8][4];
+    for (int i = 0; i < 8; ++i)
+      for (int j = 0; j < 4; ++j) c[i][j] = 0.f;
+    const uint32_t a[4] = {threadIdx.x, 1u, 2u, 3u}, b[2] = {threadIdx.x, 5u};
+    for (int it = 0; it < iters; ++it) {
+#pragma unroll
+      for (int i = 0; i < 8; ++i) mma_tf32(c[i], a, b);
+    }
+    for (int i = 0; i < 8; ++i)
+      for (int j = 0; j < 4; ++j) out += c[i][j];
+  } else if (kind == 1) {
+    double c[16];
+    for (int i = 0; i < 16; ++i) c[i] = i;
+    const double a = threadIdx.x * 1e-9 + 1.0, b = 1e-9;
+    for (int it = 0; it < iters; ++it) {
+#pragma unroll
+      for (int i = 0; i < 16; ++i) c[i] = fma(c[i], a, b);
+    }
+    for (int i = 0; i < 16; ++i) out += c[i];
+  } else {
+    float c[16];
+    for (int i = 0; i < 16; ++i) c[i] = (float)i;
+    const float a = threadIdx.x * 1e-9f + 1.0f, b = 1e-9f;
+    for (int it = 0; it < iters; ++it) {
+#pragma unroll
+      for (int i = 0; i < 16; ++i) c[i] = fmaf(c[i], a, b);
+    }
+    for (int i = 0; i < 16; ++i) out += c[i];
+  }
+  sink[(size_t)blockIdx.x * blockDim.x + threadIdx.x] = out;
+}
+
 template <typename T>
 __global__ void __launch_bounds__(256) eye_kernel(T* __restrict__ Q, long long ldq, long long m, int k) {
   const long long total = m * k;

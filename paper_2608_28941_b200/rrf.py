@@ -33,7 +33,14 @@ class rrf_result_t(C.Structure):
                 ("normA2", C.c_double), ("sigma2", C.c_double), ("E_sub", C.c_double), ("E_dir", C.c_double)]
 
 
-EXPORTS = ["rrf_create", "rrf_destroy", "rrf_workspace_bytes", "rrf_run", "rrf_panel_workspace_bytes",
+RRF_PHASES = ["init", "sample", "panel", "tfactor", "vtw", "tz", "update", "stop", "skipped"]
+
+
+class rrf_profile_t(C.Structure):
+    _fields_ = [("ms", C.c_double * 9), ("launches", C.c_int32 * 9), ("pad", C.c_int32)]
+
+
+EXPORTS = ["rrf_set_profiling", "rrf_get_profile", "rrf_measure_peak", "rrf_create", "rrf_destroy", "rrf_workspace_bytes", "rrf_run", "rrf_panel_workspace_bytes",
            "rrf_panel_qr", "rrf_apply_workspace_bytes", "rrf_apply_qt", "rrf_apply_q", "rrf_form_q",
            "rrf_fill_omega", "rrf_last_status", "rrf_status_string"]
 
@@ -61,6 +68,9 @@ def load():
     lib.rrf_form_q.argtypes = [vp, i32, i64, i32, i32, vp, i64, vp, i64, vp, i64, vp, sz, vp]
     lib.rrf_fill_omega.argtypes = [vp, i32, u64, i64, i32, i32, vp, i64, vp]
     lib.rrf_last_status.argtypes = [vp, vp]
+    lib.rrf_set_profiling.argtypes = [vp, i32]
+    lib.rrf_get_profile.argtypes = [vp, C.POINTER(rrf_profile_t)]
+    lib.rrf_measure_peak.argtypes = [vp, i32, C.c_double, C.POINTER(C.c_double)]
     lib.rrf_status_string.argtypes = [C.c_int]
     lib.rrf_status_string.restype = C.c_char_p
     for name in EXPORTS:
@@ -272,3 +282,25 @@ def rrf_fill_omega(h, n: int, nvec: int, seed: int, dtype=torch.float64, first_v
 
 def rrf_last_status(h) -> int:
     return load().rrf_last_status(h, _stream())
+
+
+def rrf_set_profiling(h, enable: bool) -> None:
+    load().rrf_set_profiling(h, 1 if enable else 0)
+
+
+def rrf_get_profile(h) -> dict:
+    """{phase: (milliseconds, launches)} of the last profiled rrf_run."""
+    p = rrf_profile_t()
+    s = load().rrf_get_profile(h, C.byref(p))
+    if s != RRF_OK:
+        raise RrfError(s, "rrf_get_profile")
+    return {name: (p.ms[i], p.launches[i]) for i, name in enumerate(RRF_PHASES)}
+
+
+def rrf_measure_peak(h, kind: int, ms: float = 50.0) -> float:
+    """Attainable TFLOP/s of one pipe: 0 f64 mma, 1 f64 FMA, 2 f32 FMA, 3 tf32 mma."""
+    out = C.c_double()
+    s = load().rrf_measure_peak(h, kind, ms, C.byref(out))
+    if s != RRF_OK:
+        raise RrfError(s, "rrf_measure_peak")
+    return out.value
