@@ -7,7 +7,7 @@
 #include <new>
 #include <vector>
 
-#include "gemm.cuh"
+#include "gemm_sk.cuh"
 #include "panel.cuh"
 
 namespace rrf {
@@ -18,6 +18,7 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
 
 constexpr int kMaxSmem = 232448;   // 227 KB opt-in dynamic shared memory per CTA on sm_100
 constexpr int kTargetCtas = 296;   // split-K until about two CTAs per SM exist
+constexpr int kMaxSms = 160;       // workspace sizes are bounds for devices with up to this many SMs
 
 }  // namespace rrf
 
@@ -41,12 +42,9 @@ static inline int ceil_div(long long a, long long b) { return (int)((a + b - 1) 
 
 // ------------------------------------------------------------------ tile configuration
 constexpr int kSampleBM = 128, kSampleStages = 4;
-constexpr int kVtwBN = 128, kVtwBK = 16, kVtwStages = 4;
-constexpr int kUpdBM = 64, kUpdBN = 64;
+constexpr int kVtwBK = 32;
 
 struct SamplePlan { int nslabs, nseg, kt_per_seg; };
-struct VtwPlan { int ntiles, nseg, kt_per_seg, npad; };
-
 static SamplePlan plan_sample(long long rows, long long n, int esize) {
   SamplePlan p;
   const int KE = 128 / esize;
@@ -57,14 +55,31 @@ static SamplePlan plan_sample(long long rows, long long n, int esize) {
   p.nseg = ceil_div(KT, p.kt_per_seg);
   return p;
 }
-static VtwPlan plan_vtw(long long rows, long long ncols) {
+
+// stream-K plan of Z = V^T C: tiles (column tile, K chunk), one CTA per SM
+struct VtwPlan { int bn, nct, KT, total, tpc, P, npad, slots; };
+static VtwPlan plan_vtw(int sms, long long rows, long long ncols, int bn) {
   VtwPlan p;
-  p.ntiles = ceil_div(ncols, kVtwBN);
-  p.npad = p.ntiles * kVtwBN;
-  const int KT = ceil_div(rows, kVtwBK);
-  int nseg = std::max(1, std::min(std::min(KT, 32), ceil_div(kTargetCtas, p.ntiles)));
-  p.kt_per_seg = ceil_div(KT, nseg);
-  p.nseg = ceil_div(KT, p.kt_per_seg);
+  p.bn = bn;
+  p.nct = ceil_div(ncols, bn);
+  p.npad = ceil_div(ncols, 128) * 128;   // Zt rows: a multiple of every tile width in use
+  p.KT = ceil_div(rows, kVtwBK);
+  p.total = p.nct * p.KT;
+  p.tpc = ceil_div(p.total, sms);
+  p.P = ceil_div(p.total, p.tpc);
+  p.slots = p.P + p.nct;
+  return p;
+}
+// stream-K plan of the fused update: tiles (row slab, column tile)
+struct UpdPlan { int NS, NC, total, tpc, P, slots; };
+static UpdPlan plan_upd(int sms, long long rows, long long ncols, int bm, int bn, int wn) {
+  UpdPlan p;
+  p.NS = ceil_div(rows, bm);
+  p.NC = ceil_div(ncols, bn);
+  p.total = p.NS * p.NC;
+  p.tpc = ceil_div(p.total, sms);
+  p.P = ceil_div(p.total, p.tpc);
+  p.slots = (p.P + p.NS) * wn;
   return p;
 }
 struct PanelPlan { int G, R, Rp; size_t smem; };
@@ -122,25 +137,38 @@ static bool b_ok(int dtype, int b) {
 // ------------------------------------------------------------------ typed launchers
 template <typename T, int B>
 struct Ops {
-  // sample
+  static constexpr int KE = 128 / (int)sizeof(T);
+  // sample (first block only)
   static constexpr int S_WM = (B == 16) ? 8 : 4, S_WN = (B == 16) ? 1 : 2;
   static constexpr int S_SMEM = kSampleStages * (kSampleBM + B) * 128 + 1024;
-  // vtw: M = B
+  // vtw: M = B, 8 consumer warps + 1 producer warp
+  static constexpr int V_BN = (B * (int)sizeof(T) >= 1024) ? 64 : 128;
   static constexpr int V_WM = (B == 16) ? 1 : (B == 128 ? 4 : 2), V_WN = 8 / V_WM;
-  static constexpr int V_SMEM = kVtwStages * kVtwBK * (B + kVtwBN) * (int)sizeof(T) + 1024;
-  // update
-  static constexpr int U_SMEM = B * (int)sizeof(T) * (kUpdBM + kUpdBN) + 1024;
+  static constexpr int V_STAGE = kVtwBK * (B + V_BN) * (int)sizeof(T);
+  static constexpr int V_STAGES = (3 * V_STAGE + 1024 > 200 * 1024) ? 2 : (4 * V_STAGE + 1024 > 200 * 1024 ? 3 : 4);
+  static constexpr int V_SMEM = V_STAGES * V_STAGE + 1024;
+  // fused update: slab height 128 (64 for the widest block), two 128-byte column groups per tile
+  static constexpr int U_BM = (B >= 128) ? 64 : 128;
+  static constexpr int U_BNB = 2;
+  static constexpr int U_WM = U_BM / 16, U_WN = 8 / U_WM;
+  static constexpr int U_BN = U_BNB * KE;
+  static constexpr int U_KB = B / KE;
+  static constexpr int U_VBYTES = U_KB * U_BM * 128;
+  static constexpr int U_STAGE = U_BNB * U_BM * 128 + U_KB * U_BN * 128 + U_BNB * B * 128;
+  static constexpr int U_STAGES = (U_VBYTES + 3 * U_STAGE + 1024 <= 226 * 1024) ? 3 : 2;
+  static constexpr int U_SMEM = U_VBYTES + U_STAGES * U_STAGE + 1024;
+  static_assert(U_SMEM + 1024 <= kMaxSmem && V_SMEM + 1024 <= kMaxSmem && S_SMEM + 1024 <= kMaxSmem, "shared memory");
 
   static cudaError_t setup() {
     cudaError_t e;
     e = cudaFuncSetAttribute(sample_kernel<T, B, kSampleBM, S_WM, S_WN, kSampleStages>,
                              cudaFuncAttributeMaxDynamicSharedMemorySize, S_SMEM);
     if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(vtw_kernel<T, B, kVtwBN, kVtwBK, V_WM, V_WN, kVtwStages>,
+    e = cudaFuncSetAttribute(vtw_sk_kernel<T, B, V_BN, kVtwBK, V_WM, V_WN, V_STAGES>,
                              cudaFuncAttributeMaxDynamicSharedMemorySize, V_SMEM);
     if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(update_kernel<T, B, kUpdBM, kUpdBN, 2, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             U_SMEM);
+    e = cudaFuncSetAttribute(upd_sk_kernel<T, B, U_BM, U_BNB, U_WM, U_WN, U_STAGES>,
+                             cudaFuncAttributeMaxDynamicSharedMemorySize, U_SMEM);
     return e;
   }
   static void sample(const CUtensorMap& tmW, const CUtensorMap& tmO, void* Ypart, int r0, int rows, int n, int j0,
@@ -149,31 +177,34 @@ struct Ops {
         <<<dim3(p.nslabs, p.nseg), S_WM * S_WN * 32, S_SMEM, st>>>(tmW, tmO, (T*)Ypart, r0, rows, n, j0, p.kt_per_seg,
                                                                      ctrl);
   }
-  static void vtw(const CUtensorMap& tmV, const CUtensorMap& tmC, void* Zpart, int r0, int rows, int cv0,
-                  const VtwPlan& p, Ctrl* ctrl, cudaStream_t st) {
-    vtw_kernel<T, B, kVtwBN, kVtwBK, V_WM, V_WN, kVtwStages>
-        <<<dim3(p.ntiles, p.nseg), 256, V_SMEM, st>>>(tmV, tmC, (T*)Zpart, r0, rows, cv0, p.npad, p.kt_per_seg, ctrl);
+  static void vtw(const CUtensorMap& tmV, const CUtensorMap& tmC, void* Zpart, int r0, int cv0, const VtwPlan& p,
+                  Ctrl* ctrl, cudaStream_t st) {
+    vtw_sk_kernel<T, B, V_BN, kVtwBK, V_WM, V_WN, V_STAGES>
+        <<<p.P, 9 * 32, V_SMEM, st>>>(tmV, tmC, (T*)Zpart, r0, cv0, p.KT, p.total, p.tpc, ctrl);
   }
-  static void update(const CUtensorMap& tmV, const CUtensorMap& tmZ, void* C, long long ldc, void* top,
-                     long long ldtop, int r0, int rows, int ncols, int cv0, int top_rows, double* norm_part,
-                     Ctrl* ctrl, cudaStream_t st) {
-    dim3 grid(ceil_div(ncols, kUpdBN), ceil_div(rows, kUpdBM));
-    update_kernel<T, B, kUpdBM, kUpdBN, 2, 2><<<grid, 128, U_SMEM, st>>>(
-        tmV, tmZ, (T*)C, ldc, (T*)top, ldtop, r0, rows, ncols, cv0, top_rows, norm_part, ctrl);
+  static void update(const CUtensorMap& tmV, const CUtensorMap& tmZ, const CUtensorMap& tmC, const CUtensorMap& tmO,
+                     void* C, long long ldc, void* top, long long ldtop, int r0, int rows, int ncols, int cv0,
+                     int top_rows, int j0, void* Ypart, double* norm_part, const UpdPlan& p, Ctrl* ctrl,
+                     cudaStream_t st) {
+    upd_sk_kernel<T, B, U_BM, U_BNB, U_WM, U_WN, U_STAGES><<<p.P, 9 * 32, U_SMEM, st>>>(
+        tmV, tmZ, tmC, tmO, (T*)C, ldc, (T*)top, ldtop, r0, rows, ncols, cv0, top_rows, j0, (T*)Ypart, norm_part, p.NC,
+        p.total, p.tpc, ctrl);
   }
 };
 
 struct OpTable {
+  int v_bn, u_bm, u_bn, u_wn;
   cudaError_t (*setup)();
   void (*sample)(const CUtensorMap&, const CUtensorMap&, void*, int, int, int, int, const SamplePlan&, Ctrl*,
                  cudaStream_t);
-  void (*vtw)(const CUtensorMap&, const CUtensorMap&, void*, int, int, int, const VtwPlan&, Ctrl*, cudaStream_t);
-  void (*update)(const CUtensorMap&, const CUtensorMap&, void*, long long, void*, long long, int, int, int, int, int,
-                 double*, Ctrl*, cudaStream_t);
+  void (*vtw)(const CUtensorMap&, const CUtensorMap&, void*, int, int, const VtwPlan&, Ctrl*, cudaStream_t);
+  void (*update)(const CUtensorMap&, const CUtensorMap&, const CUtensorMap&, const CUtensorMap&, void*, long long,
+                 void*, long long, int, int, int, int, int, int, void*, double*, const UpdPlan&, Ctrl*, cudaStream_t);
 };
 template <typename T, int B>
 static OpTable make_ops() {
-  return OpTable{&Ops<T, B>::setup, &Ops<T, B>::sample, &Ops<T, B>::vtw, &Ops<T, B>::update};
+  return OpTable{Ops<T, B>::V_BN, Ops<T, B>::U_BM, Ops<T, B>::U_BN, Ops<T, B>::U_WN, &Ops<T, B>::setup, &Ops<T, B>::sample,
+                 &Ops<T, B>::vtw,  &Ops<T, B>::update};
 }
 static const OpTable* get_ops(int dtype, int b) {
   static const OpTable d16 = make_ops<double, 16>(), d32 = make_ops<double, 32>(), d64 = make_ops<double, 64>(),
@@ -201,7 +232,7 @@ struct NoMark {
   void operator()(int, int) const {}
 };
 template <typename Mark = NoMark>
-static rrf_status_t launch_panel(rrf_ctx* h, int dtype, const void* Y, int nseg, long long seg_stride, int ldy,
+static rrf_status_t launch_panel(rrf_ctx* h, int dtype, const void* Y, PanelSource src,
                                  long long rows, int b, void* V, long long ldv, void* Tout, long long ldt,
                                  const PanelScratch& ps, Ctrl* ctrl, const int* done_flag, cudaStream_t st,
                                  Mark mark = Mark(), int step = 0) {
@@ -210,8 +241,7 @@ static rrf_status_t launch_panel(rrf_ctx* h, int dtype, const void* Y, int nseg,
   int rows_i = (int)rows, R = pp.R, Rp = pp.Rp;
   double *P = ps.P, *piv = ps.piv, *gram = ps.gram, *tau = ps.tau;
   unsigned* bar = ps.bar;
-  void* args[] = {&Y, &nseg, &seg_stride, &ldy, &rows_i, &b, &R, &Rp, &V, &ldv, &P, &piv, &gram, &tau, &bar, &ctrl,
-                  &done_flag};
+  void* args[] = {&Y, &src, &rows_i, &b, &R, &Rp, &V, &ldv, &P, &piv, &gram, &tau, &bar, &ctrl, &done_flag};
   cudaError_t e;
   const size_t tsmem = ((size_t)b * (b + 1) + b) * sizeof(double);
   mark(RRF_PHASE_PANEL, step);
@@ -237,15 +267,15 @@ static rrf_status_t launch_panel(rrf_ctx* h, int dtype, const void* Y, int nseg,
   return RRF_OK;
 }
 
-static void launch_tz(int dtype, const void* Zpart, int nseg, int npad, int b, const void* Tm, long long ldt,
+static void launch_tz(int dtype, const void* Zpart, const VtwPlan& vp, int b, const void* Tm, long long ldt,
                       int transpose_t, void* Zt, const int* done_flag, cudaStream_t st) {
   const size_t smem = ((size_t)b * (b + 1) + (size_t)kTzCols * (b + 1)) * sizeof(double);
   if (dtype == RRF_F64)
-    tz_kernel<double><<<npad / kTzCols, 256, smem, st>>>((const double*)Zpart, nseg, npad, b, (const double*)Tm, ldt,
-                                                          transpose_t, (double*)Zt, done_flag);
+    tz_kernel<double><<<vp.npad / kTzCols, 256, smem, st>>>((const double*)Zpart, vp.bn, vp.nct, vp.KT, vp.tpc, b,
+                                                            (const double*)Tm, ldt, transpose_t, (double*)Zt, done_flag);
   else
-    tz_kernel<float><<<npad / kTzCols, 256, smem, st>>>((const float*)Zpart, nseg, npad, b, (const float*)Tm, ldt,
-                                                         transpose_t, (float*)Zt, done_flag);
+    tz_kernel<float><<<vp.npad / kTzCols, 256, smem, st>>>((const float*)Zpart, vp.bn, vp.nct, vp.KT, vp.tpc, b,
+                                                           (const float*)Tm, ldt, transpose_t, (float*)Zt, done_flag);
 }
 
 static cudaError_t setup_all(int smem_optin, int* panel_smem_max) {
@@ -289,30 +319,33 @@ struct RunLayout {
 constexpr int kInitCtas = 148 * 8;
 
 static bool run_layout(const rrf_params_t* p, bool need_omega, RunLayout* L) {
+  const int sms = kMaxSms;
   const int esize = p->dtype == RRF_F64 ? 8 : 4;
   const int b = p->b, steps = p->max_rank / b;
+  const OpTable* ops = get_ops(p->dtype, b);
   size_t ymax = 0, zmax = 0;
-  int npad = 0, normmax = 0;
+  int npad = 0;
   for (int i = 0; i < steps; ++i) {
     const long long rows = p->m - (long long)i * b;
     const SamplePlan sp = plan_sample(rows, p->n, esize);
     ymax = std::max(ymax, (size_t)sp.nseg * (size_t)rows * b);
-    const VtwPlan vp = plan_vtw(rows, p->n);
-    zmax = std::max(zmax, (size_t)vp.nseg * b * (size_t)vp.npad);
+    const UpdPlan up = plan_upd(sms, rows, p->n, ops->u_bm, ops->u_bn, ops->u_wn);
+    ymax = std::max(ymax, (size_t)(sms + up.NS) * ops->u_wn * ops->u_bm * b);   // slots <= (P + NS) * wn, P <= sms
+    const VtwPlan vp = plan_vtw(sms, rows, p->n, ops->v_bn);
+    zmax = std::max(zmax, (size_t)(sms + vp.nct) * b * ops->v_bn);
     npad = vp.npad;
-    normmax = std::max(normmax, ceil_div(p->n, kUpdBN) * ceil_div(rows, kUpdBM));
   }
   size_t off = 0;
   L->ctrl = off; off += 256;
   L->traces = off; off += align_up((size_t)2 * steps * sizeof(double), 256);
   L->init_ctas = kInitCtas;
   L->init_part = off; off += align_up((size_t)kInitCtas * sizeof(double), 256);
-  L->max_norm_parts = normmax;
-  L->norm_part = off; off += align_up((size_t)2 * normmax * sizeof(double), 256);
+  L->max_norm_parts = sms;
+  L->norm_part = off; off += align_up((size_t)2 * sms * sizeof(double), 256);
   L->ypart = off; off += align_up(ymax * esize, 256);
   L->zpart = off; off += align_up(zmax * esize, 256);
   L->zt = off; off += align_up((size_t)npad * b * esize, 256);
-  L->panel = off; off += panel_scratch_bytes(148 * 2, b);
+  L->panel = off; off += panel_scratch_bytes(sms, b);
   L->w = off;
   L->ldw = (long long)align_up((size_t)p->n, 16);   // rows of the working copy start on 128-byte lines
   if (!(p->flags & RRF_FLAG_INPLACE)) off += align_up((size_t)p->m * (size_t)L->ldw * esize, 256);
@@ -369,6 +402,7 @@ rrf_status_t rrf_create(rrf_handle_t* out, int device) {
   cudaDriverEntryPointQueryResult q;
   if (e == cudaSuccess) e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q);
   if (e == cudaSuccess && (fn == nullptr || q != cudaDriverEntryPointSuccess)) e = cudaErrorUnknown;
+  if (e == cudaSuccess && h->sms > kMaxSms) e = cudaErrorInvalidConfiguration;
   h->encode = reinterpret_cast<EncodeTiledFn>(fn);
   if (e == cudaSuccess) e = setup_all(h->smem_optin, &h->panel_smem_max);
   if (e == cudaSuccess) e = cudaMalloc(&h->d_ctrl, sizeof(Ctrl));
@@ -476,7 +510,7 @@ rrf_status_t rrf_fill_omega(rrf_handle_t h, int32_t dtype, uint64_t seed, int64_
 
 rrf_status_t rrf_panel_workspace_bytes(int32_t dtype, int64_t rows, int32_t b, size_t* bytes) {
   if (bytes == nullptr || !b_ok(dtype, b) || rows < b) return RRF_ERR_INVALID_ARG;
-  *bytes = panel_scratch_bytes(148 * 2, b);
+  *bytes = panel_scratch_bytes(kMaxSms, b);
   return RRF_OK;
 }
 
@@ -487,23 +521,24 @@ rrf_status_t rrf_panel_qr(rrf_handle_t h, int32_t dtype, int64_t rows, int32_t b
     return RRF_ERR_INVALID_ARG;
   if (!b_ok(dtype, b) || rows < b || rows > 0x7fffffffLL || ldy < b || ldv < b || ldt < b || ldy > 0x7fffffffLL)
     return RRF_ERR_INVALID_ARG;
-  if (workspace_bytes < panel_scratch_bytes(148 * 2, b) || h->sms > 148 * 2) return RRF_ERR_WORKSPACE;
+  if (workspace_bytes < panel_scratch_bytes(kMaxSms, b) ) return RRF_ERR_WORKSPACE;
   cudaStream_t st = (cudaStream_t)cuda_stream;
   PanelScratch ps = carve_panel((unsigned char*)d_workspace, h->sms, b);
   if (cudaMemsetAsync(ps.bar, 0, sizeof(unsigned), st) != cudaSuccess) return RRF_ERR_CUDA;
-  return launch_panel(h, dtype, dY, 1, 0, (int)ldy, rows, b, dV, ldv, dT, ldt, ps, h->d_ctrl, &h->d_ctrl->done, st);
+  PanelSource src{};
+  src.slots = 0;
+  src.nseg = 1;
+  src.seg_stride = 0;
+  src.ldy = (int)ldy;
+  return launch_panel(h, dtype, dY, src, rows, b, dV, ldv, dT, ldt, ps, h->d_ctrl, &h->d_ctrl->done, st);
 }
 
 rrf_status_t rrf_apply_workspace_bytes(int32_t dtype, int64_t m, int64_t ncols, int32_t b, size_t* bytes) {
   if (bytes == nullptr || !b_ok(dtype, b) || m < b || ncols < 1) return RRF_ERR_INVALID_ARG;
   const int esize = dtype == RRF_F64 ? 8 : 4;
-  const VtwPlan vp = plan_vtw(m, ncols);   // the first block has the most rows and segments are capped
-  size_t zmax = 0;
-  for (long long r0 = 0; r0 + b <= m; r0 += b) {
-    const VtwPlan q = plan_vtw(m - r0, ncols);
-    zmax = std::max(zmax, (size_t)q.nseg * b * (size_t)q.npad);
-  }
-  *bytes = align_up(zmax * esize, 256) + align_up((size_t)vp.npad * b * esize, 256);
+  const VtwPlan vp = plan_vtw(kMaxSms, m, ncols, get_ops(dtype, b)->v_bn);
+  const size_t zslots = (size_t)(kMaxSms + vp.nct) * b * vp.bn;
+  *bytes = align_up((size_t)vp.npad * b * esize, 256) + align_up(zslots * esize, 256);
   return RRF_OK;
 }
 
@@ -527,23 +562,25 @@ static rrf_status_t apply_blocks(rrf_handle_t h, int dtype, long long m, int b, 
   if (workspace_bytes < need || (reinterpret_cast<uintptr_t>(d_workspace) & 255u)) return RRF_ERR_WORKSPACE;
   if (k == 0) return RRF_OK;
   const OpTable* ops = get_ops(dtype, b);
-  const VtwPlan vp0 = plan_vtw(m, ncols);
+  const VtwPlan vp0 = plan_vtw(kMaxSms, m, ncols, ops->v_bn);
   unsigned char* ws = (unsigned char*)d_workspace;
   void* Zt = ws;
   void* Zpart = ws + align_up((size_t)vp0.npad * b * esize, 256);
-  CUtensorMap tmV_k, tmC_k, tmV_u, tmZ;
+  CUtensorMap tmV_k, tmC_k, tmV_u, tmC_u, tmZ;
   if (!make_map(h, &tmV_k, dtype, dV, m, k, ldv, kVtwBK) || !make_map(h, &tmC_k, dtype, dC, m, ncols, ldc, kVtwBK) ||
-      !make_map(h, &tmV_u, dtype, dV, m, k, ldv, kUpdBM) || !make_map(h, &tmZ, dtype, Zt, vp0.npad, b, b, kUpdBN))
+      !make_map(h, &tmV_u, dtype, dV, m, k, ldv, ops->u_bm) || !make_map(h, &tmC_u, dtype, dC, m, ncols, ldc, ops->u_bm) ||
+      !make_map(h, &tmZ, dtype, Zt, vp0.npad, b, b, ops->u_bn))
     return RRF_ERR_INVALID_ARG;
   const int nblk = k / b;
   for (int q = 0; q < nblk; ++q) {
     const int l = transpose ? q : nblk - 1 - q;
     const int r0 = l * b, rows = (int)(m - r0);
-    const VtwPlan vp = plan_vtw(rows, ncols);
-    ops->vtw(tmV_k, tmC_k, Zpart, r0, rows, r0, vp, h->d_ctrl, st);
-    launch_tz(dtype, Zpart, vp.nseg, vp.npad, b, (const char*)dT + (size_t)r0 * esize, ldt, transpose ? 1 : 0, Zt,
-              &h->d_ctrl->done, st);
-    ops->update(tmV_u, tmZ, dC, ldc, (char*)dC + (size_t)r0 * ldc * esize, ldc, r0, rows, (int)ncols, r0, 0, nullptr,
+    const VtwPlan vp = plan_vtw(h->sms, rows, ncols, ops->v_bn);
+    ops->vtw(tmV_k, tmC_k, Zpart, r0, r0, vp, h->d_ctrl, st);
+    launch_tz(dtype, Zpart, vp, b, (const char*)dT + (size_t)r0 * esize, ldt, transpose ? 1 : 0, Zt, &h->d_ctrl->done,
+              st);
+    const UpdPlan up = plan_upd(h->sms, rows, ncols, ops->u_bm, ops->u_bn, ops->u_wn);
+    ops->update(tmV_u, tmZ, tmC_u, tmC_u, dC, ldc, dC, ldc, r0, rows, (int)ncols, r0, 0, -1, nullptr, nullptr, up,
                 h->d_ctrl, st);
   }
   const cudaError_t e = cudaGetLastError();
@@ -611,7 +648,6 @@ rrf_status_t rrf_run(rrf_handle_t h, const rrf_params_t* p, void* dA, int64_t ld
   RunLayout L;
   run_layout(p, dOmegaT == nullptr, &L);
   if (workspace_bytes < L.total) return fail(RRF_ERR_WORKSPACE);
-  if (h->sms > 148 * 2) return fail(RRF_ERR_WORKSPACE);
   PanelPlan pp0;
   if (!plan_panel(h, m, b, &pp0)) return fail(RRF_ERR_WORKSPACE);   // first (tallest) panel must fit on chip
 
@@ -642,14 +678,15 @@ rrf_status_t rrf_run(rrf_handle_t h, const rrf_params_t* p, void* dA, int64_t ld
     if (s != RRF_OK) return fail(s);
   }
   const OpTable* ops = get_ops(p->dtype, b);
-  const int npad = plan_vtw(m, n).npad;
-  CUtensorMap tmW_s, tmO, tmV_k, tmW_k, tmV_u, tmZ;
+  const int npad = plan_vtw(h->sms, m, n, ops->v_bn).npad;
+  CUtensorMap tmW_s, tmO, tmV_k, tmW_k, tmV_u, tmW_u, tmZ;
   if (!make_map(h, &tmW_s, p->dtype, W, m, n, ldw, kSampleBM) ||
       !make_map(h, &tmO, p->dtype, Om, p->max_rank, n, ldom, b) ||
       !make_map(h, &tmV_k, p->dtype, dV, m, p->max_rank, ldv, kVtwBK) ||
       !make_map(h, &tmW_k, p->dtype, W, m, n, ldw, kVtwBK) ||
-      !make_map(h, &tmV_u, p->dtype, dV, m, p->max_rank, ldv, kUpdBM) ||
-      !make_map(h, &tmZ, p->dtype, Zt, npad, b, b, kUpdBN))
+      !make_map(h, &tmV_u, p->dtype, dV, m, p->max_rank, ldv, ops->u_bm) ||
+      !make_map(h, &tmW_u, p->dtype, W, m, n, ldw, ops->u_bm) ||
+      !make_map(h, &tmZ, p->dtype, Zt, npad, b, b, ops->u_bn))
     return fail(RRF_ERR_INVALID_ARG);
 
   // profiling: one event before every kernel, tagged with (phase, block step)
@@ -677,32 +714,46 @@ rrf_status_t rrf_run(rrf_handle_t h, const rrf_params_t* p, void* dA, int64_t ld
   init_ctrl_kernel<<<1, 256, 0, st>>>(init_part, L.init_ctas, p->tol, p->tol_is_relative, fixed ? 1 : 0, b, p->max_rank,
                                       ctrl);
 
-  // Algorithm 2 lines 5-11: every pass is enqueued; passes after the stop return at once
+  // Algorithm 2 lines 5-11: every pass is enqueued; passes after the stop return at once.
+  // The panel of pass 0 is sampled by its own kernel; the panel of pass i+1 comes out of the
+  // fused update of pass i.
+  PanelSource src{};
+  {
+    const SamplePlan sp = plan_sample(m, n, esize);
+    mark(RRF_PHASE_SAMPLE, 0);
+    ops->sample(tmW_s, tmO, Ypart, 0, (int)m, (int)n, 0, sp, ctrl, st);
+    src.slots = 0;
+    src.nseg = sp.nseg;
+    src.seg_stride = m * b;
+    src.ldy = b;
+  }
   for (int i = 0; i < steps; ++i) {
     const int r0 = i * b, rows = (int)(m - r0);
-    const SamplePlan sp = plan_sample(rows, n, esize);
-    mark(RRF_PHASE_SAMPLE, i);
-    ops->sample(tmW_s, tmO, Ypart, r0, rows, (int)n, r0, sp, ctrl, st);
-    s = launch_panel(h, p->dtype, Ypart, sp.nseg, (long long)rows * b, b, rows, b,
-                     (char*)dV + ((size_t)r0 * ldv + r0) * esize, ldv, (char*)dT + (size_t)r0 * esize, p->max_rank, ps,
-                     ctrl, &ctrl->done, st, mark, i);
+    s = launch_panel(h, p->dtype, Ypart, src, rows, b, (char*)dV + ((size_t)r0 * ldv + r0) * esize, ldv,
+                     (char*)dT + (size_t)r0 * esize, p->max_rank, ps, ctrl, &ctrl->done, st, mark, i);
     if (s != RRF_OK) {
       out->cuda_error = h->last_cuda;
       cudaStreamSynchronize(st);
       return fail(s);
     }
-    const VtwPlan vp = plan_vtw(rows, n);
+    const VtwPlan vp = plan_vtw(h->sms, rows, n, ops->v_bn);
     mark(RRF_PHASE_VTW, i);
-    ops->vtw(tmV_k, tmW_k, Zpart, r0, rows, r0, vp, ctrl, st);
+    ops->vtw(tmV_k, tmW_k, Zpart, r0, r0, vp, ctrl, st);
     mark(RRF_PHASE_TZ, i);
-    launch_tz(p->dtype, Zpart, vp.nseg, vp.npad, b, (const char*)dT + (size_t)r0 * esize, p->max_rank, 1, Zt,
-              &ctrl->done, st);
+    launch_tz(p->dtype, Zpart, vp, b, (const char*)dT + (size_t)r0 * esize, p->max_rank, 1, Zt, &ctrl->done, st);
+    const UpdPlan up = plan_upd(h->sms, rows, n, ops->u_bm, ops->u_bn, ops->u_wn);
+    const int j0 = (i + 1 < steps) ? r0 + b : -1;   // Omega rows of the next pass, if there is one
     mark(RRF_PHASE_UPDATE, i);
-    ops->update(tmV_u, tmZ, W, ldw, (char*)dB + (size_t)r0 * ldb * esize, ldb, r0, rows, (int)n, r0, b, norm_part, ctrl,
-                st);
-    const int nparts = ceil_div(n, kUpdBN) * ceil_div(rows, kUpdBM);
+    ops->update(tmV_u, tmZ, tmW_u, tmO, W, ldw, (char*)dB + (size_t)r0 * ldb * esize, ldb, r0, rows, (int)n, r0, b, j0,
+                Ypart, norm_part, up, ctrl, st);
     mark(RRF_PHASE_STOP, i);
-    stop_kernel<<<1, 256, 0, st>>>(norm_part, nparts, b, p->max_rank, p->estimator, fixed ? 1 : 0, tr_sub, tr_dir, ctrl);
+    stop_kernel<<<1, 256, 0, st>>>(norm_part, up.P, b, p->max_rank, p->estimator, fixed ? 1 : 0, tr_sub, tr_dir, ctrl);
+    src.slots = 1;
+    src.row_off = b;
+    src.bm = ops->u_bm;
+    src.nc = up.NC;
+    src.tpc = up.tpc;
+    src.wn = ops->u_wn;
   }
   mark(RRF_PHASE_SKIPPED, steps);   // closing event
   cudaError_t e = cudaGetLastError();

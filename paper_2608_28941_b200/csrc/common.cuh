@@ -107,7 +107,9 @@ __device__ __forceinline__ void mma_tf32(float (&c)[4], const uint32_t (&a)[4], 
       : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b[0]), "r"(b[1]));
 }
 // fp32 product by the 3xTF32 split: x = hi + lo with hi = tf32(x), lo = tf32(x - hi);
-// C += A_lo*B_hi + A_hi*B_lo + A_hi*B_hi (small terms first; A_lo*B_lo is below fp32 round-off).
+// D = A_lo*B_hi + A_hi*B_lo + A_hi*B_hi (small terms first; A_lo*B_lo is below fp32 round-off),
+// then C += D with an ordinary round-to-nearest add: the tensor core's own accumulation does not
+// round to nearest, so only the eight products of one k-step are summed inside it.
 __device__ __forceinline__ void mma16x8x8(float (&c)[4], const float (&a)[4], const float (&b)[2]) {
   uint32_t ah[4], al[4], bh[2], bl[2];
 #pragma unroll
@@ -120,9 +122,12 @@ __device__ __forceinline__ void mma16x8x8(float (&c)[4], const float (&a)[4], co
     bh[i] = to_tf32(b[i]);
     bl[i] = to_tf32(b[i] - __uint_as_float(bh[i]));
   }
-  mma_tf32(c, al, bh);
-  mma_tf32(c, ah, bl);
-  mma_tf32(c, ah, bh);
+  float d[4] = {0.f, 0.f, 0.f, 0.f};
+  mma_tf32(d, al, bh);
+  mma_tf32(d, ah, bl);
+  mma_tf32(d, ah, bh);
+#pragma unroll
+  for (int i = 0; i < 4; ++i) c[i] += d[i];
 }
 
 // ---------------------------------------------------------------- small utilities

@@ -1,0 +1,409 @@
+// Persistent ("stream-K") versions of the two large contractions of a block step.
+//
+// Both kernels run one CTA per SM.  The tiles of the problem are numbered along the
+// direction in which an accumulator can stay in registers, and CTA p owns the contiguous
+// range [p*tpc, (p+1)*tpc) of them, so every SM gets the same amount of work whatever the
+// trailing matrix's height.  When a CTA's range crosses from one accumulator to the next it
+// writes a partial result to slot (p + index of the accumulator): consecutive (CTA,
+// accumulator) pairs differ in p, in the index, or in both, so the slot is unique, and the
+// consumer of the partials (panel loader, Z reduction) sums the slots of one accumulator in
+// CTA order - a fixed order, so results are reproducible bit for bit.
+//
+// One extra warp per CTA only issues TMA loads; the consumer warps never wait for each other
+// (full/empty mbarriers per stage, every wait bounded).
+//
+//   vtw_sk_kernel   Z = V_i^T W[r0:, :]                      (Algorithm 2 line 8, first product)
+//   upd_sk_kernel   W[r0:, :] -= V_i Zt^T, norms of line 9, and - fused, from the updated tile
+//                   still in registers - the next panel Y = W_new Omega_{i+1} (line 7 of the
+//                   next pass), which saves one full read of W per block step.
+#pragma once
+
+#include "gemm.cuh"
+
+namespace rrf {
+
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+
+template <typename T, int MT, int NT>
+__device__ __forceinline__ void flush_tile(T (&acc)[MT][NT][4], T* __restrict__ dst, int ld, int row0, int col0,
+                                           int g, int t) {
+#pragma unroll
+  for (int a = 0; a < MT; ++a)
+#pragma unroll
+    for (int cc = 0; cc < NT; ++cc) {
+      const int r = row0 + a * 16 + g;
+      const int col = col0 + cc * 8 + 2 * t;
+      store2(dst + (size_t)r * ld + col, acc[a][cc][0], acc[a][cc][1]);
+      store2(dst + (size_t)(r + 8) * ld + col, acc[a][cc][2], acc[a][cc][3]);
+#pragma unroll
+      for (int e = 0; e < 4; ++e) acc[a][cc][e] = T(0);
+    }
+}
+
+// ------------------------------------------------------------------------------------------
+// Z partials.  Tiles: L = c*KT + kt (column tile c of BN columns, K chunk kt of BK rows).
+// Slot (p + c) of Zpart holds a B x BN partial of column tile c.
+// ------------------------------------------------------------------------------------------
+template <typename T, int B, int BN, int BK, int WM, int WN, int STAGES>
+__global__ void __launch_bounds__((WM * WN + 1) * 32)
+    vtw_sk_kernel(const __grid_constant__ CUtensorMap tmV,  // V [m][ldv], box [BK][KE]
+                  const __grid_constant__ CUtensorMap tmC,  // C [m][ncols], box [BK][KE]
+                  T* __restrict__ Zpart, int r0, int cv0, int KT, int total, int tpc, Ctrl* ctrl) {
+  if (*reinterpret_cast<volatile int*>(&ctrl->done)) return;
+  constexpr int KE = Elem<T>::KE;
+  constexpr int NCW = WM * WN;
+  constexpr int TM = B / WM, TN = BN / WN, MT = TM / 16, NT = TN / 8;
+  static_assert(TM % 16 == 0 && TN % 8 == 0 && B % KE == 0 && BN % KE == 0 && BK % 8 == 0, "tile");
+  constexpr int NBV = B / KE, NBC = BN / KE;
+  constexpr int BOX_BYTES = BK * 128;
+  constexpr int V_BYTES = NBV * BOX_BYTES, C_BYTES = NBC * BOX_BYTES, STAGE_BYTES = V_BYTES + C_BYTES;
+
+  extern __shared__ unsigned char smem_raw[];
+  unsigned char* smem = align1024(smem_raw);
+  __shared__ uint64_t full[STAGES], empty[STAGES];
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
+  const int p = blockIdx.x;
+  const int L0 = p * tpc;
+  const int ntile = min(total, L0 + tpc) - L0;
+
+  if (tid == 0) {
+    for (int s = 0; s < STAGES; ++s) {
+      mbar_init(&full[s], 1);
+      mbar_init(&empty[s], NCW);
+    }
+    mbar_fence_init();
+  }
+  __syncthreads();
+
+  if (warp == NCW) {
+    if (lane == 0) {
+      for (int i = 0; i < ntile; ++i) {
+        const int st = i % STAGES;
+        if (i >= STAGES && !mbar_wait(&empty[st], ((i / STAGES) - 1) & 1, ctrl)) return;
+        const int L = L0 + i, c = L / KT, kt = L - c * KT;
+        unsigned char* sV = smem + st * STAGE_BYTES;
+        const int y = r0 + kt * BK;
+        mbar_expect_tx(&full[st], STAGE_BYTES);
+#pragma unroll
+        for (int v = 0; v < NBV; ++v) tma_load_2d(sV + v * BOX_BYTES, &tmV, cv0 + v * KE, y, &full[st]);
+#pragma unroll
+        for (int cb = 0; cb < NBC; ++cb)
+          tma_load_2d(sV + V_BYTES + cb * BOX_BYTES, &tmC, c * BN + cb * KE, y, &full[st]);
+      }
+    }
+    return;
+  }
+
+  const int wm = warp / WN, wn = warp % WN;
+  T acc[MT][NT][4];
+#pragma unroll
+  for (int a = 0; a < MT; ++a)
+#pragma unroll
+    for (int c = 0; c < NT; ++c)
+#pragma unroll
+      for (int e = 0; e < 4; ++e) acc[a][c][e] = T(0);
+
+  int cur_c = L0 / KT;
+  for (int i = 0; i < ntile; ++i) {
+    const int c = (L0 + i) / KT;
+    if (c != cur_c) {
+      flush_tile<T, MT, NT>(acc, Zpart + (size_t)(p + cur_c) * (size_t)(B * BN), BN, wm * TM, wn * TN, g, t);
+      cur_c = c;
+    }
+    const int st = i % STAGES;
+    if (!mbar_wait(&full[st], (i / STAGES) & 1, ctrl)) return;
+    const unsigned char* sV = smem + st * STAGE_BYTES;
+    const unsigned char* sC = sV + V_BYTES;
+#pragma unroll
+    for (int ks = 0; ks < BK / 8; ++ks) {
+      const uint32_t k = ks * 8 + 2 * t;
+      T af[MT][4], bf[NT][2];
+#pragma unroll
+      for (int a = 0; a < MT; ++a) {
+        const int j = wm * TM + a * 16 + g;
+        const unsigned char* box_lo = sV + (j / KE) * BOX_BYTES;
+        const unsigned char* box_hi = sV + ((j + 8) / KE) * BOX_BYTES;
+        const uint32_t c_lo = (j % KE) * sizeof(T), c_hi = ((j + 8) % KE) * sizeof(T);
+        af[a][0] = *reinterpret_cast<const T*>(box_lo + swz128(k * 128 + c_lo));
+        af[a][1] = *reinterpret_cast<const T*>(box_hi + swz128(k * 128 + c_hi));
+        af[a][2] = *reinterpret_cast<const T*>(box_lo + swz128((k + 1) * 128 + c_lo));
+        af[a][3] = *reinterpret_cast<const T*>(box_hi + swz128((k + 1) * 128 + c_hi));
+      }
+#pragma unroll
+      for (int cc = 0; cc < NT; ++cc) {
+        const int nn = wn * TN + cc * 8 + g;
+        const unsigned char* box = sC + (nn / KE) * BOX_BYTES;
+        const uint32_t co = (nn % KE) * sizeof(T);
+        bf[cc][0] = *reinterpret_cast<const T*>(box + swz128(k * 128 + co));
+        bf[cc][1] = *reinterpret_cast<const T*>(box + swz128((k + 1) * 128 + co));
+      }
+#pragma unroll
+      for (int a = 0; a < MT; ++a)
+#pragma unroll
+        for (int cc = 0; cc < NT; ++cc) mma16x8x8(acc[a][cc], af[a], bf[cc]);
+    }
+    __syncwarp();
+    if (lane == 0) mbar_arrive(&empty[st]);
+  }
+  if (ntile > 0)
+    flush_tile<T, MT, NT>(acc, Zpart + (size_t)(p + cur_c) * (size_t)(B * BN), BN, wm * TM, wn * TN, g, t);
+}
+
+// ------------------------------------------------------------------------------------------
+// Fused update + next sample.  Tiles: L = s*NC + c (row slab s of BM rows, column tile c of BN
+// columns); a CTA keeps V[slab] in shared memory and the slab's Y accumulator in registers.
+//   P     = V[slab, :] * Zt[col tile, :]^T                 (K = B)
+//   Wnew  = W[slab, col tile] - P   -> global (block row B_i to `top`, the rest back to C)
+//   Y    += Wnew * OmegaT[j0 .. j0+B, col tile]^T          (K = BN; only if j0 >= 0)
+// The accumulator fragment of Wnew is used directly as the A operand of the second product:
+// within one 128-byte group of columns, thread t of a quad holds the KE/4 consecutive columns
+// (KE/4)*t ..., i.e. n-tile u of the group covers columns (KE/4)*t + 2u + {0, 1}, which are
+// exactly k-slots (t, t+4) of one m16n8k8 step whose B operand is read from OmegaT with the
+// same chunk rule as every other K-contiguous operand.  No shuffles, no shared-memory round trip.
+// Slot ((p + s)*WN + wn) of Ypart holds the BM x B partial of slab s from CTA p, warp column wn.
+// ------------------------------------------------------------------------------------------
+template <typename T, int B, int BM, int BNB, int WM, int WN, int STAGES>
+__global__ void __launch_bounds__((WM * WN + 1) * 32, 1)
+    upd_sk_kernel(const __grid_constant__ CUtensorMap tmV,  // V [m][ldv], box [BM][KE]
+                  const __grid_constant__ CUtensorMap tmZ,  // Zt [npad][B], box [BN][KE]
+                  const __grid_constant__ CUtensorMap tmC,  // C [m][ncols], box [BM][KE]
+                  const __grid_constant__ CUtensorMap tmO,  // OmegaT [max_rank][n], box [B][KE]
+                  T* __restrict__ C, long long ldc, T* __restrict__ top, long long ldtop,
+                  int r0, int rows, int ncols, int cv0, int top_rows, int j0,
+                  T* __restrict__ Ypart, double* __restrict__ norm_part,
+                  int NC, int total, int tpc, Ctrl* ctrl) {
+  if (*reinterpret_cast<volatile int*>(&ctrl->done)) return;
+  constexpr int KE = Elem<T>::KE, NV = Elem<T>::NV, KS = Elem<T>::KS;
+  constexpr int U = KE / 8;            // n-tiles per 128-byte column group
+  constexpr int NCW = WM * WN;
+  constexpr int BN = BNB * KE;
+  constexpr int KB = B / KE;           // 128-byte K boxes of V and Zt
+  constexpr int TM = BM / WM, MT = TM / 16;
+  constexpr int QW = BNB / WN;         // column groups per warp
+  constexpr int NTB = B / 8;           // n-tiles of the Y accumulator
+  static_assert(TM % 16 == 0 && BNB % WN == 0 && B % KE == 0, "tile");
+  constexpr int V_BOX = BM * 128, W_BOX = BM * 128, Z_BOX = BN * 128, O_BOX = B * 128;
+  constexpr int V_BYTES = KB * V_BOX;
+  constexpr int W_BYTES = BNB * W_BOX, Z_BYTES = KB * Z_BOX, O_BYTES = BNB * O_BOX;
+  constexpr int STAGE_BYTES = W_BYTES + Z_BYTES + O_BYTES;
+
+  extern __shared__ unsigned char smem_raw[];
+  unsigned char* smem = align1024(smem_raw);
+  unsigned char* sVs = smem;
+  unsigned char* sStage = smem + V_BYTES;
+  __shared__ uint64_t full[STAGES], empty[STAGES], v_full, v_empty;
+  __shared__ double red[64];
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
+  const int p = blockIdx.x;
+  const int L0 = p * tpc;
+  const int ntile = min(total, L0 + tpc) - L0;
+  const bool do_sample = j0 >= 0;
+
+  if (tid == 0) {
+    for (int s = 0; s < STAGES; ++s) {
+      mbar_init(&full[s], 1);
+      mbar_init(&empty[s], NCW);
+    }
+    mbar_init(&v_full, 1);
+    mbar_init(&v_empty, NCW);
+    mbar_fence_init();
+  }
+  __syncthreads();
+
+  double s_top = 0.0, s_trail = 0.0;
+
+  if (warp == NCW) {
+    // ------------------------------------------------------------ producer warp
+    if (lane == 0) {
+      int cur_s = -1, nslab = 0;
+      for (int i = 0; i < ntile; ++i) {
+        const int L = L0 + i, s = L / NC, c = L - s * NC;
+        if (s != cur_s) {
+          if (nslab > 0 && !mbar_wait(&v_empty, (nslab - 1) & 1, ctrl)) break;
+          mbar_expect_tx(&v_full, V_BYTES);
+#pragma unroll
+          for (int kb = 0; kb < KB; ++kb) tma_load_2d(sVs + kb * V_BOX, &tmV, cv0 + kb * KE, r0 + s * BM, &v_full);
+          cur_s = s;
+          ++nslab;
+        }
+        const int st = i % STAGES;
+        if (i >= STAGES && !mbar_wait(&empty[st], ((i / STAGES) - 1) & 1, ctrl)) break;
+        unsigned char* sW = sStage + st * STAGE_BYTES;
+        mbar_expect_tx(&full[st], do_sample ? STAGE_BYTES : W_BYTES + Z_BYTES);
+#pragma unroll
+        for (int q = 0; q < BNB; ++q) tma_load_2d(sW + q * W_BOX, &tmC, c * BN + q * KE, r0 + s * BM, &full[st]);
+#pragma unroll
+        for (int kb = 0; kb < KB; ++kb) tma_load_2d(sW + W_BYTES + kb * Z_BOX, &tmZ, kb * KE, c * BN, &full[st]);
+        if (do_sample) {
+#pragma unroll
+          for (int q = 0; q < BNB; ++q)
+            tma_load_2d(sW + W_BYTES + Z_BYTES + q * O_BOX, &tmO, c * BN + q * KE, j0, &full[st]);
+        }
+      }
+    }
+  } else {
+    // ------------------------------------------------------------ consumer warps
+    const int wm = warp / WN, wn = warp % WN;
+    T accY[MT][NTB][4];
+#pragma unroll
+    for (int a = 0; a < MT; ++a)
+#pragma unroll
+      for (int nb = 0; nb < NTB; ++nb)
+#pragma unroll
+        for (int e = 0; e < 4; ++e) accY[a][nb][e] = T(0);
+
+    int cur_s = -1, nslab = 0;
+    bool ok = true;
+    for (int i = 0; i < ntile && ok; ++i) {
+      const int L = L0 + i, s = L / NC, c = L - s * NC;
+      if (s != cur_s) {
+        if (cur_s >= 0) {
+          if (do_sample)
+            flush_tile<T, MT, NTB>(accY, Ypart + ((size_t)(p + cur_s) * WN + wn) * (size_t)(BM * B), B, wm * TM, 0, g, t);
+          __syncwarp();
+          if (lane == 0) mbar_arrive(&v_empty);
+        }
+        if (!mbar_wait(&v_full, nslab & 1, ctrl)) { ok = false; break; }
+        cur_s = s;
+        ++nslab;
+      }
+      const int st = i % STAGES;
+      if (!mbar_wait(&full[st], (i / STAGES) & 1, ctrl)) { ok = false; break; }
+      const unsigned char* sW = sStage + st * STAGE_BYTES;
+      const unsigned char* sZ = sW + W_BYTES;
+      const unsigned char* sO = sZ + Z_BYTES;
+
+      // ---- P = V * Zt^T for this warp's rows and column groups
+      T acc[MT][QW][U][4];
+#pragma unroll
+      for (int a = 0; a < MT; ++a)
+#pragma unroll
+        for (int q = 0; q < QW; ++q)
+#pragma unroll
+          for (int u = 0; u < U; ++u)
+#pragma unroll
+            for (int e = 0; e < 4; ++e) acc[a][q][u][e] = T(0);
+#pragma unroll
+      for (int kb = 0; kb < KB; ++kb) {
+#pragma unroll
+        for (int s2 = 0; s2 < 2; ++s2) {
+          T ra[MT][2][NV];
+#pragma unroll
+          for (int a = 0; a < MT; ++a) {
+            const int rlo = wm * TM + a * 16 + g;
+            const uint32_t chunk = ((uint32_t)(2 * t + s2) ^ (uint32_t)g) << 4;
+            VecLoad16<T>::ld(sVs + kb * V_BOX + rlo * 128 + chunk, ra[a][0]);
+            VecLoad16<T>::ld(sVs + kb * V_BOX + (rlo + 8) * 128 + chunk, ra[a][1]);
+          }
+#pragma unroll
+          for (int q = 0; q < QW; ++q)
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+              // n-slot g of tile u is column (KE/4)*(g/2) + 2u + (g&1) of the group
+              const int zr = (wn * QW + q) * KE + (KE / 4) * (g >> 1) + 2 * u + (g & 1);
+              T rb[NV];
+              VecLoad16<T>::ld(sZ + kb * Z_BOX + zr * 128 + (((uint32_t)(2 * t + s2) ^ (uint32_t)(zr & 7)) << 4), rb);
+#pragma unroll
+              for (int ks = 0; ks < KS; ++ks) {
+                const T bf[2] = {rb[2 * ks], rb[2 * ks + 1]};
+#pragma unroll
+                for (int a = 0; a < MT; ++a) {
+                  const T af[4] = {ra[a][0][2 * ks], ra[a][1][2 * ks], ra[a][0][2 * ks + 1], ra[a][1][2 * ks + 1]};
+                  mma16x8x8(acc[a][q][u], af, bf);
+                }
+              }
+            }
+        }
+      }
+
+      // ---- Wnew = W - P: store, norms, and keep as the A operand of the sample product
+      const int col_base = c * BN;
+#pragma unroll
+      for (int a = 0; a < MT; ++a)
+#pragma unroll
+        for (int q = 0; q < QW; ++q) {
+          const int grp = wn * QW + q;
+#pragma unroll
+          for (int h = 0; h < 2; ++h) {
+            const int rl = wm * TM + a * 16 + g + 8 * h;     // row inside the slab
+            const int lr = s * BM + rl;                      // row relative to r0
+            T wv[2][NV];
+#pragma unroll
+            for (int s2 = 0; s2 < 2; ++s2)
+              VecLoad16<T>::ld(sW + grp * W_BOX + rl * 128 + (((uint32_t)(2 * t + s2) ^ (uint32_t)g) << 4), wv[s2]);
+            const bool row_ok = lr < rows;
+            const bool is_top = lr < top_rows;
+            T* dst = is_top ? top + (size_t)lr * ldtop : C + (size_t)(r0 + lr) * ldc;
+            const int col = col_base + grp * KE + (KE / 4) * t;   // first of KE/4 consecutive columns
+            double qsum = 0.0;
+#pragma unroll
+            for (int s2 = 0; s2 < 2; ++s2)
+#pragma unroll
+              for (int ks = 0; ks < KS; ++ks) {
+                const int u = s2 * KS + ks;
+                const T y0 = wv[s2][2 * ks] - acc[a][q][u][2 * h];
+                const T y1 = wv[s2][2 * ks + 1] - acc[a][q][u][2 * h + 1];
+                acc[a][q][u][2 * h] = y0;
+                acc[a][q][u][2 * h + 1] = y1;
+                const int cc = col + 2 * u;
+                if (row_ok) {
+                  if (cc + 1 < ncols) {
+                    store2(dst + cc, y0, y1);
+                    qsum += (double)y0 * (double)y0 + (double)y1 * (double)y1;
+                  } else if (cc < ncols) {
+                    dst[cc] = y0;
+                    qsum += (double)y0 * (double)y0;
+                  }
+                }
+              }
+            if (is_top) s_top += qsum; else s_trail += qsum;
+          }
+        }
+
+      // ---- Y += Wnew * OmegaT^T (K = this warp's columns)
+      if (do_sample) {
+#pragma unroll
+        for (int q = 0; q < QW; ++q) {
+          const int grp = wn * QW + q;
+#pragma unroll
+          for (int s2 = 0; s2 < 2; ++s2) {
+#pragma unroll
+            for (int nb = 0; nb < NTB; ++nb) {
+              const int jr = nb * 8 + g;
+              T rb[NV];
+              VecLoad16<T>::ld(sO + grp * O_BOX + jr * 128 + (((uint32_t)(2 * t + s2) ^ (uint32_t)g) << 4), rb);
+#pragma unroll
+              for (int ks = 0; ks < KS; ++ks) {
+                const int u = s2 * KS + ks;
+                const T bf[2] = {rb[2 * ks], rb[2 * ks + 1]};
+#pragma unroll
+                for (int a = 0; a < MT; ++a) {
+                  const T af[4] = {acc[a][q][u][0], acc[a][q][u][2], acc[a][q][u][1], acc[a][q][u][3]};
+                  mma16x8x8(accY[a][nb], af, bf);
+                }
+              }
+            }
+          }
+        }
+      }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&empty[st]);
+    }
+    if (ok && cur_s >= 0 && do_sample)
+      flush_tile<T, MT, NTB>(accY, Ypart + ((size_t)(p + cur_s) * WN + wn) * (size_t)(BM * B), B, wm * TM, 0, g, t);
+  }
+
+  // per-CTA norm partials (all warps join; the producer contributes zeros)
+  const double bt = block_sum(s_top, red);
+  const double br = block_sum(s_trail, red + 32);
+  if (tid == 0 && norm_part != nullptr) {
+    norm_part[2 * p] = bt;
+    norm_part[2 * p + 1] = br;
+  }
+}
+
+}  // namespace rrf

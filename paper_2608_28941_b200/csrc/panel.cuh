@@ -49,9 +49,37 @@ __device__ __forceinline__ bool grid_barrier(unsigned* ctr, unsigned target, Ctr
 //   g[c] = v_c^T v_j     = v_c[j] + p[c]/(alpha - beta)           (c < j: row j of V^T V, for T)
 // so norms, reflector application and the Gram matrix for T share one reduction.
 // ------------------------------------------------------------------------------------------
+// Where the panel's entries come from: either `nseg` partial panels stacked with a fixed
+// stride (rows x ldy each), or the slot layout written by upd_sk_kernel (gemm_sk.cuh).
+struct PanelSource {
+  int slots;               // 0: stacked segments, 1: stream-K slots
+  int nseg;                // stacked: number of partial panels
+  long long seg_stride;    // stacked: elements between partial panels
+  int ldy;                 // stacked: leading dimension
+  int row_off;             // slots: panel row 0 is row `row_off` of the producer's row numbering
+  int bm, nc, tpc, wn;     // slots: slab height, tiles per slab, tiles per CTA, warp columns
+};
+
+template <typename T>
+__device__ __forceinline__ double panel_entry(const T* __restrict__ Y, const PanelSource& src, int r, int c, int b) {
+  double s = 0.0;
+  if (!src.slots) {
+    const T* p = Y + (size_t)r * src.ldy + c;
+    for (int sg = 0; sg < src.nseg; ++sg) s += (double)p[(size_t)sg * src.seg_stride];
+  } else {
+    const int lr = r + src.row_off;
+    const int sl = lr / src.bm, rl = lr - sl * src.bm;
+    const int p_lo = (sl * src.nc) / src.tpc, p_hi = ((sl + 1) * src.nc - 1) / src.tpc;
+    for (int p = p_lo; p <= p_hi; ++p)
+      for (int w = 0; w < src.wn; ++w)
+        s += (double)Y[((size_t)(p + sl) * src.wn + w) * (size_t)(src.bm * b) + (size_t)rl * b + c];
+  }
+  return s;
+}
+
 template <typename T>
 __global__ void __launch_bounds__(kPanelThreads)
-    panel_kernel(const T* __restrict__ Y, int nseg, long long seg_stride, int ldy,  // sum of nseg partial panels
+    panel_kernel(const T* __restrict__ Y, PanelSource src,
                  int rows, int b, int R, int Rp,
                  T* __restrict__ V, long long ldv,   // rows x b block of the V array
                  double* __restrict__ P,             // [2][gridDim.x][b] per-CTA partial dots
@@ -73,13 +101,10 @@ __global__ void __launch_bounds__(kPanelThreads)
   const int gr0 = cta * R;
   const int nloc = max(0, min(R, rows - gr0));
 
-  // load the slab: sum the partial panels in segment order
+  // load the slab: sum the partial panels in their fixed order
   for (int idx = tid; idx < nloc * b; idx += kPanelThreads) {
     const int r = idx / b, c = idx - r * b;
-    const T* src = Y + (size_t)(gr0 + r) * ldy + c;
-    double s = 0.0;
-    for (int sg = 0; sg < nseg; ++sg) s += (double)src[(size_t)sg * seg_stride];
-    S[(size_t)c * Rp + r] = s;
+    S[(size_t)c * Rp + r] = panel_entry(Y, src, gr0 + r, c, b);
   }
   __syncthreads();
 
@@ -208,9 +233,11 @@ __global__ void __launch_bounds__(128)
 // Each CTA owns kTzCols columns.  Output is the transposed (K-contiguous) operand of update_kernel.
 // ------------------------------------------------------------------------------------------
 constexpr int kTzCols = 32;
+// Zpart is in the slot layout of vtw_sk_kernel: column tile c (bn columns) is the sum of slots
+// p + c for the CTAs p whose tile range [p*tpc, (p+1)*tpc) meets [c*kt, (c+1)*kt).
 template <typename T>
 __global__ void __launch_bounds__(256)
-    tz_kernel(const T* __restrict__ Zpart, int nseg, int npad, int b, const T* __restrict__ Tm, long long ldt,
+    tz_kernel(const T* __restrict__ Zpart, int bn, int nct, int kt, int tpc, int b, const T* __restrict__ Tm, long long ldt,
               int transpose_t, T* __restrict__ Zt, const int* done_flag) {
   if (*reinterpret_cast<const volatile int*>(done_flag)) return;
   extern __shared__ double zsm[];
@@ -223,10 +250,13 @@ __global__ void __launch_bounds__(256)
     const int i = idx / b, j = idx - i * b;
     Ts[i * pitch + j] = (double)Tm[(size_t)i * ldt + j];
   }
+  const int ct = col0 / bn, cin = col0 - ct * bn;   // column tiles past the last one hold no data
+  const int p_lo = (ct * kt) / tpc, p_hi = ((ct + 1) * kt - 1) / tpc;
   for (int idx = tid; idx < b * kTzCols; idx += 256) {
     const int l = idx / kTzCols, cl = idx - l * kTzCols;
     double s = 0.0;
-    for (int sg = 0; sg < nseg; ++sg) s += (double)Zpart[((size_t)sg * b + l) * npad + col0 + cl];
+    if (ct < nct)
+      for (int p = p_lo; p <= p_hi; ++p) s += (double)Zpart[(size_t)(p + ct) * (size_t)(b * bn) + (size_t)l * bn + cin + cl];
     Zs[cl * pitch + l] = s;
   }
   __syncthreads();
