@@ -18,7 +18,7 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
 
 constexpr int kMaxSmem = 232448;   // 227 KB opt-in dynamic shared memory per CTA on sm_100
 constexpr int kTargetCtas = 296;   // split-K until about two CTAs per SM exist
-constexpr int kMaxSms = 160;       // workspace sizes are bounds for devices with up to this many SMs
+constexpr int kMaxSms = kPanelMaxG;       // workspace sizes are bounds for devices with up to this many SMs
 
 }  // namespace rrf
 
@@ -84,9 +84,11 @@ static UpdPlan plan_upd(int sms, long long rows, long long ncols, int bm, int bn
 }
 struct PanelPlan { int G, R, Rp; size_t smem; };
 static bool plan_panel(const rrf_ctx* h, long long rows, int b, PanelPlan* p) {
-  int R = std::max(32, ceil_div(rows, h->sms));
+  // tall slabs keep the grid, and with it the all-to-all read of the partial sums, small
+  int R = std::max(128, ceil_div(rows, h->sms));
   p->R = R;
   p->G = ceil_div(rows, R);
+  if (R > 7 * 32) return false;   // a lane keeps at most seven rows of a column in registers
   // odd pitch keeps the transposing load/store phases bank-conflict free; the tallest panels
   // (config 5: 222 rows x 128 columns per CTA) only fit without the padding
   for (int Rp : {R | 1, R}) {
@@ -97,14 +99,15 @@ static bool plan_panel(const rrf_ctx* h, long long rows, int b, PanelPlan* p) {
   return false;
 }
 static size_t panel_scratch_bytes(int sms, int b) {
-  // P[2][sms][b] + piv[2][b] + gram[b][b] + tau[b] (+ barrier word, padded)
-  return align_up(((size_t)2 * sms * b + 2 * (size_t)b + (size_t)b * b + b) * sizeof(double) + 256, 256);
+  // P[2][b][Gp] + piv[2][b] + gram[b][b] + tau[b] (+ barrier word, padded)
+  const int gp = (sms + 31) / 32 * 32;
+  return align_up(((size_t)2 * gp * b + 2 * (size_t)b + (size_t)b * b + b) * sizeof(double) + 256, 256);
 }
 struct PanelScratch { double *P, *piv, *gram, *tau; unsigned* bar; };
 static PanelScratch carve_panel(unsigned char* base, int sms, int b) {
   PanelScratch s;
   s.P = reinterpret_cast<double*>(base);
-  s.piv = s.P + (size_t)2 * sms * b;
+  s.piv = s.P + (size_t)2 * ((sms + 31) / 32 * 32) * b;
   s.gram = s.piv + 2 * (size_t)b;
   s.tau = s.gram + (size_t)b * b;
   s.bar = reinterpret_cast<unsigned*>(s.tau + b);
@@ -245,18 +248,21 @@ static rrf_status_t launch_panel(rrf_ctx* h, int dtype, const void* Y, PanelSour
   cudaError_t e;
   const size_t tsmem = ((size_t)b * (b + 1) + b) * sizeof(double);
   mark(RRF_PHASE_PANEL, step);
+  const bool small = pp.R <= 128;
   if (dtype == RRF_F64) {
-    e = cudaLaunchCooperativeKernel((void*)panel_kernel<double>, dim3(pp.G), dim3(kPanelThreads), args, pp.smem, st);
+    e = cudaLaunchCooperativeKernel(small ? (void*)panel_kernel<double, 4> : (void*)panel_kernel<double, 7>, dim3(pp.G),
+                                    dim3(kPanelThreads), args, pp.smem, st);
     if (e == cudaSuccess) {
       mark(RRF_PHASE_TFACTOR, step);
-      tfactor_kernel<double><<<1, 128, tsmem, st>>>(gram, tau, b, (double*)Tout, ldt, done_flag);
+      tfactor_kernel<double><<<1, 256, tsmem, st>>>(gram, tau, b, (double*)Tout, ldt, done_flag);
       e = cudaGetLastError();
     }
   } else {
-    e = cudaLaunchCooperativeKernel((void*)panel_kernel<float>, dim3(pp.G), dim3(kPanelThreads), args, pp.smem, st);
+    e = cudaLaunchCooperativeKernel(small ? (void*)panel_kernel<float, 4> : (void*)panel_kernel<float, 7>, dim3(pp.G),
+                                    dim3(kPanelThreads), args, pp.smem, st);
     if (e == cudaSuccess) {
       mark(RRF_PHASE_TFACTOR, step);
-      tfactor_kernel<float><<<1, 128, tsmem, st>>>(gram, tau, b, (float*)Tout, ldt, done_flag);
+      tfactor_kernel<float><<<1, 256, tsmem, st>>>(gram, tau, b, (float*)Tout, ldt, done_flag);
       e = cudaGetLastError();
     }
   }
@@ -288,16 +294,20 @@ static cudaError_t setup_all(int smem_optin, int* panel_smem_max) {
     e = get_ops(RRF_F32, b)->setup();
     if (e != cudaSuccess) return e;
   }
-  cudaFuncAttributes fa, fb;
-  e = cudaFuncGetAttributes(&fa, panel_kernel<double>);
-  if (e != cudaSuccess) return e;
-  e = cudaFuncGetAttributes(&fb, panel_kernel<float>);
-  if (e != cudaSuccess) return e;
-  *panel_smem_max = std::min(smem_optin, kMaxSmem) - (int)std::max(fa.sharedSizeBytes, fb.sharedSizeBytes);
-  e = cudaFuncSetAttribute(panel_kernel<double>, cudaFuncAttributeMaxDynamicSharedMemorySize, *panel_smem_max);
-  if (e != cudaSuccess) return e;
-  e = cudaFuncSetAttribute(panel_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, *panel_smem_max);
-  if (e != cudaSuccess) return e;
+  const void* pk[4] = {(const void*)panel_kernel<double, 4>, (const void*)panel_kernel<double, 7>,
+                       (const void*)panel_kernel<float, 4>, (const void*)panel_kernel<float, 7>};
+  size_t stat = 0;
+  for (const void* f : pk) {
+    cudaFuncAttributes fa;
+    e = cudaFuncGetAttributes(&fa, f);
+    if (e != cudaSuccess) return e;
+    stat = std::max(stat, fa.sharedSizeBytes);
+  }
+  *panel_smem_max = std::min(smem_optin, kMaxSmem) - (int)stat;
+  for (const void* f : pk) {
+    e = cudaFuncSetAttribute(f, cudaFuncAttributeMaxDynamicSharedMemorySize, *panel_smem_max);
+    if (e != cudaSuccess) return e;
+  }
   const int tmax = (128 * 129 + 128) * 8;
   e = cudaFuncSetAttribute(tfactor_kernel<double>, cudaFuncAttributeMaxDynamicSharedMemorySize, tmax);
   if (e != cudaSuccess) return e;

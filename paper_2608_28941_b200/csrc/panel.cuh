@@ -6,10 +6,10 @@
 
 namespace rrf {
 
-constexpr int kPanelThreads = 256;
-// doubles of shared memory the panel kernel needs besides the slab: w[b] and a region that holds
-// p[b], pivot_row[b] and, at another time, one partial per thread
-__host__ __device__ constexpr int panel_extra_doubles(int b) { return b + (2 * b > kPanelThreads ? 2 * b : kPanelThreads); }
+constexpr int kPanelThreads = 512;
+constexpr int kPanelMaxG = 160;   // most CTAs a panel grid may have (one per SM)
+// doubles of shared memory the panel kernel needs besides the slab: w[b], p[b], pivot_row[b]
+__host__ __device__ constexpr int panel_extra_doubles(int b) { return 3 * b; }
 
 // Grid-wide barrier over a monotonically increasing arrival counter.  Needs all CTAs
 // co-resident (cooperative launch).  Bounded: gives up after kWaitLimitClocks.
@@ -77,12 +77,13 @@ __device__ __forceinline__ double panel_entry(const T* __restrict__ Y, const Pan
   return s;
 }
 
-template <typename T>
+// QMAX = ceil(R / 32): rows of the slab each lane looks after (template, so they live in registers).
+template <typename T, int QMAX>
 __global__ void __launch_bounds__(kPanelThreads)
     panel_kernel(const T* __restrict__ Y, PanelSource src,
                  int rows, int b, int R, int Rp,
                  T* __restrict__ V, long long ldv,   // rows x b block of the V array
-                 double* __restrict__ P,             // [2][gridDim.x][b] per-CTA partial dots
+                 double* __restrict__ P,             // [2][b][Gp] per-CTA partial dots, Gp = gridDim.x rounded up to 32
                  double* __restrict__ piv,           // [2][b] broadcast pivot row
                  double* __restrict__ gram,          // [b][b] strictly-lower part: v_c^T v_j (c < j)
                  double* __restrict__ tau_out,       // [b]
@@ -93,11 +94,12 @@ __global__ void __launch_bounds__(kPanelThreads)
   double* w_s = S + (size_t)b * Rp;       // [b]
   double* p_s = w_s + b;                  // [b]
   double* pr_s = p_s + b;                 // [b]
-  double* part_s = p_s;                   // [kPanelThreads], aliases p_s/pr_s (see panel_extra_doubles)
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   constexpr int NW = kPanelThreads / 32;
+  constexpr int CG = 4;                   // columns a warp handles at a time (independent chains)
   const int G = gridDim.x, cta = blockIdx.x;
+  const int Gp = (G + 31) & ~31;
   const int gr0 = cta * R;
   const int nloc = max(0, min(R, rows - gr0));
 
@@ -119,49 +121,101 @@ __global__ void __launch_bounds__(kPanelThreads)
         if (gr0 + r >= j) Sj[r] -= f * Sjm1[r];
     }
     __syncthreads();
-    // one pass: update trailing columns and take all dot products with column j
-    for (int c = warp; c < b; c += NW) {
-      double* Sc = S + (size_t)c * Rp;
-      const bool upd = (j > 0) && (c > j) && (tau_prev != 0.0);
-      const double f = upd ? tau_prev * w_s[c] : 0.0;
-      double acc = 0.0;
-      for (int r = lane; r < nloc; r += 32) {
+    // one pass: update trailing columns and take all dot products with column j.  Each lane keeps
+    // its rows of column j and of v_{j-1} in registers; CG columns are in flight per warp.
+    {
+      double yj[QMAX], vp[QMAX];
+#pragma unroll
+      for (int q = 0; q < QMAX; ++q) {
+        const int r = lane + 32 * q;
+        const bool in = r < nloc;
         const int grow = gr0 + r;
-        double x = Sc[r];
-        if (upd && grow >= j) {
-          x -= f * Sjm1[r];
-          Sc[r] = x;
-        }
-        if (grow > j) acc += Sj[r] * x;
+        yj[q] = (in && grow > j) ? Sj[r] : 0.0;            // rows at or above the pivot do not count
+        vp[q] = (in && grow >= j) ? Sjm1[r] : 0.0;         // rows above j are finished
       }
-      acc = warp_sum(acc);
-      if (lane == 0) p_s[c] = acc;
+      const bool pending = (j > 0) && (tau_prev != 0.0);
+      for (int c0 = warp; c0 < b; c0 += NW * CG) {
+        double x[CG][QMAX], acc[CG];
+#pragma unroll
+        for (int u = 0; u < CG; ++u) {
+          const int c = c0 + u * NW;
+          const double* Sc = S + (size_t)(c < b ? c : 0) * Rp;
+#pragma unroll
+          for (int q = 0; q < QMAX; ++q) {
+            const int r = lane + 32 * q;
+            x[u][q] = (c < b && r < nloc) ? Sc[r] : 0.0;
+          }
+        }
+#pragma unroll
+        for (int u = 0; u < CG; ++u) {
+          const int c = c0 + u * NW;
+          const bool upd = pending && c > j && c < b;
+          const double f = upd ? tau_prev * w_s[c] : 0.0;
+          double* Sc = S + (size_t)(c < b ? c : 0) * Rp;
+          double a = 0.0;
+#pragma unroll
+          for (int q = 0; q < QMAX; ++q) {
+            const int r = lane + 32 * q;
+            double xv = x[u][q];
+            if (upd) {
+              xv -= f * vp[q];
+              if (r < nloc && gr0 + r >= j) Sc[r] = xv;
+            }
+            a += yj[q] * xv;
+          }
+          acc[u] = a;
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1)
+#pragma unroll
+          for (int u = 0; u < CG; ++u) acc[u] += __shfl_xor_sync(0xffffffffu, acc[u], o);
+        if (lane == 0) {
+#pragma unroll
+          for (int u = 0; u < CG; ++u)
+            if (c0 + u * NW < b) p_s[c0 + u * NW] = acc[u];
+        }
+      }
     }
     __syncthreads();
-    double* Pj = P + (size_t)(j & 1) * G * b;
-    for (int c = tid; c < b; c += kPanelThreads) Pj[(size_t)cta * b + c] = p_s[c];
+    double* Pj = P + (size_t)(j & 1) * b * Gp;
+    for (int c = tid; c < b; c += kPanelThreads) Pj[(size_t)c * Gp + cta] = p_s[c];
     if (j >= gr0 && j < gr0 + nloc)
       for (int c = tid; c < b; c += kPanelThreads) piv[(j & 1) * b + c] = S[(size_t)c * Rp + (j - gr0)];
     if (!grid_barrier(bar, (unsigned)(j + 1) * (unsigned)G, ctrl)) return;
 
-    // every CTA: fixed-order sum of the partials (kPanelThreads/b threads per column)
+    // every CTA: sum of the per-CTA partials in a fixed order (lane x takes CTAs x, x+32, ...;
+    // then the fixed shuffle tree), one warp per column, CG columns of loads in flight at once
     {
-      const int per = kPanelThreads / b;          // b in {16,...,128} divides 256
-      const int c = tid % b, q = tid / b;
-      double s = 0.0;
-      for (int x = q; x < G; x += per) s += __ldcg(Pj + (size_t)x * b + c);
-      part_s[tid] = s;
-      __syncthreads();
-      double tot = 0.0, prv = 0.0;
-      if (tid < b) {
-        for (int qq = 0; qq < per; ++qq) tot += part_s[qq * b + tid];
-        prv = __ldcg(piv + (j & 1) * b + tid);
+      const double prv = tid < b ? __ldcg(piv + (j & 1) * b + tid) : 0.0;
+      for (int c0 = warp; c0 < b; c0 += NW * CG) {
+        double v[CG][kPanelMaxG / 32];
+#pragma unroll
+        for (int u = 0; u < CG; ++u) {
+          const int c = c0 + u * NW;
+#pragma unroll
+          for (int q = 0; q < kPanelMaxG / 32; ++q) {
+            const int xx = lane + 32 * q;
+            v[u][q] = (c < b && xx < G) ? __ldcg(Pj + (size_t)c * Gp + xx) : 0.0;
+          }
+        }
+        double sacc[CG];
+#pragma unroll
+        for (int u = 0; u < CG; ++u) {
+          sacc[u] = 0.0;
+#pragma unroll
+          for (int q = 0; q < kPanelMaxG / 32; ++q) sacc[u] += v[u][q];
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1)
+#pragma unroll
+          for (int u = 0; u < CG; ++u) sacc[u] += __shfl_xor_sync(0xffffffffu, sacc[u], o);
+        if (lane == 0) {
+#pragma unroll
+          for (int u = 0; u < CG; ++u)
+            if (c0 + u * NW < b) p_s[c0 + u * NW] = sacc[u];
+        }
       }
-      __syncthreads();
-      if (tid < b) {
-        p_s[tid] = tot;
-        pr_s[tid] = prv;
-      }
+      if (tid < b) pr_s[tid] = prv;
       __syncthreads();
     }
     const double alpha = pr_s[j], s2 = p_s[j];
@@ -198,33 +252,39 @@ __global__ void __launch_bounds__(kPanelThreads)
 // One CTA; T is built in shared memory in double and written as T (b x b, leading dim ldt).
 // ------------------------------------------------------------------------------------------
 template <typename T>
-__global__ void __launch_bounds__(128)
+__global__ void __launch_bounds__(256)
     tfactor_kernel(const double* __restrict__ gram, const double* __restrict__ tau, int b,
                    T* __restrict__ Tout, long long ldt, const int* done_flag) {
   if (*reinterpret_cast<const volatile int*>(done_flag)) return;
   extern __shared__ double tsm[];
   const int pitch = b + 1;
-  double* Ts = tsm;                        // [b][pitch]
-  double* gj = Ts + (size_t)b * pitch;     // [b]: gj[l] = v_l^T v_j, l < j
+  double* Ts = tsm;                        // [b][pitch]: T in the upper triangle, the Gram rows below it
+  double* ts = Ts + (size_t)b * pitch;     // [b]: tau
   const int tid = threadIdx.x;
-  for (int idx = tid; idx < b * pitch; idx += blockDim.x) Ts[idx] = 0.0;
+  const int per = 256 / b;                 // threads per row of T: 2, 4, 8 or 16 adjacent lanes
+  const int i = tid / per, part = tid - i * per;
+  for (int idx = tid; idx < b * b; idx += 256) {
+    const int r = idx / b, c = idx - r * b;
+    Ts[r * pitch + c] = c < r ? gram[idx] : 0.0;      // Ts[j][l] = v_l^T v_j for l < j
+  }
+  if (tid < b) ts[tid] = tau[tid];
   __syncthreads();
   for (int j = 0; j < b; ++j) {
-    const double tj = tau[j];
-    if (tid < j) gj[tid] = gram[(size_t)j * b + tid];
-    __syncthreads();
-    if (tid < j) {
-      double s = 0.0;
-      for (int l = tid; l < j; ++l) s += Ts[tid * pitch + l] * gj[l];
-      Ts[tid * pitch + j] = -tj * s;
-    } else if (tid == j) {
-      Ts[j * pitch + j] = tj;
+    const double tj = ts[j];
+    // row i of  -tau_j * T[0:j, 0:j] * g_j : the `per` lanes of a row take every per-th term
+    double s = 0.0;
+    if (i < j)
+      for (int l = i + part; l < j; l += per) s += Ts[i * pitch + l] * Ts[j * pitch + l];
+    for (int o = per >> 1; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+    if (part == 0) {
+      if (i < j) Ts[i * pitch + j] = -tj * s;
+      else if (i == j) Ts[j * pitch + j] = tj;
     }
     __syncthreads();
   }
-  for (int idx = tid; idx < b * b; idx += blockDim.x) {
-    const int i = idx / b, j = idx - i * b;
-    Tout[(size_t)i * ldt + j] = (T)Ts[i * pitch + j];
+  for (int idx = tid; idx < b * b; idx += 256) {
+    const int r = idx / b, c = idx - r * b;
+    Tout[(size_t)r * ldt + c] = c >= r ? (T)Ts[r * pitch + c] : T(0);
   }
 }
 
