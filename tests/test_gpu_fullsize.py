@@ -1,0 +1,118 @@
+"""GPU parity at the full benchmark sizes, in the launch configuration bench.py times.
+
+Configs 2, 3 and 4 are small enough for the CPU oracle to run on the same inputs in seconds,
+so k, status, the stopping trace and B are compared element by element.  Config 5
+(32768 x 16384, rank cap 2048) is checked through properties that hold at any size:
+orthogonality of Q, B = Q^T A on sampled columns, the residual against the tolerance and the
+Eckart-Young tail of the known singular values, and triangularity of Q^T A Omega (Theorem 3.1)."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import rrf_oracle as orc
+from paper_2608_28941_b200 import rrf, workloads as wl
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def h():
+    hd = rrf.rrf_create(0)
+    yield hd
+    rrf.rrf_destroy(hd)
+
+
+def _gen(w):
+    A, sig = wl.make_matrix(w, device="cuda")
+    Om = wl.make_omega(w).astype(w.np_dtype)
+    OmT = torch.from_numpy(np.ascontiguousarray(Om.T)).cuda()
+    return A, sig, Om, OmT
+
+
+def _orth_and_residual(h, w, g, A):
+    k = g.k
+    Q = rrf.rrf_form_q(h, g.V, g.T, w.b, k).double()
+    B = g.B[:k].double()
+    orth = torch.linalg.norm(Q.T @ Q - torch.eye(k, dtype=torch.float64, device="cuda")).item()
+    res = torch.linalg.norm(A.double() - Q @ B).item()
+    return Q, B, orth, res
+
+
+@pytest.mark.parametrize("name", ["cfg2", "cfg3", "cfg4"])
+def test_full_config_against_oracle(h, name):
+    w = wl.CONFIGS[name]
+    A, sig, Om, OmT = _gen(w)
+    g = rrf.rrf_run(h, A, w.b, w.tol, w.max_rank, omegaT=OmT)
+    o = orc.rrf(A.cpu().numpy().astype(np.float64), Om.astype(np.float64), w.b, w.tol, w.max_rank)
+    assert (g.k, g.steps, g.status) == (o.k, o.steps, o.status)
+    k = g.k
+    rel = 1e-10 if w.dtype == "f64" else 1e-4
+    Bg = g.B[:k].cpu().numpy().astype(np.float64)
+    assert np.max(np.abs(Bg - o.B)) <= rel * np.max(np.abs(o.B))
+    u = 1.1e-16 if w.dtype == "f64" else 6e-8
+    d = 2 * max(w.m, w.n) * u * np.sqrt(o.normA2)
+    for a, c in zip(g.E_dir_trace, o.E_dir):
+        assert abs(a - c) <= 2 * np.sqrt(c) * d + d * d + 1e-9 * c
+    Q, B, orth, res = _orth_and_residual(h, w, g, A)
+    assert orth <= (1e-12 if w.dtype == "f64" else 1e-5), orth
+    assert abs(res ** 2 - o.E_dir[-1]) <= 1e-6 * o.E_dir[-1] + 2 * np.sqrt(o.E_dir[-1]) * d + d * d
+    if o.status == orc.RRF_OK:
+        assert res <= w.tol * np.sqrt(o.normA2) * (1 + 1e-6)
+    if sig is not None:
+        assert res >= np.sqrt(np.sum(sig[k:] ** 2)) * (1 - 1e-8) - d
+    # Q*B is well-posed: full bar against the oracle's product
+    Qo = orc.form_q(o.V, o.T, w.b)
+    QB = (Q @ B).cpu().numpy()
+    ref = Qo @ o.B
+    assert np.max(np.abs(QB - ref)) <= 10 * rel * np.max(np.abs(ref))
+    # Q element-wise, block by block: the plain bar, or the oracle's own envelope where the block
+    # is an ill-conditioned function of the input (float64: the oracle re-run on the column-permuted
+    # problem, x10; float32: the same algorithm in plain float32 on the CPU, x3)
+    Qg = Q.cpu().numpy()
+    A64 = A.cpu().numpy().astype(np.float64)
+    if w.dtype == "f64":
+        op = orc.permuted_rerun(A64, Om.astype(np.float64), w.b, w.tol, w.max_rank, seed=1)
+        mult = 10
+    else:
+        op = orc.rrf(A.cpu().numpy(), Om, w.b, w.tol, w.max_rank, dtype=np.float32)
+        mult = 3
+    env = orc.form_q(op.V.astype(np.float64), op.T.astype(np.float64), w.b) if op.k == o.k else None
+    for i in range(k // w.b):
+        blk = slice(i * w.b, (i + 1) * w.b)
+        dq = np.max(np.abs(Qg[:, blk] - Qo[:, blk])) / np.max(np.abs(Qo))
+        bar = rel
+        if env is not None:
+            bar = max(bar, mult * np.max(np.abs(env[:, blk] - Qo[:, blk])) / np.max(np.abs(Qo)))
+        assert dq <= bar, (i, dq, bar)
+
+
+def test_config5_properties(h):
+    w = wl.CONFIGS["cfg5"]
+    A, sig, Om, OmT = _gen(w)
+    g = rrf.rrf_run(h, A, w.b, w.tol, w.max_rank, omegaT=OmT)
+    assert g.k == 2048 and g.steps == 16                      # rank of A: tolerance and cap fire together
+    normA = np.sqrt(g.normA2)
+    assert np.isclose(g.normA2, float(np.sum(sig ** 2)), rtol=1e-10)
+    Q, B, orth, res = _orth_and_residual(h, w, g, A)
+    assert orth <= 1e-12, orth
+    assert np.isclose(res ** 2, g.E_dir, rtol=1e-6, atol=(2 * w.m * 1.1e-16 * normA) ** 2)
+    if g.status == rrf.RRF_OK:
+        assert res <= w.tol * normA
+    # the block before the last one had not met the tolerance, and it sat above the Eckart-Young tail
+    prev = g.E_dir_trace[-2]
+    assert prev > w.tol ** 2 * g.normA2
+    assert np.sqrt(prev) >= np.sqrt(np.sum(sig[1920:] ** 2)) * (1 - 1e-8)
+    for i, e in enumerate(g.E_dir_trace[:-1]):
+        kk = (i + 1) * w.b
+        assert np.sqrt(e) >= np.sqrt(np.sum(sig[kk:] ** 2)) * (1 - 1e-8)
+    # B = Q^T A on sampled columns
+    cols = torch.arange(0, w.n, 257, device="cuda")
+    ref = Q.T @ A[:, cols]
+    assert torch.max(torch.abs(ref - B[:, cols])).item() <= 1e-10 * torch.max(torch.abs(ref)).item()
+    # Theorem 3.1: Q^T (A Omega) is upper triangular (first 512 sample vectors)
+    R = Q[:, :512].T @ (A @ OmT[:512].T)
+    low = torch.tril(R, diagonal=-1)
+    assert torch.max(torch.abs(low)).item() <= 1e-11 * torch.max(torch.abs(R)).item()
+    # E_sub and E_dir agree where the subtraction is still resolved (Frobenius identity of section 3)
+    for s, d in zip(g.E_sub_trace[:8], g.E_dir_trace[:8]):
+        assert abs(s - d) <= 1e-9 * g.normA2
