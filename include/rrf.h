@@ -135,6 +135,36 @@ rrf_status_t rrf_panel_qr(rrf_handle_t h, int32_t dtype, int64_t rows, int32_t b
                           void* d_workspace, size_t workspace_bytes, void* cuda_stream);
 
 /*
+ * rrf_panel_qr_static - the same factorisation as rrf_panel_qr for callers that cannot allocate.
+ * (The paper has no counterpart: it is an addition for embedding.)
+ *
+ * Who needs it: code that runs where device allocation is off limits - inside another
+ * framework's memory plan where every byte is pre-assigned, in a plug-in or a real-time loop
+ * that must not call cudaMalloc (which may synchronise the whole device and can fail late), or
+ * before any allocator exists.  Such a caller has no handle (rrf_create allocates) and no
+ * workspace to hand over.  This entry point needs neither: its scratch - the per-CTA partial
+ * sums, the pivot row, the Gram rows, tau, the barrier counter and the status word of the
+ * panel kernel - lives in one fixed 512 KiB array in the library's device image, which every GPU
+ * that loads the library holds until the process exits.  It calls no cudaMalloc, cudaFree or
+ * any other allocating routine; the caller still passes the input and the outputs.
+ *
+ * Limits: b in {16, 32, 64, 128} (32.. in single precision), b <= rows <= 65536, and the panel
+ * must fit on chip (rows*b*8 bytes spread over the SMs, as for rrf_panel_qr); a larger request
+ * returns RRF_ERR_WORKSPACE and launches nothing.
+ *
+ * The first call on each device looks up the array's device address (with that device current)
+ * and raises the kernels' shared-memory limits; make that first call before starting any stream
+ * capture.  Every call on a device shares the one array and finds the previous call's contents in
+ * it: the entry point clears the words that must start at zero itself, but two calls whose kernels
+ * overlap on the GPU (different streams, or different host threads) race on it - serialise them.
+ * Unlike rrf_panel_qr this call synchronises `cuda_stream` before returning and returns the
+ * device-side status (RRF_OK, or RRF_ERR_TIMEOUT if the bounded grid barrier gave up).
+ */
+rrf_status_t rrf_panel_qr_static(int32_t dtype, int64_t rows, int32_t b,
+                                 const void* dY, int64_t ldy, void* dV, int64_t ldv,
+                                 void* dT, int64_t ldt, void* cuda_stream);
+
+/*
  * rrf_apply_qt / rrf_apply_q - C <- Q^T C or C <- Q C for a device matrix C (m x ncols,
  * ldc >= ncols) with Q = Q_0 ... Q_{k/b-1} given by V (m x k) and T (b x k, leading dimension
  * ldt) as rrf_run returns them (Algorithm 2 line 8 applied block by block; "Applying Q resolves

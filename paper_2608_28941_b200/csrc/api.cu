@@ -800,3 +800,99 @@ rrf_status_t rrf_run(rrf_handle_t h, const rrf_params_t* p, void* dA, int64_t ld
 }
 
 }  // extern "C"
+
+// ------------------------------------------------------------------------------------------
+// rrf_panel_qr_static: panel QR for callers that cannot allocate (see include/rrf.h).
+// The scratch is a fixed array in the device image.  In host code its name is only a stand-in
+// for the symbol, not a device address: the address is looked up once per device with
+// cudaGetSymbolAddress and that pointer is what the kernels receive.
+// ------------------------------------------------------------------------------------------
+namespace rrf {
+
+constexpr long long kStaticMaxRows = 65536;
+constexpr size_t kStaticCtrlBytes = 256;                    // Ctrl (status, stop flag, barrier counter)
+constexpr size_t kStaticScratchBytes = 512 * 1024;
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
+
+struct StaticDevice {
+  bool ready;
+  unsigned char* ptr;      // device address of g_static_scratch on this device
+  int sms;
+  int panel_smem_max;
+};
+constexpr int kStaticMaxDevices = 64;
+static StaticDevice g_static_dev[kStaticMaxDevices];
+
+// Once per device, with that device current: symbol address, device limits, kernel attributes.
+static cudaError_t static_setup(int dev, StaticDevice* sd) {
+  void* ptr = nullptr;
+  cudaError_t e = cudaGetSymbolAddress(&ptr, g_static_scratch);
+  if (e != cudaSuccess) return e;
+  int smem_optin = 0;
+  e = cudaDeviceGetAttribute(&sd->sms, cudaDevAttrMultiProcessorCount, dev);
+  if (e != cudaSuccess) return e;
+  e = cudaDeviceGetAttribute(&smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
+  if (e != cudaSuccess) return e;
+  const void* pk[4] = {(const void*)panel_kernel<double, 4>, (const void*)panel_kernel<double, 7>,
+                       (const void*)panel_kernel<float, 4>, (const void*)panel_kernel<float, 7>};
+  size_t stat = 0;
+  for (const void* f : pk) {
+    cudaFuncAttributes fa;
+    e = cudaFuncGetAttributes(&fa, f);
+    if (e != cudaSuccess) return e;
+    stat = std::max(stat, fa.sharedSizeBytes);
+  }
+  sd->panel_smem_max = std::min(smem_optin, kMaxSmem) - (int)stat;
+  for (const void* f : pk) {
+    e = cudaFuncSetAttribute(f, cudaFuncAttributeMaxDynamicSharedMemorySize, sd->panel_smem_max);
+    if (e != cudaSuccess) return e;
+  }
+  const int tmax = (128 * 129 + 128) * 8;
+  e = cudaFuncSetAttribute(tfactor_kernel<double>, cudaFuncAttributeMaxDynamicSharedMemorySize, tmax);
+  if (e != cudaSuccess) return e;
+  e = cudaFuncSetAttribute(tfactor_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, tmax);
+  if (e != cudaSuccess) return e;
+  sd->ptr = static_cast<unsigned char*>(ptr);
+  sd->ready = true;
+  return cudaSuccess;
+}
+
+}  // namespace rrf
+
+extern "C" rrf_status_t rrf_panel_qr_static(int32_t dtype, int64_t rows, int32_t b, const void* dY, int64_t ldy,
+                                            void* dV, int64_t ldv, void* dT, int64_t ldt, void* cuda_stream) {
+  if (dY == nullptr || dV == nullptr || dT == nullptr) return RRF_ERR_INVALID_ARG;
+  if (!b_ok(dtype, b) || rows < b || ldy < b || ldv < b || ldt < b || ldy > 0x7fffffffLL) return RRF_ERR_INVALID_ARG;
+  if (rows > kStaticMaxRows) return RRF_ERR_WORKSPACE;      // beyond the built-in scratch's stated limit
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kStaticMaxDevices) return RRF_ERR_CUDA;
+  StaticDevice* sd = &g_static_dev[dev];
+  if (!sd->ready && static_setup(dev, sd) != cudaSuccess) return RRF_ERR_CUDA;
+  if (sd->sms > kMaxSms || kStaticCtrlBytes + panel_scratch_bytes(sd->sms, b) > kStaticScratchBytes)
+    return RRF_ERR_WORKSPACE;
+  rrf_ctx tmp{};                                            // host-side plan parameters only
+  tmp.device = dev;
+  tmp.sms = sd->sms;
+  tmp.panel_smem_max = sd->panel_smem_max;
+  PanelPlan pp;
+  if (!plan_panel(&tmp, rows, b, &pp)) return RRF_ERR_WORKSPACE;   // panel too tall for on-chip storage
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  Ctrl* ctrl = reinterpret_cast<Ctrl*>(sd->ptr);
+  PanelScratch ps = carve_panel(sd->ptr + kStaticCtrlBytes, sd->sms, b);
+  ps.bar = &ctrl->bar;
+  // the array keeps the last call's contents: the stop flag, the status and the barrier counter
+  // must start at zero; everything else is written by the kernels before it is read
+  if (cudaMemsetAsync(ctrl, 0, kStaticCtrlBytes, st) != cudaSuccess) return RRF_ERR_CUDA;
+  PanelSource src{};
+  src.slots = 0;
+  src.nseg = 1;
+  src.seg_stride = 0;
+  src.ldy = (int)ldy;
+  const rrf_status_t s = launch_panel(&tmp, dtype, dY, src, rows, b, dV, ldv, dT, ldt, ps, ctrl, &ctrl->done, st);
+  if (s != RRF_OK) return s;
+  int status = 0;
+  if (cudaMemcpyAsync(&status, &ctrl->status, sizeof(int), cudaMemcpyDeviceToHost, st) != cudaSuccess)
+    return RRF_ERR_CUDA;
+  if (cudaStreamSynchronize(st) != cudaSuccess) return RRF_ERR_CUDA;
+  return (rrf_status_t)status;
+}

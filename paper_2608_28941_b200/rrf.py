@@ -40,7 +40,7 @@ class rrf_profile_t(C.Structure):
     _fields_ = [("ms", C.c_double * 9), ("launches", C.c_int32 * 9), ("pad", C.c_int32)]
 
 
-EXPORTS = ["rrf_set_profiling", "rrf_get_profile", "rrf_measure_peak", "rrf_create", "rrf_destroy", "rrf_workspace_bytes", "rrf_run", "rrf_panel_workspace_bytes",
+EXPORTS = ["rrf_panel_qr_static", "rrf_set_profiling", "rrf_get_profile", "rrf_measure_peak", "rrf_create", "rrf_destroy", "rrf_workspace_bytes", "rrf_run", "rrf_panel_workspace_bytes",
            "rrf_panel_qr", "rrf_apply_workspace_bytes", "rrf_apply_qt", "rrf_apply_q", "rrf_form_q",
            "rrf_fill_omega", "rrf_last_status", "rrf_status_string"]
 
@@ -62,6 +62,7 @@ def load():
                             C.POINTER(rrf_result_t), C.POINTER(C.c_double), C.POINTER(C.c_double)]
     lib.rrf_panel_workspace_bytes.argtypes = [i32, i64, i32, C.POINTER(sz)]
     lib.rrf_panel_qr.argtypes = [vp, i32, i64, i32, vp, i64, vp, i64, vp, i64, vp, sz, vp]
+    lib.rrf_panel_qr_static.argtypes = [i32, i64, i32, vp, i64, vp, i64, vp, i64, vp]
     lib.rrf_apply_workspace_bytes.argtypes = [i32, i64, i64, i32, C.POINTER(sz)]
     for f in (lib.rrf_apply_qt, lib.rrf_apply_q):
         f.argtypes = [vp, i32, i64, i32, i32, vp, i64, vp, i64, vp, i64, i64, vp, sz, vp]
@@ -216,6 +217,19 @@ def rrf_panel_qr(h, Y: torch.Tensor):
     if s != RRF_OK:
         raise RrfError(s, "rrf_panel_qr (device)")
     return V, T
+
+
+def rrf_panel_qr_static(Y: torch.Tensor, V: torch.Tensor, T: torch.Tensor) -> int:
+    """Panel QR through the entry point that allocates nothing: no handle, no workspace.
+
+    The caller owns Y (rows x b), V (rows x b) and T (b x b); returns the status the call reports
+    (it synchronises the current stream).  Calls that overlap on the GPU race on the library's
+    built-in scratch array.
+    """
+    rows, b = Y.shape
+    return load().rrf_panel_qr_static(_dtype_code(Y), rows, b, C.c_void_p(Y.data_ptr()), _rowmajor(Y, "Y"),
+                                      C.c_void_p(V.data_ptr()), _rowmajor(V, "V"), C.c_void_p(T.data_ptr()),
+                                      _rowmajor(T, "T"), _stream())
 
 
 def _apply(fn_name: str, h, V: torch.Tensor, T: torch.Tensor, b: int, k: int, Cm: torch.Tensor) -> torch.Tensor:
