@@ -253,7 +253,7 @@ def main():
     ms_step = float(t.item()) / args.steps
     flops = method_flops(w.m, w.n, w.b, res.steps)
     value = world * flops / (ms_step * 1e-3) / 1e12
-    launches_per_run = 2 + 7 * (w.max_rank // w.b)
+    launches_per_run = 3 + 6 * (w.max_rank // w.b)   # init x2, first sample; panel, T, VtW, TZ, update, stop per pass
 
     # ---- end to end through the C ABI with host buffers
     e2e = None
@@ -307,6 +307,10 @@ def main():
             if w.dtype == "f32":
                 peak /= 3.0                       # three TF32 products per fp32 product
             work = args.steps * sum(2.0 * r * w.n * w.b for r in mi)
+            if top == "update":                   # the fused kernel also samples the next block's panel
+                work += args.steps * sum(2.0 * r * w.n * w.b for r in mi[1:])
+            if top == "sample":
+                work = args.steps * 2.0 * w.m * w.n * w.b
             achieved = work / (ms * 1e-3) / 1e12
             recipe = peaks.get("bf16_tflops", 1590.0) * NOMINAL_FP64_OVER_BF16 if w.dtype == "f64" else None
             roofline = {"kernel": top, "bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TFLOP/s",

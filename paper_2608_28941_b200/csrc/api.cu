@@ -31,6 +31,8 @@ struct rrf_ctx {
   int last_cuda;
   int panel_smem_max;    // dynamic shared memory the panel kernel may use (opt-in limit minus its static part)
   int profiling;
+  cudaStream_t aux;                      // side stream: the T factor is built while V^T W runs
+  std::vector<cudaEvent_t> sync_events;  // fork/join events between the caller's stream and `aux`
   std::vector<cudaEvent_t> events;
   rrf_profile_t profile;
 };
@@ -42,7 +44,7 @@ static inline int ceil_div(long long a, long long b) { return (int)((a + b - 1) 
 
 // ------------------------------------------------------------------ tile configuration
 constexpr int kSampleBM = 128, kSampleStages = 4;
-constexpr int kVtwBK = 32;
+constexpr int kVtwBK = 64;
 
 struct SamplePlan { int nslabs, nseg, kt_per_seg; };
 static SamplePlan plan_sample(long long rows, long long n, int esize) {
@@ -85,7 +87,7 @@ static UpdPlan plan_upd(int sms, long long rows, long long ncols, int bm, int bn
 struct PanelPlan { int G, R, Rp; size_t smem; };
 static bool plan_panel(const rrf_ctx* h, long long rows, int b, PanelPlan* p) {
   // tall slabs keep the grid, and with it the all-to-all read of the partial sums, small
-  int R = std::max(128, ceil_div(rows, h->sms));
+  int R = std::max(64, ceil_div(rows, h->sms));
   p->R = R;
   p->G = ceil_div(rows, R);
   if (R > 7 * 32) return false;   // a lane keeps at most seven rows of a column in registers
@@ -238,7 +240,8 @@ template <typename Mark = NoMark>
 static rrf_status_t launch_panel(rrf_ctx* h, int dtype, const void* Y, PanelSource src,
                                  long long rows, int b, void* V, long long ldv, void* Tout, long long ldt,
                                  const PanelScratch& ps, Ctrl* ctrl, const int* done_flag, cudaStream_t st,
-                                 Mark mark = Mark(), int step = 0) {
+                                 Mark mark = Mark(), int step = 0, cudaStream_t st_t = nullptr,
+                                 cudaEvent_t ev_fork = nullptr, cudaEvent_t ev_join = nullptr) {
   PanelPlan pp;
   if (!plan_panel(h, rows, b, &pp)) return RRF_ERR_WORKSPACE;
   int rows_i = (int)rows, R = pp.R, Rp = pp.Rp;
@@ -246,24 +249,40 @@ static rrf_status_t launch_panel(rrf_ctx* h, int dtype, const void* Y, PanelSour
   unsigned* bar = ps.bar;
   void* args[] = {&Y, &src, &rows_i, &b, &R, &Rp, &V, &ldv, &P, &piv, &gram, &tau, &bar, &ctrl, &done_flag};
   cudaError_t e;
-  const size_t tsmem = ((size_t)b * (b + 1) + b) * sizeof(double);
+  const size_t tsmem = ((size_t)b * (b + 1) + (size_t)(b / 2) * (b / 2 + 1)) * sizeof(double);
   mark(RRF_PHASE_PANEL, step);
   const bool small = pp.R <= 128;
   if (dtype == RRF_F64) {
     e = cudaLaunchCooperativeKernel(small ? (void*)panel_kernel<double, 4> : (void*)panel_kernel<double, 7>, dim3(pp.G),
                                     dim3(kPanelThreads), args, pp.smem, st);
     if (e == cudaSuccess) {
-      mark(RRF_PHASE_TFACTOR, step);
-      tfactor_kernel<double><<<1, 256, tsmem, st>>>(gram, tau, b, (double*)Tout, ldt, done_flag);
+      cudaStream_t tt = st;
+      if (ev_fork != nullptr) {          // fork: the T factor runs on the side stream after the panel
+        cudaEventRecord(ev_fork, st);
+        cudaStreamWaitEvent(st_t, ev_fork, 0);
+        tt = st_t;
+      } else {
+        mark(RRF_PHASE_TFACTOR, step);
+      }
+      tfactor_kernel<double><<<1, 256, tsmem, tt>>>(gram, tau, b, (double*)Tout, ldt, done_flag);
       e = cudaGetLastError();
+      if (ev_join != nullptr) cudaEventRecord(ev_join, st_t);
     }
   } else {
     e = cudaLaunchCooperativeKernel(small ? (void*)panel_kernel<float, 4> : (void*)panel_kernel<float, 7>, dim3(pp.G),
                                     dim3(kPanelThreads), args, pp.smem, st);
     if (e == cudaSuccess) {
-      mark(RRF_PHASE_TFACTOR, step);
-      tfactor_kernel<float><<<1, 256, tsmem, st>>>(gram, tau, b, (float*)Tout, ldt, done_flag);
+      cudaStream_t tt = st;
+      if (ev_fork != nullptr) {
+        cudaEventRecord(ev_fork, st);
+        cudaStreamWaitEvent(st_t, ev_fork, 0);
+        tt = st_t;
+      } else {
+        mark(RRF_PHASE_TFACTOR, step);
+      }
+      tfactor_kernel<float><<<1, 256, tsmem, tt>>>(gram, tau, b, (float*)Tout, ldt, done_flag);
       e = cudaGetLastError();
+      if (ev_join != nullptr) cudaEventRecord(ev_join, st_t);
     }
   }
   if (e != cudaSuccess) {
@@ -308,7 +327,7 @@ static cudaError_t setup_all(int smem_optin, int* panel_smem_max) {
     e = cudaFuncSetAttribute(f, cudaFuncAttributeMaxDynamicSharedMemorySize, *panel_smem_max);
     if (e != cudaSuccess) return e;
   }
-  const int tmax = (128 * 129 + 128) * 8;
+  const int tmax = (128 * 129 + 64 * 65) * 8;
   e = cudaFuncSetAttribute(tfactor_kernel<double>, cudaFuncAttributeMaxDynamicSharedMemorySize, tmax);
   if (e != cudaSuccess) return e;
   e = cudaFuncSetAttribute(tfactor_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, tmax);
@@ -405,6 +424,7 @@ rrf_status_t rrf_create(rrf_handle_t* out, int device) {
   h->device = device;
   h->last_cuda = 0;
   h->profiling = 0;
+  h->aux = nullptr;
   std::memset(&h->profile, 0, sizeof(h->profile));
   cudaError_t e = cudaDeviceGetAttribute(&h->sms, cudaDevAttrMultiProcessorCount, device);
   if (e == cudaSuccess) e = cudaDeviceGetAttribute(&h->smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, device);
@@ -415,6 +435,7 @@ rrf_status_t rrf_create(rrf_handle_t* out, int device) {
   if (e == cudaSuccess && h->sms > kMaxSms) e = cudaErrorInvalidConfiguration;
   h->encode = reinterpret_cast<EncodeTiledFn>(fn);
   if (e == cudaSuccess) e = setup_all(h->smem_optin, &h->panel_smem_max);
+  if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&h->aux, cudaStreamNonBlocking);
   if (e == cudaSuccess) e = cudaMalloc(&h->d_ctrl, sizeof(Ctrl));
   if (e == cudaSuccess) e = cudaMemset(h->d_ctrl, 0, sizeof(Ctrl));
   if (e != cudaSuccess) {
@@ -432,6 +453,8 @@ rrf_status_t rrf_destroy(rrf_handle_t h) {
   cudaSetDevice(h->device);
   cudaFree(h->d_ctrl);
   for (cudaEvent_t ev : h->events) cudaEventDestroy(ev);
+  for (cudaEvent_t ev : h->sync_events) cudaEventDestroy(ev);
+  if (h->aux != nullptr) cudaStreamDestroy(h->aux);
   delete h;
   return RRF_OK;
 }
@@ -724,6 +747,13 @@ rrf_status_t rrf_run(rrf_handle_t h, const rrf_params_t* p, void* dA, int64_t ld
   init_ctrl_kernel<<<1, 256, 0, st>>>(init_part, L.init_ctas, p->tol, p->tol_is_relative, fixed ? 1 : 0, b, p->max_rank,
                                       ctrl);
 
+  // fork/join events for the side stream (two per pass), created once and kept in the handle
+  while (h->sync_events.size() < (size_t)2 * steps) {
+    cudaEvent_t ev;
+    if (cudaEventCreateWithFlags(&ev, cudaEventDisableTiming) != cudaSuccess) return fail(RRF_ERR_CUDA);
+    h->sync_events.push_back(ev);
+  }
+
   // Algorithm 2 lines 5-11: every pass is enqueued; passes after the stop return at once.
   // The panel of pass 0 is sampled by its own kernel; the panel of pass i+1 comes out of the
   // fused update of pass i.
@@ -740,7 +770,8 @@ rrf_status_t rrf_run(rrf_handle_t h, const rrf_params_t* p, void* dA, int64_t ld
   for (int i = 0; i < steps; ++i) {
     const int r0 = i * b, rows = (int)(m - r0);
     s = launch_panel(h, p->dtype, Ypart, src, rows, b, (char*)dV + ((size_t)r0 * ldv + r0) * esize, ldv,
-                     (char*)dT + (size_t)r0 * esize, p->max_rank, ps, ctrl, &ctrl->done, st, mark, i);
+                     (char*)dT + (size_t)r0 * esize, p->max_rank, ps, ctrl, &ctrl->done, st, mark, i, h->aux,
+                     h->sync_events[2 * i], h->sync_events[2 * i + 1]);
     if (s != RRF_OK) {
       out->cuda_error = h->last_cuda;
       cudaStreamSynchronize(st);
@@ -750,6 +781,7 @@ rrf_status_t rrf_run(rrf_handle_t h, const rrf_params_t* p, void* dA, int64_t ld
     mark(RRF_PHASE_VTW, i);
     ops->vtw(tmV_k, tmW_k, Zpart, r0, r0, vp, ctrl, st);
     mark(RRF_PHASE_TZ, i);
+    cudaStreamWaitEvent(st, h->sync_events[2 * i + 1], 0);   // join: T_i is needed from here on
     launch_tz(p->dtype, Zpart, vp, b, (const char*)dT + (size_t)r0 * esize, p->max_rank, 1, Zt, &ctrl->done, st);
     const UpdPlan up = plan_upd(h->sms, rows, n, ops->u_bm, ops->u_bn, ops->u_wn);
     const int j0 = (i + 1 < steps) ? r0 + b : -1;   // Omega rows of the next pass, if there is one
@@ -847,7 +879,7 @@ static cudaError_t static_setup(int dev, StaticDevice* sd) {
     e = cudaFuncSetAttribute(f, cudaFuncAttributeMaxDynamicSharedMemorySize, sd->panel_smem_max);
     if (e != cudaSuccess) return e;
   }
-  const int tmax = (128 * 129 + 128) * 8;
+  const int tmax = (128 * 129 + 64 * 65) * 8;
   e = cudaFuncSetAttribute(tfactor_kernel<double>, cudaFuncAttributeMaxDynamicSharedMemorySize, tmax);
   if (e != cudaSuccess) return e;
   e = cudaFuncSetAttribute(tfactor_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, tmax);

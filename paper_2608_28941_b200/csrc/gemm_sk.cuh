@@ -107,14 +107,14 @@ __global__ void __launch_bounds__((WM * WN + 1) * 32)
       for (int e = 0; e < 4; ++e) acc[a][c][e] = T(0);
 
   int cur_c = L0 / KT;
+  int c = cur_c, kt = L0 - cur_c * KT, st = 0;
+  uint32_t ph = 0;
   for (int i = 0; i < ntile; ++i) {
-    const int c = (L0 + i) / KT;
     if (c != cur_c) {
       flush_tile<T, MT, NT>(acc, Zpart + (size_t)(p + cur_c) * (size_t)(B * BN), BN, wm * TM, wn * TN, g, t);
       cur_c = c;
     }
-    const int st = i % STAGES;
-    if (!mbar_wait(&full[st], (i / STAGES) & 1, ctrl)) return;
+    if (!mbar_wait(&full[st], ph, ctrl)) return;
     const unsigned char* sV = smem + st * STAGE_BYTES;
     const unsigned char* sC = sV + V_BYTES;
 #pragma unroll
@@ -147,6 +147,8 @@ __global__ void __launch_bounds__((WM * WN + 1) * 32)
     }
     __syncwarp();
     if (lane == 0) mbar_arrive(&empty[st]);
+    if (++st == STAGES) { st = 0; ph ^= 1u; }
+    if (++kt == KT) { kt = 0; ++c; }
   }
   if (ntile > 0)
     flush_tile<T, MT, NT>(acc, Zpart + (size_t)(p + cur_c) * (size_t)(B * BN), BN, wm * TM, wn * TN, g, t);
@@ -220,8 +222,8 @@ __global__ void __launch_bounds__((WM * WN + 1) * 32, 1)
     // ------------------------------------------------------------ producer warp
     if (lane == 0) {
       int cur_s = -1, nslab = 0;
-      for (int i = 0; i < ntile; ++i) {
-        const int L = L0 + i, s = L / NC, c = L - s * NC;
+      int s = L0 / NC, c = L0 - s * NC;
+      for (int i = 0; i < ntile; ++i, c = (c + 1 == NC ? 0 : c + 1), s += (c == 0)) {
         if (s != cur_s) {
           if (nslab > 0 && !mbar_wait(&v_empty, (nslab - 1) & 1, ctrl)) break;
           mbar_expect_tx(&v_full, V_BYTES);
@@ -258,8 +260,12 @@ __global__ void __launch_bounds__((WM * WN + 1) * 32, 1)
 
     int cur_s = -1, nslab = 0;
     bool ok = true;
+    int s = L0 / NC, c = L0 - s * NC, st = 0;
+    uint32_t ph = 0;
+    // per slab: where this thread's rows go, and to which norm they count (hoisted out of the tile loop)
+    T* rowp[MT][2];
+    bool rtop[MT][2];
     for (int i = 0; i < ntile && ok; ++i) {
-      const int L = L0 + i, s = L / NC, c = L - s * NC;
       if (s != cur_s) {
         if (cur_s >= 0) {
           if (do_sample)
@@ -270,9 +276,16 @@ __global__ void __launch_bounds__((WM * WN + 1) * 32, 1)
         if (!mbar_wait(&v_full, nslab & 1, ctrl)) { ok = false; break; }
         cur_s = s;
         ++nslab;
+#pragma unroll
+        for (int a = 0; a < MT; ++a)
+#pragma unroll
+          for (int h = 0; h < 2; ++h) {
+            const int lr = s * BM + wm * TM + a * 16 + g + 8 * h;     // row relative to r0
+            rtop[a][h] = lr < top_rows;
+            rowp[a][h] = lr >= rows ? nullptr : (rtop[a][h] ? top + (size_t)lr * ldtop : C + (size_t)(r0 + lr) * ldc);
+          }
       }
-      const int st = i % STAGES;
-      if (!mbar_wait(&full[st], (i / STAGES) & 1, ctrl)) { ok = false; break; }
+      if (!mbar_wait(&full[st], ph, ctrl)) { ok = false; break; }
       const unsigned char* sW = sStage + st * STAGE_BYTES;
       const unsigned char* sZ = sW + W_BYTES;
       const unsigned char* sO = sZ + Z_BYTES;
@@ -322,24 +335,22 @@ __global__ void __launch_bounds__((WM * WN + 1) * 32, 1)
 
       // ---- Wnew = W - P: store, norms, and keep as the A operand of the sample product
       const int col_base = c * BN;
+      const bool interior = col_base + BN <= ncols;      // no column guards needed
 #pragma unroll
       for (int a = 0; a < MT; ++a)
 #pragma unroll
         for (int q = 0; q < QW; ++q) {
           const int grp = wn * QW + q;
+          const int col = col_base + grp * KE + (KE / 4) * t;   // first of this thread's KE/4 consecutive columns
 #pragma unroll
           for (int h = 0; h < 2; ++h) {
             const int rl = wm * TM + a * 16 + g + 8 * h;     // row inside the slab
-            const int lr = s * BM + rl;                      // row relative to r0
             T wv[2][NV];
 #pragma unroll
             for (int s2 = 0; s2 < 2; ++s2)
               VecLoad16<T>::ld(sW + grp * W_BOX + rl * 128 + (((uint32_t)(2 * t + s2) ^ (uint32_t)g) << 4), wv[s2]);
-            const bool row_ok = lr < rows;
-            const bool is_top = lr < top_rows;
-            T* dst = is_top ? top + (size_t)lr * ldtop : C + (size_t)(r0 + lr) * ldc;
-            const int col = col_base + grp * KE + (KE / 4) * t;   // first of KE/4 consecutive columns
-            double qsum = 0.0;
+            T* dst = rowp[a][h];
+            double q0 = 0.0, q1 = 0.0;
 #pragma unroll
             for (int s2 = 0; s2 < 2; ++s2)
 #pragma unroll
@@ -350,17 +361,20 @@ __global__ void __launch_bounds__((WM * WN + 1) * 32, 1)
                 acc[a][q][u][2 * h] = y0;
                 acc[a][q][u][2 * h + 1] = y1;
                 const int cc = col + 2 * u;
-                if (row_ok) {
-                  if (cc + 1 < ncols) {
+                if (dst != nullptr) {
+                  if (interior || cc + 1 < ncols) {
                     store2(dst + cc, y0, y1);
-                    qsum += (double)y0 * (double)y0 + (double)y1 * (double)y1;
+                    q0 += (double)y0 * (double)y0;
+                    q1 += (double)y1 * (double)y1;
                   } else if (cc < ncols) {
                     dst[cc] = y0;
-                    qsum += (double)y0 * (double)y0;
+                    q0 += (double)y0 * (double)y0;
                   }
                 }
               }
-            if (is_top) s_top += qsum; else s_trail += qsum;
+            const double qs = q0 + q1;
+            s_top += rtop[a][h] ? qs : 0.0;
+            s_trail += rtop[a][h] ? 0.0 : qs;
           }
         }
 
@@ -392,6 +406,8 @@ __global__ void __launch_bounds__((WM * WN + 1) * 32, 1)
       }
       __syncwarp();
       if (lane == 0) mbar_arrive(&empty[st]);
+      if (++st == STAGES) { st = 0; ph ^= 1u; }
+      if (++c == NC) { c = 0; ++s; }
     }
     if (ok && cur_s >= 0 && do_sample)
       flush_tile<T, MT, NTB>(accY, Ypart + ((size_t)(p + cur_s) * WN + wn) * (size_t)(BM * B), B, wm * TM, 0, g, t);

@@ -247,9 +247,13 @@ __global__ void __launch_bounds__(kPanelThreads)
 }
 
 // ------------------------------------------------------------------------------------------
-// Compact-WY factor from the Gram rows:  T[j][j] = tau_j,
-// T[0:j, j] = -tau_j * T[0:j, 0:j] * (V[:, 0:j]^T v_j)   (Eq. "Q_i = I_m - V_i T_i V_i^T").
-// One CTA; T is built in shared memory in double and written as T (b x b, leading dim ldt).
+// Compact-WY factor from the Gram rows (Eq. "Q_i = I_m - V_i T_i V_i^T").  The column recurrence
+// T[0:j, j] = -tau_j T[0:j, 0:j] (V[:, 0:j]^T v_j) is applied a block at a time: if T11 and T22 are
+// the factors of two adjacent groups of s reflectors, the factor of the 2s reflectors is
+//   [ T11   -T11 (V1^T V2) T22 ]
+//   [  0            T22        ]
+// so log2(b) rounds of independent s x s products build T from its diagonal tau.  One CTA; T and the
+// Gram rows share one shared-memory array (upper / strictly lower triangle).
 // ------------------------------------------------------------------------------------------
 template <typename T>
 __global__ void __launch_bounds__(256)
@@ -257,28 +261,31 @@ __global__ void __launch_bounds__(256)
                    T* __restrict__ Tout, long long ldt, const int* done_flag) {
   if (*reinterpret_cast<const volatile int*>(done_flag)) return;
   extern __shared__ double tsm[];
-  const int pitch = b + 1;
-  double* Ts = tsm;                        // [b][pitch]: T in the upper triangle, the Gram rows below it
-  double* ts = Ts + (size_t)b * pitch;     // [b]: tau
+  const int pitch = b + 1, mp = b / 2 + 1;
+  double* Ts = tsm;                        // [b][pitch]: T above and on the diagonal, Gram rows below
+  double* Ms = Ts + (size_t)b * pitch;     // [b/2][mp]: (V1^T V2) T22 of every pair of the current round
   const int tid = threadIdx.x;
-  const int per = 256 / b;                 // threads per row of T: 2, 4, 8 or 16 adjacent lanes
-  const int i = tid / per, part = tid - i * per;
   for (int idx = tid; idx < b * b; idx += 256) {
     const int r = idx / b, c = idx - r * b;
-    Ts[r * pitch + c] = c < r ? gram[idx] : 0.0;      // Ts[j][l] = v_l^T v_j for l < j
+    Ts[r * pitch + c] = c < r ? gram[idx] : (c == r ? tau[r] : 0.0);    // Ts[j][l] = v_l^T v_j for l < j
   }
-  if (tid < b) ts[tid] = tau[tid];
   __syncthreads();
-  for (int j = 0; j < b; ++j) {
-    const double tj = ts[j];
-    // row i of  -tau_j * T[0:j, 0:j] * g_j : the `per` lanes of a row take every per-th term
-    double s = 0.0;
-    if (i < j)
-      for (int l = i + part; l < j; l += per) s += Ts[i * pitch + l] * Ts[j * pitch + l];
-    for (int o = per >> 1; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
-    if (part == 0) {
-      if (i < j) Ts[i * pitch + j] = -tj * s;
-      else if (i == j) Ts[j * pitch + j] = tj;
+  for (int s = 1; s < b; s <<= 1) {
+    const int per_level = b * s / 2;       // (b / 2s) pairs x s x s entries
+    for (int idx = tid; idx < per_level; idx += 256) {
+      const int q = idx / (s * s), rc = idx - q * s * s, r = rc / s, c = rc - r * s;
+      const int o = 2 * s * q;
+      double acc = 0.0;                    // M[r][c] = sum_k (v_{o+r}^T v_{o+s+k}) T22[k][c], k <= c
+      for (int k = 0; k <= c; ++k) acc += Ts[(o + s + k) * pitch + (o + r)] * Ts[(o + s + k) * pitch + (o + s + c)];
+      Ms[(s * q + r) * mp + c] = acc;
+    }
+    __syncthreads();
+    for (int idx = tid; idx < per_level; idx += 256) {
+      const int q = idx / (s * s), rc = idx - q * s * s, r = rc / s, c = rc - r * s;
+      const int o = 2 * s * q;
+      double acc = 0.0;                    // T12[r][c] = -sum_k T11[r][k] M[k][c], k >= r
+      for (int k = r; k < s; ++k) acc += Ts[(o + r) * pitch + (o + k)] * Ms[(s * q + k) * mp + c];
+      Ts[(o + r) * pitch + (o + s + c)] = -acc;
     }
     __syncthreads();
   }
@@ -342,25 +349,23 @@ __global__ void __launch_bounds__(256)
     init_kernel(const T* __restrict__ A, long long lda, T* __restrict__ W, long long ldw, long long m, long long n,
                 T* __restrict__ V, long long ldv, int vcols, double* __restrict__ part) {
   __shared__ double red[32];
-  const long long total = m * n;
-  const long long chunk = (total + gridDim.x - 1) / gridDim.x;
-  const long long lo = (long long)blockIdx.x * chunk, hi = min(total, lo + chunk);
+  // CTA c owns rows [c*rpc, (c+1)*rpc): fixed chunking, so the partial sums do not depend on scheduling
+  const long long rpc = (m + gridDim.x - 1) / gridDim.x;
+  const long long r_lo = (long long)blockIdx.x * rpc, r_hi = min(m, r_lo + rpc);
   double s = 0.0;
-  for (long long idx = lo + threadIdx.x; idx < hi; idx += 256) {
-    const long long r = idx / n, c = idx - r * n;
-    const T x = A[r * lda + c];
-    if (W != nullptr) W[r * ldw + c] = x;
-    s += (double)x * (double)x;
+  for (long long r = r_lo; r < r_hi; ++r) {
+    const T* src = A + r * lda;
+    T* dst = W != nullptr ? W + r * ldw : nullptr;
+    for (long long c = threadIdx.x; c < n; c += 256) {
+      const T x = src[c];
+      if (dst != nullptr) dst[c] = x;
+      s += (double)x * (double)x;
+    }
+    T* vrow = V + r * ldv;
+    for (int c = threadIdx.x; c < vcols; c += 256) vrow[c] = T(0);
   }
   const double tot = block_sum(s, red);
   if (threadIdx.x == 0) part[blockIdx.x] = tot;
-  const long long vtotal = m * vcols;
-  const long long vchunk = (vtotal + gridDim.x - 1) / gridDim.x;
-  const long long vlo = (long long)blockIdx.x * vchunk, vhi = min(vtotal, vlo + vchunk);
-  for (long long idx = vlo + threadIdx.x; idx < vhi; idx += 256) {
-    const long long r = idx / vcols, c = idx - r * vcols;
-    V[r * ldv + c] = T(0);
-  }
 }
 
 __global__ void __launch_bounds__(256)
