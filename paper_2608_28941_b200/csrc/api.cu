@@ -174,6 +174,8 @@ struct Ops {
     if (e != cudaSuccess) return e;
     e = cudaFuncSetAttribute(upd_sk_kernel<T, B, U_BM, U_BNB, U_WM, U_WN, U_STAGES>,
                              cudaFuncAttributeMaxDynamicSharedMemorySize, U_SMEM);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(tz_kernel<T, B>, cudaFuncAttributeMaxDynamicSharedMemorySize, Z_SMEM);
     return e;
   }
   static void sample(const CUtensorMap& tmW, const CUtensorMap& tmO, void* Ypart, int r0, int rows, int n, int j0,
@@ -186,6 +188,12 @@ struct Ops {
                   Ctrl* ctrl, cudaStream_t st) {
     vtw_sk_kernel<T, B, V_BN, kVtwBK, V_WM, V_WN, V_STAGES>
         <<<p.P, 9 * 32, V_SMEM, st>>>(tmV, tmC, (T*)Zpart, r0, cv0, p.KT, p.total, p.tpc, ctrl);
+  }
+  static constexpr int Z_SMEM = (B * (B + 4) + B * (kTzCols + 4)) * (int)sizeof(T);
+  static void tz(const void* Zpart, const VtwPlan& vp, const void* Tm, long long ldt, int transpose_t, void* Zt,
+                 const int* done_flag, cudaStream_t st) {
+    tz_kernel<T, B><<<vp.npad / kTzCols, kTzThreads, Z_SMEM, st>>>((const T*)Zpart, vp.bn, vp.nct, vp.KT, vp.tpc, (const T*)Tm,
+                                                            ldt, transpose_t, (T*)Zt, done_flag);
   }
   static void update(const CUtensorMap& tmV, const CUtensorMap& tmZ, const CUtensorMap& tmC, const CUtensorMap& tmO,
                      void* C, long long ldc, void* top, long long ldtop, int r0, int rows, int ncols, int cv0,
@@ -203,13 +211,14 @@ struct OpTable {
   void (*sample)(const CUtensorMap&, const CUtensorMap&, void*, int, int, int, int, const SamplePlan&, Ctrl*,
                  cudaStream_t);
   void (*vtw)(const CUtensorMap&, const CUtensorMap&, void*, int, int, const VtwPlan&, Ctrl*, cudaStream_t);
+  void (*tz)(const void*, const VtwPlan&, const void*, long long, int, void*, const int*, cudaStream_t);
   void (*update)(const CUtensorMap&, const CUtensorMap&, const CUtensorMap&, const CUtensorMap&, void*, long long,
                  void*, long long, int, int, int, int, int, int, void*, double*, const UpdPlan&, Ctrl*, cudaStream_t);
 };
 template <typename T, int B>
 static OpTable make_ops() {
   return OpTable{Ops<T, B>::V_BN, Ops<T, B>::U_BM, Ops<T, B>::U_BN, Ops<T, B>::U_WN, &Ops<T, B>::setup, &Ops<T, B>::sample,
-                 &Ops<T, B>::vtw,  &Ops<T, B>::update};
+                 &Ops<T, B>::vtw,  &Ops<T, B>::tz, &Ops<T, B>::update};
 }
 static const OpTable* get_ops(int dtype, int b) {
   static const OpTable d16 = make_ops<double, 16>(), d32 = make_ops<double, 32>(), d64 = make_ops<double, 64>(),
@@ -292,17 +301,6 @@ static rrf_status_t launch_panel(rrf_ctx* h, int dtype, const void* Y, PanelSour
   return RRF_OK;
 }
 
-static void launch_tz(int dtype, const void* Zpart, const VtwPlan& vp, int b, const void* Tm, long long ldt,
-                      int transpose_t, void* Zt, const int* done_flag, cudaStream_t st) {
-  const size_t smem = ((size_t)b * (b + 1) + (size_t)kTzCols * (b + 1)) * sizeof(double);
-  if (dtype == RRF_F64)
-    tz_kernel<double><<<vp.npad / kTzCols, 256, smem, st>>>((const double*)Zpart, vp.bn, vp.nct, vp.KT, vp.tpc, b,
-                                                            (const double*)Tm, ldt, transpose_t, (double*)Zt, done_flag);
-  else
-    tz_kernel<float><<<vp.npad / kTzCols, 256, smem, st>>>((const float*)Zpart, vp.bn, vp.nct, vp.KT, vp.tpc, b,
-                                                           (const float*)Tm, ldt, transpose_t, (float*)Zt, done_flag);
-}
-
 static cudaError_t setup_all(int smem_optin, int* panel_smem_max) {
   cudaError_t e;
   for (int b : {16, 32, 64, 128}) {
@@ -332,10 +330,6 @@ static cudaError_t setup_all(int smem_optin, int* panel_smem_max) {
   if (e != cudaSuccess) return e;
   e = cudaFuncSetAttribute(tfactor_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, tmax);
   if (e != cudaSuccess) return e;
-  const int zmax = (128 * 129 + kTzCols * 129) * 8;
-  e = cudaFuncSetAttribute(tz_kernel<double>, cudaFuncAttributeMaxDynamicSharedMemorySize, zmax);
-  if (e != cudaSuccess) return e;
-  e = cudaFuncSetAttribute(tz_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, zmax);
   return e;
 }
 
@@ -610,8 +604,7 @@ static rrf_status_t apply_blocks(rrf_handle_t h, int dtype, long long m, int b, 
     const int r0 = l * b, rows = (int)(m - r0);
     const VtwPlan vp = plan_vtw(h->sms, rows, ncols, ops->v_bn);
     ops->vtw(tmV_k, tmC_k, Zpart, r0, r0, vp, h->d_ctrl, st);
-    launch_tz(dtype, Zpart, vp, b, (const char*)dT + (size_t)r0 * esize, ldt, transpose ? 1 : 0, Zt, &h->d_ctrl->done,
-              st);
+    ops->tz(Zpart, vp, (const char*)dT + (size_t)r0 * esize, ldt, transpose ? 1 : 0, Zt, &h->d_ctrl->done, st);
     const UpdPlan up = plan_upd(h->sms, rows, ncols, ops->u_bm, ops->u_bn, ops->u_wn);
     ops->update(tmV_u, tmZ, tmC_u, tmC_u, dC, ldc, dC, ldc, r0, rows, (int)ncols, r0, 0, -1, nullptr, nullptr, up,
                 h->d_ctrl, st);
@@ -782,7 +775,7 @@ rrf_status_t rrf_run(rrf_handle_t h, const rrf_params_t* p, void* dA, int64_t ld
     ops->vtw(tmV_k, tmW_k, Zpart, r0, r0, vp, ctrl, st);
     mark(RRF_PHASE_TZ, i);
     cudaStreamWaitEvent(st, h->sync_events[2 * i + 1], 0);   // join: T_i is needed from here on
-    launch_tz(p->dtype, Zpart, vp, b, (const char*)dT + (size_t)r0 * esize, p->max_rank, 1, Zt, &ctrl->done, st);
+    ops->tz(Zpart, vp, (const char*)dT + (size_t)r0 * esize, p->max_rank, 1, Zt, &ctrl->done, st);
     const UpdPlan up = plan_upd(h->sms, rows, n, ops->u_bm, ops->u_bn, ops->u_wn);
     const int j0 = (i + 1 < steps) ? r0 + b : -1;   // Omega rows of the next pass, if there is one
     mark(RRF_PHASE_UPDATE, i);

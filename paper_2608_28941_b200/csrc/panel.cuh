@@ -265,27 +265,58 @@ __global__ void __launch_bounds__(256)
   double* Ts = tsm;                        // [b][pitch]: T above and on the diagonal, Gram rows below
   double* Ms = Ts + (size_t)b * pitch;     // [b/2][mp]: (V1^T V2) T22 of every pair of the current round
   const int tid = threadIdx.x;
-  for (int idx = tid; idx < b * b; idx += 256) {
-    const int r = idx / b, c = idx - r * b;
-    Ts[r * pitch + c] = c < r ? gram[idx] : (c == r ? tau[r] : 0.0);    // Ts[j][l] = v_l^T v_j for l < j
+  // stage the Gram rows (strictly lower triangle) and tau: eight independent loads in flight per thread
+  for (int base = 0; base < b * b; base += 256 * 8) {
+    double v[8];
+#pragma unroll
+    for (int e = 0; e < 8; ++e) {
+      const int idx = base + e * 256 + tid;
+      const int r = idx / b, c = idx - r * b;
+      v[e] = (idx < b * b && c < r) ? __ldcg(gram + idx) : 0.0;
+    }
+#pragma unroll
+    for (int e = 0; e < 8; ++e) {
+      const int idx = base + e * 256 + tid;
+      const int r = idx / b, c = idx - r * b;
+      if (idx < b * b) Ts[r * pitch + c] = v[e];
+    }
   }
+  __syncthreads();
+  if (tid < b) Ts[tid * pitch + tid] = __ldcg(tau + tid);
   __syncthreads();
   for (int s = 1; s < b; s <<= 1) {
     const int per_level = b * s / 2;       // (b / 2s) pairs x s x s entries
+    const int ls = 31 - __clz(s);          // s is a power of two
     for (int idx = tid; idx < per_level; idx += 256) {
-      const int q = idx / (s * s), rc = idx - q * s * s, r = rc / s, c = rc - r * s;
+      const int q = idx >> (2 * ls), rc = idx & (s * s - 1), r = rc >> ls, c = rc & (s - 1);
       const int o = 2 * s * q;
-      double acc = 0.0;                    // M[r][c] = sum_k (v_{o+r}^T v_{o+s+k}) T22[k][c], k <= c
-      for (int k = 0; k <= c; ++k) acc += Ts[(o + s + k) * pitch + (o + r)] * Ts[(o + s + k) * pitch + (o + s + c)];
-      Ms[(s * q + r) * mp + c] = acc;
+      // M[r][c] = sum_{k <= c} (v_{o+r}^T v_{o+s+k}) T22[k][c]; two independent partial sums
+      const double* ga = Ts + (size_t)(o + s) * pitch + (o + r);
+      const double* tb = Ts + (size_t)(o + s) * pitch + (o + s + c);
+      double a0 = 0.0, a1 = 0.0;
+      int k = 0;
+      for (; k + 1 <= c; k += 2) {
+        a0 += ga[k * pitch] * tb[k * pitch];
+        a1 += ga[(k + 1) * pitch] * tb[(k + 1) * pitch];
+      }
+      if (k <= c) a0 += ga[k * pitch] * tb[k * pitch];
+      Ms[(s * q + r) * mp + c] = a0 + a1;
     }
     __syncthreads();
     for (int idx = tid; idx < per_level; idx += 256) {
-      const int q = idx / (s * s), rc = idx - q * s * s, r = rc / s, c = rc - r * s;
+      const int q = idx >> (2 * ls), rc = idx & (s * s - 1), r = rc >> ls, c = rc & (s - 1);
       const int o = 2 * s * q;
-      double acc = 0.0;                    // T12[r][c] = -sum_k T11[r][k] M[k][c], k >= r
-      for (int k = r; k < s; ++k) acc += Ts[(o + r) * pitch + (o + k)] * Ms[(s * q + k) * mp + c];
-      Ts[(o + r) * pitch + (o + s + c)] = -acc;
+      // T12[r][c] = -sum_{k >= r} T11[r][k] M[k][c]
+      const double* ta = Ts + (size_t)(o + r) * pitch + o;
+      const double* mb = Ms + (size_t)(s * q) * mp + c;
+      double a0 = 0.0, a1 = 0.0;
+      int k = r;
+      for (; k + 1 < s; k += 2) {
+        a0 += ta[k] * mb[k * mp];
+        a1 += ta[k + 1] * mb[(k + 1) * mp];
+      }
+      if (k < s) a0 += ta[k] * mb[k * mp];
+      Ts[(o + r) * pitch + (o + s + c)] = -(a0 + a1);
     }
     __syncthreads();
   }
@@ -296,47 +327,98 @@ __global__ void __launch_bounds__(256)
 }
 
 // ------------------------------------------------------------------------------------------
-// Zt[col][0:b] = (op(T) * sum_seg Zpart[seg][:, col])   with op(T) = T^T (apply Q^T) or T (apply Q).
-// Each CTA owns kTzCols columns.  Output is the transposed (K-contiguous) operand of update_kernel.
+// Zt[col][0:B] = (op(T) * sum of the partial slots of Z[:, col])   with op(T) = T^T (apply Q^T) or
+// T (apply Q).  Zpart is in the slot layout of vtw_sk_kernel: column tile ct (bn columns) is the sum
+// of slots p + ct for the CTAs p whose tile range [p*tpc, (p+1)*tpc) meets [ct*kt, (ct+1)*kt),
+// summed in CTA order.  Each CTA owns kTzCols columns: it stages op(T) (as the A operand, K = row)
+// and the summed columns in shared memory with a pitch of 4 mod 16 elements, which makes the scalar
+// fragment loads conflict free, and multiplies on the tensor cores.  The output is the transposed
+// (K-contiguous) operand of upd_sk_kernel.
 // ------------------------------------------------------------------------------------------
 constexpr int kTzCols = 32;
-// Zpart is in the slot layout of vtw_sk_kernel: column tile c (bn columns) is the sum of slots
-// p + c for the CTAs p whose tile range [p*tpc, (p+1)*tpc) meets [c*kt, (c+1)*kt).
-template <typename T>
-__global__ void __launch_bounds__(256)
-    tz_kernel(const T* __restrict__ Zpart, int bn, int nct, int kt, int tpc, int b, const T* __restrict__ Tm, long long ldt,
+constexpr int kTzThreads = 512;
+template <typename T, int B>
+__global__ void __launch_bounds__(kTzThreads)
+    tz_kernel(const T* __restrict__ Zpart, int bn, int nct, int kt, int tpc, const T* __restrict__ Tm, long long ldt,
               int transpose_t, T* __restrict__ Zt, const int* done_flag) {
   if (*reinterpret_cast<const volatile int*>(done_flag)) return;
-  extern __shared__ double zsm[];
-  const int pitch = b + 1;
-  double* Ts = zsm;                         // [b][pitch]
-  double* Zs = Ts + (size_t)b * pitch;      // [kTzCols][pitch]
-  const int tid = threadIdx.x;
+  constexpr int PA = B + 4, PB = kTzCols + 4;
+  constexpr int NWARP = kTzThreads / 32;
+  constexpr int MTILES = B / 16, NTILES = kTzCols / 8;
+  extern __shared__ unsigned char zsm_raw[];
+  T* As = reinterpret_cast<T*>(zsm_raw);          // [B][PA]: As[l][j] = op(T)[j][l]
+  T* Bs = As + (size_t)B * PA;                    // [B][PB]: summed Z[l][col]
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
   const int col0 = blockIdx.x * kTzCols;
-  for (int idx = tid; idx < b * b; idx += 256) {
-    const int i = idx / b, j = idx - i * b;
-    Ts[i * pitch + j] = (double)Tm[(size_t)i * ldt + j];
+  {
+    constexpr int EA = (B * B + kTzThreads - 1) / kTzThreads;
+    T v[EA];
+#pragma unroll
+    for (int e = 0; e < EA; ++e) {
+      const int idx = tid + e * kTzThreads, l = idx / B, j = idx - l * B;
+      v[e] = T(0);
+      if (idx < B * B) {
+        if (transpose_t) { if (l <= j) v[e] = Tm[(size_t)l * ldt + j]; }     // (T^T)[j][l] = T[l][j], upper triangular
+        else             { if (j <= l) v[e] = Tm[(size_t)j * ldt + l]; }     // T[j][l]
+      }
+    }
+#pragma unroll
+    for (int e = 0; e < EA; ++e) {
+      const int idx = tid + e * kTzThreads, l = idx / B, j = idx - l * B;
+      if (idx < B * B) As[l * PA + j] = v[e];
+    }
   }
-  const int ct = col0 / bn, cin = col0 - ct * bn;   // column tiles past the last one hold no data
+  const int ct = col0 / bn, cin = col0 - ct * bn;   // kTzCols divides bn; tiles past the last hold no data
   const int p_lo = (ct * kt) / tpc, p_hi = ((ct + 1) * kt - 1) / tpc;
-  for (int idx = tid; idx < b * kTzCols; idx += 256) {
-    const int l = idx / kTzCols, cl = idx - l * kTzCols;
-    double s = 0.0;
-    if (ct < nct)
-      for (int p = p_lo; p <= p_hi; ++p) s += (double)Zpart[(size_t)(p + ct) * (size_t)(b * bn) + (size_t)l * bn + cin + cl];
-    Zs[cl * pitch + l] = s;
+  {
+    // every thread owns EPT entries; the loads of up to eight slots are in flight together and are
+    // then added in slot (= CTA) order
+    constexpr int EPT = (B * kTzCols + kTzThreads - 1) / kTzThreads;
+    constexpr int SB = EPT >= 8 ? 4 : 8;            // slots per batch, bounded by registers
+    double sum[EPT];
+#pragma unroll
+    for (int e = 0; e < EPT; ++e) sum[e] = 0.0;
+    if (ct < nct) {
+      for (int p0 = p_lo; p0 <= p_hi; p0 += SB) {
+        T v[SB][EPT];
+#pragma unroll
+        for (int u = 0; u < SB; ++u) {
+          const T* slot = Zpart + (size_t)(p0 + u + ct) * (size_t)(B * bn) + cin;
+#pragma unroll
+          for (int e = 0; e < EPT; ++e) {
+            const int idx = tid + e * kTzThreads, l = idx / kTzCols, cl = idx - l * kTzCols;
+            v[u][e] = (p0 + u <= p_hi && idx < B * kTzCols) ? __ldcg(slot + (size_t)l * bn + cl) : T(0);
+          }
+        }
+#pragma unroll
+        for (int u = 0; u < SB; ++u)
+#pragma unroll
+          for (int e = 0; e < EPT; ++e) sum[e] += (double)v[u][e];
+      }
+    }
+#pragma unroll
+    for (int e = 0; e < EPT; ++e) {
+      const int idx = tid + e * kTzThreads, l = idx / kTzCols, cl = idx - l * kTzCols;
+      if (idx < B * kTzCols) Bs[l * PB + cl] = (T)sum[e];
+    }
   }
   __syncthreads();
-  const int j = tid % b, cq = tid / b, ncq = 256 / b;
-  for (int cl = cq; cl < kTzCols; cl += ncq) {
-    const double* z = Zs + cl * pitch;
-    double s = 0.0;
-    if (transpose_t) {
-      for (int l = 0; l <= j; ++l) s += Ts[l * pitch + j] * z[l];
-    } else {
-      for (int l = j; l < b; ++l) s += Ts[j * pitch + l] * z[l];
+  for (int tile = warp; tile < MTILES * NTILES; tile += NWARP) {
+    const int j0 = (tile / NTILES) * 16, n0 = (tile % NTILES) * 8;
+    T acc[4] = {T(0), T(0), T(0), T(0)};
+#pragma unroll 4
+    for (int ks = 0; ks < B / 8; ++ks) {
+      const int k = ks * 8 + t;
+      const T af[4] = {As[k * PA + j0 + g], As[k * PA + j0 + g + 8], As[(k + 4) * PA + j0 + g],
+                       As[(k + 4) * PA + j0 + g + 8]};
+      const T bf[2] = {Bs[k * PB + n0 + g], Bs[(k + 4) * PB + n0 + g]};
+      mma16x8x8(acc, af, bf);
     }
-    Zt[(size_t)(col0 + cl) * b + j] = (T)s;
+    const int j = j0 + g, col = col0 + n0 + 2 * t;
+    Zt[(size_t)col * B + j] = acc[0];
+    Zt[(size_t)(col + 1) * B + j] = acc[1];
+    Zt[(size_t)col * B + j + 8] = acc[2];
+    Zt[(size_t)(col + 1) * B + j + 8] = acc[3];
   }
 }
 
