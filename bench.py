@@ -27,9 +27,10 @@ if ROOT not in sys.path:
 
 import numpy as np  # noqa: E402
 
-# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu
-# capture summarised under profiles/ (None until a capture of the current kernel exists).
-NCU_TRAFFIC_BYTES = {}
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel of the default
+# workload, from the ncu capture summarised in profiles/kernels_cfg2_4096x4096_b64.md (captured on a
+# 4096 x 4096 case and scaled to the bench's average launch by the elements processed).
+NCU_TRAFFIC_BYTES = {("cfg2", "update"): 1.07e9, ("cfg2", "vtw"): 136.3e6 * 3.875}
 
 NOMINAL_FP64_OVER_BF16 = 37.0 / 2250.0   # HGX B200 dense figures: FP64 tensor 37 TF, bf16 2250 TF
 
@@ -94,6 +95,22 @@ class ClockSampler:
                     reasons.add(nm)
         return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": mx, "reasons": sorted(reasons),
                 "samples": len(sm)}
+
+
+def max_over_ranks(ms: float, world: int, device) -> float:
+    """Slowest rank's time: every multi-GPU number is the maximum over ranks."""
+    if world == 1:
+        return float(ms)
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def job_tflops(flops_per_replica: float, world: int, ms_step: float) -> float:
+    """Whole-job rate of `world` independent replicas that all took `ms_step` (the slowest rank's time)."""
+    return world * flops_per_replica / (ms_step * 1e-3) / 1e12
 
 
 def oracle_run(A, Om, w, blocks=None):
@@ -246,13 +263,9 @@ def main():
     e1.record()
     barrier()
     clocks = sampler.stop()
-    ms_total = e0.elapsed_time(e1)
-    t = torch.tensor([ms_total], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    ms_step = float(t.item()) / args.steps
+    ms_step = max_over_ranks(e0.elapsed_time(e1), world, dev) / args.steps
     flops = method_flops(w.m, w.n, w.b, res.steps)
-    value = world * flops / (ms_step * 1e-3) / 1e12
+    value = job_tflops(flops, world, ms_step)
     launches_per_run = 3 + 6 * (w.max_rank // w.b)   # init x2, first sample; panel, T, VtW, TZ, update, stop per pass
 
     # ---- end to end through the C ABI with host buffers
@@ -284,11 +297,8 @@ def main():
             e2e_step()
         e1.record()
         barrier()
-        t = torch.tensor([e0.elapsed_time(e1)], dtype=torch.float64, device=dev)
-        if world > 1:
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_e2e = float(t.item()) / n_e2e
-        e2e = {"value": world * flops / (ms_e2e * 1e-3) / 1e12, "unit": "TFLOP/s", "ms_per_step": ms_e2e,
+        ms_e2e = max_over_ranks(e0.elapsed_time(e1), world, dev) / n_e2e
+        e2e = {"value": job_tflops(flops, world, ms_e2e), "unit": "TFLOP/s", "ms_per_step": ms_e2e,
                "h2d_bytes_per_step": int((A_h.numel() + O_h.numel()) * esize),
                "d2h_bytes_per_step": int((k * w.n + w.m * k + w.b * k) * esize)}
 
@@ -314,7 +324,7 @@ def main():
             achieved = work / (ms * 1e-3) / 1e12
             recipe = peaks.get("bf16_tflops", 1590.0) * NOMINAL_FP64_OVER_BF16 if w.dtype == "f64" else None
             roofline = {"kernel": top, "bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
-                        "frac": achieved / peak, "traffic": NCU_TRAFFIC_BYTES.get(top),
+                        "frac": achieved / peak, "traffic": NCU_TRAFFIC_BYTES.get((w.name, top)),
                         "peak_source": "FP64 mma.sync rate measured live by rrf_measure_peak" if w.dtype == "f64"
                         else "TF32 mma.sync rate / 3 measured live by rrf_measure_peak",
                         "peak_recipe": recipe,
@@ -327,7 +337,7 @@ def main():
             byts = args.steps * sum(2.0 * r * w.b * esize for r in mi)
             achieved = byts / (ms * 1e-3) / 1e9
             roofline = {"kernel": top, "bound": "hbm", "achieved": achieved, "peak": hbm, "unit": "GB/s",
-                        "frac": achieved / hbm, "traffic": NCU_TRAFFIC_BYTES.get(top),
+                        "frac": achieved / hbm, "traffic": NCU_TRAFFIC_BYTES.get((w.name, top)),
                         "peak_source": "MEASURED_PEAKS.json (of measured)" if "hbm_gbs" in peaks else "of fallback",
                         "avg_launch_ms": ms / max(cnt, 1), "launches": cnt}
         roofline["phases_ms_per_step"] = {nm: prof[nm][0] / args.steps for nm in prof}
