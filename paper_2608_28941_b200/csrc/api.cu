@@ -162,6 +162,7 @@ struct Ops {
   static constexpr int U_STAGE = U_BNB * U_BM * 128 + U_KB * U_BN * 128 + U_BNB * B * 128;
   static constexpr int U_STAGES = (U_VBYTES + 3 * U_STAGE + 1024 <= 226 * 1024) ? 3 : 2;
   static constexpr int U_SMEM = U_VBYTES + U_STAGES * U_STAGE + 1024;
+  static constexpr bool U_PW = false;   // the widest fp64 block needs the registers of 8 warps
   static_assert(U_SMEM + 1024 <= kMaxSmem && V_SMEM + 1024 <= kMaxSmem && S_SMEM + 1024 <= kMaxSmem, "shared memory");
 
   static cudaError_t setup() {
@@ -172,7 +173,7 @@ struct Ops {
     e = cudaFuncSetAttribute(vtw_sk_kernel<T, B, V_BN, kVtwBK, V_WM, V_WN, V_STAGES>,
                              cudaFuncAttributeMaxDynamicSharedMemorySize, V_SMEM);
     if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(upd_sk_kernel<T, B, U_BM, U_BNB, U_WM, U_WN, U_STAGES>,
+    e = cudaFuncSetAttribute(upd_sk_kernel<T, B, U_BM, U_BNB, U_WM, U_WN, U_STAGES, U_PW>,
                              cudaFuncAttributeMaxDynamicSharedMemorySize, U_SMEM);
     if (e != cudaSuccess) return e;
     e = cudaFuncSetAttribute(tz_kernel<T, B>, cudaFuncAttributeMaxDynamicSharedMemorySize, Z_SMEM);
@@ -199,7 +200,7 @@ struct Ops {
                      void* C, long long ldc, void* top, long long ldtop, int r0, int rows, int ncols, int cv0,
                      int top_rows, int j0, void* Ypart, double* norm_part, const UpdPlan& p, Ctrl* ctrl,
                      cudaStream_t st) {
-    upd_sk_kernel<T, B, U_BM, U_BNB, U_WM, U_WN, U_STAGES><<<p.P, 9 * 32, U_SMEM, st>>>(
+    upd_sk_kernel<T, B, U_BM, U_BNB, U_WM, U_WN, U_STAGES, U_PW><<<p.P, (U_PW ? 9 : 8) * 32, U_SMEM, st>>>(
         tmV, tmZ, tmC, tmO, (T*)C, ldc, (T*)top, ldtop, r0, rows, ncols, cv0, top_rows, j0, (T*)Ypart, norm_part, p.NC,
         p.total, p.tpc, ctrl);
   }

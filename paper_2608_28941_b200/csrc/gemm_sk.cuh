@@ -167,8 +167,11 @@ __global__ void __launch_bounds__((WM * WN + 1) * 32)
 // same chunk rule as every other K-contiguous operand.  No shuffles, no shared-memory round trip.
 // Slot ((p + s)*WN + wn) of Ypart holds the BM x B partial of slab s from CTA p, warp column wn.
 // ------------------------------------------------------------------------------------------
-template <typename T, int B, int BM, int BNB, int WM, int WN, int STAGES>
-__global__ void __launch_bounds__((WM * WN + 1) * 32, 1)
+// PW: a dedicated producer warp issues the TMA loads.  Without it (PW = false) lane 0 of consumer
+// warp 0 issues them at the top of each tile, which leaves the CTA at eight warps - two per SM
+// sub-partition, hence up to 255 registers per thread for the widest block size.
+template <typename T, int B, int BM, int BNB, int WM, int WN, int STAGES, bool PW>
+__global__ void __launch_bounds__((WM * WN + (PW ? 1 : 0)) * 32, 1)
     upd_sk_kernel(const __grid_constant__ CUtensorMap tmV,  // V [m][ldv], box [BM][KE]
                   const __grid_constant__ CUtensorMap tmZ,  // Zt [npad][B], box [BN][KE]
                   const __grid_constant__ CUtensorMap tmC,  // C [m][ncols], box [BM][KE]
@@ -218,7 +221,28 @@ __global__ void __launch_bounds__((WM * WN + 1) * 32, 1)
 
   double s_top = 0.0, s_trail = 0.0;
 
-  if (warp == NCW) {
+  // loads of one tile (and of V when the tile opens a new row slab); called by one thread
+  auto load_slab = [&](int s) {
+    mbar_expect_tx(&v_full, V_BYTES);
+#pragma unroll
+    for (int kb = 0; kb < KB; ++kb) tma_load_2d(sVs + kb * V_BOX, &tmV, cv0 + kb * KE, r0 + s * BM, &v_full);
+  };
+  auto load_tile = [&](int i, int s, int c) {
+    const int st = i % STAGES;
+    unsigned char* sW = sStage + st * STAGE_BYTES;
+    mbar_expect_tx(&full[st], do_sample ? STAGE_BYTES : W_BYTES + Z_BYTES);
+#pragma unroll
+    for (int q = 0; q < BNB; ++q) tma_load_2d(sW + q * W_BOX, &tmC, c * BN + q * KE, r0 + s * BM, &full[st]);
+#pragma unroll
+    for (int kb = 0; kb < KB; ++kb) tma_load_2d(sW + W_BYTES + kb * Z_BOX, &tmZ, kb * KE, c * BN, &full[st]);
+    if (do_sample) {
+#pragma unroll
+      for (int q = 0; q < BNB; ++q)
+        tma_load_2d(sW + W_BYTES + Z_BYTES + q * O_BOX, &tmO, c * BN + q * KE, j0, &full[st]);
+    }
+  };
+
+  if (PW && warp == NCW) {
     // ------------------------------------------------------------ producer warp
     if (lane == 0) {
       int cur_s = -1, nslab = 0;
@@ -226,25 +250,12 @@ __global__ void __launch_bounds__((WM * WN + 1) * 32, 1)
       for (int i = 0; i < ntile; ++i, c = (c + 1 == NC ? 0 : c + 1), s += (c == 0)) {
         if (s != cur_s) {
           if (nslab > 0 && !mbar_wait(&v_empty, (nslab - 1) & 1, ctrl)) break;
-          mbar_expect_tx(&v_full, V_BYTES);
-#pragma unroll
-          for (int kb = 0; kb < KB; ++kb) tma_load_2d(sVs + kb * V_BOX, &tmV, cv0 + kb * KE, r0 + s * BM, &v_full);
+          load_slab(s);
           cur_s = s;
           ++nslab;
         }
-        const int st = i % STAGES;
-        if (i >= STAGES && !mbar_wait(&empty[st], ((i / STAGES) - 1) & 1, ctrl)) break;
-        unsigned char* sW = sStage + st * STAGE_BYTES;
-        mbar_expect_tx(&full[st], do_sample ? STAGE_BYTES : W_BYTES + Z_BYTES);
-#pragma unroll
-        for (int q = 0; q < BNB; ++q) tma_load_2d(sW + q * W_BOX, &tmC, c * BN + q * KE, r0 + s * BM, &full[st]);
-#pragma unroll
-        for (int kb = 0; kb < KB; ++kb) tma_load_2d(sW + W_BYTES + kb * Z_BOX, &tmZ, kb * KE, c * BN, &full[st]);
-        if (do_sample) {
-#pragma unroll
-          for (int q = 0; q < BNB; ++q)
-            tma_load_2d(sW + W_BYTES + Z_BYTES + q * O_BOX, &tmO, c * BN + q * KE, j0, &full[st]);
-        }
+        if (i >= STAGES && !mbar_wait(&empty[i % STAGES], ((i / STAGES) - 1) & 1, ctrl)) break;
+        load_tile(i, s, c);
       }
     }
   } else {
@@ -262,17 +273,39 @@ __global__ void __launch_bounds__((WM * WN + 1) * 32, 1)
     bool ok = true;
     int s = L0 / NC, c = L0 - s * NC, st = 0;
     uint32_t ph = 0;
+    // state of the inline producer (PW = false; used by lane 0 of warp 0 only)
+    int nxt = 0, p_s = s, p_c = c, p_cur_s = -1, p_nslab = 0;
     // per slab: where this thread's rows go, and to which norm they count (hoisted out of the tile loop)
     T* rowp[MT][2];
     bool rtop[MT][2];
     for (int i = 0; i < ntile && ok; ++i) {
-      if (s != cur_s) {
-        if (cur_s >= 0) {
-          if (do_sample)
-            flush_tile<T, MT, NTB>(accY, Ypart + ((size_t)(p + cur_s) * WN + wn) * (size_t)(BM * B), B, wm * TM, 0, g, t);
-          __syncwarp();
-          if (lane == 0) mbar_arrive(&v_empty);
+      if (s != cur_s && cur_s >= 0) {
+        if (do_sample)
+          flush_tile<T, MT, NTB>(accY, Ypart + ((size_t)(p + cur_s) * WN + wn) * (size_t)(BM * B), B, wm * TM, 0, g, t);
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&v_empty);
+      }
+      if (!PW) {
+        if (warp == 0 && lane == 0) {
+          // issue every tile up to STAGES-1 ahead; a tile that opens a new slab waits until the
+          // consumers stand at it (the V buffer is single)
+          while (nxt < ntile && nxt <= i + STAGES - 1) {
+            if (p_s != p_cur_s) {
+              if (nxt != i) break;
+              if (p_nslab > 0 && !mbar_wait(&v_empty, (p_nslab - 1) & 1, ctrl)) break;
+              load_slab(p_s);
+              p_cur_s = p_s;
+              ++p_nslab;
+            }
+            if (nxt >= STAGES && !mbar_wait(&empty[nxt % STAGES], ((nxt / STAGES) - 1) & 1, ctrl)) break;
+            load_tile(nxt, p_s, p_c);
+            ++nxt;
+            if (++p_c == NC) { p_c = 0; ++p_s; }
+          }
         }
+        __syncwarp();
+      }
+      if (s != cur_s) {
         if (!mbar_wait(&v_full, nslab & 1, ctrl)) { ok = false; break; }
         cur_s = s;
         ++nslab;
