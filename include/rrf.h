@@ -227,6 +227,15 @@ rrf_status_t rrf_set_profiling(rrf_handle_t h, int32_t enable);
 rrf_status_t rrf_get_profile(rrf_handle_t h, rrf_profile_t* out);
 rrf_status_t rrf_measure_peak(rrf_handle_t h, int32_t kind, double ms, double* tflops);
 
+/*
+ * rrf_selftest_timeout - failure-detection self test (no counterpart in the paper).  Launches one
+ * small CTA that waits, with the library's bounded grid-barrier wait shortened to `limit_ms`
+ * milliseconds, for an arrival that never comes.  The wait gives up, the kernel records
+ * RRF_ERR_TIMEOUT in the handle's device status word and returns normally: nothing traps, faults or
+ * hangs, and the context stays usable.  The next rrf_last_status() call reports and clears it.
+ */
+rrf_status_t rrf_selftest_timeout(rrf_handle_t h, double limit_ms, void* cuda_stream);
+
 /* Status word of the handle's device side (set by bounded waits), read with one small
  * device-to-host copy after synchronising `cuda_stream`; clears it. */
 rrf_status_t rrf_last_status(rrf_handle_t h, void* cuda_stream);

@@ -507,6 +507,14 @@ rrf_status_t rrf_measure_peak(rrf_handle_t h, int32_t kind, double ms, double* t
   return cudaGetLastError() == cudaSuccess ? RRF_OK : RRF_ERR_CUDA;
 }
 
+rrf_status_t rrf_selftest_timeout(rrf_handle_t h, double limit_ms, void* cuda_stream) {
+  if (h == nullptr || !(limit_ms > 0.0) || limit_ms > 1000.0) return RRF_ERR_INVALID_ARG;
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  if (cudaMemsetAsync(&h->d_ctrl->bar, 0, sizeof(unsigned), st) != cudaSuccess) return RRF_ERR_CUDA;
+  timeout_selftest_kernel<<<1, 32, 0, st>>>(&h->d_ctrl->bar, h->d_ctrl, (long long)(limit_ms * 2.0e6));
+  return cudaGetLastError() == cudaSuccess ? RRF_OK : RRF_ERR_CUDA;
+}
+
 rrf_status_t rrf_workspace_bytes(const rrf_params_t* p, size_t* bytes) {
   if (bytes == nullptr) return RRF_ERR_INVALID_ARG;
   const rrf_status_t s = check_params(p);

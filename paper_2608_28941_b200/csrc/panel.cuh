@@ -13,7 +13,8 @@ __host__ __device__ constexpr int panel_extra_doubles(int b) { return 3 * b; }
 
 // Grid-wide barrier over a monotonically increasing arrival counter.  Needs all CTAs
 // co-resident (cooperative launch).  Bounded: gives up after kWaitLimitClocks.
-__device__ __forceinline__ bool grid_barrier(unsigned* ctr, unsigned target, Ctrl* ctrl) {
+__device__ __forceinline__ bool grid_barrier(unsigned* ctr, unsigned target, Ctrl* ctrl,
+                                             long long limit = kWaitLimitClocks) {
   __shared__ int ok_s;
   __syncthreads();
   if (threadIdx.x == 0) {
@@ -25,7 +26,7 @@ __device__ __forceinline__ bool grid_barrier(unsigned* ctr, unsigned target, Ctr
       unsigned v;
       asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(ctr) : "memory");
       if (v >= target) break;
-      if (clock64() - t0 > kWaitLimitClocks) {
+      if (clock64() - t0 > limit) {
         atomicExch(&ctrl->status, (int)RRF_ERR_TIMEOUT);
         ok = 0;
         break;
@@ -35,6 +36,11 @@ __device__ __forceinline__ bool grid_barrier(unsigned* ctr, unsigned target, Ctr
   }
   __syncthreads();
   return ok_s != 0;
+}
+
+// Self test of the bounded wait: one CTA arrives at a barrier that expects two.
+__global__ void __launch_bounds__(32) timeout_selftest_kernel(unsigned* ctr, Ctrl* ctrl, long long limit) {
+  grid_barrier(ctr, 2u, ctrl, limit);
 }
 
 // ------------------------------------------------------------------------------------------

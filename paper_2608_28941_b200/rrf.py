@@ -40,7 +40,7 @@ class rrf_profile_t(C.Structure):
     _fields_ = [("ms", C.c_double * 9), ("launches", C.c_int32 * 9), ("pad", C.c_int32)]
 
 
-EXPORTS = ["rrf_panel_qr_static", "rrf_set_profiling", "rrf_get_profile", "rrf_measure_peak", "rrf_create", "rrf_destroy", "rrf_workspace_bytes", "rrf_run", "rrf_panel_workspace_bytes",
+EXPORTS = ["rrf_selftest_timeout", "rrf_panel_qr_static", "rrf_set_profiling", "rrf_get_profile", "rrf_measure_peak", "rrf_create", "rrf_destroy", "rrf_workspace_bytes", "rrf_run", "rrf_panel_workspace_bytes",
            "rrf_panel_qr", "rrf_apply_workspace_bytes", "rrf_apply_qt", "rrf_apply_q", "rrf_form_q",
            "rrf_fill_omega", "rrf_last_status", "rrf_status_string"]
 
@@ -69,6 +69,7 @@ def load():
     lib.rrf_form_q.argtypes = [vp, i32, i64, i32, i32, vp, i64, vp, i64, vp, i64, vp, sz, vp]
     lib.rrf_fill_omega.argtypes = [vp, i32, u64, i64, i32, i32, vp, i64, vp]
     lib.rrf_last_status.argtypes = [vp, vp]
+    lib.rrf_selftest_timeout.argtypes = [vp, C.c_double, vp]
     lib.rrf_set_profiling.argtypes = [vp, i32]
     lib.rrf_get_profile.argtypes = [vp, C.POINTER(rrf_profile_t)]
     lib.rrf_measure_peak.argtypes = [vp, i32, C.c_double, C.POINTER(C.c_double)]
@@ -318,3 +319,11 @@ def rrf_measure_peak(h, kind: int, ms: float = 50.0) -> float:
     if s != RRF_OK:
         raise RrfError(s, "rrf_measure_peak")
     return out.value
+
+
+def rrf_selftest_timeout(h, limit_ms: float = 50.0) -> int:
+    """Make a bounded device-side wait run out; returns the status the device recorded."""
+    s = load().rrf_selftest_timeout(h, limit_ms, _stream())
+    if s != RRF_OK:
+        raise RrfError(s, "rrf_selftest_timeout")
+    return rrf_last_status(h)
