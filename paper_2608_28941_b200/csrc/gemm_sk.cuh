@@ -106,6 +106,29 @@ __global__ void __launch_bounds__((WM * WN + 1) * 32)
 #pragma unroll
       for (int e = 0; e < 4; ++e) acc[a][c][e] = T(0);
 
+  // per-thread byte offsets of the fragment elements inside a stage (rows 2t and 2t+1 of each box)
+  uint32_t offA[MT][4], offB[NT][2];
+  {
+    const uint32_t x0 = ((uint32_t)(2 * t) & 7u) << 4, x1 = ((uint32_t)(2 * t + 1) & 7u) << 4;
+    const uint32_t r0b = (uint32_t)(2 * t) * 128u, r1b = r0b + 128u;
+#pragma unroll
+    for (int a = 0; a < MT; ++a) {
+      const int j = wm * TM + a * 16 + g;
+      const uint32_t b_lo = (uint32_t)(j / KE) * BOX_BYTES, b_hi = (uint32_t)((j + 8) / KE) * BOX_BYTES;
+      const uint32_t c_lo = (uint32_t)(j % KE) * sizeof(T), c_hi = (uint32_t)((j + 8) % KE) * sizeof(T);
+      offA[a][0] = b_lo + r0b + (c_lo ^ x0);
+      offA[a][1] = b_hi + r0b + (c_hi ^ x0);
+      offA[a][2] = b_lo + r1b + (c_lo ^ x1);
+      offA[a][3] = b_hi + r1b + (c_hi ^ x1);
+    }
+#pragma unroll
+    for (int cc = 0; cc < NT; ++cc) {
+      const int nn = wn * TN + cc * 8 + g;
+      const uint32_t bb = (uint32_t)(nn / KE) * BOX_BYTES, co = (uint32_t)(nn % KE) * sizeof(T);
+      offB[cc][0] = bb + r0b + (co ^ x0);
+      offB[cc][1] = bb + r1b + (co ^ x1);
+    }
+  }
   int cur_c = L0 / KT;
   int c = cur_c, kt = L0 - cur_c * KT, st = 0;
   uint32_t ph = 0;
@@ -117,28 +140,23 @@ __global__ void __launch_bounds__((WM * WN + 1) * 32)
     if (!mbar_wait(&full[st], ph, ctrl)) return;
     const unsigned char* sV = smem + st * STAGE_BYTES;
     const unsigned char* sC = sV + V_BYTES;
+    // Rows k = 8*ks + 2t and k + 1 of a box: the swizzle XORs the 16-byte chunk index with k & 7,
+    // which is 2t or 2t + 1 whatever ks is, so every fragment address is a per-thread constant
+    // plus ks * 1024 bytes.
 #pragma unroll
     for (int ks = 0; ks < BK / 8; ++ks) {
-      const uint32_t k = ks * 8 + 2 * t;
       T af[MT][4], bf[NT][2];
 #pragma unroll
       for (int a = 0; a < MT; ++a) {
-        const int j = wm * TM + a * 16 + g;
-        const unsigned char* box_lo = sV + (j / KE) * BOX_BYTES;
-        const unsigned char* box_hi = sV + ((j + 8) / KE) * BOX_BYTES;
-        const uint32_t c_lo = (j % KE) * sizeof(T), c_hi = ((j + 8) % KE) * sizeof(T);
-        af[a][0] = *reinterpret_cast<const T*>(box_lo + swz128(k * 128 + c_lo));
-        af[a][1] = *reinterpret_cast<const T*>(box_hi + swz128(k * 128 + c_hi));
-        af[a][2] = *reinterpret_cast<const T*>(box_lo + swz128((k + 1) * 128 + c_lo));
-        af[a][3] = *reinterpret_cast<const T*>(box_hi + swz128((k + 1) * 128 + c_hi));
+        af[a][0] = *reinterpret_cast<const T*>(sV + offA[a][0] + ks * 1024);
+        af[a][1] = *reinterpret_cast<const T*>(sV + offA[a][1] + ks * 1024);
+        af[a][2] = *reinterpret_cast<const T*>(sV + offA[a][2] + ks * 1024);
+        af[a][3] = *reinterpret_cast<const T*>(sV + offA[a][3] + ks * 1024);
       }
 #pragma unroll
       for (int cc = 0; cc < NT; ++cc) {
-        const int nn = wn * TN + cc * 8 + g;
-        const unsigned char* box = sC + (nn / KE) * BOX_BYTES;
-        const uint32_t co = (nn % KE) * sizeof(T);
-        bf[cc][0] = *reinterpret_cast<const T*>(box + swz128(k * 128 + co));
-        bf[cc][1] = *reinterpret_cast<const T*>(box + swz128((k + 1) * 128 + co));
+        bf[cc][0] = *reinterpret_cast<const T*>(sC + offB[cc][0] + ks * 1024);
+        bf[cc][1] = *reinterpret_cast<const T*>(sC + offB[cc][1] + ks * 1024);
       }
 #pragma unroll
       for (int a = 0; a < MT; ++a)
