@@ -43,17 +43,28 @@ static inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; 
 static inline int ceil_div(long long a, long long b) { return (int)((a + b - 1) / b); }
 
 // ------------------------------------------------------------------ tile configuration
-constexpr int kSampleBM = 128, kSampleStages = 4;
+constexpr int kSampleBM = 128, kSampleStages = 2;
 constexpr int kVtwBK = 64;
 
 struct SamplePlan { int nslabs, nseg, kt_per_seg; };
-static SamplePlan plan_sample(long long rows, long long n, int esize) {
+constexpr int kSampleMaxSeg = 12;
+// K segments are chosen to fill whole waves of one CTA per SM with equal K ranges
+static SamplePlan plan_sample(int sms, long long rows, long long n, int esize, int kbs) {
   SamplePlan p;
   const int KE = 128 / esize;
   p.nslabs = ceil_div(rows, kSampleBM);
-  const int KT = ceil_div(n, KE);
-  int nseg = std::max(1, std::min(std::min(KT, 16), ceil_div(kTargetCtas, p.nslabs)));
-  p.kt_per_seg = ceil_div(KT, nseg);
+  const int KT = ceil_div(n, KE * kbs);
+  int best = 1;
+  double best_eff = 0.0;
+  for (int nseg = 1; nseg <= std::min(KT, kSampleMaxSeg); ++nseg) {
+    const int ctas = p.nslabs * nseg, waves = ceil_div(ctas, sms), per = ceil_div(KT, nseg);
+    const double eff = (double)ctas / ((double)waves * sms) * (double)KT / ((double)per * nseg);
+    if (eff > best_eff + 1e-9) {
+      best_eff = eff;
+      best = nseg;
+    }
+  }
+  p.kt_per_seg = ceil_div(KT, best);
   p.nseg = ceil_div(KT, p.kt_per_seg);
   return p;
 }
@@ -145,7 +156,8 @@ struct Ops {
   static constexpr int KE = 128 / (int)sizeof(T);
   // sample (first block only)
   static constexpr int S_WM = (B == 16) ? 8 : 4, S_WN = (B == 16) ? 1 : 2;
-  static constexpr int S_SMEM = kSampleStages * (kSampleBM + B) * 128 + 1024;
+  static constexpr int S_KBS = (B >= 128) ? 2 : 4;   // 128-byte K boxes per pipeline stage
+  static constexpr int S_SMEM = kSampleStages * S_KBS * (kSampleBM + B) * 128 + 1024;
   // vtw: M = B, 8 consumer warps + 1 producer warp
   static constexpr int V_BN = (B * (int)sizeof(T) >= 1024) ? 64 : 128;
   static constexpr int V_WM = (B == 16) ? 1 : (B == 128 ? 4 : 2), V_WN = 8 / V_WM;
@@ -167,7 +179,7 @@ struct Ops {
 
   static cudaError_t setup() {
     cudaError_t e;
-    e = cudaFuncSetAttribute(sample_kernel<T, B, kSampleBM, S_WM, S_WN, kSampleStages>,
+    e = cudaFuncSetAttribute(sample_kernel<T, B, kSampleBM, S_WM, S_WN, kSampleStages, S_KBS>,
                              cudaFuncAttributeMaxDynamicSharedMemorySize, S_SMEM);
     if (e != cudaSuccess) return e;
     e = cudaFuncSetAttribute(vtw_sk_kernel<T, B, V_BN, kVtwBK, V_WM, V_WN, V_STAGES>,
@@ -181,7 +193,7 @@ struct Ops {
   }
   static void sample(const CUtensorMap& tmW, const CUtensorMap& tmO, void* Ypart, int r0, int rows, int n, int j0,
                      const SamplePlan& p, Ctrl* ctrl, cudaStream_t st) {
-    sample_kernel<T, B, kSampleBM, S_WM, S_WN, kSampleStages>
+    sample_kernel<T, B, kSampleBM, S_WM, S_WN, kSampleStages, S_KBS>
         <<<dim3(p.nslabs, p.nseg), S_WM * S_WN * 32, S_SMEM, st>>>(tmW, tmO, (T*)Ypart, r0, rows, n, j0, p.kt_per_seg,
                                                                      ctrl);
   }
@@ -207,7 +219,7 @@ struct Ops {
 };
 
 struct OpTable {
-  int v_bn, u_bm, u_bn, u_wn;
+  int s_kbs, v_bn, u_bm, u_bn, u_wn;
   cudaError_t (*setup)();
   void (*sample)(const CUtensorMap&, const CUtensorMap&, void*, int, int, int, int, const SamplePlan&, Ctrl*,
                  cudaStream_t);
@@ -218,7 +230,7 @@ struct OpTable {
 };
 template <typename T, int B>
 static OpTable make_ops() {
-  return OpTable{Ops<T, B>::V_BN, Ops<T, B>::U_BM, Ops<T, B>::U_BN, Ops<T, B>::U_WN, &Ops<T, B>::setup, &Ops<T, B>::sample,
+  return OpTable{Ops<T, B>::S_KBS, Ops<T, B>::V_BN, Ops<T, B>::U_BM, Ops<T, B>::U_BN, Ops<T, B>::U_WN, &Ops<T, B>::setup, &Ops<T, B>::sample,
                  &Ops<T, B>::vtw,  &Ops<T, B>::tz, &Ops<T, B>::update};
 }
 static const OpTable* get_ops(int dtype, int b) {
@@ -351,8 +363,7 @@ static bool run_layout(const rrf_params_t* p, bool need_omega, RunLayout* L) {
   int npad = 0;
   for (int i = 0; i < steps; ++i) {
     const long long rows = p->m - (long long)i * b;
-    const SamplePlan sp = plan_sample(rows, p->n, esize);
-    ymax = std::max(ymax, (size_t)sp.nseg * (size_t)rows * b);
+    ymax = std::max(ymax, (size_t)kSampleMaxSeg * (size_t)rows * b);   // first block only, any SM count
     const UpdPlan up = plan_upd(sms, rows, p->n, ops->u_bm, ops->u_bn, ops->u_wn);
     ymax = std::max(ymax, (size_t)(sms + up.NS) * ops->u_wn * ops->u_bm * b);   // slots <= (P + NS) * wn, P <= sms
     const VtwPlan vp = plan_vtw(sms, rows, p->n, ops->v_bn);
@@ -761,7 +772,7 @@ rrf_status_t rrf_run(rrf_handle_t h, const rrf_params_t* p, void* dA, int64_t ld
   // fused update of pass i.
   PanelSource src{};
   {
-    const SamplePlan sp = plan_sample(m, n, esize);
+    const SamplePlan sp = plan_sample(h->sms, m, n, esize, ops->s_kbs);
     mark(RRF_PHASE_SAMPLE, 0);
     ops->sample(tmW_s, tmO, Ypart, 0, (int)m, (int)n, 0, sp, ctrl, st);
     src.slots = 0;

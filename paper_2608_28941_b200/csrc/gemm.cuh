@@ -46,7 +46,8 @@ __device__ __forceinline__ void store2<float>(float* p, float a, float b) {
 // Y_part[seg] = W[r0 + slab*BM ..., k-range(seg)] * OmegaT[j0 .. j0+B, k-range(seg)]^T
 // grid = (row slabs, K segments); both operands K-contiguous.
 // ------------------------------------------------------------------------------------------
-template <typename T, int B, int BM, int WM, int WN, int STAGES>
+// KBS 128-byte K boxes of both operands form one pipeline stage.
+template <typename T, int B, int BM, int WM, int WN, int STAGES, int KBS>
 __global__ void __launch_bounds__(WM* WN * 32)
     sample_kernel(const __grid_constant__ CUtensorMap tmW,  // W [m][n], box [BM][KE]
                   const __grid_constant__ CUtensorMap tmO,  // OmegaT [max_rank][n], box [B][KE]
@@ -56,7 +57,7 @@ __global__ void __launch_bounds__(WM* WN * 32)
   constexpr int KE = Elem<T>::KE, NV = Elem<T>::NV, KS = Elem<T>::KS;
   constexpr int TM = BM / WM, TN = B / WN, MT = TM / 16, NT = TN / 8;
   static_assert(TM % 16 == 0 && TN % 8 == 0, "warp tile");
-  constexpr int A_BYTES = BM * 128, B_BYTES = B * 128, STAGE_BYTES = A_BYTES + B_BYTES;
+  constexpr int A_BYTES = BM * 128, B_BYTES = B * 128, STAGE_BYTES = KBS * (A_BYTES + B_BYTES);
 
   extern __shared__ unsigned char smem_raw[];
   unsigned char* smem = align1024(smem_raw);
@@ -65,7 +66,7 @@ __global__ void __launch_bounds__(WM* WN * 32)
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
   const int wm = warp / WN, wn = warp % WN;
   const int slab = blockIdx.x, seg = blockIdx.y;
-  const int KT = (n + KE - 1) / KE;
+  const int KT = (n + KBS * KE - 1) / (KBS * KE);    // K tiles of KBS boxes
   const int kt0 = seg * kt_per_seg;
   const int nkt = max(0, min(KT, kt0 + kt_per_seg) - kt0);
   const int grow0 = r0 + slab * BM;
@@ -80,8 +81,11 @@ __global__ void __launch_bounds__(WM* WN * 32)
     const int st = i % STAGES;
     unsigned char* sA = smem + st * STAGE_BYTES;
     mbar_expect_tx(&full[st], STAGE_BYTES);
-    tma_load_2d(sA, &tmW, (kt0 + i) * KE, grow0, &full[st]);
-    tma_load_2d(sA + A_BYTES, &tmO, (kt0 + i) * KE, j0, &full[st]);
+#pragma unroll
+    for (int kb = 0; kb < KBS; ++kb) {
+      tma_load_2d(sA + kb * A_BYTES, &tmW, ((kt0 + i) * KBS + kb) * KE, grow0, &full[st]);
+      tma_load_2d(sA + KBS * A_BYTES + kb * B_BYTES, &tmO, ((kt0 + i) * KBS + kb) * KE, j0, &full[st]);
+    }
   };
   if (tid == 0)
     for (int i = 0; i < STAGES - 1 && i < nkt; ++i) issue(i);
@@ -98,8 +102,10 @@ __global__ void __launch_bounds__(WM* WN * 32)
     if (tid == 0 && i + STAGES - 1 < nkt) issue(i + STAGES - 1);
     const int st = i % STAGES;
     if (!mbar_wait(&full[st], (i / STAGES) & 1, ctrl)) return;
-    const unsigned char* sA = smem + st * STAGE_BYTES;
-    const unsigned char* sB = sA + A_BYTES;
+#pragma unroll
+    for (int kb = 0; kb < KBS; ++kb) {
+    const unsigned char* sA = smem + st * STAGE_BYTES + kb * A_BYTES;
+    const unsigned char* sB = smem + st * STAGE_BYTES + KBS * A_BYTES + kb * B_BYTES;
 #pragma unroll
     for (int s2 = 0; s2 < 2; ++s2) {
       const uint32_t chunk = ((uint32_t)(2 * t + s2) ^ (uint32_t)g) << 4;
@@ -126,6 +132,7 @@ __global__ void __launch_bounds__(WM* WN * 32)
             mma16x8x8(acc[a][c], af, bf);
           }
         }
+    }
     }
     __syncthreads();  // everyone is done with stage st before it is refilled
   }
