@@ -273,10 +273,11 @@ static rrf_status_t launch_panel(rrf_ctx* h, int dtype, const void* Y, PanelSour
   cudaError_t e;
   const size_t tsmem = ((size_t)b * (b + 1) + (size_t)(b / 2) * (b / 2 + 1)) * sizeof(double);
   mark(RRF_PHASE_PANEL, step);
-  const bool small = pp.R <= 128;
+  // rows per lane kept in registers: the smallest of 2, 4, 7 that covers the slab
+  const int qsel = pp.R <= 64 ? 0 : (pp.R <= 128 ? 1 : 2);
   if (dtype == RRF_F64) {
-    e = cudaLaunchCooperativeKernel(small ? (void*)panel_kernel<double, 4> : (void*)panel_kernel<double, 7>, dim3(pp.G),
-                                    dim3(kPanelThreads), args, pp.smem, st);
+    void* const fn[3] = {(void*)panel_kernel<double, 2>, (void*)panel_kernel<double, 4>, (void*)panel_kernel<double, 7>};
+    e = cudaLaunchCooperativeKernel(fn[qsel], dim3(pp.G), dim3(kPanelThreads), args, pp.smem, st);
     if (e == cudaSuccess) {
       cudaStream_t tt = st;
       if (ev_fork != nullptr) {          // fork: the T factor runs on the side stream after the panel
@@ -291,8 +292,8 @@ static rrf_status_t launch_panel(rrf_ctx* h, int dtype, const void* Y, PanelSour
       if (ev_join != nullptr) cudaEventRecord(ev_join, st_t);
     }
   } else {
-    e = cudaLaunchCooperativeKernel(small ? (void*)panel_kernel<float, 4> : (void*)panel_kernel<float, 7>, dim3(pp.G),
-                                    dim3(kPanelThreads), args, pp.smem, st);
+    void* const fn[3] = {(void*)panel_kernel<float, 2>, (void*)panel_kernel<float, 4>, (void*)panel_kernel<float, 7>};
+    e = cudaLaunchCooperativeKernel(fn[qsel], dim3(pp.G), dim3(kPanelThreads), args, pp.smem, st);
     if (e == cudaSuccess) {
       cudaStream_t tt = st;
       if (ev_fork != nullptr) {
@@ -324,8 +325,9 @@ static cudaError_t setup_all(int smem_optin, int* panel_smem_max) {
     e = get_ops(RRF_F32, b)->setup();
     if (e != cudaSuccess) return e;
   }
-  const void* pk[4] = {(const void*)panel_kernel<double, 4>, (const void*)panel_kernel<double, 7>,
-                       (const void*)panel_kernel<float, 4>, (const void*)panel_kernel<float, 7>};
+  const void* pk[6] = {(const void*)panel_kernel<double, 2>, (const void*)panel_kernel<double, 4>,
+                       (const void*)panel_kernel<double, 7>, (const void*)panel_kernel<float, 2>,
+                       (const void*)panel_kernel<float, 4>,  (const void*)panel_kernel<float, 7>};
   size_t stat = 0;
   for (const void* f : pk) {
     cudaFuncAttributes fa;
@@ -878,8 +880,9 @@ static cudaError_t static_setup(int dev, StaticDevice* sd) {
   if (e != cudaSuccess) return e;
   e = cudaDeviceGetAttribute(&smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
   if (e != cudaSuccess) return e;
-  const void* pk[4] = {(const void*)panel_kernel<double, 4>, (const void*)panel_kernel<double, 7>,
-                       (const void*)panel_kernel<float, 4>, (const void*)panel_kernel<float, 7>};
+  const void* pk[6] = {(const void*)panel_kernel<double, 2>, (const void*)panel_kernel<double, 4>,
+                       (const void*)panel_kernel<double, 7>, (const void*)panel_kernel<float, 2>,
+                       (const void*)panel_kernel<float, 4>,  (const void*)panel_kernel<float, 7>};
   size_t stat = 0;
   for (const void* f : pk) {
     cudaFuncAttributes fa;

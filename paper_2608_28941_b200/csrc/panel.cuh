@@ -8,8 +8,8 @@ namespace rrf {
 
 constexpr int kPanelThreads = 512;
 constexpr int kPanelMaxG = 160;   // most CTAs a panel grid may have (one per SM)
-// doubles of shared memory the panel kernel needs besides the slab: w[b], p[b], pivot_row[b]
-__host__ __device__ constexpr int panel_extra_doubles(int b) { return 3 * b; }
+// doubles of shared memory the panel kernel needs besides the slab: w[b], p[b], pivot_row[b], scalars
+__host__ __device__ constexpr int panel_extra_doubles(int b) { return 3 * b + 4; }
 
 // Grid-wide barrier over a monotonically increasing arrival counter.  Needs all CTAs
 // co-resident (cooperative launch).  Bounded: gives up after kWaitLimitClocks.
@@ -38,6 +38,25 @@ __device__ __forceinline__ bool grid_barrier(unsigned* ctr, unsigned target, Ctr
   return ok_s != 0;
 }
 
+// Sums four per-lane values over the warp with 6 adds and 6 shuffles instead of 20: after the
+// exchanges with lanes ^16 and ^8 every lane carries one of the four sums (number 2*bit4 + bit3 of
+// its lane index), which three more butterfly steps complete.  Fixed order, so reproducible.
+__device__ __forceinline__ double warp_sum4(const double (&v)[4], int lane) {
+  const bool hi = lane & 16;
+  double a0 = hi ? v[2] : v[0], a1 = hi ? v[3] : v[1];
+  const double s0 = hi ? v[0] : v[2], s1 = hi ? v[1] : v[3];
+  a0 += __shfl_xor_sync(0xffffffffu, s0, 16);
+  a1 += __shfl_xor_sync(0xffffffffu, s1, 16);
+  const bool mid = lane & 8;
+  double k = mid ? a1 : a0;
+  const double snd = mid ? a0 : a1;
+  k += __shfl_xor_sync(0xffffffffu, snd, 8);
+  k += __shfl_xor_sync(0xffffffffu, k, 4);
+  k += __shfl_xor_sync(0xffffffffu, k, 2);
+  k += __shfl_xor_sync(0xffffffffu, k, 1);
+  return k;
+}
+
 // Self test of the bounded wait: one CTA arrives at a barrier that expects two.
 __global__ void __launch_bounds__(32) timeout_selftest_kernel(unsigned* ctr, Ctrl* ctrl, long long limit) {
   grid_barrier(ctr, 2u, ctrl, limit);
@@ -50,7 +69,7 @@ __global__ void __launch_bounds__(32) timeout_selftest_kernel(unsigned* ctr, Ctr
 // H_{j-1} and accumulates p[c] = sum_{row > j} Y[row, j] * X[row, c] for every column c, where
 // X[:, c] is the finished vector v_c for c < j and the current Y[:, c] for c >= j.  After the
 // barrier every CTA sums the per-CTA partials in CTA order and derives, with alpha = Y[j, j]:
-//   beta = -sign(alpha) sqrt(alpha^2 + p[j]),  tau = (beta - alpha)/beta,  v = Y[j+1:, j]/(alpha - beta)
+//   beta = -sign(alpha) sqrt(alpha^2 + p[j]),  tau = (beta - alpha)/beta,  v = Y[j+1:, j] * (1/(alpha - beta))
 //   w[c] = v^T Y[:, c]   = Y[j, c] + p[c]/(alpha - beta)           (c > j: needed by H_j)
 //   g[c] = v_c^T v_j     = v_c[j] + p[c]/(alpha - beta)           (c < j: row j of V^T V, for T)
 // so norms, reflector application and the Gram matrix for T share one reduction.
@@ -100,6 +119,7 @@ __global__ void __launch_bounds__(kPanelThreads)
   double* w_s = S + (size_t)b * Rp;       // [b]
   double* p_s = w_s + b;                  // [b]
   double* pr_s = p_s + b;                 // [b]
+  double* sc_s = pr_s + b;                // [4]: tau_j, 1/(alpha - beta)
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   constexpr int NW = kPanelThreads / 32;
@@ -171,14 +191,10 @@ __global__ void __launch_bounds__(kPanelThreads)
           }
           acc[u] = a;
         }
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1)
-#pragma unroll
-          for (int u = 0; u < CG; ++u) acc[u] += __shfl_xor_sync(0xffffffffu, acc[u], o);
-        if (lane == 0) {
-#pragma unroll
-          for (int u = 0; u < CG; ++u)
-            if (c0 + u * NW < b) p_s[c0 + u * NW] = acc[u];
+        {
+          const double tot = warp_sum4(acc, lane);
+          const int u = ((lane >> 4) << 1) | ((lane >> 3) & 1);
+          if ((lane & 7) == 0 && c0 + u * NW < b) p_s[c0 + u * NW] = tot;
         }
       }
     }
@@ -211,36 +227,43 @@ __global__ void __launch_bounds__(kPanelThreads)
 #pragma unroll
           for (int q = 0; q < kPanelMaxG / 32; ++q) sacc[u] += v[u][q];
         }
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1)
-#pragma unroll
-          for (int u = 0; u < CG; ++u) sacc[u] += __shfl_xor_sync(0xffffffffu, sacc[u], o);
-        if (lane == 0) {
-#pragma unroll
-          for (int u = 0; u < CG; ++u)
-            if (c0 + u * NW < b) p_s[c0 + u * NW] = sacc[u];
+        {
+          const double tot = warp_sum4(sacc, lane);
+          const int u = ((lane >> 4) << 1) | ((lane >> 3) & 1);
+          if ((lane & 7) == 0 && c0 + u * NW < b) p_s[c0 + u * NW] = tot;
         }
       }
       if (tid < b) pr_s[tid] = prv;
       __syncthreads();
     }
-    const double alpha = pr_s[j], s2 = p_s[j];
-    double tau = 0.0, denom = 1.0;
-    if (s2 != 0.0) {
-      const double beta = -copysign(sqrt(alpha * alpha + s2), alpha);
-      tau = (beta - alpha) / beta;
-      denom = alpha - beta;
+    // The reflector's scalars are computed once (square root and divisions are long FP64 sequences
+    // and the SM has few FP64 lanes) and shared: tau, 1/(alpha - beta), and whether there is
+    // anything to annihilate.
+    if (warp == 0) {
+      const double alpha = pr_s[j], s2 = p_s[j];
+      double tau = 0.0, rdenom = 0.0;
+      if (s2 != 0.0) {
+        const double beta = -copysign(sqrt(alpha * alpha + s2), alpha);
+        tau = (beta - alpha) / beta;
+        rdenom = 1.0 / (alpha - beta);
+      }
+      if (lane == 0) {
+        sc_s[0] = tau;
+        sc_s[1] = rdenom;
+        if (cta == 0) tau_out[j] = tau;
+      }
     }
+    __syncthreads();
+    const double tau = sc_s[0], rdenom = sc_s[1];     // rdenom == 0 marks H_j = I
     if (tid < b && tid != j) {
-      const double wv = (s2 != 0.0) ? pr_s[tid] + p_s[tid] / denom : pr_s[tid];
+      const double wv = pr_s[tid] + p_s[tid] * rdenom;
       w_s[tid] = wv;
       if (cta == 0 && tid < j) gram[(size_t)j * b + tid] = wv;
     }
-    if (cta == 0 && tid == 0) tau_out[j] = tau;
     // column j becomes v_j (unit lower trapezoidal, explicit ones and zeros)
     for (int r = tid; r < nloc; r += kPanelThreads) {
       const int grow = gr0 + r;
-      Sj[r] = grow > j ? (s2 != 0.0 ? Sj[r] / denom : 0.0) : (grow == j ? 1.0 : 0.0);
+      Sj[r] = grow > j ? Sj[r] * rdenom : (grow == j ? 1.0 : 0.0);
     }
     tau_prev = tau;
     __syncthreads();
