@@ -195,6 +195,8 @@ def main():
     ap.add_argument("--max-rank", type=int, default=0, help="override the workload's rank cap")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--schedule", default="auto", choices=["auto", "one", "two"],
+                    help="one queue (sequential), two queues (look-ahead), or the library's own rule")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 0)
 
@@ -236,8 +238,10 @@ def main():
     T = torch.empty((w.b, w.max_rank), dtype=tdt, device=dev)
     B = torch.empty((w.max_rank, w.n), dtype=tdt, device=dev)
 
+    sched = {"auto": 0, "one": rrf.RRF_FLAG_ONE_QUEUE, "two": rrf.RRF_FLAG_TWO_QUEUES}[args.schedule]
+
     def step():
-        return rrf.rrf_run(h, A, w.b, w.tol, w.max_rank, omegaT=OmT, V=V, T=T, B=B, workspace=ws)
+        return rrf.rrf_run(h, A, w.b, w.tol, w.max_rank, omegaT=OmT, V=V, T=T, B=B, workspace=ws, flags=sched)
 
     def barrier():
         torch.cuda.synchronize()
@@ -266,7 +270,8 @@ def main():
     ms_step = max_over_ranks(e0.elapsed_time(e1), world, dev) / args.steps
     flops = method_flops(w.m, w.n, w.b, res.steps)
     value = job_tflops(flops, world, ms_step)
-    launches_per_run = 3 + 6 * (w.max_rank // w.b)   # init x2, first sample; panel, T, VtW, TZ, update, stop per pass
+    # init x2, first sample (two with look-ahead); panel, T, VtW, TZ, update, stop per pass
+    launches_per_run = 3 + (1 if res.queues == 2 else 0) + 6 * (w.max_rank // w.b)
 
     # ---- end to end through the C ABI with host buffers
     e2e = None
@@ -283,7 +288,7 @@ def main():
         def e2e_step():
             A_d.copy_(A_h, non_blocking=True)
             O_d.copy_(O_h, non_blocking=True)
-            r = rrf.rrf_run(h, A_d, w.b, w.tol, w.max_rank, omegaT=O_d, V=V, T=T, B=B, workspace=ws)
+            r = rrf.rrf_run(h, A_d, w.b, w.tol, w.max_rank, omegaT=O_d, V=V, T=T, B=B, workspace=ws, flags=sched)
             B_h[:r.k].copy_(B[:r.k], non_blocking=True)
             V_h[:, :r.k].copy_(V[:, :r.k], non_blocking=True)
             T_h[:, :r.k].copy_(T[:, :r.k], non_blocking=True)
@@ -362,6 +367,7 @@ def main():
                 "config": {"workload": w.name, "m": w.m, "n": w.n, "b": w.b, "tol": w.tol, "max_rank": w.max_rank,
                            "k": res.k, "block_steps": res.steps, "status": res.status,
                            "l2": "inputs larger than L2 (A is %.0f MB)" % (w.m * w.n * esize / 1e6),
+                           "queues": res.queues, "panel_ctas": res.panel_ctas,
                            "parallelism": "replicas only" if world > 1 else "single GPU"},
                 "clocks": clocks, "e2e": e2e, "gpu_launches": args.steps * launches_per_run,
                 "roofline": roofline, "cpu_baseline": cpu}

@@ -51,6 +51,9 @@ typedef enum {
 /* Flags for rrf_params_t.flags */
 #define RRF_FLAG_INPLACE 1u     /* A itself is the working matrix (it is overwritten) */
 #define RRF_FLAG_FIXED_RANK 2u  /* ignore the tolerance, always run to max_rank (fixed-rank mode) */
+#define RRF_FLAG_ONE_QUEUE 4u   /* force the sequential schedule: panel, V^T W, update one after the other */
+#define RRF_FLAG_TWO_QUEUES 8u  /* use the look-ahead schedule whenever the panel can be confined to a few SMs,
+                                   also where the built-in rule would pick the sequential one */
 
 typedef struct {
   int32_t dtype;            /* rrf_dtype_t: element type of A, Omega, V, T, B, Q */
@@ -74,6 +77,9 @@ typedef struct {
   double sigma2;            /* squared absolute tolerance the loop compared against */
   double E_sub;             /* final value of Algorithm 2's E = ||A||_F^2 - sum ||B_i||_F^2 */
   double E_dir;             /* final ||W[k:, :]||_F^2 = ||A - Q B||_F^2 */
+  int32_t queues;           /* schedule used: 1 = sequential, 2 = look-ahead (panel QR of the next block runs
+                               beside the update of the current one) */
+  int32_t panel_ctas;       /* look-ahead: SMs the panel kernel was confined to; sequential: 0 */
 } rrf_result_t;
 
 /* Create / destroy a context bound to one CUDA device.  rrf_create makes `device`

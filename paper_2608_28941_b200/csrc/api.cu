@@ -17,7 +17,6 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
 constexpr int kMaxSmem = 232448;   // 227 KB opt-in dynamic shared memory per CTA on sm_100
-constexpr int kTargetCtas = 296;   // split-K until about two CTAs per SM exist
 constexpr int kMaxSms = kPanelMaxG;       // workspace sizes are bounds for devices with up to this many SMs
 
 }  // namespace rrf
@@ -95,26 +94,69 @@ static UpdPlan plan_upd(int sms, long long rows, long long ncols, int bm, int bn
   p.slots = (p.P + p.NS) * wn;
   return p;
 }
-struct PanelPlan { int G, R, Rp; size_t smem; };
-static bool plan_panel(const rrf_ctx* h, long long rows, int b, PanelPlan* p) {
+// The panel kernel's variants: rows a lane keeps in registers, row groups, and whether the slab is
+// allocated at its full height (32 * rows per lane * groups, zero filled) or exactly (the fallback for
+// the one shape that only fits unpadded).
+constexpr int kPanelVariants = 6;
+static const int kVariantRows[kPanelVariants] = {64, 128, 224, 320, 512, 224};
+static const bool kVariantPad[kPanelVariants] = {true, true, true, true, true, false};
+template <typename T>
+static const void* panel_variant(int q) {
+  switch (q) {
+    case 0: return (const void*)panel_kernel<T, 2, 1>;
+    case 1: return (const void*)panel_kernel<T, 4, 1>;
+    case 2: return (const void*)panel_kernel<T, 7, 1>;
+    case 3: return (const void*)panel_kernel<T, 5, 2>;
+    case 4: return (const void*)panel_kernel<T, 8, 2>;
+    default: return (const void*)panel_kernel<T, 7, 1, false>;
+  }
+}
+struct PanelPlan { int G, R, Rp, variant; size_t smem; };
+// ctas == 0: the panel is spread over every SM (short slabs, short passes).  ctas > 0: the panel is
+// confined to that many CTAs so that the other SMs stay free for the GEMM kernels of the look-ahead
+// schedule; `fix` adds the b rows above the panel and the shared memory of the late reflector
+// application.
+static bool plan_panel(const rrf_ctx* h, long long rows, int b, PanelPlan* p, int ctas = 0, bool fix = false) {
+  if (fix && b > 64) return false;
+  const long long ext = rows + (fix ? b : 0);
   // tall slabs keep the grid, and with it the all-to-all read of the partial sums, small
-  int R = std::max(64, ceil_div(rows, h->sms));
+  const int R = std::max(64, ceil_div(ext, ctas > 0 ? ctas : h->sms));
   p->R = R;
-  p->G = ceil_div(rows, R);
-  if (R > 7 * 32) return false;   // a lane keeps at most seven rows of a column in registers
-  // odd pitch keeps the transposing load/store phases bank-conflict free; the tallest panels
-  // (config 5: 222 rows x 128 columns per CTA) only fit without the padding
-  for (int Rp : {R | 1, R}) {
-    p->Rp = Rp;
-    p->smem = ((size_t)b * Rp + panel_extra_doubles(b)) * sizeof(double);
-    if (p->smem <= (size_t)h->panel_smem_max) return p->G <= h->sms;
+  p->G = ceil_div(ext, R);
+  if (p->G > h->sms) return false;
+  const size_t extra = (size_t)panel_extra_doubles(b) + (fix ? panel_fix_doubles(b) : 0);
+  for (int q = 0; q < kPanelVariants; ++q) {
+    if (R > kVariantRows[q]) continue;
+    if (kVariantPad[q]) {
+      p->Rp = kVariantRows[q] + 1;          // odd pitch: the transposing load/store phases stay conflict free
+    } else {
+      if (fix) continue;
+      p->Rp = ((size_t)b * (R | 1) + extra) * sizeof(double) <= (size_t)h->panel_smem_max ? (R | 1) : R;
+    }
+    p->variant = q;
+    p->smem = ((size_t)b * p->Rp + extra) * sizeof(double);
+    if (p->smem <= (size_t)h->panel_smem_max) return true;
   }
   return false;
+}
+// Fewest CTAs whose shared memory holds a rows x b panel with the fix-up staging; 0 if none.
+static int panel_min_ctas(const rrf_ctx* h, long long rows, int b) {
+  if (b > 64) return 0;
+  const size_t extra = (size_t)panel_extra_doubles(b) + panel_fix_doubles(b);
+  int best = 0;
+  for (int q = 0; q < kPanelVariants; ++q)
+    if (kVariantPad[q] && ((size_t)b * (kVariantRows[q] + 1) + extra) * sizeof(double) <= (size_t)h->panel_smem_max)
+      best = std::max(best, kVariantRows[q]);
+  return best > 0 ? ceil_div(rows + b, best) : 0;
 }
 static size_t panel_scratch_bytes(int sms, int b) {
   // P[2][b][Gp] + piv[2][b] + gram[b][b] + tau[b] (+ barrier word, padded)
   const int gp = (sms + 31) / 32 * 32;
   return align_up(((size_t)2 * gp * b + 2 * (size_t)b + (size_t)b * b + b) * sizeof(double) + 256, 256);
+}
+constexpr int kLookMaxCtas = 40;   // most CTAs a confined panel may take
+static size_t look_scratch_bytes(int b) {   // Gpart[kLookMaxCtas][b*b] + M[b*b]
+  return align_up((size_t)(kLookMaxCtas + 1) * b * b * sizeof(double), 256);
 }
 struct PanelScratch { double *P, *piv, *gram, *tau; unsigned* bar; };
 static PanelScratch carve_panel(unsigned char* base, int sms, int b) {
@@ -258,55 +300,44 @@ static const OpTable* get_ops(int dtype, int b) {
 struct NoMark {
   void operator()(int, int) const {}
 };
+struct PanelOpts {
+  PanelFix fix{};                  // look-ahead fix-up (enabled == 0: none)
+  int ctas = 0;                    // 0: one slab per SM; > 0: confine the panel to this many CTAs
+  unsigned* bar_reset = nullptr;   // the T-factor kernel zeroes this word (the panel's barrier counter)
+  cudaStream_t st_t = nullptr;     // side stream for the T factor, with its fork / join events
+  cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
+};
 template <typename Mark = NoMark>
 static rrf_status_t launch_panel(rrf_ctx* h, int dtype, const void* Y, PanelSource src,
                                  long long rows, int b, void* V, long long ldv, void* Tout, long long ldt,
                                  const PanelScratch& ps, Ctrl* ctrl, const int* done_flag, cudaStream_t st,
-                                 Mark mark = Mark(), int step = 0, cudaStream_t st_t = nullptr,
-                                 cudaEvent_t ev_fork = nullptr, cudaEvent_t ev_join = nullptr) {
+                                 Mark mark = Mark(), int step = 0, const PanelOpts& o = PanelOpts()) {
   PanelPlan pp;
-  if (!plan_panel(h, rows, b, &pp)) return RRF_ERR_WORKSPACE;
+  if (!plan_panel(h, rows, b, &pp, o.ctas, o.fix.enabled != 0)) return RRF_ERR_WORKSPACE;
   int rows_i = (int)rows, R = pp.R, Rp = pp.Rp;
   double *P = ps.P, *piv = ps.piv, *gram = ps.gram, *tau = ps.tau;
   unsigned* bar = ps.bar;
-  void* args[] = {&Y, &src, &rows_i, &b, &R, &Rp, &V, &ldv, &P, &piv, &gram, &tau, &bar, &ctrl, &done_flag};
-  cudaError_t e;
+  PanelFix fix = o.fix;
+  void* args[] = {&Y, &src, &rows_i, &b, &R, &Rp, &V, &ldv, &P, &piv, &gram, &tau, &bar, &ctrl, &done_flag, &fix};
   const size_t tsmem = ((size_t)b * (b + 1) + (size_t)(b / 2) * (b / 2 + 1)) * sizeof(double);
   mark(RRF_PHASE_PANEL, step);
-  // rows per lane kept in registers: the smallest of 2, 4, 7 that covers the slab
-  const int qsel = pp.R <= 64 ? 0 : (pp.R <= 128 ? 1 : 2);
-  if (dtype == RRF_F64) {
-    void* const fn[3] = {(void*)panel_kernel<double, 2>, (void*)panel_kernel<double, 4>, (void*)panel_kernel<double, 7>};
-    e = cudaLaunchCooperativeKernel(fn[qsel], dim3(pp.G), dim3(kPanelThreads), args, pp.smem, st);
-    if (e == cudaSuccess) {
-      cudaStream_t tt = st;
-      if (ev_fork != nullptr) {          // fork: the T factor runs on the side stream after the panel
-        cudaEventRecord(ev_fork, st);
-        cudaStreamWaitEvent(st_t, ev_fork, 0);
-        tt = st_t;
-      } else {
-        mark(RRF_PHASE_TFACTOR, step);
-      }
-      tfactor_kernel<double><<<1, 256, tsmem, tt>>>(gram, tau, b, (double*)Tout, ldt, done_flag);
-      e = cudaGetLastError();
-      if (ev_join != nullptr) cudaEventRecord(ev_join, st_t);
+  const void* fn = dtype == RRF_F64 ? panel_variant<double>(pp.variant) : panel_variant<float>(pp.variant);
+  cudaError_t e = cudaLaunchCooperativeKernel(fn, dim3(pp.G), dim3(kPanelThreads), args, pp.smem, st);
+  if (e == cudaSuccess) {
+    cudaStream_t tt = st;
+    if (o.ev_fork != nullptr) {          // fork: the T factor runs on the side stream after the panel
+      cudaEventRecord(o.ev_fork, st);
+      cudaStreamWaitEvent(o.st_t, o.ev_fork, 0);
+      tt = o.st_t;
+    } else {
+      mark(RRF_PHASE_TFACTOR, step);
     }
-  } else {
-    void* const fn[3] = {(void*)panel_kernel<float, 2>, (void*)panel_kernel<float, 4>, (void*)panel_kernel<float, 7>};
-    e = cudaLaunchCooperativeKernel(fn[qsel], dim3(pp.G), dim3(kPanelThreads), args, pp.smem, st);
-    if (e == cudaSuccess) {
-      cudaStream_t tt = st;
-      if (ev_fork != nullptr) {
-        cudaEventRecord(ev_fork, st);
-        cudaStreamWaitEvent(st_t, ev_fork, 0);
-        tt = st_t;
-      } else {
-        mark(RRF_PHASE_TFACTOR, step);
-      }
-      tfactor_kernel<float><<<1, 256, tsmem, tt>>>(gram, tau, b, (float*)Tout, ldt, done_flag);
-      e = cudaGetLastError();
-      if (ev_join != nullptr) cudaEventRecord(ev_join, st_t);
-    }
+    if (dtype == RRF_F64)
+      tfactor_kernel<double><<<1, 256, tsmem, tt>>>(gram, tau, b, (double*)Tout, ldt, done_flag, o.bar_reset);
+    else
+      tfactor_kernel<float><<<1, 256, tsmem, tt>>>(gram, tau, b, (float*)Tout, ldt, done_flag, o.bar_reset);
+    e = cudaGetLastError();
+    if (o.ev_join != nullptr) cudaEventRecord(o.ev_join, o.st_t);
   }
   if (e != cudaSuccess) {
     h->last_cuda = (int)e;
@@ -315,19 +346,14 @@ static rrf_status_t launch_panel(rrf_ctx* h, int dtype, const void* Y, PanelSour
   return RRF_OK;
 }
 
-static cudaError_t setup_all(int smem_optin, int* panel_smem_max) {
+// attributes of the panel and T-factor kernels; reports the dynamic shared memory a panel may use
+static cudaError_t setup_panel_kernels(int smem_optin, int* panel_smem_max) {
   cudaError_t e;
-  for (int b : {16, 32, 64, 128}) {
-    e = get_ops(RRF_F64, b)->setup();
-    if (e != cudaSuccess) return e;
+  const void* pk[2 * kPanelVariants];
+  for (int q = 0; q < kPanelVariants; ++q) {
+    pk[q] = panel_variant<double>(q);
+    pk[kPanelVariants + q] = panel_variant<float>(q);
   }
-  for (int b : {32, 64, 128}) {
-    e = get_ops(RRF_F32, b)->setup();
-    if (e != cudaSuccess) return e;
-  }
-  const void* pk[6] = {(const void*)panel_kernel<double, 2>, (const void*)panel_kernel<double, 4>,
-                       (const void*)panel_kernel<double, 7>, (const void*)panel_kernel<float, 2>,
-                       (const void*)panel_kernel<float, 4>,  (const void*)panel_kernel<float, 7>};
   size_t stat = 0;
   for (const void* f : pk) {
     cudaFuncAttributes fa;
@@ -343,14 +369,25 @@ static cudaError_t setup_all(int smem_optin, int* panel_smem_max) {
   const int tmax = (128 * 129 + 64 * 65) * 8;
   e = cudaFuncSetAttribute(tfactor_kernel<double>, cudaFuncAttributeMaxDynamicSharedMemorySize, tmax);
   if (e != cudaSuccess) return e;
-  e = cudaFuncSetAttribute(tfactor_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, tmax);
-  if (e != cudaSuccess) return e;
-  return e;
+  return cudaFuncSetAttribute(tfactor_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, tmax);
+}
+
+static cudaError_t setup_all(int smem_optin, int* panel_smem_max) {
+  cudaError_t e;
+  for (int b : {16, 32, 64, 128}) {
+    e = get_ops(RRF_F64, b)->setup();
+    if (e != cudaSuccess) return e;
+  }
+  for (int b : {32, 64, 128}) {
+    e = get_ops(RRF_F32, b)->setup();
+    if (e != cudaSuccess) return e;
+  }
+  return setup_panel_kernels(smem_optin, panel_smem_max);
 }
 
 // ------------------------------------------------------------------ workspace of rrf_run
 struct RunLayout {
-  size_t ctrl, traces, norm_part, init_part, ypart, zpart, zt, panel, w, omega, total;
+  size_t ctrl, traces, done_after, norm_part, init_part, ypart, ypart2, zpart, zt, panel, look, w, omega, total;
   int init_ctas, max_norm_parts;
   long long ldw;
 };
@@ -375,14 +412,17 @@ static bool run_layout(const rrf_params_t* p, bool need_omega, RunLayout* L) {
   size_t off = 0;
   L->ctrl = off; off += 256;
   L->traces = off; off += align_up((size_t)2 * steps * sizeof(double), 256);
+  L->done_after = off; off += align_up((size_t)(steps + 2) * sizeof(int), 256);   // + the look-ahead barrier word
   L->init_ctas = kInitCtas;
   L->init_part = off; off += align_up((size_t)kInitCtas * sizeof(double), 256);
   L->max_norm_parts = sms;
   L->norm_part = off; off += align_up((size_t)2 * sms * sizeof(double), 256);
   L->ypart = off; off += align_up(ymax * esize, 256);
+  L->ypart2 = off; off += align_up(ymax * esize, 256);   // the look-ahead schedule keeps two sampled panels
   L->zpart = off; off += align_up(zmax * esize, 256);
   L->zt = off; off += align_up((size_t)npad * b * esize, 256);
   L->panel = off; off += panel_scratch_bytes(sms, b);
+  L->look = off; off += look_scratch_bytes(b);
   L->w = off;
   L->ldw = (long long)align_up((size_t)p->n, 16);   // rows of the working copy start on 128-byte lines
   if (!(p->flags & RRF_FLAG_INPLACE)) off += align_up((size_t)p->m * (size_t)L->ldw * esize, 256);
@@ -696,8 +736,20 @@ rrf_status_t rrf_run(rrf_handle_t h, const rrf_params_t* p, void* dA, int64_t ld
   RunLayout L;
   run_layout(p, dOmegaT == nullptr, &L);
   if (workspace_bytes < L.total) return fail(RRF_ERR_WORKSPACE);
+  // Schedule.  Two queues (look-ahead) when the tallest panel fits in the shared memory of a small
+  // share of the SMs, so that confining the panel there costs the GEMM kernels little; else one queue.
+  const int steps_total = p->max_rank / b;
+  int look_ctas = 0;
+  if (!(p->flags & RRF_FLAG_ONE_QUEUE) && steps_total >= 2) {
+    const int fewest = panel_min_ctas(h, m, b);
+    int want = std::max(fewest, h->sms / 9);
+    if (const char* ev = std::getenv("RRF_LOOKAHEAD_CTAS")) want = std::max(fewest, std::atoi(ev));
+    const int cap = (p->flags & RRF_FLAG_TWO_QUEUES) ? kLookMaxCtas : std::min(kLookMaxCtas, h->sms / 5);
+    PanelPlan ppl;
+    if (fewest > 0 && want <= cap && want < h->sms && plan_panel(h, m, b, &ppl, want, true)) look_ctas = want;
+  }
   PanelPlan pp0;
-  if (!plan_panel(h, m, b, &pp0)) return fail(RRF_ERR_WORKSPACE);   // first (tallest) panel must fit on chip
+  if (look_ctas == 0 && !plan_panel(h, m, b, &pp0)) return fail(RRF_ERR_WORKSPACE);   // tallest panel must fit on chip
 
   cudaStream_t st = (cudaStream_t)cuda_stream;
   if (cudaSetDevice(h->device) != cudaSuccess) return fail(RRF_ERR_CUDA);
@@ -706,6 +758,9 @@ rrf_status_t rrf_run(rrf_handle_t h, const rrf_params_t* p, void* dA, int64_t ld
   const int steps = p->max_rank / b;
   double* tr_sub = reinterpret_cast<double*>(ws + L.traces);
   double* tr_dir = tr_sub + steps;
+  int* done_after = reinterpret_cast<int*>(ws + L.done_after);
+  unsigned* look_bar = reinterpret_cast<unsigned*>(done_after + steps + 1);
+  double* look_G = reinterpret_cast<double*>(ws + L.look);
   double* init_part = reinterpret_cast<double*>(ws + L.init_part);
   double* norm_part = reinterpret_cast<double*>(ws + L.norm_part);
   void* Ypart = ws + L.ypart;
@@ -713,6 +768,8 @@ rrf_status_t rrf_run(rrf_handle_t h, const rrf_params_t* p, void* dA, int64_t ld
   void* Zt = ws + L.zt;
   PanelScratch ps = carve_panel(ws + L.panel, h->sms, b);
   ps.bar = &ctrl->bar;
+  if (look_ctas > 0 && cudaMemsetAsync(look_bar, 0, sizeof(unsigned), (cudaStream_t)cuda_stream) != cudaSuccess)
+    return fail(RRF_ERR_CUDA);
   const bool inplace = (p->flags & RRF_FLAG_INPLACE) != 0;
   const bool fixed = (p->flags & RRF_FLAG_FIXED_RANK) != 0;
   void* W = inplace ? dA : (void*)(ws + L.w);
@@ -760,57 +817,141 @@ rrf_status_t rrf_run(rrf_handle_t h, const rrf_params_t* p, void* dA, int64_t ld
     init_kernel<float><<<L.init_ctas, 256, 0, st>>>((const float*)dA, lda, inplace ? nullptr : (float*)W, ldw, m, n,
                                                     (float*)dV, ldv, p->max_rank, init_part);
   init_ctrl_kernel<<<1, 256, 0, st>>>(init_part, L.init_ctas, p->tol, p->tol_is_relative, fixed ? 1 : 0, b, p->max_rank,
-                                      ctrl);
+                                      ctrl, done_after, steps);
 
-  // fork/join events for the side stream (two per pass), created once and kept in the handle
-  while (h->sync_events.size() < (size_t)2 * steps) {
+  // fork/join events for the side stream, created once and kept in the handle
+  while (h->sync_events.size() < (size_t)2 * steps + 1) {
     cudaEvent_t ev;
     if (cudaEventCreateWithFlags(&ev, cudaEventDisableTiming) != cudaSuccess) return fail(RRF_ERR_CUDA);
     h->sync_events.push_back(ev);
   }
 
   // Algorithm 2 lines 5-11: every pass is enqueued; passes after the stop return at once.
-  // The panel of pass 0 is sampled by its own kernel; the panel of pass i+1 comes out of the
-  // fused update of pass i.
+  auto panel_failed = [&](rrf_status_t ps_status) {
+    out->cuda_error = h->last_cuda;
+    cudaStreamSynchronize(st);
+    cudaStreamSynchronize(h->aux);
+    return fail(ps_status);
+  };
+  void* const V0 = dV;
+  auto Vblk = [&](int r0) { return (void*)((char*)V0 + ((size_t)r0 * ldv + r0) * esize); };
+  auto Tblk = [&](int r0) { return (void*)((char*)dT + (size_t)r0 * esize); };
+  const SamplePlan sp = plan_sample(h->sms, m, n, esize, ops->s_kbs);
   PanelSource src{};
-  {
-    const SamplePlan sp = plan_sample(h->sms, m, n, esize, ops->s_kbs);
-    mark(RRF_PHASE_SAMPLE, 0);
-    ops->sample(tmW_s, tmO, Ypart, 0, (int)m, (int)n, 0, sp, ctrl, st);
-    src.slots = 0;
-    src.nseg = sp.nseg;
-    src.seg_stride = m * b;
-    src.ldy = b;
-  }
-  for (int i = 0; i < steps; ++i) {
-    const int r0 = i * b, rows = (int)(m - r0);
-    s = launch_panel(h, p->dtype, Ypart, src, rows, b, (char*)dV + ((size_t)r0 * ldv + r0) * esize, ldv,
-                     (char*)dT + (size_t)r0 * esize, p->max_rank, ps, ctrl, &ctrl->done, st, mark, i, h->aux,
-                     h->sync_events[2 * i], h->sync_events[2 * i + 1]);
-    if (s != RRF_OK) {
-      out->cuda_error = h->last_cuda;
-      cudaStreamSynchronize(st);
-      return fail(s);
+  src.slots = 0;
+  src.nseg = sp.nseg;
+  src.seg_stride = m * b;
+  src.ldy = b;
+  src.row_off = 0;
+  mark(RRF_PHASE_SAMPLE, 0);
+  ops->sample(tmW_s, tmO, Ypart, 0, (int)m, (int)n, 0, sp, ctrl, st);
+
+  if (look_ctas == 0) {
+    // One queue.  The panel of pass 0 is sampled by its own kernel; the panel of pass i+1 comes out
+    // of the fused update of pass i.
+    for (int i = 0; i < steps; ++i) {
+      const int r0 = i * b, rows = (int)(m - r0);
+      PanelOpts po;
+      po.st_t = h->aux;
+      po.ev_fork = h->sync_events[2 * i];
+      po.ev_join = h->sync_events[2 * i + 1];
+      s = launch_panel(h, p->dtype, Ypart, src, rows, b, Vblk(r0), ldv, Tblk(r0), p->max_rank, ps, ctrl, &ctrl->done,
+                       st, mark, i, po);
+      if (s != RRF_OK) return panel_failed(s);
+      const VtwPlan vp = plan_vtw(h->sms, rows, n, ops->v_bn);
+      mark(RRF_PHASE_VTW, i);
+      ops->vtw(tmV_k, tmW_k, Zpart, r0, r0, vp, ctrl, st);
+      mark(RRF_PHASE_TZ, i);
+      cudaStreamWaitEvent(st, h->sync_events[2 * i + 1], 0);   // join: T_i is needed from here on
+      ops->tz(Zpart, vp, Tblk(r0), p->max_rank, 1, Zt, &ctrl->done, st);
+      const UpdPlan up = plan_upd(h->sms, rows, n, ops->u_bm, ops->u_bn, ops->u_wn);
+      const int j0 = (i + 1 < steps) ? r0 + b : -1;   // Omega rows of the next pass, if there is one
+      mark(RRF_PHASE_UPDATE, i);
+      ops->update(tmV_u, tmZ, tmW_u, tmO, W, ldw, (char*)dB + (size_t)r0 * ldb * esize, ldb, r0, rows, (int)n, r0, b,
+                  j0, Ypart, norm_part, up, ctrl, st);
+      mark(RRF_PHASE_STOP, i);
+      stop_kernel<<<1, 256, 0, st>>>(norm_part, up.P, b, p->max_rank, p->estimator, fixed ? 1 : 0, tr_sub, tr_dir, ctrl,
+                                     done_after, 1);
+      src.slots = 1;
+      src.row_off = b;
+      src.bm = ops->u_bm;
+      src.nc = up.NC;
+      src.tpc = up.tpc;
+      src.wn = ops->u_wn;
     }
-    const VtwPlan vp = plan_vtw(h->sms, rows, n, ops->v_bn);
-    mark(RRF_PHASE_VTW, i);
-    ops->vtw(tmV_k, tmW_k, Zpart, r0, r0, vp, ctrl, st);
-    mark(RRF_PHASE_TZ, i);
-    cudaStreamWaitEvent(st, h->sync_events[2 * i + 1], 0);   // join: T_i is needed from here on
-    ops->tz(Zpart, vp, (const char*)dT + (size_t)r0 * esize, p->max_rank, 1, Zt, &ctrl->done, st);
-    const UpdPlan up = plan_upd(h->sms, rows, n, ops->u_bm, ops->u_bn, ops->u_wn);
-    const int j0 = (i + 1 < steps) ? r0 + b : -1;   // Omega rows of the next pass, if there is one
-    mark(RRF_PHASE_UPDATE, i);
-    ops->update(tmV_u, tmZ, tmW_u, tmO, W, ldw, (char*)dB + (size_t)r0 * ldb * esize, ldb, r0, rows, (int)n, r0, b, j0,
-                Ypart, norm_part, up, ctrl, st);
-    mark(RRF_PHASE_STOP, i);
-    stop_kernel<<<1, 256, 0, st>>>(norm_part, up.P, b, p->max_rank, p->estimator, fixed ? 1 : 0, tr_sub, tr_dir, ctrl);
-    src.slots = 1;
-    src.row_off = b;
-    src.bm = ops->u_bm;
-    src.nc = up.NC;
-    src.tpc = up.tpc;
-    src.wn = ops->u_wn;
+  } else {
+    // Two queues (the paper's look-ahead variant, Figure "DAG" (b)).  The fused update of pass i-1
+    // samples the panel of pass i+1 from the matrix as it stands after pass i-1; the panel kernel of
+    // pass i+1 applies the reflectors of pass i to that panel itself (PanelFix) and factors it on
+    // `look_ctas` SMs while the GEMM kernels of pass i run on the other SMs.
+    //   side stream : panel_0 | fix + panel_1 | fix + panel_2 | ...
+    //   main stream :           V^T W, T Z, update, stop of pass 0 | of pass 1 | ...
+    const int gsms = h->sms - look_ctas;
+    void* Ybuf[2] = {Ypart, ws + L.ypart2};
+    cudaEvent_t evS = h->sync_events[2 * steps];
+    auto evP = [&](int i) { return h->sync_events[2 * i]; };
+    auto evU = [&](int i) { return h->sync_events[2 * i + 1]; };
+    PanelSource src1 = src;           // panel 1: sampled from A by the sample kernel
+    src1.row_off = b;
+    if (steps > 1) {
+      mark(RRF_PHASE_SAMPLE, 0);
+      ops->sample(tmW_s, tmO, Ybuf[1], 0, (int)m, (int)n, b, sp, ctrl, st);
+    }
+    cudaEventRecord(evS, st);
+    cudaStreamWaitEvent(h->aux, evS, 0);
+    ps.bar = look_bar;
+    PanelOpts po;
+    po.ctas = look_ctas;
+    po.bar_reset = look_bar;
+    s = launch_panel(h, p->dtype, Ybuf[0], src, m, b, Vblk(0), ldv, Tblk(0), p->max_rank, ps, ctrl, done_after, h->aux,
+                     NoMark(), 0, po);
+    if (s != RRF_OK) return panel_failed(s);
+    cudaEventRecord(evP(0), h->aux);
+    UpdPlan up_prev{};
+    for (int i = 0; i < steps; ++i) {
+      const int r0 = i * b, rows = (int)(m - r0);
+      if (i + 1 < steps) {
+        PanelSource sn = src1;
+        if (i >= 1) {
+          cudaStreamWaitEvent(h->aux, evU(i - 1), 0);   // the panel sampled by the update of pass i-1
+          sn.slots = 1;
+          sn.row_off = 2 * b;
+          sn.bm = ops->u_bm;
+          sn.nc = up_prev.NC;
+          sn.tpc = up_prev.tpc;
+          sn.wn = ops->u_wn;
+        }
+        PanelOpts pn = po;
+        pn.fix.enabled = 1;
+        pn.fix.Vp = Vblk(r0);
+        pn.fix.ldvp = ldv;
+        pn.fix.Tp = Tblk(r0);
+        pn.fix.ldtp = p->max_rank;
+        pn.fix.Gpart = look_G;
+        pn.fix.M = look_G + (size_t)kLookMaxCtas * b * b;
+        s = launch_panel(h, p->dtype, Ybuf[(i + 1) & 1], sn, rows - b, b, Vblk(r0 + b), ldv, Tblk(r0 + b), p->max_rank,
+                         ps, ctrl, done_after + i, h->aux, NoMark(), i + 1, pn);
+        if (s != RRF_OK) return panel_failed(s);
+        cudaEventRecord(evP(i + 1), h->aux);
+      }
+      mark(RRF_PHASE_PANEL, i);                        // time the main stream waits for V_i, T_i
+      cudaStreamWaitEvent(st, evP(i), 0);
+      const VtwPlan vp = plan_vtw(gsms, rows, n, ops->v_bn);
+      mark(RRF_PHASE_VTW, i);
+      ops->vtw(tmV_k, tmW_k, Zpart, r0, r0, vp, ctrl, st);
+      mark(RRF_PHASE_TZ, i);
+      ops->tz(Zpart, vp, Tblk(r0), p->max_rank, 1, Zt, &ctrl->done, st);
+      const UpdPlan up = plan_upd(gsms, rows, n, ops->u_bm, ops->u_bn, ops->u_wn);
+      const int j0 = (i + 2 < steps) ? r0 + 2 * b : -1;   // Omega rows of the pass after the next
+      mark(RRF_PHASE_UPDATE, i);
+      ops->update(tmV_u, tmZ, tmW_u, tmO, W, ldw, (char*)dB + (size_t)r0 * ldb * esize, ldb, r0, rows, (int)n, r0, b,
+                  j0, Ybuf[i & 1], norm_part, up, ctrl, st);
+      mark(RRF_PHASE_STOP, i);
+      stop_kernel<<<1, 256, 0, st>>>(norm_part, up.P, b, p->max_rank, p->estimator, fixed ? 1 : 0, tr_sub, tr_dir, ctrl,
+                                     done_after, 0);
+      cudaEventRecord(evU(i), st);
+      up_prev = up;
+    }
   }
   mark(RRF_PHASE_SKIPPED, steps);   // closing event
   cudaError_t e = cudaGetLastError();
@@ -839,6 +980,8 @@ rrf_status_t rrf_run(rrf_handle_t h, const rrf_params_t* p, void* dA, int64_t ld
   out->sigma2 = hc.sigma2;
   out->E_sub = hc.E_sub;
   out->E_dir = hc.E_dir;
+  out->queues = look_ctas > 0 ? 2 : 1;
+  out->panel_ctas = look_ctas;
   if (hc.steps > 0) {
     if (h_E_sub_trace != nullptr) cudaMemcpy(h_E_sub_trace, tr_sub, sizeof(double) * hc.steps, cudaMemcpyDeviceToHost);
     if (h_E_dir_trace != nullptr) cudaMemcpy(h_E_dir_trace, tr_dir, sizeof(double) * hc.steps, cudaMemcpyDeviceToHost);
@@ -880,25 +1023,7 @@ static cudaError_t static_setup(int dev, StaticDevice* sd) {
   if (e != cudaSuccess) return e;
   e = cudaDeviceGetAttribute(&smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
   if (e != cudaSuccess) return e;
-  const void* pk[6] = {(const void*)panel_kernel<double, 2>, (const void*)panel_kernel<double, 4>,
-                       (const void*)panel_kernel<double, 7>, (const void*)panel_kernel<float, 2>,
-                       (const void*)panel_kernel<float, 4>,  (const void*)panel_kernel<float, 7>};
-  size_t stat = 0;
-  for (const void* f : pk) {
-    cudaFuncAttributes fa;
-    e = cudaFuncGetAttributes(&fa, f);
-    if (e != cudaSuccess) return e;
-    stat = std::max(stat, fa.sharedSizeBytes);
-  }
-  sd->panel_smem_max = std::min(smem_optin, kMaxSmem) - (int)stat;
-  for (const void* f : pk) {
-    e = cudaFuncSetAttribute(f, cudaFuncAttributeMaxDynamicSharedMemorySize, sd->panel_smem_max);
-    if (e != cudaSuccess) return e;
-  }
-  const int tmax = (128 * 129 + 64 * 65) * 8;
-  e = cudaFuncSetAttribute(tfactor_kernel<double>, cudaFuncAttributeMaxDynamicSharedMemorySize, tmax);
-  if (e != cudaSuccess) return e;
-  e = cudaFuncSetAttribute(tfactor_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, tmax);
+  e = setup_panel_kernels(smem_optin, &sd->panel_smem_max);
   if (e != cudaSuccess) return e;
   sd->ptr = static_cast<unsigned char*>(ptr);
   sd->ready = true;

@@ -8,8 +8,8 @@ namespace rrf {
 
 constexpr int kPanelThreads = 512;
 constexpr int kPanelMaxG = 160;   // most CTAs a panel grid may have (one per SM)
-// doubles of shared memory the panel kernel needs besides the slab: w[b], p[b], pivot_row[b], scalars
-__host__ __device__ constexpr int panel_extra_doubles(int b) { return 3 * b + 4; }
+// doubles of shared memory the panel kernel needs besides the slab: w[b], p[2][b], pivot_row[b], scalars
+__host__ __device__ constexpr int panel_extra_doubles(int b) { return 4 * b + 4; }
 
 // Grid-wide barrier over a monotonically increasing arrival counter.  Needs all CTAs
 // co-resident (cooperative launch).  Bounded: gives up after kWaitLimitClocks.
@@ -81,15 +81,33 @@ struct PanelSource {
   int nseg;                // stacked: number of partial panels
   long long seg_stride;    // stacked: elements between partial panels
   int ldy;                 // stacked: leading dimension
-  int row_off;             // slots: panel row 0 is row `row_off` of the producer's row numbering
+  int row_off;             // panel row 0 is row `row_off` of the producer's row numbering
   int bm, nc, tpc, wn;     // slots: slab height, tiles per slab, tiles per CTA, warp columns
 };
+
+// Look-ahead schedule (Section "Implementation", the two-queue variant): the panel was sampled from
+// the matrix BEFORE the previous block's reflectors were applied, P = W_old * Omega, so the kernel
+// first applies them to the panel itself, Y = (P - Vp (Tp^T (Vp^T P)))[b:, :], where Vp is the previous
+// (rows + b) x b block of Householder vectors and Tp its triangular factor.
+struct PanelFix {
+  int enabled;
+  const void* Vp;          // previous V block, element type T, row 0 = b rows above the panel's row 0
+  long long ldvp;
+  const void* Tp;          // previous T block (b x b, upper triangular), element type T
+  long long ldtp;
+  double* Gpart;           // [gridDim.x][b*b] per-CTA partial Vp^T P
+  double* M;               // [b*b] Tp^T (Vp^T P)
+};
+constexpr int kFixChunk = 32;   // rows of Vp staged in shared memory at a time
+// doubles of shared memory the fix-up needs on top of panel_extra_doubles: the staged rows of Vp
+// (pitch b + 8 or b + 4) and a b x (b + 8) matrix (Tp, then M)
+__host__ __device__ constexpr int panel_fix_doubles(int b) { return kFixChunk * (b + 8) + b * (b + 8); }
 
 template <typename T>
 __device__ __forceinline__ double panel_entry(const T* __restrict__ Y, const PanelSource& src, int r, int c, int b) {
   double s = 0.0;
   if (!src.slots) {
-    const T* p = Y + (size_t)r * src.ldy + c;
+    const T* p = Y + (size_t)(r + src.row_off) * src.ldy + c;
     for (int sg = 0; sg < src.nseg; ++sg) s += (double)p[(size_t)sg * src.seg_stride];
   } else {
     const int lr = r + src.row_off;
@@ -102,8 +120,12 @@ __device__ __forceinline__ double panel_entry(const T* __restrict__ Y, const Pan
   return s;
 }
 
-// QMAX = ceil(R / 32): rows of the slab each lane looks after (template, so they live in registers).
-template <typename T, int QMAX>
+// The 16 warps of a CTA form RH row groups of 16/RH warps; a lane looks after QMAX rows of its
+// group (kept in registers during a pass), so a slab holds up to 32 * QMAX * RH rows.  With PAD the
+// slab is allocated at that full height and zero filled below its last row, which removes every
+// per-element bounds test from the pass; PAD = false keeps the tests (for the one shape whose slab only
+// fits unpadded).
+template <typename T, int QMAX, int RH, bool PAD = true>
 __global__ void __launch_bounds__(kPanelThreads)
     panel_kernel(const T* __restrict__ Y, PanelSource src,
                  int rows, int b, int R, int Rp,
@@ -112,98 +134,266 @@ __global__ void __launch_bounds__(kPanelThreads)
                  double* __restrict__ piv,           // [2][b] broadcast pivot row
                  double* __restrict__ gram,          // [b][b] strictly-lower part: v_c^T v_j (c < j)
                  double* __restrict__ tau_out,       // [b]
-                 unsigned* bar, Ctrl* ctrl, const int* done_flag) {
+                 unsigned* bar, Ctrl* ctrl, const int* done_flag, PanelFix fix) {
   if (*reinterpret_cast<const volatile int*>(done_flag)) return;
   extern __shared__ double psm[];
   double* S = psm;                        // [b][Rp]
   double* w_s = S + (size_t)b * Rp;       // [b]
-  double* p_s = w_s + b;                  // [b]
-  double* pr_s = p_s + b;                 // [b]
+  double* p_s = w_s + b;                  // [2][b]: per row group, then (first b) the grid-wide sums
+  double* pr_s = p_s + 2 * b;             // [b]
   double* sc_s = pr_s + b;                // [4]: tau_j, 1/(alpha - beta)
 
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  constexpr int NW = kPanelThreads / 32;
+  constexpr int NT = kPanelThreads, NW = NT / 32;
+  constexpr int NWC = NW / RH;            // warps that share the columns within one row group
   constexpr int CG = 4;                   // columns a warp handles at a time (independent chains)
+  constexpr int RS = 32 * QMAX * RH;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int rg = warp / NWC, wc = warp - rg * NWC;
   const int G = gridDim.x, cta = blockIdx.x;
   const int Gp = (G + 31) & ~31;
+  // Slab rows are numbered from the first row this kernel touches: with the fix-up that is b rows
+  // above the panel (the rows of P that only enter Vp^T P), so the panel starts at slab row `row0`.
+  const int row0 = fix.enabled ? b : 0;
+  const int ext = rows + row0;
   const int gr0 = cta * R;
-  const int nloc = max(0, min(R, rows - gr0));
+  const int nloc = max(0, min(R, ext - gr0));
+  const int lb = 31 - __clz(b);           // b is a power of two
+  unsigned nbar = 0;                      // grid barriers passed so far
 
   // load the slab: sum the partial panels in their fixed order
-  for (int idx = tid; idx < nloc * b; idx += kPanelThreads) {
-    const int r = idx / b, c = idx - r * b;
-    S[(size_t)c * Rp + r] = panel_entry(Y, src, gr0 + r, c, b);
+  for (int idx = tid; idx < nloc * b; idx += NT) {
+    const int r = idx >> lb, c = idx & (b - 1);
+    S[(size_t)c * Rp + r] = panel_entry(Y, src, gr0 + r - row0, c, b);
+  }
+  if (PAD) {
+    const int npad = RS - nloc;
+    for (int idx = tid; idx < npad * b; idx += NT) {
+      const int c = idx / npad, r = nloc + (idx - c * npad);
+      S[(size_t)c * Rp + r] = 0.0;
+    }
   }
   __syncthreads();
 
+  if (fix.enabled) {
+    // ---- S <- P - Vp (Tp^T (Vp^T P)) on the tensor cores (FP64 m16n8k8)
+    const int g = lane >> 2, t = lane & 3;
+    double* Vst = sc_s + 4;                              // [kFixChunk][b + 8] or [kFixChunk][b + 4]
+    double* Mst = Vst + (size_t)kFixChunk * (b + 8);     // [b][b + 8]: Tp (pitch b + 1), then M
+    const T* Vp = reinterpret_cast<const T*>(fix.Vp);
+    const T* Tp = reinterpret_cast<const T*>(fix.Tp);
+    const int nch = (nloc + kFixChunk - 1) / kFixChunk;
+    constexpr int EPT = 4;                               // kFixChunk * 64 / NT staged elements per thread
+    T pre[EPT];
+    auto fetch = [&](int ch) {                           // rows of Vp for chunk ch, into registers
+#pragma unroll
+      for (int e = 0; e < EPT; ++e) {
+        const int idx = tid + e * NT, rr = idx >> lb, c = idx & (b - 1), r = ch * kFixChunk + rr;
+        pre[e] = (rr < kFixChunk && r < nloc) ? Vp[(size_t)(gr0 + r) * fix.ldvp + c] : T(0);
+      }
+    };
+    auto stash = [&](int pitch) {                        // registers -> Vst[rr][c]
+#pragma unroll
+      for (int e = 0; e < EPT; ++e) {
+        const int idx = tid + e * NT, rr = idx >> lb, c = idx & (b - 1);
+        if (rr < kFixChunk) Vst[rr * pitch + c] = (double)pre[e];
+      }
+    };
+    // Tp into shared memory (pitch b + 1), zero below the diagonal
+    for (int idx = tid; idx < b * b; idx += NT) {
+      const int l = idx >> lb, k = idx & (b - 1);
+      Mst[l * (b + 1) + k] = l <= k ? (double)Tp[(size_t)l * fix.ldtp + k] : 0.0;
+    }
+    // Phase 1: Gpart[cta] = Vp[slab]^T S.  Warp (mt, np) owns G[16 mt .., 16 np ..] (two n-tiles).
+    {
+      const int nmt = b >> 4;
+      const bool act = warp < nmt * nmt;
+      const int mt = act ? warp / nmt : 0, np = act ? warp - mt * nmt : 0;
+      const int PV = b + 8;
+      double acc[2][4];
+#pragma unroll
+      for (int i = 0; i < 2; ++i)
+#pragma unroll
+        for (int e = 0; e < 4; ++e) acc[i][e] = 0.0;
+      if (nch > 0) fetch(0);
+      for (int ch = 0; ch < nch; ++ch) {
+        __syncthreads();
+        stash(PV);
+        __syncthreads();
+        if (ch + 1 < nch) fetch(ch + 1);
+        if (act) {
+          const int rc = ch * kFixChunk;
+#pragma unroll
+          for (int ks = 0; ks < kFixChunk / 8; ++ks) {
+            const double* va = Vst + (ks * 8 + t) * PV + mt * 16 + g;
+            const double af[4] = {va[0], va[8], va[4 * PV], va[4 * PV + 8]};
+#pragma unroll
+            for (int i = 0; i < 2; ++i) {
+              const double* sb = S + (size_t)((np * 2 + i) * 8 + g) * Rp + rc + ks * 8 + t;
+              const double bf[2] = {sb[0], sb[4]};
+              mma16x8x8(acc[i], af, bf);
+            }
+          }
+        }
+      }
+      if (act) {
+        double* gp = fix.Gpart + (size_t)cta * b * b;
+#pragma unroll
+        for (int i = 0; i < 2; ++i) {
+          const int col = (np * 2 + i) * 8 + 2 * t, row = mt * 16 + g;
+          gp[(size_t)row * b + col] = acc[i][0];
+          gp[(size_t)row * b + col + 1] = acc[i][1];
+          gp[(size_t)(row + 8) * b + col] = acc[i][2];
+          gp[(size_t)(row + 8) * b + col + 1] = acc[i][3];
+        }
+      }
+    }
+    if (!grid_barrier(bar, (++nbar) * (unsigned)G, ctrl)) return;
+    // Phase 2: CTA c owns columns c, c + G, ... of G = sum of the partials (in CTA order) and of
+    // M = Tp^T G, column by column: M[k][c2] = sum_{l <= k} Tp[l][k] G[l][c2].
+    {
+      const int ncol = cta < b ? (b - cta + G - 1) / G : 0;
+      double* Gs = Vst;                                  // up to kFixChunk columns of G at a time
+      for (int q0 = 0; q0 < ncol; q0 += kFixChunk) {
+        const int nq = min(kFixChunk, ncol - q0);
+        __syncthreads();
+        for (int idx = tid; idx < nq * b; idx += NT) {
+          const int q = idx >> lb, l = idx & (b - 1), c2 = cta + (q0 + q) * G;
+          const double* gp = fix.Gpart + (size_t)l * b + c2;
+          double sum = 0.0;
+          int x = 0;
+          for (; x + 8 <= G; x += 8) {
+            double v[8];
+#pragma unroll
+            for (int e = 0; e < 8; ++e) v[e] = __ldcg(gp + (size_t)(x + e) * b * b);
+#pragma unroll
+            for (int e = 0; e < 8; ++e) sum += v[e];
+          }
+          for (; x < G; ++x) sum += __ldcg(gp + (size_t)x * b * b);
+          Gs[q * b + l] = sum;
+        }
+        __syncthreads();
+        for (int idx = tid; idx < nq * b; idx += NT) {
+          const int q = idx >> lb, k = idx & (b - 1), c2 = cta + (q0 + q) * G;
+          double s0 = 0.0, s1 = 0.0;
+          int l = 0;
+          for (; l + 1 <= k; l += 2) {
+            s0 += Mst[l * (b + 1) + k] * Gs[q * b + l];
+            s1 += Mst[(l + 1) * (b + 1) + k] * Gs[q * b + l + 1];
+          }
+          if (l <= k) s0 += Mst[l * (b + 1) + k] * Gs[q * b + l];
+          fix.M[(size_t)k * b + c2] = s0 + s1;
+        }
+      }
+    }
+    if (!grid_barrier(bar, (++nbar) * (unsigned)G, ctrl)) return;
+    // Phase 3: S -= Vp[slab] M.  A task is a 16-row x 8-column tile of a chunk.
+    {
+      const int PV = b + 4, PM = b + 8;
+      for (int idx = tid; idx < b * b; idx += NT) Mst[(idx >> lb) * PM + (idx & (b - 1))] = __ldcg(fix.M + idx);
+      const int ntask = (kFixChunk / 16) * (b >> 3);
+      if (nch > 0) fetch(0);
+      for (int ch = 0; ch < nch; ++ch) {
+        __syncthreads();
+        stash(PV);
+        __syncthreads();
+        if (ch + 1 < nch) fetch(ch + 1);
+        const int rc = ch * kFixChunk;
+        for (int task = warp; task < ntask; task += NW) {
+          const int r0 = (task & 1) * 16, n0 = (task >> 1) * 8;
+          double acc[4] = {0.0, 0.0, 0.0, 0.0};
+          for (int k0 = 0; k0 < b; k0 += 8) {
+            const double* va = Vst + (r0 + g) * PV + k0 + t;
+            const double af[4] = {va[0], va[8 * PV], va[4], va[8 * PV + 4]};
+            const double* mb = Mst + (k0 + t) * PM + n0 + g;
+            const double bf[2] = {mb[0], mb[4 * PM]};
+            mma16x8x8(acc, af, bf);
+          }
+          double* s0 = S + (size_t)(n0 + 2 * t) * Rp + rc + r0 + g;
+          s0[0] -= acc[0];
+          s0[Rp] -= acc[1];
+          s0[8] -= acc[2];
+          s0[Rp + 8] -= acc[3];
+        }
+      }
+    }
+    __syncthreads();
+  }
+
   double tau_prev = 0.0;
   for (int j = 0; j < b; ++j) {
+    const int pr = row0 + j;                           // slab-numbering row of the pivot
     double* Sj = S + (size_t)j * Rp;
     const double* Sjm1 = S + (size_t)(j > 0 ? j - 1 : 0) * Rp;
     // finish column j: pending reflector H_{j-1}
     if (j > 0 && tau_prev != 0.0) {
       const double f = tau_prev * w_s[j];
-      for (int r = tid; r < nloc; r += kPanelThreads)
-        if (gr0 + r >= j) Sj[r] -= f * Sjm1[r];
+      for (int r = tid; r < nloc; r += NT)
+        if (gr0 + r >= pr) Sj[r] -= f * Sjm1[r];
     }
     __syncthreads();
     // one pass: update trailing columns and take all dot products with column j.  Each lane keeps
-    // its rows of column j and of v_{j-1} in registers; CG columns are in flight per warp.
+    // its rows of column j and of v_{j-1} in registers, masked once per column: rows at or above the
+    // pivot do not count in the dot products, and rows the pending reflector must not change see
+    // v_{j-1} = 0, so the inner loop needs no tests.  CG columns are in flight per warp.
     {
       double yj[QMAX], vp[QMAX];
+      const int rbase = rg * (32 * QMAX) + lane;
 #pragma unroll
       for (int q = 0; q < QMAX; ++q) {
-        const int r = lane + 32 * q;
-        const bool in = r < nloc;
+        const int r = rbase + 32 * q;
+        const bool in = PAD || r < nloc;
         const int grow = gr0 + r;
-        yj[q] = (in && grow > j) ? Sj[r] : 0.0;            // rows at or above the pivot do not count
-        vp[q] = (in && grow >= j) ? Sjm1[r] : 0.0;         // rows above j are finished
+        yj[q] = (in && grow > pr) ? Sj[r] : 0.0;
+        vp[q] = (in && grow >= pr) ? Sjm1[r] : 0.0;
       }
       const bool pending = (j > 0) && (tau_prev != 0.0);
-      for (int c0 = warp; c0 < b; c0 += NW * CG) {
+      for (int c0 = wc; c0 < b; c0 += NWC * CG) {
         double x[CG][QMAX], acc[CG];
 #pragma unroll
         for (int u = 0; u < CG; ++u) {
-          const int c = c0 + u * NW;
-          const double* Sc = S + (size_t)(c < b ? c : 0) * Rp;
+          const int c = c0 + u * NWC;
+          const double* Sc = S + (size_t)(c < b ? c : 0) * Rp + rbase;
 #pragma unroll
-          for (int q = 0; q < QMAX; ++q) {
-            const int r = lane + 32 * q;
-            x[u][q] = (c < b && r < nloc) ? Sc[r] : 0.0;
-          }
+          for (int q = 0; q < QMAX; ++q) x[u][q] = (PAD || rbase + 32 * q < nloc) ? Sc[32 * q] : 0.0;
         }
 #pragma unroll
         for (int u = 0; u < CG; ++u) {
-          const int c = c0 + u * NW;
+          const int c = c0 + u * NWC;
           const bool upd = pending && c > j && c < b;
-          const double f = upd ? tau_prev * w_s[c] : 0.0;
-          double* Sc = S + (size_t)(c < b ? c : 0) * Rp;
           double a = 0.0;
+          if (upd) {
+            const double f = tau_prev * w_s[c];
+            double* Sc = S + (size_t)c * Rp + rbase;
 #pragma unroll
-          for (int q = 0; q < QMAX; ++q) {
-            const int r = lane + 32 * q;
-            double xv = x[u][q];
-            if (upd) {
-              xv -= f * vp[q];
-              if (r < nloc && gr0 + r >= j) Sc[r] = xv;
+            for (int q = 0; q < QMAX; ++q) {
+              const double xv = x[u][q] - f * vp[q];
+              if (PAD || rbase + 32 * q < nloc) Sc[32 * q] = xv;
+              a += yj[q] * xv;
             }
-            a += yj[q] * xv;
+          } else {
+#pragma unroll
+            for (int q = 0; q < QMAX; ++q) a += yj[q] * x[u][q];
           }
-          acc[u] = a;
+          acc[u] = c < b ? a : 0.0;
         }
         {
           const double tot = warp_sum4(acc, lane);
           const int u = ((lane >> 4) << 1) | ((lane >> 3) & 1);
-          if ((lane & 7) == 0 && c0 + u * NW < b) p_s[c0 + u * NW] = tot;
+          if ((lane & 7) == 0 && c0 + u * NWC < b) p_s[rg * b + c0 + u * NWC] = tot;
         }
       }
     }
     __syncthreads();
     double* Pj = P + (size_t)(j & 1) * b * Gp;
-    for (int c = tid; c < b; c += kPanelThreads) Pj[(size_t)c * Gp + cta] = p_s[c];
-    if (j >= gr0 && j < gr0 + nloc)
-      for (int c = tid; c < b; c += kPanelThreads) piv[(j & 1) * b + c] = S[(size_t)c * Rp + (j - gr0)];
-    if (!grid_barrier(bar, (unsigned)(j + 1) * (unsigned)G, ctrl)) return;
+    for (int c = tid; c < b; c += NT) {
+      double v = p_s[c];
+#pragma unroll
+      for (int h = 1; h < RH; ++h) v += p_s[h * b + c];
+      Pj[(size_t)c * Gp + cta] = v;
+    }
+    if (pr >= gr0 && pr < gr0 + nloc)
+      for (int c = tid; c < b; c += NT) piv[(j & 1) * b + c] = S[(size_t)c * Rp + (pr - gr0)];
+    if (!grid_barrier(bar, (++nbar) * (unsigned)G, ctrl)) return;
 
     // every CTA: sum of the per-CTA partials in a fixed order (lane x takes CTAs x, x+32, ...;
     // then the fixed shuffle tree), one warp per column, CG columns of loads in flight at once
@@ -261,17 +451,17 @@ __global__ void __launch_bounds__(kPanelThreads)
       if (cta == 0 && tid < j) gram[(size_t)j * b + tid] = wv;
     }
     // column j becomes v_j (unit lower trapezoidal, explicit ones and zeros)
-    for (int r = tid; r < nloc; r += kPanelThreads) {
+    for (int r = tid; r < nloc; r += NT) {
       const int grow = gr0 + r;
-      Sj[r] = grow > j ? Sj[r] * rdenom : (grow == j ? 1.0 : 0.0);
+      Sj[r] = grow > pr ? Sj[r] * rdenom : (grow == pr ? 1.0 : 0.0);
     }
     tau_prev = tau;
     __syncthreads();
   }
 
-  for (int idx = tid; idx < nloc * b; idx += kPanelThreads) {
-    const int r = idx / b, c = idx - r * b;
-    V[(size_t)(gr0 + r) * ldv + c] = (T)S[(size_t)c * Rp + r];
+  for (int idx = tid; idx < nloc * b; idx += NT) {
+    const int r = idx >> lb, c = idx & (b - 1);
+    if (gr0 + r >= row0) V[(size_t)(gr0 + r - row0) * ldv + c] = (T)S[(size_t)c * Rp + r];
   }
 }
 
@@ -287,8 +477,9 @@ __global__ void __launch_bounds__(kPanelThreads)
 template <typename T>
 __global__ void __launch_bounds__(256)
     tfactor_kernel(const double* __restrict__ gram, const double* __restrict__ tau, int b,
-                   T* __restrict__ Tout, long long ldt, const int* done_flag) {
+                   T* __restrict__ Tout, long long ldt, const int* done_flag, unsigned* bar_reset) {
   if (*reinterpret_cast<const volatile int*>(done_flag)) return;
+  if (threadIdx.x == 0 && bar_reset != nullptr) *bar_reset = 0;   // the panel before this kernel is finished with it
   extern __shared__ double tsm[];
   const int pitch = b + 1, mp = b / 2 + 1;
   double* Ts = tsm;                        // [b][pitch]: T above and on the diagonal, Gram rows below
@@ -481,7 +672,7 @@ __global__ void __launch_bounds__(256)
 
 __global__ void __launch_bounds__(256)
     init_ctrl_kernel(const double* __restrict__ part, int npart, double tol, int relative, int fixed_rank,
-                     int b, int max_rank, Ctrl* ctrl) {
+                     int b, int max_rank, Ctrl* ctrl, int* __restrict__ done_after, int nsteps) {
   __shared__ double red[32];
   double s = 0.0;
   for (int i = threadIdx.x; i < npart; i += 256) s += part[i];
@@ -506,13 +697,19 @@ __global__ void __launch_bounds__(256)
     }
     ctrl->status = status;
     ctrl->done = done;
+    // done_after[q] = value of `done` when block step q is about to start; steps that never run keep 1
+    if (done_after != nullptr) {
+      done_after[0] = done;
+      for (int q = 1; q <= nsteps; ++q) done_after[q] = 1;
+    }
   }
 }
 
 // Algorithm 2 lines 9-10 and the test of line 5 for the next pass, on the device.
 __global__ void __launch_bounds__(256)
     stop_kernel(const double* __restrict__ norm_part, int npart, int b, int max_rank, int estimator,
-                int fixed_rank, double* __restrict__ tr_sub, double* __restrict__ tr_dir, Ctrl* ctrl) {
+                int fixed_rank, double* __restrict__ tr_sub, double* __restrict__ tr_dir, Ctrl* ctrl,
+                int* __restrict__ done_after, int reset_bar) {
   if (*reinterpret_cast<volatile int*>(&ctrl->done)) return;
   __shared__ double red[64];
   double st = 0.0, sr = 0.0;
@@ -531,13 +728,14 @@ __global__ void __launch_bounds__(256)
     tr_dir[i] = trail;
     ctrl->steps = i + 1;
     ctrl->k = (i + 1) * b;
-    ctrl->bar = 0;
+    if (reset_bar) ctrl->bar = 0;
     const double E = estimator == 0 ? trail : e_sub;
     const bool below = !(E > ctrl->sigma2);
     const bool met = !fixed_rank && below;
     const bool cap = (i + 2) * b > max_rank;
     if (ctrl->status == RRF_OK && !below && cap) ctrl->status = RRF_MAX_RANK_REACHED;
     if (met || cap) ctrl->done = 1;
+    if (done_after != nullptr) done_after[i + 1] = (met || cap) ? 1 : 0;
   }
 }
 

@@ -172,10 +172,15 @@ def test_apply_and_form_q_match_oracle(h, m, ncols, b, k, dtype):
 # ------------------------------------------------------------------ whole runs
 
 
-def test_cfg1_full(h):
+SCHEDULES = [pytest.param(rrf.RRF_FLAG_ONE_QUEUE, id="one-queue"), pytest.param(rrf.RRF_FLAG_TWO_QUEUES, id="two-queues")]
+
+
+@pytest.mark.parametrize("sched", SCHEDULES)
+def test_cfg1_full(h, sched):
     w = wl.CONFIGS["cfg1"]
-    g, o, A, Om = run_both(h, w)
+    g, o, A, Om = run_both(h, w, flags=sched)
     assert o.k == 256 and o.status == orc.RRF_MAX_RANK_REACHED
+    assert g.queues == (1 if sched == rrf.RRF_FLAG_ONE_QUEUE else 2)
     check_run(h, w, g, o, A, Om)
 
 
@@ -191,10 +196,32 @@ def test_cfg1_full(h):
     ("cfg4b", dict(m=1200, n=1024, max_rank=256, rank=128, b=128)),
     ("cfg1", dict(m=900, n=700, max_rank=256, b=128)),                 # fp64, widest block, ragged
 ])
-def test_reduced_configs(h, name, kw):
+@pytest.mark.parametrize("sched", SCHEDULES)
+def test_reduced_configs(h, name, kw, sched):
     w = wl.CONFIGS[name].scaled(**kw)
-    g, o, A, Om = run_both(h, w)
+    g, o, A, Om = run_both(h, w, flags=sched)
+    # the look-ahead schedule needs the panel (plus its staging) in a few SMs' shared memory
+    assert g.queues == (2 if sched == rrf.RRF_FLAG_TWO_QUEUES and w.b <= 64 else 1)
     check_run(h, w, g, o, A, Om)
+
+
+def test_schedules_agree_and_stop_mid_way(h):
+    # stops after a few blocks: the look-ahead has factored one panel too many by then, which must
+    # not show in k, B, the traces, or the defined part of V and T
+    w = wl.CONFIGS["cfg2"].scaled(m=2048, n=1536, max_rank=512)
+    A, _ = wl.make_matrix(w)
+    Om = wl.make_omega(w)
+    dA, dOmT = torch.from_numpy(A).cuda(), torch.from_numpy(np.ascontiguousarray(Om.T)).cuda()
+    g1 = rrf.rrf_run(h, dA, w.b, 1e-2, w.max_rank, omegaT=dOmT, flags=rrf.RRF_FLAG_ONE_QUEUE)
+    g2 = rrf.rrf_run(h, dA, w.b, 1e-2, w.max_rank, omegaT=dOmT, flags=rrf.RRF_FLAG_TWO_QUEUES)
+    assert (g1.queues, g2.queues) == (1, 2) and g2.panel_ctas > 0
+    assert 0 < g1.k < w.max_rank and g1.k == g2.k and g1.status == g2.status == rrf.RRF_OK
+    k = g1.k
+    assert relmax(g2.B[:k].cpu().numpy(), g1.B[:k].cpu().numpy()) <= 1e-10
+    assert np.allclose(g1.E_dir_trace, g2.E_dir_trace, rtol=1e-9)
+    Q1 = rrf.rrf_form_q(h, g1.V, g1.T, w.b, k).cpu().numpy()
+    Q2 = rrf.rrf_form_q(h, g2.V, g2.T, w.b, k).cpu().numpy()
+    assert relmax(Q2 @ g2.B[:k].cpu().numpy(), Q1 @ g1.B[:k].cpu().numpy()) <= 1e-10
 
 
 def test_subtractive_estimator_and_fixed_rank(h):
