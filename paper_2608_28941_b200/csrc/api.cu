@@ -3,6 +3,7 @@
 #include <algorithm>
 #include <cstdio>
 #include <cstdlib>
+#include <cmath>
 #include <cstring>
 #include <new>
 #include <vector>
@@ -154,7 +155,29 @@ static size_t panel_scratch_bytes(int sms, int b) {
   const int gp = (sms + 31) / 32 * 32;
   return align_up(((size_t)2 * gp * b + 2 * (size_t)b + (size_t)b * b + b) * sizeof(double) + 256, 256);
 }
-constexpr int kLookMaxCtas = 40;   // most CTAs a confined panel may take
+constexpr int kLookMaxCtas = 48;   // most CTAs a confined panel may take
+// Rough cost model of one pass, in microseconds, used only to choose the schedule (fitted to event
+// timings on a B200; the look-ahead is right or wrong by its measured time, not by this model).
+struct PassModel {
+  int sms;
+  double rows, n;
+  int b;
+  bool f64;
+  // flop per microsecond the two GEMM kernels sustain on the whole device
+  double vtw() const { return 2.0 * rows * n * b / (f64 ? 33e6 : 45e6) + 10.0; }
+  double upd() const { return 4.0 * rows * n * b / (f64 ? 27e6 : 32e6) + 15.0; }
+  // fix-up + panel + T factor on `ctas` SMs, with the launch and event hand-overs of the side stream
+  double panel_chain(int ctas) const {
+    const double R = std::max(64.0, (rows + b) / ctas);
+    const double cycles = b * (7000.0 + 0.14 * R * b) + 20000.0 + 0.07 * R * b * b;
+    return cycles / 1965.0 + 0.3 * b + (f64 ? 45.0 : 85.0);
+  }
+  // the stream-K GEMMs lose a little more than the SMs they give up (tile quantisation)
+  double scale(int ctas) const { return std::pow((double)sms / (sms - ctas), 1.15); }
+  double step_ungated(int ctas) const { return std::max(panel_chain(ctas), (vtw() + upd()) * scale(ctas)); }
+  double step_gated(int ctas) const { return vtw() + std::max(panel_chain(ctas), upd() * scale(ctas)); }
+  double step_serial() const { return vtw() + upd() + b * 4.2 + 25.0; }
+};
 static size_t look_scratch_bytes(int b) {   // Gpart[kLookMaxCtas][b*b] + M[b*b]
   return align_up((size_t)(kLookMaxCtas + 1) * b * b * sizeof(double), 256);
 }
@@ -742,11 +765,23 @@ rrf_status_t rrf_run(rrf_handle_t h, const rrf_params_t* p, void* dA, int64_t ld
   int look_ctas = 0;
   if (!(p->flags & RRF_FLAG_ONE_QUEUE) && steps_total >= 2) {
     const int fewest = panel_min_ctas(h, m, b);
-    int want = std::max(fewest, h->sms / 9);
-    if (const char* ev = std::getenv("RRF_LOOKAHEAD_CTAS")) want = std::max(fewest, std::atoi(ev));
-    const int cap = (p->flags & RRF_FLAG_TWO_QUEUES) ? kLookMaxCtas : std::min(kLookMaxCtas, h->sms / 5);
-    PanelPlan ppl;
-    if (fewest > 0 && want <= cap && want < h->sms && plan_panel(h, m, b, &ppl, want, true)) look_ctas = want;
+    const int cap = std::min(kLookMaxCtas, h->sms / 3);
+    if (fewest > 0 && fewest <= cap) {
+      const PassModel pm{h->sms, (double)m, (double)n, b, p->dtype == RRF_F64};
+      int best = fewest;
+      double best_t = std::min(pm.step_ungated(fewest), pm.step_gated(fewest));
+      for (int c = fewest + 1; c <= cap; ++c) {
+        const double t = std::min(pm.step_ungated(c), pm.step_gated(c));
+        if (t < best_t * 0.995) {
+          best_t = t;
+          best = c;
+        }
+      }
+      if (const char* ev = std::getenv("RRF_LOOKAHEAD_CTAS")) best = std::min(cap, std::max(fewest, std::atoi(ev)));
+      PanelPlan ppl;
+      const bool wanted = (p->flags & RRF_FLAG_TWO_QUEUES) || best_t < pm.step_serial();
+      if (wanted && plan_panel(h, m, b, &ppl, best, true)) look_ctas = best;
+    }
   }
   PanelPlan pp0;
   if (look_ctas == 0 && !plan_panel(h, m, b, &pp0)) return fail(RRF_ERR_WORKSPACE);   // tallest panel must fit on chip
@@ -820,7 +855,7 @@ rrf_status_t rrf_run(rrf_handle_t h, const rrf_params_t* p, void* dA, int64_t ld
                                       ctrl, done_after, steps);
 
   // fork/join events for the side stream, created once and kept in the handle
-  while (h->sync_events.size() < (size_t)2 * steps + 1) {
+  while (h->sync_events.size() < (size_t)3 * steps + 2) {
     cudaEvent_t ev;
     if (cudaEventCreateWithFlags(&ev, cudaEventDisableTiming) != cudaSuccess) return fail(RRF_ERR_CUDA);
     h->sync_events.push_back(ev);
@@ -888,15 +923,21 @@ rrf_status_t rrf_run(rrf_handle_t h, const rrf_params_t* p, void* dA, int64_t ld
     //   main stream :           V^T W, T Z, update, stop of pass 0 | of pass 1 | ...
     const int gsms = h->sms - look_ctas;
     void* Ybuf[2] = {Ypart, ws + L.ypart2};
-    cudaEvent_t evS = h->sync_events[2 * steps];
-    auto evP = [&](int i) { return h->sync_events[2 * i]; };
-    auto evU = [&](int i) { return h->sync_events[2 * i + 1]; };
+    cudaEvent_t evS = h->sync_events[3 * steps], evS2 = h->sync_events[3 * steps + 1];
+    auto evP = [&](int i) { return h->sync_events[3 * i]; };
+    auto evU = [&](int i) { return h->sync_events[3 * i + 1]; };
+    auto evZ = [&](int i) { return h->sync_events[3 * i + 2]; };
+    // Where the update alone outlasts the next panel, the panel is held back until V^T W and T Z of
+    // the pass are done, and V^T W gets every SM; otherwise the panel chain is the critical path and
+    // starts as early as its inputs allow.
+    const char* gate_env = std::getenv("RRF_LOOKAHEAD_GATE");
+    auto gated = [&](int rows_i) {
+      if (gate_env != nullptr) return std::atoi(gate_env) != 0;
+      const PassModel pm{h->sms, (double)rows_i, (double)n, b, p->dtype == RRF_F64};
+      return pm.step_gated(look_ctas) < pm.step_ungated(look_ctas);
+    };
     PanelSource src1 = src;           // panel 1: sampled from A by the sample kernel
     src1.row_off = b;
-    if (steps > 1) {
-      mark(RRF_PHASE_SAMPLE, 0);
-      ops->sample(tmW_s, tmO, Ybuf[1], 0, (int)m, (int)n, b, sp, ctrl, st);
-    }
     cudaEventRecord(evS, st);
     cudaStreamWaitEvent(h->aux, evS, 0);
     ps.bar = look_bar;
@@ -907,11 +948,18 @@ rrf_status_t rrf_run(rrf_handle_t h, const rrf_params_t* p, void* dA, int64_t ld
                      NoMark(), 0, po);
     if (s != RRF_OK) return panel_failed(s);
     cudaEventRecord(evP(0), h->aux);
+    if (steps > 1) {                  // the second panel is sampled while the first is factored
+      mark(RRF_PHASE_SAMPLE, 0);
+      ops->sample(tmW_s, tmO, Ybuf[1], 0, (int)m, (int)n, b, sp, ctrl, st);
+      cudaEventRecord(evS2, st);
+    }
     UpdPlan up_prev{};
     for (int i = 0; i < steps; ++i) {
       const int r0 = i * b, rows = (int)(m - r0);
-      if (i + 1 < steps) {
+      const bool gate = gated(rows);
+      auto next_panel = [&]() -> rrf_status_t {
         PanelSource sn = src1;
+        if (i == 0) cudaStreamWaitEvent(h->aux, evS2, 0);
         if (i >= 1) {
           cudaStreamWaitEvent(h->aux, evU(i - 1), 0);   // the panel sampled by the update of pass i-1
           sn.slots = 1;
@@ -929,18 +977,29 @@ rrf_status_t rrf_run(rrf_handle_t h, const rrf_params_t* p, void* dA, int64_t ld
         pn.fix.ldtp = p->max_rank;
         pn.fix.Gpart = look_G;
         pn.fix.M = look_G + (size_t)kLookMaxCtas * b * b;
-        s = launch_panel(h, p->dtype, Ybuf[(i + 1) & 1], sn, rows - b, b, Vblk(r0 + b), ldv, Tblk(r0 + b), p->max_rank,
-                         ps, ctrl, done_after + i, h->aux, NoMark(), i + 1, pn);
+        if (gate) cudaStreamWaitEvent(h->aux, evZ(i), 0);
+        const rrf_status_t ls = launch_panel(h, p->dtype, Ybuf[(i + 1) & 1], sn, rows - b, b, Vblk(r0 + b), ldv,
+                                             Tblk(r0 + b), p->max_rank, ps, ctrl, done_after + i, h->aux, NoMark(),
+                                             i + 1, pn);
+        if (ls == RRF_OK) cudaEventRecord(evP(i + 1), h->aux);
+        return ls;
+      };
+      if (i + 1 < steps && !gate) {
+        s = next_panel();
         if (s != RRF_OK) return panel_failed(s);
-        cudaEventRecord(evP(i + 1), h->aux);
       }
       mark(RRF_PHASE_PANEL, i);                        // time the main stream waits for V_i, T_i
       cudaStreamWaitEvent(st, evP(i), 0);
-      const VtwPlan vp = plan_vtw(gsms, rows, n, ops->v_bn);
+      const VtwPlan vp = plan_vtw(gate ? h->sms : gsms, rows, n, ops->v_bn);
       mark(RRF_PHASE_VTW, i);
       ops->vtw(tmV_k, tmW_k, Zpart, r0, r0, vp, ctrl, st);
       mark(RRF_PHASE_TZ, i);
       ops->tz(Zpart, vp, Tblk(r0), p->max_rank, 1, Zt, &ctrl->done, st);
+      if (i + 1 < steps && gate) {
+        cudaEventRecord(evZ(i), st);
+        s = next_panel();
+        if (s != RRF_OK) return panel_failed(s);
+      }
       const UpdPlan up = plan_upd(gsms, rows, n, ops->u_bm, ops->u_bn, ops->u_wn);
       const int j0 = (i + 2 < steps) ? r0 + 2 * b : -1;   // Omega rows of the pass after the next
       mark(RRF_PHASE_UPDATE, i);
