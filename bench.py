@@ -249,24 +249,39 @@ def main():
             dist.barrier()
             torch.cuda.synchronize()
 
-    rrf.rrf_set_profiling(h, True)
+    # Timed region: the call as a user makes it (no per-kernel events).  The per-kernel event profile
+    # that feeds `roofline` is taken over the same number of steps right after it, because an event
+    # between every two kernels lengthens a step by several percent.
+    rrf.rrf_set_profiling(h, False)
     for _ in range(max(args.warmup, 1)):
         res = step()
     sampler = ClockSampler(local)
     barrier()
     sampler.start()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    prof = {}
     e0.record()
     for _ in range(args.steps):
         res = step()
+    e1.record()
+    barrier()
+    p0, p1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    rrf.rrf_set_profiling(h, True)
+    for _ in range(2):
+        step()
+    prof = {}
+    barrier()
+    p0.record()
+    for _ in range(args.steps):
+        step()
         for name, (ms, cnt) in rrf.rrf_get_profile(h).items():
             a = prof.setdefault(name, [0.0, 0])
             a[0] += ms
             a[1] += cnt
-    e1.record()
+    p1.record()
     barrier()
     clocks = sampler.stop()
+    rrf.rrf_set_profiling(h, False)
+    ms_profiled = p0.elapsed_time(p1) / args.steps
     ms_step = max_over_ranks(e0.elapsed_time(e1), world, dev) / args.steps
     flops = method_flops(w.m, w.n, w.b, res.steps)
     value = job_tflops(flops, world, ms_step)
@@ -337,6 +352,12 @@ def main():
                         "peak_recipe_source": ("MEASURED_PEAKS.json bf16 x nominal FP64/bf16 ratio (of measured)"
                                                if "bf16_tflops" in peaks else "fallback bf16 x nominal ratio (of fallback)"),
                         "avg_launch_ms": ms / max(cnt, 1), "launches": cnt}
+            # with the look-ahead schedule the update runs beside the panel kernel, on the SMs left to it
+            sms = torch.cuda.get_device_properties(local).multi_processor_count
+            share = (sms - res.panel_ctas) / sms if (res.queues == 2 and top == "update") else 1.0
+            roofline["sm_share"] = share
+            roofline["frac_of_share"] = achieved / (peak * share)
+            roofline["whole_step_frac"] = value / world / peak
         else:
             hbm = peaks.get("hbm_gbs", 6650.0)
             byts = args.steps * sum(2.0 * r * w.b * esize for r in mi)
@@ -346,6 +367,8 @@ def main():
                         "peak_source": "MEASURED_PEAKS.json (of measured)" if "hbm_gbs" in peaks else "of fallback",
                         "avg_launch_ms": ms / max(cnt, 1), "launches": cnt}
         roofline["phases_ms_per_step"] = {nm: prof[nm][0] / args.steps for nm in prof}
+        roofline["profiled_over"] = ("%d steps right after the timed region, with an event before every kernel "
+                                     "(%.3f ms per step with the events, %.3f without)" % (args.steps, ms_profiled, ms_step))
 
     # ---- CPU baseline: the oracle on the host cores (rank 0, single-GPU runs only)
     cpu = None

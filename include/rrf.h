@@ -52,6 +52,8 @@ typedef enum {
 #define RRF_FLAG_INPLACE 1u     /* A itself is the working matrix (it is overwritten) */
 #define RRF_FLAG_FIXED_RANK 2u  /* ignore the tolerance, always run to max_rank (fixed-rank mode) */
 #define RRF_FLAG_ONE_QUEUE 4u   /* force the sequential schedule: panel, V^T W, update one after the other */
+#define RRF_FLAG_NO_GRAPH 16u    /* always enqueue the kernels one by one (by default a call that repeats the
+                                   previous call's arguments is captured into a CUDA graph and replayed) */
 #define RRF_FLAG_TWO_QUEUES 8u  /* use the look-ahead schedule whenever the panel can be confined to a few SMs,
                                    also where the built-in rule would pick the sequential one */
 

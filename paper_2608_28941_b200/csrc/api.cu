@@ -35,6 +35,14 @@ struct rrf_ctx {
   std::vector<cudaEvent_t> sync_events;  // fork/join events between the caller's stream and `aux`
   std::vector<cudaEvent_t> events;
   rrf_profile_t profile;
+  // rrf_run as a CUDA graph: captured on the second call with the same arguments, replayed after that
+  cudaStream_t cap;                      // stream the capture runs on (the caller's may be the legacy stream)
+  cudaGraph_t graph;
+  cudaGraphExec_t gexec;
+  std::vector<unsigned char> gkey;       // arguments the instantiated graph was captured for
+  std::vector<unsigned char> gcand;      // arguments of the last directly enqueued call
+  std::vector<std::pair<int, int>> gmarks;
+  int graph_off;                         // set when a capture failed: enqueue directly from then on
 };
 
 namespace rrf {
@@ -496,6 +504,10 @@ rrf_status_t rrf_create(rrf_handle_t* out, int device) {
   h->last_cuda = 0;
   h->profiling = 0;
   h->aux = nullptr;
+  h->cap = nullptr;
+  h->graph = nullptr;
+  h->gexec = nullptr;
+  h->graph_off = 0;
   std::memset(&h->profile, 0, sizeof(h->profile));
   cudaError_t e = cudaDeviceGetAttribute(&h->sms, cudaDevAttrMultiProcessorCount, device);
   if (e == cudaSuccess) e = cudaDeviceGetAttribute(&h->smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, device);
@@ -507,6 +519,7 @@ rrf_status_t rrf_create(rrf_handle_t* out, int device) {
   h->encode = reinterpret_cast<EncodeTiledFn>(fn);
   if (e == cudaSuccess) e = setup_all(h->smem_optin, &h->panel_smem_max);
   if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&h->aux, cudaStreamNonBlocking);
+  if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&h->cap, cudaStreamNonBlocking);
   if (e == cudaSuccess) e = cudaMalloc(&h->d_ctrl, sizeof(Ctrl));
   if (e == cudaSuccess) e = cudaMemset(h->d_ctrl, 0, sizeof(Ctrl));
   if (e != cudaSuccess) {
@@ -525,7 +538,10 @@ rrf_status_t rrf_destroy(rrf_handle_t h) {
   cudaFree(h->d_ctrl);
   for (cudaEvent_t ev : h->events) cudaEventDestroy(ev);
   for (cudaEvent_t ev : h->sync_events) cudaEventDestroy(ev);
+  if (h->gexec != nullptr) cudaGraphExecDestroy(h->gexec);
+  if (h->graph != nullptr) cudaGraphDestroy(h->graph);
   if (h->aux != nullptr) cudaStreamDestroy(h->aux);
+  if (h->cap != nullptr) cudaStreamDestroy(h->cap);
   delete h;
   return RRF_OK;
 }
@@ -786,7 +802,8 @@ rrf_status_t rrf_run(rrf_handle_t h, const rrf_params_t* p, void* dA, int64_t ld
   PanelPlan pp0;
   if (look_ctas == 0 && !plan_panel(h, m, b, &pp0)) return fail(RRF_ERR_WORKSPACE);   // tallest panel must fit on chip
 
-  cudaStream_t st = (cudaStream_t)cuda_stream;
+  cudaStream_t const user_st = (cudaStream_t)cuda_stream;
+  cudaStream_t st = user_st;
   if (cudaSetDevice(h->device) != cudaSuccess) return fail(RRF_ERR_CUDA);
   unsigned char* ws = (unsigned char*)d_workspace;
   Ctrl* ctrl = reinterpret_cast<Ctrl*>(ws + L.ctrl);
@@ -803,10 +820,15 @@ rrf_status_t rrf_run(rrf_handle_t h, const rrf_params_t* p, void* dA, int64_t ld
   void* Zt = ws + L.zt;
   PanelScratch ps = carve_panel(ws + L.panel, h->sms, b);
   ps.bar = &ctrl->bar;
-  if (look_ctas > 0 && cudaMemsetAsync(look_bar, 0, sizeof(unsigned), (cudaStream_t)cuda_stream) != cudaSuccess)
-    return fail(RRF_ERR_CUDA);
   const bool inplace = (p->flags & RRF_FLAG_INPLACE) != 0;
   const bool fixed = (p->flags & RRF_FLAG_FIXED_RANK) != 0;
+  std::vector<std::pair<int, int>> marks;   // profiling: (phase, block step) of every recorded event
+  size_t nev = 0;
+  bool capturing = false;
+  // Everything rrf_run puts on the device, on stream `st` (and the side stream, forked from and joined
+  // back to it): enqueued directly, or recorded into a CUDA graph.
+  auto enqueue = [&]() -> rrf_status_t {
+  if (look_ctas > 0 && cudaMemsetAsync(look_bar, 0, sizeof(unsigned), st) != cudaSuccess) return RRF_ERR_CUDA;
   void* W = inplace ? dA : (void*)(ws + L.w);
   const long long ldw = inplace ? lda : L.ldw;
   const void* Om = dOmegaT;
@@ -815,7 +837,7 @@ rrf_status_t rrf_run(rrf_handle_t h, const rrf_params_t* p, void* dA, int64_t ld
     Om = ws + L.omega;
     ldom = n;
     s = rrf_fill_omega(h, p->dtype, p->seed, n, p->max_rank, 0, ws + L.omega, n, st);
-    if (s != RRF_OK) return fail(s);
+    if (s != RRF_OK) return s;
   }
   const OpTable* ops = get_ops(p->dtype, b);
   const int npad = plan_vtw(h->sms, m, n, ops->v_bn).npad;
@@ -827,11 +849,9 @@ rrf_status_t rrf_run(rrf_handle_t h, const rrf_params_t* p, void* dA, int64_t ld
       !make_map(h, &tmV_u, p->dtype, dV, m, p->max_rank, ldv, ops->u_bm) ||
       !make_map(h, &tmW_u, p->dtype, W, m, n, ldw, ops->u_bm) ||
       !make_map(h, &tmZ, p->dtype, Zt, npad, b, b, ops->u_bn))
-    return fail(RRF_ERR_INVALID_ARG);
+    return RRF_ERR_INVALID_ARG;
 
   // profiling: one event before every kernel, tagged with (phase, block step)
-  std::vector<std::pair<int, int>> marks;
-  size_t nev = 0;
   auto mark = [&](int phase, int step) {
     if (!h->profiling) return;
     if (nev == h->events.size()) {
@@ -839,7 +859,7 @@ rrf_status_t rrf_run(rrf_handle_t h, const rrf_params_t* p, void* dA, int64_t ld
       if (cudaEventCreate(&ev) != cudaSuccess) return;
       h->events.push_back(ev);
     }
-    cudaEventRecord(h->events[nev++], st);
+    cudaEventRecordWithFlags(h->events[nev++], st, capturing ? cudaEventRecordExternal : cudaEventRecordDefault);
     marks.emplace_back(phase, step);
   };
 
@@ -857,16 +877,18 @@ rrf_status_t rrf_run(rrf_handle_t h, const rrf_params_t* p, void* dA, int64_t ld
   // fork/join events for the side stream, created once and kept in the handle
   while (h->sync_events.size() < (size_t)3 * steps + 2) {
     cudaEvent_t ev;
-    if (cudaEventCreateWithFlags(&ev, cudaEventDisableTiming) != cudaSuccess) return fail(RRF_ERR_CUDA);
+    if (cudaEventCreateWithFlags(&ev, cudaEventDisableTiming) != cudaSuccess) return RRF_ERR_CUDA;
     h->sync_events.push_back(ev);
   }
 
   // Algorithm 2 lines 5-11: every pass is enqueued; passes after the stop return at once.
   auto panel_failed = [&](rrf_status_t ps_status) {
     out->cuda_error = h->last_cuda;
-    cudaStreamSynchronize(st);
-    cudaStreamSynchronize(h->aux);
-    return fail(ps_status);
+    if (!capturing) {
+      cudaStreamSynchronize(st);
+      cudaStreamSynchronize(h->aux);
+    }
+    return ps_status;
   };
   void* const V0 = dV;
   auto Vblk = [&](int r0) { return (void*)((char*)V0 + ((size_t)r0 * ldv + r0) * esize); };
@@ -1013,6 +1035,79 @@ rrf_status_t rrf_run(rrf_handle_t h, const rrf_params_t* p, void* dA, int64_t ld
     }
   }
   mark(RRF_PHASE_SKIPPED, steps);   // closing event
+  return RRF_OK;
+  };
+
+  // The sequence of launches depends only on the arguments.  The first call with a given set is
+  // enqueued directly; if the next call repeats it, the sequence is captured into a graph, and every
+  // further repeat is one graph launch (no per-kernel launch cost on the host).
+  std::vector<unsigned char> key;
+  {
+    auto put = [&](const void* ptr, size_t nbytes) {
+      const unsigned char* c = static_cast<const unsigned char*>(ptr);
+      key.insert(key.end(), c, c + nbytes);
+    };
+    const void* ptrs[6] = {dA, dOmegaT, dV, dT, dB, d_workspace};
+    const long long lds[4] = {lda, ldo, ldv, ldb};
+    const char* ge = std::getenv("RRF_LOOKAHEAD_GATE");
+    const int ints[3] = {look_ctas, h->profiling, ge != nullptr ? 1 + std::atoi(ge) : 0};
+    put(p, sizeof(*p));
+    put(ptrs, sizeof(ptrs));
+    put(lds, sizeof(lds));
+    put(&workspace_bytes, sizeof(workspace_bytes));
+    put(ints, sizeof(ints));
+  }
+  const bool graphs_ok = !h->graph_off && !(p->flags & RRF_FLAG_NO_GRAPH);
+  bool launched = false;
+  if (graphs_ok && h->gexec != nullptr && key == h->gkey) {
+    marks = h->gmarks;
+    nev = marks.size();
+    launched = cudaGraphLaunch(h->gexec, user_st) == cudaSuccess;
+    if (!launched) h->graph_off = 1;
+  } else if (graphs_ok && key == h->gcand) {
+    if (h->gexec != nullptr) cudaGraphExecDestroy(h->gexec);
+    if (h->graph != nullptr) cudaGraphDestroy(h->graph);
+    h->gexec = nullptr;
+    h->graph = nullptr;
+    h->gkey.clear();
+    st = h->cap;
+    capturing = true;
+    rrf_status_t cs = RRF_ERR_CUDA;
+    if (cudaStreamBeginCapture(st, cudaStreamCaptureModeRelaxed) == cudaSuccess) {
+      cs = enqueue();
+      cudaGraph_t g = nullptr;
+      const cudaError_t ce = cudaStreamEndCapture(st, &g);
+      if (cs == RRF_OK && ce == cudaSuccess && g != nullptr &&
+          cudaGraphInstantiate(&h->gexec, g, 0) == cudaSuccess) {
+        h->graph = g;
+        h->gkey = key;
+        h->gmarks = marks;
+        launched = cudaGraphLaunch(h->gexec, user_st) == cudaSuccess;
+      } else if (g != nullptr) {
+        cudaGraphDestroy(g);
+      }
+    }
+    if (!launched) {               // capture is not available here: enqueue directly from now on
+      cudaGetLastError();
+      if (h->gexec != nullptr) cudaGraphExecDestroy(h->gexec);
+      if (h->graph != nullptr) cudaGraphDestroy(h->graph);
+      h->gexec = nullptr;
+      h->graph = nullptr;
+      h->gkey.clear();
+      h->graph_off = 1;
+      if (cs != RRF_OK && cs != RRF_ERR_CUDA) return fail(cs);
+    }
+    capturing = false;
+    st = user_st;
+  }
+  if (!launched) {
+    marks.clear();
+    nev = 0;
+    s = enqueue();
+    if (s != RRF_OK) return fail(s);
+    h->gcand = key;
+  }
+  st = user_st;
   cudaError_t e = cudaGetLastError();
   Ctrl hc;
   if (e == cudaSuccess) e = cudaMemcpyAsync(&hc, ctrl, sizeof(Ctrl), cudaMemcpyDeviceToHost, st);

@@ -16,7 +16,7 @@ import torch
 RRF_F64, RRF_F32 = 0, 1
 RRF_OK, RRF_MAX_RANK_REACHED = 0, 1
 RRF_ERR_INVALID_ARG, RRF_ERR_WORKSPACE, RRF_ERR_CUDA, RRF_ERR_TIMEOUT, RRF_ERR_NONFINITE = -1, -2, -3, -4, -5
-RRF_FLAG_INPLACE, RRF_FLAG_FIXED_RANK, RRF_FLAG_ONE_QUEUE, RRF_FLAG_TWO_QUEUES = 1, 2, 4, 8
+RRF_FLAG_INPLACE, RRF_FLAG_FIXED_RANK, RRF_FLAG_ONE_QUEUE, RRF_FLAG_TWO_QUEUES, RRF_FLAG_NO_GRAPH = 1, 2, 4, 8, 16
 
 _LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "librrf.so")
 _lib = None

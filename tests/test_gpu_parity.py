@@ -281,6 +281,35 @@ def test_runs_are_bitwise_reproducible(h):
     assert torch.equal(g1.B[:k], g2.B[:k]) and torch.equal(g1.V[:, :k], g2.V[:, :k]) and torch.equal(g1.T[:, :k], g2.T[:, :k])
 
 
+def test_graph_replay_follows_the_data(h):
+    # Repeating a call with the same buffers replays a captured CUDA graph (third call on); the replay
+    # must read the buffers' current contents and give what a direct enqueue gives, bit for bit.
+    w = wl.CONFIGS["cfg2"].scaled(m=1280, n=1024, max_rank=256)
+    A1, _ = wl.make_matrix(w)
+    A2 = np.ascontiguousarray(A1[::-1] * 0.5 + np.roll(A1, 7, axis=1))
+    Om = wl.make_omega(w)
+    dA = torch.empty((w.m, w.n), dtype=torch.float64, device="cuda")
+    dOmT = torch.from_numpy(np.ascontiguousarray(Om.T)).cuda()
+    p = rrf.make_params(rrf.RRF_F64, w.m, w.n, w.b, w.tol, w.max_rank)
+    ws = torch.empty(rrf.rrf_workspace_bytes(p), dtype=torch.uint8, device="cuda")
+    V = torch.empty((w.m, w.max_rank), dtype=torch.float64, device="cuda")
+    T = torch.empty((w.b, w.max_rank), dtype=torch.float64, device="cuda")
+    B = torch.empty((w.max_rank, w.n), dtype=torch.float64, device="cuda")
+
+    def run(A, flags):
+        dA.copy_(torch.from_numpy(A))
+        g = rrf.rrf_run(h, dA, w.b, w.tol, w.max_rank, omegaT=dOmT, V=V, T=T, B=B, workspace=ws, flags=flags)
+        return g.k, g.status, list(g.E_dir_trace), B[:g.k].clone(), V[:, :g.k].clone(), T[:, :g.k].clone()
+
+    for sched in (rrf.RRF_FLAG_ONE_QUEUE, rrf.RRF_FLAG_TWO_QUEUES):
+        ref1 = run(A1, sched | rrf.RRF_FLAG_NO_GRAPH)
+        ref2 = run(A2, sched | rrf.RRF_FLAG_NO_GRAPH)
+        for A, ref in ((A1, ref1), (A1, ref1), (A1, ref1), (A2, ref2), (A1, ref1), (A2, ref2)):
+            got = run(A, sched)          # direct, capture, then replays; the data changes under the graph
+            assert got[:3] == ref[:3]
+            assert all(torch.equal(x, y) for x, y in zip(got[3:], ref[3:]))
+
+
 def test_bounded_wait_times_out_and_context_survives(h):
     # a wait that nothing satisfies gives up after its limit and reports it; no trap, no hang
     assert rrf.rrf_selftest_timeout(h, 20.0) == rrf.RRF_ERR_TIMEOUT
