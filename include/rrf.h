@@ -103,12 +103,16 @@ rrf_status_t rrf_workspace_bytes(const rrf_params_t* p, size_t* bytes);
  *   dV       m x max_rank (ldv >= max_rank): Householder vectors, unit lower trapezoidal,
  *            block column i holds V_i in rows i*b.. and zeros above.  Columns >= k are
  *            unspecified on return.
- *   dT       b x max_rank, leading dimension max_rank: T_i (upper triangular) in columns i*b...
+ *   dT       b x max_rank, leading dimension max_rank: T_i (upper triangular) in columns i*b...;
+ *            columns >= k are unspecified on return (the look-ahead schedule factors one panel
+ *            past the stop).
  *   dB       max_rank x n (ldb >= n): rows 0..k-1 are B = Q^T A.  With RRF_FLAG_INPLACE,
  *            dB may alias dA (ldb == lda).
  *   d_workspace / workspace_bytes   at least rrf_workspace_bytes(), 256-byte aligned.
- *   cuda_stream   a cudaStream_t (NULL: the default stream).  All work is enqueued on it;
- *            the call synchronises it once, at the end, to read back the result.
+ *   cuda_stream   a cudaStream_t (NULL: the default stream).  All work is ordered after what
+ *            is on it and the call synchronises it once, at the end, to read back the result.
+ *            Part of the work runs on a stream the handle owns, forked from and joined back
+ *            to cuda_stream with events.
  *   h_E_sub_trace, h_E_dir_trace   optional HOST arrays of max_rank/b doubles receiving
  *            both stopping quantities after every block step.
  *
@@ -116,6 +120,17 @@ rrf_status_t rrf_workspace_bytes(const rrf_params_t* p, size_t* bytes);
  * reads a device flag and returns at once when the stop rule has fired, so there is no
  * host round-trip per block.  Returns RRF_OK / RRF_MAX_RANK_REACHED, or an error (out->status
  * is the same value).
+ *
+ * Schedule (Section "Implementation" of the paper, Figure "DAG").  One queue: panel QR, V^T W,
+ * T^T Z and the update follow one another.  Two queues: the panel of block i+1 is sampled one
+ * block early, corrected with block i's reflectors and factored on a few SMs while the update of
+ * block i runs on the others; this needs b <= 64 and a panel that fits in the shared memory of
+ * at most a third of the SMs.  The library picks the faster one for the sizes given; the flags
+ * RRF_FLAG_ONE_QUEUE / RRF_FLAG_TWO_QUEUES override that, and out->queues / out->panel_ctas say
+ * what ran.  The two schedules compute the same quantities up to rounding.
+ * A call whose arguments (parameters, pointers, leading dimensions, workspace) repeat those of
+ * the previous call on this handle is captured into a CUDA graph and replayed on later repeats;
+ * the buffers' CONTENTS may change freely between calls.  RRF_FLAG_NO_GRAPH disables this.
  */
 rrf_status_t rrf_run(rrf_handle_t h, const rrf_params_t* p,
                      void* dA, int64_t lda,
