@@ -341,119 +341,259 @@ __global__ void __launch_bounds__((WM * WN + (PW ? 1 : 0)) * 32, 1)
       const unsigned char* sZ = sW + W_BYTES;
       const unsigned char* sO = sZ + Z_BYTES;
 
-      // ---- P = V * Zt^T for this warp's rows and column groups
-      T acc[MT][QW][U][4];
+      if constexpr (sizeof(T) == 8) {
+        // ---- P = V * Zt^T for this warp's rows and column groups
+        T acc[MT][QW][U][4];
 #pragma unroll
-      for (int a = 0; a < MT; ++a)
-#pragma unroll
-        for (int q = 0; q < QW; ++q)
-#pragma unroll
-          for (int u = 0; u < U; ++u)
-#pragma unroll
-            for (int e = 0; e < 4; ++e) acc[a][q][u][e] = T(0);
-#pragma unroll
-      for (int kb = 0; kb < KB; ++kb) {
-#pragma unroll
-        for (int s2 = 0; s2 < 2; ++s2) {
-          T ra[MT][2][NV];
-#pragma unroll
-          for (int a = 0; a < MT; ++a) {
-            const int rlo = wm * TM + a * 16 + g;
-            const uint32_t chunk = ((uint32_t)(2 * t + s2) ^ (uint32_t)g) << 4;
-            VecLoad16<T>::ld(sVs + kb * V_BOX + rlo * 128 + chunk, ra[a][0]);
-            VecLoad16<T>::ld(sVs + kb * V_BOX + (rlo + 8) * 128 + chunk, ra[a][1]);
-          }
+        for (int a = 0; a < MT; ++a)
 #pragma unroll
           for (int q = 0; q < QW; ++q)
 #pragma unroll
-            for (int u = 0; u < U; ++u) {
-              // n-slot g of tile u is column (KE/4)*(g/2) + 2u + (g&1) of the group
-              const int zr = (wn * QW + q) * KE + (KE / 4) * (g >> 1) + 2 * u + (g & 1);
-              T rb[NV];
-              VecLoad16<T>::ld(sZ + kb * Z_BOX + zr * 128 + (((uint32_t)(2 * t + s2) ^ (uint32_t)(zr & 7)) << 4), rb);
+            for (int u = 0; u < U; ++u)
 #pragma unroll
-              for (int ks = 0; ks < KS; ++ks) {
-                const T bf[2] = {rb[2 * ks], rb[2 * ks + 1]};
+              for (int e = 0; e < 4; ++e) acc[a][q][u][e] = T(0);
 #pragma unroll
-                for (int a = 0; a < MT; ++a) {
-                  const T af[4] = {ra[a][0][2 * ks], ra[a][1][2 * ks], ra[a][0][2 * ks + 1], ra[a][1][2 * ks + 1]};
-                  mma16x8x8(acc[a][q][u], af, bf);
-                }
-              }
+        for (int kb = 0; kb < KB; ++kb) {
+#pragma unroll
+          for (int s2 = 0; s2 < 2; ++s2) {
+            T ra[MT][2][NV];
+#pragma unroll
+            for (int a = 0; a < MT; ++a) {
+              const int rlo = wm * TM + a * 16 + g;
+              const uint32_t chunk = ((uint32_t)(2 * t + s2) ^ (uint32_t)g) << 4;
+              VecLoad16<T>::ld(sVs + kb * V_BOX + rlo * 128 + chunk, ra[a][0]);
+              VecLoad16<T>::ld(sVs + kb * V_BOX + (rlo + 8) * 128 + chunk, ra[a][1]);
             }
-        }
-      }
-
-      // ---- Wnew = W - P: store, norms, and keep as the A operand of the sample product
-      const int col_base = c * BN;
-      const bool interior = col_base + BN <= ncols;      // no column guards needed
 #pragma unroll
-      for (int a = 0; a < MT; ++a)
+            for (int q = 0; q < QW; ++q)
 #pragma unroll
-        for (int q = 0; q < QW; ++q) {
-          const int grp = wn * QW + q;
-          const int col = col_base + grp * KE + (KE / 4) * t;   // first of this thread's KE/4 consecutive columns
+              for (int u = 0; u < U; ++u) {
+                // n-slot g of tile u is column (KE/4)*(g/2) + 2u + (g&1) of the group
+                const int zr = (wn * QW + q) * KE + (KE / 4) * (g >> 1) + 2 * u + (g & 1);
+                T rb[NV];
+                VecLoad16<T>::ld(sZ + kb * Z_BOX + zr * 128 + (((uint32_t)(2 * t + s2) ^ (uint32_t)(zr & 7)) << 4), rb);
 #pragma unroll
-          for (int h = 0; h < 2; ++h) {
-            const int rl = wm * TM + a * 16 + g + 8 * h;     // row inside the slab
-            T wv[2][NV];
+                for (int ks = 0; ks < KS; ++ks) {
+                  const T bf[2] = {rb[2 * ks], rb[2 * ks + 1]};
 #pragma unroll
-            for (int s2 = 0; s2 < 2; ++s2)
-              VecLoad16<T>::ld(sW + grp * W_BOX + rl * 128 + (((uint32_t)(2 * t + s2) ^ (uint32_t)g) << 4), wv[s2]);
-            T* dst = rowp[a][h];
-            double q0 = 0.0, q1 = 0.0;
-#pragma unroll
-            for (int s2 = 0; s2 < 2; ++s2)
-#pragma unroll
-              for (int ks = 0; ks < KS; ++ks) {
-                const int u = s2 * KS + ks;
-                const T y0 = wv[s2][2 * ks] - acc[a][q][u][2 * h];
-                const T y1 = wv[s2][2 * ks + 1] - acc[a][q][u][2 * h + 1];
-                acc[a][q][u][2 * h] = y0;
-                acc[a][q][u][2 * h + 1] = y1;
-                const int cc = col + 2 * u;
-                if (dst != nullptr) {
-                  if (interior || cc + 1 < ncols) {
-                    store2(dst + cc, y0, y1);
-                    q0 += (double)y0 * (double)y0;
-                    q1 += (double)y1 * (double)y1;
-                  } else if (cc < ncols) {
-                    dst[cc] = y0;
-                    q0 += (double)y0 * (double)y0;
+                  for (int a = 0; a < MT; ++a) {
+                    const T af[4] = {ra[a][0][2 * ks], ra[a][1][2 * ks], ra[a][0][2 * ks + 1], ra[a][1][2 * ks + 1]};
+                    mma16x8x8(acc[a][q][u], af, bf);
                   }
                 }
               }
-            const double qs = q0 + q1;
-            s_top += rtop[a][h] ? qs : 0.0;
-            s_trail += rtop[a][h] ? 0.0 : qs;
           }
         }
 
-      // ---- Y += Wnew * OmegaT^T (K = this warp's columns)
-      if (do_sample) {
+        // ---- Wnew = W - P: store, norms, and keep as the A operand of the sample product
+        const int col_base = c * BN;
+        const bool interior = col_base + BN <= ncols;      // no column guards needed
 #pragma unroll
-        for (int q = 0; q < QW; ++q) {
-          const int grp = wn * QW + q;
+        for (int a = 0; a < MT; ++a)
 #pragma unroll
-          for (int s2 = 0; s2 < 2; ++s2) {
+          for (int q = 0; q < QW; ++q) {
+            const int grp = wn * QW + q;
+            const int col = col_base + grp * KE + (KE / 4) * t;   // first of this thread's KE/4 consecutive columns
 #pragma unroll
-            for (int nb = 0; nb < NTB; ++nb) {
-              const int jr = nb * 8 + g;
-              T rb[NV];
-              VecLoad16<T>::ld(sO + grp * O_BOX + jr * 128 + (((uint32_t)(2 * t + s2) ^ (uint32_t)g) << 4), rb);
+            for (int h = 0; h < 2; ++h) {
+              const int rl = wm * TM + a * 16 + g + 8 * h;     // row inside the slab
+              T wv[2][NV];
 #pragma unroll
-              for (int ks = 0; ks < KS; ++ks) {
-                const int u = s2 * KS + ks;
-                const T bf[2] = {rb[2 * ks], rb[2 * ks + 1]};
+              for (int s2 = 0; s2 < 2; ++s2)
+                VecLoad16<T>::ld(sW + grp * W_BOX + rl * 128 + (((uint32_t)(2 * t + s2) ^ (uint32_t)g) << 4), wv[s2]);
+              T* dst = rowp[a][h];
+              double q0 = 0.0, q1 = 0.0;
 #pragma unroll
-                for (int a = 0; a < MT; ++a) {
-                  const T af[4] = {acc[a][q][u][0], acc[a][q][u][2], acc[a][q][u][1], acc[a][q][u][3]};
-                  mma16x8x8(accY[a][nb], af, bf);
+              for (int s2 = 0; s2 < 2; ++s2)
+#pragma unroll
+                for (int ks = 0; ks < KS; ++ks) {
+                  const int u = s2 * KS + ks;
+                  const T y0 = wv[s2][2 * ks] - acc[a][q][u][2 * h];
+                  const T y1 = wv[s2][2 * ks + 1] - acc[a][q][u][2 * h + 1];
+                  acc[a][q][u][2 * h] = y0;
+                  acc[a][q][u][2 * h + 1] = y1;
+                  const int cc = col + 2 * u;
+                  if (dst != nullptr) {
+                    if (interior || cc + 1 < ncols) {
+                      store2(dst + cc, y0, y1);
+                      q0 += (double)y0 * (double)y0;
+                      q1 += (double)y1 * (double)y1;
+                    } else if (cc < ncols) {
+                      dst[cc] = y0;
+                      q0 += (double)y0 * (double)y0;
+                    }
+                  }
+                }
+              const double qs = q0 + q1;
+              s_top += rtop[a][h] ? qs : 0.0;
+              s_trail += rtop[a][h] ? 0.0 : qs;
+            }
+          }
+
+        // ---- Y += Wnew * OmegaT^T (K = this warp's columns)
+        if (do_sample) {
+#pragma unroll
+          for (int q = 0; q < QW; ++q) {
+            const int grp = wn * QW + q;
+#pragma unroll
+            for (int s2 = 0; s2 < 2; ++s2) {
+#pragma unroll
+              for (int nb = 0; nb < NTB; ++nb) {
+                const int jr = nb * 8 + g;
+                T rb[NV];
+                VecLoad16<T>::ld(sO + grp * O_BOX + jr * 128 + (((uint32_t)(2 * t + s2) ^ (uint32_t)g) << 4), rb);
+#pragma unroll
+                for (int ks = 0; ks < KS; ++ks) {
+                  const int u = s2 * KS + ks;
+                  const T bf[2] = {rb[2 * ks], rb[2 * ks + 1]};
+#pragma unroll
+                  for (int a = 0; a < MT; ++a) {
+                    const T af[4] = {acc[a][q][u][0], acc[a][q][u][2], acc[a][q][u][1], acc[a][q][u][3]};
+                    mma16x8x8(accY[a][nb], af, bf);
+                  }
                 }
               }
             }
           }
         }
+      } else {
+        // The tile runs as a pipeline over this warp's QW column groups so that the tensor pipe always
+        // has a product to work on while the element-wise part of another group is in flight:
+        //   VZ(0) | VZ(1) + EPI(0) | S(0) + EPI(1) | S(1)          (QW = 2)
+        // Single precision only (three TF32 products and their splitting per MMA leave issue slots for
+        // this to pay: 11 % on the 4096 x 11008 workload); in double precision the plain order above is
+        // faster by 4 %.
+        // VZ(q): P = V * Zt^T for group q.  EPI(q): Wnew = W - P, store, norms (2 MT pieces, one per 8
+        // rows).  S(q): Y += Wnew * OmegaT^T with the accumulator fragment of Wnew as the A operand.
+        // The pieces of EPI are placed between the unrolled MMA iterations of the neighbouring product.
+        T acc[MT][QW][U][4];
+        const int col_base = c * BN;
+        const bool interior = col_base + BN <= ncols;      // no column guards needed
+        constexpr int NP = 2 * MT;                          // pieces of one group's epilogue
+#define RRF_VZ_ITER(qa_, qb_, it_)                                                                                   \
+        {                                                                                                         \
+          const int kb_ = (it_) >> 1, s2_ = (it_) & 1;                                                            \
+          T ra_[MT][2][NV];                                                                                       \
+          _Pragma("unroll") for (int a = 0; a < MT; ++a) {                                                        \
+            const int rlo = wm * TM + a * 16 + g;                                                                 \
+            const uint32_t chunk = ((uint32_t)(2 * t + s2_) ^ (uint32_t)g) << 4;                                  \
+            VecLoad16<T>::ld(sVs + kb_ * V_BOX + rlo * 128 + chunk, ra_[a][0]);                                   \
+            VecLoad16<T>::ld(sVs + kb_ * V_BOX + (rlo + 8) * 128 + chunk, ra_[a][1]);                             \
+          }                                                                                                       \
+          _Pragma("unroll") for (int q_ = (qa_); q_ < (qb_); ++q_)                                                \
+          _Pragma("unroll") for (int u = 0; u < U; ++u) {                                                         \
+            /* n-slot g of tile u is column (KE/4)*(g/2) + 2u + (g&1) of the group */                             \
+            const int zr = (wn * QW + (q_)) * KE + (KE / 4) * (g >> 1) + 2 * u + (g & 1);                         \
+            T rb_[NV];                                                                                            \
+            VecLoad16<T>::ld(sZ + kb_ * Z_BOX + zr * 128 + (((uint32_t)(2 * t + s2_) ^ (uint32_t)(zr & 7)) << 4), rb_); \
+            _Pragma("unroll") for (int ks = 0; ks < KS; ++ks) {                                                   \
+              const T bf[2] = {rb_[2 * ks], rb_[2 * ks + 1]};                                                     \
+              _Pragma("unroll") for (int a = 0; a < MT; ++a) {                                                    \
+                const T af[4] = {ra_[a][0][2 * ks], ra_[a][1][2 * ks], ra_[a][0][2 * ks + 1], ra_[a][1][2 * ks + 1]}; \
+                mma16x8x8(acc[a][q_][u], af, bf);                                                                 \
+              }                                                                                                   \
+            }                                                                                                     \
+          }                                                                                                       \
+        }
+#define RRF_EPI_PIECE(q_, e_)                                                                                  \
+        {                                                                                                         \
+          const int a_ = (e_) >> 1, h_ = (e_) & 1;                                                                \
+          const int grp = wn * QW + (q_);                                                                         \
+          const int col = col_base + grp * KE + (KE / 4) * t;   /* first of this thread's KE/4 consecutive columns */ \
+          const int rl = wm * TM + a_ * 16 + g + 8 * h_;        /* row inside the slab */                         \
+          T wv[2][NV];                                                                                            \
+          _Pragma("unroll") for (int s2 = 0; s2 < 2; ++s2)                                                        \
+            VecLoad16<T>::ld(sW + grp * W_BOX + rl * 128 + (((uint32_t)(2 * t + s2) ^ (uint32_t)g) << 4), wv[s2]); \
+          T* dst = rowp[a_][h_];                                                                                  \
+          double q0 = 0.0, q1 = 0.0;                                                                              \
+          _Pragma("unroll") for (int s2 = 0; s2 < 2; ++s2)                                                        \
+            _Pragma("unroll") for (int ks = 0; ks < KS; ++ks) {                                                   \
+              const int u = s2 * KS + ks;                                                                         \
+              const T y0 = wv[s2][2 * ks] - acc[a_][q_][u][2 * h_];                                               \
+              const T y1 = wv[s2][2 * ks + 1] - acc[a_][q_][u][2 * h_ + 1];                                       \
+              acc[a_][q_][u][2 * h_] = y0;                                                                        \
+              acc[a_][q_][u][2 * h_ + 1] = y1;                                                                    \
+              const int cc = col + 2 * u;                                                                         \
+              if (dst != nullptr) {                                                                               \
+                if (interior || cc + 1 < ncols) {                                                                 \
+                  store2(dst + cc, y0, y1);                                                                       \
+                  q0 += (double)y0 * (double)y0;                                                                  \
+                  q1 += (double)y1 * (double)y1;                                                                  \
+                } else if (cc < ncols) {                                                                          \
+                  dst[cc] = y0;                                                                                   \
+                  q0 += (double)y0 * (double)y0;                                                                  \
+                }                                                                                                 \
+              }                                                                                                   \
+            }                                                                                                     \
+          const double qs = q0 + q1;                                                                              \
+          s_top += rtop[a_][h_] ? qs : 0.0;                                                                       \
+          s_trail += rtop[a_][h_] ? 0.0 : qs;                                                                     \
+        }
+#define RRF_S_ITER(q_, it_)                                                                                    \
+        {                                                                                                         \
+          const int s2_ = (it_) / NTB, nb_ = (it_) % NTB;                                                         \
+          const int grp = wn * QW + (q_);                                                                         \
+          const int jr = nb_ * 8 + g;                                                                             \
+          T rb_[NV];                                                                                              \
+          VecLoad16<T>::ld(sO + grp * O_BOX + jr * 128 + (((uint32_t)(2 * t + s2_) ^ (uint32_t)g) << 4), rb_);    \
+          _Pragma("unroll") for (int ks = 0; ks < KS; ++ks) {                                                     \
+            const int u = s2_ * KS + ks;                                                                          \
+            const T bf[2] = {rb_[2 * ks], rb_[2 * ks + 1]};                                                       \
+            _Pragma("unroll") for (int a = 0; a < MT; ++a) {                                                      \
+              const T af[4] = {acc[a][q_][u][0], acc[a][q_][u][2], acc[a][q_][u][1], acc[a][q_][u][3]};           \
+              mma16x8x8(accY[a][nb_], af, bf);                                                                    \
+            }                                                                                                     \
+          }                                                                                                       \
+        }
+#pragma unroll
+        for (int a = 0; a < MT; ++a)
+#pragma unroll
+          for (int q = 0; q < QW; ++q)
+#pragma unroll
+            for (int u = 0; u < U; ++u)
+#pragma unroll
+              for (int e = 0; e < 4; ++e) acc[a][q][u][e] = T(0);
+        constexpr int NVZ = 2 * KB, NSI = 2 * NTB;          // unrolled iterations of VZ and of S(q)
+        static_assert(QW == 1 || QW == 2, "column groups per warp");
+          constexpr bool kSplitVZ = true;
+        if (QW == 2 && kSplitVZ) {
+#pragma unroll
+          for (int it = 0; it < NVZ; ++it) RRF_VZ_ITER(0, 1, it)
+#pragma unroll
+          for (int it = 0; it < NVZ; ++it) {
+            RRF_VZ_ITER(QW - 1, QW, it)
+#pragma unroll
+            for (int e = 0; e < NP; ++e)
+              if (it == (((e + 1) * NVZ) / (NP + 1) > 0 ? ((e + 1) * NVZ) / (NP + 1) - 1 : 0)) RRF_EPI_PIECE(0, e)
+          }
+        } else {
+#pragma unroll
+          for (int it = 0; it < NVZ; ++it) RRF_VZ_ITER(0, QW, it)
+#pragma unroll
+          for (int e = 0; e < NP; ++e) RRF_EPI_PIECE(0, e)
+        }
+        if (QW == 2 && !do_sample) {
+#pragma unroll
+          for (int e = 0; e < NP; ++e) RRF_EPI_PIECE(QW - 1, e)
+        }
+        if (do_sample) {
+#pragma unroll
+          for (int it = 0; it < NSI; ++it) {
+            RRF_S_ITER(0, it)
+            if (QW == 2) {
+#pragma unroll
+              for (int e = 0; e < NP; ++e)
+                if (it == ((e + 1) * NSI) / (NP + 1) - 1) RRF_EPI_PIECE(QW - 1, e)
+            }
+          }
+          if (QW == 2) {
+#pragma unroll
+            for (int it = 0; it < NSI; ++it) RRF_S_ITER(QW - 1, it)
+          }
+        }
+#undef RRF_VZ_ITER
+#undef RRF_EPI_PIECE
+#undef RRF_S_ITER
       }
       __syncwarp();
       if (lane == 0) mbar_arrive(&empty[st]);
