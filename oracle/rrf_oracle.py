@@ -208,6 +208,14 @@ def permuted_rerun(A, Omega, b, tol, max_rank, seed=0, **kw) -> OracleResult:
     return res
 
 
+def subspace_transfer(V_old, T_old, V_new, T_new, b: int, M: np.ndarray) -> np.ndarray:
+    """Section "Towards Efficient Low-Rank Deep Learning": an optimiser state M (k_old x n) held in the
+    basis Q_old is replaced by Q_new^T Q_old M (k_new x n).  Written out with the explicit bases."""
+    Q_old = form_q(V_old, T_old, b)
+    Q_new = form_q(V_new, T_new, b)
+    return Q_new.T @ (Q_old @ np.asarray(M, dtype=np.float64))
+
+
 def form_q(V: np.ndarray, T: np.ndarray, b: int) -> np.ndarray:
     """Explicit Q = (Q_0 ... Q_{i-1}) I[:, 0:k]  (Algorithm 2, Ensure line)."""
     m, k = V.shape

@@ -230,3 +230,38 @@ def test_fp32_subtractive_estimator_stops_tracking_near_384():
     Q = orc.form_q(r.V.astype(np.float64), r.T.astype(np.float64), b)
     assert np.linalg.norm(Q.T @ Q - np.eye(640), 2) < 5e-6
     assert np.linalg.norm(A - Q @ (Q.T @ A), 2) < 2e-6
+
+
+def test_subspace_transfer_pins():
+    """Q_new^T Q_old M: identity when the bases coincide, an isometry that pads with zeros when the new
+    basis extends the old one, and equal to the same product with bases taken from LAPACK's QR."""
+    import scipy.linalg as sla
+    rng = np.random.default_rng(77)
+    m, n, b = 240, 150, 16
+    A = rng.standard_normal((m, 40)) @ rng.standard_normal((40, n))
+    Om = rng.standard_normal((n, 64))
+    small = orc.rrf(A, Om, b, 0.0, 32)
+    large = orc.rrf(A, Om, b, 0.0, 64)
+    M = rng.standard_normal((32, 70))
+    same = orc.subspace_transfer(small.V, small.T, small.V, small.T, b, M)
+    assert np.max(np.abs(same - M)) < 1e-13
+    # the first 32 basis vectors of the longer run are the basis of the shorter one
+    ext = orc.subspace_transfer(small.V, small.T, large.V, large.T, b, M)
+    assert ext.shape == (64, 70)
+    assert np.max(np.abs(ext[:32] - M)) < 1e-12 and np.max(np.abs(ext[32:])) < 1e-12
+    # unrelated bases: against thin Q factors from LAPACK (sign-fixed to the Householder convention)
+    A2 = rng.standard_normal((m, n))
+    other = orc.rrf(A2, Om, b, 0.0, 48)
+
+    def lapack_basis(Amat, k):
+        Q, R = sla.qr(Amat @ Om[:, :k], mode="economic")
+        return Q
+
+    Qo, Qn = lapack_basis(A, 32), lapack_basis(A2, 48)
+    # geqrf and the blocked run span the same subspaces and agree column by column up to sign
+    So = np.sign(np.sum(Qo * orc.form_q(small.V, small.T, b), axis=0))
+    Sn = np.sign(np.sum(Qn * orc.form_q(other.V, other.T, b), axis=0))
+    want = (Qn * Sn).T @ ((Qo * So) @ M)
+    got = orc.subspace_transfer(small.V, small.T, other.V, other.T, b, M)
+    assert got.shape == (48, 70)
+    assert np.max(np.abs(got - want)) < 1e-9 * np.max(np.abs(want))
