@@ -210,6 +210,28 @@ rrf_status_t rrf_form_q(rrf_handle_t h, int32_t dtype, int64_t m, int32_t b, int
                         void* d_workspace, size_t workspace_bytes, void* cuda_stream);
 
 /*
+ * rrf_subspace_transfer - the subspace-consistency transform of the paper's Section "Towards
+ * Efficient Low-Rank Deep Learning": a low-rank optimiser state M (k_old x ncols) held in the basis
+ * Q_old of the previous step is re-expressed in the current basis Q_new,
+ *     Mout (k_new x ncols) = Q_new^T (Q_old M),
+ * both bases given by their reflectors (V m x k, T b x k) as rrf_run returns them, for the same m
+ * and b; k_old and k_new may differ (the adaptive ranks of two training steps).  Computed as
+ * [M; 0] (m x ncols) -> Q_old [M; 0] -> Q_new^T (.) -> first k_new rows, with the same kernels as
+ * rrf_apply_q / rrf_apply_qt.  M and Mout are device matrices (ldm, ldmo >= ncols, 16-byte aligned
+ * rows); they may not overlap.  Workspace: rrf_transfer_workspace_bytes(), 256-byte aligned.  Does
+ * not synchronise the stream.
+ */
+rrf_status_t rrf_transfer_workspace_bytes(int32_t dtype, int64_t m, int64_t ncols, int32_t b, size_t* bytes);
+rrf_status_t rrf_subspace_transfer(rrf_handle_t h, int32_t dtype, int64_t m, int32_t b,
+                                   int32_t k_old, const void* dV_old, int64_t ldv_old,
+                                   const void* dT_old, int64_t ldt_old,
+                                   int32_t k_new, const void* dV_new, int64_t ldv_new,
+                                   const void* dT_new, int64_t ldt_new,
+                                   const void* dM, int64_t ldm, int64_t ncols,
+                                   void* dMout, int64_t ldmo,
+                                   void* d_workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
  * rrf_fill_omega - Algorithm 2 line 6: fill dOmegaT (nvec x n, ldo >= n) with i.i.d. standard
  * Gaussians.  Counter-based: element (j, c) depends only on (seed, j, c) - Philox-4x32-10 keyed
  * by the seed with counter (c/2, j), Box-Muller in double precision, rounded to dtype - so any

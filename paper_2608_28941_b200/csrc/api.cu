@@ -750,6 +750,56 @@ rrf_status_t rrf_form_q(rrf_handle_t h, int32_t dtype, int64_t m, int32_t b, int
   return apply_blocks(h, dtype, m, b, k, dV, ldv, dT, ldt, dQ, ldq, k, d_workspace, workspace_bytes, st, false);
 }
 
+rrf_status_t rrf_transfer_workspace_bytes(int32_t dtype, int64_t m, int64_t ncols, int32_t b, size_t* bytes) {
+  size_t apply = 0;
+  const rrf_status_t s = rrf_apply_workspace_bytes(dtype, m, ncols, b, &apply);
+  if (s != RRF_OK) return s;
+  const int esize = dtype == RRF_F64 ? 8 : 4;
+  *bytes = align_up((size_t)m * align_up((size_t)ncols, 16) * esize, 256) + apply;
+  return RRF_OK;
+}
+
+rrf_status_t rrf_subspace_transfer(rrf_handle_t h, int32_t dtype, int64_t m, int32_t b, int32_t k_old,
+                                   const void* dV_old, int64_t ldv_old, const void* dT_old, int64_t ldt_old,
+                                   int32_t k_new, const void* dV_new, int64_t ldv_new, const void* dT_new,
+                                   int64_t ldt_new, const void* dM, int64_t ldm, int64_t ncols, void* dMout,
+                                   int64_t ldmo, void* d_workspace, size_t workspace_bytes, void* cuda_stream) {
+  if (h == nullptr || dM == nullptr || dMout == nullptr || d_workspace == nullptr) return RRF_ERR_INVALID_ARG;
+  if (!b_ok(dtype, b) || k_old < 1 || k_new < 1 || k_old > m || k_new > m || ncols < 1 || ldm < ncols || ldmo < ncols)
+    return RRF_ERR_INVALID_ARG;
+  size_t need = 0;
+  if (rrf_transfer_workspace_bytes(dtype, m, ncols, b, &need) != RRF_OK) return RRF_ERR_INVALID_ARG;
+  if (workspace_bytes < need || (reinterpret_cast<uintptr_t>(d_workspace) & 255u)) return RRF_ERR_WORKSPACE;
+  const int esize = dtype == RRF_F64 ? 8 : 4;
+  const long long ldc = (long long)align_up((size_t)ncols, 16);
+  const size_t cbytes = align_up((size_t)m * ldc * esize, 256);
+  unsigned char* ws = (unsigned char*)d_workspace;
+  void* Cm = ws;
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  const int grid = (int)std::min<long long>(((long long)m * ncols + 255) / 256, (long long)h->sms * 16);
+  if (dtype == RRF_F64)
+    copy_rows_kernel<double><<<grid, 256, 0, st>>>((double*)Cm, ldc, (const double*)dM, ldm, k_old, m, ncols);
+  else
+    copy_rows_kernel<float><<<grid, 256, 0, st>>>((float*)Cm, ldc, (const float*)dM, ldm, k_old, m, ncols);
+  rrf_status_t s = apply_blocks(h, dtype, m, b, k_old, dV_old, ldv_old, dT_old, ldt_old, Cm, ldc, ncols, ws + cbytes,
+                                workspace_bytes - cbytes, st, false);
+  if (s != RRF_OK) return s;
+  s = apply_blocks(h, dtype, m, b, k_new, dV_new, ldv_new, dT_new, ldt_new, Cm, ldc, ncols, ws + cbytes,
+                   workspace_bytes - cbytes, st, true);
+  if (s != RRF_OK) return s;
+  const int grid2 = (int)std::min<long long>(((long long)k_new * ncols + 255) / 256, (long long)h->sms * 16);
+  if (dtype == RRF_F64)
+    copy_rows_kernel<double><<<grid2, 256, 0, st>>>((double*)dMout, ldmo, (const double*)Cm, ldc, k_new, k_new, ncols);
+  else
+    copy_rows_kernel<float><<<grid2, 256, 0, st>>>((float*)dMout, ldmo, (const float*)Cm, ldc, k_new, k_new, ncols);
+  const cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) {
+    h->last_cuda = (int)e;
+    return RRF_ERR_CUDA;
+  }
+  return RRF_OK;
+}
+
 rrf_status_t rrf_run(rrf_handle_t h, const rrf_params_t* p, void* dA, int64_t lda, const void* dOmegaT, int64_t ldo,
                      void* dV, int64_t ldv, void* dT, void* dB, int64_t ldb, void* d_workspace, size_t workspace_bytes,
                      void* cuda_stream, rrf_result_t* out, double* h_E_sub_trace, double* h_E_dir_trace) {

@@ -838,4 +838,16 @@ __global__ void __launch_bounds__(256) eye_kernel(T* __restrict__ Q, long long l
   }
 }
 
+// dst (rows_total x ncols) <- first rows_copy rows of src, zeros below
+template <typename T>
+__global__ void __launch_bounds__(256)
+    copy_rows_kernel(T* __restrict__ dst, long long ldd, const T* __restrict__ src, long long lds, long long rows_copy,
+                     long long rows_total, long long ncols) {
+  const long long total = rows_total * ncols;
+  for (long long idx = (long long)blockIdx.x * 256 + threadIdx.x; idx < total; idx += (long long)gridDim.x * 256) {
+    const long long r = idx / ncols, c = idx - r * ncols;
+    dst[r * ldd + c] = r < rows_copy ? src[r * lds + c] : T(0);
+  }
+}
+
 }  // namespace rrf

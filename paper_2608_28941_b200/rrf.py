@@ -41,7 +41,7 @@ class rrf_profile_t(C.Structure):
     _fields_ = [("ms", C.c_double * 9), ("launches", C.c_int32 * 9), ("pad", C.c_int32)]
 
 
-EXPORTS = ["rrf_selftest_timeout", "rrf_panel_qr_static", "rrf_set_profiling", "rrf_get_profile", "rrf_measure_peak", "rrf_create", "rrf_destroy", "rrf_workspace_bytes", "rrf_run", "rrf_panel_workspace_bytes",
+EXPORTS = ["rrf_transfer_workspace_bytes", "rrf_subspace_transfer", "rrf_selftest_timeout", "rrf_panel_qr_static", "rrf_set_profiling", "rrf_get_profile", "rrf_measure_peak", "rrf_create", "rrf_destroy", "rrf_workspace_bytes", "rrf_run", "rrf_panel_workspace_bytes",
            "rrf_panel_qr", "rrf_apply_workspace_bytes", "rrf_apply_qt", "rrf_apply_q", "rrf_form_q",
            "rrf_fill_omega", "rrf_last_status", "rrf_status_string"]
 
@@ -69,6 +69,9 @@ def load():
         f.argtypes = [vp, i32, i64, i32, i32, vp, i64, vp, i64, vp, i64, i64, vp, sz, vp]
     lib.rrf_form_q.argtypes = [vp, i32, i64, i32, i32, vp, i64, vp, i64, vp, i64, vp, sz, vp]
     lib.rrf_fill_omega.argtypes = [vp, i32, u64, i64, i32, i32, vp, i64, vp]
+    lib.rrf_transfer_workspace_bytes.argtypes = [i32, i64, i64, i32, C.POINTER(sz)]
+    lib.rrf_subspace_transfer.argtypes = [vp, i32, i64, i32, i32, vp, i64, vp, i64, i32, vp, i64, vp, i64, vp, i64, i64,
+                                          vp, i64, vp, sz, vp]
     lib.rrf_last_status.argtypes = [vp, vp]
     lib.rrf_selftest_timeout.argtypes = [vp, C.c_double, vp]
     lib.rrf_set_profiling.argtypes = [vp, i32]
@@ -282,6 +285,30 @@ def rrf_form_q(h, V: torch.Tensor, T: torch.Tensor, b: int, k: int) -> torch.Ten
         raise RrfError(s, "rrf_form_q")
     torch.cuda.current_stream().synchronize()
     return Q
+
+
+def rrf_subspace_transfer(h, V_old, T_old, k_old: int, V_new, T_new, k_new: int, b: int, M: torch.Tensor) -> torch.Tensor:
+    """Mout (k_new x n) = Q_new^T (Q_old M) for M (k_old x n)."""
+    lib = load()
+    m, ncols = V_old.shape[0], M.shape[1]
+    dt = _dtype_code(M)
+    out = _empty(k_new, ncols, M.dtype, M.device)
+    need = C.c_size_t()
+    s = lib.rrf_transfer_workspace_bytes(dt, m, ncols, b, C.byref(need))
+    if s != RRF_OK:
+        raise RrfError(s, "rrf_transfer_workspace_bytes")
+    ws = torch.empty(need.value, dtype=torch.uint8, device=M.device)
+    s = lib.rrf_subspace_transfer(h, dt, m, b, k_old, C.c_void_p(V_old.data_ptr()), _rowmajor(V_old, "V_old"),
+                                  C.c_void_p(T_old.data_ptr()), _rowmajor(T_old, "T_old"), k_new,
+                                  C.c_void_p(V_new.data_ptr()), _rowmajor(V_new, "V_new"),
+                                  C.c_void_p(T_new.data_ptr()), _rowmajor(T_new, "T_new"),
+                                  C.c_void_p(M.data_ptr()), _rowmajor(M, "M"), ncols,
+                                  C.c_void_p(out.data_ptr()), _rowmajor(out, "Mout"), C.c_void_p(ws.data_ptr()),
+                                  ws.numel(), _stream())
+    if s != RRF_OK:
+        raise RrfError(s, "rrf_subspace_transfer")
+    torch.cuda.current_stream().synchronize()
+    return out
 
 
 def rrf_fill_omega(h, n: int, nvec: int, seed: int, dtype=torch.float64, first_vec: int = 0,

@@ -169,6 +169,25 @@ def test_apply_and_form_q_match_oracle(h, m, ncols, b, k, dtype):
     assert relmax(Q, orc.form_q(o.V, o.T, b)) <= tol
 
 
+@pytest.mark.parametrize("m,n,b,k_old,k_new,ncols,dtype", [(700, 400, 16, 48, 80, 333, "f64"),
+                                                          (1500, 900, 64, 192, 128, 1000, "f64"),
+                                                          (1024, 640, 32, 96, 96, 520, "f32")])
+def test_subspace_transfer_matches_oracle(h, m, n, b, k_old, k_new, ncols, dtype):
+    # the bases of two unrelated matrices (two "training steps"), different ranks
+    rng = np.random.default_rng(m + k_old)
+    Om = rng.standard_normal((n, max(k_old, k_new)))
+    old = orc.rrf(rng.standard_normal((m, n)), Om, b, 0.0, k_old)
+    new = orc.rrf(rng.standard_normal((m, n)), Om, b, 0.0, k_new)
+    M = rng.standard_normal((k_old, ncols))
+    npdt = np.float64 if dtype == "f64" else np.float32
+    mult = 2 if dtype == "f64" else 4
+    dev = lambda x: _pad_cols(np.ascontiguousarray(x.astype(npdt)), mult)
+    got = rrf.rrf_subspace_transfer(h, dev(old.V), dev(old.T), k_old, dev(new.V), dev(new.T), k_new, b, dev(M))
+    want = orc.subspace_transfer(old.V, old.T, new.V, new.T, b, M)
+    assert got.shape == (k_new, ncols)
+    assert relmax(got.cpu().numpy().astype(np.float64), want) <= (1e-12 if dtype == "f64" else 3e-5)
+
+
 # ------------------------------------------------------------------ whole runs
 
 
