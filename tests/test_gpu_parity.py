@@ -329,6 +329,34 @@ def test_graph_replay_follows_the_data(h):
             assert all(torch.equal(x, y) for x, y in zip(got[3:], ref[3:]))
 
 
+def test_runs_on_a_caller_stream(h):
+    # all work is ordered on the caller's stream, also when the launches come from a replayed graph:
+    # the input is produced on that stream right before the call and the output consumed right after
+    w = wl.CONFIGS["cfg2"].scaled(m=1024, n=896, max_rank=192)
+    A, _ = wl.make_matrix(w)
+    Om = wl.make_omega(w)
+    dOmT = torch.from_numpy(np.ascontiguousarray(Om.T)).cuda()
+    dA0 = torch.from_numpy(A).cuda()
+    ref = rrf.rrf_run(h, dA0, w.b, w.tol, w.max_rank, omegaT=dOmT, flags=rrf.RRF_FLAG_NO_GRAPH)
+    refB = ref.B[:ref.k].clone()
+    p = rrf.make_params(rrf.RRF_F64, w.m, w.n, w.b, w.tol, w.max_rank)
+    ws = torch.empty(rrf.rrf_workspace_bytes(p), dtype=torch.uint8, device="cuda")
+    V = torch.empty((w.m, w.max_rank), dtype=torch.float64, device="cuda")
+    T = torch.empty((w.b, w.max_rank), dtype=torch.float64, device="cuda")
+    B = torch.empty((w.max_rank, w.n), dtype=torch.float64, device="cuda")
+    dA = torch.empty_like(dA0)
+    side = torch.cuda.Stream()
+    torch.cuda.synchronize()
+    with torch.cuda.stream(side):
+        for _ in range(4):
+            dA.zero_()
+            dA.add_(dA0)                 # the input only exists once this has run on `side`
+            g = rrf.rrf_run(h, dA, w.b, w.tol, w.max_rank, omegaT=dOmT, V=V, T=T, B=B, workspace=ws)
+            out = B[:g.k] * 1.0          # consumer on the same stream
+            assert g.k == ref.k and torch.equal(out, refB)
+    torch.cuda.synchronize()
+
+
 def test_bounded_wait_times_out_and_context_survives(h):
     # a wait that nothing satisfies gives up after its limit and reports it; no trap, no hang
     assert rrf.rrf_selftest_timeout(h, 20.0) == rrf.RRF_ERR_TIMEOUT
