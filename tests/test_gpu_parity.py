@@ -376,6 +376,15 @@ def test_invalid_arguments_are_rejected(h):
     odd = torch.randn((128, 97), dtype=torch.float64, device="cuda")       # ld = 97 doubles: not 16-byte rows
     with pytest.raises(rrf.RrfError):
         rrf.rrf_run(h, odd, 16, 1e-3, 32)
+    # a panel taller than the SMs' shared memory holds is refused before anything is launched
+    tall = torch.zeros((40000, 128), dtype=torch.float64, device="cuda")
+    with pytest.raises(rrf.RrfError) as e:
+        rrf.rrf_panel_qr(h, tall)
+    assert e.value.status == rrf.RRF_ERR_WORKSPACE
+    assert rrf.rrf_last_status(h) == rrf.RRF_OK
+    # the tallest panel of the largest configuration (32768 x 128) does fit
+    V, T = rrf.rrf_panel_qr(h, torch.randn((32768, 128), dtype=torch.float64, device="cuda"))
+    assert torch.isfinite(V).all() and float(V[0, 0]) == 1.0 and torch.count_nonzero(torch.triu(V[:128], 1)) == 0
 
 
 # ------------------------------------------------------------------ built-in Gaussian generator
