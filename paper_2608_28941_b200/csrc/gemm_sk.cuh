@@ -1,6 +1,7 @@
 // Persistent ("stream-K") versions of the two large contractions of a block step.
 //
-// Both kernels run one CTA per SM.  The tiles of the problem are numbered along the
+// Both kernels run one CTA per SM they are given (every SM under the sequential schedule; all but the
+// SMs of the panel kernel under the look-ahead schedule, where they run beside it).  The tiles of the problem are numbered along the
 // direction in which an accumulator can stay in registers, and CTA p owns the contiguous
 // range [p*tpc, (p+1)*tpc) of them, so every SM gets the same amount of work whatever the
 // trailing matrix's height.  When a CTA's range crosses from one accumulator to the next it
@@ -9,13 +10,14 @@
 // consumer of the partials (panel loader, Z reduction) sums the slots of one accumulator in
 // CTA order - a fixed order, so results are reproducible bit for bit.
 //
-// One extra warp per CTA only issues TMA loads; the consumer warps never wait for each other
-// (full/empty mbarriers per stage, every wait bounded).
+// TMA loads are issued by one extra warp (vtw) or by one lane of the first warp (upd); the consumer
+// warps never wait for each other (full/empty mbarriers per stage, every wait bounded).
 //
 //   vtw_sk_kernel   Z = V_i^T W[r0:, :]                      (Algorithm 2 line 8, first product)
 //   upd_sk_kernel   W[r0:, :] -= V_i Zt^T, norms of line 9, and - fused, from the updated tile
-//                   still in registers - the next panel Y = W_new Omega_{i+1} (line 7 of the
-//                   next pass), which saves one full read of W per block step.
+//                   still in registers - a later panel Y = W_new Omega_j (line 7 of a later pass:
+//                   j = i+1 under the sequential schedule, j = i+2 under look-ahead), which saves
+//                   one full read of W per block step.
 #pragma once
 
 #include "gemm.cuh"
