@@ -243,18 +243,19 @@ def test_schedules_agree_and_stop_mid_way(h):
     assert relmax(Q2 @ g2.B[:k].cpu().numpy(), Q1 @ g1.B[:k].cpu().numpy()) <= 1e-10
 
 
-def test_subtractive_estimator_and_fixed_rank(h):
+@pytest.mark.parametrize("sched", SCHEDULES)
+def test_subtractive_estimator_and_fixed_rank(h, sched):
     w = wl.CONFIGS["cfg2"].scaled(m=1024, n=768, max_rank=256)
-    g, o, A, Om = run_both(h, w, estimator=1)
+    g, o, A, Om = run_both(h, w, estimator=1, flags=sched)
     check_run(h, w, g, o, A, Om, q_envelope=False)
     assert np.allclose(g.E_sub_trace, o.E_sub, rtol=1e-6, atol=1e-18 * o.normA2)
     dA, dOmT = torch.from_numpy(A).cuda(), torch.from_numpy(np.ascontiguousarray(Om.T)).cuda()
-    ga = rrf.rrf_run(h, dA, w.b, 1e-2, w.max_rank, omegaT=dOmT)
+    ga = rrf.rrf_run(h, dA, w.b, 1e-2, w.max_rank, omegaT=dOmT, flags=sched)
     assert ga.k < w.max_rank and ga.status == rrf.RRF_OK
-    gf = rrf.rrf_run(h, dA, w.b, 1e-2, w.max_rank, omegaT=dOmT, flags=rrf.RRF_FLAG_FIXED_RANK)
+    gf = rrf.rrf_run(h, dA, w.b, 1e-2, w.max_rank, omegaT=dOmT, flags=sched | rrf.RRF_FLAG_FIXED_RANK)
     assert gf.k == w.max_rank and gf.status == rrf.RRF_OK   # tolerance met on the way, ran to the cap
     assert torch.equal(gf.B[:ga.k], ga.B[:ga.k])
-    gf = rrf.rrf_run(h, dA, w.b, 1e-9, w.max_rank, omegaT=dOmT, flags=rrf.RRF_FLAG_FIXED_RANK)
+    gf = rrf.rrf_run(h, dA, w.b, 1e-9, w.max_rank, omegaT=dOmT, flags=sched | rrf.RRF_FLAG_FIXED_RANK)
     assert gf.k == w.max_rank and gf.status == rrf.RRF_MAX_RANK_REACHED
 
 
@@ -281,12 +282,13 @@ def test_edge_cases(h):
     assert g.status == rrf.RRF_ERR_NONFINITE and g.k == 0
 
 
-def test_inplace_aliasing_b(h):
+@pytest.mark.parametrize("sched", SCHEDULES)
+def test_inplace_aliasing_b(h, sched):
     w = wl.CONFIGS["cfg2"].scaled(m=768, n=512, max_rank=128)
-    g, o, A, Om = run_both(h, w)
+    g, o, A, Om = run_both(h, w, flags=sched)
     dA = torch.from_numpy(A).cuda()
     gi = rrf.rrf_run(h, dA, w.b, w.tol, w.max_rank, omegaT=torch.from_numpy(np.ascontiguousarray(Om.T)).cuda(),
-                     flags=rrf.RRF_FLAG_INPLACE, B=dA[:w.max_rank])
+                     flags=sched | rrf.RRF_FLAG_INPLACE, B=dA[:w.max_rank])
     assert gi.k == g.k
     assert torch.equal(dA[:g.k], g.B[:g.k])
 
