@@ -119,7 +119,8 @@ def check_run(h, w, g, o, A, Om, q_envelope=True):
 
 @pytest.mark.parametrize("rows,b,dtype", [(200, 16, "f64"), (1024, 16, "f64"), (4096, 32, "f64"),
                                           (8192, 64, "f64"), (5001, 64, "f64"), (300, 128, "f64"),
-                                          (20000, 128, "f64"), (4096, 64, "f32"), (777, 32, "f32")])
+                                          (20000, 128, "f64"), (4096, 64, "f32"), (777, 32, "f32"),
+                                          (60000, 32, "f64"), (45000, 64, "f64")])      # slabs of 512 / 320 rows
 def test_panel_qr_matches_oracle(h, rows, b, dtype):
     rng = np.random.default_rng(rows + b)
     Y = rng.standard_normal((rows, b))
