@@ -352,11 +352,18 @@ def main():
                         "peak_recipe_source": ("MEASURED_PEAKS.json bf16 x nominal FP64/bf16 ratio (of measured)"
                                                if "bf16_tflops" in peaks else "fallback bf16 x nominal ratio (of fallback)"),
                         "avg_launch_ms": ms / max(cnt, 1), "launches": cnt}
-            # with the look-ahead schedule the update runs beside the panel kernel, on the SMs left to it
+            # With the look-ahead schedule the update is launched on the SMs the panel kernel leaves it and
+            # the two run at the same time, so the roofline that bounds this kernel is that of its SMs.
             sms = torch.cuda.get_device_properties(local).multi_processor_count
             share = (sms - res.panel_ctas) / sms if (res.queues == 2 and top == "update") else 1.0
             roofline["sm_share"] = share
-            roofline["frac_of_share"] = achieved / (peak * share)
+            roofline["peak_device"] = peak
+            roofline["frac_device"] = achieved / peak
+            if share < 1.0:
+                roofline["peak"] = peak * share
+                roofline["frac"] = achieved / (peak * share)
+                roofline["peak_source"] += " x %d/%d SMs (the kernel runs on %d SMs beside the panel kernel on %d)" % (
+                    sms - res.panel_ctas, sms, sms - res.panel_ctas, res.panel_ctas)
             roofline["whole_step_frac"] = value / world / peak
         else:
             hbm = peaks.get("hbm_gbs", 6650.0)
