@@ -285,8 +285,10 @@ def main():
     ms_step = max_over_ranks(e0.elapsed_time(e1), world, dev) / args.steps
     flops = method_flops(w.m, w.n, w.b, res.steps)
     value = job_tflops(flops, world, ms_step)
-    # init x2, first sample (two with look-ahead); panel, T, VtW, TZ, update, stop per pass
-    launches_per_run = 3 + (1 if res.queues == 2 else 0) + 6 * (w.max_rank // w.b)
+    # init x2, first sample (two with look-ahead); panel, T, VtW, TZ, update, stop per pass, and with the
+    # sampling predictor one more (the separate sample kernel, which returns at once unless needed)
+    predicting = w.dtype == "f64" and w.b < 128 and (res.fused_samples < res.steps - 1 or res.extra_samples > 0)
+    launches_per_run = 3 + (1 if res.queues == 2 else 0) + (7 if predicting else 6) * (w.max_rank // w.b)
 
     # ---- end to end through the C ABI with host buffers
     e2e = None
@@ -337,8 +339,8 @@ def main():
             if w.dtype == "f32":
                 peak /= 3.0                       # three TF32 products per fp32 product
             work = args.steps * sum(2.0 * r * w.n * w.b for r in mi)
-            if top == "update":                   # the fused kernel also samples the next block's panel
-                work += args.steps * sum(2.0 * r * w.n * w.b for r in mi[1:])
+            if top == "update":                   # the fused kernel also samples a later panel in most passes
+                work += args.steps * sum(2.0 * r * w.n * w.b for r in mi[:res.fused_samples])
             if top == "sample":
                 work = args.steps * 2.0 * w.m * w.n * w.b
             achieved = work / (ms * 1e-3) / 1e12
@@ -398,6 +400,7 @@ def main():
                            "k": res.k, "block_steps": res.steps, "status": res.status,
                            "l2": "inputs larger than L2 (A is %.0f MB)" % (w.m * w.n * esize / 1e6),
                            "queues": res.queues, "panel_ctas": res.panel_ctas,
+                           "fused_samples": res.fused_samples, "extra_samples": res.extra_samples,
                            "parallelism": "replicas only" if world > 1 else "single GPU"},
                 "clocks": clocks, "e2e": e2e, "gpu_launches": args.steps * launches_per_run,
                 "roofline": roofline, "cpu_baseline": cpu}

@@ -52,6 +52,10 @@ typedef enum {
 #define RRF_FLAG_INPLACE 1u     /* A itself is the working matrix (it is overwritten) */
 #define RRF_FLAG_FIXED_RANK 2u  /* ignore the tolerance, always run to max_rank (fixed-rank mode) */
 #define RRF_FLAG_ONE_QUEUE 4u   /* force the sequential schedule: panel, V^T W, update one after the other */
+#define RRF_FLAG_SAMPLE_ALWAYS 32u /* every update samples a later panel (no prediction of the last passes) */
+#define RRF_FLAG_SAMPLE_NEVER 64u  /* no update samples; every panel comes from the separate sample kernel
+                                      (slower; exercises the path a wrong prediction takes).  Ignored in
+                                      single precision and for b = 128, where the updates always sample */
 #define RRF_FLAG_NO_GRAPH 16u    /* always enqueue the kernels one by one (by default a call that repeats the
                                    previous call's arguments is captured into a CUDA graph and replayed) */
 #define RRF_FLAG_TWO_QUEUES 8u  /* use the look-ahead schedule whenever the panel can be confined to a few SMs,
@@ -82,6 +86,9 @@ typedef struct {
   int32_t queues;           /* schedule used: 1 = sequential, 2 = look-ahead (panel QR of the next block runs
                                beside the update of the current one) */
   int32_t panel_ctas;       /* look-ahead: SMs the panel kernel was confined to; sequential: 0 */
+  int32_t fused_samples;    /* passes whose update also sampled a later panel */
+  int32_t extra_samples;    /* panels the separate sample kernel had to provide (wrong "the loop will end"
+                               predictions, or RRF_FLAG_SAMPLE_NEVER) */
 } rrf_result_t;
 
 /* Create / destroy a context bound to one CUDA device.  rrf_create makes `device`

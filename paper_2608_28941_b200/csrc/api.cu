@@ -54,7 +54,7 @@ static inline int ceil_div(long long a, long long b) { return (int)((a + b - 1) 
 constexpr int kSampleBM = 128, kSampleStages = 2;
 constexpr int kVtwBK = 64;
 
-struct SamplePlan { int nslabs, nseg, kt_per_seg; };
+struct SamplePlan { int nslabs, nseg, kt_per_seg, ctas; };
 constexpr int kSampleMaxSeg = 12;
 // K segments are chosen to fill whole waves of one CTA per SM with equal K ranges
 static SamplePlan plan_sample(int sms, long long rows, long long n, int esize, int kbs) {
@@ -74,6 +74,7 @@ static SamplePlan plan_sample(int sms, long long rows, long long n, int esize, i
   }
   p.kt_per_seg = ceil_div(KT, best);
   p.nseg = ceil_div(KT, p.kt_per_seg);
+  p.ctas = sms;   // one CTA per SM walks the items
   return p;
 }
 
@@ -265,10 +266,10 @@ struct Ops {
     return e;
   }
   static void sample(const CUtensorMap& tmW, const CUtensorMap& tmO, void* Ypart, int r0, int rows, int n, int j0,
-                     const SamplePlan& p, Ctrl* ctrl, cudaStream_t st) {
+                     const SamplePlan& p, Ctrl* ctrl, const int* only_if_zero, cudaStream_t st) {
     sample_kernel<T, B, kSampleBM, S_WM, S_WN, kSampleStages, S_KBS>
-        <<<dim3(p.nslabs, p.nseg), S_WM * S_WN * 32, S_SMEM, st>>>(tmW, tmO, (T*)Ypart, r0, rows, n, j0, p.kt_per_seg,
-                                                                     ctrl);
+        <<<std::min(p.nslabs * p.nseg, p.ctas), S_WM * S_WN * 32, S_SMEM, st>>>(tmW, tmO, (T*)Ypart, r0, rows, n, j0, p.nslabs,
+                                                                                  p.nseg, p.kt_per_seg, ctrl, only_if_zero);
   }
   static void vtw(const CUtensorMap& tmV, const CUtensorMap& tmC, void* Zpart, int r0, int cv0, const VtwPlan& p,
                   Ctrl* ctrl, cudaStream_t st) {
@@ -284,10 +285,10 @@ struct Ops {
   static void update(const CUtensorMap& tmV, const CUtensorMap& tmZ, const CUtensorMap& tmC, const CUtensorMap& tmO,
                      void* C, long long ldc, void* top, long long ldtop, int r0, int rows, int ncols, int cv0,
                      int top_rows, int j0, void* Ypart, double* norm_part, const UpdPlan& p, Ctrl* ctrl,
-                     cudaStream_t st) {
+                     const int* samp_flag, cudaStream_t st) {
     upd_sk_kernel<T, B, U_BM, U_BNB, U_WM, U_WN, U_STAGES, U_PW><<<p.P, (U_PW ? 9 : 8) * 32, U_SMEM, st>>>(
         tmV, tmZ, tmC, tmO, (T*)C, ldc, (T*)top, ldtop, r0, rows, ncols, cv0, top_rows, j0, (T*)Ypart, norm_part, p.NC,
-        p.total, p.tpc, ctrl);
+        p.total, p.tpc, ctrl, samp_flag);
   }
 };
 
@@ -295,11 +296,12 @@ struct OpTable {
   int s_kbs, v_bn, u_bm, u_bn, u_wn;
   cudaError_t (*setup)();
   void (*sample)(const CUtensorMap&, const CUtensorMap&, void*, int, int, int, int, const SamplePlan&, Ctrl*,
-                 cudaStream_t);
+                 const int*, cudaStream_t);
   void (*vtw)(const CUtensorMap&, const CUtensorMap&, void*, int, int, const VtwPlan&, Ctrl*, cudaStream_t);
   void (*tz)(const void*, const VtwPlan&, const void*, long long, int, void*, const int*, cudaStream_t);
   void (*update)(const CUtensorMap&, const CUtensorMap&, const CUtensorMap&, const CUtensorMap&, void*, long long,
-                 void*, long long, int, int, int, int, int, int, void*, double*, const UpdPlan&, Ctrl*, cudaStream_t);
+                 void*, long long, int, int, int, int, int, int, void*, double*, const UpdPlan&, Ctrl*, const int*,
+                 cudaStream_t);
 };
 template <typename T, int B>
 static OpTable make_ops() {
@@ -332,6 +334,8 @@ struct NoMark {
   void operator()(int, int) const {}
 };
 struct PanelOpts {
+  PanelSource alt{};               // where the panel is if the fused update skipped sampling it ...
+  const int* fused_flag = nullptr; // ... which is the case when this device word is 0 (NULL: always `src`)
   PanelFix fix{};                  // look-ahead fix-up (enabled == 0: none)
   int ctas = 0;                    // 0: one slab per SM; > 0: confine the panel to this many CTAs
   unsigned* bar_reset = nullptr;   // the T-factor kernel zeroes this word (the panel's barrier counter)
@@ -349,7 +353,10 @@ static rrf_status_t launch_panel(rrf_ctx* h, int dtype, const void* Y, PanelSour
   double *P = ps.P, *piv = ps.piv, *gram = ps.gram, *tau = ps.tau;
   unsigned* bar = ps.bar;
   PanelFix fix = o.fix;
-  void* args[] = {&Y, &src, &rows_i, &b, &R, &Rp, &V, &ldv, &P, &piv, &gram, &tau, &bar, &ctrl, &done_flag, &fix};
+  PanelSource alt = o.alt;
+  const int* fused_flag = o.fused_flag;
+  void* args[] = {&Y,   &src, &alt, &fused_flag, &rows_i, &b,    &R,         &Rp, &V,
+                  &ldv, &P,   &piv, &gram,       &tau,    &bar,  &ctrl, &done_flag, &fix};
   const size_t tsmem = ((size_t)b * (b + 1) + (size_t)(b / 2) * (b / 2 + 1)) * sizeof(double);
   mark(RRF_PHASE_PANEL, step);
   const void* fn = dtype == RRF_F64 ? panel_variant<double>(pp.variant) : panel_variant<float>(pp.variant);
@@ -443,7 +450,7 @@ static bool run_layout(const rrf_params_t* p, bool need_omega, RunLayout* L) {
   size_t off = 0;
   L->ctrl = off; off += 256;
   L->traces = off; off += align_up((size_t)2 * steps * sizeof(double), 256);
-  L->done_after = off; off += align_up((size_t)(steps + 2) * sizeof(int), 256);   // + the look-ahead barrier word
+  L->done_after = off; off += align_up((size_t)(2 * steps + 3) * sizeof(int), 256);   // + the look-ahead barrier word + samp[]
   L->init_ctas = kInitCtas;
   L->init_part = off; off += align_up((size_t)kInitCtas * sizeof(double), 256);
   L->max_norm_parts = sms;
@@ -708,7 +715,7 @@ static rrf_status_t apply_blocks(rrf_handle_t h, int dtype, long long m, int b, 
     ops->tz(Zpart, vp, (const char*)dT + (size_t)r0 * esize, ldt, transpose ? 1 : 0, Zt, &h->d_ctrl->done, st);
     const UpdPlan up = plan_upd(h->sms, rows, ncols, ops->u_bm, ops->u_bn, ops->u_wn);
     ops->update(tmV_u, tmZ, tmC_u, tmC_u, dC, ldc, dC, ldc, r0, rows, (int)ncols, r0, 0, -1, nullptr, nullptr, up,
-                h->d_ctrl, st);
+                h->d_ctrl, nullptr, st);
   }
   const cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) {
@@ -862,6 +869,20 @@ rrf_status_t rrf_run(rrf_handle_t h, const rrf_params_t* p, void* dA, int64_t ld
   double* tr_dir = tr_sub + steps;
   int* done_after = reinterpret_cast<int*>(ws + L.done_after);
   unsigned* look_bar = reinterpret_cast<unsigned*>(done_after + steps + 1);
+  int* samp = done_after + steps + 2;   // [steps + 1]: does the update of pass q sample a later panel
+  // Sampling predictor (see stop_kernel): worth its one skipped-kernel launch per pass only where a pass is
+  // long, i.e. where the sample it can save is worth more than those launches cost.
+  int predict = 1;
+  const bool predictor_built = b < 128 && p->dtype == RRF_F64;   // see upd_sk_kernel
+  if (!predictor_built) {
+    predict = 1;
+  } else if (p->flags & RRF_FLAG_SAMPLE_NEVER) {
+    predict = 2;
+  } else if (!(p->flags & RRF_FLAG_SAMPLE_ALWAYS) && !(p->flags & RRF_FLAG_FIXED_RANK)) {
+    const PassModel pm{h->sms, (double)m, (double)n, b, p->dtype == RRF_F64};
+    if (pm.vtw() + pm.upd() > 600.0) predict = 0;
+  }
+  const bool predicting = predict != 1;
   double* look_G = reinterpret_cast<double*>(ws + L.look);
   double* init_part = reinterpret_cast<double*>(ws + L.init_part);
   double* norm_part = reinterpret_cast<double*>(ws + L.norm_part);
@@ -922,7 +943,7 @@ rrf_status_t rrf_run(rrf_handle_t h, const rrf_params_t* p, void* dA, int64_t ld
     init_kernel<float><<<L.init_ctas, 256, 0, st>>>((const float*)dA, lda, inplace ? nullptr : (float*)W, ldw, m, n,
                                                     (float*)dV, ldv, p->max_rank, init_part);
   init_ctrl_kernel<<<1, 256, 0, st>>>(init_part, L.init_ctas, p->tol, p->tol_is_relative, fixed ? 1 : 0, b, p->max_rank,
-                                      ctrl, done_after, steps);
+                                      ctrl, done_after, samp, steps, predict);
 
   // fork/join events for the side stream, created once and kept in the handle
   while (h->sync_events.size() < (size_t)3 * steps + 2) {
@@ -951,17 +972,21 @@ rrf_status_t rrf_run(rrf_handle_t h, const rrf_params_t* p, void* dA, int64_t ld
   src.ldy = b;
   src.row_off = 0;
   mark(RRF_PHASE_SAMPLE, 0);
-  ops->sample(tmW_s, tmO, Ypart, 0, (int)m, (int)n, 0, sp, ctrl, st);
+  ops->sample(tmW_s, tmO, Ypart, 0, (int)m, (int)n, 0, sp, ctrl, nullptr, st);
 
   if (look_ctas == 0) {
     // One queue.  The panel of pass 0 is sampled by its own kernel; the panel of pass i+1 comes out
     // of the fused update of pass i.
+    PanelSource alt{};             // the upcoming panel as the separate sample kernel would leave it
+    const int* fused_flag = nullptr;
     for (int i = 0; i < steps; ++i) {
       const int r0 = i * b, rows = (int)(m - r0);
       PanelOpts po;
       po.st_t = h->aux;
       po.ev_fork = h->sync_events[2 * i];
       po.ev_join = h->sync_events[2 * i + 1];
+      po.alt = alt;
+      po.fused_flag = fused_flag;
       s = launch_panel(h, p->dtype, Ypart, src, rows, b, Vblk(r0), ldv, Tblk(r0), p->max_rank, ps, ctrl, &ctrl->done,
                        st, mark, i, po);
       if (s != RRF_OK) return panel_failed(s);
@@ -975,10 +1000,20 @@ rrf_status_t rrf_run(rrf_handle_t h, const rrf_params_t* p, void* dA, int64_t ld
       const int j0 = (i + 1 < steps) ? r0 + b : -1;   // Omega rows of the next pass, if there is one
       mark(RRF_PHASE_UPDATE, i);
       ops->update(tmV_u, tmZ, tmW_u, tmO, W, ldw, (char*)dB + (size_t)r0 * ldb * esize, ldb, r0, rows, (int)n, r0, b,
-                  j0, Ypart, norm_part, up, ctrl, st);
+                  j0, Ypart, norm_part, up, ctrl, samp + i, st);
       mark(RRF_PHASE_STOP, i);
       stop_kernel<<<1, 256, 0, st>>>(norm_part, up.P, b, p->max_rank, p->estimator, fixed ? 1 : 0, tr_sub, tr_dir, ctrl,
-                                     done_after, 1);
+                                     done_after, 1, predicting ? samp : nullptr, predict);
+      if (j0 >= 0 && predicting) {
+        // the next panel, sampled on its own if the loop goes on and the update had been told to skip it
+        const SamplePlan sp2 = plan_sample(h->sms, rows - b, n, esize, ops->s_kbs);
+        ops->sample(tmW_s, tmO, Ypart, r0 + b, rows - b, (int)n, j0, sp2, ctrl, samp + i, st);
+        alt = PanelSource{};
+        alt.nseg = sp2.nseg;
+        alt.seg_stride = (long long)(rows - b) * b;
+        alt.ldy = b;
+        fused_flag = samp + i;
+      }
       src.slots = 1;
       src.row_off = b;
       src.bm = ops->u_bm;
@@ -1010,6 +1045,7 @@ rrf_status_t rrf_run(rrf_handle_t h, const rrf_params_t* p, void* dA, int64_t ld
     };
     PanelSource src1 = src;           // panel 1: sampled from A by the sample kernel
     src1.row_off = b;
+    src1.nseg = plan_sample(gsms, m, n, esize, ops->s_kbs).nseg;
     cudaEventRecord(evS, st);
     cudaStreamWaitEvent(h->aux, evS, 0);
     ps.bar = look_bar;
@@ -1022,10 +1058,12 @@ rrf_status_t rrf_run(rrf_handle_t h, const rrf_params_t* p, void* dA, int64_t ld
     cudaEventRecord(evP(0), h->aux);
     if (steps > 1) {                  // the second panel is sampled while the first is factored
       mark(RRF_PHASE_SAMPLE, 0);
-      ops->sample(tmW_s, tmO, Ybuf[1], 0, (int)m, (int)n, b, sp, ctrl, st);
+      const SamplePlan sp1 = plan_sample(gsms, m, n, esize, ops->s_kbs);   // beside the first panel
+      ops->sample(tmW_s, tmO, Ybuf[1], 0, (int)m, (int)n, b, sp1, ctrl, nullptr, st);
       cudaEventRecord(evS2, st);
     }
     UpdPlan up_prev{};
+    PanelSource alt_prev{};        // the panel of pass i+1 as the separate sample kernel would leave it
     for (int i = 0; i < steps; ++i) {
       const int r0 = i * b, rows = (int)(m - r0);
       const bool gate = gated(rows);
@@ -1042,6 +1080,10 @@ rrf_status_t rrf_run(rrf_handle_t h, const rrf_params_t* p, void* dA, int64_t ld
           sn.wn = ops->u_wn;
         }
         PanelOpts pn = po;
+        if (i >= 1) {
+          pn.alt = alt_prev;
+          pn.fused_flag = predicting ? samp + (i - 1) : nullptr;
+        }
         pn.fix.enabled = 1;
         pn.fix.Vp = Vblk(r0);
         pn.fix.ldvp = ldv;
@@ -1076,10 +1118,21 @@ rrf_status_t rrf_run(rrf_handle_t h, const rrf_params_t* p, void* dA, int64_t ld
       const int j0 = (i + 2 < steps) ? r0 + 2 * b : -1;   // Omega rows of the pass after the next
       mark(RRF_PHASE_UPDATE, i);
       ops->update(tmV_u, tmZ, tmW_u, tmO, W, ldw, (char*)dB + (size_t)r0 * ldb * esize, ldb, r0, rows, (int)n, r0, b,
-                  j0, Ybuf[i & 1], norm_part, up, ctrl, st);
+                  j0, Ybuf[i & 1], norm_part, up, ctrl, samp + i, st);
       mark(RRF_PHASE_STOP, i);
       stop_kernel<<<1, 256, 0, st>>>(norm_part, up.P, b, p->max_rank, p->estimator, fixed ? 1 : 0, tr_sub, tr_dir, ctrl,
-                                     done_after, 0);
+                                     done_after, 0, predicting ? samp : nullptr, predict);
+      if (j0 >= 0 && predicting) {
+        // the panel of pass i+2, sampled on its own if the loop goes on and the update had been told to skip it;
+        // its first b rows are the rows above that panel which the fix-up needs
+        const SamplePlan sp2 = plan_sample(gsms, rows - b, n, esize, ops->s_kbs);
+        ops->sample(tmW_s, tmO, Ybuf[i & 1], r0 + b, rows - b, (int)n, j0, sp2, ctrl, samp + i, st);
+        alt_prev = PanelSource{};
+        alt_prev.nseg = sp2.nseg;
+        alt_prev.seg_stride = (long long)(rows - b) * b;
+        alt_prev.ldy = b;
+        alt_prev.row_off = b;
+      }
       cudaEventRecord(evU(i), st);
       up_prev = up;
     }
@@ -1185,6 +1238,8 @@ rrf_status_t rrf_run(rrf_handle_t h, const rrf_params_t* p, void* dA, int64_t ld
   out->E_sub = hc.E_sub;
   out->E_dir = hc.E_dir;
   out->queues = look_ctas > 0 ? 2 : 1;
+  out->fused_samples = hc.fused_samples;
+  out->extra_samples = hc.extra_samples;
   out->panel_ctas = look_ctas;
   if (hc.steps > 0) {
     if (h_E_sub_trace != nullptr) cudaMemcpy(h_E_sub_trace, tr_sub, sizeof(double) * hc.steps, cudaMemcpyDeviceToHost);

@@ -23,6 +23,10 @@ struct Ctrl {
   double sigma2;   // squared absolute tolerance
   double E_sub;    // Algorithm 2 line 9
   double E_dir;    // ||W[r0+b:, :]||_F^2
+  double E_prev;   // stopping quantity after the previous pass, and the ratio of the two before that:
+  double r_prev;   // the history the sampling predictor extrapolates (negative: no ratio yet)
+  int fused_samples;   // passes whose update also sampled a later panel
+  int extra_samples;   // panels sampled by the separate kernel because the predictor had skipped them
 };
 
 // ~1 s at 2 GHz: every spin in this library gives up after this many SM clocks.

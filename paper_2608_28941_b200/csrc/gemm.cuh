@@ -44,7 +44,7 @@ __device__ __forceinline__ void store2<float>(float* p, float a, float b) {
 
 // ------------------------------------------------------------------------------------------
 // Y_part[seg] = W[r0 + slab*BM ..., k-range(seg)] * OmegaT[j0 .. j0+B, k-range(seg)]^T
-// grid = (row slabs, K segments); both operands K-contiguous.
+// Items (row slab, K segment), walked by one CTA per SM; both operands K-contiguous.
 // ------------------------------------------------------------------------------------------
 // KBS 128-byte K boxes of both operands form one pipeline stage.
 template <typename T, int B, int BM, int WM, int WN, int STAGES, int KBS>
@@ -52,8 +52,13 @@ __global__ void __launch_bounds__(WM* WN * 32)
     sample_kernel(const __grid_constant__ CUtensorMap tmW,  // W [m][n], box [BM][KE]
                   const __grid_constant__ CUtensorMap tmO,  // OmegaT [max_rank][n], box [B][KE]
                   T* __restrict__ Ypart,                    // [nseg][rows][B]
-                  int r0, int rows, int n, int j0, int kt_per_seg, Ctrl* ctrl) {
+                  int r0, int rows, int n, int j0, int nslabs, int nseg, int kt_per_seg, Ctrl* ctrl,
+                  const int* __restrict__ only_if_zero) {   // non-NULL: run only where the fused update skipped this panel
   if (*reinterpret_cast<volatile int*>(&ctrl->done)) return;
+  if (only_if_zero != nullptr) {
+    if (*only_if_zero != 0) return;
+    if (blockIdx.x == 0 && threadIdx.x == 0) atomicAdd(&ctrl->extra_samples, 1);
+  }
   constexpr int KE = Elem<T>::KE, NV = Elem<T>::NV, KS = Elem<T>::KS;
   constexpr int TM = BM / WM, TN = B / WN, MT = TM / 16, NT = TN / 8;
   static_assert(TM % 16 == 0 && TN % 8 == 0, "warp tile");
@@ -65,11 +70,7 @@ __global__ void __launch_bounds__(WM* WN * 32)
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
   const int wm = warp / WN, wn = warp % WN;
-  const int slab = blockIdx.x, seg = blockIdx.y;
   const int KT = (n + KBS * KE - 1) / (KBS * KE);    // K tiles of KBS boxes
-  const int kt0 = seg * kt_per_seg;
-  const int nkt = max(0, min(KT, kt0 + kt_per_seg) - kt0);
-  const int grow0 = r0 + slab * BM;
 
   if (tid == 0) {
     for (int s = 0; s < STAGES; ++s) mbar_init(&full[s], 1);
@@ -77,76 +78,87 @@ __global__ void __launch_bounds__(WM* WN * 32)
   }
   __syncthreads();
 
-  auto issue = [&](int i) {
-    const int st = i % STAGES;
-    unsigned char* sA = smem + st * STAGE_BYTES;
-    mbar_expect_tx(&full[st], STAGE_BYTES);
-#pragma unroll
-    for (int kb = 0; kb < KBS; ++kb) {
-      tma_load_2d(sA + kb * A_BYTES, &tmW, ((kt0 + i) * KBS + kb) * KE, grow0, &full[st]);
-      tma_load_2d(sA + KBS * A_BYTES + kb * B_BYTES, &tmO, ((kt0 + i) * KBS + kb) * KE, j0, &full[st]);
-    }
-  };
-  if (tid == 0)
-    for (int i = 0; i < STAGES - 1 && i < nkt; ++i) issue(i);
+  // One CTA per SM walks the (row slab, K segment) items; `base` counts the K tiles this CTA has been
+  // through, which is what the stage ring and the barrier phases follow across items.
+  int base = 0;
+  for (int item = blockIdx.x; item < nslabs * nseg; item += gridDim.x) {
+    const int slab = item % nslabs, seg = item / nslabs;
+    const int kt0 = seg * kt_per_seg;
+    const int nkt = max(0, min(KT, kt0 + kt_per_seg) - kt0);
+    const int grow0 = r0 + slab * BM;
 
-  T acc[MT][NT][4];
+    auto issue = [&](int i) {
+      const int st = (base + i) % STAGES;
+      unsigned char* sA = smem + st * STAGE_BYTES;
+      mbar_expect_tx(&full[st], STAGE_BYTES);
 #pragma unroll
-  for (int a = 0; a < MT; ++a)
-#pragma unroll
-    for (int c = 0; c < NT; ++c)
-#pragma unroll
-      for (int e = 0; e < 4; ++e) acc[a][c][e] = T(0);
+      for (int kb = 0; kb < KBS; ++kb) {
+        tma_load_2d(sA + kb * A_BYTES, &tmW, ((kt0 + i) * KBS + kb) * KE, grow0, &full[st]);
+        tma_load_2d(sA + KBS * A_BYTES + kb * B_BYTES, &tmO, ((kt0 + i) * KBS + kb) * KE, j0, &full[st]);
+      }
+    };
+    if (tid == 0)
+      for (int i = 0; i < STAGES - 1 && i < nkt; ++i) issue(i);
 
-  for (int i = 0; i < nkt; ++i) {
-    if (tid == 0 && i + STAGES - 1 < nkt) issue(i + STAGES - 1);
-    const int st = i % STAGES;
-    if (!mbar_wait(&full[st], (i / STAGES) & 1, ctrl)) return;
+    T acc[MT][NT][4];
 #pragma unroll
-    for (int kb = 0; kb < KBS; ++kb) {
-    const unsigned char* sA = smem + st * STAGE_BYTES + kb * A_BYTES;
-    const unsigned char* sB = smem + st * STAGE_BYTES + KBS * A_BYTES + kb * B_BYTES;
+    for (int a = 0; a < MT; ++a)
 #pragma unroll
-    for (int s2 = 0; s2 < 2; ++s2) {
-      const uint32_t chunk = ((uint32_t)(2 * t + s2) ^ (uint32_t)g) << 4;
-      T ra[MT][2][NV], rb[NT][NV];
+      for (int c = 0; c < NT; ++c)
 #pragma unroll
-      for (int a = 0; a < MT; ++a) {
-        const int rlo = wm * TM + a * 16 + g;
-        VecLoad16<T>::ld(sA + rlo * 128 + chunk, ra[a][0]);
-        VecLoad16<T>::ld(sA + (rlo + 8) * 128 + chunk, ra[a][1]);
-      }
+        for (int e = 0; e < 4; ++e) acc[a][c][e] = T(0);
+
+    for (int i = 0; i < nkt; ++i) {
+      if (tid == 0 && i + STAGES - 1 < nkt) issue(i + STAGES - 1);
+      const int st = (base + i) % STAGES;
+      if (!mbar_wait(&full[st], ((base + i) / STAGES) & 1, ctrl)) return;
 #pragma unroll
-      for (int c = 0; c < NT; ++c) {
-        const int rn = wn * TN + c * 8 + g;
-        VecLoad16<T>::ld(sB + rn * 128 + chunk, rb[c]);
-      }
+      for (int kb = 0; kb < KBS; ++kb) {
+        const unsigned char* sA = smem + st * STAGE_BYTES + kb * A_BYTES;
+        const unsigned char* sB = smem + st * STAGE_BYTES + KBS * A_BYTES + kb * B_BYTES;
 #pragma unroll
-      for (int ks = 0; ks < KS; ++ks)
+        for (int s2 = 0; s2 < 2; ++s2) {
+          const uint32_t chunk = ((uint32_t)(2 * t + s2) ^ (uint32_t)g) << 4;
+          T ra[MT][2][NV], rb[NT][NV];
 #pragma unroll
-        for (int a = 0; a < MT; ++a) {
-          const T af[4] = {ra[a][0][2 * ks], ra[a][1][2 * ks], ra[a][0][2 * ks + 1], ra[a][1][2 * ks + 1]};
+          for (int a = 0; a < MT; ++a) {
+            const int rlo = wm * TM + a * 16 + g;
+            VecLoad16<T>::ld(sA + rlo * 128 + chunk, ra[a][0]);
+            VecLoad16<T>::ld(sA + (rlo + 8) * 128 + chunk, ra[a][1]);
+          }
 #pragma unroll
           for (int c = 0; c < NT; ++c) {
-            const T bf[2] = {rb[c][2 * ks], rb[c][2 * ks + 1]};
-            mma16x8x8(acc[a][c], af, bf);
+            const int rn = wn * TN + c * 8 + g;
+            VecLoad16<T>::ld(sB + rn * 128 + chunk, rb[c]);
           }
+#pragma unroll
+          for (int ks = 0; ks < KS; ++ks)
+#pragma unroll
+            for (int a = 0; a < MT; ++a) {
+              const T af[4] = {ra[a][0][2 * ks], ra[a][1][2 * ks], ra[a][0][2 * ks + 1], ra[a][1][2 * ks + 1]};
+#pragma unroll
+              for (int c = 0; c < NT; ++c) {
+                const T bf[2] = {rb[c][2 * ks], rb[c][2 * ks + 1]};
+                mma16x8x8(acc[a][c], af, bf);
+              }
+            }
         }
+      }
+      __syncthreads();  // everyone is done with stage st before it is refilled
     }
-    }
-    __syncthreads();  // everyone is done with stage st before it is refilled
-  }
+    base += nkt;
 
-  T* Y = Ypart + (size_t)seg * (size_t)rows * B;
+    T* Y = Ypart + (size_t)seg * (size_t)rows * B;
 #pragma unroll
-  for (int a = 0; a < MT; ++a)
+    for (int a = 0; a < MT; ++a)
 #pragma unroll
-    for (int c = 0; c < NT; ++c) {
-      const int row = slab * BM + wm * TM + a * 16 + g;
-      const int col = wn * TN + c * 8 + 2 * t;
-      if (row < rows) store2(Y + (size_t)row * B + col, acc[a][c][0], acc[a][c][1]);
-      if (row + 8 < rows) store2(Y + (size_t)(row + 8) * B + col, acc[a][c][2], acc[a][c][3]);
-    }
+      for (int c = 0; c < NT; ++c) {
+        const int row = slab * BM + wm * TM + a * 16 + g;
+        const int col = wn * TN + c * 8 + 2 * t;
+        if (row < rows) store2(Y + (size_t)row * B + col, acc[a][c][0], acc[a][c][1]);
+        if (row + 8 < rows) store2(Y + (size_t)(row + 8) * B + col, acc[a][c][2], acc[a][c][3]);
+      }
+  }
 }
 
 }  // namespace rrf

@@ -199,7 +199,8 @@ __global__ void __launch_bounds__((WM * WN + (PW ? 1 : 0)) * 32, 1)
                   T* __restrict__ C, long long ldc, T* __restrict__ top, long long ldtop,
                   int r0, int rows, int ncols, int cv0, int top_rows, int j0,
                   T* __restrict__ Ypart, double* __restrict__ norm_part,
-                  int NC, int total, int tpc, Ctrl* ctrl) {
+                  int NC, int total, int tpc, Ctrl* ctrl,
+                  const int* __restrict__ samp_flag) {   // non-NULL: sample only if *samp_flag != 0
   if (*reinterpret_cast<volatile int*>(&ctrl->done)) return;
   constexpr int KE = Elem<T>::KE, NV = Elem<T>::NV, KS = Elem<T>::KS;
   constexpr int U = KE / 8;            // n-tiles per 128-byte column group
@@ -226,7 +227,11 @@ __global__ void __launch_bounds__((WM * WN + (PW ? 1 : 0)) * 32, 1)
   const int p = blockIdx.x;
   const int L0 = p * tpc;
   const int ntile = min(total, L0 + tpc) - L0;
-  const bool do_sample = j0 >= 0;
+  // the widest block size and single precision keep the host's decision (those instantiations are at
+  // the register limit and lose 3-4 % with the extra test)
+  constexpr bool kPredicted = B < 128 && sizeof(T) == 8;
+  const bool do_sample = j0 >= 0 && (!kPredicted || samp_flag == nullptr || *samp_flag != 0);
+  if (kPredicted && do_sample && samp_flag != nullptr && p == 0 && tid == 0) atomicAdd(&ctrl->fused_samples, 1);
 
   if (tid == 0) {
     for (int s = 0; s < STAGES; ++s) {

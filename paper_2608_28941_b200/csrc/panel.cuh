@@ -127,7 +127,7 @@ __device__ __forceinline__ double panel_entry(const T* __restrict__ Y, const Pan
 // fits unpadded).
 template <typename T, int QMAX, int RH, bool PAD = true>
 __global__ void __launch_bounds__(kPanelThreads)
-    panel_kernel(const T* __restrict__ Y, PanelSource src,
+    panel_kernel(const T* __restrict__ Y, PanelSource src_fused, PanelSource src_alt, const int* __restrict__ fused_flag,
                  int rows, int b, int R, int Rp,
                  T* __restrict__ V, long long ldv,   // rows x b block of the V array
                  double* __restrict__ P,             // [2][b][Gp] per-CTA partial dots, Gp = gridDim.x rounded up to 32
@@ -136,6 +136,10 @@ __global__ void __launch_bounds__(kPanelThreads)
                  double* __restrict__ tau_out,       // [b]
                  unsigned* bar, Ctrl* ctrl, const int* done_flag, PanelFix fix) {
   if (*reinterpret_cast<const volatile int*>(done_flag)) return;
+  // the panel's entries were sampled by the fused update, or - where the predictor had skipped that - by
+  // the separate sample kernel, in its layout
+  const bool use_alt = fused_flag != nullptr && *fused_flag == 0;
+  const PanelSource src = use_alt ? src_alt : src_fused;   // a copy in registers, not a pointer into the parameters
   extern __shared__ double psm[];
   double* S = psm;                        // [b][Rp]
   double* w_s = S + (size_t)b * Rp;       // [b]
@@ -672,7 +676,8 @@ __global__ void __launch_bounds__(256)
 
 __global__ void __launch_bounds__(256)
     init_ctrl_kernel(const double* __restrict__ part, int npart, double tol, int relative, int fixed_rank,
-                     int b, int max_rank, Ctrl* ctrl, int* __restrict__ done_after, int nsteps) {
+                     int b, int max_rank, Ctrl* ctrl, int* __restrict__ done_after, int* __restrict__ samp, int nsteps,
+                     int predict) {
   __shared__ double red[32];
   double s = 0.0;
   for (int i = threadIdx.x; i < npart; i += 256) s += part[i];
@@ -682,6 +687,10 @@ __global__ void __launch_bounds__(256)
     ctrl->sigma2 = relative ? tol * tol * tot : tol * tol;
     ctrl->E_sub = tot;
     ctrl->E_dir = tot;
+    ctrl->E_prev = tot;
+    ctrl->r_prev = -1.0;
+    ctrl->fused_samples = 0;
+    ctrl->extra_samples = 0;
     ctrl->steps = 0;
     ctrl->k = 0;
     ctrl->bar = 0;
@@ -702,6 +711,9 @@ __global__ void __launch_bounds__(256)
       done_after[0] = done;
       for (int q = 1; q <= nsteps; ++q) done_after[q] = 1;
     }
+    // samp[q] != 0: the update of pass q also samples a later panel; the stop rule of pass q-1 decides it
+    if (samp != nullptr)
+      for (int q = 0; q <= nsteps; ++q) samp[q] = predict == 2 ? 0 : 1;
   }
 }
 
@@ -709,7 +721,7 @@ __global__ void __launch_bounds__(256)
 __global__ void __launch_bounds__(256)
     stop_kernel(const double* __restrict__ norm_part, int npart, int b, int max_rank, int estimator,
                 int fixed_rank, double* __restrict__ tr_sub, double* __restrict__ tr_dir, Ctrl* ctrl,
-                int* __restrict__ done_after, int reset_bar) {
+                int* __restrict__ done_after, int reset_bar, int* __restrict__ samp, int predict) {
   if (*reinterpret_cast<volatile int*>(&ctrl->done)) return;
   __shared__ double red[64];
   double st = 0.0, sr = 0.0;
@@ -736,6 +748,28 @@ __global__ void __launch_bounds__(256)
     if (ctrl->status == RRF_OK && !below && cap) ctrl->status = RRF_MAX_RANK_REACHED;
     if (met || cap) ctrl->done = 1;
     if (done_after != nullptr) done_after[i + 1] = (met || cap) ? 1 : 0;
+    // Sampling predictor.  The update of pass i+1 also samples a later panel, which is wasted work if
+    // pass i+1 turns out to be the last.  Extrapolate the stopping quantity one pass ahead (last reduction
+    // ratio, moved on by its last change) and let that update skip the sampling when the two last ratios
+    // agree to 30 % and the prediction is below the tolerance.  If the loop goes on after all, the
+    // skipped panel is sampled by a kernel of its own.  predict: 0 = by this rule, 1 = always sample,
+    // 2 = never sample.
+    if (samp != nullptr) {
+      const double Ep = ctrl->E_prev;
+      double r = (Ep > 0.0) ? E / Ep : 1.0;
+      r = r < 0.0 ? 0.0 : (r > 1.0 ? 1.0 : r);
+      const double rp = ctrl->r_prev;
+      const double dr = (rp >= 0.0 && r > rp) ? r - rp : 0.0;
+      const double rr = r + dr > 1.0 ? 1.0 : r + dr;
+      const double e = E * rr;
+      const bool steady = rp >= 0.0 && fabs(r - rp) <= 0.3 * fmax(r, rp);
+      int want = fixed_rank || !steady || e > 0.9 * ctrl->sigma2;
+      if (predict == 1) want = 1;
+      if (predict == 2) want = 0;
+      samp[i + 1] = want;
+      ctrl->E_prev = E;
+      ctrl->r_prev = r;
+    }
   }
 }
 

@@ -17,6 +17,7 @@ RRF_F64, RRF_F32 = 0, 1
 RRF_OK, RRF_MAX_RANK_REACHED = 0, 1
 RRF_ERR_INVALID_ARG, RRF_ERR_WORKSPACE, RRF_ERR_CUDA, RRF_ERR_TIMEOUT, RRF_ERR_NONFINITE = -1, -2, -3, -4, -5
 RRF_FLAG_INPLACE, RRF_FLAG_FIXED_RANK, RRF_FLAG_ONE_QUEUE, RRF_FLAG_TWO_QUEUES, RRF_FLAG_NO_GRAPH = 1, 2, 4, 8, 16
+RRF_FLAG_SAMPLE_ALWAYS, RRF_FLAG_SAMPLE_NEVER = 32, 64
 
 _LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "librrf.so")
 _lib = None
@@ -31,7 +32,8 @@ class rrf_params_t(C.Structure):
 class rrf_result_t(C.Structure):
     _fields_ = [("status", C.c_int32), ("k", C.c_int32), ("steps", C.c_int32), ("cuda_error", C.c_int32),
                 ("normA2", C.c_double), ("sigma2", C.c_double), ("E_sub", C.c_double), ("E_dir", C.c_double),
-                ("queues", C.c_int32), ("panel_ctas", C.c_int32)]
+                ("queues", C.c_int32), ("panel_ctas", C.c_int32), ("fused_samples", C.c_int32),
+                ("extra_samples", C.c_int32)]
 
 
 RRF_PHASES = ["init", "sample", "panel", "tfactor", "vtw", "tz", "update", "stop", "skipped"]
@@ -164,6 +166,8 @@ class RunResult:
     B: torch.Tensor   # max_rank x n buffer; rows [:k] are defined
     queues: int = 1   # schedule used: 1 sequential, 2 look-ahead
     panel_ctas: int = 0
+    fused_samples: int = 0
+    extra_samples: int = 0
 
 
 def rrf_run(h, A: torch.Tensor, b: int, tol: float, max_rank: int, omegaT: torch.Tensor | None = None,
@@ -200,7 +204,8 @@ def rrf_run(h, A: torch.Tensor, b: int, tol: float, max_rank: int, omegaT: torch
     if check and s < 0:
         raise RrfError(s, "rrf_run")
     return RunResult(res.status, res.k, res.steps, res.normA2, res.sigma2, res.E_sub, res.E_dir,
-                     list(tr_sub)[:res.steps], list(tr_dir)[:res.steps], V, T, B, res.queues, res.panel_ctas)
+                     list(tr_sub)[:res.steps], list(tr_dir)[:res.steps], V, T, B, res.queues, res.panel_ctas,
+                     res.fused_samples, res.extra_samples)
 
 
 def rrf_panel_qr(h, Y: torch.Tensor):

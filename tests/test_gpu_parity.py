@@ -225,6 +225,24 @@ def test_reduced_configs(h, name, kw, sched):
     check_run(h, w, g, o, A, Om)
 
 
+@pytest.mark.parametrize("sched", SCHEDULES)
+@pytest.mark.parametrize("sampling", [pytest.param(rrf.RRF_FLAG_SAMPLE_ALWAYS, id="always-fused"),
+                                      pytest.param(rrf.RRF_FLAG_SAMPLE_NEVER, id="never-fused")])
+@pytest.mark.parametrize("name,kw", [("cfg2", dict(m=1536, n=1280, max_rank=512)),
+                                     ("cfg3", dict(m=1024, n=1024, max_rank=512)),
+                                     ("cfg1", dict(m=900, n=700, max_rank=256))])
+def test_panel_from_either_sampler(h, name, kw, sched, sampling):
+    # the update samples a later panel unless the stop rule predicts that the loop ends first; a panel
+    # skipped wrongly comes from the separate sample kernel.  Both extremes must give the oracle's result.
+    w = wl.CONFIGS[name].scaled(**kw)
+    g, o, A, Om = run_both(h, w, flags=sched | sampling)
+    if sampling == rrf.RRF_FLAG_SAMPLE_NEVER:
+        assert g.fused_samples == 0 and g.extra_samples >= g.steps - (2 if g.queues == 2 else 1)
+    else:
+        assert g.extra_samples == 0 and g.fused_samples >= g.steps - (2 if g.queues == 2 else 1)
+    check_run(h, w, g, o, A, Om)
+
+
 def test_schedules_agree_and_stop_mid_way(h):
     # stops after a few blocks: the look-ahead has factored one panel too many by then, which must
     # not show in k, B, the traces, or the defined part of V and T
