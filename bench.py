@@ -285,10 +285,7 @@ def main():
     ms_step = max_over_ranks(e0.elapsed_time(e1), world, dev) / args.steps
     flops = method_flops(w.m, w.n, w.b, res.steps)
     value = job_tflops(flops, world, ms_step)
-    # init x2, first sample (two with look-ahead); panel, T, VtW, TZ, update, stop per pass, and with the
-    # sampling predictor one more (the separate sample kernel, which returns at once unless needed)
-    predicting = w.dtype == "f64" and w.b < 128 and (res.fused_samples < res.steps - 1 or res.extra_samples > 0)
-    launches_per_run = 3 + (1 if res.queues == 2 else 0) + (7 if predicting else 6) * (w.max_rank // w.b)
+    launches_per_run = res.kernel_launches     # counted by the library: every kernel it put on the device
 
     # ---- end to end through the C ABI with host buffers
     e2e = None
@@ -340,7 +337,7 @@ def main():
                 peak /= 3.0                       # three TF32 products per fp32 product
             work = args.steps * sum(2.0 * r * w.n * w.b for r in mi)
             if top == "update":                   # the fused kernel also samples a later panel in most passes
-                work += args.steps * sum(2.0 * r * w.n * w.b for r in mi[:res.fused_samples])
+                work += args.steps * sum(2.0 * (r - w.b) * w.n * w.b for r in mi[:res.fused_samples])   # rows below B_i
             if top == "sample":
                 work = args.steps * 2.0 * w.m * w.n * w.b
             achieved = work / (ms * 1e-3) / 1e12

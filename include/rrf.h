@@ -89,6 +89,9 @@ typedef struct {
   int32_t fused_samples;    /* passes whose update also sampled a later panel */
   int32_t extra_samples;    /* panels the separate sample kernel had to provide (wrong "the loop will end"
                                predictions, or RRF_FLAG_SAMPLE_NEVER) */
+  int32_t kernel_launches;  /* kernels of this library the call put on the device, passes after the stop
+                               included (their kernels start, read the stop flag and return) */
+  int32_t reserved;
 } rrf_result_t;
 
 /* Create / destroy a context bound to one CUDA device.  rrf_create makes `device`

@@ -1239,6 +1239,12 @@ rrf_status_t rrf_run(rrf_handle_t h, const rrf_params_t* p, void* dA, int64_t ld
   out->E_dir = hc.E_dir;
   out->queues = look_ctas > 0 ? 2 : 1;
   out->fused_samples = hc.fused_samples;
+  {
+    // kernels this call put on the device (passes after the stop included: they start and return)
+    const int lag = look_ctas > 0 ? 2 : 1;
+    out->kernel_launches = 2 + (dOmegaT == nullptr ? 1 : 0) + 1 + ((look_ctas > 0 && steps > 1) ? 1 : 0) + 6 * steps +
+                           (predicting ? std::max(0, steps - lag) : 0);
+  }
   out->extra_samples = hc.extra_samples;
   out->panel_ctas = look_ctas;
   if (hc.steps > 0) {

@@ -33,7 +33,7 @@ class rrf_result_t(C.Structure):
     _fields_ = [("status", C.c_int32), ("k", C.c_int32), ("steps", C.c_int32), ("cuda_error", C.c_int32),
                 ("normA2", C.c_double), ("sigma2", C.c_double), ("E_sub", C.c_double), ("E_dir", C.c_double),
                 ("queues", C.c_int32), ("panel_ctas", C.c_int32), ("fused_samples", C.c_int32),
-                ("extra_samples", C.c_int32)]
+                ("extra_samples", C.c_int32), ("kernel_launches", C.c_int32), ("reserved", C.c_int32)]
 
 
 RRF_PHASES = ["init", "sample", "panel", "tfactor", "vtw", "tz", "update", "stop", "skipped"]
@@ -168,6 +168,7 @@ class RunResult:
     panel_ctas: int = 0
     fused_samples: int = 0
     extra_samples: int = 0
+    kernel_launches: int = 0
 
 
 def rrf_run(h, A: torch.Tensor, b: int, tol: float, max_rank: int, omegaT: torch.Tensor | None = None,
@@ -205,7 +206,7 @@ def rrf_run(h, A: torch.Tensor, b: int, tol: float, max_rank: int, omegaT: torch
         raise RrfError(s, "rrf_run")
     return RunResult(res.status, res.k, res.steps, res.normA2, res.sigma2, res.E_sub, res.E_dir,
                      list(tr_sub)[:res.steps], list(tr_dir)[:res.steps], V, T, B, res.queues, res.panel_ctas,
-                     res.fused_samples, res.extra_samples)
+                     res.fused_samples, res.extra_samples, res.kernel_launches)
 
 
 def rrf_panel_qr(h, Y: torch.Tensor):
