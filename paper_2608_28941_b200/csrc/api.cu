@@ -266,10 +266,10 @@ struct Ops {
     return e;
   }
   static void sample(const CUtensorMap& tmW, const CUtensorMap& tmO, void* Ypart, int r0, int rows, int n, int j0,
-                     const SamplePlan& p, Ctrl* ctrl, const int* only_if_zero, cudaStream_t st) {
+                     const SamplePlan& p, Ctrl* ctrl, const int* only_if_zero, double* sq_part, cudaStream_t st) {
     sample_kernel<T, B, kSampleBM, S_WM, S_WN, kSampleStages, S_KBS>
         <<<std::min(p.nslabs * p.nseg, p.ctas), S_WM * S_WN * 32, S_SMEM, st>>>(tmW, tmO, (T*)Ypart, r0, rows, n, j0, p.nslabs,
-                                                                                  p.nseg, p.kt_per_seg, ctrl, only_if_zero);
+                                                                                  p.nseg, p.kt_per_seg, ctrl, only_if_zero, sq_part);
   }
   static void vtw(const CUtensorMap& tmV, const CUtensorMap& tmC, void* Zpart, int r0, int cv0, const VtwPlan& p,
                   Ctrl* ctrl, cudaStream_t st) {
@@ -296,7 +296,7 @@ struct OpTable {
   int s_kbs, v_bn, u_bm, u_bn, u_wn;
   cudaError_t (*setup)();
   void (*sample)(const CUtensorMap&, const CUtensorMap&, void*, int, int, int, int, const SamplePlan&, Ctrl*,
-                 const int*, cudaStream_t);
+                 const int*, double*, cudaStream_t);
   void (*vtw)(const CUtensorMap&, const CUtensorMap&, void*, int, int, const VtwPlan&, Ctrl*, cudaStream_t);
   void (*tz)(const void*, const VtwPlan&, const void*, long long, int, void*, const int*, cudaStream_t);
   void (*update)(const CUtensorMap&, const CUtensorMap&, const CUtensorMap&, const CUtensorMap&, void*, long long,
@@ -912,8 +912,12 @@ rrf_status_t rrf_run(rrf_handle_t h, const rrf_params_t* p, void* dA, int64_t ld
   }
   const OpTable* ops = get_ops(p->dtype, b);
   const int npad = plan_vtw(h->sms, m, n, ops->v_bn).npad;
-  CUtensorMap tmW_s, tmO, tmV_k, tmW_k, tmV_u, tmW_u, tmZ;
-  if (!make_map(h, &tmW_s, p->dtype, W, m, n, ldw, kSampleBM) ||
+  // Pass 0 reads A itself and writes W (no copy W <- A): the first panels are sampled from A, V_0^T A is taken
+  // from A, and the update of pass 0 loads its tiles from A and stores them to W.
+  CUtensorMap tmW_s, tmA_s, tmA_k, tmA_u, tmO, tmV_k, tmW_k, tmV_u, tmW_u, tmZ;
+  if (!make_map(h, &tmA_s, p->dtype, dA, m, n, lda, kSampleBM) || !make_map(h, &tmA_k, p->dtype, dA, m, n, lda, kVtwBK) ||
+      !make_map(h, &tmA_u, p->dtype, dA, m, n, lda, ops->u_bm) ||
+      !make_map(h, &tmW_s, p->dtype, W, m, n, ldw, kSampleBM) ||
       !make_map(h, &tmO, p->dtype, Om, p->max_rank, n, ldom, b) ||
       !make_map(h, &tmV_k, p->dtype, dV, m, p->max_rank, ldv, kVtwBK) ||
       !make_map(h, &tmW_k, p->dtype, W, m, n, ldw, kVtwBK) ||
@@ -934,16 +938,12 @@ rrf_status_t rrf_run(rrf_handle_t h, const rrf_params_t* p, void* dA, int64_t ld
     marks.emplace_back(phase, step);
   };
 
-  // Algorithm 2 lines 1-4
+  // Algorithm 2 lines 1-4.  V <- 0 and the loop state are memsets; ||A||_F^2 is summed by the first sample
+  // kernel, which reads all of A anyway, and W <- A never happens as a copy (pass 0 reads A, writes W).
   mark(RRF_PHASE_INIT, -1);
-  if (p->dtype == RRF_F64)
-    init_kernel<double><<<L.init_ctas, 256, 0, st>>>((const double*)dA, lda, inplace ? nullptr : (double*)W, ldw, m, n,
-                                                     (double*)dV, ldv, p->max_rank, init_part);
-  else
-    init_kernel<float><<<L.init_ctas, 256, 0, st>>>((const float*)dA, lda, inplace ? nullptr : (float*)W, ldw, m, n,
-                                                    (float*)dV, ldv, p->max_rank, init_part);
-  init_ctrl_kernel<<<1, 256, 0, st>>>(init_part, L.init_ctas, p->tol, p->tol_is_relative, fixed ? 1 : 0, b, p->max_rank,
-                                      ctrl, done_after, samp, steps, predict);
+  if (cudaMemsetAsync(ctrl, 0, 256, st) != cudaSuccess) return RRF_ERR_CUDA;   // also: the stop flag of the last run
+  if (cudaMemset2DAsync(dV, (size_t)ldv * esize, 0, (size_t)p->max_rank * esize, (size_t)m, st) != cudaSuccess)
+    return RRF_ERR_CUDA;
 
   // fork/join events for the side stream, created once and kept in the handle
   while (h->sync_events.size() < (size_t)3 * steps + 2) {
@@ -972,7 +972,9 @@ rrf_status_t rrf_run(rrf_handle_t h, const rrf_params_t* p, void* dA, int64_t ld
   src.ldy = b;
   src.row_off = 0;
   mark(RRF_PHASE_SAMPLE, 0);
-  ops->sample(tmW_s, tmO, Ypart, 0, (int)m, (int)n, 0, sp, ctrl, nullptr, st);
+  ops->sample(tmA_s, tmO, Ypart, 0, (int)m, (int)n, 0, sp, ctrl, nullptr, init_part, st);
+  init_ctrl_kernel<<<1, 256, 0, st>>>(init_part, std::min(sp.nslabs * sp.nseg, sp.ctas), p->tol, p->tol_is_relative,
+                                      fixed ? 1 : 0, b, p->max_rank, ctrl, done_after, samp, steps, predict);
 
   if (look_ctas == 0) {
     // One queue.  The panel of pass 0 is sampled by its own kernel; the panel of pass i+1 comes out
@@ -992,14 +994,14 @@ rrf_status_t rrf_run(rrf_handle_t h, const rrf_params_t* p, void* dA, int64_t ld
       if (s != RRF_OK) return panel_failed(s);
       const VtwPlan vp = plan_vtw(h->sms, rows, n, ops->v_bn);
       mark(RRF_PHASE_VTW, i);
-      ops->vtw(tmV_k, tmW_k, Zpart, r0, r0, vp, ctrl, st);
+      ops->vtw(tmV_k, i == 0 ? tmA_k : tmW_k, Zpart, r0, r0, vp, ctrl, st);
       mark(RRF_PHASE_TZ, i);
       cudaStreamWaitEvent(st, h->sync_events[2 * i + 1], 0);   // join: T_i is needed from here on
       ops->tz(Zpart, vp, Tblk(r0), p->max_rank, 1, Zt, &ctrl->done, st);
       const UpdPlan up = plan_upd(h->sms, rows, n, ops->u_bm, ops->u_bn, ops->u_wn);
       const int j0 = (i + 1 < steps) ? r0 + b : -1;   // Omega rows of the next pass, if there is one
       mark(RRF_PHASE_UPDATE, i);
-      ops->update(tmV_u, tmZ, tmW_u, tmO, W, ldw, (char*)dB + (size_t)r0 * ldb * esize, ldb, r0, rows, (int)n, r0, b,
+      ops->update(tmV_u, tmZ, i == 0 ? tmA_u : tmW_u, tmO, W, ldw, (char*)dB + (size_t)r0 * ldb * esize, ldb, r0, rows, (int)n, r0, b,
                   j0, Ypart, norm_part, up, ctrl, samp + i, st);
       mark(RRF_PHASE_STOP, i);
       stop_kernel<<<1, 256, 0, st>>>(norm_part, up.P, b, p->max_rank, p->estimator, fixed ? 1 : 0, tr_sub, tr_dir, ctrl,
@@ -1007,7 +1009,7 @@ rrf_status_t rrf_run(rrf_handle_t h, const rrf_params_t* p, void* dA, int64_t ld
       if (j0 >= 0 && predicting) {
         // the next panel, sampled on its own if the loop goes on and the update had been told to skip it
         const SamplePlan sp2 = plan_sample(h->sms, rows - b, n, esize, ops->s_kbs);
-        ops->sample(tmW_s, tmO, Ypart, r0 + b, rows - b, (int)n, j0, sp2, ctrl, samp + i, st);
+        ops->sample(tmW_s, tmO, Ypart, r0 + b, rows - b, (int)n, j0, sp2, ctrl, samp + i, nullptr, st);
         alt = PanelSource{};
         alt.nseg = sp2.nseg;
         alt.seg_stride = (long long)(rows - b) * b;
@@ -1059,7 +1061,7 @@ rrf_status_t rrf_run(rrf_handle_t h, const rrf_params_t* p, void* dA, int64_t ld
     if (steps > 1) {                  // the second panel is sampled while the first is factored
       mark(RRF_PHASE_SAMPLE, 0);
       const SamplePlan sp1 = plan_sample(gsms, m, n, esize, ops->s_kbs);   // beside the first panel
-      ops->sample(tmW_s, tmO, Ybuf[1], 0, (int)m, (int)n, b, sp1, ctrl, nullptr, st);
+      ops->sample(tmA_s, tmO, Ybuf[1], 0, (int)m, (int)n, b, sp1, ctrl, nullptr, nullptr, st);
       cudaEventRecord(evS2, st);
     }
     UpdPlan up_prev{};
@@ -1106,7 +1108,7 @@ rrf_status_t rrf_run(rrf_handle_t h, const rrf_params_t* p, void* dA, int64_t ld
       cudaStreamWaitEvent(st, evP(i), 0);
       const VtwPlan vp = plan_vtw(gate ? h->sms : gsms, rows, n, ops->v_bn);
       mark(RRF_PHASE_VTW, i);
-      ops->vtw(tmV_k, tmW_k, Zpart, r0, r0, vp, ctrl, st);
+      ops->vtw(tmV_k, i == 0 ? tmA_k : tmW_k, Zpart, r0, r0, vp, ctrl, st);
       mark(RRF_PHASE_TZ, i);
       ops->tz(Zpart, vp, Tblk(r0), p->max_rank, 1, Zt, &ctrl->done, st);
       if (i + 1 < steps && gate) {
@@ -1117,7 +1119,7 @@ rrf_status_t rrf_run(rrf_handle_t h, const rrf_params_t* p, void* dA, int64_t ld
       const UpdPlan up = plan_upd(gsms, rows, n, ops->u_bm, ops->u_bn, ops->u_wn);
       const int j0 = (i + 2 < steps) ? r0 + 2 * b : -1;   // Omega rows of the pass after the next
       mark(RRF_PHASE_UPDATE, i);
-      ops->update(tmV_u, tmZ, tmW_u, tmO, W, ldw, (char*)dB + (size_t)r0 * ldb * esize, ldb, r0, rows, (int)n, r0, b,
+      ops->update(tmV_u, tmZ, i == 0 ? tmA_u : tmW_u, tmO, W, ldw, (char*)dB + (size_t)r0 * ldb * esize, ldb, r0, rows, (int)n, r0, b,
                   j0, Ybuf[i & 1], norm_part, up, ctrl, samp + i, st);
       mark(RRF_PHASE_STOP, i);
       stop_kernel<<<1, 256, 0, st>>>(norm_part, up.P, b, p->max_rank, p->estimator, fixed ? 1 : 0, tr_sub, tr_dir, ctrl,
@@ -1126,7 +1128,7 @@ rrf_status_t rrf_run(rrf_handle_t h, const rrf_params_t* p, void* dA, int64_t ld
         // the panel of pass i+2, sampled on its own if the loop goes on and the update had been told to skip it;
         // its first b rows are the rows above that panel which the fix-up needs
         const SamplePlan sp2 = plan_sample(gsms, rows - b, n, esize, ops->s_kbs);
-        ops->sample(tmW_s, tmO, Ybuf[i & 1], r0 + b, rows - b, (int)n, j0, sp2, ctrl, samp + i, st);
+        ops->sample(tmW_s, tmO, Ybuf[i & 1], r0 + b, rows - b, (int)n, j0, sp2, ctrl, samp + i, nullptr, st);
         alt_prev = PanelSource{};
         alt_prev.nseg = sp2.nseg;
         alt_prev.seg_stride = (long long)(rows - b) * b;

@@ -53,7 +53,8 @@ __global__ void __launch_bounds__(WM* WN * 32)
                   const __grid_constant__ CUtensorMap tmO,  // OmegaT [max_rank][n], box [B][KE]
                   T* __restrict__ Ypart,                    // [nseg][rows][B]
                   int r0, int rows, int n, int j0, int nslabs, int nseg, int kt_per_seg, Ctrl* ctrl,
-                  const int* __restrict__ only_if_zero) {   // non-NULL: run only where the fused update skipped this panel
+                  const int* __restrict__ only_if_zero,     // non-NULL: run only where the fused update skipped this panel
+                  double* __restrict__ sq_part) {           // non-NULL: also per-CTA partial sums of squares of W
   if (*reinterpret_cast<volatile int*>(&ctrl->done)) return;
   if (only_if_zero != nullptr) {
     if (*only_if_zero != 0) return;
@@ -67,10 +68,15 @@ __global__ void __launch_bounds__(WM* WN * 32)
   extern __shared__ unsigned char smem_raw[];
   unsigned char* smem = align1024(smem_raw);
   __shared__ uint64_t full[STAGES];
+  __shared__ double red[32];
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
   const int wm = warp / WN, wn = warp % WN;
   const int KT = (n + KBS * KE - 1) / (KBS * KE);    // K tiles of KBS boxes
+  // ||W||_F^2 on the side (Algorithm 2 line 2): the warps of warp column 0 between them load every element
+  // of a W tile exactly once, and the items of the launch partition W
+  const bool take_sq = sq_part != nullptr && wn == 0;
+  double sq = 0.0;
 
   if (tid == 0) {
     for (int s = 0; s < STAGES; ++s) mbar_init(&full[s], 1);
@@ -126,6 +132,14 @@ __global__ void __launch_bounds__(WM* WN * 32)
             VecLoad16<T>::ld(sA + rlo * 128 + chunk, ra[a][0]);
             VecLoad16<T>::ld(sA + (rlo + 8) * 128 + chunk, ra[a][1]);
           }
+          if (take_sq) {
+#pragma unroll
+            for (int a = 0; a < MT; ++a)
+#pragma unroll
+              for (int h = 0; h < 2; ++h)
+#pragma unroll
+                for (int e = 0; e < NV; ++e) sq += (double)ra[a][h][e] * (double)ra[a][h][e];
+          }
 #pragma unroll
           for (int c = 0; c < NT; ++c) {
             const int rn = wn * TN + c * 8 + g;
@@ -158,6 +172,10 @@ __global__ void __launch_bounds__(WM* WN * 32)
         if (row < rows) store2(Y + (size_t)row * B + col, acc[a][c][0], acc[a][c][1]);
         if (row + 8 < rows) store2(Y + (size_t)(row + 8) * B + col, acc[a][c][2], acc[a][c][3]);
       }
+  }
+  if (sq_part != nullptr) {
+    const double tot = block_sum(sq, red);     // fixed order within the CTA; the CTA's items in their order
+    if (tid == 0) sq_part[blockIdx.x] = tot;
   }
 }
 

@@ -647,33 +647,9 @@ __global__ void __launch_bounds__(kTzThreads)
 }
 
 // ------------------------------------------------------------------------------------------
-// Algorithm 2 lines 1-3: W <- A (unless in place), partial sums of ||A||_F^2, V <- 0.
-// Fixed chunking and fixed-order reductions: the result does not depend on scheduling.
+// Algorithm 2 lines 2-4: ||A||_F^2 from the first sample kernel's per-CTA partial sums (fixed order), the
+// squared tolerance, and the loop state.
 // ------------------------------------------------------------------------------------------
-template <typename T>
-__global__ void __launch_bounds__(256)
-    init_kernel(const T* __restrict__ A, long long lda, T* __restrict__ W, long long ldw, long long m, long long n,
-                T* __restrict__ V, long long ldv, int vcols, double* __restrict__ part) {
-  __shared__ double red[32];
-  // CTA c owns rows [c*rpc, (c+1)*rpc): fixed chunking, so the partial sums do not depend on scheduling
-  const long long rpc = (m + gridDim.x - 1) / gridDim.x;
-  const long long r_lo = (long long)blockIdx.x * rpc, r_hi = min(m, r_lo + rpc);
-  double s = 0.0;
-  for (long long r = r_lo; r < r_hi; ++r) {
-    const T* src = A + r * lda;
-    T* dst = W != nullptr ? W + r * ldw : nullptr;
-    for (long long c = threadIdx.x; c < n; c += 256) {
-      const T x = src[c];
-      if (dst != nullptr) dst[c] = x;
-      s += (double)x * (double)x;
-    }
-    T* vrow = V + r * ldv;
-    for (int c = threadIdx.x; c < vcols; c += 256) vrow[c] = T(0);
-  }
-  const double tot = block_sum(s, red);
-  if (threadIdx.x == 0) part[blockIdx.x] = tot;
-}
-
 __global__ void __launch_bounds__(256)
     init_ctrl_kernel(const double* __restrict__ part, int npart, double tol, int relative, int fixed_rank,
                      int b, int max_rank, Ctrl* ctrl, int* __restrict__ done_after, int* __restrict__ samp, int nsteps,
