@@ -1245,7 +1245,7 @@ rrf_status_t rrf_run(rrf_handle_t h, const rrf_params_t* p, void* dA, int64_t ld
     const int lag = look_ctas > 0 ? 2 : 1;
     // without the predictor every executed pass that has a later panel to sample samples it
     out->fused_samples = predicting ? hc.fused_samples : std::min(hc.steps, std::max(0, steps - lag));
-    out->kernel_launches = 2 + (dOmegaT == nullptr ? 1 : 0) + 1 + ((look_ctas > 0 && steps > 1) ? 1 : 0) + 6 * steps +
+    out->kernel_launches = 1 + (dOmegaT == nullptr ? 1 : 0) + 1 + ((look_ctas > 0 && steps > 1) ? 1 : 0) + 6 * steps +
                            (predicting ? std::max(0, steps - lag) : 0);
   }
   out->extra_samples = hc.extra_samples;
