@@ -339,6 +339,10 @@ struct PanelOpts {
   PanelFix fix{};                  // look-ahead fix-up (enabled == 0: none)
   int ctas = 0;                    // 0: one slab per SM; > 0: confine the panel to this many CTAs
   unsigned* bar_reset = nullptr;   // the T-factor kernel zeroes this word (the panel's barrier counter)
+  bool merge_t = false;            // CTA 0 of the panel kernel builds T itself: no T-factor launch
+  unsigned bar_base = 0;           // value of the barrier counter when this launch starts (it is not reset
+                                   // between the launches of the look-ahead schedule)
+  unsigned* bar_used = nullptr;    // out: what this launch adds to the counter
   cudaStream_t st_t = nullptr;     // side stream for the T factor, with its fork / join events
   cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
 };
@@ -355,13 +359,17 @@ static rrf_status_t launch_panel(rrf_ctx* h, int dtype, const void* Y, PanelSour
   PanelFix fix = o.fix;
   PanelSource alt = o.alt;
   const int* fused_flag = o.fused_flag;
-  void* args[] = {&Y,   &src, &alt, &fused_flag, &rows_i, &b,    &R,         &Rp, &V,
-                  &ldv, &P,   &piv, &gram,       &tau,    &bar,  &ctrl, &done_flag, &fix};
+  unsigned bar_base = o.bar_base;
+  void* Tmerged = o.merge_t ? Tout : nullptr;
+  void* args[] = {&Y,   &src, &alt, &fused_flag, &rows_i, &b,    &R,    &Rp,        &V,   &ldv,      &P,
+                  &piv, &gram, &tau, &bar,       &ctrl,   &done_flag, &fix, &bar_base, &Tmerged, &ldt};
   const size_t tsmem = ((size_t)b * (b + 1) + (size_t)(b / 2) * (b / 2 + 1)) * sizeof(double);
+  if (o.merge_t) pp.smem = std::max(pp.smem, tsmem);
+  if (o.bar_used != nullptr) *o.bar_used = (unsigned)(b + (o.fix.enabled ? 2 : 0)) * (unsigned)pp.G;
   mark(RRF_PHASE_PANEL, step);
   const void* fn = dtype == RRF_F64 ? panel_variant<double>(pp.variant) : panel_variant<float>(pp.variant);
   cudaError_t e = cudaLaunchCooperativeKernel(fn, dim3(pp.G), dim3(kPanelThreads), args, pp.smem, st);
-  if (e == cudaSuccess) {
+  if (e == cudaSuccess && !o.merge_t) {
     cudaStream_t tt = st;
     if (o.ev_fork != nullptr) {          // fork: the T factor runs on the side stream after the panel
       cudaEventRecord(o.ev_fork, st);
@@ -1051,12 +1059,17 @@ rrf_status_t rrf_run(rrf_handle_t h, const rrf_params_t* p, void* dA, int64_t ld
     cudaEventRecord(evS, st);
     cudaStreamWaitEvent(h->aux, evS, 0);
     ps.bar = look_bar;
+    // the barrier counter is zeroed once per run and runs on from panel to panel (a panel that does not
+    // run because the loop has ended adds nothing, and then no later panel runs either)
+    unsigned bar_next = 0, bar_used = 0;
     PanelOpts po;
     po.ctas = look_ctas;
-    po.bar_reset = look_bar;
+    po.merge_t = true;
+    po.bar_used = &bar_used;
     s = launch_panel(h, p->dtype, Ybuf[0], src, m, b, Vblk(0), ldv, Tblk(0), p->max_rank, ps, ctrl, done_after, h->aux,
                      NoMark(), 0, po);
     if (s != RRF_OK) return panel_failed(s);
+    bar_next += bar_used;
     cudaEventRecord(evP(0), h->aux);
     if (steps > 1) {                  // the second panel is sampled while the first is factored
       mark(RRF_PHASE_SAMPLE, 0);
@@ -1082,6 +1095,7 @@ rrf_status_t rrf_run(rrf_handle_t h, const rrf_params_t* p, void* dA, int64_t ld
           sn.wn = ops->u_wn;
         }
         PanelOpts pn = po;
+        pn.bar_base = bar_next;
         if (i >= 1) {
           pn.alt = alt_prev;
           pn.fused_flag = predicting ? samp + (i - 1) : nullptr;
@@ -1097,7 +1111,10 @@ rrf_status_t rrf_run(rrf_handle_t h, const rrf_params_t* p, void* dA, int64_t ld
         const rrf_status_t ls = launch_panel(h, p->dtype, Ybuf[(i + 1) & 1], sn, rows - b, b, Vblk(r0 + b), ldv,
                                              Tblk(r0 + b), p->max_rank, ps, ctrl, done_after + i, h->aux, NoMark(),
                                              i + 1, pn);
-        if (ls == RRF_OK) cudaEventRecord(evP(i + 1), h->aux);
+        if (ls == RRF_OK) {
+          cudaEventRecord(evP(i + 1), h->aux);
+          bar_next += bar_used;
+        }
         return ls;
       };
       if (i + 1 < steps && !gate) {
@@ -1245,7 +1262,9 @@ rrf_status_t rrf_run(rrf_handle_t h, const rrf_params_t* p, void* dA, int64_t ld
     const int lag = look_ctas > 0 ? 2 : 1;
     // without the predictor every executed pass that has a later panel to sample samples it
     out->fused_samples = predicting ? hc.fused_samples : std::min(hc.steps, std::max(0, steps - lag));
-    out->kernel_launches = 1 + (dOmegaT == nullptr ? 1 : 0) + 1 + ((look_ctas > 0 && steps > 1) ? 1 : 0) + 6 * steps +
+    out->kernel_launches = 1 + (dOmegaT == nullptr ? 1 : 0) + 1 + ((look_ctas > 0 && steps > 1) ? 1 : 0) +
+                           (look_ctas > 0 ? 5 : 6) * steps +   // look-ahead: the panel kernel builds T itself
+                          
                            (predicting ? std::max(0, steps - lag) : 0);
   }
   out->extra_samples = hc.extra_samples;

@@ -120,6 +120,78 @@ __device__ __forceinline__ double panel_entry(const T* __restrict__ Y, const Pan
   return s;
 }
 
+// Compact-WY factor T from the Gram rows and tau, by recursive doubling (see tfactor_kernel below).
+// The block-level body: every thread of one CTA calls it; `tsm` holds b*(b+1) + (b/2)*(b/2+1) doubles.
+template <typename T>
+__device__ __forceinline__ void tfactor_block(const double* __restrict__ gram, const double* __restrict__ tau, int b,
+                                              T* __restrict__ Tout, long long ldt, double* tsm) {
+  const int pitch = b + 1, mp = b / 2 + 1;
+  double* Ts = tsm;                        // [b][pitch]: T above and on the diagonal, Gram rows below
+  double* Ms = Ts + (size_t)b * pitch;     // [b/2][mp]: (V1^T V2) T22 of every pair of the current round
+  const int tid = threadIdx.x;
+  const int nthr = blockDim.x;
+  // stage the Gram rows (strictly lower triangle) and tau: eight independent loads in flight per thread
+  for (int base = 0; base < b * b; base += nthr * 8) {
+    double v[8];
+#pragma unroll
+    for (int e = 0; e < 8; ++e) {
+      const int idx = base + e * nthr + tid;
+      const int r = idx / b, c = idx - r * b;
+      v[e] = (idx < b * b && c < r) ? __ldcg(gram + idx) : 0.0;
+    }
+#pragma unroll
+    for (int e = 0; e < 8; ++e) {
+      const int idx = base + e * nthr + tid;
+      const int r = idx / b, c = idx - r * b;
+      if (idx < b * b) Ts[r * pitch + c] = v[e];
+    }
+  }
+  __syncthreads();
+  if (tid < b) Ts[tid * pitch + tid] = __ldcg(tau + tid);
+  __syncthreads();
+  for (int s = 1; s < b; s <<= 1) {
+    const int per_level = b * s / 2;       // (b / 2s) pairs x s x s entries
+    const int ls = 31 - __clz(s);          // s is a power of two
+    for (int idx = tid; idx < per_level; idx += nthr) {
+      const int q = idx >> (2 * ls), rc = idx & (s * s - 1), r = rc >> ls, c = rc & (s - 1);
+      const int o = 2 * s * q;
+      // M[r][c] = sum_{k <= c} (v_{o+r}^T v_{o+s+k}) T22[k][c]; two independent partial sums
+      const double* ga = Ts + (size_t)(o + s) * pitch + (o + r);
+      const double* tb = Ts + (size_t)(o + s) * pitch + (o + s + c);
+      double a0 = 0.0, a1 = 0.0;
+      int k = 0;
+      for (; k + 1 <= c; k += 2) {
+        a0 += ga[k * pitch] * tb[k * pitch];
+        a1 += ga[(k + 1) * pitch] * tb[(k + 1) * pitch];
+      }
+      if (k <= c) a0 += ga[k * pitch] * tb[k * pitch];
+      Ms[(s * q + r) * mp + c] = a0 + a1;
+    }
+    __syncthreads();
+    for (int idx = tid; idx < per_level; idx += nthr) {
+      const int q = idx >> (2 * ls), rc = idx & (s * s - 1), r = rc >> ls, c = rc & (s - 1);
+      const int o = 2 * s * q;
+      // T12[r][c] = -sum_{k >= r} T11[r][k] M[k][c]
+      const double* ta = Ts + (size_t)(o + r) * pitch + o;
+      const double* mb = Ms + (size_t)(s * q) * mp + c;
+      double a0 = 0.0, a1 = 0.0;
+      int k = r;
+      for (; k + 1 < s; k += 2) {
+        a0 += ta[k] * mb[k * mp];
+        a1 += ta[k + 1] * mb[(k + 1) * mp];
+      }
+      if (k < s) a0 += ta[k] * mb[k * mp];
+      Ts[(o + r) * pitch + (o + s + c)] = -(a0 + a1);
+    }
+    __syncthreads();
+  }
+  for (int idx = tid; idx < b * b; idx += nthr) {
+    const int r = idx / b, c = idx - r * b;
+    Tout[(size_t)r * ldt + c] = c >= r ? (T)Ts[r * pitch + c] : T(0);
+  }
+}
+
+
 // The 16 warps of a CTA form RH row groups of 16/RH warps; a lane looks after QMAX rows of its
 // group (kept in registers during a pass), so a slab holds up to 32 * QMAX * RH rows.  With PAD the
 // slab is allocated at that full height and zero filled below its last row, which removes every
@@ -134,7 +206,9 @@ __global__ void __launch_bounds__(kPanelThreads)
                  double* __restrict__ piv,           // [2][b] broadcast pivot row
                  double* __restrict__ gram,          // [b][b] strictly-lower part: v_c^T v_j (c < j)
                  double* __restrict__ tau_out,       // [b]
-                 unsigned* bar, Ctrl* ctrl, const int* done_flag, PanelFix fix) {
+                 unsigned* bar, Ctrl* ctrl, const int* done_flag, PanelFix fix,
+                 unsigned bar_base,                 // value of the barrier counter when this launch starts
+                 T* __restrict__ Tout, long long ldt) {   // non-NULL: CTA 0 also builds the T factor at the end
   if (*reinterpret_cast<const volatile int*>(done_flag)) return;
   // the panel's entries were sampled by the fused update, or - where the predictor had skipped that - by
   // the separate sample kernel, in its layout
@@ -251,7 +325,7 @@ __global__ void __launch_bounds__(kPanelThreads)
         }
       }
     }
-    if (!grid_barrier(bar, (++nbar) * (unsigned)G, ctrl)) return;
+    if (!grid_barrier(bar, bar_base + (++nbar) * (unsigned)G, ctrl)) return;
     // Phase 2: CTA c owns columns c, c + G, ... of G = sum of the partials (in CTA order) and of
     // M = Tp^T G, column by column: M[k][c2] = sum_{l <= k} Tp[l][k] G[l][c2].
     {
@@ -289,7 +363,7 @@ __global__ void __launch_bounds__(kPanelThreads)
         }
       }
     }
-    if (!grid_barrier(bar, (++nbar) * (unsigned)G, ctrl)) return;
+    if (!grid_barrier(bar, bar_base + (++nbar) * (unsigned)G, ctrl)) return;
     // Phase 3: S -= Vp[slab] M.  A task is a 16-row x 8-column tile of a chunk.
     {
       const int PV = b + 4, PM = b + 8;
@@ -397,7 +471,7 @@ __global__ void __launch_bounds__(kPanelThreads)
     }
     if (pr >= gr0 && pr < gr0 + nloc)
       for (int c = tid; c < b; c += NT) piv[(j & 1) * b + c] = S[(size_t)c * Rp + (pr - gr0)];
-    if (!grid_barrier(bar, (++nbar) * (unsigned)G, ctrl)) return;
+    if (!grid_barrier(bar, bar_base + (++nbar) * (unsigned)G, ctrl)) return;
 
     // every CTA: sum of the per-CTA partials in a fixed order (lane x takes CTAs x, x+32, ...;
     // then the fixed shuffle tree), one warp per column, CG columns of loads in flight at once
@@ -467,6 +541,11 @@ __global__ void __launch_bounds__(kPanelThreads)
     const int r = idx >> lb, c = idx & (b - 1);
     if (gr0 + r >= row0) V[(size_t)(gr0 + r - row0) * ldv + c] = (T)S[(size_t)c * Rp + r];
   }
+  // CTA 0 wrote the Gram rows and tau itself: it can go on to the T factor without another launch
+  if (Tout != nullptr && cta == 0) {
+    __syncthreads();
+    tfactor_block<T>(gram, tau_out, b, Tout, ldt, psm);
+  }
 }
 
 // ------------------------------------------------------------------------------------------
@@ -484,70 +563,8 @@ __global__ void __launch_bounds__(256)
                    T* __restrict__ Tout, long long ldt, const int* done_flag, unsigned* bar_reset) {
   if (*reinterpret_cast<const volatile int*>(done_flag)) return;
   if (threadIdx.x == 0 && bar_reset != nullptr) *bar_reset = 0;   // the panel before this kernel is finished with it
-  extern __shared__ double tsm[];
-  const int pitch = b + 1, mp = b / 2 + 1;
-  double* Ts = tsm;                        // [b][pitch]: T above and on the diagonal, Gram rows below
-  double* Ms = Ts + (size_t)b * pitch;     // [b/2][mp]: (V1^T V2) T22 of every pair of the current round
-  const int tid = threadIdx.x;
-  // stage the Gram rows (strictly lower triangle) and tau: eight independent loads in flight per thread
-  for (int base = 0; base < b * b; base += 256 * 8) {
-    double v[8];
-#pragma unroll
-    for (int e = 0; e < 8; ++e) {
-      const int idx = base + e * 256 + tid;
-      const int r = idx / b, c = idx - r * b;
-      v[e] = (idx < b * b && c < r) ? __ldcg(gram + idx) : 0.0;
-    }
-#pragma unroll
-    for (int e = 0; e < 8; ++e) {
-      const int idx = base + e * 256 + tid;
-      const int r = idx / b, c = idx - r * b;
-      if (idx < b * b) Ts[r * pitch + c] = v[e];
-    }
-  }
-  __syncthreads();
-  if (tid < b) Ts[tid * pitch + tid] = __ldcg(tau + tid);
-  __syncthreads();
-  for (int s = 1; s < b; s <<= 1) {
-    const int per_level = b * s / 2;       // (b / 2s) pairs x s x s entries
-    const int ls = 31 - __clz(s);          // s is a power of two
-    for (int idx = tid; idx < per_level; idx += 256) {
-      const int q = idx >> (2 * ls), rc = idx & (s * s - 1), r = rc >> ls, c = rc & (s - 1);
-      const int o = 2 * s * q;
-      // M[r][c] = sum_{k <= c} (v_{o+r}^T v_{o+s+k}) T22[k][c]; two independent partial sums
-      const double* ga = Ts + (size_t)(o + s) * pitch + (o + r);
-      const double* tb = Ts + (size_t)(o + s) * pitch + (o + s + c);
-      double a0 = 0.0, a1 = 0.0;
-      int k = 0;
-      for (; k + 1 <= c; k += 2) {
-        a0 += ga[k * pitch] * tb[k * pitch];
-        a1 += ga[(k + 1) * pitch] * tb[(k + 1) * pitch];
-      }
-      if (k <= c) a0 += ga[k * pitch] * tb[k * pitch];
-      Ms[(s * q + r) * mp + c] = a0 + a1;
-    }
-    __syncthreads();
-    for (int idx = tid; idx < per_level; idx += 256) {
-      const int q = idx >> (2 * ls), rc = idx & (s * s - 1), r = rc >> ls, c = rc & (s - 1);
-      const int o = 2 * s * q;
-      // T12[r][c] = -sum_{k >= r} T11[r][k] M[k][c]
-      const double* ta = Ts + (size_t)(o + r) * pitch + o;
-      const double* mb = Ms + (size_t)(s * q) * mp + c;
-      double a0 = 0.0, a1 = 0.0;
-      int k = r;
-      for (; k + 1 < s; k += 2) {
-        a0 += ta[k] * mb[k * mp];
-        a1 += ta[k + 1] * mb[(k + 1) * mp];
-      }
-      if (k < s) a0 += ta[k] * mb[k * mp];
-      Ts[(o + r) * pitch + (o + s + c)] = -(a0 + a1);
-    }
-    __syncthreads();
-  }
-  for (int idx = tid; idx < b * b; idx += 256) {
-    const int r = idx / b, c = idx - r * b;
-    Tout[(size_t)r * ldt + c] = c >= r ? (T)Ts[r * pitch + c] : T(0);
-  }
+  extern __shared__ double tsm_k[];
+  tfactor_block<T>(gram, tau, b, Tout, ldt, tsm_k);
 }
 
 // ------------------------------------------------------------------------------------------
