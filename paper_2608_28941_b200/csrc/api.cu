@@ -1264,7 +1264,6 @@ rrf_status_t rrf_run(rrf_handle_t h, const rrf_params_t* p, void* dA, int64_t ld
     out->fused_samples = predicting ? hc.fused_samples : std::min(hc.steps, std::max(0, steps - lag));
     out->kernel_launches = 1 + (dOmegaT == nullptr ? 1 : 0) + 1 + ((look_ctas > 0 && steps > 1) ? 1 : 0) +
                            (look_ctas > 0 ? 5 : 6) * steps +   // look-ahead: the panel kernel builds T itself
-                          
                            (predicting ? std::max(0, steps - lag) : 0);
   }
   out->extra_samples = hc.extra_samples;
