@@ -95,7 +95,9 @@ typedef struct {
 } rrf_result_t;
 
 /* Create / destroy a context bound to one CUDA device.  rrf_create makes `device`
- * current, queries its limits and allocates the context's status words. */
+ * current, queries its limits and allocates the context's status words.  A handle keeps per-call
+ * state (events, a side stream, the captured graph of the last repeated call): use it from one thread
+ * at a time, and do not overlap two rrf_run calls on the same handle. */
 rrf_status_t rrf_create(rrf_handle_t* out, int device);
 rrf_status_t rrf_destroy(rrf_handle_t h);
 
