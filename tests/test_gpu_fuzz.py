@@ -1,0 +1,83 @@
+"""Seeded random sweep of shapes, block sizes, schedules and sampling modes against the oracle.
+
+Sixty small problems (ragged sizes, ranks from 1 to full, tolerances over eight decades, both precisions, both
+estimators, fixed-rank mode, one and two queues, every sampling mode).  Compared: k (unless the oracle's own
+stopping quantity sits within 1e-6 / 1e-2 of the threshold, where either answer is right), B, Q^T Q and Q B.
+Where a late block is sampled from a residual that is pure rounding noise (exactly rank-deficient inputs) B and
+Q are not unique, and the test falls back to what is: the residual norm and the orthogonality."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import rrf_oracle as orc
+from paper_2608_28941_b200 import rrf
+
+pytestmark = pytest.mark.gpu
+
+
+def _relmax(x, ref):
+    s = np.max(np.abs(ref)) if ref.size else 1.0
+    return np.max(np.abs(x - ref)) / (s if s > 0 else 1.0) if ref.size else 0.0
+
+
+def _pad(x, mult):
+    r, c = x.shape
+    ld = (c + mult - 1) // mult * mult
+    buf = torch.zeros((r, ld), dtype=torch.from_numpy(x).dtype, device="cuda")
+    buf[:, :c] = torch.from_numpy(x).cuda()
+    return buf[:, :c]
+
+
+@pytest.mark.parametrize("seed", range(60))
+def test_random_problem(seed):
+    rng = np.random.default_rng(9000 + seed)
+    h = rrf.rrf_create(0)
+    try:
+        dt = "f64" if rng.random() < 0.75 else "f32"
+        b = int(rng.choice([16, 32, 64, 128] if dt == "f64" else [32, 64, 128]))
+        maxr = b * int(rng.integers(1, 7))
+        m = int(rng.integers(maxr, maxr + 1500))
+        n = int(rng.integers(maxr, maxr + 1500))
+        rank = int(rng.integers(1, max(2, min(m, n))))
+        sv = np.logspace(0, -float(rng.choice([2.0, 6.0, 12.0])), rank)
+        A = (rng.standard_normal((m, rank)) * sv) @ rng.standard_normal((rank, n))
+        Om = rng.standard_normal((n, maxr))
+        est = int(rng.integers(0, 2))
+        if est == 0:
+            tol = float(10.0 ** rng.uniform(-9, -1)) if dt == "f64" else float(10.0 ** rng.uniform(-4, -1))
+        else:   # Algorithm 2 line 9 cancels: keep the tolerance above its rounding floor
+            tol = float(10.0 ** rng.uniform(-6, -1)) if dt == "f64" else float(10.0 ** rng.uniform(-2.3, -1))
+        sched = int(rng.choice([0, rrf.RRF_FLAG_ONE_QUEUE, rrf.RRF_FLAG_TWO_QUEUES]))
+        samp = int(rng.choice([0, rrf.RRF_FLAG_SAMPLE_ALWAYS, rrf.RRF_FLAG_SAMPLE_NEVER]))
+        fixed = rrf.RRF_FLAG_FIXED_RANK if rng.random() < 0.15 else 0
+        npdt = np.float64 if dt == "f64" else np.float32
+        A = np.ascontiguousarray(A.astype(npdt))
+        OmT = np.ascontiguousarray(Om.T.astype(npdt))
+        mult = 2 if dt == "f64" else 4
+        g = rrf.rrf_run(h, _pad(A, mult), b, tol, maxr, omegaT=_pad(OmT, mult), estimator=est, flags=sched | samp | fixed)
+        A64, Om64 = A.astype(np.float64), OmT.T.astype(np.float64)
+        if fixed:   # the oracle has no fixed-rank switch: tolerance 0 on the residual norm runs it to the cap
+            o = orc.rrf(A64, Om64, b, 0.0, maxr, estimator="direct")
+        else:
+            o = orc.rrf(A64, Om64, b, tol, maxr, estimator="direct" if est == 0 else "subtractive")
+        trace = o.E_dir if est == 0 else o.E_sub
+        near = 1e-6 if dt == "f64" else 1e-2
+        marginal = (not fixed) and any(abs(e / max(o.normA2 * tol * tol, 1e-300) - 1.0) < near for e in trace)
+        if not marginal:
+            assert g.k == o.k, (g.k, o.k)
+        k = min(g.k, o.k)
+        if k == 0:
+            return
+        B = g.B[:k].cpu().numpy().astype(np.float64)
+        Q = rrf.rrf_form_q(h, g.V, g.T, b, k).cpu().numpy().astype(np.float64)
+        orth = np.linalg.norm(Q.T @ Q - np.eye(k))
+        assert orth <= (1e-11 if dt == "f64" else 1e-4), orth
+        bar = 5e-8 if dt == "f64" else 1e-2
+        eB = _relmax(B, o.B[:k])
+        eQB = _relmax(Q @ B, orc.form_q(o.V[:, :k], o.T[:, :k], b) @ o.B[:k])
+        if eB > bar or eQB > bar:
+            res_g = np.linalg.norm(A64 - Q @ B)
+            res_o = np.sqrt(max(o.E_dir[k // b - 1], 0.0))
+            assert abs(res_g - res_o) <= 1e-6 * np.linalg.norm(A64) + 0.05 * res_o, (eB, eQB, res_g, res_o)
+    finally:
+        rrf.rrf_destroy(h)
