@@ -265,3 +265,40 @@ def test_subspace_transfer_pins():
     got = orc.subspace_transfer(small.V, small.T, other.V, other.T, b, M)
     assert got.shape == (48, 70)
     assert np.max(np.abs(got - want)) < 1e-9 * np.max(np.abs(want))
+
+
+def test_householder_keeps_orthogonality_where_block_gram_schmidt_loses_it():
+    """The paper's stability experiment (1024 x 1024, singular values 1 ... 1e-14, b = 64, single precision),
+    qualitatively: without reorthogonalisation the Gram-Schmidt range finder loses orthogonality while its own
+    stopping quantity keeps falling; with it, and for the Householder method, Q stays orthonormal to single
+    precision and the projection residual follows the singular values down to the fp32 floor."""
+    from oracle import bcgs_foil
+    rng = np.random.default_rng(2024)
+    n, b, passes = 1024, 64, 10
+    U, _ = np.linalg.qr(rng.standard_normal((n, n)))
+    Vv, _ = np.linalg.qr(rng.standard_normal((n, n)))
+    s = np.logspace(0, -14, n)
+    A = ((U * s) @ Vv.T).astype(np.float32)
+    Om = rng.standard_normal((n, passes * b)).astype(np.float32)
+    A64 = A.astype(np.float64)
+
+    def orth_loss(Q):
+        Q = Q.astype(np.float64)
+        return np.linalg.norm(Q.T @ Q - np.eye(Q.shape[1]), 2)
+
+    def proj_res(Q):
+        Q = Q.astype(np.float64)
+        return np.linalg.norm(A64 - Q @ (Q.T @ A64), 2)
+
+    Q_plain, _, tracked_plain = bcgs_foil.bcgs_range_finder(A, Om, b, passes, reorth=False)
+    Q_re, _, _ = bcgs_foil.bcgs_range_finder(A, Om, b, passes, reorth=True)
+    hh = orc.rrf(A, Om, b, 0.0, passes * b, dtype=np.float32)
+    Q_hh = orc.form_q(hh.V.astype(np.float64), hh.T.astype(np.float64), b)
+    u32 = 6e-8
+    assert orth_loss(Q_hh) < 100 * u32 and orth_loss(Q_re) < 100 * u32
+    assert orth_loss(Q_plain) > 1e4 * u32                          # orthogonality gone ...
+    assert proj_res(Q_plain) > 30 * proj_res(Q_hh)                 # ... and with it the approximation,
+    assert tracked_plain[-1] < 0.1 * proj_res(Q_plain)             # which its stopping quantity does not see
+    # Householder and reorthogonalised Gram-Schmidt both reach the single-precision floor of this matrix
+    floor = np.linalg.svd(A64, compute_uv=False)[passes * b]
+    assert proj_res(Q_hh) < 50 * max(floor, u32) and proj_res(Q_re) < 50 * max(floor, u32)
