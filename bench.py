@@ -296,30 +296,49 @@ def main():
         B_h = torch.empty((w.max_rank, w.n), dtype=tdt).pin_memory()
         V_h = torch.empty((w.m, w.max_rank), dtype=tdt).pin_memory()
         T_h = torch.empty((w.b, w.max_rank), dtype=tdt).pin_memory()
-        A_d = torch.empty_like(A)
-        O_d = torch.empty_like(OmT)
+        # Two sets of device input buffers: the inputs of step s+1 travel on a copy stream while step s
+        # computes and its results go back, as a caller that streams problems through the library would do.
+        # Every step still pays its own host-to-device copy and device-to-host read inside the timed region.
+        A_d = [torch.empty_like(A), torch.empty_like(A)]
+        O_d = [torch.empty_like(OmT), torch.empty_like(OmT)]
+        arrived = [torch.cuda.Event(), torch.cuda.Event()]
+        copy_stream = torch.cuda.Stream()
 
-        def e2e_step():
-            A_d.copy_(A_h, non_blocking=True)
-            O_d.copy_(O_h, non_blocking=True)
-            r = rrf.rrf_run(h, A_d, w.b, w.tol, w.max_rank, omegaT=O_d, V=V, T=T, B=B, workspace=ws, flags=sched)
-            B_h[:r.k].copy_(B[:r.k], non_blocking=True)
-            V_h[:, :r.k].copy_(V[:, :r.k], non_blocking=True)
-            T_h[:, :r.k].copy_(T[:, :r.k], non_blocking=True)
+        def send(slot):
+            with torch.cuda.stream(copy_stream):
+                A_d[slot].copy_(A_h, non_blocking=True)
+                O_d[slot].copy_(O_h, non_blocking=True)
+                arrived[slot].record(copy_stream)
+
+        def e2e_loop(nsteps):
+            copy_stream.wait_stream(torch.cuda.current_stream())
+            send(0)
+            r = None
+            for s in range(nsteps):
+                slot = s & 1
+                if s + 1 < nsteps:
+                    send(1 - slot)                 # the previous user of that slot has finished: rrf_run synchronises
+                torch.cuda.current_stream().wait_event(arrived[slot])
+                r = rrf.rrf_run(h, A_d[slot], w.b, w.tol, w.max_rank, omegaT=O_d[slot], V=V, T=T, B=B, workspace=ws,
+                                flags=sched | rrf.RRF_FLAG_NO_GRAPH)     # the input buffers alternate: nothing to replay
+                B_h[:r.k].copy_(B[:r.k], non_blocking=True)
+                V_h[:, :r.k].copy_(V[:, :r.k], non_blocking=True)
+                T_h[:, :r.k].copy_(T[:, :r.k], non_blocking=True)
             torch.cuda.current_stream().synchronize()
             return r
-        e2e_step()
+        e2e_loop(2)
         barrier()
-        n_e2e = max(2, min(args.steps, 5))
+        n_e2e = max(2, min(args.steps, 6))
         e0.record()
-        for _ in range(n_e2e):
-            e2e_step()
+        e2e_loop(n_e2e)
         e1.record()
         barrier()
         ms_e2e = max_over_ranks(e0.elapsed_time(e1), world, dev) / n_e2e
         e2e = {"value": job_tflops(flops, world, ms_e2e), "unit": "TFLOP/s", "ms_per_step": ms_e2e,
                "h2d_bytes_per_step": int((A_h.numel() + O_h.numel()) * esize),
-               "d2h_bytes_per_step": int((k * w.n + w.m * k + w.b * k) * esize)}
+               "d2h_bytes_per_step": int((k * w.n + w.m * k + w.b * k) * esize),
+               "pipelined": "inputs of step s+1 are copied on a second stream while step s computes; %d steps timed, "
+                            "first copy not overlapped" % n_e2e}
 
     # ---- roofline of the dominant kernel, from the event profile of the timed region
     roofline = None
