@@ -11,12 +11,15 @@ Readings of the paper taken here:
   * Algorithm 2 line 8 applies Q_i^T = I - V_i T_i^T V_i^T (Theorem 3.1 and
     step 3 of the recursive QB recipe say "A <- Q_1^T A").
   * "qr(.)" / geqrt: LAPACK's Householder convention, beta = -sign(alpha)*||x||,
-    v[0] = 1, tau = (beta - alpha)/beta, H = I - tau v v^T; sign(0) = +1.
+    v[0] = 1, tau = (beta - alpha)/beta, H = I - tau v v^T.  The sign of a zero pivot is
+    the sign of the zero, as in LAPACK (beta = -SIGN(||x||, alpha)): alpha = +0.0 gives
+    beta = -||x||, alpha = -0.0 gives beta = +||x||.
   * tolerance: Frobenius norm, relative to ||A||_F when `relative` is set;
     the loop continues while E > sigma^2 (strict).
   * stopping quantity: `estimator="direct"` uses E = ||W[r0+b:, :]||_F^2, the
-    residual itself (section 3: the norm of the lower part of the updated
-    matrix); `estimator="subtractive"` is Algorithm 2 line 9 literally,
+    residual itself (section 3, after the Frobenius identity: the rows below
+    block row i of the updated matrix carry the whole remaining error);
+    `estimator="subtractive"` is Algorithm 2 line 9 literally,
     E <- E - ||B_i||_F^2.  Both are always recorded.
   * rank cap: the loop also ends when another block would exceed `max_rank`
     (the paper's fixed-rank mode).
@@ -55,7 +58,7 @@ def house(x: np.ndarray):
     v[0] = 1.0
     if xnorm == 0.0:
         return v, dt(0.0), alpha
-    sign = dt(1.0) if alpha >= 0.0 else dt(-1.0)
+    sign = dt(np.copysign(1.0, alpha))          # LAPACK's SIGN(., alpha): honours the sign of a zero
     beta = -sign * np.sqrt(alpha * alpha + xnorm * xnorm)
     tau = (beta - alpha) / beta
     v[1:] = tail / (alpha - beta)

@@ -67,6 +67,27 @@ def test_house_closed_form():
     assert tau == 0.0 and beta == 2.0 and np.allclose(v, [1, 0, 0])
 
 
+def test_house_at_a_zero_pivot():
+    # alpha = +0.0: beta = -||x||, tau = 1, v = [1, x_1/||x||, ...]; alpha = -0.0 takes the other sign
+    # (LAPACK's SIGN(., alpha) honours the sign of a zero, and "geqrt" is LAPACK's routine)
+    v, tau, beta = orc.house(np.array([0.0, 3.0, 4.0]))
+    assert beta == -5.0 and tau == 1.0 and np.allclose(v, [1.0, 0.6, 0.8], atol=1e-16)
+    v, tau, beta = orc.house(np.array([-0.0, 3.0, 4.0]))
+    assert beta == 5.0 and tau == 1.0 and np.allclose(v, [1.0, -0.6, -0.8], atol=1e-16)
+
+
+@pytest.mark.parametrize("zero", [0.0, -0.0])
+def test_panel_qr_with_a_zero_pivot_matches_lapack(zero):
+    rng = np.random.default_rng(5)
+    Y = rng.standard_normal((30, 5))
+    Y[0, 0] = zero                       # the first pivot is an exact (signed) zero
+    V, tau, T, R = orc.panel_qr(Y)
+    V_ref, tau_ref, R_ref = _lapack_vtau(Y)
+    assert np.allclose(V, V_ref, atol=1e-14) and np.allclose(tau, tau_ref, atol=1e-14)
+    assert np.allclose(R, R_ref, atol=1e-13)
+    assert np.sign(R[0, 0]) == (-1.0 if np.copysign(1.0, zero) > 0 else 1.0)
+
+
 # ---- P5: compact WY factor
 
 
