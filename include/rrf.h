@@ -72,6 +72,9 @@ typedef struct {
   int32_t tol_is_relative;  /* ... taken as tol*||A||_F if non-zero */
   uint32_t flags;
   uint64_t seed;            /* seed of the built-in Gaussian generator (used when dOmegaT == NULL) */
+  int32_t tune_panel_ctas;  /* look-ahead schedule: SMs given to the panel chain; 0 = the library's own rule */
+  int32_t tune_gate;        /* look-ahead schedule: 0 = own rule, 1 = start each panel as early as its inputs
+                               allow, 2 = hold it back until T^T Z of the pass is done (V^T W keeps every SM) */
 } rrf_params_t;
 
 typedef struct {
@@ -189,11 +192,14 @@ rrf_status_t rrf_panel_qr(rrf_handle_t h, int32_t dtype, int64_t rows, int32_t b
  *
  * The first call on each device looks up the array's device address (with that device current)
  * and raises the kernels' shared-memory limits; make that first call before starting any stream
- * capture.  Every call on a device shares the one array and finds the previous call's contents in
- * it: the entry point clears the words that must start at zero itself, but two calls whose kernels
- * overlap on the GPU (different streams, or different host threads) race on it - serialise them.
- * Unlike rrf_panel_qr this call synchronises `cuda_stream` before returning and returns the
- * device-side status (RRF_OK, or RRF_ERR_TIMEOUT if the bounded grid barrier gave up).
+ * capture.  That one-time set-up is guarded (std::call_once per device), so first calls from
+ * several host threads are safe.  Every call on a device shares the one array and finds the
+ * previous call's contents in it: the entry point clears the words that must start at zero
+ * itself, but two calls whose kernels overlap on the GPU (different streams, or different host
+ * threads) race on it - serialise them.
+ * Unlike rrf_panel_qr, EVERY call copies the device-side status back and synchronises
+ * `cuda_stream` before returning (RRF_OK, or RRF_ERR_TIMEOUT if the bounded grid barrier gave
+ * up), so it blocks the calling thread until the panel is factored.
  */
 rrf_status_t rrf_panel_qr_static(int32_t dtype, int64_t rows, int32_t b,
                                  const void* dY, int64_t ldy, void* dV, int64_t ldv,
@@ -202,8 +208,8 @@ rrf_status_t rrf_panel_qr_static(int32_t dtype, int64_t rows, int32_t b,
 /*
  * rrf_apply_qt / rrf_apply_q - C <- Q^T C or C <- Q C for a device matrix C (m x ncols,
  * ldc >= ncols) with Q = Q_0 ... Q_{k/b-1} given by V (m x k) and T (b x k, leading dimension
- * ldt) as rrf_run returns them (Algorithm 2 line 8 applied block by block; "Applying Q resolves
- * into a series of matrix-matrix products").  Workspace: rrf_apply_workspace_bytes().
+ * ldt) as rrf_run returns them (Algorithm 2 line 8 and Eq. "Q_i = I_m - V_i T_i V_i^T": Q is applied
+ * one block reflector after the other, each as three GEMMs).  Workspace: rrf_apply_workspace_bytes().
  * rrf_form_q writes the explicit basis Q = Q I[:, 0:k] (m x k, ldq >= k).  None of the three
  * synchronises the stream.
  */

@@ -5,6 +5,7 @@
 #include <cstdlib>
 #include <cmath>
 #include <cstring>
+#include <mutex>
 #include <new>
 #include <vector>
 
@@ -487,6 +488,7 @@ static rrf_status_t check_params(const rrf_params_t* p) {
   if (p->max_rank > p->m || p->max_rank > p->n) return RRF_ERR_INVALID_ARG;
   if (!(p->tol >= 0.0)) return RRF_ERR_INVALID_ARG;
   if (p->estimator != 0 && p->estimator != 1) return RRF_ERR_INVALID_ARG;
+  if (p->tune_panel_ctas < 0 || p->tune_gate < 0 || p->tune_gate > 2) return RRF_ERR_INVALID_ARG;
   return RRF_OK;
 }
 
@@ -538,7 +540,6 @@ rrf_status_t rrf_create(rrf_handle_t* out, int device) {
   if (e == cudaSuccess) e = cudaMalloc(&h->d_ctrl, sizeof(Ctrl));
   if (e == cudaSuccess) e = cudaMemset(h->d_ctrl, 0, sizeof(Ctrl));
   if (e != cudaSuccess) {
-    if (std::getenv("RRF_VERBOSE")) std::fprintf(stderr, "rrf_create: %s\n", cudaGetErrorString(e));
     delete h;
     return RRF_ERR_CUDA;
   }
@@ -858,7 +859,7 @@ rrf_status_t rrf_run(rrf_handle_t h, const rrf_params_t* p, void* dA, int64_t ld
           best = c;
         }
       }
-      if (const char* ev = std::getenv("RRF_LOOKAHEAD_CTAS")) best = std::min(cap, std::max(fewest, std::atoi(ev)));
+      if (p->tune_panel_ctas > 0) best = std::min(cap, std::max(fewest, (int)p->tune_panel_ctas));
       PanelPlan ppl;
       const bool wanted = (p->flags & RRF_FLAG_TWO_QUEUES) || best_t < pm.step_serial();
       if (wanted && plan_panel(h, m, b, &ppl, best, true)) look_ctas = best;
@@ -1047,9 +1048,8 @@ rrf_status_t rrf_run(rrf_handle_t h, const rrf_params_t* p, void* dA, int64_t ld
     // Where the update alone outlasts the next panel, the panel is held back until V^T W and T Z of
     // the pass are done, and V^T W gets every SM; otherwise the panel chain is the critical path and
     // starts as early as its inputs allow.
-    const char* gate_env = std::getenv("RRF_LOOKAHEAD_GATE");
     auto gated = [&](int rows_i) {
-      if (gate_env != nullptr) return std::atoi(gate_env) != 0;
+      if (p->tune_gate != 0) return p->tune_gate == 2;
       const PassModel pm{h->sms, (double)rows_i, (double)n, b, p->dtype == RRF_F64};
       return pm.step_gated(look_ctas) < pm.step_ungated(look_ctas);
     };
@@ -1171,8 +1171,7 @@ rrf_status_t rrf_run(rrf_handle_t h, const rrf_params_t* p, void* dA, int64_t ld
     };
     const void* ptrs[6] = {dA, dOmegaT, dV, dT, dB, d_workspace};
     const long long lds[4] = {lda, ldo, ldv, ldb};
-    const char* ge = std::getenv("RRF_LOOKAHEAD_GATE");
-    const int ints[3] = {look_ctas, h->profiling, ge != nullptr ? 1 + std::atoi(ge) : 0};
+    const int ints[2] = {look_ctas, h->profiling};
     put(p, sizeof(*p));
     put(ptrs, sizeof(ptrs));
     put(lds, sizeof(lds));
@@ -1291,7 +1290,8 @@ constexpr size_t kStaticScratchBytes = 512 * 1024;
 static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
 
 struct StaticDevice {
-  bool ready;
+  std::once_flag once;     // the set-up below runs once per device, whichever host thread calls first
+  cudaError_t err;
   unsigned char* ptr;      // device address of g_static_scratch on this device
   int sms;
   int panel_smem_max;
@@ -1312,7 +1312,6 @@ static cudaError_t static_setup(int dev, StaticDevice* sd) {
   e = setup_panel_kernels(smem_optin, &sd->panel_smem_max);
   if (e != cudaSuccess) return e;
   sd->ptr = static_cast<unsigned char*>(ptr);
-  sd->ready = true;
   return cudaSuccess;
 }
 
@@ -1326,7 +1325,8 @@ extern "C" rrf_status_t rrf_panel_qr_static(int32_t dtype, int64_t rows, int32_t
   int dev = -1;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kStaticMaxDevices) return RRF_ERR_CUDA;
   StaticDevice* sd = &g_static_dev[dev];
-  if (!sd->ready && static_setup(dev, sd) != cudaSuccess) return RRF_ERR_CUDA;
+  std::call_once(sd->once, [&] { sd->err = static_setup(dev, sd); });
+  if (sd->err != cudaSuccess || sd->ptr == nullptr) return RRF_ERR_CUDA;
   if (sd->sms > kMaxSms || kStaticCtrlBytes + panel_scratch_bytes(sd->sms, b) > kStaticScratchBytes)
     return RRF_ERR_WORKSPACE;
   rrf_ctx tmp{};                                            // host-side plan parameters only

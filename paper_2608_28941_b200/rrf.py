@@ -26,7 +26,7 @@ _lib = None
 class rrf_params_t(C.Structure):
     _fields_ = [("dtype", C.c_int32), ("b", C.c_int32), ("max_rank", C.c_int32), ("estimator", C.c_int32),
                 ("m", C.c_int64), ("n", C.c_int64), ("tol", C.c_double), ("tol_is_relative", C.c_int32),
-                ("flags", C.c_uint32), ("seed", C.c_uint64)]
+                ("flags", C.c_uint32), ("seed", C.c_uint64), ("tune_panel_ctas", C.c_int32), ("tune_gate", C.c_int32)]
 
 
 class rrf_result_t(C.Structure):
@@ -137,9 +137,10 @@ def rrf_destroy(h) -> None:
 
 
 def make_params(dtype: int, m: int, n: int, b: int, tol: float, max_rank: int, relative: bool = True,
-                estimator: int = 0, flags: int = 0, seed: int = 0) -> rrf_params_t:
+                estimator: int = 0, flags: int = 0, seed: int = 0, panel_ctas: int = 0, gate: int = 0) -> rrf_params_t:
     return rrf_params_t(dtype=dtype, b=b, max_rank=max_rank, estimator=estimator, m=m, n=n, tol=tol,
-                        tol_is_relative=1 if relative else 0, flags=flags, seed=seed)
+                        tol_is_relative=1 if relative else 0, flags=flags, seed=seed,
+                        tune_panel_ctas=panel_ctas, tune_gate=gate)
 
 
 def rrf_workspace_bytes(p: rrf_params_t) -> int:
@@ -174,12 +175,12 @@ class RunResult:
 def rrf_run(h, A: torch.Tensor, b: int, tol: float, max_rank: int, omegaT: torch.Tensor | None = None,
             relative: bool = True, estimator: int = 0, flags: int = 0, seed: int = 0,
             V: torch.Tensor | None = None, T: torch.Tensor | None = None, B: torch.Tensor | None = None,
-            workspace: torch.Tensor | None = None, check: bool = True) -> RunResult:
+            workspace: torch.Tensor | None = None, check: bool = True, panel_ctas: int = 0, gate: int = 0) -> RunResult:
     """Algorithm 2 on the device.  `omegaT` is max_rank x n (row j = j-th Gaussian vector) or None."""
     lib = load()
     m, n = A.shape
     dt = _dtype_code(A)
-    p = make_params(dt, m, n, b, tol, max_rank, relative, estimator, flags, seed)
+    p = make_params(dt, m, n, b, tol, max_rank, relative, estimator, flags, seed, panel_ctas, gate)
     need = C.c_size_t()
     s = lib.rrf_workspace_bytes(C.byref(p), C.byref(need))
     if s != RRF_OK:

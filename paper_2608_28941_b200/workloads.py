@@ -2,8 +2,8 @@
 
 This module only *generates inputs* (test matrices A with a prescribed
 spectrum and Gaussian sampling matrices Omega).  It contains none of the
-method's arithmetic and is imported by the tests, by the benchmark and by the
-golden-value script.  The CPU oracle and the CUDA library never import it:
+method's arithmetic and is imported by the tests, by the smoke check and by the
+benchmark.  The CPU oracle and the CUDA library never import it:
 they receive its arrays as arguments, so both sides see the same bytes.
 
 Workloads mirror the paper's experiments: matrices with prescribed singular

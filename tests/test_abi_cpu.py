@@ -24,7 +24,7 @@ def test_library_exports_every_declared_symbol(lib):
 
 
 def test_struct_layouts_match_header():
-    assert ctypes.sizeof(rrf.rrf_params_t) == 56
+    assert ctypes.sizeof(rrf.rrf_params_t) == 64
     assert ctypes.sizeof(rrf.rrf_result_t) == 72
 
 

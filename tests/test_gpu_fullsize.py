@@ -1,10 +1,11 @@
 """GPU parity at the full benchmark sizes, in the launch configuration bench.py times.
 
-Configs 2, 3 and 4 are small enough for the CPU oracle to run on the same inputs in seconds,
-so k, status, the stopping trace and B are compared element by element.  Config 5
-(32768 x 16384, rank cap 2048) is checked through properties that hold at any size:
-orthogonality of Q, B = Q^T A on sampled columns, the residual against the tolerance and the
-Eckart-Young tail of the known singular values, and triangularity of Q^T A Omega (Theorem 3.1)."""
+Every configuration is run through the CPU oracle on the same inputs, and k, status, the stopping
+trace, B, Q B and Q (per block, against the oracle's own envelope) are compared element by element;
+the oracle needs seconds for configs 2-4 and about a minute for config 5 (32768 x 16384, rank cap
+2048).  Config 5 is also checked through properties that hold at any size: orthogonality of Q,
+B = Q^T A on sampled columns, the residual against the tolerance and the Eckart-Young tail of the
+known singular values, and triangularity of Q^T A Omega (Theorem 3.1)."""
 import numpy as np
 import pytest
 import torch
@@ -38,7 +39,7 @@ def _orth_and_residual(h, w, g, A):
     return Q, B, orth, res
 
 
-@pytest.mark.parametrize("name", ["cfg2", "cfg3", "cfg4"])
+@pytest.mark.parametrize("name", ["cfg2", "cfg3", "cfg4", "cfg5"])
 def test_full_config_against_oracle(h, name):
     w = wl.CONFIGS[name]
     A, sig, Om, OmT = _gen(w)
@@ -51,8 +52,19 @@ def test_full_config_against_oracle(h, name):
     assert np.max(np.abs(Bg - o.B)) <= rel * np.max(np.abs(o.B))
     u = 1.1e-16 if w.dtype == "f64" else 6e-8
     d = 2 * max(w.m, w.n) * u * np.sqrt(o.normA2)
-    for a, c in zip(g.E_dir_trace, o.E_dir):
-        assert abs(a - c) <= 2 * np.sqrt(c) * d + d * d + 1e-9 * c
+    # the oracle's own envelope (float64: the column-permuted problem, x10; float32: the same steps in
+    # plain float32 on the CPU, x3) bounds what two correct implementations may differ by
+    A64 = A.cpu().numpy().astype(np.float64)
+    if w.dtype == "f64":
+        op = orc.permuted_rerun(A64, Om.astype(np.float64), w.b, w.tol, w.max_rank, seed=1)
+        mult = 10
+    else:
+        op = orc.rrf(A.cpu().numpy(), Om, w.b, w.tol, w.max_rank, dtype=np.float32)
+        mult = 3
+    same_k = op.k == o.k
+    for i, (a, c) in enumerate(zip(g.E_dir_trace, o.E_dir)):
+        slack = 1e-9 * c + (mult * abs(op.E_dir[i] - c) if same_k else 2 * np.sqrt(c) * d + d * d)
+        assert abs(a - c) <= slack, (i, a, c, slack)
     Q, B, orth, res = _orth_and_residual(h, w, g, A)
     assert orth <= (1e-12 if w.dtype == "f64" else 1e-5), orth
     assert abs(res ** 2 - o.E_dir[-1]) <= 1e-6 * o.E_dir[-1] + 2 * np.sqrt(o.E_dir[-1]) * d + d * d
@@ -69,14 +81,7 @@ def test_full_config_against_oracle(h, name):
     # is an ill-conditioned function of the input (float64: the oracle re-run on the column-permuted
     # problem, x10; float32: the same algorithm in plain float32 on the CPU, x3)
     Qg = Q.cpu().numpy()
-    A64 = A.cpu().numpy().astype(np.float64)
-    if w.dtype == "f64":
-        op = orc.permuted_rerun(A64, Om.astype(np.float64), w.b, w.tol, w.max_rank, seed=1)
-        mult = 10
-    else:
-        op = orc.rrf(A.cpu().numpy(), Om, w.b, w.tol, w.max_rank, dtype=np.float32)
-        mult = 3
-    env = orc.form_q(op.V.astype(np.float64), op.T.astype(np.float64), w.b) if op.k == o.k else None
+    env = orc.form_q(op.V.astype(np.float64), op.T.astype(np.float64), w.b) if same_k else None
     for i in range(k // w.b):
         blk = slice(i * w.b, (i + 1) * w.b)
         dq = np.max(np.abs(Qg[:, blk] - Qo[:, blk])) / np.max(np.abs(Qo))

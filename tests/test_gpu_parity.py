@@ -1,5 +1,5 @@
 """GPU parity: the CUDA library, called through the C ABI, against the CPU oracle on the
-same seeded inputs.  Bars (from the benchmark spec of this path):
+same seeded inputs.  Bars:
   k, status, steps: exact;  B and Q: relative max-norm 1e-10 (f64) / 1e-4 (f32);
   ||Q^T Q - I||_F <= 1e-12 (f64) / 1e-5 (f32).
 Q's late column blocks are ill-conditioned functions of the input (two correct float64
@@ -72,19 +72,32 @@ def check_run(h, w, g, o, A, Om, q_envelope=True):
     assert relmax(B, o.B) <= tol["rel"], ("B", relmax(B, o.B))
     u = 1.1e-16 if w.dtype == "f64" else 6e-8
     d = 2 * max(w.m, w.n) * u * np.sqrt(o.normA2)     # Frobenius size of the residual's rounding noise
-    # stopping quantities after every block.  The residual W[r0+b:, :] carries rounding noise
-    # of Frobenius size about d = 2 max(m, n) u ||A||_F (inner products of length m and n), so
-    # its squared norm E is only defined to 2 sqrt(E) d + d^2; above that floor the bar is 1e-9.
-    for a, c in zip(g.E_dir_trace, o.E_dir):
-        slack = 2 * np.sqrt(c) * d + d * d + 1e-9 * c
-        assert abs(a - c) <= slack, ("E_dir", a, c, slack)
+    A64 = A.astype(np.float64)
+    # The oracle's own envelope: the same problem with another summation order (float64: columns of A
+    # and rows of Omega permuted; float32: the same steps in plain float32 on the CPU).
+    op = None
+    if q_envelope and w.dtype == "f64":
+        op = orc.permuted_rerun(A64, Om.astype(np.float64), b, w.tol, w.max_rank, seed=1)
+        assert op.k == o.k
+    elif q_envelope:
+        op = orc.rrf(A, Om, b, w.tol, w.max_rank, dtype=np.float32)
+        if op.k != o.k:
+            op = None
+    # Stopping quantities after every block: 1e-9 relative, widened only by what the oracle's own trace
+    # moves under the reordering (x10; x3 against the float32 rerun).  Without an envelope the bound is
+    # the rounding noise of the residual itself, 2 sqrt(E) d + d^2.
+    for i, (a, c) in enumerate(zip(g.E_dir_trace, o.E_dir)):
+        if op is not None:
+            slack = 1e-9 * c + (10 if w.dtype == "f64" else 3) * abs(op.E_dir[i] - c) + 1e-300
+        else:
+            slack = 2 * np.sqrt(c) * d + d * d + 1e-9 * c
+        assert abs(a - c) <= slack, ("E_dir", i, a, c, slack)
     # Q explicitly, on the device
     Qg = rrf.rrf_form_q(h, g.V, g.T, b, k).cpu().numpy().astype(np.float64)
     Qo = orc.form_q(o.V, o.T, b)
     orth = np.linalg.norm(Qg.T @ Qg - np.eye(k))
     assert orth <= tol["orth"], ("orth", orth)
     # Q*B and the residual are well-posed: full bar
-    A64 = A.astype(np.float64)
     assert relmax(Qg @ B, Qo @ o.B) <= 10 * tol["rel"], ("QB", relmax(Qg @ B, Qo @ o.B))
     res = np.linalg.norm(A64 - Qg @ B)
     assert abs(res ** 2 - o.E_dir[-1]) <= 1e-6 * o.E_dir[-1] + 2 * np.sqrt(o.E_dir[-1]) * d + d * d
@@ -92,15 +105,8 @@ def check_run(h, w, g, o, A, Om, q_envelope=True):
         assert res <= w.tol * np.sqrt(o.normA2) * (1 + 1e-6)
     # Q element-wise, block by block, against the oracle's own envelope
     env = None
-    if q_envelope and w.dtype == "f64":
-        op = orc.permuted_rerun(A64, Om.astype(np.float64), b, w.tol, w.max_rank, seed=1)
-        assert op.k == o.k
-        env = orc.form_q(op.V, op.T, b)
-    elif q_envelope:
-        # single precision: the yardstick is the same algorithm in plain float32 on the CPU
-        op = orc.rrf(A, Om, b, w.tol, w.max_rank, dtype=np.float32)
-        if op.k == o.k:
-            env = orc.form_q(op.V.astype(np.float64), op.T.astype(np.float64), b)
+    if op is not None:
+        env = orc.form_q(op.V.astype(np.float64), op.T.astype(np.float64), b)
     worst = 0.0
     for i in range(k // b):
         blk = slice(i * b, (i + 1) * b)
@@ -131,6 +137,19 @@ def test_panel_qr_matches_oracle(h, rows, b, dtype):
     tol = 1e-12 if dtype == "f64" else 2e-6
     assert np.max(np.abs(V.cpu().numpy() - Vo)) <= tol
     assert np.max(np.abs(T.cpu().numpy() - To)) <= tol * 10
+
+
+@pytest.mark.parametrize("zero", [0.0, -0.0])
+def test_panel_qr_with_a_zero_first_pivot(h, zero):
+    # the reflector of a zero pivot takes the sign of the zero on both sides (LAPACK's SIGN)
+    rng = np.random.default_rng(17)
+    Y = rng.standard_normal((700, 16))
+    Y[0, 0] = zero
+    V, T = rrf.rrf_panel_qr(h, torch.from_numpy(Y).cuda())
+    Vo, tau, To, _ = orc.panel_qr(Y)
+    assert np.max(np.abs(V.cpu().numpy() - Vo)) <= 1e-12
+    assert np.max(np.abs(T.cpu().numpy() - To)) <= 1e-11
+    assert np.sign(Vo[1, 0]) == np.sign(Y[1, 0]) * (1.0 if np.copysign(1.0, zero) > 0 else -1.0)
 
 
 def test_panel_qr_zero_column_and_rank_deficient(h):
@@ -241,6 +260,44 @@ def test_panel_from_either_sampler(h, name, kw, sched, sampling):
     else:
         assert g.extra_samples == 0 and g.fused_samples >= g.steps - (2 if g.queues == 2 else 1)
     check_run(h, w, g, o, A, Om)
+
+
+@pytest.mark.parametrize("sched", SCHEDULES)
+@pytest.mark.parametrize("name,kw", [("cfg2", dict(m=1536, n=1280, max_rank=512)),
+                                     ("cfg3", dict(m=1024, n=1024, max_rank=384)),
+                                     ("cfg4", dict(m=1024, n=2752, max_rank=256, rank=64))])
+def test_each_block_factors_the_residual_it_was_given(h, name, kw, sched):
+    # Block by block, without the conditioning that compounds over a run: stop the GPU after i blocks
+    # (in place, so the residual W it leaves can be read back), sample Y_i = W[i b:, :] Omega_i from THAT
+    # residual on the CPU, factor it with the oracle, and compare with block i of the full GPU run at
+    # the plain bar (1e-10 / 1e-4, scaled by the panel's own condition number only; under the look-ahead
+    # schedule the panel was sampled one update earlier, from a residual that was larger by the factor
+    # `amp`, whose rounding noise it carries).
+    w = wl.CONFIGS[name].scaled(**kw)
+    A, _ = wl.make_matrix(w)
+    Om = wl.make_omega(w).astype(w.np_dtype)
+    dOmT = torch.from_numpy(np.ascontiguousarray(Om.T)).cuda()
+    full = rrf.rrf_run(h, torch.from_numpy(A).cuda(), w.b, w.tol, w.max_rank, omegaT=dOmT,
+                       flags=sched | rrf.RRF_FLAG_FIXED_RANK)
+    assert full.k == w.max_rank
+    Vf, Tf = full.V.cpu().numpy().astype(np.float64), full.T.cpu().numpy().astype(np.float64)
+    b = w.b
+    bar = TOL[w.dtype]["rel"]
+    E = [full.normA2] + list(full.E_dir_trace)      # E[j]: squared residual norm after j blocks
+    for i in (1, 2, 3):
+        dA = torch.from_numpy(A).cuda()
+        part = rrf.rrf_run(h, dA, b, w.tol, i * b, omegaT=dOmT[:i * b],
+                           flags=sched | rrf.RRF_FLAG_FIXED_RANK | rrf.RRF_FLAG_INPLACE, B=dA[:i * b])
+        assert part.k == i * b
+        Wres = dA[i * b:].cpu().numpy().astype(np.float64)
+        Y = Wres @ Om[:, i * b:(i + 1) * b].astype(np.float64)
+        Vo, _, To, R = orc.panel_qr(Y)
+        cond = np.linalg.cond(R)
+        amp = np.sqrt(E[i - 1] / E[i]) if full.queues == 2 else 1.0
+        tol = bar * max(1.0, cond / 100.0) * amp
+        dv = np.max(np.abs(Vf[i * b:, i * b:(i + 1) * b] - Vo))
+        dt = np.max(np.abs(Tf[:, i * b:(i + 1) * b] - To))
+        assert dv <= tol and dt <= 10 * tol, (i, dv, dt, cond)
 
 
 def test_schedules_agree_and_stop_mid_way(h):

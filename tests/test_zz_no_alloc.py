@@ -3,13 +3,14 @@
 Some embedders - a framework with a fixed memory plan, a plug-in or control loop that must
 never call cudaMalloc - can use neither a handle (creating one allocates) nor a workspace.
 rrf_panel_qr_static keeps its scratch in a fixed array inside the library instead.  This test
-calls it through the C ABI twice in a row, on different panels, and checks both results against
-the ordinary entry point: the second call must not be disturbed by what the first one left in
+calls it through the C ABI several times in a row, on different panels, and checks every result
+against the ordinary entry point and the CPU oracle: a later call must not be disturbed by what an earlier one left in
 the shared array.  It lives in its own file, collected last, and also passes on its own."""
 import numpy as np
 import pytest
 import torch
 
+from oracle import rrf_oracle as orc
 from paper_2608_28941_b200 import rrf
 
 pytestmark = pytest.mark.gpu
@@ -34,7 +35,11 @@ def test_static_scratch_panel_qr_matches_workspace_version_twice():
             tol = 1e-12 if dtype == torch.float64 else 2e-6
             assert torch.max(torch.abs(V - V_ref)).item() <= tol
             assert torch.max(torch.abs(T - T_ref)).item() <= 10 * tol
-            # and the factorisation itself is right: (I - V T V^T)^T Y is upper triangular
+            # ... against the CPU oracle's panel factorisation of the same panel ...
+            Vo, _, To, _ = orc.panel_qr(Y.cpu().numpy().astype("float64"))
+            assert abs(V.double().cpu().numpy() - Vo).max() <= tol
+            assert abs(T.double().cpu().numpy() - To).max() <= 10 * tol
+            # ... and the factorisation itself is right: (I - V T V^T)^T Y is upper triangular
             Vd, Td, Yd = V.double(), T.double(), Y.double()
             R = Yd - Vd @ (Td.T @ (Vd.T @ Yd))
             assert torch.max(torch.abs(torch.tril(R, -1))).item() <= (1e-11 if dtype == torch.float64 else 1e-4)
