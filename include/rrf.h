@@ -58,6 +58,10 @@ typedef enum {
                                       single precision and for b = 128, where the updates always sample */
 #define RRF_FLAG_NO_GRAPH 16u    /* always enqueue the kernels one by one (by default a call that repeats the
                                    previous call's arguments is captured into a CUDA graph and replayed) */
+#define RRF_FLAG_PANEL_TREE 128u /* b <= 64: factor the panels with the tree kernel (see rrf_panel_qr_tree) instead of
+                                    the kernel that pays one grid barrier per column.  Off by default: it is the
+                                    slower of the two on the sizes measured so far.  The look-ahead schedule is
+                                    then used only if RRF_FLAG_TWO_QUEUES asks for it */
 #define RRF_FLAG_TWO_QUEUES 8u  /* use the look-ahead schedule whenever the panel can be confined to a few SMs,
                                    also where the built-in rule would pick the sequential one */
 
@@ -171,6 +175,21 @@ rrf_status_t rrf_panel_qr(rrf_handle_t h, int32_t dtype, int64_t rows, int32_t b
                           const void* dY, int64_t ldy, void* dV, int64_t ldv,
                           void* dT, int64_t ldt,
                           void* d_workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
+ * rrf_panel_qr_tree - the same factorisation (Algorithm 2 line 7) by another route, for b <= 64: a tall-skinny QR
+ * over row slabs (every CTA factors its slab on its own, the b x b triangular factors are reduced up a tree
+ * of Householder QRs) followed by a reconstruction of the panel's Householder vectors and of T from the explicit
+ * orthonormal factor.  It needs 2 * levels - 1 grid barriers instead of b, is built from orthogonal
+ * transformations only, and returns the same V and T as rrf_panel_qr up to rounding, except where a column is
+ * exactly zero below its pivot (LAPACK then takes H = I; this route returns another valid reflector).
+ * Same arguments, workspace and error behaviour as rrf_panel_qr; RRF_ERR_WORKSPACE if the slabs and tree nodes
+ * need more CTAs than the device has SMs (about 40000 rows for b = 64).
+ */
+rrf_status_t rrf_panel_qr_tree(rrf_handle_t h, int32_t dtype, int64_t rows, int32_t b,
+                               const void* dY, int64_t ldy, void* dV, int64_t ldv,
+                               void* dT, int64_t ldt,
+                               void* d_workspace, size_t workspace_bytes, void* cuda_stream);
 
 /*
  * rrf_panel_qr_static - the same factorisation as rrf_panel_qr for callers that cannot allocate.

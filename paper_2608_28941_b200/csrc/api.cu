@@ -10,7 +10,7 @@
 #include <vector>
 
 #include "gemm_sk.cuh"
-#include "panel.cuh"
+#include "panel_tsqr.cuh"
 
 namespace rrf {
 
@@ -31,6 +31,7 @@ struct rrf_ctx {
   rrf::Ctrl* d_ctrl;     // status words for the calls that do not run Algorithm 2's loop
   int last_cuda;
   int panel_smem_max;    // dynamic shared memory the panel kernel may use (opt-in limit minus its static part)
+  int tsqr_smem_max;     // the same for the tree panel kernel
   int profiling;
   cudaStream_t aux;                      // side stream: the T factor is built while V^T W runs
   std::vector<cudaEvent_t> sync_events;  // fork/join events between the caller's stream and `aux`
@@ -150,6 +151,64 @@ static bool plan_panel(const rrf_ctx* h, long long rows, int b, PanelPlan* p, in
   }
   return false;
 }
+constexpr int kTsqrMaxB = 64;      // widest panel the tree kernel factors (wider ones take the per-column kernel)
+// Plan of the tree panel kernel: leaf slab height (one of the factorisation's tilings), fan-in, levels.
+struct TreePlan { TsqrPlan t; int ctas, Rp, nbar; size_t smem; double est_us; };
+static size_t tsqr_smem_bytes(int b, int slab_rows) {
+  return ((size_t)b * (slab_rows + 1) + panel_fix_doubles(b) + tsqr_small_doubles(b)) * sizeof(double);
+}
+// rough time of one CTA-local factorisation of `rows` x b (microseconds): b dependent columns
+static double tsqr_level_us(int rows, int b) { return b * (1100.0 + 0.09 * rows * b) / 1965.0 + 6.0; }
+// max_ctas == 0: any number up to the SM count.  Returns false if no tiling fits.
+static bool plan_tree(const rrf_ctx* h, long long rows, int b, int max_ctas, bool fix, TreePlan* out) {
+  if (b > kTsqrMaxB) return false;
+  const long long ext = rows + (fix ? b : 0);
+  const int limit = max_ctas > 0 ? std::min(max_ctas, h->sms) : h->sms;
+  int vmax = -1;                                     // tallest tiling that fits in shared memory
+  for (int v = 0; v < 5; ++v)
+    if (tsqr_smem_bytes(b, tsqr_variant_rows(v)) <= (size_t)h->tsqr_smem_max) vmax = v;
+  if (vmax < 0) return false;
+  const int f = tsqr_variant_rows(vmax) / b;
+  bool found = false;
+  for (int v = 0; v <= vmax; ++v) {
+    const int R = tsqr_variant_rows(v);
+    if (R < (fix ? 2 * b : b)) continue;
+    TreePlan p{};
+    p.t.R = R;
+    p.t.f = f;
+    p.t.cnt[0] = ceil_div(ext, R);
+    p.t.var[0] = v;
+    p.t.off[0] = 0;
+    int l = 0, top = v;
+    double est = tsqr_level_us(R, b);
+    bool ok = true;
+    while (p.t.cnt[l] > 1) {
+      if (f < 2 || l + 1 >= 6) { ok = false; break; }
+      p.t.cnt[l + 1] = ceil_div(p.t.cnt[l], f);
+      p.t.off[l + 1] = p.t.off[l] + p.t.cnt[l];
+      const int need = std::min(f, p.t.cnt[l]) * b;
+      int nv = 0;
+      while (tsqr_variant_rows(nv) < need) ++nv;
+      p.t.var[l + 1] = nv;
+      top = std::max(top, nv);
+      est += tsqr_level_us(tsqr_variant_rows(nv), b) + 8.0;   // + the way down and two barriers
+      ++l;
+    }
+    if (!ok) continue;
+    p.t.nlev = l + 1;
+    p.ctas = p.t.off[l] + p.t.cnt[l];
+    if (p.ctas > limit) continue;
+    p.Rp = tsqr_variant_rows(top) + 1;
+    p.smem = tsqr_smem_bytes(b, tsqr_variant_rows(top));
+    p.nbar = 2 * p.t.nlev - 1 + (fix ? 2 : 0);
+    p.est_us = est + 0.25 * b + 10.0 + (fix ? 25.0 : 0.0);     // + elimination, final product, fix-up
+    if (!found || p.est_us < out->est_us) {
+      *out = p;
+      found = true;
+    }
+  }
+  return found;
+}
 // Fewest CTAs whose shared memory holds a rows x b panel with the fix-up staging; 0 if none.
 static int panel_min_ctas(const rrf_ctx* h, long long rows, int b) {
   if (b > 64) return 0;
@@ -160,11 +219,16 @@ static int panel_min_ctas(const rrf_ctx* h, long long rows, int b) {
       best = std::max(best, kVariantRows[q]);
   return best > 0 ? ceil_div(rows + b, best) : 0;
 }
-static size_t panel_scratch_bytes(int sms, int b) {
+static size_t direct_scratch_bytes(int sms, int b) {
   // P[2][b][Gp] + piv[2][b] + gram[b][b] + tau[b] (+ barrier word, padded)
   const int gp = (sms + 31) / 32 * 32;
   return align_up(((size_t)2 * gp * b + 2 * (size_t)b + (size_t)b * b + b) * sizeof(double) + 256, 256);
 }
+static size_t tsqr_scratch_bytes(int sms, int b) {
+  // Rbuf, Xbuf, Kbuf [CTA][b*b] + Ubuf [2][b*b]
+  return b <= kTsqrMaxB ? align_up(((size_t)3 * sms + 2) * b * b * sizeof(double), 256) : 0;
+}
+static size_t panel_scratch_bytes(int sms, int b) { return direct_scratch_bytes(sms, b) + tsqr_scratch_bytes(sms, b); }
 constexpr int kLookMaxCtas = 48;   // most CTAs a confined panel may take
 // Rough cost model of one pass, in microseconds, used only to choose the schedule (fitted to event
 // timings on a B200; the look-ahead is right or wrong by its measured time, not by this model).
@@ -191,14 +255,21 @@ struct PassModel {
 static size_t look_scratch_bytes(int b) {   // Gpart[kLookMaxCtas][b*b] + M[b*b]
   return align_up((size_t)(kLookMaxCtas + 1) * b * b * sizeof(double), 256);
 }
-struct PanelScratch { double *P, *piv, *gram, *tau; unsigned* bar; };
-static PanelScratch carve_panel(unsigned char* base, int sms, int b) {
+struct PanelScratch { double *P, *piv, *gram, *tau; unsigned* bar; TsqrScratch ts; };
+// `sms`: the SM count the buffers were sized for (the handle's bound kMaxSms for caller workspaces)
+static PanelScratch carve_panel(unsigned char* base, int sms, int b, bool with_tree = true) {
   PanelScratch s;
   s.P = reinterpret_cast<double*>(base);
   s.piv = s.P + (size_t)2 * ((sms + 31) / 32 * 32) * b;
   s.gram = s.piv + 2 * (size_t)b;
   s.tau = s.gram + (size_t)b * b;
   s.bar = reinterpret_cast<unsigned*>(s.tau + b);
+  s.ts = TsqrScratch{nullptr, nullptr, nullptr, nullptr};
+  if (with_tree && b <= kTsqrMaxB) {
+    double* t = reinterpret_cast<double*>(base + direct_scratch_bytes(sms, b));
+    const size_t blk = (size_t)sms * b * b;
+    s.ts = TsqrScratch{t, t + blk, t + 2 * blk, t + 3 * blk};
+  }
   return s;
 }
 
@@ -346,12 +417,38 @@ struct PanelOpts {
   unsigned* bar_used = nullptr;    // out: what this launch adds to the counter
   cudaStream_t st_t = nullptr;     // side stream for the T factor, with its fork / join events
   cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
+  bool tree = false;               // b <= 64: use the tree kernel (no grid barrier per column)
 };
 template <typename Mark = NoMark>
 static rrf_status_t launch_panel(rrf_ctx* h, int dtype, const void* Y, PanelSource src,
                                  long long rows, int b, void* V, long long ldv, void* Tout, long long ldt,
                                  const PanelScratch& ps, Ctrl* ctrl, const int* done_flag, cudaStream_t st,
                                  Mark mark = Mark(), int step = 0, const PanelOpts& o = PanelOpts()) {
+  if (b <= kTsqrMaxB && o.tree && ps.ts.Rbuf != nullptr) {
+    // tree kernel: factorisation, T factor and all, in one cooperative launch
+    TreePlan tp;
+    if (!plan_tree(h, rows, b, o.ctas, o.fix.enabled != 0, &tp)) return RRF_ERR_WORKSPACE;
+    int rows_i = (int)rows, Rp = tp.Rp;
+    PanelFix fix = o.fix;
+    PanelSource alt = o.alt;
+    const int* fused_flag = o.fused_flag;
+    unsigned bar_base = o.bar_base;
+    unsigned* bar = ps.bar;
+    TsqrPlan plan = tp.t;
+    TsqrScratch tsc = ps.ts;
+    void* args[] = {&Y, &src, &alt, &fused_flag, &rows_i, &b, &Rp, &V, &ldv, &plan, &tsc,
+                    &bar, &ctrl, &done_flag, &fix, &bar_base, &Tout, &ldt};
+    if (o.bar_used != nullptr) *o.bar_used = (unsigned)tp.nbar * (unsigned)tp.ctas;
+    mark(RRF_PHASE_PANEL, step);
+    const void* fn = dtype == RRF_F64 ? (const void*)panel_tsqr_kernel<double> : (const void*)panel_tsqr_kernel<float>;
+    const cudaError_t e = cudaLaunchCooperativeKernel(fn, dim3(tp.ctas), dim3(kPanelThreads), args, tp.smem, st);
+    if (e != cudaSuccess) {
+      h->last_cuda = (int)e;
+      return RRF_ERR_CUDA;
+    }
+    if (o.ev_join != nullptr) cudaEventRecord(o.ev_join, st);   // T is ready when the panel kernel is
+    return RRF_OK;
+  }
   PanelPlan pp;
   if (!plan_panel(h, rows, b, &pp, o.ctas, o.fix.enabled != 0)) return RRF_ERR_WORKSPACE;
   int rows_i = (int)rows, R = pp.R, Rp = pp.Rp;
@@ -417,6 +514,23 @@ static cudaError_t setup_panel_kernels(int smem_optin, int* panel_smem_max) {
   e = cudaFuncSetAttribute(tfactor_kernel<double>, cudaFuncAttributeMaxDynamicSharedMemorySize, tmax);
   if (e != cudaSuccess) return e;
   return cudaFuncSetAttribute(tfactor_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, tmax);
+}
+
+static cudaError_t setup_tree_kernels(int smem_optin, int* tsqr_smem_max) {
+  const void* fk[2] = {(const void*)panel_tsqr_kernel<double>, (const void*)panel_tsqr_kernel<float>};
+  size_t stat = 0;
+  for (const void* f : fk) {
+    cudaFuncAttributes fa;
+    const cudaError_t e = cudaFuncGetAttributes(&fa, f);
+    if (e != cudaSuccess) return e;
+    stat = std::max(stat, fa.sharedSizeBytes);
+  }
+  *tsqr_smem_max = std::min(smem_optin, kMaxSmem) - (int)stat;
+  for (const void* f : fk) {
+    const cudaError_t e = cudaFuncSetAttribute(f, cudaFuncAttributeMaxDynamicSharedMemorySize, *tsqr_smem_max);
+    if (e != cudaSuccess) return e;
+  }
+  return cudaSuccess;
 }
 
 static cudaError_t setup_all(int smem_optin, int* panel_smem_max) {
@@ -535,6 +649,7 @@ rrf_status_t rrf_create(rrf_handle_t* out, int device) {
   if (e == cudaSuccess && h->sms > kMaxSms) e = cudaErrorInvalidConfiguration;
   h->encode = reinterpret_cast<EncodeTiledFn>(fn);
   if (e == cudaSuccess) e = setup_all(h->smem_optin, &h->panel_smem_max);
+  if (e == cudaSuccess) e = setup_tree_kernels(h->smem_optin, &h->tsqr_smem_max);
   if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&h->aux, cudaStreamNonBlocking);
   if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&h->cap, cudaStreamNonBlocking);
   if (e == cudaSuccess) e = cudaMalloc(&h->d_ctrl, sizeof(Ctrl));
@@ -658,13 +773,14 @@ rrf_status_t rrf_panel_workspace_bytes(int32_t dtype, int64_t rows, int32_t b, s
   return RRF_OK;
 }
 
-rrf_status_t rrf_panel_qr(rrf_handle_t h, int32_t dtype, int64_t rows, int32_t b, const void* dY, int64_t ldy,
-                          void* dV, int64_t ldv, void* dT, int64_t ldt, void* d_workspace, size_t workspace_bytes,
-                          void* cuda_stream) {
+static rrf_status_t panel_qr_entry(rrf_handle_t h, int32_t dtype, int64_t rows, int32_t b, const void* dY, int64_t ldy,
+                                   void* dV, int64_t ldv, void* dT, int64_t ldt, void* d_workspace,
+                                   size_t workspace_bytes, void* cuda_stream, bool tree) {
   if (h == nullptr || dY == nullptr || dV == nullptr || dT == nullptr || d_workspace == nullptr)
     return RRF_ERR_INVALID_ARG;
   if (!b_ok(dtype, b) || rows < b || rows > 0x7fffffffLL || ldy < b || ldv < b || ldt < b || ldy > 0x7fffffffLL)
     return RRF_ERR_INVALID_ARG;
+  if (tree && b > kTsqrMaxB) return RRF_ERR_INVALID_ARG;
   if (workspace_bytes < panel_scratch_bytes(kMaxSms, b) ) return RRF_ERR_WORKSPACE;
   cudaStream_t st = (cudaStream_t)cuda_stream;
   PanelScratch ps = carve_panel((unsigned char*)d_workspace, h->sms, b);
@@ -674,7 +790,21 @@ rrf_status_t rrf_panel_qr(rrf_handle_t h, int32_t dtype, int64_t rows, int32_t b
   src.nseg = 1;
   src.seg_stride = 0;
   src.ldy = (int)ldy;
-  return launch_panel(h, dtype, dY, src, rows, b, dV, ldv, dT, ldt, ps, h->d_ctrl, &h->d_ctrl->done, st);
+  PanelOpts po;
+  po.tree = tree;
+  return launch_panel(h, dtype, dY, src, rows, b, dV, ldv, dT, ldt, ps, h->d_ctrl, &h->d_ctrl->done, st, NoMark(), 0, po);
+}
+
+rrf_status_t rrf_panel_qr(rrf_handle_t h, int32_t dtype, int64_t rows, int32_t b, const void* dY, int64_t ldy,
+                          void* dV, int64_t ldv, void* dT, int64_t ldt, void* d_workspace, size_t workspace_bytes,
+                          void* cuda_stream) {
+  return panel_qr_entry(h, dtype, rows, b, dY, ldy, dV, ldv, dT, ldt, d_workspace, workspace_bytes, cuda_stream, false);
+}
+
+rrf_status_t rrf_panel_qr_tree(rrf_handle_t h, int32_t dtype, int64_t rows, int32_t b, const void* dY, int64_t ldy,
+                               void* dV, int64_t ldv, void* dT, int64_t ldt, void* d_workspace,
+                               size_t workspace_bytes, void* cuda_stream) {
+  return panel_qr_entry(h, dtype, rows, b, dY, ldy, dV, ldv, dT, ldt, d_workspace, workspace_bytes, cuda_stream, true);
 }
 
 rrf_status_t rrf_apply_workspace_bytes(int32_t dtype, int64_t m, int64_t ncols, int32_t b, size_t* bytes) {
@@ -844,8 +974,16 @@ rrf_status_t rrf_run(rrf_handle_t h, const rrf_params_t* p, void* dA, int64_t ld
   // Schedule.  Two queues (look-ahead) when the tallest panel fits in the shared memory of a small
   // share of the SMs, so that confining the panel there costs the GEMM kernels little; else one queue.
   const int steps_total = p->max_rank / b;
+  // the tree panel kernel is opt-in: it is the slower of the two on every size measured so far
+  const bool tree = (p->flags & RRF_FLAG_PANEL_TREE) != 0 && b <= kTsqrMaxB;
   int look_ctas = 0;
-  if (!(p->flags & RRF_FLAG_ONE_QUEUE) && steps_total >= 2) {
+  if (tree) {
+    TreePlan tl;
+    const int cap = std::min(kLookMaxCtas, h->sms / 3);
+    const int lim = p->tune_panel_ctas > 0 ? std::min(cap, (int)p->tune_panel_ctas) : cap;
+    if ((p->flags & RRF_FLAG_TWO_QUEUES) && steps_total >= 2 && plan_tree(h, m, b, lim, true, &tl)) look_ctas = tl.ctas;
+    if (look_ctas == 0 && !plan_tree(h, m, b, 0, false, &tl)) return fail(RRF_ERR_WORKSPACE);
+  } else if (!(p->flags & RRF_FLAG_ONE_QUEUE) && steps_total >= 2) {
     const int fewest = panel_min_ctas(h, m, b);
     const int cap = std::min(kLookMaxCtas, h->sms / 3);
     if (fewest > 0 && fewest <= cap) {
@@ -866,7 +1004,7 @@ rrf_status_t rrf_run(rrf_handle_t h, const rrf_params_t* p, void* dA, int64_t ld
     }
   }
   PanelPlan pp0;
-  if (look_ctas == 0 && !plan_panel(h, m, b, &pp0)) return fail(RRF_ERR_WORKSPACE);   // tallest panel must fit on chip
+  if (!tree && look_ctas == 0 && !plan_panel(h, m, b, &pp0)) return fail(RRF_ERR_WORKSPACE);   // tallest panel must fit on chip
 
   cudaStream_t const user_st = (cudaStream_t)cuda_stream;
   cudaStream_t st = user_st;
@@ -998,6 +1136,7 @@ rrf_status_t rrf_run(rrf_handle_t h, const rrf_params_t* p, void* dA, int64_t ld
       po.ev_join = h->sync_events[2 * i + 1];
       po.alt = alt;
       po.fused_flag = fused_flag;
+      po.tree = tree;
       s = launch_panel(h, p->dtype, Ypart, src, rows, b, Vblk(r0), ldv, Tblk(r0), p->max_rank, ps, ctrl, &ctrl->done,
                        st, mark, i, po);
       if (s != RRF_OK) return panel_failed(s);
@@ -1064,6 +1203,7 @@ rrf_status_t rrf_run(rrf_handle_t h, const rrf_params_t* p, void* dA, int64_t ld
     unsigned bar_next = 0, bar_used = 0;
     PanelOpts po;
     po.ctas = look_ctas;
+    po.tree = tree;
     po.merge_t = true;
     po.bar_used = &bar_used;
     s = launch_panel(h, p->dtype, Ybuf[0], src, m, b, Vblk(0), ldv, Tblk(0), p->max_rank, ps, ctrl, done_after, h->aux,
@@ -1262,7 +1402,7 @@ rrf_status_t rrf_run(rrf_handle_t h, const rrf_params_t* p, void* dA, int64_t ld
     // without the predictor every executed pass that has a later panel to sample samples it
     out->fused_samples = predicting ? hc.fused_samples : std::min(hc.steps, std::max(0, steps - lag));
     out->kernel_launches = 1 + (dOmegaT == nullptr ? 1 : 0) + 1 + ((look_ctas > 0 && steps > 1) ? 1 : 0) +
-                           (look_ctas > 0 ? 5 : 6) * steps +   // look-ahead: the panel kernel builds T itself
+                           ((look_ctas > 0 || tree) ? 5 : 6) * steps +   // look-ahead, tree kernel: the panel kernel builds T itself
                            (predicting ? std::max(0, steps - lag) : 0);
   }
   out->extra_samples = hc.extra_samples;
@@ -1327,7 +1467,7 @@ extern "C" rrf_status_t rrf_panel_qr_static(int32_t dtype, int64_t rows, int32_t
   StaticDevice* sd = &g_static_dev[dev];
   std::call_once(sd->once, [&] { sd->err = static_setup(dev, sd); });
   if (sd->err != cudaSuccess || sd->ptr == nullptr) return RRF_ERR_CUDA;
-  if (sd->sms > kMaxSms || kStaticCtrlBytes + panel_scratch_bytes(sd->sms, b) > kStaticScratchBytes)
+  if (sd->sms > kMaxSms || kStaticCtrlBytes + direct_scratch_bytes(sd->sms, b) > kStaticScratchBytes)
     return RRF_ERR_WORKSPACE;
   rrf_ctx tmp{};                                            // host-side plan parameters only
   tmp.device = dev;
@@ -1337,7 +1477,7 @@ extern "C" rrf_status_t rrf_panel_qr_static(int32_t dtype, int64_t rows, int32_t
   if (!plan_panel(&tmp, rows, b, &pp)) return RRF_ERR_WORKSPACE;   // panel too tall for on-chip storage
   cudaStream_t st = (cudaStream_t)cuda_stream;
   Ctrl* ctrl = reinterpret_cast<Ctrl*>(sd->ptr);
-  PanelScratch ps = carve_panel(sd->ptr + kStaticCtrlBytes, sd->sms, b);
+  PanelScratch ps = carve_panel(sd->ptr + kStaticCtrlBytes, sd->sms, b, false);
   ps.bar = &ctrl->bar;
   // the array keeps the last call's contents: the stop flag, the status and the barrier counter
   // must start at zero; everything else is written by the kernels before it is read
@@ -1355,3 +1495,9 @@ extern "C" rrf_status_t rrf_panel_qr_static(int32_t dtype, int64_t rows, int32_t
   if (cudaStreamSynchronize(st) != cudaSuccess) return RRF_ERR_CUDA;
   return (rrf_status_t)status;
 }
+
+#ifdef RRF_TSQR_TRACE
+extern "C" int rrf_debug_trace(unsigned long long* out) {
+  return (int)cudaMemcpyFromSymbol(out, rrf::g_tsqr_trace, sizeof(unsigned long long) * 64);
+}
+#endif

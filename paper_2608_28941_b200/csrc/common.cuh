@@ -66,6 +66,7 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, Ctrl* 
   while (!mbar_try_wait(bar, parity)) {
     if (clock64() - t0 > kWaitLimitClocks) {
       atomicExch(&ctrl->status, (int)RRF_ERR_TIMEOUT);
+      atomicExch(&ctrl->done, 1);          // kernels already enqueued behind this one return at once
       return false;
     }
   }
@@ -126,6 +127,44 @@ __device__ __forceinline__ void mma16x8x8(float (&c)[4], const float (&a)[4], co
     bh[i] = to_tf32(b[i]);
     bl[i] = to_tf32(b[i] - __uint_as_float(bh[i]));
   }
+  float d[4] = {0.f, 0.f, 0.f, 0.f};
+  mma_tf32(d, al, bh);
+  mma_tf32(d, ah, bl);
+  mma_tf32(d, ah, bh);
+#pragma unroll
+  for (int i = 0; i < 4; ++i) c[i] += d[i];
+}
+
+// Operands prepared once and used by several products.  In double precision an operand is the value; in single
+// precision it is the value split into two TF32 numbers, so that a fragment that feeds several m16n8k8 products
+// is split once and not once per product.
+template <typename T>
+struct Op;
+template <>
+struct Op<double> {
+  double v;
+};
+template <>
+struct Op<float> {
+  uint32_t hi, lo;
+};
+__device__ __forceinline__ Op<double> prep(double x) { return Op<double>{x}; }
+__device__ __forceinline__ Op<float> prep(float x) {
+  Op<float> o;
+  o.hi = to_tf32(x);
+  o.lo = to_tf32(x - __uint_as_float(o.hi));
+  return o;
+}
+__device__ __forceinline__ void mma_op(double (&c)[4], const Op<double>& a0, const Op<double>& a1, const Op<double>& a2,
+                                       const Op<double>& a3, const Op<double>& b0, const Op<double>& b1) {
+  const double a[4] = {a0.v, a1.v, a2.v, a3.v}, b[2] = {b0.v, b1.v};
+  mma16x8x8(c, a, b);
+}
+// D = A_lo*B_hi + A_hi*B_lo + A_hi*B_hi inside the tensor core, then C += D rounded to nearest (see above)
+__device__ __forceinline__ void mma_op(float (&c)[4], const Op<float>& a0, const Op<float>& a1, const Op<float>& a2,
+                                       const Op<float>& a3, const Op<float>& b0, const Op<float>& b1) {
+  const uint32_t ah[4] = {a0.hi, a1.hi, a2.hi, a3.hi}, al[4] = {a0.lo, a1.lo, a2.lo, a3.lo};
+  const uint32_t bh[2] = {b0.hi, b1.hi}, bl[2] = {b0.lo, b1.lo};
   float d[4] = {0.f, 0.f, 0.f, 0.f};
   mma_tf32(d, al, bh);
   mma_tf32(d, ah, bl);

@@ -145,17 +145,26 @@ __global__ void __launch_bounds__(WM* WN * 32)
             const int rn = wn * TN + c * 8 + g;
             VecLoad16<T>::ld(sB + rn * 128 + chunk, rb[c]);
           }
+          Op<T> oa[MT][2][NV], ob[NT][NV];     // split once, used by NT (resp. MT) products each
+#pragma unroll
+          for (int a = 0; a < MT; ++a)
+#pragma unroll
+            for (int e = 0; e < NV; ++e) {
+              oa[a][0][e] = prep(ra[a][0][e]);
+              oa[a][1][e] = prep(ra[a][1][e]);
+            }
+#pragma unroll
+          for (int c = 0; c < NT; ++c)
+#pragma unroll
+            for (int e = 0; e < NV; ++e) ob[c][e] = prep(rb[c][e]);
 #pragma unroll
           for (int ks = 0; ks < KS; ++ks)
 #pragma unroll
-            for (int a = 0; a < MT; ++a) {
-              const T af[4] = {ra[a][0][2 * ks], ra[a][1][2 * ks], ra[a][0][2 * ks + 1], ra[a][1][2 * ks + 1]};
+            for (int a = 0; a < MT; ++a)
 #pragma unroll
-              for (int c = 0; c < NT; ++c) {
-                const T bf[2] = {rb[c][2 * ks], rb[c][2 * ks + 1]};
-                mma16x8x8(acc[a][c], af, bf);
-              }
-            }
+              for (int c = 0; c < NT; ++c)
+                mma_op(acc[a][c], oa[a][0][2 * ks], oa[a][1][2 * ks], oa[a][0][2 * ks + 1], oa[a][1][2 * ks + 1],
+                       ob[c][2 * ks], ob[c][2 * ks + 1]);
         }
       }
       __syncthreads();  // everyone is done with stage st before it is refilled

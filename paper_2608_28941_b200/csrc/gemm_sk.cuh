@@ -147,23 +147,24 @@ __global__ void __launch_bounds__((WM * WN + 1) * 32)
     // plus ks * 1024 bytes.
 #pragma unroll
     for (int ks = 0; ks < BK / 8; ++ks) {
-      T af[MT][4], bf[NT][2];
+      Op<T> af[MT][4], bf[NT][2];
 #pragma unroll
       for (int a = 0; a < MT; ++a) {
-        af[a][0] = *reinterpret_cast<const T*>(sV + offA[a][0] + ks * 1024);
-        af[a][1] = *reinterpret_cast<const T*>(sV + offA[a][1] + ks * 1024);
-        af[a][2] = *reinterpret_cast<const T*>(sV + offA[a][2] + ks * 1024);
-        af[a][3] = *reinterpret_cast<const T*>(sV + offA[a][3] + ks * 1024);
+        af[a][0] = prep(*reinterpret_cast<const T*>(sV + offA[a][0] + ks * 1024));
+        af[a][1] = prep(*reinterpret_cast<const T*>(sV + offA[a][1] + ks * 1024));
+        af[a][2] = prep(*reinterpret_cast<const T*>(sV + offA[a][2] + ks * 1024));
+        af[a][3] = prep(*reinterpret_cast<const T*>(sV + offA[a][3] + ks * 1024));
       }
 #pragma unroll
       for (int cc = 0; cc < NT; ++cc) {
-        bf[cc][0] = *reinterpret_cast<const T*>(sC + offB[cc][0] + ks * 1024);
-        bf[cc][1] = *reinterpret_cast<const T*>(sC + offB[cc][1] + ks * 1024);
+        bf[cc][0] = prep(*reinterpret_cast<const T*>(sC + offB[cc][0] + ks * 1024));
+        bf[cc][1] = prep(*reinterpret_cast<const T*>(sC + offB[cc][1] + ks * 1024));
       }
 #pragma unroll
       for (int a = 0; a < MT; ++a)
 #pragma unroll
-        for (int cc = 0; cc < NT; ++cc) mma16x8x8(acc[a][cc], af[a], bf[cc]);
+        for (int cc = 0; cc < NT; ++cc)
+          mma_op(acc[a][cc], af[a][0], af[a][1], af[a][2], af[a][3], bf[cc][0], bf[cc][1]);
     }
     __syncwarp();
     if (lane == 0) mbar_arrive(&empty[st]);
@@ -480,12 +481,17 @@ __global__ void __launch_bounds__((WM * WN + (PW ? 1 : 0)) * 32, 1)
 #define RRF_VZ_ITER(qa_, qb_, it_)                                                                                   \
         {                                                                                                         \
           const int kb_ = (it_) >> 1, s2_ = (it_) & 1;                                                            \
-          T ra_[MT][2][NV];                                                                                       \
+          Op<T> oa_[MT][2][NV];                                                                                   \
           _Pragma("unroll") for (int a = 0; a < MT; ++a) {                                                        \
             const int rlo = wm * TM + a * 16 + g;                                                                 \
             const uint32_t chunk = ((uint32_t)(2 * t + s2_) ^ (uint32_t)g) << 4;                                  \
-            VecLoad16<T>::ld(sVs + kb_ * V_BOX + rlo * 128 + chunk, ra_[a][0]);                                   \
-            VecLoad16<T>::ld(sVs + kb_ * V_BOX + (rlo + 8) * 128 + chunk, ra_[a][1]);                             \
+            T ra0_[NV], ra1_[NV];                                                                                 \
+            VecLoad16<T>::ld(sVs + kb_ * V_BOX + rlo * 128 + chunk, ra0_);                                        \
+            VecLoad16<T>::ld(sVs + kb_ * V_BOX + (rlo + 8) * 128 + chunk, ra1_);                                  \
+            _Pragma("unroll") for (int e = 0; e < NV; ++e) {                                                      \
+              oa_[a][0][e] = prep(ra0_[e]);                                                                       \
+              oa_[a][1][e] = prep(ra1_[e]);                                                                       \
+            }                                                                                                     \
           }                                                                                                       \
           _Pragma("unroll") for (int q_ = (qa_); q_ < (qb_); ++q_)                                                \
           _Pragma("unroll") for (int u = 0; u < U; ++u) {                                                         \
@@ -494,11 +500,10 @@ __global__ void __launch_bounds__((WM * WN + (PW ? 1 : 0)) * 32, 1)
             T rb_[NV];                                                                                            \
             VecLoad16<T>::ld(sZ + kb_ * Z_BOX + zr * 128 + (((uint32_t)(2 * t + s2_) ^ (uint32_t)(zr & 7)) << 4), rb_); \
             _Pragma("unroll") for (int ks = 0; ks < KS; ++ks) {                                                   \
-              const T bf[2] = {rb_[2 * ks], rb_[2 * ks + 1]};                                                     \
-              _Pragma("unroll") for (int a = 0; a < MT; ++a) {                                                    \
-                const T af[4] = {ra_[a][0][2 * ks], ra_[a][1][2 * ks], ra_[a][0][2 * ks + 1], ra_[a][1][2 * ks + 1]}; \
-                mma16x8x8(acc[a][q_][u], af, bf);                                                                 \
-              }                                                                                                   \
+              const Op<T> b0_ = prep(rb_[2 * ks]), b1_ = prep(rb_[2 * ks + 1]);                                   \
+              _Pragma("unroll") for (int a = 0; a < MT; ++a)                                                      \
+                mma_op(acc[a][q_][u], oa_[a][0][2 * ks], oa_[a][1][2 * ks], oa_[a][0][2 * ks + 1],                \
+                       oa_[a][1][2 * ks + 1], b0_, b1_);                                                          \
             }                                                                                                     \
           }                                                                                                       \
         }
@@ -545,13 +550,17 @@ __global__ void __launch_bounds__((WM * WN + (PW ? 1 : 0)) * 32, 1)
           VecLoad16<T>::ld(sO + grp * O_BOX + jr * 128 + (((uint32_t)(2 * t + s2_) ^ (uint32_t)g) << 4), rb_);    \
           _Pragma("unroll") for (int ks = 0; ks < KS; ++ks) {                                                     \
             const int u = s2_ * KS + ks;                                                                          \
-            const T bf[2] = {rb_[2 * ks], rb_[2 * ks + 1]};                                                       \
-            _Pragma("unroll") for (int a = 0; a < MT; ++a) {                                                      \
-              const T af[4] = {acc[a][q_][u][0], acc[a][q_][u][2], acc[a][q_][u][1], acc[a][q_][u][3]};           \
-              mma16x8x8(accY[a][nb_], af, bf);                                                                    \
-            }                                                                                                     \
+            const Op<T> b0_ = prep(rb_[2 * ks]), b1_ = prep(rb_[2 * ks + 1]);                                     \
+            _Pragma("unroll") for (int a = 0; a < MT; ++a)                                                        \
+              mma_op(accY[a][nb_], oW[a][u][0], oW[a][u][2], oW[a][u][1], oW[a][u][3], b0_, b1_);                 \
           }                                                                                                       \
         }
+        /* the updated tile of group q_ as the A operand of the sample product, split once for all its n-tiles */ \
+#define RRF_SPLIT_W(q_)                                                                                           \
+        _Pragma("unroll") for (int a = 0; a < MT; ++a)                                                            \
+          _Pragma("unroll") for (int u = 0; u < U; ++u)                                                           \
+            _Pragma("unroll") for (int e = 0; e < 4; ++e) oW[a][u][e] = prep(acc[a][q_][u][e]);
+        Op<T> oW[MT][U][4];
 #pragma unroll
         for (int a = 0; a < MT; ++a)
 #pragma unroll
@@ -584,6 +593,7 @@ __global__ void __launch_bounds__((WM * WN + (PW ? 1 : 0)) * 32, 1)
           for (int e = 0; e < NP; ++e) RRF_EPI_PIECE(QW - 1, e)
         }
         if (do_sample) {
+          RRF_SPLIT_W(0)
 #pragma unroll
           for (int it = 0; it < NSI; ++it) {
             RRF_S_ITER(0, it)
@@ -594,10 +604,12 @@ __global__ void __launch_bounds__((WM * WN + (PW ? 1 : 0)) * 32, 1)
             }
           }
           if (QW == 2) {
+            RRF_SPLIT_W(QW - 1)
 #pragma unroll
             for (int it = 0; it < NSI; ++it) RRF_S_ITER(QW - 1, it)
           }
         }
+#undef RRF_SPLIT_W
 #undef RRF_VZ_ITER
 #undef RRF_EPI_PIECE
 #undef RRF_S_ITER

@@ -28,6 +28,7 @@ __device__ __forceinline__ bool grid_barrier(unsigned* ctr, unsigned target, Ctr
       if (v >= target) break;
       if (clock64() - t0 > limit) {
         atomicExch(&ctrl->status, (int)RRF_ERR_TIMEOUT);
+        atomicExch(&ctrl->done, 1);        // kernels already enqueued behind this one return at once
         ok = 0;
         break;
       }
@@ -108,7 +109,8 @@ __device__ __forceinline__ double panel_entry(const T* __restrict__ Y, const Pan
   double s = 0.0;
   if (!src.slots) {
     const T* p = Y + (size_t)(r + src.row_off) * src.ldy + c;
-    for (int sg = 0; sg < src.nseg; ++sg) s += (double)p[(size_t)sg * src.seg_stride];
+    s = (double)p[0];                     // not 0.0 + p[0]: a lone -0.0 keeps its sign (it decides a reflector's)
+    for (int sg = 1; sg < src.nseg; ++sg) s += (double)p[(size_t)sg * src.seg_stride];
   } else {
     const int lr = r + src.row_off;
     const int sl = lr / src.bm, rl = lr - sl * src.bm;
@@ -209,7 +211,7 @@ __global__ void __launch_bounds__(kPanelThreads)
                  unsigned* bar, Ctrl* ctrl, const int* done_flag, PanelFix fix,
                  unsigned bar_base,                 // value of the barrier counter when this launch starts
                  T* __restrict__ Tout, long long ldt) {   // non-NULL: CTA 0 also builds the T factor at the end
-  if (*reinterpret_cast<const volatile int*>(done_flag)) return;
+  if (*reinterpret_cast<const volatile int*>(done_flag) || *reinterpret_cast<const volatile int*>(&ctrl->status) < 0) return;
   // the panel's entries were sampled by the fused update, or - where the predictor had skipped that - by
   // the separate sample kernel, in its layout
   const bool use_alt = fused_flag != nullptr && *fused_flag == 0;
