@@ -163,7 +163,7 @@ def run_reference(args, w, rank, world):
         blocks = max(1, int(budget / (t_full / 2)))
     for _ in range(args.warmup):
         oracle_run(A, Om, w, blocks)
-    times, steps_done = [], 0
+    times, steps_done, r = [], 0, None
     for _ in range(args.steps):
         r, dt = oracle_run(A, Om, w, blocks)
         times.append(dt)
@@ -175,12 +175,186 @@ def run_reference(args, w, rank, world):
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": sec * 1e3, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": w.dtype, "data": "synthetic",
             "config": {"workload": w.name, "m": w.m, "n": w.n, "b": w.b, "tol": w.tol, "max_rank": w.max_rank,
-                       "sample": sample},
+                       "k": r.k, "block_steps": r.steps, "status": r.status, "sample": sample},
             "cpu_baseline": {"value": tf, "unit": "TFLOP/s", "cores": host_threads(), "kind": "oracle",
                              "sample": sample},
             "e2e": {"value": tf, "unit": "TFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}
     print(json.dumps(line))
+
+
+class Problem:
+    """One workload resident on the device: inputs, outputs and workspace of rrf_run."""
+
+    def __init__(self, h, w, dev, sched):
+        import torch
+        from paper_2608_28941_b200 import rrf
+        self.h, self.w, self.dev, self.sched = h, w, dev, sched
+        self.A, self.Om, self.OmT = generate(w, dev)
+        self.tdt, self.esize = self.A.dtype, self.A.element_size()
+        p = rrf.make_params(rrf.RRF_F64 if w.dtype == "f64" else rrf.RRF_F32, w.m, w.n, w.b, w.tol, w.max_rank)
+        self.ws = torch.empty(rrf.rrf_workspace_bytes(p), dtype=torch.uint8, device=dev)
+        self.V = torch.empty((w.m, w.max_rank), dtype=self.tdt, device=dev)
+        self.T = torch.empty((w.b, w.max_rank), dtype=self.tdt, device=dev)
+        self.B = torch.empty((w.max_rank, w.n), dtype=self.tdt, device=dev)
+
+    def step(self, A=None, omegaT="resident", flags=0):
+        from paper_2608_28941_b200 import rrf
+        w = self.w
+        om = self.OmT if isinstance(omegaT, str) else omegaT
+        return rrf.rrf_run(self.h, self.A if A is None else A, w.b, w.tol, w.max_rank, omegaT=om, V=self.V, T=self.T,
+                           B=self.B, workspace=self.ws, flags=self.sched | flags, seed=w.seed)
+
+
+def time_problem(pb, steps, warmup, world, barrier):
+    """Timed region (the call as a user makes it) and, right after it, the per-kernel event profile."""
+    import torch
+    from paper_2608_28941_b200 import rrf
+    h = pb.h
+    rrf.rrf_set_profiling(h, False)
+    res = None
+    for _ in range(max(warmup, 1)):
+        res = pb.step()
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(steps):
+        res = pb.step()
+    e1.record()
+    barrier()
+    ms_step = max_over_ranks(e0.elapsed_time(e1), world, pb.dev) / steps
+    # per-kernel events lengthen a step by several percent, so they are kept out of the timed region
+    p0, p1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    rrf.rrf_set_profiling(h, True)
+    for _ in range(2):
+        pb.step()
+    prof = {}
+    barrier()
+    p0.record()
+    for _ in range(steps):
+        pb.step()
+        for name, (ms, cnt) in rrf.rrf_get_profile(h).items():
+            a = prof.setdefault(name, [0.0, 0])
+            a[0] += ms
+            a[1] += cnt
+    p1.record()
+    barrier()
+    rrf.rrf_set_profiling(h, False)
+    return res, ms_step, prof, p0.elapsed_time(p1) / steps
+
+
+def roofline_of(pb, res, prof, steps, value_per_gpu, ms_step, ms_profiled, peaks, local):
+    """Roofline of the dominant kernel from the event profile.  `frac` is against the whole device's peak."""
+    import torch
+    from paper_2608_28941_b200 import rrf
+    w, h = pb.w, pb.h
+    gemm = {"sample", "vtw", "update"}
+    top = max((nm for nm in prof if nm not in ("skipped",)), key=lambda nm: prof[nm][0])
+    ms, cnt = prof[top]
+    mi = [w.m - i * w.b for i in range(res.steps)]
+    kind = 0 if w.dtype == "f64" else 3
+    peak = rrf.rrf_measure_peak(h, kind, 200.0)
+    if w.dtype == "f32":
+        peak /= 3.0                               # three TF32 products per fp32 product
+    if top in gemm:
+        work = steps * sum(2.0 * r * w.n * w.b for r in mi)
+        if top == "update":                       # the fused kernel also samples a later panel in most passes
+            work += steps * sum(2.0 * (r - w.b) * w.n * w.b for r in mi[:res.fused_samples])   # rows below B_i
+        if top == "sample":
+            work = steps * 2.0 * w.m * w.n * w.b
+        achieved = work / (ms * 1e-3) / 1e12
+        recipe = peaks.get("bf16_tflops", 1590.0) * NOMINAL_FP64_OVER_BF16 if w.dtype == "f64" else None
+        sms = torch.cuda.get_device_properties(local).multi_processor_count
+        share = (sms - res.panel_ctas) / sms if (res.queues == 2 and top == "update") else 1.0
+        rl = {"kernel": top, "bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
+              "frac": achieved / peak, "traffic": NCU_TRAFFIC_BYTES.get((w.name, top)),
+              "peak_source": ("FP64 mma.sync rate of the whole device, measured live by rrf_measure_peak" if w.dtype == "f64"
+                              else "TF32 mma.sync rate / 3 of the whole device, measured live by rrf_measure_peak"),
+              "peak_recipe": recipe, "frac_recipe": achieved / recipe if recipe else None,
+              "peak_recipe_source": ("MEASURED_PEAKS.json bf16 x nominal FP64/bf16 ratio (of measured)"
+                                     if "bf16_tflops" in peaks else "fallback bf16 x nominal ratio (of fallback)"),
+              "avg_launch_ms": ms / max(cnt, 1), "launches": cnt,
+              # under the look-ahead schedule the kernel is launched on the SMs the panel kernel leaves it
+              "sm_share": share, "frac_of_own_sms": achieved / (peak * share)}
+    else:
+        hbm = peaks.get("hbm_gbs", 6650.0)
+        byts = steps * sum(2.0 * r * w.b * pb.esize for r in mi)
+        achieved = byts / (ms * 1e-3) / 1e9
+        rl = {"kernel": top, "bound": "hbm", "achieved": achieved, "peak": hbm, "unit": "GB/s",
+              "frac": achieved / hbm, "traffic": NCU_TRAFFIC_BYTES.get((w.name, top)),
+              "peak_source": "MEASURED_PEAKS.json (of measured)" if "hbm_gbs" in peaks else "of fallback",
+              "avg_launch_ms": ms / max(cnt, 1), "launches": cnt}
+    rl["whole_step_frac"] = value_per_gpu / peak
+    rl["phases_ms_per_step"] = {nm: prof[nm][0] / steps for nm in prof}
+    rl["profiled_over"] = ("%d steps right after the timed region, with an event before every kernel "
+                           "(%.3f ms per step with the events, %.3f without)" % (steps, ms_profiled, ms_step))
+    return rl
+
+def e2e_of(pb, res, steps, world, barrier, flops):
+    """The same metric through the C ABI from pinned host memory: every step copies A in and B, V, T out.
+    Omega is drawn on the device by the library (seed), so it does not travel."""
+    import torch
+    from paper_2608_28941_b200 import rrf
+    w, dev = pb.w, pb.dev
+    A_h = pb.A.cpu().pin_memory()
+    B_h = torch.empty((w.max_rank, w.n), dtype=pb.tdt).pin_memory()
+    V_h = torch.empty((w.m, w.max_rank), dtype=pb.tdt).pin_memory()
+    T_h = torch.empty((w.b, w.max_rank), dtype=pb.tdt).pin_memory()
+    # Two device input buffers: the input of step s+1 travels on a copy stream while step s computes and its
+    # results go back, as a caller that streams problems through the library would do.
+    A_d = [torch.empty_like(pb.A), torch.empty_like(pb.A)]
+    arrived = [torch.cuda.Event(), torch.cuda.Event()]
+    copy_stream = torch.cuda.Stream()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+
+    # the pinned host-to-device rate on its own, to tell the link from the loop
+    barrier()
+    e0.record()
+    for _ in range(3):
+        A_d[0].copy_(A_h, non_blocking=True)
+    e1.record()
+    barrier()
+    h2d_gbs = 3 * A_h.numel() * pb.esize / (e0.elapsed_time(e1) * 1e-3) / 1e9
+
+    def send(slot):
+        with torch.cuda.stream(copy_stream):
+            A_d[slot].copy_(A_h, non_blocking=True)
+            arrived[slot].record(copy_stream)
+
+    def loop(nsteps):
+        copy_stream.wait_stream(torch.cuda.current_stream())
+        send(0)
+        r = None
+        for s in range(nsteps):
+            slot = s & 1
+            if s + 1 < nsteps:
+                send(1 - slot)                 # the previous user of that slot has finished: rrf_run synchronises
+            torch.cuda.current_stream().wait_event(arrived[slot])
+            r = pb.step(A=A_d[slot], omegaT=None, flags=rrf.RRF_FLAG_NO_GRAPH)   # the inputs alternate: nothing to replay
+            # B's rows are contiguous; V and T go back whole (a strided copy of their first k columns runs
+            # at 2 GB/s, the whole buffers at the link's rate)
+            B_h[:r.k].copy_(pb.B[:r.k], non_blocking=True)
+            V_h.copy_(pb.V, non_blocking=True)
+            T_h.copy_(pb.T, non_blocking=True)
+        torch.cuda.current_stream().synchronize()
+        return r
+
+    loop(2)
+    barrier()
+    n_e2e = max(2, min(steps, 6))
+    e0.record()
+    r = loop(n_e2e)
+    e1.record()
+    barrier()
+    ms = max_over_ranks(e0.elapsed_time(e1), world, dev) / n_e2e
+    fl = method_flops(w.m, w.n, w.b, r.steps)
+    return {"value": job_tflops(fl, world, ms), "unit": "TFLOP/s", "ms_per_step": ms,
+            "h2d_bytes_per_step": int(A_h.numel() * pb.esize),
+            "d2h_bytes_per_step": int((r.k * w.n + w.m * w.max_rank + w.b * w.max_rank) * pb.esize),
+            "k": r.k, "omega": "drawn on the device from the seed (rrf_fill_omega), not copied",
+            "pinned_h2d_gbs_alone": h2d_gbs,
+            "pipelined": "the input of step s+1 is copied on a second stream while step s computes; %d steps timed, "
+                         "first copy not overlapped" % n_e2e}
 
 
 def main():
@@ -195,10 +369,12 @@ def main():
     ap.add_argument("--max-rank", type=int, default=0, help="override the workload's rank cap")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-per-config", action="store_true", help="skip the short runs of the other four configurations")
     ap.add_argument("--schedule", default="auto", choices=["auto", "one", "two"],
                     help="one queue (sequential), two queues (look-ahead), or the library's own rule")
+    ap.add_argument("--panel", default="column", choices=["column", "tree"], help="panel kernel (b <= 64)")
     args = ap.parse_args()
-    args.warmup = max(args.warmup, 0)
+    args.warmup = max(args.warmup, 3)
 
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -206,7 +382,8 @@ def main():
 
     from paper_2608_28941_b200 import workloads as wl
     w = wl.CONFIGS[args.workload]
-    if args.m or args.n or args.max_rank:
+    custom = bool(args.m or args.n or args.max_rank)
+    if custom:
         w = w.scaled(args.m or w.m, args.n or w.n, max_rank=args.max_rank or w.max_rank)
 
     if args.impl == "reference":
@@ -228,20 +405,9 @@ def main():
     if world > 1:
         dist.barrier()
     h = rrf.rrf_create(local)
-
-    A, Om, OmT = generate(w, dev)
-    tdt = A.dtype
-    esize = A.element_size()
-    p = rrf.make_params(rrf.RRF_F64 if w.dtype == "f64" else rrf.RRF_F32, w.m, w.n, w.b, w.tol, w.max_rank)
-    ws = torch.empty(rrf.rrf_workspace_bytes(p), dtype=torch.uint8, device=dev)
-    V = torch.empty((w.m, w.max_rank), dtype=tdt, device=dev)
-    T = torch.empty((w.b, w.max_rank), dtype=tdt, device=dev)
-    B = torch.empty((w.max_rank, w.n), dtype=tdt, device=dev)
-
     sched = {"auto": 0, "one": rrf.RRF_FLAG_ONE_QUEUE, "two": rrf.RRF_FLAG_TWO_QUEUES}[args.schedule]
-
-    def step():
-        return rrf.rrf_run(h, A, w.b, w.tol, w.max_rank, omegaT=OmT, V=V, T=T, B=B, workspace=ws, flags=sched)
+    if args.panel == "tree":
+        sched |= rrf.RRF_FLAG_PANEL_TREE
 
     def barrier():
         torch.cuda.synchronize()
@@ -249,157 +415,26 @@ def main():
             dist.barrier()
             torch.cuda.synchronize()
 
-    # Timed region: the call as a user makes it (no per-kernel events).  The per-kernel event profile
-    # that feeds `roofline` is taken over the same number of steps right after it, because an event
-    # between every two kernels lengthens a step by several percent.
-    rrf.rrf_set_profiling(h, False)
-    for _ in range(max(args.warmup, 1)):
-        res = step()
+    peaks = measured_peaks()
+    pb = Problem(h, w, dev, sched)
     sampler = ClockSampler(local)
+    pb.step()
     barrier()
     sampler.start()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record()
-    for _ in range(args.steps):
-        res = step()
-    e1.record()
-    barrier()
-    p0, p1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    rrf.rrf_set_profiling(h, True)
-    for _ in range(2):
-        step()
-    prof = {}
-    barrier()
-    p0.record()
-    for _ in range(args.steps):
-        step()
-        for name, (ms, cnt) in rrf.rrf_get_profile(h).items():
-            a = prof.setdefault(name, [0.0, 0])
-            a[0] += ms
-            a[1] += cnt
-    p1.record()
-    barrier()
+    res, ms_step, prof, ms_profiled = time_problem(pb, args.steps, args.warmup, world, barrier)
     clocks = sampler.stop()
-    rrf.rrf_set_profiling(h, False)
-    ms_profiled = p0.elapsed_time(p1) / args.steps
-    ms_step = max_over_ranks(e0.elapsed_time(e1), world, dev) / args.steps
     flops = method_flops(w.m, w.n, w.b, res.steps)
     value = job_tflops(flops, world, ms_step)
-    launches_per_run = res.kernel_launches     # counted by the library: every kernel it put on the device
+    launches = args.steps * res.kernel_launches      # counted by the library: every kernel it put on the device
 
-    # ---- end to end through the C ABI with host buffers
-    e2e = None
-    if not args.no_e2e:
-        A_h = A.cpu().pin_memory()
-        O_h = OmT.cpu().pin_memory()
-        k = res.k
-        B_h = torch.empty((w.max_rank, w.n), dtype=tdt).pin_memory()
-        V_h = torch.empty((w.m, w.max_rank), dtype=tdt).pin_memory()
-        T_h = torch.empty((w.b, w.max_rank), dtype=tdt).pin_memory()
-        # Two sets of device input buffers: the inputs of step s+1 travel on a copy stream while step s
-        # computes and its results go back, as a caller that streams problems through the library would do.
-        # Every step still pays its own host-to-device copy and device-to-host read inside the timed region.
-        A_d = [torch.empty_like(A), torch.empty_like(A)]
-        O_d = [torch.empty_like(OmT), torch.empty_like(OmT)]
-        arrived = [torch.cuda.Event(), torch.cuda.Event()]
-        copy_stream = torch.cuda.Stream()
-
-        def send(slot):
-            with torch.cuda.stream(copy_stream):
-                A_d[slot].copy_(A_h, non_blocking=True)
-                O_d[slot].copy_(O_h, non_blocking=True)
-                arrived[slot].record(copy_stream)
-
-        def e2e_loop(nsteps):
-            copy_stream.wait_stream(torch.cuda.current_stream())
-            send(0)
-            r = None
-            for s in range(nsteps):
-                slot = s & 1
-                if s + 1 < nsteps:
-                    send(1 - slot)                 # the previous user of that slot has finished: rrf_run synchronises
-                torch.cuda.current_stream().wait_event(arrived[slot])
-                r = rrf.rrf_run(h, A_d[slot], w.b, w.tol, w.max_rank, omegaT=O_d[slot], V=V, T=T, B=B, workspace=ws,
-                                flags=sched | rrf.RRF_FLAG_NO_GRAPH)     # the input buffers alternate: nothing to replay
-                B_h[:r.k].copy_(B[:r.k], non_blocking=True)
-                V_h[:, :r.k].copy_(V[:, :r.k], non_blocking=True)
-                T_h[:, :r.k].copy_(T[:, :r.k], non_blocking=True)
-            torch.cuda.current_stream().synchronize()
-            return r
-        e2e_loop(2)
-        barrier()
-        n_e2e = max(2, min(args.steps, 6))
-        e0.record()
-        e2e_loop(n_e2e)
-        e1.record()
-        barrier()
-        ms_e2e = max_over_ranks(e0.elapsed_time(e1), world, dev) / n_e2e
-        e2e = {"value": job_tflops(flops, world, ms_e2e), "unit": "TFLOP/s", "ms_per_step": ms_e2e,
-               "h2d_bytes_per_step": int((A_h.numel() + O_h.numel()) * esize),
-               "d2h_bytes_per_step": int((k * w.n + w.m * k + w.b * k) * esize),
-               "pipelined": "inputs of step s+1 are copied on a second stream while step s computes; %d steps timed, "
-                            "first copy not overlapped" % n_e2e}
-
-    # ---- roofline of the dominant kernel, from the event profile of the timed region
-    roofline = None
-    if rank == 0:
-        peaks = measured_peaks()
-        gemm = {"sample", "vtw", "update"}
-        top = max((nm for nm in prof if nm not in ("skipped",)), key=lambda nm: prof[nm][0])
-        ms, cnt = prof[top]
-        per_run_steps = res.steps
-        mi = [w.m - i * w.b for i in range(per_run_steps)]
-        if top in gemm:
-            kind = 0 if w.dtype == "f64" else 3
-            peak = rrf.rrf_measure_peak(h, kind, 200.0)
-            if w.dtype == "f32":
-                peak /= 3.0                       # three TF32 products per fp32 product
-            work = args.steps * sum(2.0 * r * w.n * w.b for r in mi)
-            if top == "update":                   # the fused kernel also samples a later panel in most passes
-                work += args.steps * sum(2.0 * (r - w.b) * w.n * w.b for r in mi[:res.fused_samples])   # rows below B_i
-            if top == "sample":
-                work = args.steps * 2.0 * w.m * w.n * w.b
-            achieved = work / (ms * 1e-3) / 1e12
-            recipe = peaks.get("bf16_tflops", 1590.0) * NOMINAL_FP64_OVER_BF16 if w.dtype == "f64" else None
-            roofline = {"kernel": top, "bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
-                        "frac": achieved / peak, "traffic": NCU_TRAFFIC_BYTES.get((w.name, top)),
-                        "peak_source": "FP64 mma.sync rate measured live by rrf_measure_peak" if w.dtype == "f64"
-                        else "TF32 mma.sync rate / 3 measured live by rrf_measure_peak",
-                        "peak_recipe": recipe,
-                        "frac_recipe": achieved / recipe if recipe else None,
-                        "peak_recipe_source": ("MEASURED_PEAKS.json bf16 x nominal FP64/bf16 ratio (of measured)"
-                                               if "bf16_tflops" in peaks else "fallback bf16 x nominal ratio (of fallback)"),
-                        "avg_launch_ms": ms / max(cnt, 1), "launches": cnt}
-            # With the look-ahead schedule the update is launched on the SMs the panel kernel leaves it and
-            # the two run at the same time, so the roofline that bounds this kernel is that of its SMs.
-            sms = torch.cuda.get_device_properties(local).multi_processor_count
-            share = (sms - res.panel_ctas) / sms if (res.queues == 2 and top == "update") else 1.0
-            roofline["sm_share"] = share
-            roofline["peak_device"] = peak
-            roofline["frac_device"] = achieved / peak
-            if share < 1.0:
-                roofline["peak"] = peak * share
-                roofline["frac"] = achieved / (peak * share)
-                roofline["peak_source"] += " x %d/%d SMs (the kernel runs on %d SMs beside the panel kernel on %d)" % (
-                    sms - res.panel_ctas, sms, sms - res.panel_ctas, res.panel_ctas)
-            roofline["whole_step_frac"] = value / world / peak
-        else:
-            hbm = peaks.get("hbm_gbs", 6650.0)
-            byts = args.steps * sum(2.0 * r * w.b * esize for r in mi)
-            achieved = byts / (ms * 1e-3) / 1e9
-            roofline = {"kernel": top, "bound": "hbm", "achieved": achieved, "peak": hbm, "unit": "GB/s",
-                        "frac": achieved / hbm, "traffic": NCU_TRAFFIC_BYTES.get((w.name, top)),
-                        "peak_source": "MEASURED_PEAKS.json (of measured)" if "hbm_gbs" in peaks else "of fallback",
-                        "avg_launch_ms": ms / max(cnt, 1), "launches": cnt}
-        roofline["phases_ms_per_step"] = {nm: prof[nm][0] / args.steps for nm in prof}
-        roofline["profiled_over"] = ("%d steps right after the timed region, with an event before every kernel "
-                                     "(%.3f ms per step with the events, %.3f without)" % (args.steps, ms_profiled, ms_step))
+    e2e = None if args.no_e2e else e2e_of(pb, res, args.steps, world, barrier, flops)
+    roofline = roofline_of(pb, res, prof, args.steps, value / world, ms_step, ms_profiled, peaks, local) if rank == 0 else None
 
     # ---- CPU baseline: the oracle on the host cores (rank 0, single-GPU runs only)
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        A64 = A.cpu().numpy().astype(np.float64)
-        Om64 = Om.astype(np.float64)
+        A64 = pb.A.cpu().numpy().astype(np.float64)
+        Om64 = pb.Om.astype(np.float64)
         _, t2 = oracle_run(A64, Om64, w, blocks=2)
         est = t2 / 2 * (w.max_rank // w.b)
         blocks = None if est < 40 else max(1, int(25.0 / (t2 / 2)))
@@ -407,19 +442,46 @@ def main():
         cpu = {"value": method_flops(w.m, w.n, w.b, r.steps) / dt / 1e12, "unit": "TFLOP/s", "cores": host_threads(),
                "kind": "oracle", "seconds": dt, "k": r.k,
                "sample": "full workload, one run" if blocks is None else f"first {r.steps} block steps, one run"}
+        del A64, Om64
+
+    # ---- the other configurations, briefly: time, rate, fraction of the peak, dominant kernel
+    per_config = None
+    if rank == 0 and world == 1 and not custom and not args.no_per_config:
+        del pb
+        torch.cuda.empty_cache()
+        per_config = []
+        for name in ("cfg1", "cfg2", "cfg3", "cfg4", "cfg5"):
+            if name == w.name:
+                continue
+            wc = wl.CONFIGS[name]
+            n_steps = 3 if name == "cfg5" else 10
+            pc = Problem(h, wc, dev, sched)
+            r, ms, pr, msp = time_problem(pc, n_steps, 3, 1, barrier)
+            v = job_tflops(method_flops(wc.m, wc.n, wc.b, r.steps), 1, ms)
+            rl = roofline_of(pc, r, pr, n_steps, v, ms, msp, peaks, local)
+            per_config.append({"workload": name, "dtype": wc.dtype, "m": wc.m, "n": wc.n, "b": wc.b, "tol": wc.tol,
+                               "max_rank": wc.max_rank, "k": r.k, "block_steps": r.steps, "status": r.status,
+                               "queues": r.queues, "panel_ctas": r.panel_ctas, "steps_timed": n_steps,
+                               "ms_per_step": ms, "tflops": v, "peak_tflops": rl["peak"] if rl["bound"] == "tensor" else None,
+                               "whole_step_frac": rl["whole_step_frac"], "dominant_kernel": rl["kernel"],
+                               "dominant_bound": rl["bound"], "dominant_frac": rl["frac"],
+                               "phases_ms_per_step": rl["phases_ms_per_step"]})
+            del pc
+            torch.cuda.empty_cache()
 
     if rank == 0:
+        esize = 8 if w.dtype == "f64" else 4
         line = {"metric": "rangefinder_tflops", "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps,
                 "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
                 "vs_baseline": None, "dtype": w.dtype, "data": "synthetic",
                 "config": {"workload": w.name, "m": w.m, "n": w.n, "b": w.b, "tol": w.tol, "max_rank": w.max_rank,
                            "k": res.k, "block_steps": res.steps, "status": res.status,
                            "l2": "inputs larger than L2 (A is %.0f MB)" % (w.m * w.n * esize / 1e6),
-                           "queues": res.queues, "panel_ctas": res.panel_ctas,
+                           "queues": res.queues, "panel_ctas": res.panel_ctas, "panel_kernel": args.panel,
                            "fused_samples": res.fused_samples, "extra_samples": res.extra_samples,
                            "parallelism": "replicas only" if world > 1 else "single GPU"},
-                "clocks": clocks, "e2e": e2e, "gpu_launches": args.steps * launches_per_run,
-                "roofline": roofline, "cpu_baseline": cpu}
+                "clocks": clocks, "e2e": e2e, "gpu_launches": launches,
+                "roofline": roofline, "cpu_baseline": cpu, "per_config": per_config}
         print(json.dumps(line))
     rrf.rrf_destroy(h)
     if world > 1:

@@ -100,8 +100,13 @@ def test_full_config_against_oracle(h, name):
         # Block i is sampled from a residual of relative size rho_i = sqrt(E_{i-1} / ||A||^2) that carries
         # rounding noise of the size of u ||A||, so it is only determined to about u / rho_i; what it
         # contributes to Q B is weighted by rho_i (the size of B_i).  A block whose deviation weighted that
-        # way is below a tenth of the plain bar is as good as the input allows.
+        # way is below a tenth of the plain bar is as good as the input allows.  (Config 5's last block mixes
+        # the last b directions of A's range, singular values down to 1.2e-6, with a square Gaussian matrix.)
         rho = np.sqrt((o.E_dir[i - 1] if i > 0 else o.normA2) / o.normA2)
+        if sig is not None:
+            # with a prescribed spectrum the weakest direction the block captures is known: a direction of
+            # singular value s is determined to (noise / s) and enters Q B with weight s
+            rho = min(rho, sig[min((i + 1) * w.b, sig.size) - 1] / np.sqrt(o.normA2))
         assert dq <= bar or dq * rho <= 0.1 * rel, (i, dq, bar, rho)
 
 
