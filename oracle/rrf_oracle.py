@@ -23,6 +23,21 @@ Readings of the paper taken here:
     E <- E - ||B_i||_F^2.  Both are always recorded.
   * rank cap: the loop also ends when another block would exceed `max_rank`
     (the paper's fixed-rank mode).
+  * stopping rules that need neither B nor the updated matrix (the outlook's "alternative stopping
+    criteria ... estimating the spectral norm of the remaining part", and its variant that leaves A
+    unchanged): the sampled panel itself is a randomized probe of the residual.  With Omega_i
+    standard Gaussian (n x b) and W the residual before block i,
+        E[ ||W Omega_i||_F^2 ] = b ||W||_F^2,
+    so `estimator="sampled_fro"` tests E = ||Y_i||_F^2 / b, and (Halko, Martinsson, Tropp 2011,
+    Lemma 4.1) ||W||_2 <= 10 sqrt(2/pi) max_j ||W omega_j||_2 with probability 1 - 10^-b, so
+    `estimator="sampled_spectral"` tests E = (200/pi) max_j ||Y_i[:, j]||_2^2, a bound on the squared
+    SPECTRAL norm of the residual (the norm of Eq. "tolerance").  Both are evaluated when panel i has
+    been sampled and before it is factored: the loop stops with k = i b if E <= sigma^2.  If the rank
+    cap ends the loop instead, nothing certifies the last block and the status is "cap reached".
+  * `schedule="a_unchanged"`: the outlook's variant that never updates A and returns no B.  The
+    panel is sampled from A itself, Y_i = A Omega_i, and the reflector blocks found so far are applied
+    to it, Y_i <- Q_{i-1}^T ... Q_0^T Y_i, before its rows i b.. are factored.  By Theorem 3.1 this is
+    the same panel as the in-place schedule's.  Only the sampled estimators can stop this loop.
 
 Parity status: every function below is pinned by tests/test_oracle_pins.py
 (dense Householder QR of A*Omega via LAPACK, the compact-WY identities, the
@@ -108,6 +123,9 @@ class OracleResult:
     B: np.ndarray            # k x n
     E_sub: list = field(default_factory=list)   # after each block: Algorithm 2 line 9
     E_dir: list = field(default_factory=list)   # after each block: ||W[r0+b:, :]||_F^2
+    E_est: list = field(default_factory=list)   # sampled estimators: per sampled panel, the estimate of the
+                                                # residual BEFORE that block (one entry more than blocks if the
+                                                # estimate stopped the loop)
     W: np.ndarray | None = None                 # final working matrix (m x n)
 
 
@@ -117,9 +135,22 @@ def _sumsq(X: np.ndarray) -> float:
     return float(np.sum(X64 * X64))
 
 
+SPECTRAL_FACTOR = 200.0 / np.pi      # (10 sqrt(2/pi))^2
+
+
+def sampled_estimate(Y: np.ndarray, estimator: str) -> float:
+    """Randomized estimate of the squared residual norm from a sampled panel Y = W Omega_i."""
+    colsq = np.sum(Y.astype(np.float64) ** 2, axis=0)
+    if estimator == "sampled_fro":
+        return float(np.sum(colsq)) / Y.shape[1]
+    if estimator == "sampled_spectral":
+        return SPECTRAL_FACTOR * float(np.max(colsq))
+    raise ValueError(estimator)
+
+
 def rrf(A: np.ndarray, Omega: np.ndarray, b: int, tol: float, max_rank: int,
         relative: bool = True, estimator: str = "direct", keep_w: bool = False,
-        dtype=np.float64) -> OracleResult:
+        dtype=np.float64, schedule: str = "in_place", fixed_rank: bool = False) -> OracleResult:
     """Algorithm 2, in the paper's order.
 
     A: m x n; Omega: n x max_rank (block i uses columns i*b:(i+1)*b, i.e. the
@@ -127,12 +158,19 @@ def rrf(A: np.ndarray, Omega: np.ndarray, b: int, tol: float, max_rank: int,
     if `relative`).  `dtype` is the working precision: float64 is the oracle
     proper; float32 reruns the same steps in single precision (the paper's
     experiments are in single precision) and serves as the plain-fp32 yardstick.
+    `estimator`: "direct", "subtractive", "sampled_fro", "sampled_spectral" (see the header).
+    `schedule`: "in_place" (Algorithm 2) or "a_unchanged" (no update of A, no B; sampled estimators
+    or `fixed_rank` only).  `fixed_rank`: ignore the tolerance and run to the cap.
     """
     W = np.array(A, dtype=dtype, copy=True)                 # line 2: B <- A
     Omega = np.asarray(Omega, dtype=dtype)
     m, n = W.shape
     assert b >= 1 and max_rank % b == 0 and max_rank <= min(m, n)
     assert Omega.shape[0] == n and Omega.shape[1] >= max_rank
+    sampled = estimator in ("sampled_fro", "sampled_spectral")
+    unchanged = schedule == "a_unchanged"
+    assert schedule in ("in_place", "a_unchanged")
+    assert not unchanged or sampled or fixed_rank
     normA2 = _sumsq(W)                                      # line 1: E <- ||A||_F^2
     sigma2 = (tol * tol * normA2) if relative else tol * tol
     V = np.zeros((m, max_rank), dtype=dtype)                # line 3
@@ -140,33 +178,55 @@ def rrf(A: np.ndarray, Omega: np.ndarray, b: int, tol: float, max_rank: int,
     res = OracleResult(0, RRF_OK, 0, normA2, sigma2, V, T, W)
     E_sub = normA2
     E = normA2
+    met = (not fixed_rank) and not (E > sigma2)
     i = 0                                                   # line 4
-    while E > sigma2 and (i + 1) * b <= max_rank:           # line 5 (+ rank cap)
+    while not met and (i + 1) * b <= max_rank:              # line 5 (+ rank cap)
         r0 = i * b
         Om = Omega[:, r0:r0 + b]                            # line 6
-        Y = W[r0:, :] @ Om                                  # line 7: sample ...
+        if unchanged:
+            Y = W @ Om                                      # W is A itself here: it is never updated
+            for l in range(i):                              # Q_{i-1}^T ... Q_0^T, in the order Q_0^T first
+                q0 = l * b
+                Vl = V[q0:, q0:q0 + b]
+                Tl = T[:, q0:q0 + b]
+                Y[q0:, :] -= Vl @ (Tl.T @ (Vl.T @ Y[q0:, :]))
+            Y = Y[r0:, :]
+        else:
+            Y = W[r0:, :] @ Om                              # line 7: sample ...
+        if sampled:
+            E = sampled_estimate(Y, estimator)
+            res.E_est.append(E)
+            if not fixed_rank and not (E > sigma2):
+                met = True
+                break
         Vi, _, Ti, _ = panel_qr(Y)                          # ... and factor
         V[r0:, r0:r0 + b] = Vi
         T[:, r0:r0 + b] = Ti
-        Z = Vi.T @ W[r0:, :]                                # line 8: W <- Q_i^T W
-        Z = Ti.T @ Z
-        W[r0:, :] -= Vi @ Z
-        Bi = W[r0:r0 + b, :]
-        E_sub = E_sub - _sumsq(Bi)                          # line 9
-        trail = W[r0 + b:, :]
-        E_dir = _sumsq(trail)
-        res.E_sub.append(E_sub)
-        res.E_dir.append(E_dir)
-        E = E_dir if estimator == "direct" else E_sub
+        if not unchanged:
+            Z = Vi.T @ W[r0:, :]                            # line 8: W <- Q_i^T W
+            Z = Ti.T @ Z
+            W[r0:, :] -= Vi @ Z
+            Bi = W[r0:r0 + b, :]
+            E_sub = E_sub - _sumsq(Bi)                      # line 9
+            trail = W[r0 + b:, :]
+            E_dir = _sumsq(trail)
+            res.E_sub.append(E_sub)
+            res.E_dir.append(E_dir)
+            if not sampled:
+                E = E_dir if estimator == "direct" else E_sub
+                met = (not fixed_rank) and not (E > sigma2)
         i += 1                                              # line 10
     k = i * b                                               # lines 12-14
     res.k = k
     res.steps = i
-    res.status = RRF_OK if E <= sigma2 else RRF_MAX_RANK_REACHED
+    if sampled or unchanged:
+        res.status = RRF_OK if met else RRF_MAX_RANK_REACHED     # only an estimate that stopped the loop certifies
+    else:
+        res.status = RRF_OK if E <= sigma2 else RRF_MAX_RANK_REACHED
     res.V = V[:, :k]
     res.T = T[:, :k]
-    res.B = W[:k, :].copy()
-    res.W = W if keep_w else None
+    res.B = None if unchanged else W[:k, :].copy()
+    res.W = W if (keep_w and not unchanged) else None
     return res
 
 

@@ -323,3 +323,71 @@ def test_householder_keeps_orthogonality_where_block_gram_schmidt_loses_it():
     # Householder and reorthogonalised Gram-Schmidt both reach the single-precision floor of this matrix
     floor = np.linalg.svd(A64, compute_uv=False)[passes * b]
     assert proj_res(Q_hh) < 50 * max(floor, u32) and proj_res(Q_re) < 50 * max(floor, u32)
+
+
+# ---- sampled stopping estimators and the schedule that leaves A unchanged
+
+
+def test_sampled_frobenius_estimate_is_exact_for_an_orthogonal_probe():
+    # closed form: with Omega_i = sqrt(b) O, O orthogonal n x n (b = n), ||W Omega_i||_F^2 / b = ||W||_F^2
+    rng = np.random.default_rng(21)
+    W = rng.standard_normal((30, 12))
+    O, _ = np.linalg.qr(rng.standard_normal((12, 12)))
+    est = orc.sampled_estimate(W @ (np.sqrt(12.0) * O), "sampled_fro")
+    assert np.isclose(est, np.linalg.norm(W) ** 2, rtol=1e-13)
+
+
+def test_sampled_estimates_are_unbiased_and_bound_the_spectral_norm():
+    rng = np.random.default_rng(22)
+    W = rng.standard_normal((60, 40)) * np.exp(-np.arange(40) / 6.0)
+    fro2, two2 = np.linalg.norm(W) ** 2, np.linalg.norm(W, 2) ** 2
+    b, draws = 8, 400
+    est_f = np.array([orc.sampled_estimate(W @ rng.standard_normal((40, b)), "sampled_fro") for _ in range(draws)])
+    # E[est] = ||W||_F^2; Var[est] = 2 ||W^T W||_F^2 / b
+    std = np.sqrt(2.0 * np.linalg.norm(W.T @ W) ** 2 / b / draws)
+    assert abs(est_f.mean() - fro2) < 5 * std
+    est_s = np.array([orc.sampled_estimate(W @ rng.standard_normal((40, b)), "sampled_spectral") for _ in range(draws)])
+    assert np.all(est_s >= two2)                      # fails with probability 10^-b per draw
+    assert np.median(est_s) < 64 * 40 * two2          # and it is not vacuous
+
+
+@pytest.mark.parametrize("estimator", ["sampled_fro", "sampled_spectral"])
+def test_sampled_rules_stop_on_the_panel_before_it_is_factored(estimator):
+    A, Om, s, b, max_rank = _case(m=120, n=100, b=10, max_rank=80, seed=5, decay=4.0)
+    tol = 1e-3
+    r = orc.rrf(A, Om, b, tol, max_rank, estimator=estimator, keep_w=True)
+    assert r.status == orc.RRF_OK and 0 < r.k < max_rank
+    assert len(r.E_est) == r.steps + 1                # the estimate that stopped the loop has no block
+    # brute force from the recorded residuals: entry i was computed from the residual after i blocks
+    sigma2 = tol * tol * r.normA2
+    assert all(e > sigma2 for e in r.E_est[:-1]) and r.E_est[-1] <= sigma2
+    Q = orc.form_q(r.V, r.T, b)
+    res2 = np.linalg.norm(A - Q @ (Q.T @ A)) ** 2
+    if estimator == "sampled_spectral":               # certifies the 2-norm of the residual
+        assert np.linalg.norm(A - Q @ (Q.T @ A), 2) ** 2 <= r.E_est[-1] <= sigma2
+    else:                                             # tracks the Frobenius residual within its spread
+        assert 0.3 * res2 <= r.E_est[-1] <= 3.0 * res2
+    # the first estimate probes A itself
+    assert np.isclose(r.E_est[0], orc.sampled_estimate(A @ Om[:, :b], estimator), rtol=1e-12)
+
+
+def test_schedule_that_leaves_a_unchanged_gives_the_same_reflectors():
+    # Theorem 3.1: the panel sampled from A and pulled through the reflectors found so far is the panel the
+    # in-place schedule samples from the updated matrix, so V, T (and k under a sampled rule) agree
+    A, Om, s, b, max_rank = _case(m=90, n=70, b=6, max_rank=36, seed=8, decay=5.0)
+    r1 = orc.rrf(A, Om, b, 0.0, max_rank, fixed_rank=True)
+    r2 = orc.rrf(A, Om, b, 0.0, max_rank, fixed_rank=True, schedule="a_unchanged")
+    assert r2.k == r1.k == max_rank and r2.B is None
+    prev = [r1.normA2] + r1.E_dir[:-1]
+    for i in range(max_rank // b):
+        amp = np.sqrt(r1.normA2 / prev[i])
+        blk = slice(i * b, (i + 1) * b)
+        assert np.max(np.abs(r1.V[:, blk] - r2.V[:, blk])) < 1e-13 * amp, i
+        assert np.max(np.abs(r1.T[:, blk] - r2.T[:, blk])) < 1e-12 * amp, i
+    # against LAPACK directly: the reflectors are those of the dense QR of A Omega
+    V_ref, tau_ref, _ = _lapack_vtau(A @ Om[:, :max_rank])
+    assert np.max(np.abs(r2.V[:, :b] - V_ref[:, :b])) < 1e-13
+    a = orc.rrf(A, Om, b, 5e-2, max_rank, estimator="sampled_fro")
+    u = orc.rrf(A, Om, b, 5e-2, max_rank, estimator="sampled_fro", schedule="a_unchanged")
+    assert 0 < a.k < max_rank and a.k == u.k and a.status == u.status == orc.RRF_OK
+    assert np.allclose(a.E_est, u.E_est, rtol=1e-9)
