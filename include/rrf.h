@@ -62,6 +62,10 @@ typedef enum {
                                     the kernel that pays one grid barrier per column.  Off by default: it is the
                                     slower of the two on the sizes measured so far.  The look-ahead schedule is
                                     then used only if RRF_FLAG_TWO_QUEUES asks for it */
+#define RRF_FLAG_NO_UPDATE 256u /* the variant of the paper's outlook that leaves A unchanged and returns no B: each
+                                  panel is sampled from A itself and pulled through the reflector blocks found so
+                                  far.  One pass over A per block instead of three.  Needs estimator 2 or 3, or
+                                  RRF_FLAG_FIXED_RANK; dB may be NULL; sequential schedule, per-column panel kernel */
 #define RRF_FLAG_TWO_QUEUES 8u  /* use the look-ahead schedule whenever the panel can be confined to a few SMs,
                                    also where the built-in rule would pick the sequential one */
 
@@ -70,7 +74,14 @@ typedef struct {
   int32_t b;                /* block size */
   int32_t max_rank;         /* rank cap, multiple of b, <= min(m, n) */
   int32_t estimator;        /* 0: stop on the residual norm ||W[r0+b:, :]||_F^2 (default);
-                               1: stop on the paper's E <- E - ||B_i||_F^2 (Algorithm 2, line 9) */
+                               1: stop on the paper's E <- E - ||B_i||_F^2 (Algorithm 2, line 9);
+                               2, 3: sampled rules, evaluated on panel i = W Omega_i before block i is applied and
+                               ending the loop with k = i b if E <= sigma^2 (W: the residual left by i blocks):
+                               2: E = ||Y_i||_F^2 / b, an unbiased estimate of ||W||_F^2;
+                               3: E = (200/pi) max_j ||Y_i[:, j]||^2 >= ||W||_2^2 with probability 1 - 10^-b
+                                  (a bound on the SPECTRAL norm of the residual, the norm of Eq. "tolerance").
+                               If the rank cap ends the loop under 2 or 3 the status is RRF_MAX_RANK_REACHED:
+                               nothing has certified the last block. */
   int64_t m, n;             /* A is m x n */
   double tol;               /* the tolerance sigma of Algorithm 2 ... */
   int32_t tol_is_relative;  /* ... taken as tol*||A||_F if non-zero */
@@ -98,7 +109,7 @@ typedef struct {
                                predictions, or RRF_FLAG_SAMPLE_NEVER) */
   int32_t kernel_launches;  /* kernels of this library the call put on the device, passes after the stop
                                included (their kernels start, read the stop flag and return) */
-  int32_t reserved;
+  int32_t n_est;            /* estimators 2, 3: estimates evaluated (steps + 1 if an estimate ended the loop) */
 } rrf_result_t;
 
 /* Create / destroy a context bound to one CUDA device.  rrf_create makes `device`
@@ -134,6 +145,8 @@ rrf_status_t rrf_workspace_bytes(const rrf_params_t* p, size_t* bytes);
  *            to cuda_stream with events.
  *   h_E_sub_trace, h_E_dir_trace   optional HOST arrays of max_rank/b doubles receiving
  *            both stopping quantities after every block step.
+ *   h_E_est_trace   optional HOST array of max_rank/b + 1 doubles: under estimator 2 or 3, entry i is
+ *            the estimate of the residual left by i blocks (out->n_est entries).
  *
  * The loop `while E > sigma^2` runs on the device: each kernel of a block step first
  * reads a device flag and returns at once when the stop rule has fired, so there is no
@@ -159,7 +172,7 @@ rrf_status_t rrf_run(rrf_handle_t h, const rrf_params_t* p,
                      void* dB, int64_t ldb,
                      void* d_workspace, size_t workspace_bytes,
                      void* cuda_stream, rrf_result_t* out,
-                     double* h_E_sub_trace, double* h_E_dir_trace);
+                     double* h_E_sub_trace, double* h_E_dir_trace, double* h_E_est_trace);
 
 /*
  * rrf_panel_qr - Algorithm 2 line 7 on its own (LAPACK geqrt semantics): Householder QR of a

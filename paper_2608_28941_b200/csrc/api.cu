@@ -418,6 +418,8 @@ struct PanelOpts {
   cudaStream_t st_t = nullptr;     // side stream for the T factor, with its fork / join events
   cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
   bool tree = false;               // b <= 64: use the tree kernel (no grid barrier per column)
+  double* csq = nullptr;           // [b][Gp]: the panel kernel leaves the column sums of squares of the panel here
+  int* g_out = nullptr;            // out: CTAs of the per-column panel kernel (Gp = g rounded up to 32)
 };
 template <typename Mark = NoMark>
 static rrf_status_t launch_panel(rrf_ctx* h, int dtype, const void* Y, PanelSource src,
@@ -459,11 +461,13 @@ static rrf_status_t launch_panel(rrf_ctx* h, int dtype, const void* Y, PanelSour
   const int* fused_flag = o.fused_flag;
   unsigned bar_base = o.bar_base;
   void* Tmerged = o.merge_t ? Tout : nullptr;
+  double* csq = o.csq;
   void* args[] = {&Y,   &src, &alt, &fused_flag, &rows_i, &b,    &R,    &Rp,        &V,   &ldv,      &P,
-                  &piv, &gram, &tau, &bar,       &ctrl,   &done_flag, &fix, &bar_base, &Tmerged, &ldt};
+                  &piv, &gram, &tau, &bar,       &ctrl,   &done_flag, &fix, &bar_base, &Tmerged, &ldt, &csq};
   const size_t tsmem = ((size_t)b * (b + 1) + (size_t)(b / 2) * (b / 2 + 1)) * sizeof(double);
   if (o.merge_t) pp.smem = std::max(pp.smem, tsmem);
   if (o.bar_used != nullptr) *o.bar_used = (unsigned)(b + (o.fix.enabled ? 2 : 0)) * (unsigned)pp.G;
+  if (o.g_out != nullptr) *o.g_out = pp.G;
   mark(RRF_PHASE_PANEL, step);
   const void* fn = dtype == RRF_F64 ? panel_variant<double>(pp.variant) : panel_variant<float>(pp.variant);
   cudaError_t e = cudaLaunchCooperativeKernel(fn, dim3(pp.G), dim3(kPanelThreads), args, pp.smem, st);
@@ -548,7 +552,7 @@ static cudaError_t setup_all(int smem_optin, int* panel_smem_max) {
 
 // ------------------------------------------------------------------ workspace of rrf_run
 struct RunLayout {
-  size_t ctrl, traces, done_after, norm_part, init_part, ypart, ypart2, zpart, zt, panel, look, w, omega, total;
+  size_t ctrl, traces, done_after, norm_part, init_part, ypart, ypart2, zpart, zt, panel, look, csq, w, omega, total;
   int init_ctas, max_norm_parts;
   long long ldw;
 };
@@ -572,7 +576,7 @@ static bool run_layout(const rrf_params_t* p, bool need_omega, RunLayout* L) {
   }
   size_t off = 0;
   L->ctrl = off; off += 256;
-  L->traces = off; off += align_up((size_t)2 * steps * sizeof(double), 256);
+  L->traces = off; off += align_up(((size_t)3 * steps + 1) * sizeof(double), 256);   // E_sub, E_dir, estimates
   L->done_after = off; off += align_up((size_t)(2 * steps + 3) * sizeof(int), 256);   // + the look-ahead barrier word + samp[]
   L->init_ctas = kInitCtas;
   L->init_part = off; off += align_up((size_t)kInitCtas * sizeof(double), 256);
@@ -584,6 +588,7 @@ static bool run_layout(const rrf_params_t* p, bool need_omega, RunLayout* L) {
   L->zt = off; off += align_up((size_t)npad * b * esize, 256);
   L->panel = off; off += panel_scratch_bytes(sms, b);
   L->look = off; off += look_scratch_bytes(b);
+  L->csq = off; off += align_up((size_t)2 * b * ((sms + 31) / 32 * 32) * sizeof(double), 256);   // two panels in flight
   L->w = off;
   L->ldw = (long long)align_up((size_t)p->n, 16);   // rows of the working copy start on 128-byte lines
   if (!(p->flags & RRF_FLAG_INPLACE)) off += align_up((size_t)p->m * (size_t)L->ldw * esize, 256);
@@ -601,7 +606,13 @@ static rrf_status_t check_params(const rrf_params_t* p) {
   if (p->max_rank < p->b || p->max_rank % p->b != 0) return RRF_ERR_INVALID_ARG;
   if (p->max_rank > p->m || p->max_rank > p->n) return RRF_ERR_INVALID_ARG;
   if (!(p->tol >= 0.0)) return RRF_ERR_INVALID_ARG;
-  if (p->estimator != 0 && p->estimator != 1) return RRF_ERR_INVALID_ARG;
+  if (p->estimator < 0 || p->estimator > 3) return RRF_ERR_INVALID_ARG;
+  if (p->estimator >= 2 && (p->flags & RRF_FLAG_PANEL_TREE)) return RRF_ERR_INVALID_ARG;
+  if (p->flags & RRF_FLAG_NO_UPDATE) {
+    // without the update there is no residual to measure: only a sampled rule or the rank cap ends the loop
+    if (p->estimator < 2 && !(p->flags & RRF_FLAG_FIXED_RANK)) return RRF_ERR_INVALID_ARG;
+    if (p->flags & (RRF_FLAG_INPLACE | RRF_FLAG_PANEL_TREE | RRF_FLAG_TWO_QUEUES)) return RRF_ERR_INVALID_ARG;
+  }
   if (p->tune_panel_ctas < 0 || p->tune_gate < 0 || p->tune_gate > 2) return RRF_ERR_INVALID_ARG;
   return RRF_OK;
 }
@@ -948,7 +959,8 @@ rrf_status_t rrf_subspace_transfer(rrf_handle_t h, int32_t dtype, int64_t m, int
 
 rrf_status_t rrf_run(rrf_handle_t h, const rrf_params_t* p, void* dA, int64_t lda, const void* dOmegaT, int64_t ldo,
                      void* dV, int64_t ldv, void* dT, void* dB, int64_t ldb, void* d_workspace, size_t workspace_bytes,
-                     void* cuda_stream, rrf_result_t* out, double* h_E_sub_trace, double* h_E_dir_trace) {
+                     void* cuda_stream, rrf_result_t* out, double* h_E_sub_trace, double* h_E_dir_trace,
+                     double* h_E_est_trace) {
   if (out == nullptr) return RRF_ERR_INVALID_ARG;
   std::memset(out, 0, sizeof(*out));
   auto fail = [&](rrf_status_t s) {
@@ -961,12 +973,13 @@ rrf_status_t rrf_run(rrf_handle_t h, const rrf_params_t* p, void* dA, int64_t ld
   const int esize = p->dtype == RRF_F64 ? 8 : 4;
   const int b = p->b;
   const long long m = p->m, n = p->n;
-  if (dA == nullptr || dV == nullptr || dT == nullptr || dB == nullptr || d_workspace == nullptr)
+  const bool unchanged = (p->flags & RRF_FLAG_NO_UPDATE) != 0;     // A is never updated, B is not produced
+  if (dA == nullptr || dV == nullptr || dT == nullptr || (dB == nullptr && !unchanged) || d_workspace == nullptr)
     return fail(RRF_ERR_INVALID_ARG);
-  if (!ld_ok(lda, n, esize) || !ld_ok(ldv, p->max_rank, esize) || !ld_ok(ldb, n, esize))
+  if (!ld_ok(lda, n, esize) || !ld_ok(ldv, p->max_rank, esize) || (dB != nullptr && !ld_ok(ldb, n, esize)))
     return fail(RRF_ERR_INVALID_ARG);
   if (dOmegaT != nullptr && (!ld_ok(ldo, n, esize) || !aligned16(dOmegaT))) return fail(RRF_ERR_INVALID_ARG);
-  if (!aligned16(dA) || !aligned16(dV) || !aligned16(dB) || (reinterpret_cast<uintptr_t>(d_workspace) & 255u))
+  if (!aligned16(dA) || !aligned16(dV) || (dB != nullptr && !aligned16(dB)) || (reinterpret_cast<uintptr_t>(d_workspace) & 255u))
     return fail(RRF_ERR_INVALID_ARG);
   RunLayout L;
   run_layout(p, dOmegaT == nullptr, &L);
@@ -983,7 +996,7 @@ rrf_status_t rrf_run(rrf_handle_t h, const rrf_params_t* p, void* dA, int64_t ld
     const int lim = p->tune_panel_ctas > 0 ? std::min(cap, (int)p->tune_panel_ctas) : cap;
     if ((p->flags & RRF_FLAG_TWO_QUEUES) && steps_total >= 2 && plan_tree(h, m, b, lim, true, &tl)) look_ctas = tl.ctas;
     if (look_ctas == 0 && !plan_tree(h, m, b, 0, false, &tl)) return fail(RRF_ERR_WORKSPACE);
-  } else if (!(p->flags & RRF_FLAG_ONE_QUEUE) && steps_total >= 2) {
+  } else if (!(p->flags & RRF_FLAG_ONE_QUEUE) && !unchanged && steps_total >= 2) {
     const int fewest = panel_min_ctas(h, m, b);
     const int cap = std::min(kLookMaxCtas, h->sms / 3);
     if (fewest > 0 && fewest <= cap) {
@@ -1014,6 +1027,11 @@ rrf_status_t rrf_run(rrf_handle_t h, const rrf_params_t* p, void* dA, int64_t ld
   const int steps = p->max_rank / b;
   double* tr_sub = reinterpret_cast<double*>(ws + L.traces);
   double* tr_dir = tr_sub + steps;
+  double* tr_est = tr_dir + steps;                   // [steps + 1]
+  const bool sampled = p->estimator >= 2;
+  double* csq0 = reinterpret_cast<double*>(ws + L.csq);
+  const int csq_gp = (h->sms + 31) / 32 * 32;
+  auto csq_buf = [&](int i) { return csq0 + (size_t)(i & 1) * b * csq_gp; };
   int* done_after = reinterpret_cast<int*>(ws + L.done_after);
   unsigned* look_bar = reinterpret_cast<unsigned*>(done_after + steps + 1);
   int* samp = done_after + steps + 2;   // [steps + 1]: does the update of pass q sample a later panel
@@ -1123,7 +1141,59 @@ rrf_status_t rrf_run(rrf_handle_t h, const rrf_params_t* p, void* dA, int64_t ld
   init_ctrl_kernel<<<1, 256, 0, st>>>(init_part, std::min(sp.nslabs * sp.nseg, sp.ctas), p->tol, p->tol_is_relative,
                                       fixed ? 1 : 0, b, p->max_rank, ctrl, done_after, samp, steps, predict);
 
-  if (look_ctas == 0) {
+  if (unchanged) {
+    // The variant of the paper's outlook that leaves A unchanged and returns no B: every panel is sampled from
+    // A itself, Y_i = A Omega_i, pulled through the reflector blocks found so far (Q_0^T first), and its rows
+    // i b.. are factored.  One pass over A per block instead of three; only a sampled rule (or the cap) stops it.
+    void* Pbuf = ws + L.w;             // m x b panel, dense (the working copy of A is not needed here)
+    const int npad_p = plan_vtw(h->sms, m, b, ops->v_bn).npad;
+    CUtensorMap tmP_k, tmP_u, tmZp;
+    if (!make_map(h, &tmP_k, p->dtype, Pbuf, m, b, b, kVtwBK) || !make_map(h, &tmP_u, p->dtype, Pbuf, m, b, b, ops->u_bm) ||
+        !make_map(h, &tmZp, p->dtype, Zt, npad_p, b, b, ops->u_bn))
+      return RRF_ERR_INVALID_ARG;
+    unsigned bar_next = 0, bar_used = 0;
+    const int sum_grid = (int)std::min<long long>((m * b + 255) / 256, (long long)h->sms * 8);
+    for (int i = 0; i < steps; ++i) {
+      const int r0 = i * b, rows = (int)(m - r0);
+      if (i > 0) {
+        mark(RRF_PHASE_SAMPLE, i);
+        ops->sample(tmA_s, tmO, Ypart, 0, (int)m, (int)n, r0, sp, ctrl, nullptr, nullptr, st);
+      }
+      if (p->dtype == RRF_F64)
+        panel_sum_kernel<double><<<sum_grid, 256, 0, st>>>((const double*)Ypart, sp.nseg, m * b, m, b, (double*)Pbuf, ctrl);
+      else
+        panel_sum_kernel<float><<<sum_grid, 256, 0, st>>>((const float*)Ypart, sp.nseg, m * b, m, b, (float*)Pbuf, ctrl);
+      for (int l = 0; l < i; ++l) {
+        const int q0 = l * b, rl = (int)(m - q0);
+        const VtwPlan vp = plan_vtw(h->sms, rl, b, ops->v_bn);
+        mark(RRF_PHASE_VTW, i);
+        ops->vtw(tmV_k, tmP_k, Zpart, q0, q0, vp, ctrl, st);
+        mark(RRF_PHASE_TZ, i);
+        ops->tz(Zpart, vp, Tblk(q0), p->max_rank, 1, Zt, &ctrl->done, st);
+        const UpdPlan up = plan_upd(h->sms, rl, b, ops->u_bm, ops->u_bn, ops->u_wn);
+        mark(RRF_PHASE_UPDATE, i);
+        ops->update(tmV_u, tmZp, tmP_u, tmP_u, Pbuf, b, Pbuf, b, q0, rl, b, q0, 0, -1, nullptr, nullptr, up, ctrl, nullptr, st);
+      }
+      PanelSource sd{};
+      sd.nseg = 1;
+      sd.ldy = b;
+      sd.row_off = r0;
+      PanelOpts po;
+      po.merge_t = true;
+      po.bar_base = bar_next;
+      po.bar_used = &bar_used;
+      po.csq = csq_buf(i);
+      int pg = 0;
+      po.g_out = &pg;
+      s = launch_panel(h, p->dtype, Pbuf, sd, rows, b, Vblk(r0), ldv, Tblk(r0), p->max_rank, ps, ctrl, &ctrl->done, st,
+                       mark, i, po);
+      if (s != RRF_OK) return panel_failed(s);
+      bar_next += bar_used;
+      mark(RRF_PHASE_STOP, i);
+      est_kernel<<<1, 128, 0, st>>>(csq_buf(i), pg, (pg + 31) & ~31, b, p->max_rank, sampled ? p->estimator : 2,
+                                    fixed ? 1 : 0, 1, i, tr_est, ctrl);
+    }
+  } else if (look_ctas == 0) {
     // One queue.  The panel of pass 0 is sampled by its own kernel; the panel of pass i+1 comes out
     // of the fused update of pass i.
     PanelSource alt{};             // the upcoming panel as the separate sample kernel would leave it
@@ -1137,9 +1207,15 @@ rrf_status_t rrf_run(rrf_handle_t h, const rrf_params_t* p, void* dA, int64_t ld
       po.alt = alt;
       po.fused_flag = fused_flag;
       po.tree = tree;
+      int pg = 0;
+      if (sampled) po.csq = csq_buf(i);
+      po.g_out = &pg;
       s = launch_panel(h, p->dtype, Ypart, src, rows, b, Vblk(r0), ldv, Tblk(r0), p->max_rank, ps, ctrl, &ctrl->done,
                        st, mark, i, po);
       if (s != RRF_OK) return panel_failed(s);
+      if (sampled)                     // the sampled rule looks at panel i before block i is applied
+        est_kernel<<<1, 128, 0, st>>>(csq_buf(i), pg, (pg + 31) & ~31, b, p->max_rank, p->estimator, fixed ? 1 : 0, 0, i,
+                                      tr_est, ctrl);
       const VtwPlan vp = plan_vtw(h->sms, rows, n, ops->v_bn);
       mark(RRF_PHASE_VTW, i);
       ops->vtw(tmV_k, i == 0 ? tmA_k : tmW_k, Zpart, r0, r0, vp, ctrl, st);
@@ -1206,6 +1282,9 @@ rrf_status_t rrf_run(rrf_handle_t h, const rrf_params_t* p, void* dA, int64_t ld
     po.tree = tree;
     po.merge_t = true;
     po.bar_used = &bar_used;
+    std::vector<int> panel_g(steps + 1, 0);
+    po.g_out = &panel_g[0];
+    if (sampled) po.csq = csq_buf(0);
     s = launch_panel(h, p->dtype, Ybuf[0], src, m, b, Vblk(0), ldv, Tblk(0), p->max_rank, ps, ctrl, done_after, h->aux,
                      NoMark(), 0, po);
     if (s != RRF_OK) return panel_failed(s);
@@ -1248,6 +1327,8 @@ rrf_status_t rrf_run(rrf_handle_t h, const rrf_params_t* p, void* dA, int64_t ld
         pn.fix.Gpart = look_G;
         pn.fix.M = look_G + (size_t)kLookMaxCtas * b * b;
         if (gate) cudaStreamWaitEvent(h->aux, evZ(i), 0);
+        pn.g_out = &panel_g[i + 1];
+        if (sampled) pn.csq = csq_buf(i + 1);
         const rrf_status_t ls = launch_panel(h, p->dtype, Ybuf[(i + 1) & 1], sn, rows - b, b, Vblk(r0 + b), ldv,
                                              Tblk(r0 + b), p->max_rank, ps, ctrl, done_after + i, h->aux, NoMark(),
                                              i + 1, pn);
@@ -1263,6 +1344,9 @@ rrf_status_t rrf_run(rrf_handle_t h, const rrf_params_t* p, void* dA, int64_t ld
       }
       mark(RRF_PHASE_PANEL, i);                        // time the main stream waits for V_i, T_i
       cudaStreamWaitEvent(st, evP(i), 0);
+      if (sampled)                     // the sampled rule looks at panel i before block i is applied
+        est_kernel<<<1, 128, 0, st>>>(csq_buf(i), panel_g[i], (panel_g[i] + 31) & ~31, b, p->max_rank, p->estimator,
+                                      fixed ? 1 : 0, 0, i, tr_est, ctrl);
       const VtwPlan vp = plan_vtw(gate ? h->sms : gsms, rows, n, ops->v_bn);
       mark(RRF_PHASE_VTW, i);
       ops->vtw(tmV_k, i == 0 ? tmA_k : tmW_k, Zpart, r0, r0, vp, ctrl, st);
@@ -1401,7 +1485,10 @@ rrf_status_t rrf_run(rrf_handle_t h, const rrf_params_t* p, void* dA, int64_t ld
     const int lag = look_ctas > 0 ? 2 : 1;
     // without the predictor every executed pass that has a later panel to sample samples it
     out->fused_samples = predicting ? hc.fused_samples : std::min(hc.steps, std::max(0, steps - lag));
-    out->kernel_launches = 1 + (dOmegaT == nullptr ? 1 : 0) + 1 + ((look_ctas > 0 && steps > 1) ? 1 : 0) +
+    if (unchanged)
+      out->kernel_launches = (dOmegaT == nullptr ? 1 : 0) + 1 + 4 * steps + 3 * steps * (steps - 1) / 2;
+    else
+    out->kernel_launches = (sampled ? steps : 0) + 1 + (dOmegaT == nullptr ? 1 : 0) + 1 + ((look_ctas > 0 && steps > 1) ? 1 : 0) +
                            ((look_ctas > 0 || tree) ? 5 : 6) * steps +   // look-ahead, tree kernel: the panel kernel builds T itself
                            (predicting ? std::max(0, steps - lag) : 0);
   }
@@ -1411,6 +1498,9 @@ rrf_status_t rrf_run(rrf_handle_t h, const rrf_params_t* p, void* dA, int64_t ld
     if (h_E_sub_trace != nullptr) cudaMemcpy(h_E_sub_trace, tr_sub, sizeof(double) * hc.steps, cudaMemcpyDeviceToHost);
     if (h_E_dir_trace != nullptr) cudaMemcpy(h_E_dir_trace, tr_dir, sizeof(double) * hc.steps, cudaMemcpyDeviceToHost);
   }
+  out->n_est = hc.n_est;
+  if (hc.n_est > 0 && h_E_est_trace != nullptr)
+    cudaMemcpy(h_E_est_trace, tr_est, sizeof(double) * hc.n_est, cudaMemcpyDeviceToHost);
   return (rrf_status_t)hc.status;
 }
 

@@ -27,7 +27,11 @@ struct Ctrl {
   double r_prev;   // the history the sampling predictor extrapolates (negative: no ratio yet)
   int fused_samples;   // passes whose update also sampled a later panel
   int extra_samples;   // panels sampled by the separate kernel because the predictor had skipped them
+  int n_est;           // sampled stopping rules: panels whose estimate was evaluated
+  int pad2;
+  double E_est;        // sampled stopping rules: the last estimate
 };
+static_assert(sizeof(Ctrl) <= 256, "the control block has 256 bytes of workspace");
 
 // ~1 s at 2 GHz: every spin in this library gives up after this many SM clocks.
 constexpr long long kWaitLimitClocks = 2000000000LL;

@@ -210,7 +210,8 @@ __global__ void __launch_bounds__(kPanelThreads)
                  double* __restrict__ tau_out,       // [b]
                  unsigned* bar, Ctrl* ctrl, const int* done_flag, PanelFix fix,
                  unsigned bar_base,                 // value of the barrier counter when this launch starts
-                 T* __restrict__ Tout, long long ldt) {   // non-NULL: CTA 0 also builds the T factor at the end
+                 T* __restrict__ Tout, long long ldt,     // non-NULL: CTA 0 also builds the T factor at the end
+                 double* __restrict__ csq) {              // non-NULL: [b][Gp] per-CTA sums of squares of the panel's columns
   if (*reinterpret_cast<const volatile int*>(done_flag) || *reinterpret_cast<const volatile int*>(&ctrl->status) < 0) return;
   // the panel's entries were sampled by the fused update, or - where the predictor had skipped that - by
   // the separate sample kernel, in its layout
@@ -397,6 +398,20 @@ __global__ void __launch_bounds__(kPanelThreads)
       }
     }
     __syncthreads();
+  }
+
+  // Sums of squares of the columns of the panel as sampled (after the fix-up): the sampled stopping rules
+  // estimate the residual from them (est_kernel).  One warp per column, fixed order.
+  if (csq != nullptr) {
+    for (int c = warp; c < b; c += NW) {
+      double a = 0.0;
+      for (int r = lane; r < nloc; r += 32) {
+        const double v = (gr0 + r >= row0) ? S[(size_t)c * Rp + r] : 0.0;
+        a += v * v;
+      }
+      a = warp_sum(a);
+      if (lane == 0) csq[(size_t)c * Gp + cta] = a;
+    }
   }
 
   double tau_prev = 0.0;
@@ -686,6 +701,8 @@ __global__ void __launch_bounds__(256)
     ctrl->r_prev = -1.0;
     ctrl->fused_samples = 0;
     ctrl->extra_samples = 0;
+    ctrl->n_est = 0;
+    ctrl->E_est = 0.0;
     ctrl->steps = 0;
     ctrl->k = 0;
     ctrl->bar = 0;
@@ -737,7 +754,8 @@ __global__ void __launch_bounds__(256)
     ctrl->k = (i + 1) * b;
     if (reset_bar) ctrl->bar = 0;
     const double E = estimator == 0 ? trail : e_sub;
-    const bool below = !(E > ctrl->sigma2);
+    // the sampled rules (estimator >= 2) decide in est_kernel; here only the rank cap ends the loop
+    const bool below = estimator < 2 && !(E > ctrl->sigma2);
     const bool met = !fixed_rank && below;
     const bool cap = (i + 2) * b > max_rank;
     if (ctrl->status == RRF_OK && !below && cap) ctrl->status = RRF_MAX_RANK_REACHED;
@@ -765,6 +783,66 @@ __global__ void __launch_bounds__(256)
       ctrl->E_prev = E;
       ctrl->r_prev = r;
     }
+  }
+}
+
+// ------------------------------------------------------------------------------------------
+// Sampled stopping rules (the paper's outlook: criteria based on the spectral norm of the remaining part, and
+// a criterion for the variant that never updates A).  Panel i, Y_i = W Omega_i with Omega_i standard Gaussian,
+// probes the residual W left by the first i blocks:
+//   estimator 2:  E = ||Y_i||_F^2 / b            (E[E] = ||W||_F^2)
+//   estimator 3:  E = (200/pi) max_j ||y_j||^2   (||W||_2^2 <= E with probability 1 - 10^-b; Halko et al., Lemma 4.1)
+// from the per-CTA column sums of squares the panel kernel left in csq.  If E <= sigma^2 the loop ends with
+// k = i b (panel i is discarded).  advance != 0 (no update kernels in the loop): this kernel also counts the
+// block and applies the rank cap.
+// ------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(128)
+    est_kernel(const double* __restrict__ csq, int G, int Gp, int b, int max_rank, int estimator, int fixed_rank,
+               int advance, int step, double* __restrict__ tr_est, Ctrl* ctrl) {
+  if (*reinterpret_cast<volatile int*>(&ctrl->done)) return;
+  __shared__ double col[128];
+  const int c = threadIdx.x;
+  double s = 0.0;
+  if (c < b)
+    for (int x = 0; x < G; ++x) s += __ldcg(csq + (size_t)c * Gp + x);
+  col[c] = c < b ? s : 0.0;
+  __syncthreads();
+  if (c == 0) {
+    double E = 0.0;
+    if (estimator == 2) {
+      for (int j = 0; j < b; ++j) E += col[j];
+      E /= (double)b;
+    } else {
+      for (int j = 0; j < b; ++j) E = fmax(E, col[j]);
+      E *= 63.66197723675813;                     // 200 / pi
+    }
+    tr_est[step] = E;
+    ctrl->E_est = E;
+    ctrl->n_est = step + 1;
+    if (!fixed_rank && !(E > ctrl->sigma2)) {
+      ctrl->done = 1;
+    } else if (advance) {
+      ctrl->steps = step + 1;
+      ctrl->k = (step + 1) * b;
+      if ((step + 2) * b > max_rank) {
+        ctrl->done = 1;
+        if (ctrl->status == RRF_OK) ctrl->status = RRF_MAX_RANK_REACHED;
+      }
+    }
+  }
+}
+
+// dst (rows x b, dense) = sum of the nseg stacked partial panels the sample kernel wrote, in their fixed order
+template <typename T>
+__global__ void __launch_bounds__(256)
+    panel_sum_kernel(const T* __restrict__ Ypart, int nseg, long long seg_stride, long long rows, int b,
+                     T* __restrict__ dst, const Ctrl* ctrl) {
+  if (*reinterpret_cast<const volatile int*>(&ctrl->done)) return;
+  const long long total = rows * b;
+  for (long long idx = (long long)blockIdx.x * 256 + threadIdx.x; idx < total; idx += (long long)gridDim.x * 256) {
+    double s = (double)Ypart[idx];
+    for (int sg = 1; sg < nseg; ++sg) s += (double)Ypart[idx + (long long)sg * seg_stride];
+    dst[idx] = (T)s;
   }
 }
 

@@ -18,6 +18,7 @@ RRF_OK, RRF_MAX_RANK_REACHED = 0, 1
 RRF_ERR_INVALID_ARG, RRF_ERR_WORKSPACE, RRF_ERR_CUDA, RRF_ERR_TIMEOUT, RRF_ERR_NONFINITE = -1, -2, -3, -4, -5
 RRF_FLAG_INPLACE, RRF_FLAG_FIXED_RANK, RRF_FLAG_ONE_QUEUE, RRF_FLAG_TWO_QUEUES, RRF_FLAG_NO_GRAPH = 1, 2, 4, 8, 16
 RRF_FLAG_SAMPLE_ALWAYS, RRF_FLAG_SAMPLE_NEVER, RRF_FLAG_PANEL_TREE = 32, 64, 128
+RRF_FLAG_NO_UPDATE = 256
 
 _LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "librrf.so")
 _lib = None
@@ -33,7 +34,7 @@ class rrf_result_t(C.Structure):
     _fields_ = [("status", C.c_int32), ("k", C.c_int32), ("steps", C.c_int32), ("cuda_error", C.c_int32),
                 ("normA2", C.c_double), ("sigma2", C.c_double), ("E_sub", C.c_double), ("E_dir", C.c_double),
                 ("queues", C.c_int32), ("panel_ctas", C.c_int32), ("fused_samples", C.c_int32),
-                ("extra_samples", C.c_int32), ("kernel_launches", C.c_int32), ("reserved", C.c_int32)]
+                ("extra_samples", C.c_int32), ("kernel_launches", C.c_int32), ("n_est", C.c_int32)]
 
 
 RRF_PHASES = ["init", "sample", "panel", "tfactor", "vtw", "tz", "update", "stop", "skipped"]
@@ -62,7 +63,8 @@ def load():
     lib.rrf_destroy.argtypes = [vp]
     lib.rrf_workspace_bytes.argtypes = [C.POINTER(rrf_params_t), C.POINTER(sz)]
     lib.rrf_run.argtypes = [vp, C.POINTER(rrf_params_t), vp, i64, vp, i64, vp, i64, vp, vp, i64, vp, sz, vp,
-                            C.POINTER(rrf_result_t), C.POINTER(C.c_double), C.POINTER(C.c_double)]
+                            C.POINTER(rrf_result_t), C.POINTER(C.c_double), C.POINTER(C.c_double),
+                            C.POINTER(C.c_double)]
     lib.rrf_panel_workspace_bytes.argtypes = [i32, i64, i32, C.POINTER(sz)]
     lib.rrf_panel_qr.argtypes = [vp, i32, i64, i32, vp, i64, vp, i64, vp, i64, vp, sz, vp]
     lib.rrf_panel_qr_tree.argtypes = [vp, i32, i64, i32, vp, i64, vp, i64, vp, i64, vp, sz, vp]
@@ -171,6 +173,7 @@ class RunResult:
     fused_samples: int = 0
     extra_samples: int = 0
     kernel_launches: int = 0
+    E_est_trace: list = None   # estimators 2, 3: estimate of the residual before each sampled panel
 
 
 def rrf_run(h, A: torch.Tensor, b: int, tol: float, max_rank: int, omegaT: torch.Tensor | None = None,
@@ -191,7 +194,8 @@ def rrf_run(h, A: torch.Tensor, b: int, tol: float, max_rank: int, omegaT: torch
         V = _empty(m, max_rank, A.dtype, dev)
     if T is None:
         T = torch.empty((b, max_rank), dtype=A.dtype, device=dev)   # leading dimension max_rank
-    if B is None:
+    no_update = bool(flags & RRF_FLAG_NO_UPDATE)
+    if B is None and not no_update:
         B = _empty(max_rank, n, A.dtype, dev)
     if workspace is None:
         workspace = torch.empty(need.value, dtype=torch.uint8, device=dev)
@@ -199,16 +203,17 @@ def rrf_run(h, A: torch.Tensor, b: int, tol: float, max_rank: int, omegaT: torch
     steps = max_rank // b
     tr_sub = (C.c_double * steps)()
     tr_dir = (C.c_double * steps)()
+    tr_est = (C.c_double * (steps + 1))()
     om_ptr, ldo = (None, 0) if omegaT is None else (C.c_void_p(omegaT.data_ptr()), _rowmajor(omegaT, "omegaT"))
     s = lib.rrf_run(h, C.byref(p), C.c_void_p(A.data_ptr()), _rowmajor(A, "A"), om_ptr, ldo,
                     C.c_void_p(V.data_ptr()), _rowmajor(V, "V"), C.c_void_p(T.data_ptr()),
-                    C.c_void_p(B.data_ptr()), _rowmajor(B, "B"), C.c_void_p(workspace.data_ptr()),
-                    workspace.numel(), _stream(), C.byref(res), tr_sub, tr_dir)
+                    None if B is None else C.c_void_p(B.data_ptr()), 0 if B is None else _rowmajor(B, "B"),
+                    C.c_void_p(workspace.data_ptr()), workspace.numel(), _stream(), C.byref(res), tr_sub, tr_dir, tr_est)
     if check and s < 0:
         raise RrfError(s, "rrf_run")
     return RunResult(res.status, res.k, res.steps, res.normA2, res.sigma2, res.E_sub, res.E_dir,
                      list(tr_sub)[:res.steps], list(tr_dir)[:res.steps], V, T, B, res.queues, res.panel_ctas,
-                     res.fused_samples, res.extra_samples, res.kernel_launches)
+                     res.fused_samples, res.extra_samples, res.kernel_launches, list(tr_est)[:res.n_est])
 
 
 def rrf_panel_qr(h, Y: torch.Tensor, tree: bool = False):

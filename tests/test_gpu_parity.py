@@ -17,6 +17,7 @@ from philox_ref import omega_reference as _omega_reference
 pytestmark = pytest.mark.gpu
 
 TOL = {"f64": dict(rel=1e-10, orth=1e-12), "f32": dict(rel=1e-4, orth=1e-5)}
+ESTIMATORS = ["direct", "subtractive", "sampled_fro", "sampled_spectral"]
 
 
 @pytest.fixture(scope="module")
@@ -50,8 +51,7 @@ def run_both(h, w, estimator=0, flags=0, A=None, Om=None):
     dA = _pad_cols(A, mult)
     dOmT = _pad_cols(np.ascontiguousarray(Om_t.T), mult)
     g = rrf.rrf_run(h, dA, w.b, w.tol, w.max_rank, omegaT=dOmT, estimator=estimator, flags=flags)
-    o = orc.rrf(A.astype(np.float64), Om_t.astype(np.float64), w.b, w.tol, w.max_rank,
-                estimator="direct" if estimator == 0 else "subtractive")
+    o = orc.rrf(A.astype(np.float64), Om_t.astype(np.float64), w.b, w.tol, w.max_rank, estimator=ESTIMATORS[estimator])
     return g, o, A, Om_t
 
 
@@ -61,7 +61,7 @@ def relmax(x, ref):
     return d / s if s > 0 else d
 
 
-def check_run(h, w, g, o, A, Om, q_envelope=True):
+def check_run(h, w, g, o, A, Om, q_envelope=True, estimator="direct"):
     tol = TOL[w.dtype]
     assert g.k == o.k and g.steps == o.steps and g.status == o.status, (g.k, o.k, g.status, o.status)
     k, b = g.k, w.b
@@ -77,10 +77,10 @@ def check_run(h, w, g, o, A, Om, q_envelope=True):
     # and rows of Omega permuted; float32: the same steps in plain float32 on the CPU).
     op = None
     if q_envelope and w.dtype == "f64":
-        op = orc.permuted_rerun(A64, Om.astype(np.float64), b, w.tol, w.max_rank, seed=1)
+        op = orc.permuted_rerun(A64, Om.astype(np.float64), b, w.tol, w.max_rank, seed=1, estimator=estimator)
         assert op.k == o.k
     elif q_envelope:
-        op = orc.rrf(A, Om, b, w.tol, w.max_rank, dtype=np.float32)
+        op = orc.rrf(A, Om, b, w.tol, w.max_rank, dtype=np.float32, estimator=estimator)
         if op.k != o.k:
             op = None
     # Stopping quantities after every block: 1e-9 relative, plus what the oracle's own trace moves under
@@ -325,6 +325,70 @@ def test_whole_runs_with_the_tree_panel_kernel(h, name, kw, sched):
     g, o, A, Om = run_both(h, w, flags=sched | rrf.RRF_FLAG_PANEL_TREE)
     assert g.queues == (2 if sched == rrf.RRF_FLAG_TWO_QUEUES else 1)
     check_run(h, w, g, o, A, Om)
+
+
+@pytest.mark.parametrize("sched", SCHEDULES)
+@pytest.mark.parametrize("estimator", [2, 3])
+@pytest.mark.parametrize("name,kw,tol", [("cfg2", dict(m=1536, n=1280, max_rank=512), 3e-3),
+                                         ("cfg1", dict(m=900, n=700, max_rank=256), 1e-3),
+                                         ("cfg4b", dict(m=1024, n=2752, max_rank=256, rank=64), 1e-2)])
+def test_sampled_stopping_rules_match_the_oracle(h, name, kw, tol, estimator, sched):
+    # the rules that look at the sampled panel instead of B or the updated matrix: same k, same estimates
+    w = wl.CONFIGS[name].scaled(**kw)
+    w = w.__class__(**{**w.__dict__, "tol": tol})
+    g, o, A, Om = run_both(h, w, estimator=estimator, flags=sched)
+    assert len(g.E_est_trace) == len(o.E_est) and g.status == o.status
+    rt = 1e-9 if w.dtype == "f64" else 1e-4
+    assert np.allclose(g.E_est_trace, o.E_est, rtol=rt, atol=rt * 1e-6 * o.normA2), (g.E_est_trace, o.E_est)
+    if estimator == 2 or name != "cfg4b":
+        assert 0 < g.k < w.max_rank and g.status == rrf.RRF_OK
+    check_run(h, w, g, o, A, Om, estimator=ESTIMATORS[estimator])
+
+
+@pytest.mark.parametrize("name,kw,tol", [("cfg2", dict(m=1536, n=1280, max_rank=512), 3e-3),
+                                         ("cfg1", dict(m=900, n=700, max_rank=256), 1e-3),
+                                         ("cfg5", dict(m=2048, n=1024, max_rank=512, rank=384), 1e-4),
+                                         ("cfg4b", dict(m=1024, n=2752, max_rank=256, rank=64), 1e-2)])
+def test_variant_that_leaves_a_unchanged(h, name, kw, tol):
+    # no update of A, no B: panels are sampled from A and pulled through the reflectors found so far
+    w = wl.CONFIGS[name].scaled(**kw)
+    A, _ = wl.make_matrix(w)
+    Om = wl.make_omega(w).astype(w.np_dtype)
+    dA = torch.from_numpy(A).cuda()
+    keep = dA.clone()
+    dOmT = torch.from_numpy(np.ascontiguousarray(Om.T)).cuda()
+    g = rrf.rrf_run(h, dA, w.b, tol, w.max_rank, omegaT=dOmT, estimator=2, flags=rrf.RRF_FLAG_NO_UPDATE)
+    o = orc.rrf(A.astype(np.float64), Om.astype(np.float64), w.b, tol, w.max_rank, estimator="sampled_fro",
+                schedule="a_unchanged")
+    oi = orc.rrf(A.astype(np.float64), Om.astype(np.float64), w.b, tol, w.max_rank, estimator="sampled_fro")
+    assert torch.equal(dA, keep) and g.B is None
+    assert (g.k, g.steps, g.status) == (o.k, o.steps, o.status) and 0 < g.k < w.max_rank
+    rt = 1e-9 if w.dtype == "f64" else 1e-4
+    assert np.allclose(g.E_est_trace, o.E_est, rtol=rt, atol=rt * 1e-6 * o.normA2)
+    k, b = g.k, w.b
+    Qg = rrf.rrf_form_q(h, g.V, g.T, b, k).cpu().numpy().astype(np.float64)
+    Qo = orc.form_q(o.V, o.T, b)
+    tl = TOL[w.dtype]
+    assert np.linalg.norm(Qg.T @ Qg - np.eye(k)) <= tl["orth"]
+    A64 = A.astype(np.float64)
+    # the projection is what a user of this variant gets: Q Q^T A against the oracle's, and the residual it leaves
+    assert relmax(Qg @ (Qg.T @ A64), Qo @ (Qo.T @ A64)) <= 10 * tl["rel"]
+    assert np.linalg.norm(A64 - Qg @ (Qg.T @ A64)) <= tol * np.sqrt(o.normA2) * 3.0
+    prev = [oi.normA2] + oi.E_dir
+    for i in range(k // b):
+        blk = slice(i * b, (i + 1) * b)
+        d = np.max(np.abs(Qg[:, blk] - Qo[:, blk])) / np.max(np.abs(Qo))
+        rho = np.sqrt(prev[i] / oi.normA2)
+        assert d <= tl["rel"] or d * rho <= tl["rel"], (i, d, rho)
+    # fixed-rank mode of the same variant
+    gf = rrf.rrf_run(h, dA, w.b, tol, w.max_rank, omegaT=dOmT, flags=rrf.RRF_FLAG_NO_UPDATE | rrf.RRF_FLAG_FIXED_RANK)
+    of = orc.rrf(A.astype(np.float64), Om.astype(np.float64), w.b, tol, w.max_rank, schedule="a_unchanged",
+                 fixed_rank=True, estimator="sampled_fro")
+    assert gf.k == of.k == w.max_rank and gf.status == of.status
+    Qf = rrf.rrf_form_q(h, gf.V, gf.T, b, gf.k).cpu().numpy().astype(np.float64)
+    assert np.linalg.norm(Qf.T @ Qf - np.eye(gf.k)) <= tl["orth"]
+    Qof = orc.form_q(of.V, of.T, b)
+    assert relmax(Qf @ (Qf.T @ A64), Qof @ (Qof.T @ A64)) <= 10 * tl["rel"]
 
 
 def test_schedules_agree_and_stop_mid_way(h):
