@@ -186,10 +186,10 @@ def run_reference(args, w, rank, world):
 class Problem:
     """One workload resident on the device: inputs, outputs and workspace of rrf_run."""
 
-    def __init__(self, h, w, dev, sched):
+    def __init__(self, h, w, dev, sched, estimator=0):
         import torch
         from paper_2608_28941_b200 import rrf
-        self.h, self.w, self.dev, self.sched = h, w, dev, sched
+        self.h, self.w, self.dev, self.sched, self.estimator = h, w, dev, sched, estimator
         self.A, self.Om, self.OmT = generate(w, dev)
         self.tdt, self.esize = self.A.dtype, self.A.element_size()
         p = rrf.make_params(rrf.RRF_F64 if w.dtype == "f64" else rrf.RRF_F32, w.m, w.n, w.b, w.tol, w.max_rank)
@@ -203,7 +203,7 @@ class Problem:
         w = self.w
         om = self.OmT if isinstance(omegaT, str) else omegaT
         return rrf.rrf_run(self.h, self.A if A is None else A, w.b, w.tol, w.max_rank, omegaT=om, V=self.V, T=self.T,
-                           B=self.B, workspace=self.ws, flags=self.sched | flags, seed=w.seed)
+                           B=self.B, workspace=self.ws, flags=self.sched | flags, seed=w.seed, estimator=self.estimator)
 
 
 def time_problem(pb, steps, warmup, world, barrier):
@@ -373,6 +373,10 @@ def main():
     ap.add_argument("--schedule", default="auto", choices=["auto", "one", "two"],
                     help="one queue (sequential), two queues (look-ahead), or the library's own rule")
     ap.add_argument("--panel", default="column", choices=["column", "tree"], help="panel kernel (b <= 64)")
+    ap.add_argument("--variant", default="in-place", choices=["in-place", "no-update"],
+                    help="no-update: A is left unchanged and B is not formed (one pass over A per block instead of "
+                         "three); stops on the sampled Frobenius estimate.  Flops are counted as the in-place schedule's")
+    ap.add_argument("--estimator", type=int, default=0, choices=[0, 1, 2, 3])
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
 
@@ -415,8 +419,14 @@ def main():
             dist.barrier()
             torch.cuda.synchronize()
 
+    estimator = args.estimator
+    if args.variant == "no-update":
+        sched = rrf.RRF_FLAG_NO_UPDATE
+        estimator = estimator if estimator >= 2 else 2
+        args.no_e2e = True
+        args.no_per_config = True
     peaks = measured_peaks()
-    pb = Problem(h, w, dev, sched)
+    pb = Problem(h, w, dev, sched, estimator)
     sampler = ClockSampler(local)
     pb.step()
     barrier()
@@ -478,6 +488,8 @@ def main():
                            "k": res.k, "block_steps": res.steps, "status": res.status,
                            "l2": "inputs larger than L2 (A is %.0f MB)" % (w.m * w.n * esize / 1e6),
                            "queues": res.queues, "panel_ctas": res.panel_ctas, "panel_kernel": args.panel,
+                           "variant": args.variant, "estimator": estimator,
+                           "passes_over_A_per_block": 1 if args.variant == "no-update" else 3,
                            "fused_samples": res.fused_samples, "extra_samples": res.extra_samples,
                            "parallelism": "replicas only" if world > 1 else "single GPU"},
                 "clocks": clocks, "e2e": e2e, "gpu_launches": launches,

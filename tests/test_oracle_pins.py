@@ -391,3 +391,25 @@ def test_schedule_that_leaves_a_unchanged_gives_the_same_reflectors():
     u = orc.rrf(A, Om, b, 5e-2, max_rank, estimator="sampled_fro", schedule="a_unchanged")
     assert 0 < a.k < max_rank and a.k == u.k and a.status == u.status == orc.RRF_OK
     assert np.allclose(a.E_est, u.E_est, rtol=1e-9)
+
+
+def test_foil_on_the_stability_stress_configuration():
+    """The third configuration's recipe (fifteen decades of singular values, then a 1e-16 floor) at 1024 x 1024 in
+    double precision, b = 32: the regime where block Gram-Schmidt without reorthogonalisation loses orthogonality
+    while the Householder range finder keeps it at round-off."""
+    from oracle import bcgs_foil
+    w = wl.CONFIGS["cfg3"].scaled(m=1024, n=1024, max_rank=384)
+    A, _ = wl.make_matrix(w)
+    Om = wl.make_omega(w)
+    passes = w.max_rank // w.b
+    Q_plain, _, _ = bcgs_foil.bcgs_range_finder(A, Om, w.b, passes, reorth=False, dtype=np.float64)
+    Q_re, _, _ = bcgs_foil.bcgs_range_finder(A, Om, w.b, passes, reorth=True, dtype=np.float64)
+    hh = orc.rrf(A, Om, w.b, 0.0, w.max_rank)
+    Q_hh = orc.form_q(hh.V, hh.T, w.b)
+
+    def loss(Q):
+        return np.linalg.norm(Q.T @ Q - np.eye(Q.shape[1]))
+
+    assert loss(Q_hh) < 1e-13                       # the bar the GPU path is held to is 1e-12
+    assert loss(Q_re) < 1e-12
+    assert loss(Q_plain) > 1e-6                     # orthogonality lost by ten orders of magnitude
