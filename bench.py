@@ -372,7 +372,8 @@ def main():
     ap.add_argument("--no-per-config", action="store_true", help="skip the short runs of the other four configurations")
     ap.add_argument("--schedule", default="auto", choices=["auto", "one", "two"],
                     help="one queue (sequential), two queues (look-ahead), or the library's own rule")
-    ap.add_argument("--panel", default="column", choices=["column", "tree"], help="panel kernel (b <= 64)")
+    ap.add_argument("--panel", default="column", choices=["column", "blocked", "tree"],
+                    help="panel kernel: column by column (default), blocked in micro-panels of eight, or the tree kernel (b <= 64)")
     ap.add_argument("--variant", default="in-place", choices=["in-place", "no-update"],
                     help="no-update: A is left unchanged and B is not formed (one pass over A per block instead of "
                          "three); stops on the sampled Frobenius estimate.  Flops are counted as the in-place schedule's")
@@ -412,6 +413,8 @@ def main():
     sched = {"auto": 0, "one": rrf.RRF_FLAG_ONE_QUEUE, "two": rrf.RRF_FLAG_TWO_QUEUES}[args.schedule]
     if args.panel == "tree":
         sched |= rrf.RRF_FLAG_PANEL_TREE
+    if args.panel == "blocked":
+        sched |= rrf.RRF_FLAG_PANEL_BLOCKED
 
     def barrier():
         torch.cuda.synchronize()

@@ -62,6 +62,8 @@ typedef enum {
                                     the kernel that pays one grid barrier per column.  Off by default: it is the
                                     slower of the two on the sizes measured so far.  The look-ahead schedule is
                                     then used only if RRF_FLAG_TWO_QUEUES asks for it */
+#define RRF_FLAG_PANEL_BLOCKED 512u /* factor the panels with the blocked kernel (see rrf_panel_qr_blocked) where it
+                                      fits.  Off by default: slower than the column-by-column kernel in whole runs */
 #define RRF_FLAG_NO_UPDATE 256u /* the variant of the paper's outlook that leaves A unchanged and returns no B: each
                                   panel is sampled from A itself and pulled through the reflector blocks found so
                                   far.  One pass over A per block instead of three.  Needs estimator 2 or 3, or
@@ -188,6 +190,16 @@ rrf_status_t rrf_panel_qr(rrf_handle_t h, int32_t dtype, int64_t rows, int32_t b
                           const void* dY, int64_t ldy, void* dV, int64_t ldv,
                           void* dT, int64_t ldt,
                           void* d_workspace, size_t workspace_bytes, void* cuda_stream);
+
+/* rrf_panel_qr_blocked - the same call with the blocked kernel: the columns are factored in micro-panels of eight
+ * (a column step touches eight columns of the slab instead of all b), each finished micro-panel is applied to the
+ * rest of the panel as a block reflector on the FP64 tensor cores, and the CTAs exchange their partial sums through
+ * flagged words in global memory instead of a grid barrier followed by a read.  Same V and T up to rounding.  Falls
+ * back to the column-by-column kernel when the slab and its small matrices do not fit in shared memory. */
+rrf_status_t rrf_panel_qr_blocked(rrf_handle_t h, int32_t dtype, int64_t rows, int32_t b,
+                                  const void* dY, int64_t ldy, void* dV, int64_t ldv,
+                                  void* dT, int64_t ldt,
+                                  void* d_workspace, size_t workspace_bytes, void* cuda_stream);
 
 /*
  * rrf_panel_qr_tree - the same factorisation (Algorithm 2 line 7) by another route, for b <= 64: a tall-skinny QR

@@ -10,7 +10,7 @@
 #include <vector>
 
 #include "gemm_sk.cuh"
-#include "panel_tsqr.cuh"
+#include "panel_blk.cuh"
 
 namespace rrf {
 
@@ -32,6 +32,7 @@ struct rrf_ctx {
   int last_cuda;
   int panel_smem_max;    // dynamic shared memory the panel kernel may use (opt-in limit minus its static part)
   int tsqr_smem_max;     // the same for the tree panel kernel
+  int blk_smem_max;      // the same for the blocked panel kernel
   int profiling;
   cudaStream_t aux;                      // side stream: the T factor is built while V^T W runs
   std::vector<cudaEvent_t> sync_events;  // fork/join events between the caller's stream and `aux`
@@ -209,6 +210,39 @@ static bool plan_tree(const rrf_ctx* h, long long rows, int b, int max_ctas, boo
   }
   return found;
 }
+// Plan of the blocked panel kernel (panel_blk.cuh): slab height per CTA and which of its small matrices fit in
+// shared memory beside the slab.
+struct BlkPlan { int G, R, RS, Rp, ksplit, c_in_smem; size_t smem; };
+static bool plan_blk(const rrf_ctx* h, long long rows, int b, BlkPlan* p, int ctas = 0, bool fix = false) {
+  if (fix && b > 64) return false;
+  const long long ext = rows + (fix ? b : 0);
+  const size_t small = 16 + 8 + 8 + 8 + 64 + 64 + 8 + 8;
+  const size_t fixd = fix ? (size_t)panel_fix_doubles(b) : 0;
+  int R = std::max(64, ceil_div(ext, ctas > 0 ? ctas : h->sms));
+  if (ctas == 0) {
+    // Every column costs one exchange among all CTAs, whose latency grows with their number, while the pass
+    // over a slab is cheap: prefer few tall slabs (up to 320 rows) where shared memory allows.
+    const size_t room = (size_t)h->blk_smem_max / sizeof(double) - std::max(fixd, (size_t)kBlkDw) - (size_t)kMB * (b + 8) - small;
+    const int tall = std::min(320, (int)(room / b - 1) / 16 * 16);
+    if (tall > R) R = tall;
+  }
+  p->R = R;
+  p->G = ceil_div(ext, R);
+  if (p->G > h->sms) return false;
+  p->RS = (R + 15) / 16 * 16;
+  // roomy: odd pitch, D partials of the K-split warps and C staged in shared memory
+  p->ksplit = std::max(1, 16 / (b / 16));
+  p->c_in_smem = 1;
+  p->Rp = p->RS + 1;
+  p->smem = ((size_t)b * p->Rp + std::max(fixd, p->ksplit > 1 ? (size_t)kBlkDw : 0) + (size_t)kMB * (b + 8) + small) * sizeof(double);
+  if (p->smem <= (size_t)h->blk_smem_max) return true;
+  // tight: nothing but the slab (and the fix-up staging)
+  p->ksplit = 1;
+  p->c_in_smem = 0;
+  p->Rp = p->RS;
+  p->smem = ((size_t)b * p->Rp + fixd + small) * sizeof(double);
+  return p->smem <= (size_t)h->blk_smem_max;
+}
 // Fewest CTAs whose shared memory holds a rows x b panel with the fix-up staging; 0 if none.
 static int panel_min_ctas(const rrf_ctx* h, long long rows, int b) {
   if (b > 64) return 0;
@@ -228,7 +262,18 @@ static size_t tsqr_scratch_bytes(int sms, int b) {
   // Rbuf, Xbuf, Kbuf [CTA][b*b] + Ubuf [2][b*b]
   return b <= kTsqrMaxB ? align_up(((size_t)3 * sms + 2) * b * b * sizeof(double), 256) : 0;
 }
-static size_t panel_scratch_bytes(int sms, int b) { return direct_scratch_bytes(sms, b) + tsqr_scratch_bytes(sms, b); }
+// blocked panel kernel: exchange lines, per-CTA partials, reduced block, and three tag arrays (zeroed before use)
+// zeroed before use: the flagged words of the exchanges, Lw [2][16][Gp][2], Pw [8 b][Gp][2], Rw [16 b][2]
+static size_t blk_tag_bytes(int sms, int b) {
+  const size_t gp = (size_t)(sms + 31) / 32 * 32;
+  return align_up(((size_t)2 * 16 * gp * 2 + (size_t)kMB * b * gp * 2 + (size_t)16 * b * 2) * sizeof(unsigned long long), 256);
+}
+static size_t blk_scratch_bytes(int sms, int b) {
+  return blk_tag_bytes(sms, b) + align_up((size_t)sms * kMB * b * sizeof(double), 256);
+}
+static size_t panel_scratch_bytes(int sms, int b) {
+  return direct_scratch_bytes(sms, b) + tsqr_scratch_bytes(sms, b) + blk_scratch_bytes(sms, b);
+}
 constexpr int kLookMaxCtas = 48;   // most CTAs a confined panel may take
 // Rough cost model of one pass, in microseconds, used only to choose the schedule (fitted to event
 // timings on a B200; the look-ahead is right or wrong by its measured time, not by this model).
@@ -255,7 +300,7 @@ struct PassModel {
 static size_t look_scratch_bytes(int b) {   // Gpart[kLookMaxCtas][b*b] + M[b*b]
   return align_up((size_t)(kLookMaxCtas + 1) * b * b * sizeof(double), 256);
 }
-struct PanelScratch { double *P, *piv, *gram, *tau; unsigned* bar; TsqrScratch ts; };
+struct PanelScratch { double *P, *piv, *gram, *tau; unsigned* bar; TsqrScratch ts; BlkScratch bk; unsigned* blk_tags; size_t blk_tag_bytes; };
 // `sms`: the SM count the buffers were sized for (the handle's bound kMaxSms for caller workspaces)
 static PanelScratch carve_panel(unsigned char* base, int sms, int b, bool with_tree = true) {
   PanelScratch s;
@@ -265,10 +310,23 @@ static PanelScratch carve_panel(unsigned char* base, int sms, int b, bool with_t
   s.tau = s.gram + (size_t)b * b;
   s.bar = reinterpret_cast<unsigned*>(s.tau + b);
   s.ts = TsqrScratch{nullptr, nullptr, nullptr, nullptr};
+  s.bk = BlkScratch{nullptr, nullptr, nullptr, nullptr};
+  s.blk_tags = nullptr;
+  s.blk_tag_bytes = 0;
   if (with_tree && b <= kTsqrMaxB) {
     double* t = reinterpret_cast<double*>(base + direct_scratch_bytes(sms, b));
     const size_t blk = (size_t)sms * b * b;
     s.ts = TsqrScratch{t, t + blk, t + 2 * blk, t + 3 * blk};
+  }
+  if (with_tree) {
+    unsigned char* q = base + direct_scratch_bytes(sms, b) + tsqr_scratch_bytes(sms, b);
+    const size_t gp = (size_t)(sms + 31) / 32 * 32;
+    s.blk_tags = reinterpret_cast<unsigned*>(q);
+    s.blk_tag_bytes = blk_tag_bytes(sms, b);
+    s.bk.Lw = reinterpret_cast<unsigned long long*>(q);
+    s.bk.Pw = s.bk.Lw + (size_t)2 * 16 * gp * 2;
+    s.bk.Rw = s.bk.Pw + (size_t)kMB * b * gp * 2;
+    s.bk.Cg = reinterpret_cast<double*>(q + blk_tag_bytes(sms, b));
   }
   return s;
 }
@@ -418,6 +476,8 @@ struct PanelOpts {
   cudaStream_t st_t = nullptr;     // side stream for the T factor, with its fork / join events
   cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
   bool tree = false;               // b <= 64: use the tree kernel (no grid barrier per column)
+  bool blocked = false;            // use the blocked kernel (micro-panels of eight columns, panel_blk.cuh) if it fits
+  unsigned seq_base = 0;           // blocked kernel: first tag value of this launch (tags only grow within a run)
   double* csq = nullptr;           // [b][Gp]: the panel kernel leaves the column sums of squares of the panel here
   int* g_out = nullptr;            // out: CTAs of the per-column panel kernel (Gp = g rounded up to 32)
 };
@@ -451,9 +511,7 @@ static rrf_status_t launch_panel(rrf_ctx* h, int dtype, const void* Y, PanelSour
     if (o.ev_join != nullptr) cudaEventRecord(o.ev_join, st);   // T is ready when the panel kernel is
     return RRF_OK;
   }
-  PanelPlan pp;
-  if (!plan_panel(h, rows, b, &pp, o.ctas, o.fix.enabled != 0)) return RRF_ERR_WORKSPACE;
-  int rows_i = (int)rows, R = pp.R, Rp = pp.Rp;
+  int rows_i = (int)rows;
   double *P = ps.P, *piv = ps.piv, *gram = ps.gram, *tau = ps.tau;
   unsigned* bar = ps.bar;
   PanelFix fix = o.fix;
@@ -462,15 +520,36 @@ static rrf_status_t launch_panel(rrf_ctx* h, int dtype, const void* Y, PanelSour
   unsigned bar_base = o.bar_base;
   void* Tmerged = o.merge_t ? Tout : nullptr;
   double* csq = o.csq;
-  void* args[] = {&Y,   &src, &alt, &fused_flag, &rows_i, &b,    &R,    &Rp,        &V,   &ldv,      &P,
-                  &piv, &gram, &tau, &bar,       &ctrl,   &done_flag, &fix, &bar_base, &Tmerged, &ldt, &csq};
   const size_t tsmem = ((size_t)b * (b + 1) + (size_t)(b / 2) * (b / 2 + 1)) * sizeof(double);
-  if (o.merge_t) pp.smem = std::max(pp.smem, tsmem);
-  if (o.bar_used != nullptr) *o.bar_used = (unsigned)(b + (o.fix.enabled ? 2 : 0)) * (unsigned)pp.G;
-  if (o.g_out != nullptr) *o.g_out = pp.G;
-  mark(RRF_PHASE_PANEL, step);
-  const void* fn = dtype == RRF_F64 ? panel_variant<double>(pp.variant) : panel_variant<float>(pp.variant);
-  cudaError_t e = cudaLaunchCooperativeKernel(fn, dim3(pp.G), dim3(kPanelThreads), args, pp.smem, st);
+  cudaError_t e;
+  BlkPlan bp;
+  if (o.blocked && ps.bk.Lw != nullptr && plan_blk(h, rows, b, &bp, o.ctas, o.fix.enabled != 0)) {
+    // blocked kernel: micro-panels of eight columns, exchanges instead of grid barriers
+    int R = bp.R, Rp = bp.Rp, RS = bp.RS, ksplit = bp.ksplit, c_in_smem = bp.c_in_smem;
+    BlkScratch bk = ps.bk;
+    unsigned seq_base = o.seq_base;
+    void* args[] = {&Y, &src, &alt, &fused_flag, &rows_i, &b, &R, &Rp, &RS, &V, &ldv, &gram, &tau, &bk, &seq_base,
+                    &ksplit, &c_in_smem, &bar, &ctrl, &done_flag, &fix, &bar_base, &Tmerged, &ldt, &csq};
+    size_t smem = bp.smem;
+    if (o.merge_t) smem = std::max(smem, tsmem);
+    if (o.bar_used != nullptr) *o.bar_used = (unsigned)(o.fix.enabled ? 2 : 0) * (unsigned)bp.G;
+    if (o.g_out != nullptr) *o.g_out = bp.G;
+    mark(RRF_PHASE_PANEL, step);
+    const void* fn = dtype == RRF_F64 ? (const void*)panel_blk_kernel<double> : (const void*)panel_blk_kernel<float>;
+    e = cudaLaunchCooperativeKernel(fn, dim3(bp.G), dim3(kPanelThreads), args, smem, st);
+  } else {
+    PanelPlan pp;
+    if (!plan_panel(h, rows, b, &pp, o.ctas, o.fix.enabled != 0)) return RRF_ERR_WORKSPACE;
+    int R = pp.R, Rp = pp.Rp;
+    void* args[] = {&Y,   &src, &alt, &fused_flag, &rows_i, &b,    &R,    &Rp,        &V,   &ldv,      &P,
+                    &piv, &gram, &tau, &bar,       &ctrl,   &done_flag, &fix, &bar_base, &Tmerged, &ldt, &csq};
+    if (o.merge_t) pp.smem = std::max(pp.smem, tsmem);
+    if (o.bar_used != nullptr) *o.bar_used = (unsigned)(b + (o.fix.enabled ? 2 : 0)) * (unsigned)pp.G;
+    if (o.g_out != nullptr) *o.g_out = pp.G;
+    mark(RRF_PHASE_PANEL, step);
+    const void* fn = dtype == RRF_F64 ? panel_variant<double>(pp.variant) : panel_variant<float>(pp.variant);
+    e = cudaLaunchCooperativeKernel(fn, dim3(pp.G), dim3(kPanelThreads), args, pp.smem, st);
+  }
   if (e == cudaSuccess && !o.merge_t) {
     cudaStream_t tt = st;
     if (o.ev_fork != nullptr) {          // fork: the T factor runs on the side stream after the panel
@@ -532,6 +611,23 @@ static cudaError_t setup_tree_kernels(int smem_optin, int* tsqr_smem_max) {
   *tsqr_smem_max = std::min(smem_optin, kMaxSmem) - (int)stat;
   for (const void* f : fk) {
     const cudaError_t e = cudaFuncSetAttribute(f, cudaFuncAttributeMaxDynamicSharedMemorySize, *tsqr_smem_max);
+    if (e != cudaSuccess) return e;
+  }
+  return cudaSuccess;
+}
+
+static cudaError_t setup_blk_kernels(int smem_optin, int* blk_smem_max) {
+  const void* fk[2] = {(const void*)panel_blk_kernel<double>, (const void*)panel_blk_kernel<float>};
+  size_t stat = 0;
+  for (const void* f : fk) {
+    cudaFuncAttributes fa;
+    const cudaError_t e = cudaFuncGetAttributes(&fa, f);
+    if (e != cudaSuccess) return e;
+    stat = std::max(stat, fa.sharedSizeBytes);
+  }
+  *blk_smem_max = std::min(smem_optin, kMaxSmem) - (int)stat;
+  for (const void* f : fk) {
+    const cudaError_t e = cudaFuncSetAttribute(f, cudaFuncAttributeMaxDynamicSharedMemorySize, *blk_smem_max);
     if (e != cudaSuccess) return e;
   }
   return cudaSuccess;
@@ -661,6 +757,7 @@ rrf_status_t rrf_create(rrf_handle_t* out, int device) {
   h->encode = reinterpret_cast<EncodeTiledFn>(fn);
   if (e == cudaSuccess) e = setup_all(h->smem_optin, &h->panel_smem_max);
   if (e == cudaSuccess) e = setup_tree_kernels(h->smem_optin, &h->tsqr_smem_max);
+  if (e == cudaSuccess) e = setup_blk_kernels(h->smem_optin, &h->blk_smem_max);
   if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&h->aux, cudaStreamNonBlocking);
   if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&h->cap, cudaStreamNonBlocking);
   if (e == cudaSuccess) e = cudaMalloc(&h->d_ctrl, sizeof(Ctrl));
@@ -786,7 +883,7 @@ rrf_status_t rrf_panel_workspace_bytes(int32_t dtype, int64_t rows, int32_t b, s
 
 static rrf_status_t panel_qr_entry(rrf_handle_t h, int32_t dtype, int64_t rows, int32_t b, const void* dY, int64_t ldy,
                                    void* dV, int64_t ldv, void* dT, int64_t ldt, void* d_workspace,
-                                   size_t workspace_bytes, void* cuda_stream, bool tree) {
+                                   size_t workspace_bytes, void* cuda_stream, bool tree, bool blocked = false) {
   if (h == nullptr || dY == nullptr || dV == nullptr || dT == nullptr || d_workspace == nullptr)
     return RRF_ERR_INVALID_ARG;
   if (!b_ok(dtype, b) || rows < b || rows > 0x7fffffffLL || ldy < b || ldv < b || ldt < b || ldy > 0x7fffffffLL)
@@ -796,6 +893,7 @@ static rrf_status_t panel_qr_entry(rrf_handle_t h, int32_t dtype, int64_t rows, 
   cudaStream_t st = (cudaStream_t)cuda_stream;
   PanelScratch ps = carve_panel((unsigned char*)d_workspace, h->sms, b);
   if (cudaMemsetAsync(ps.bar, 0, sizeof(unsigned), st) != cudaSuccess) return RRF_ERR_CUDA;
+  if (cudaMemsetAsync(ps.blk_tags, 0, ps.blk_tag_bytes, st) != cudaSuccess) return RRF_ERR_CUDA;
   PanelSource src{};
   src.slots = 0;
   src.nseg = 1;
@@ -803,6 +901,7 @@ static rrf_status_t panel_qr_entry(rrf_handle_t h, int32_t dtype, int64_t rows, 
   src.ldy = (int)ldy;
   PanelOpts po;
   po.tree = tree;
+  po.blocked = blocked;
   return launch_panel(h, dtype, dY, src, rows, b, dV, ldv, dT, ldt, ps, h->d_ctrl, &h->d_ctrl->done, st, NoMark(), 0, po);
 }
 
@@ -810,6 +909,12 @@ rrf_status_t rrf_panel_qr(rrf_handle_t h, int32_t dtype, int64_t rows, int32_t b
                           void* dV, int64_t ldv, void* dT, int64_t ldt, void* d_workspace, size_t workspace_bytes,
                           void* cuda_stream) {
   return panel_qr_entry(h, dtype, rows, b, dY, ldy, dV, ldv, dT, ldt, d_workspace, workspace_bytes, cuda_stream, false);
+}
+
+rrf_status_t rrf_panel_qr_blocked(rrf_handle_t h, int32_t dtype, int64_t rows, int32_t b, const void* dY, int64_t ldy,
+                                 void* dV, int64_t ldv, void* dT, int64_t ldt, void* d_workspace,
+                                 size_t workspace_bytes, void* cuda_stream) {
+  return panel_qr_entry(h, dtype, rows, b, dY, ldy, dV, ldv, dT, ldt, d_workspace, workspace_bytes, cuda_stream, false, true);
 }
 
 rrf_status_t rrf_panel_qr_tree(rrf_handle_t h, int32_t dtype, int64_t rows, int32_t b, const void* dY, int64_t ldy,
@@ -989,6 +1094,7 @@ rrf_status_t rrf_run(rrf_handle_t h, const rrf_params_t* p, void* dA, int64_t ld
   const int steps_total = p->max_rank / b;
   // the tree panel kernel is opt-in: it is the slower of the two on every size measured so far
   const bool tree = (p->flags & RRF_FLAG_PANEL_TREE) != 0 && b <= kTsqrMaxB;
+  const bool blocked = (p->flags & RRF_FLAG_PANEL_BLOCKED) != 0;
   int look_ctas = 0;
   if (tree) {
     TreePlan tl;
@@ -1065,6 +1171,7 @@ rrf_status_t rrf_run(rrf_handle_t h, const rrf_params_t* p, void* dA, int64_t ld
   // back to it): enqueued directly, or recorded into a CUDA graph.
   auto enqueue = [&]() -> rrf_status_t {
   if (look_ctas > 0 && cudaMemsetAsync(look_bar, 0, sizeof(unsigned), st) != cudaSuccess) return RRF_ERR_CUDA;
+  if (cudaMemsetAsync(ps.blk_tags, 0, ps.blk_tag_bytes, st) != cudaSuccess) return RRF_ERR_CUDA;   // exchange tags of the blocked panel kernel
   void* W = inplace ? dA : (void*)(ws + L.w);
   const long long ldw = inplace ? lda : L.ldw;
   const void* Om = dOmegaT;
@@ -1180,6 +1287,8 @@ rrf_status_t rrf_run(rrf_handle_t h, const rrf_params_t* p, void* dA, int64_t ld
       sd.row_off = r0;
       PanelOpts po;
       po.merge_t = true;
+      po.blocked = blocked;
+      po.seq_base = 256u * (unsigned)i;
       po.bar_base = bar_next;
       po.bar_used = &bar_used;
       po.csq = csq_buf(i);
@@ -1207,6 +1316,8 @@ rrf_status_t rrf_run(rrf_handle_t h, const rrf_params_t* p, void* dA, int64_t ld
       po.alt = alt;
       po.fused_flag = fused_flag;
       po.tree = tree;
+      po.blocked = blocked;
+      po.seq_base = 256u * (unsigned)i;
       int pg = 0;
       if (sampled) po.csq = csq_buf(i);
       po.g_out = &pg;
@@ -1280,6 +1391,7 @@ rrf_status_t rrf_run(rrf_handle_t h, const rrf_params_t* p, void* dA, int64_t ld
     PanelOpts po;
     po.ctas = look_ctas;
     po.tree = tree;
+    po.blocked = blocked;
     po.merge_t = true;
     po.bar_used = &bar_used;
     std::vector<int> panel_g(steps + 1, 0);
@@ -1328,6 +1440,7 @@ rrf_status_t rrf_run(rrf_handle_t h, const rrf_params_t* p, void* dA, int64_t ld
         pn.fix.M = look_G + (size_t)kLookMaxCtas * b * b;
         if (gate) cudaStreamWaitEvent(h->aux, evZ(i), 0);
         pn.g_out = &panel_g[i + 1];
+        pn.seq_base = 256u * (unsigned)(i + 1);
         if (sampled) pn.csq = csq_buf(i + 1);
         const rrf_status_t ls = launch_panel(h, p->dtype, Ybuf[(i + 1) & 1], sn, rows - b, b, Vblk(r0 + b), ldv,
                                              Tblk(r0 + b), p->max_rank, ps, ctrl, done_after + i, h->aux, NoMark(),

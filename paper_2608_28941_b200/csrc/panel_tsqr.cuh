@@ -41,7 +41,9 @@ __device__ __forceinline__ void tsqr_stamp(int slot, bool who) {
 }
 #define RRF_STAMP(slot, who) tsqr_stamp(slot, who)
 #define RRF_CSTAMP(slot, who) if ((who) && threadIdx.x == 0) g_tsqr_trace[slot] = (unsigned long long)clock64()
+#define RRF_CSTAMP_T(slot, who, thr) if ((who) && threadIdx.x == (thr)) g_tsqr_trace[slot] = (unsigned long long)clock64()
 #else
+#define RRF_CSTAMP_T(slot, who, thr)
 #define RRF_STAMP(slot, who)
 #define RRF_CSTAMP(slot, who)
 #endif

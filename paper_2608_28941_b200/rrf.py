@@ -19,6 +19,7 @@ RRF_ERR_INVALID_ARG, RRF_ERR_WORKSPACE, RRF_ERR_CUDA, RRF_ERR_TIMEOUT, RRF_ERR_N
 RRF_FLAG_INPLACE, RRF_FLAG_FIXED_RANK, RRF_FLAG_ONE_QUEUE, RRF_FLAG_TWO_QUEUES, RRF_FLAG_NO_GRAPH = 1, 2, 4, 8, 16
 RRF_FLAG_SAMPLE_ALWAYS, RRF_FLAG_SAMPLE_NEVER, RRF_FLAG_PANEL_TREE = 32, 64, 128
 RRF_FLAG_NO_UPDATE = 256
+RRF_FLAG_PANEL_BLOCKED = 512
 
 _LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "librrf.so")
 _lib = None
@@ -44,7 +45,7 @@ class rrf_profile_t(C.Structure):
     _fields_ = [("ms", C.c_double * 9), ("launches", C.c_int32 * 9), ("pad", C.c_int32)]
 
 
-EXPORTS = ["rrf_panel_qr_tree", "rrf_transfer_workspace_bytes", "rrf_subspace_transfer", "rrf_selftest_timeout", "rrf_panel_qr_static", "rrf_set_profiling", "rrf_get_profile", "rrf_measure_peak", "rrf_create", "rrf_destroy", "rrf_workspace_bytes", "rrf_run", "rrf_panel_workspace_bytes",
+EXPORTS = ["rrf_panel_qr_blocked", "rrf_panel_qr_tree", "rrf_transfer_workspace_bytes", "rrf_subspace_transfer", "rrf_selftest_timeout", "rrf_panel_qr_static", "rrf_set_profiling", "rrf_get_profile", "rrf_measure_peak", "rrf_create", "rrf_destroy", "rrf_workspace_bytes", "rrf_run", "rrf_panel_workspace_bytes",
            "rrf_panel_qr", "rrf_apply_workspace_bytes", "rrf_apply_qt", "rrf_apply_q", "rrf_form_q",
            "rrf_fill_omega", "rrf_last_status", "rrf_status_string"]
 
@@ -68,6 +69,7 @@ def load():
     lib.rrf_panel_workspace_bytes.argtypes = [i32, i64, i32, C.POINTER(sz)]
     lib.rrf_panel_qr.argtypes = [vp, i32, i64, i32, vp, i64, vp, i64, vp, i64, vp, sz, vp]
     lib.rrf_panel_qr_tree.argtypes = [vp, i32, i64, i32, vp, i64, vp, i64, vp, i64, vp, sz, vp]
+    lib.rrf_panel_qr_blocked.argtypes = [vp, i32, i64, i32, vp, i64, vp, i64, vp, i64, vp, sz, vp]
     lib.rrf_panel_qr_static.argtypes = [i32, i64, i32, vp, i64, vp, i64, vp, i64, vp]
     lib.rrf_apply_workspace_bytes.argtypes = [i32, i64, i64, i32, C.POINTER(sz)]
     for f in (lib.rrf_apply_qt, lib.rrf_apply_q):
@@ -216,8 +218,9 @@ def rrf_run(h, A: torch.Tensor, b: int, tol: float, max_rank: int, omegaT: torch
                      res.fused_samples, res.extra_samples, res.kernel_launches, list(tr_est)[:res.n_est])
 
 
-def rrf_panel_qr(h, Y: torch.Tensor, tree: bool = False):
-    """Householder QR of a tall panel: returns (V, T) as the library writes them (`tree`: rrf_panel_qr_tree)."""
+def rrf_panel_qr(h, Y: torch.Tensor, tree: bool = False, blocked: bool = False):
+    """Householder QR of a tall panel: returns (V, T) as the library writes them
+    (`tree`: rrf_panel_qr_tree, `blocked`: rrf_panel_qr_blocked)."""
     lib = load()
     rows, b = Y.shape
     dt = _dtype_code(Y)
@@ -228,7 +231,8 @@ def rrf_panel_qr(h, Y: torch.Tensor, tree: bool = False):
     ws = torch.empty(need.value, dtype=torch.uint8, device=Y.device)
     V = torch.empty_like(Y)
     T = torch.empty((b, b), dtype=Y.dtype, device=Y.device)
-    s = (lib.rrf_panel_qr_tree if tree else lib.rrf_panel_qr)(h, dt, rows, b, C.c_void_p(Y.data_ptr()), _rowmajor(Y, "Y"), C.c_void_p(V.data_ptr()),
+    fn = lib.rrf_panel_qr_tree if tree else (lib.rrf_panel_qr_blocked if blocked else lib.rrf_panel_qr)
+    s = fn(h, dt, rows, b, C.c_void_p(Y.data_ptr()), _rowmajor(Y, "Y"), C.c_void_p(V.data_ptr()),
                          _rowmajor(V, "V"), C.c_void_p(T.data_ptr()), b, C.c_void_p(ws.data_ptr()), ws.numel(),
                          _stream())
     if s != RRF_OK:

@@ -18,6 +18,7 @@ pytestmark = pytest.mark.gpu
 
 TOL = {"f64": dict(rel=1e-10, orth=1e-12), "f32": dict(rel=1e-4, orth=1e-5)}
 ESTIMATORS = ["direct", "subtractive", "sampled_fro", "sampled_spectral"]
+ALGOS = [pytest.param("column", id="per-column"), pytest.param("blocked", id="blocked"), pytest.param("tree", id="tree")]
 
 
 @pytest.fixture(scope="module")
@@ -135,43 +136,44 @@ def check_run(h, w, g, o, A, Om, q_envelope=True, estimator="direct"):
                                           (8192, 64, "f64"), (5001, 64, "f64"), (300, 128, "f64"),
                                           (20000, 128, "f64"), (4096, 64, "f32"), (777, 32, "f32"),
                                           (60000, 32, "f64"), (45000, 64, "f64")])      # slabs of 512 / 320 rows
-@pytest.mark.parametrize("tree", [pytest.param(False, id="per-column"), pytest.param(True, id="tree")])
-def test_panel_qr_matches_oracle(h, rows, b, dtype, tree):
+@pytest.mark.parametrize("algo", ALGOS)
+def test_panel_qr_matches_oracle(h, rows, b, dtype, algo):
+    tree, blocked = algo == "tree", algo == "blocked"
     if tree and (b > 64 or rows * b > 35000 * 64):
         pytest.skip("the tree kernel takes b <= 64 and at most one slab or node per SM")
     rng = np.random.default_rng(rows + b)
     Y = rng.standard_normal((rows, b))
     if dtype == "f32":
         Y = Y.astype(np.float32)
-    V, T = rrf.rrf_panel_qr(h, torch.from_numpy(Y).cuda(), tree=tree)
+    V, T = rrf.rrf_panel_qr(h, torch.from_numpy(Y).cuda(), tree=tree, blocked=blocked)
     Vo, tau, To, _ = orc.panel_qr(Y.astype(np.float64))
     tol = 1e-12 if dtype == "f64" else 2e-6
     assert np.max(np.abs(V.cpu().numpy() - Vo)) <= tol
     assert np.max(np.abs(T.cpu().numpy() - To)) <= tol * 10
 
 
-@pytest.mark.parametrize("tree", [pytest.param(False, id="per-column"), pytest.param(True, id="tree")])
+@pytest.mark.parametrize("algo", ALGOS)
 @pytest.mark.parametrize("zero", [0.0, -0.0])
-def test_panel_qr_with_a_zero_first_pivot(h, zero, tree):
+def test_panel_qr_with_a_zero_first_pivot(h, zero, algo):
     # the reflector of a zero pivot takes the sign of the zero on both sides (LAPACK's SIGN)
     rng = np.random.default_rng(17)
     Y = rng.standard_normal((700, 16))
     Y[0, 0] = zero
-    V, T = rrf.rrf_panel_qr(h, torch.from_numpy(Y).cuda(), tree=tree)
+    V, T = rrf.rrf_panel_qr(h, torch.from_numpy(Y).cuda(), tree=algo == "tree", blocked=algo == "blocked")
     Vo, tau, To, _ = orc.panel_qr(Y)
     assert np.max(np.abs(V.cpu().numpy() - Vo)) <= 1e-12
     assert np.max(np.abs(T.cpu().numpy() - To)) <= 1e-11
     assert np.sign(Vo[1, 0]) == np.sign(Y[1, 0]) * (1.0 if np.copysign(1.0, zero) > 0 else -1.0)
 
 
-@pytest.mark.parametrize("tree", [pytest.param(False, id="per-column"), pytest.param(True, id="tree")])
-def test_panel_qr_zero_column_and_rank_deficient(h, tree):
+@pytest.mark.parametrize("algo", ALGOS)
+def test_panel_qr_zero_column_and_rank_deficient(h, algo):
     rng = np.random.default_rng(0)
     Y = rng.standard_normal((500, 16))
     Y[:, 3] = 0.0
     Y[:, 7] = Y[:, 2] * 2.0          # exactly dependent column
     Y[5:, 0] = 0.0                   # nothing to annihilate below... except rows 1..4
-    V, T = rrf.rrf_panel_qr(h, torch.from_numpy(Y).cuda(), tree=tree)
+    V, T = rrf.rrf_panel_qr(h, torch.from_numpy(Y).cuda(), tree=algo == "tree", blocked=algo == "blocked")
     Vg, Tg = V.cpu().numpy(), T.cpu().numpy()
     Q = np.eye(500) - Vg @ Tg @ Vg.T
     assert np.linalg.norm(Q.T @ Q - np.eye(500)) < 1e-12
@@ -319,10 +321,11 @@ def test_each_block_factors_the_residual_it_was_given(h, name, kw, sched):
                                      ("cfg3", dict(m=1024, n=1024, max_rank=512)),
                                      ("cfg2", dict(m=6000, n=1111, max_rank=256)),      # several tree levels
                                      ("cfg4", dict(m=1024, n=2752, max_rank=256, rank=64))])
-def test_whole_runs_with_the_tree_panel_kernel(h, name, kw, sched):
-    # the opt-in panel kernel (tall-skinny QR + reconstruction of the reflectors) under both schedules
+@pytest.mark.parametrize("panel", [pytest.param(rrf.RRF_FLAG_PANEL_TREE, id="tree"), pytest.param(rrf.RRF_FLAG_PANEL_BLOCKED, id="blocked")])
+def test_whole_runs_with_the_other_panel_kernels(h, name, kw, sched, panel):
+    # the opt-in panel kernels (tall-skinny QR + reconstruction; micro-panels of eight columns) under both schedules
     w = wl.CONFIGS[name].scaled(**kw)
-    g, o, A, Om = run_both(h, w, flags=sched | rrf.RRF_FLAG_PANEL_TREE)
+    g, o, A, Om = run_both(h, w, flags=sched | panel)
     assert g.queues == (2 if sched == rrf.RRF_FLAG_TWO_QUEUES else 1)
     check_run(h, w, g, o, A, Om)
 
