@@ -186,10 +186,10 @@ def run_reference(args, w, rank, world):
 class Problem:
     """One workload resident on the device: inputs, outputs and workspace of rrf_run."""
 
-    def __init__(self, h, w, dev, sched, estimator=0):
+    def __init__(self, h, w, dev, sched, estimator=0, panel_ctas=0):
         import torch
         from paper_2608_28941_b200 import rrf
-        self.h, self.w, self.dev, self.sched, self.estimator = h, w, dev, sched, estimator
+        self.h, self.w, self.dev, self.sched, self.estimator, self.panel_ctas = h, w, dev, sched, estimator, panel_ctas
         self.A, self.Om, self.OmT = generate(w, dev)
         self.tdt, self.esize = self.A.dtype, self.A.element_size()
         p = rrf.make_params(rrf.RRF_F64 if w.dtype == "f64" else rrf.RRF_F32, w.m, w.n, w.b, w.tol, w.max_rank)
@@ -203,7 +203,7 @@ class Problem:
         w = self.w
         om = self.OmT if isinstance(omegaT, str) else omegaT
         return rrf.rrf_run(self.h, self.A if A is None else A, w.b, w.tol, w.max_rank, omegaT=om, V=self.V, T=self.T,
-                           B=self.B, workspace=self.ws, flags=self.sched | flags, seed=w.seed, estimator=self.estimator)
+                           B=self.B, workspace=self.ws, flags=self.sched | flags, seed=w.seed, estimator=self.estimator, panel_ctas=self.panel_ctas)
 
 
 def time_problem(pb, steps, warmup, world, barrier):
@@ -378,6 +378,7 @@ def main():
                     help="no-update: A is left unchanged and B is not formed (one pass over A per block instead of "
                          "three); stops on the sampled Frobenius estimate.  Flops are counted as the in-place schedule's")
     ap.add_argument("--estimator", type=int, default=0, choices=[0, 1, 2, 3])
+    ap.add_argument("--panel-ctas", type=int, default=0, help="look-ahead schedule: SMs given to the panel chain (0: library's rule)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
 
@@ -429,7 +430,7 @@ def main():
         args.no_e2e = True
         args.no_per_config = True
     peaks = measured_peaks()
-    pb = Problem(h, w, dev, sched, estimator)
+    pb = Problem(h, w, dev, sched, estimator, args.panel_ctas)
     sampler = ClockSampler(local)
     pb.step()
     barrier()

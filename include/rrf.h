@@ -42,7 +42,7 @@ typedef enum {
   RRF_OK = 0,
   RRF_MAX_RANK_REACHED = 1,   /* success with information: rank cap hit before the tolerance */
   RRF_ERR_INVALID_ARG = -1,
-  RRF_ERR_WORKSPACE = -2,     /* workspace too small, or a panel too tall for on-chip storage */
+  RRF_ERR_WORKSPACE = -2,     /* workspace too small, or (tree kernel, static entry point) a panel too tall for on-chip storage */
   RRF_ERR_CUDA = -3,          /* a CUDA call failed; the raw code is in rrf_result_t.cuda_error */
   RRF_ERR_TIMEOUT = -4,       /* a bounded device-side wait gave up */
   RRF_ERR_NONFINITE = -5      /* A contains NaN or Inf */
@@ -182,6 +182,8 @@ rrf_status_t rrf_run(rrf_handle_t h, const rrf_params_t* p,
  * explicit ones and zeros) and the compact-WY factor T (b x b, ldt >= b, upper triangular) with
  * H_0 ... H_{b-1} = I - V T V^T.  Reflector convention: beta = -sign(alpha) ||x||, v_0 = 1,
  * tau = (beta - alpha)/beta.  R is not returned.  Workspace: rrf_panel_workspace_bytes().
+ * Any height: a panel whose slabs do not fit in the SMs' shared memory (more than about 32000 x 128 or
+ * 47000 x 64 doubles on 148 SMs) is factored by the blocked kernel with its slabs in global memory.
  * Does not synchronise the stream; a timeout of the in-kernel grid barrier is reported by
  * the next rrf_last_status() call.
  */

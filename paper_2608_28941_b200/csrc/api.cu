@@ -212,9 +212,25 @@ static bool plan_tree(const rrf_ctx* h, long long rows, int b, int max_ctas, boo
 }
 // Plan of the blocked panel kernel (panel_blk.cuh): slab height per CTA and which of its small matrices fit in
 // shared memory beside the slab.
-struct BlkPlan { int G, R, RS, Rp, ksplit, c_in_smem; size_t smem; };
-static bool plan_blk(const rrf_ctx* h, long long rows, int b, BlkPlan* p, int ctas = 0, bool fix = false) {
+struct BlkPlan { int G, R, RS, Rp, ksplit, c_in_smem, gslab; size_t smem; };
+// `global_slab`: keep the slabs in global memory (no height limit; the panel can be confined to very few SMs)
+static bool plan_blk(const rrf_ctx* h, long long rows, int b, BlkPlan* p, int ctas = 0, bool fix = false,
+                     bool global_slab = false) {
   if (fix && b > 64) return false;
+  p->gslab = 0;
+  if (global_slab) {
+    const long long ext = rows + (fix ? b : 0);
+    const size_t fixd = fix ? (size_t)panel_fix_doubles(b) : 0;
+    p->R = std::max(64, ceil_div(ext, ctas > 0 ? ctas : h->sms));
+    p->G = ceil_div(ext, p->R);
+    p->RS = (p->R + 15) / 16 * 16;
+    p->Rp = p->RS + 1;
+    p->ksplit = std::max(1, 16 / (b / 16));
+    p->c_in_smem = 1;
+    p->gslab = 1;
+    p->smem = (std::max(fixd, p->ksplit > 1 ? (size_t)kBlkDw : 0) + (size_t)kMB * (b + 8) + 16 + 8 + 8 + 8 + 64 + 64 + 8 + 8) * sizeof(double);
+    return p->G <= h->sms;
+  }
   const long long ext = rows + (fix ? b : 0);
   const size_t small = 16 + 8 + 8 + 8 + 64 + 64 + 8 + 8;
   const size_t fixd = fix ? (size_t)panel_fix_doubles(b) : 0;
@@ -268,11 +284,14 @@ static size_t blk_tag_bytes(int sms, int b) {
   const size_t gp = (size_t)(sms + 31) / 32 * 32;
   return align_up(((size_t)2 * 16 * gp * 2 + (size_t)kMB * b * gp * 2 + (size_t)16 * b * 2) * sizeof(unsigned long long), 256);
 }
-static size_t blk_scratch_bytes(int sms, int b) {
-  return blk_tag_bytes(sms, b) + align_up((size_t)sms * kMB * b * sizeof(double), 256);
+static size_t blk_slab_bytes(int sms, int b, long long rows) {   // slabs in global memory: [G][b][Rp], Rp <= R + 17
+  return align_up((size_t)b * (size_t)(2 * (rows + b) + 17LL * sms) * sizeof(double), 256);   // G R < 2 (rows + b)
 }
-static size_t panel_scratch_bytes(int sms, int b) {
-  return direct_scratch_bytes(sms, b) + tsqr_scratch_bytes(sms, b) + blk_scratch_bytes(sms, b);
+static size_t blk_scratch_bytes(int sms, int b, long long rows) {
+  return blk_tag_bytes(sms, b) + align_up((size_t)sms * kMB * b * sizeof(double), 256) + blk_slab_bytes(sms, b, rows);
+}
+static size_t panel_scratch_bytes(int sms, int b, long long rows) {
+  return direct_scratch_bytes(sms, b) + tsqr_scratch_bytes(sms, b) + blk_scratch_bytes(sms, b, rows);
 }
 constexpr int kLookMaxCtas = 48;   // most CTAs a confined panel may take
 // Rough cost model of one pass, in microseconds, used only to choose the schedule (fitted to event
@@ -300,7 +319,7 @@ struct PassModel {
 static size_t look_scratch_bytes(int b) {   // Gpart[kLookMaxCtas][b*b] + M[b*b]
   return align_up((size_t)(kLookMaxCtas + 1) * b * b * sizeof(double), 256);
 }
-struct PanelScratch { double *P, *piv, *gram, *tau; unsigned* bar; TsqrScratch ts; BlkScratch bk; unsigned* blk_tags; size_t blk_tag_bytes; };
+struct PanelScratch { double *P, *piv, *gram, *tau; unsigned* bar; TsqrScratch ts; BlkScratch bk; unsigned* blk_tags; size_t blk_tag_bytes; double* gslab; };
 // `sms`: the SM count the buffers were sized for (the handle's bound kMaxSms for caller workspaces)
 static PanelScratch carve_panel(unsigned char* base, int sms, int b, bool with_tree = true) {
   PanelScratch s;
@@ -313,6 +332,7 @@ static PanelScratch carve_panel(unsigned char* base, int sms, int b, bool with_t
   s.bk = BlkScratch{nullptr, nullptr, nullptr, nullptr};
   s.blk_tags = nullptr;
   s.blk_tag_bytes = 0;
+  s.gslab = nullptr;
   if (with_tree && b <= kTsqrMaxB) {
     double* t = reinterpret_cast<double*>(base + direct_scratch_bytes(sms, b));
     const size_t blk = (size_t)sms * b * b;
@@ -327,6 +347,7 @@ static PanelScratch carve_panel(unsigned char* base, int sms, int b, bool with_t
     s.bk.Pw = s.bk.Lw + (size_t)2 * 16 * gp * 2;
     s.bk.Rw = s.bk.Pw + (size_t)kMB * b * gp * 2;
     s.bk.Cg = reinterpret_cast<double*>(q + blk_tag_bytes(sms, b));
+    s.gslab = reinterpret_cast<double*>(q + blk_tag_bytes(sms, b) + align_up((size_t)sms * kMB * b * sizeof(double), 256));
   }
   return s;
 }
@@ -477,6 +498,7 @@ struct PanelOpts {
   cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
   bool tree = false;               // b <= 64: use the tree kernel (no grid barrier per column)
   bool blocked = false;            // use the blocked kernel (micro-panels of eight columns, panel_blk.cuh) if it fits
+  bool global_slab = false;        // blocked kernel: keep the slabs in global memory
   unsigned seq_base = 0;           // blocked kernel: first tag value of this launch (tags only grow within a run)
   double* csq = nullptr;           // [b][Gp]: the panel kernel leaves the column sums of squares of the panel here
   int* g_out = nullptr;            // out: CTAs of the per-column panel kernel (Gp = g rounded up to 32)
@@ -523,13 +545,21 @@ static rrf_status_t launch_panel(rrf_ctx* h, int dtype, const void* Y, PanelSour
   const size_t tsmem = ((size_t)b * (b + 1) + (size_t)(b / 2) * (b / 2 + 1)) * sizeof(double);
   cudaError_t e;
   BlkPlan bp;
-  if (o.blocked && ps.bk.Lw != nullptr && plan_blk(h, rows, b, &bp, o.ctas, o.fix.enabled != 0)) {
+  // a panel too tall for shared memory goes to the blocked kernel with its slabs in global memory
+  PanelPlan pp_probe;
+  const bool too_tall = ps.bk.Lw != nullptr && !plan_panel(h, rows, b, &pp_probe, o.ctas, o.fix.enabled != 0) &&
+                        !(o.fix.enabled && b > 64);
+  const bool want_global = o.global_slab || too_tall;
+  if ((o.blocked || too_tall) && ps.bk.Lw != nullptr &&
+      ((!want_global && plan_blk(h, rows, b, &bp, o.ctas, o.fix.enabled != 0)) ||
+       plan_blk(h, rows, b, &bp, o.ctas, o.fix.enabled != 0, true))) {
     // blocked kernel: micro-panels of eight columns, exchanges instead of grid barriers
     int R = bp.R, Rp = bp.Rp, RS = bp.RS, ksplit = bp.ksplit, c_in_smem = bp.c_in_smem;
     BlkScratch bk = ps.bk;
     unsigned seq_base = o.seq_base;
+    double* gslab = bp.gslab ? ps.gslab : nullptr;
     void* args[] = {&Y, &src, &alt, &fused_flag, &rows_i, &b, &R, &Rp, &RS, &V, &ldv, &gram, &tau, &bk, &seq_base,
-                    &ksplit, &c_in_smem, &bar, &ctrl, &done_flag, &fix, &bar_base, &Tmerged, &ldt, &csq};
+                    &ksplit, &c_in_smem, &bar, &ctrl, &done_flag, &fix, &bar_base, &Tmerged, &ldt, &csq, &gslab};
     size_t smem = bp.smem;
     if (o.merge_t) smem = std::max(smem, tsmem);
     if (o.bar_used != nullptr) *o.bar_used = (unsigned)(o.fix.enabled ? 2 : 0) * (unsigned)bp.G;
@@ -682,7 +712,7 @@ static bool run_layout(const rrf_params_t* p, bool need_omega, RunLayout* L) {
   L->ypart2 = off; off += align_up(ymax * esize, 256);   // the look-ahead schedule keeps two sampled panels
   L->zpart = off; off += align_up(zmax * esize, 256);
   L->zt = off; off += align_up((size_t)npad * b * esize, 256);
-  L->panel = off; off += panel_scratch_bytes(sms, b);
+  L->panel = off; off += panel_scratch_bytes(sms, b, p->m);
   L->look = off; off += look_scratch_bytes(b);
   L->csq = off; off += align_up((size_t)2 * b * ((sms + 31) / 32 * 32) * sizeof(double), 256);   // two panels in flight
   L->w = off;
@@ -877,7 +907,7 @@ rrf_status_t rrf_fill_omega(rrf_handle_t h, int32_t dtype, uint64_t seed, int64_
 
 rrf_status_t rrf_panel_workspace_bytes(int32_t dtype, int64_t rows, int32_t b, size_t* bytes) {
   if (bytes == nullptr || !b_ok(dtype, b) || rows < b) return RRF_ERR_INVALID_ARG;
-  *bytes = panel_scratch_bytes(kMaxSms, b);
+  *bytes = panel_scratch_bytes(kMaxSms, b, rows);
   return RRF_OK;
 }
 
@@ -889,7 +919,7 @@ static rrf_status_t panel_qr_entry(rrf_handle_t h, int32_t dtype, int64_t rows, 
   if (!b_ok(dtype, b) || rows < b || rows > 0x7fffffffLL || ldy < b || ldv < b || ldt < b || ldy > 0x7fffffffLL)
     return RRF_ERR_INVALID_ARG;
   if (tree && b > kTsqrMaxB) return RRF_ERR_INVALID_ARG;
-  if (workspace_bytes < panel_scratch_bytes(kMaxSms, b) ) return RRF_ERR_WORKSPACE;
+  if (workspace_bytes < panel_scratch_bytes(kMaxSms, b, rows)) return RRF_ERR_WORKSPACE;
   cudaStream_t st = (cudaStream_t)cuda_stream;
   PanelScratch ps = carve_panel((unsigned char*)d_workspace, h->sms, b);
   if (cudaMemsetAsync(ps.bar, 0, sizeof(unsigned), st) != cudaSuccess) return RRF_ERR_CUDA;
@@ -1096,7 +1126,12 @@ rrf_status_t rrf_run(rrf_handle_t h, const rrf_params_t* p, void* dA, int64_t ld
   const bool tree = (p->flags & RRF_FLAG_PANEL_TREE) != 0 && b <= kTsqrMaxB;
   const bool blocked = (p->flags & RRF_FLAG_PANEL_BLOCKED) != 0;
   int look_ctas = 0;
-  if (tree) {
+  if (blocked && !tree) {
+    // opt-in blocked panel kernel: under look-ahead (only if asked for) the panel is confined to a few SMs, its
+    // slabs in global memory when shared memory does not hold them
+    if ((p->flags & RRF_FLAG_TWO_QUEUES) && steps_total >= 2 && b <= 64 && !unchanged)
+      look_ctas = p->tune_panel_ctas > 0 ? std::min((int)p->tune_panel_ctas, h->sms / 3) : 12;
+  } else if (tree) {
     TreePlan tl;
     const int cap = std::min(kLookMaxCtas, h->sms / 3);
     const int lim = p->tune_panel_ctas > 0 ? std::min(cap, (int)p->tune_panel_ctas) : cap;
@@ -1122,8 +1157,7 @@ rrf_status_t rrf_run(rrf_handle_t h, const rrf_params_t* p, void* dA, int64_t ld
       if (wanted && plan_panel(h, m, b, &ppl, best, true)) look_ctas = best;
     }
   }
-  PanelPlan pp0;
-  if (!tree && look_ctas == 0 && !plan_panel(h, m, b, &pp0)) return fail(RRF_ERR_WORKSPACE);   // tallest panel must fit on chip
+  // (a panel too tall for shared memory is factored by the blocked kernel with its slabs in global memory)
 
   cudaStream_t const user_st = (cudaStream_t)cuda_stream;
   cudaStream_t st = user_st;

@@ -90,7 +90,7 @@ __device__ __forceinline__ bool ll_sum(const unsigned long long* rowp, int G, un
 // above the panel).  R rows per CTA, RS >= R rows allocated (a multiple of 16, zero filled), pitch Rp.
 // `ksplit`: warps that share the rows of one tile in the D product (1: no shared-memory staging of D);
 // `c_in_smem`: C of the block step is staged in shared memory (else read from global memory, for slabs that
-// leave no room).
+// leave no room).  `gslab`: the slabs themselves live in global memory (any height, any number of CTAs).
 // ------------------------------------------------------------------------------------------
 template <typename T>
 __global__ void __launch_bounds__(kPanelThreads)
@@ -98,7 +98,8 @@ __global__ void __launch_bounds__(kPanelThreads)
                      int rows, int b, int R, int Rp, int RS, T* __restrict__ V, long long ldv,
                      double* __restrict__ gram, double* __restrict__ tau_out, BlkScratch bs, unsigned seq_base,
                      int ksplit, int c_in_smem, unsigned* bar, Ctrl* ctrl, const int* done_flag, PanelFix fix,
-                     unsigned bar_base, T* __restrict__ Tout, long long ldt, double* __restrict__ csq) {
+                     unsigned bar_base, T* __restrict__ Tout, long long ldt, double* __restrict__ csq,
+                     double* __restrict__ gslab) {      // non-NULL: the slabs live in global memory ([CTA][b][Rp])
   if (*reinterpret_cast<const volatile int*>(done_flag) || *reinterpret_cast<const volatile int*>(&ctrl->status) < 0) return;
   const bool use_alt = fused_flag != nullptr && *fused_flag == 0;
   const PanelSource src = use_alt ? src_alt : src_fused;
@@ -115,8 +116,10 @@ __global__ void __launch_bounds__(kPanelThreads)
   const int lb = 31 - __clz(b);
   const int aux_n = max(fix.enabled ? panel_fix_doubles(b) : 0, ksplit > 1 ? kBlkDw : 0);
   const int cp = b + 8;
-  double* S = psm;                                  // [b][Rp]
-  double* aux = S + (size_t)b * Rp;                 // fix-up staging, then the D partials of the K-split warps
+  // The slab [b][Rp]: in shared memory, or - for slabs taller than shared memory holds, or to confine a tall
+  // panel to a few SMs - in this CTA's own stretch of global memory (served by L1 / L2; nobody else touches it).
+  double* S = gslab != nullptr ? gslab + (size_t)blockIdx.x * b * Rp : psm;
+  double* aux = gslab != nullptr ? psm : psm + (size_t)b * Rp;   // fix-up staging, then the D partials of the K-split warps
   double* Cs = aux + aux_n;                         // [8][b + 8] (c_in_smem)
   double* p_s = Cs + (c_in_smem ? kMB * cp : 0);    // [2][8]
   double* pr_s = p_s + 16;                          // [8] pivot row of the micro-panel's columns
