@@ -274,6 +274,25 @@ rrf_status_t rrf_form_q(rrf_handle_t h, int32_t dtype, int64_t m, int32_t b, int
                         void* d_workspace, size_t workspace_bytes, void* cuda_stream);
 
 /*
+ * Building blocks of the column-sharded variant (outlook of the paper: "extensions to distributed matrix
+ * layouts"; driver: paper_2608_28941_b200/sharded.py).  With the columns of A split over the GPUs, A = [A_1 .. A_P],
+ * and the rows of Omega split to match, a block step needs one exchange: the m_i x b panel Y_i = sum_p W_p Omega_{i,p}
+ * (an all-reduce, left to the caller's communication library); everything else is local.
+ *
+ * rrf_sample_panel: dY (rows x b, dense, leading dimension b) = C (rows x n, ldc) * OmegaT (b x n, ldo)^T, i.e. line 7
+ *   of Algorithm 2 for one rank's column block.  Workspace: rrf_sample_workspace_bytes(), 256-byte aligned.
+ * rrf_frobenius_sq: *d_out (a double in DEVICE memory) = squared Frobenius norm of C (rows x cols, ldc), summed in a fixed
+ *   order in double precision; rows may be 0.  Workspace: 8 * 4 * (number of SMs) bytes (5 KB is always enough).
+ * Neither synchronises the stream.
+ */
+rrf_status_t rrf_sample_workspace_bytes(int32_t dtype, int64_t rows, int32_t b, size_t* bytes);
+rrf_status_t rrf_sample_panel(rrf_handle_t h, int32_t dtype, int64_t rows, int64_t n, int32_t b,
+                              const void* dC, int64_t ldc, const void* dOmegaT, int64_t ldo, void* dY,
+                              void* d_workspace, size_t workspace_bytes, void* cuda_stream);
+rrf_status_t rrf_frobenius_sq(rrf_handle_t h, int32_t dtype, int64_t rows, int64_t cols, const void* dC, int64_t ldc,
+                       double* d_out, void* d_workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
  * rrf_subspace_transfer - the subspace-consistency transform of the paper's Section "Towards
  * Efficient Low-Rank Deep Learning": a low-rank optimiser state M (k_old x ncols) held in the basis
  * Q_old of the previous step is re-expressed in the current basis Q_new,

@@ -254,6 +254,49 @@ def apply_q(V: np.ndarray, T: np.ndarray, b: int, C: np.ndarray) -> np.ndarray:
     return C
 
 
+def rrf_column_sharded(A_loc: np.ndarray, Omega_loc: np.ndarray, b: int, tol: float, max_rank: int, allreduce,
+                       relative: bool = True, fixed_rank: bool = False) -> OracleResult:
+    """One rank of the column-sharded variant (outlook: "extensions to distributed matrix layouts").
+
+    The columns of A are split over the ranks, A = [A_1 ... A_P]; rank p holds A_p (m x n_p) and the matching
+    ROWS of Omega (n_p x max_rank), since A Omega_i = sum_p A_p Omega_{i,p}.  `allreduce(x)` returns the sum of the
+    ranks' arrays (or floats).  Per block there is exactly one exchange of data, the m_i x b panel:
+        Y_i = allreduce(W_p[r0:, :] Omega_{i,p});  every rank factors the same Y_i;  the update is local;
+    plus two scalars (||A||_F^2 once, the residual norm per block).  V, T, k and the traces come out identical on
+    every rank; B is this rank's column block of B.  Stops on the residual norm (estimator "direct").
+    """
+    W = np.array(A_loc, dtype=np.float64, copy=True)
+    Omega_loc = np.asarray(Omega_loc, dtype=np.float64)
+    m = W.shape[0]
+    normA2 = float(allreduce(_sumsq(W)))
+    sigma2 = (tol * tol * normA2) if relative else tol * tol
+    V = np.zeros((m, max_rank))
+    T = np.zeros((b, max_rank))
+    res = OracleResult(0, RRF_OK, 0, normA2, sigma2, V, T, None)
+    E = normA2
+    E_sub = normA2
+    met = (not fixed_rank) and not (E > sigma2)
+    i = 0
+    while not met and (i + 1) * b <= max_rank:
+        r0 = i * b
+        Y = allreduce(W[r0:, :] @ Omega_loc[:, r0:r0 + b])           # the one exchange of a block step
+        Vi, _, Ti, _ = panel_qr(Y)
+        V[r0:, r0:r0 + b] = Vi
+        T[:, r0:r0 + b] = Ti
+        W[r0:, :] -= Vi @ (Ti.T @ (Vi.T @ W[r0:, :]))
+        E_sub = E_sub - float(allreduce(_sumsq(W[r0:r0 + b, :])))
+        E = float(allreduce(_sumsq(W[r0 + b:, :])))
+        res.E_sub.append(E_sub)
+        res.E_dir.append(E)
+        met = (not fixed_rank) and not (E > sigma2)
+        i += 1
+    k = i * b
+    res.k, res.steps = k, i
+    res.status = RRF_OK if E <= sigma2 else RRF_MAX_RANK_REACHED
+    res.V, res.T, res.B = V[:, :k], T[:, :k], W[:k, :].copy()
+    return res
+
+
 def permuted_rerun(A, Omega, b, tol, max_rank, seed=0, **kw) -> OracleResult:
     """The same problem with the columns of A and the rows of Omega permuted.
 

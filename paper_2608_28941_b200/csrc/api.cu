@@ -953,6 +953,67 @@ rrf_status_t rrf_panel_qr_tree(rrf_handle_t h, int32_t dtype, int64_t rows, int3
   return panel_qr_entry(h, dtype, rows, b, dY, ldy, dV, ldv, dT, ldt, d_workspace, workspace_bytes, cuda_stream, true);
 }
 
+// ---- building blocks of the column-sharded variant: sample one panel, squared Frobenius norm
+rrf_status_t rrf_sample_workspace_bytes(int32_t dtype, int64_t rows, int32_t b, size_t* bytes) {
+  if (bytes == nullptr || !b_ok(dtype, b) || rows < 1) return RRF_ERR_INVALID_ARG;
+  const int esize = dtype == RRF_F64 ? 8 : 4;
+  *bytes = align_up((size_t)kSampleMaxSeg * (size_t)rows * b * esize, 256) + 256;
+  return RRF_OK;
+}
+
+rrf_status_t rrf_sample_panel(rrf_handle_t h, int32_t dtype, int64_t rows, int64_t n, int32_t b, const void* dC,
+                              int64_t ldc, const void* dOmegaT, int64_t ldo, void* dY, void* d_workspace,
+                              size_t workspace_bytes, void* cuda_stream) {
+  if (h == nullptr || dC == nullptr || dOmegaT == nullptr || dY == nullptr || d_workspace == nullptr)
+    return RRF_ERR_INVALID_ARG;
+  const int esize = dtype == RRF_F64 ? 8 : 4;
+  if (!b_ok(dtype, b) || rows < 1 || n < 1 || rows > 0x7fffffffLL || n > 0x7fffffffLL) return RRF_ERR_INVALID_ARG;
+  if (!ld_ok(ldc, n, esize) || !ld_ok(ldo, n, esize) || !aligned16(dC) || !aligned16(dOmegaT)) return RRF_ERR_INVALID_ARG;
+  size_t need = 0;
+  rrf_sample_workspace_bytes(dtype, rows, b, &need);
+  if (workspace_bytes < need || (reinterpret_cast<uintptr_t>(d_workspace) & 255u)) return RRF_ERR_WORKSPACE;
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  const OpTable* ops = get_ops(dtype, b);
+  CUtensorMap tmC, tmO;
+  if (!make_map(h, &tmC, dtype, dC, rows, n, ldc, kSampleBM) || !make_map(h, &tmO, dtype, dOmegaT, b, n, ldo, b))
+    return RRF_ERR_INVALID_ARG;
+  const SamplePlan sp = plan_sample(h->sms, rows, n, esize, ops->s_kbs);
+  ops->sample(tmC, tmO, d_workspace, 0, (int)rows, (int)n, 0, sp, h->d_ctrl, nullptr, nullptr, st);
+  const int grid = (int)std::min<long long>((rows * b + 255) / 256, (long long)h->sms * 8);
+  if (dtype == RRF_F64)
+    panel_sum_kernel<double><<<grid, 256, 0, st>>>((const double*)d_workspace, sp.nseg, rows * b, rows, b, (double*)dY, h->d_ctrl);
+  else
+    panel_sum_kernel<float><<<grid, 256, 0, st>>>((const float*)d_workspace, sp.nseg, rows * b, rows, b, (float*)dY, h->d_ctrl);
+  const cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) {
+    h->last_cuda = (int)e;
+    return RRF_ERR_CUDA;
+  }
+  return RRF_OK;
+}
+
+rrf_status_t rrf_frobenius_sq(rrf_handle_t h, int32_t dtype, int64_t rows, int64_t cols, const void* dC, int64_t ldc,
+                       double* d_out, void* d_workspace, size_t workspace_bytes, void* cuda_stream) {
+  if (h == nullptr || d_out == nullptr || d_workspace == nullptr || rows < 0 || cols < 1 || ldc < cols) return RRF_ERR_INVALID_ARG;
+  if (dtype != RRF_F64 && dtype != RRF_F32) return RRF_ERR_INVALID_ARG;
+  if (rows > 0 && dC == nullptr) return RRF_ERR_INVALID_ARG;
+  const int grid = h->sms * 4;
+  if (workspace_bytes < (size_t)grid * sizeof(double)) return RRF_ERR_WORKSPACE;
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  double* part = (double*)d_workspace;
+  if (dtype == RRF_F64)
+    frob2_part_kernel<double><<<grid, 256, 0, st>>>((const double*)dC, ldc, rows, cols, part);
+  else
+    frob2_part_kernel<float><<<grid, 256, 0, st>>>((const float*)dC, ldc, rows, cols, part);
+  frob2_final_kernel<<<1, 256, 0, st>>>(part, grid, d_out);
+  const cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) {
+    h->last_cuda = (int)e;
+    return RRF_ERR_CUDA;
+  }
+  return RRF_OK;
+}
+
 rrf_status_t rrf_apply_workspace_bytes(int32_t dtype, int64_t m, int64_t ncols, int32_t b, size_t* bytes) {
   if (bytes == nullptr || !b_ok(dtype, b) || m < b || ncols < 1) return RRF_ERR_INVALID_ARG;
   const int esize = dtype == RRF_F64 ? 8 : 4;

@@ -832,6 +832,31 @@ __global__ void __launch_bounds__(128)
   }
 }
 
+// Squared Frobenius norm of a rows x cols matrix, in two fixed-order stages (accumulated in double): every CTA
+// sums a contiguous range of rows, CTA 0's successor kernel adds the partials in CTA order.
+template <typename T>
+__global__ void __launch_bounds__(256)
+    frob2_part_kernel(const T* __restrict__ C, long long ldc, long long rows, long long cols, double* __restrict__ part) {
+  __shared__ double red[32];
+  const long long per = (rows + gridDim.x - 1) / gridDim.x;
+  const long long r_lo = per * blockIdx.x, r_hi = min(rows, r_lo + per);
+  double s = 0.0;
+  for (long long r = r_lo; r < r_hi; ++r)
+    for (long long c = threadIdx.x; c < cols; c += 256) {
+      const double v = (double)C[r * ldc + c];
+      s += v * v;
+    }
+  const double tot = block_sum(s, red);
+  if (threadIdx.x == 0) part[blockIdx.x] = tot;
+}
+__global__ void __launch_bounds__(256) frob2_final_kernel(const double* __restrict__ part, int n, double* __restrict__ out) {
+  __shared__ double red[32];
+  double s = 0.0;
+  for (int i = threadIdx.x; i < n; i += 256) s += part[i];
+  const double tot = block_sum(s, red);
+  if (threadIdx.x == 0) *out = tot;
+}
+
 // dst (rows x b, dense) = sum of the nseg stacked partial panels the sample kernel wrote, in their fixed order
 template <typename T>
 __global__ void __launch_bounds__(256)

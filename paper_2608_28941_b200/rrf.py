@@ -45,7 +45,7 @@ class rrf_profile_t(C.Structure):
     _fields_ = [("ms", C.c_double * 9), ("launches", C.c_int32 * 9), ("pad", C.c_int32)]
 
 
-EXPORTS = ["rrf_panel_qr_blocked", "rrf_panel_qr_tree", "rrf_transfer_workspace_bytes", "rrf_subspace_transfer", "rrf_selftest_timeout", "rrf_panel_qr_static", "rrf_set_profiling", "rrf_get_profile", "rrf_measure_peak", "rrf_create", "rrf_destroy", "rrf_workspace_bytes", "rrf_run", "rrf_panel_workspace_bytes",
+EXPORTS = ["rrf_sample_workspace_bytes", "rrf_sample_panel", "rrf_frobenius_sq", "rrf_panel_qr_blocked", "rrf_panel_qr_tree", "rrf_transfer_workspace_bytes", "rrf_subspace_transfer", "rrf_selftest_timeout", "rrf_panel_qr_static", "rrf_set_profiling", "rrf_get_profile", "rrf_measure_peak", "rrf_create", "rrf_destroy", "rrf_workspace_bytes", "rrf_run", "rrf_panel_workspace_bytes",
            "rrf_panel_qr", "rrf_apply_workspace_bytes", "rrf_apply_qt", "rrf_apply_q", "rrf_form_q",
            "rrf_fill_omega", "rrf_last_status", "rrf_status_string"]
 
@@ -72,6 +72,9 @@ def load():
     lib.rrf_panel_qr_blocked.argtypes = [vp, i32, i64, i32, vp, i64, vp, i64, vp, i64, vp, sz, vp]
     lib.rrf_panel_qr_static.argtypes = [i32, i64, i32, vp, i64, vp, i64, vp, i64, vp]
     lib.rrf_apply_workspace_bytes.argtypes = [i32, i64, i64, i32, C.POINTER(sz)]
+    lib.rrf_sample_workspace_bytes.argtypes = [i32, i64, i32, C.POINTER(sz)]
+    lib.rrf_sample_panel.argtypes = [vp, i32, i64, i64, i32, vp, i64, vp, i64, vp, vp, sz, vp]
+    lib.rrf_frobenius_sq.argtypes = [vp, i32, i64, i64, vp, i64, vp, vp, sz, vp]
     for f in (lib.rrf_apply_qt, lib.rrf_apply_q):
         f.argtypes = [vp, i32, i64, i32, i32, vp, i64, vp, i64, vp, i64, i64, vp, sz, vp]
     lib.rrf_form_q.argtypes = [vp, i32, i64, i32, i32, vp, i64, vp, i64, vp, i64, vp, sz, vp]

@@ -591,3 +591,28 @@ def test_run_with_builtin_omega(h):
     o = orc.rrf(A, OmT.T, w.b, w.tol, w.max_rank)
     assert g.k == o.k and g.status == o.status
     assert relmax(g.B[:g.k].cpu().numpy(), o.B) <= 1e-10
+
+
+# ------------------------------------------------------------------ column-sharded driver (one rank on one GPU)
+
+
+@pytest.mark.parametrize("name,kw", [("cfg2", dict(m=1536, n=1280, max_rank=512)), ("cfg1", dict(m=900, n=700, max_rank=256)),
+                                     ("cfg4b", dict(m=1024, n=2752, max_rank=256, rank=64))])
+def test_column_sharded_driver_as_a_single_rank(h, name, kw):
+    # the multi-GPU variant's code path (sample, exchange, panel QR, local update, norms) with a one-rank "exchange";
+    # its host logic across ranks is covered on the CPU with gloo (tests/test_column_sharded_cpu.py)
+    from paper_2608_28941_b200 import sharded
+    w = wl.CONFIGS[name].scaled(**kw)
+    A, _ = wl.make_matrix(w)
+    Om = wl.make_omega(w).astype(w.np_dtype)
+    mult = 2 if w.dtype == "f64" else 4
+    g = sharded.rrf_run_column_sharded(h, _pad_cols(A, mult), _pad_cols(np.ascontiguousarray(Om.T), mult), w.b, w.tol, w.max_rank)
+    o = orc.rrf(A.astype(np.float64), Om.astype(np.float64), w.b, w.tol, w.max_rank)
+    assert (g.k, g.steps, g.status) == (o.k, o.steps, o.status)
+    tl = TOL[w.dtype]
+    assert relmax(g.B[:g.k].cpu().numpy().astype(np.float64), o.B) <= tl["rel"]
+    assert np.allclose(g.E_dir_trace, o.E_dir, rtol=1e-8 if w.dtype == "f64" else 1e-3, atol=1e-24 * o.normA2)
+    Q = rrf.rrf_form_q(h, _pad_cols(g.V[:, :g.k].cpu().numpy(), mult), _pad_cols(g.T[:, :g.k].cpu().numpy(), mult), w.b, g.k)
+    Q = Q.cpu().numpy().astype(np.float64)
+    assert np.linalg.norm(Q.T @ Q - np.eye(g.k)) <= tl["orth"]
+    assert relmax(Q @ g.B[:g.k].cpu().numpy().astype(np.float64), orc.form_q(o.V, o.T, w.b) @ o.B) <= 10 * tl["rel"]
