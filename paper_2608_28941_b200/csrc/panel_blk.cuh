@@ -11,11 +11,13 @@
 // tensor cores:  D = X^T V8 (every column against the eight new vectors; for finished columns these are the
 // entries of V^T V that the T factor needs), one two-stage exchange, C = T8^T D, X -= V8 C.
 //
-// Exchanges replace the grid barrier: every CTA publishes its values in its own line of a global buffer,
-// followed by a tag (release); every CTA reads all lines after seeing their tags (acquire) and sums them in CTA
-// order, so all CTAs hold the same bits.  A line is reused two rounds later, which is safe because a CTA can
-// only write round r+2 after it has read every CTA's round r+1, i.e. after every CTA has finished reading
-// round r.  All CTAs must be co-resident (cooperative launch); every wait is bounded.
+// Exchanges replace the grid barrier: every CTA writes its values as flagged words (see ll_store: the value and
+// the tag of the round in the same 64-bit words) into its own slots of a global buffer; every CTA reads all slots,
+// spinning until the round's tag is there, and sums them in CTA order, so all CTAs hold the same bits.  A slot is
+// reused two rounds later, which is safe because a CTA can only write round r+2 after it has read every CTA's
+// round r+1, i.e. after every CTA has finished reading round r.  All CTAs must be co-resident (cooperative
+// launch); every wait is bounded.  The slab can live in shared memory or, for panels that do not fit there, in a
+// stretch of global memory private to the CTA.
 #pragma once
 
 #include "panel_tsqr.cuh"
@@ -23,7 +25,6 @@
 namespace rrf {
 
 constexpr int kMB = 8;                       // columns of a micro-panel
-constexpr int kBlkLine = 16;                 // doubles per exchange line: 8 partial sums, 8 pivot-row values
 
 struct BlkScratch {
   unsigned long long* Lw;  // [2][16][Gp][2]: per-column exchange, flagged words (see ll_store); Gp = G rounded up to 32
