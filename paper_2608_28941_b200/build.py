@@ -1,6 +1,7 @@
 """Build the C-ABI library (librrf.so) for sm_100a with nvcc, in-tree.
 
-Usage: python -m paper_2608_28941_b200.build [--force]
+Usage: python -m paper_2608_28941_b200.build [--force] [-v] [--nvtx]
+(--nvtx: NVTX ranges around the phases of rrf_run, for timeline tools; off by default)
 """
 from __future__ import annotations
 
@@ -22,7 +23,7 @@ def _stale() -> bool:
     return any(os.path.getmtime(f) > t for f in deps)
 
 
-def build(force: bool = False, verbose: bool = False) -> str:
+def build(force: bool = False, verbose: bool = False, nvtx: bool = False) -> str:
     if not force and not _stale():
         return LIB
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
@@ -31,9 +32,11 @@ def build(force: bool = False, verbose: bool = False) -> str:
     if verbose:
         cmd.insert(1, "-Xptxas")
         cmd.insert(2, "-v")
+    if nvtx:
+        cmd += ["-DRRF_NVTX", "-ldl"]
     subprocess.run(cmd, check=True)
     return LIB
 
 
 if __name__ == "__main__":
-    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv))
+    print(build(force="--force" in sys.argv or "--nvtx" in sys.argv, verbose="-v" in sys.argv, nvtx="--nvtx" in sys.argv))

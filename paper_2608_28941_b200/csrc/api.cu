@@ -12,6 +12,29 @@
 #include "gemm_sk.cuh"
 #include "panel_blk.cuh"
 
+// NVTX ranges around the phases of rrf_run (host-side enqueue order), compiled in with -DRRF_NVTX only
+// (python -m paper_2608_28941_b200.build --nvtx); one range per kernel group, named "<phase> <block step>".
+#ifdef RRF_NVTX
+#include <nvtx3/nvToolsExt.h>
+static const char* const kNvtxPhase[] = {"init", "sample", "panel", "tfactor", "vtw", "tz", "update", "stop", "end"};
+#define RRF_NVTX_MARK(open, phase, step)                                   \
+  do {                                                                     \
+    if (open) nvtxRangePop();                                              \
+    char nm_[48];                                                          \
+    std::snprintf(nm_, sizeof nm_, "rrf %s %d", kNvtxPhase[phase], step);  \
+    nvtxRangePushA(nm_);                                                   \
+    open = true;                                                           \
+  } while (0)
+#define RRF_NVTX_CLOSE(open) \
+  do {                       \
+    if (open) nvtxRangePop(); \
+    open = false;            \
+  } while (0)
+#else
+#define RRF_NVTX_MARK(open, phase, step) (void)(open)
+#define RRF_NVTX_CLOSE(open) (void)(open)
+#endif
+
 namespace rrf {
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
@@ -1294,7 +1317,9 @@ rrf_status_t rrf_run(rrf_handle_t h, const rrf_params_t* p, void* dA, int64_t ld
     return RRF_ERR_INVALID_ARG;
 
   // profiling: one event before every kernel, tagged with (phase, block step)
+  bool nvtx_open = false;
   auto mark = [&](int phase, int step) {
+    RRF_NVTX_MARK(nvtx_open, phase, step);
     if (!h->profiling) return;
     if (nev == h->events.size()) {
       cudaEvent_t ev;
@@ -1589,6 +1614,7 @@ rrf_status_t rrf_run(rrf_handle_t h, const rrf_params_t* p, void* dA, int64_t ld
     }
   }
   mark(RRF_PHASE_SKIPPED, steps);   // closing event
+  RRF_NVTX_CLOSE(nvtx_open);
   return RRF_OK;
   };
 

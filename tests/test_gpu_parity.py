@@ -405,6 +405,43 @@ def test_variant_that_leaves_a_unchanged(h, name, kw, tol):
     assert relmax(Qf @ (Qf.T @ A64), Qof @ (Qof.T @ A64)) <= 10 * tl["rel"]
 
 
+def test_single_precision_subtractive_rule_leaves_the_track_near_384_on_the_device(h):
+    # The paper's stability experiment (1024 x 1024, singular values 1 ... 1e-14, b = 64, single precision) on the
+    # GPU: Algorithm 2 line 9 (estimator 1) follows the residual for a few blocks and then stops tracking it
+    # (cancellation: it stalls, or turns negative), while the residual norm itself (always recorded) and the
+    # sampled Frobenius rule keep following the singular values down to the single-precision floor.
+    rng = np.random.default_rng(2024)
+    n, b, cap = 1024, 64, 640
+    U, _ = np.linalg.qr(rng.standard_normal((n, n)))
+    Vv, _ = np.linalg.qr(rng.standard_normal((n, n)))
+    sv = np.logspace(0, -14, n)
+    A = ((U * sv) @ Vv.T).astype(np.float32)
+    Om = rng.standard_normal((n, cap)).astype(np.float32)
+    dA, dOmT = torch.from_numpy(A).cuda(), torch.from_numpy(np.ascontiguousarray(Om.T)).cuda()
+    g = rrf.rrf_run(h, dA, b, 0.0, cap, omegaT=dOmT, estimator=1, flags=rrf.RRF_FLAG_FIXED_RANK)
+    o = orc.rrf(A, Om, b, 0.0, cap, dtype=np.float32)
+    assert g.k == cap
+    tail2 = np.array([np.sum(sv[(i + 1) * b:] ** 2) for i in range(cap // b)])   # Eckart-Young tails
+    e_dir, e_sub = np.array(g.E_dir_trace), np.array(g.E_sub_trace)
+    # the first blocks: both quantities are the residual (within 20 %) ...
+    assert np.all(np.abs(e_sub[:3] - e_dir[:3]) <= 0.2 * e_dir[:3])
+    # ... by block 6 (k = 384) and after, the subtractive one is off by more than a factor of two or negative
+    lost = (e_sub[5:] <= 0.0) | (np.abs(e_sub[5:] - e_dir[5:]) > e_dir[5:])
+    assert lost.all(), (e_sub, e_dir)
+    # the residual norm keeps following the spectrum until the fp32 floor (about 1e-13 of ||A||^2)
+    floor = 1e-12 * g.normA2
+    assert np.all(e_dir >= 0.5 * tail2) and np.all(e_dir <= 100.0 * tail2 + floor)
+    # same loss in the oracle's single-precision rerun (the paper's observation, pinned on the CPU too)
+    o_sub, o_dir = np.array(o.E_sub), np.array(o.E_dir)
+    assert ((o_sub[5:] <= 0.0) | (np.abs(o_sub[5:] - o_dir[5:]) > o_dir[5:])).all()
+    # the sampled rule (estimator 2) looks at panel i = residual after i blocks: stays within its spread of it
+    g2 = rrf.rrf_run(h, dA, b, 0.0, cap, omegaT=dOmT, estimator=2, flags=rrf.RRF_FLAG_FIXED_RANK)
+    est = np.array(g2.E_est_trace)
+    prev = np.concatenate([[g2.normA2], np.array(g2.E_dir_trace)[:-1]])
+    ok = prev > floor
+    assert np.all(est[ok] >= 0.3 * prev[ok]) and np.all(est[ok] <= 3.0 * prev[ok])
+
+
 def test_schedules_agree_and_stop_mid_way(h):
     # stops after a few blocks: the look-ahead has factored one panel too many by then, which must
     # not show in k, B, the traces, or the defined part of V and T
@@ -538,6 +575,28 @@ def test_runs_on_a_caller_stream(h):
             out = B[:g.k] * 1.0          # consumer on the same stream
             assert g.k == ref.k and torch.equal(out, refB)
     torch.cuda.synchronize()
+
+
+def test_kernels_behind_a_timed_out_wait_return_at_once(h):
+    # a wait that gives up also raises the stop flag, so work already enqueued behind it does not run on
+    # half-written data (and cannot wait out its own limit): here a panel QR enqueued after the self test
+    import ctypes as C
+    lib = rrf.load()
+    Y = torch.randn((512, 16), dtype=torch.float64, device="cuda")
+    V = torch.full_like(Y, 7.0)
+    T = torch.full((16, 16), 7.0, dtype=torch.float64, device="cuda")
+    need = C.c_size_t()
+    lib.rrf_panel_workspace_bytes(rrf.RRF_F64, 512, 16, C.byref(need))
+    ws = torch.empty(need.value, dtype=torch.uint8, device="cuda")
+    st = rrf._stream()
+    assert lib.rrf_selftest_timeout(h, C.c_double(20.0), st) == rrf.RRF_OK          # enqueue only
+    assert lib.rrf_panel_qr(h, rrf.RRF_F64, 512, 16, C.c_void_p(Y.data_ptr()), 16, C.c_void_p(V.data_ptr()), 16,
+                            C.c_void_p(T.data_ptr()), 16, C.c_void_p(ws.data_ptr()), ws.numel(), st) == rrf.RRF_OK
+    assert rrf.rrf_last_status(h) == rrf.RRF_ERR_TIMEOUT            # synchronises, reports, clears
+    assert float(V.min()) == 7.0 and float(T.max()) == 7.0          # the panel kernels saw the flag and left at once
+    Vg, Tg = rrf.rrf_panel_qr(h, Y)                                 # and the context works again
+    Vo, _, To, _ = orc.panel_qr(Y.cpu().numpy())
+    assert np.max(np.abs(Vg.cpu().numpy() - Vo)) <= 1e-12
 
 
 def test_bounded_wait_times_out_and_context_survives(h):
