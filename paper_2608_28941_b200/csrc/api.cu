@@ -7,9 +7,11 @@
 #include <cstring>
 #include <mutex>
 #include <new>
+#include <type_traits>
 #include <vector>
 
 #include "gemm_sk.cuh"
+#include "gemm_tc.cuh"
 #include "panel_blk.cuh"
 
 // NVTX ranges around the phases of rrf_run (host-side enqueue order), compiled in with -DRRF_NVTX only
@@ -69,6 +71,8 @@ struct rrf_ctx {
   std::vector<unsigned char> gcand;      // arguments of the last directly enqueued call
   std::vector<std::pair<int, int>> gmarks;
   int graph_off;                         // set when a capture failed: enqueue directly from then on
+  int f32_engine;                        // single-precision V^T W: 0 = mma.sync 3xTF32, 1 = tcgen05 3xTF32
+  int tc_chunk;                          // tcgen05: 64-row tiles summed in tensor memory between round-to-nearest adds
 };
 
 namespace rrf {
@@ -105,7 +109,7 @@ static SamplePlan plan_sample(int sms, long long rows, long long n, int esize, i
 }
 
 // stream-K plan of Z = V^T C: tiles (column tile, K chunk), one CTA per SM
-struct VtwPlan { int bn, nct, KT, total, tpc, P, npad, slots; };
+struct VtwPlan { int bn, nct, KT, total, tpc, P, npad, slots, tc, chunk; };
 static VtwPlan plan_vtw(int sms, long long rows, long long ncols, int bn) {
   VtwPlan p;
   p.bn = bn;
@@ -116,6 +120,8 @@ static VtwPlan plan_vtw(int sms, long long rows, long long ncols, int bn) {
   p.tpc = ceil_div(p.total, sms);
   p.P = ceil_div(p.total, p.tpc);
   p.slots = p.P + p.nct;
+  p.tc = 0;
+  p.chunk = 0;
   return p;
 }
 // stream-K plan of the fused update: tiles (row slab, column tile)
@@ -377,7 +383,7 @@ static PanelScratch carve_panel(unsigned char* base, int sms, int b, bool with_t
 
 // ------------------------------------------------------------------ tensor maps
 static bool make_map(const rrf_ctx* h, CUtensorMap* map, int dtype, const void* base, unsigned long long rows,
-                     unsigned long long cols, unsigned long long ld, unsigned box_rows) {
+                     unsigned long long cols, unsigned long long ld, unsigned box_rows, bool atom32 = false) {
   const int esize = dtype == RRF_F64 ? 8 : 4;
   cuuint64_t gdim[2] = {cols, rows};
   cuuint64_t gstr[1] = {ld * (unsigned long long)esize};
@@ -385,7 +391,8 @@ static bool make_map(const rrf_ctx* h, CUtensorMap* map, int dtype, const void* 
   cuuint32_t estr[2] = {1, 1};
   const CUresult r = h->encode(map, dtype == RRF_F64 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT64 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32,
                                2, const_cast<void*>(base), gdim, gstr, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                               CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                               atom32 ? CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B : CU_TENSOR_MAP_SWIZZLE_128B,
+                               CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
                                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return r == CUDA_SUCCESS;
 }
@@ -412,6 +419,10 @@ struct Ops {
   static constexpr int V_STAGE = kVtwBK * (B + V_BN) * (int)sizeof(T);
   static constexpr int V_STAGES = (3 * V_STAGE + 1024 > 200 * 1024) ? 2 : (4 * V_STAGE + 1024 > 200 * 1024 ? 3 : 4);
   static constexpr int V_SMEM = V_STAGES * V_STAGE + 1024;
+  // vtw on tcgen05 (single precision only): stages of the TMA ring and of the (hi, lo) operand ring
+  static constexpr int TC_B = (B == 16) ? 32 : B;
+  static constexpr int TC_RS = (B >= 128) ? 3 : 4, TC_OS = (B == 32) ? 3 : 2;
+  static_assert(TcCfg<TC_B, TC_RS, TC_OS>::SMEM + 1024 <= kMaxSmem, "shared memory");
   // fused update: slab height 128 (64 for the widest block), two 128-byte column groups per tile
   static constexpr int U_BM = (B >= 128) ? 64 : 128;
   static constexpr int U_BNB = 2;
@@ -436,6 +447,11 @@ struct Ops {
     e = cudaFuncSetAttribute(upd_sk_kernel<T, B, U_BM, U_BNB, U_WM, U_WN, U_STAGES, U_PW>,
                              cudaFuncAttributeMaxDynamicSharedMemorySize, U_SMEM);
     if (e != cudaSuccess) return e;
+    if constexpr (std::is_same<T, float>::value) {
+      e = cudaFuncSetAttribute(vtw_tc_kernel<B, TC_RS, TC_OS>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                               TcCfg<B, TC_RS, TC_OS>::SMEM);
+      if (e != cudaSuccess) return e;
+    }
     e = cudaFuncSetAttribute(tz_kernel<T, B>, cudaFuncAttributeMaxDynamicSharedMemorySize, Z_SMEM);
     return e;
   }
@@ -447,6 +463,13 @@ struct Ops {
   }
   static void vtw(const CUtensorMap& tmV, const CUtensorMap& tmC, void* Zpart, int r0, int cv0, const VtwPlan& p,
                   Ctrl* ctrl, cudaStream_t st) {
+    if constexpr (std::is_same<T, float>::value) {
+      if (p.tc) {     // the maps then have 32-row boxes
+        vtw_tc_kernel<B, TC_RS, TC_OS><<<p.P, kTcThreads, TcCfg<B, TC_RS, TC_OS>::SMEM, st>>>(
+            tmV, tmC, (float*)Zpart, r0, cv0, p.KT, p.total, p.tpc, p.chunk, ctrl);
+        return;
+      }
+    }
     vtw_sk_kernel<T, B, V_BN, kVtwBK, V_WM, V_WN, V_STAGES>
         <<<p.P, 9 * 32, V_SMEM, st>>>(tmV, tmC, (T*)Zpart, r0, cv0, p.KT, p.total, p.tpc, ctrl);
   }
@@ -799,6 +822,8 @@ rrf_status_t rrf_create(rrf_handle_t* out, int device) {
   h->graph = nullptr;
   h->gexec = nullptr;
   h->graph_off = 0;
+  h->f32_engine = 0;
+  h->tc_chunk = 0;
   std::memset(&h->profile, 0, sizeof(h->profile));
   cudaError_t e = cudaDeviceGetAttribute(&h->sms, cudaDevAttrMultiProcessorCount, device);
   if (e == cudaSuccess) e = cudaDeviceGetAttribute(&h->smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, device);
@@ -846,6 +871,13 @@ rrf_status_t rrf_last_status(rrf_handle_t h, void* cuda_stream) {
   if (cudaStreamSynchronize(st) != cudaSuccess) return RRF_ERR_CUDA;
   if (c.status != 0) cudaMemsetAsync(h->d_ctrl, 0, sizeof(Ctrl), st);
   return (rrf_status_t)c.status;
+}
+
+rrf_status_t rrf_set_f32_engine(rrf_handle_t h, int32_t engine, int32_t chunk_tiles) {
+  if (h == nullptr || engine < 0 || engine > 1 || chunk_tiles < 0) return RRF_ERR_INVALID_ARG;
+  h->f32_engine = engine;
+  h->tc_chunk = chunk_tiles;
+  return RRF_OK;
 }
 
 rrf_status_t rrf_set_profiling(rrf_handle_t h, int32_t enable) {
@@ -1071,7 +1103,9 @@ static rrf_status_t apply_blocks(rrf_handle_t h, int dtype, long long m, int b, 
   void* Zt = ws;
   void* Zpart = ws + align_up((size_t)vp0.npad * b * esize, 256);
   CUtensorMap tmV_k, tmC_k, tmV_u, tmC_u, tmZ;
-  if (!make_map(h, &tmV_k, dtype, dV, m, k, ldv, kVtwBK) || !make_map(h, &tmC_k, dtype, dC, m, ncols, ldc, kVtwBK) ||
+  const bool tc = dtype == RRF_F32 && h->f32_engine == 1;
+  const unsigned kbox = tc ? kTcSub : kVtwBK;     // rows of a TMA box of the V^T C kernel in use
+  if (!make_map(h, &tmV_k, dtype, dV, m, k, ldv, kbox, tc) || !make_map(h, &tmC_k, dtype, dC, m, ncols, ldc, kbox, tc) ||
       !make_map(h, &tmV_u, dtype, dV, m, k, ldv, ops->u_bm) || !make_map(h, &tmC_u, dtype, dC, m, ncols, ldc, ops->u_bm) ||
       !make_map(h, &tmZ, dtype, Zt, vp0.npad, b, b, ops->u_bn))
     return RRF_ERR_INVALID_ARG;
@@ -1079,7 +1113,9 @@ static rrf_status_t apply_blocks(rrf_handle_t h, int dtype, long long m, int b, 
   for (int q = 0; q < nblk; ++q) {
     const int l = transpose ? q : nblk - 1 - q;
     const int r0 = l * b, rows = (int)(m - r0);
-    const VtwPlan vp = plan_vtw(h->sms, rows, ncols, ops->v_bn);
+    VtwPlan vp = plan_vtw(h->sms, rows, ncols, ops->v_bn);
+    vp.tc = tc;
+    vp.chunk = h->tc_chunk;
     ops->vtw(tmV_k, tmC_k, Zpart, r0, r0, vp, h->d_ctrl, st);
     ops->tz(Zpart, vp, (const char*)dT + (size_t)r0 * esize, ldt, transpose ? 1 : 0, Zt, &h->d_ctrl->done, st);
     const UpdPlan up = plan_upd(h->sms, rows, ncols, ops->u_bm, ops->u_bn, ops->u_wn);
@@ -1305,12 +1341,14 @@ rrf_status_t rrf_run(rrf_handle_t h, const rrf_params_t* p, void* dA, int64_t ld
   // Pass 0 reads A itself and writes W (no copy W <- A): the first panels are sampled from A, V_0^T A is taken
   // from A, and the update of pass 0 loads its tiles from A and stores them to W.
   CUtensorMap tmW_s, tmA_s, tmA_k, tmA_u, tmO, tmV_k, tmW_k, tmV_u, tmW_u, tmZ;
-  if (!make_map(h, &tmA_s, p->dtype, dA, m, n, lda, kSampleBM) || !make_map(h, &tmA_k, p->dtype, dA, m, n, lda, kVtwBK) ||
+  const bool tc = p->dtype == RRF_F32 && h->f32_engine == 1;
+  const unsigned kbox = tc ? kTcSub : kVtwBK;     // rows of a TMA box of the V^T W kernel in use
+  if (!make_map(h, &tmA_s, p->dtype, dA, m, n, lda, kSampleBM) || !make_map(h, &tmA_k, p->dtype, dA, m, n, lda, kbox, tc) ||
       !make_map(h, &tmA_u, p->dtype, dA, m, n, lda, ops->u_bm) ||
       !make_map(h, &tmW_s, p->dtype, W, m, n, ldw, kSampleBM) ||
       !make_map(h, &tmO, p->dtype, Om, p->max_rank, n, ldom, b) ||
-      !make_map(h, &tmV_k, p->dtype, dV, m, p->max_rank, ldv, kVtwBK) ||
-      !make_map(h, &tmW_k, p->dtype, W, m, n, ldw, kVtwBK) ||
+      !make_map(h, &tmV_k, p->dtype, dV, m, p->max_rank, ldv, kbox, tc) ||
+      !make_map(h, &tmW_k, p->dtype, W, m, n, ldw, kbox, tc) ||
       !make_map(h, &tmV_u, p->dtype, dV, m, p->max_rank, ldv, ops->u_bm) ||
       !make_map(h, &tmW_u, p->dtype, W, m, n, ldw, ops->u_bm) ||
       !make_map(h, &tmZ, p->dtype, Zt, npad, b, b, ops->u_bn))
@@ -1375,7 +1413,7 @@ rrf_status_t rrf_run(rrf_handle_t h, const rrf_params_t* p, void* dA, int64_t ld
     void* Pbuf = ws + L.w;             // m x b panel, dense (the working copy of A is not needed here)
     const int npad_p = plan_vtw(h->sms, m, b, ops->v_bn).npad;
     CUtensorMap tmP_k, tmP_u, tmZp;
-    if (!make_map(h, &tmP_k, p->dtype, Pbuf, m, b, b, kVtwBK) || !make_map(h, &tmP_u, p->dtype, Pbuf, m, b, b, ops->u_bm) ||
+    if (!make_map(h, &tmP_k, p->dtype, Pbuf, m, b, b, kbox, tc) || !make_map(h, &tmP_u, p->dtype, Pbuf, m, b, b, ops->u_bm) ||
         !make_map(h, &tmZp, p->dtype, Zt, npad_p, b, b, ops->u_bn))
       return RRF_ERR_INVALID_ARG;
     unsigned bar_next = 0, bar_used = 0;
@@ -1392,7 +1430,9 @@ rrf_status_t rrf_run(rrf_handle_t h, const rrf_params_t* p, void* dA, int64_t ld
         panel_sum_kernel<float><<<sum_grid, 256, 0, st>>>((const float*)Ypart, sp.nseg, m * b, m, b, (float*)Pbuf, ctrl);
       for (int l = 0; l < i; ++l) {
         const int q0 = l * b, rl = (int)(m - q0);
-        const VtwPlan vp = plan_vtw(h->sms, rl, b, ops->v_bn);
+        VtwPlan vp = plan_vtw(h->sms, rl, b, ops->v_bn);
+        vp.tc = tc;
+        vp.chunk = h->tc_chunk;
         mark(RRF_PHASE_VTW, i);
         ops->vtw(tmV_k, tmP_k, Zpart, q0, q0, vp, ctrl, st);
         mark(RRF_PHASE_TZ, i);
@@ -1447,7 +1487,9 @@ rrf_status_t rrf_run(rrf_handle_t h, const rrf_params_t* p, void* dA, int64_t ld
       if (sampled)                     // the sampled rule looks at panel i before block i is applied
         est_kernel<<<1, 128, 0, st>>>(csq_buf(i), pg, (pg + 31) & ~31, b, p->max_rank, p->estimator, fixed ? 1 : 0, 0, i,
                                       tr_est, ctrl);
-      const VtwPlan vp = plan_vtw(h->sms, rows, n, ops->v_bn);
+      VtwPlan vp = plan_vtw(h->sms, rows, n, ops->v_bn);
+      vp.tc = tc;
+      vp.chunk = h->tc_chunk;
       mark(RRF_PHASE_VTW, i);
       ops->vtw(tmV_k, i == 0 ? tmA_k : tmW_k, Zpart, r0, r0, vp, ctrl, st);
       mark(RRF_PHASE_TZ, i);
@@ -1580,7 +1622,9 @@ rrf_status_t rrf_run(rrf_handle_t h, const rrf_params_t* p, void* dA, int64_t ld
       if (sampled)                     // the sampled rule looks at panel i before block i is applied
         est_kernel<<<1, 128, 0, st>>>(csq_buf(i), panel_g[i], (panel_g[i] + 31) & ~31, b, p->max_rank, p->estimator,
                                       fixed ? 1 : 0, 0, i, tr_est, ctrl);
-      const VtwPlan vp = plan_vtw(gate ? h->sms : gsms, rows, n, ops->v_bn);
+      VtwPlan vp = plan_vtw(gate ? h->sms : gsms, rows, n, ops->v_bn);
+      vp.tc = tc;
+      vp.chunk = h->tc_chunk;
       mark(RRF_PHASE_VTW, i);
       ops->vtw(tmV_k, i == 0 ? tmA_k : tmW_k, Zpart, r0, r0, vp, ctrl, st);
       mark(RRF_PHASE_TZ, i);
@@ -1629,7 +1673,7 @@ rrf_status_t rrf_run(rrf_handle_t h, const rrf_params_t* p, void* dA, int64_t ld
     };
     const void* ptrs[6] = {dA, dOmegaT, dV, dT, dB, d_workspace};
     const long long lds[4] = {lda, ldo, ldv, ldb};
-    const int ints[2] = {look_ctas, h->profiling};
+    const int ints[4] = {look_ctas, h->profiling, h->f32_engine, h->tc_chunk};
     put(p, sizeof(*p));
     put(ptrs, sizeof(ptrs));
     put(lds, sizeof(lds));

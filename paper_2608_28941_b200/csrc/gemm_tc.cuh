@@ -1,0 +1,270 @@
+// Single-precision Z = V_i^T W[r0:, :] (Algorithm 2 line 8, first product) on the fifth-generation tensor
+// cores: tcgen05.mma kind::tf32, operands in shared memory, accumulator in tensor memory.
+//
+// Same tiling, same stream-K ranges and the same partial-result slots as vtw_sk_kernel, so the
+// consumer of the partials does not know which of the two ran.  What differs is the engine:
+//
+//   * The instruction computes D[128 x B] (+)= A[128 x 8] * B[8 x B] with A = (W tile)^T and B = V tile.
+//     Both tiles arrive by TMA with a 128-byte line holding one contraction index and 32 consecutive
+//     columns, which is the instruction's transposed ("MN-major") operand form; for 32-bit operands
+//     that form needs the swizzle with 32-byte atoms, so these tensor maps differ from the mma.sync
+//     kernel's in the swizzle mode (and in the box height).  No transposition anywhere.
+//   * fp32 accuracy comes from the same 3xTF32 split as the mma.sync path, x = hi + lo with
+//     hi = tf32(x), lo = tf32(x - hi), D += A_lo B_hi + A_hi B_lo + A_hi B_hi.  The split is an
+//     element-wise pass by four warps from the TMA ring into a second ring of (hi, lo) planes at
+//     the same byte offsets, so the swizzle never has to be decoded.
+//   * The tensor core's own accumulation does not round to nearest.  `chunk` bounds how many
+//     64-row tiles are summed inside tensor memory before the four warps add the accumulator into
+//     registers with ordinary round-to-nearest adds (0: a whole accumulator stays in tensor memory).
+//
+// Warp roles: 0-3 split operands and drain the accumulator (warp w owns tensor-memory lanes
+// 32w .. 32w+31, i.e. those columns of the tile), 4 issues TMA loads, 5 issues the MMAs.
+// Every wait is bounded; on a time-out all roles fall through to the common exit, where tensor
+// memory is released.
+#pragma once
+
+#include "gemm_sk.cuh"
+
+namespace rrf {
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void proxy_fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+
+// whole warp; writes the base address of `ncols` tensor-memory columns (a power of two >= 32) to *slot
+__device__ __forceinline__ void tmem_alloc(uint32_t* slot, uint32_t ncols) {
+  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(slot)), "r"(ncols)
+               : "memory");
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t base, uint32_t ncols) {
+  asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(base), "r"(ncols) : "memory");
+}
+// mbarrier arrival once every MMA this thread has issued so far is complete
+__device__ __forceinline__ void tc_commit(uint64_t* bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
+               : "memory");
+}
+// Shared-memory operand descriptor for a 32-bit operand whose rows are contraction indices ("MN-major"):
+// 128-byte lines of 32 elements along M or N, consecutive lines are consecutive contraction indices,
+// and the 32-byte quarter of a line is XORed with the line index modulo 4.  This is the one layout in
+// which the tensor core accepts a transposed TF32 operand (with the ordinary 16-byte-chunk swizzle it
+// returns zeros), and TMA writes it with CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B.
+// `addr` is the first of the eight lines of one K step, `lbo` the byte distance between groups of
+// 32 elements along M or N; groups of four lines follow each other at 512 bytes.
+__device__ __forceinline__ uint64_t tc_desc(uint32_t addr, uint32_t lbo) {
+  return (uint64_t)((addr & 0x3FFFFu) >> 4) | ((uint64_t)((lbo >> 4) & 0x3FFFu) << 16) |
+         ((uint64_t)(512u >> 4) << 32) | (1ull << 46) | (1ull << 61);
+}
+// fp32 accumulator, TF32 operands, both MN-major, D is M x N
+__host__ __device__ constexpr uint32_t tc_idesc_tf32(int M, int N) {
+  return (1u << 4) | (2u << 7) | (2u << 10) | (1u << 15) | (1u << 16) | ((uint32_t)(N >> 3) << 17) |
+         ((uint32_t)(M >> 4) << 24);
+}
+__device__ __forceinline__ void tc_mma_tf32(uint32_t d_tmem, uint64_t a, uint64_t b, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(a), "l"(b), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+// 16 consecutive columns of this thread's tensor-memory lane
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, float (&v)[16]) {
+  uint32_t r[16];
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr));
+  // the registers are named as operands so that no use of them can be scheduled before the wait
+  asm volatile("tcgen05.wait::ld.sync.aligned;"
+               : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]), "+r"(r[8]),
+                 "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]), "+r"(r[14]), "+r"(r[15])
+               :
+               : "memory");
+#pragma unroll
+  for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
+}
+
+constexpr int kTcBN = 128;     // columns of W per accumulator = rows of D = tensor-memory lanes
+constexpr int kTcSub = 32;     // rows (contraction indices) per ring stage; a 64-row tile is two stages
+constexpr int kTcThreads = 192;
+
+template <int B, int RS, int OS>
+struct TcCfg {
+  static constexpr int NBV = B / 32, NBC = kTcBN / 32;
+  static constexpr int BOX = kTcSub * 128;
+  static constexpr int RAW = (NBV + NBC) * BOX;       // one stage of the TMA ring
+  static constexpr int OPS = 2 * RAW;                 // one stage of the operand ring: hi plane, lo plane
+  static constexpr int SMEM = RS * RAW + OS * OPS + 1024;
+};
+
+template <int B, int RS, int OS>
+__global__ void __launch_bounds__(kTcThreads, 1)
+    vtw_tc_kernel(const __grid_constant__ CUtensorMap tmV,  // V [m][ldv], box [32][32]
+                  const __grid_constant__ CUtensorMap tmC,  // C [m][ncols], box [32][32]
+                  float* __restrict__ Zpart, int r0, int cv0, int KT, int total, int tpc, int chunk, Ctrl* ctrl) {
+  if (*reinterpret_cast<volatile int*>(&ctrl->done)) return;
+  using Cfg = TcCfg<B, RS, OS>;
+  constexpr int NBV = Cfg::NBV, NBC = Cfg::NBC, BOX = Cfg::BOX, RAW = Cfg::RAW, OPS = Cfg::OPS;
+  static_assert(B == 32 || B == 64 || B == 128, "tensor-memory columns: a power of two, at least 32");
+
+  extern __shared__ unsigned char smem_raw[];
+  unsigned char* smem = align1024(smem_raw);
+  unsigned char* ops = smem + RS * RAW;
+  __shared__ uint64_t raw_full[RS], raw_empty[RS], op_full[OS], op_empty[OS], acc_full, acc_empty;
+  __shared__ uint32_t tmem_slot;
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int p = blockIdx.x;
+  const int L0 = p * tpc;
+  const int ntile = min(total, L0 + tpc) - L0;
+  const int nsub = 2 * ntile;
+
+  if (tid == 0) {
+    for (int s = 0; s < RS; ++s) {
+      mbar_init(&raw_full[s], 1);
+      mbar_init(&raw_empty[s], 4);
+    }
+    for (int s = 0; s < OS; ++s) {
+      mbar_init(&op_full[s], 4);
+      mbar_init(&op_empty[s], 1);
+    }
+    mbar_init(&acc_full, 1);
+    mbar_init(&acc_empty, 4);
+    mbar_fence_init();
+  }
+  __syncthreads();
+  if (warp == 0) tmem_alloc(&tmem_slot, B);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = *reinterpret_cast<volatile uint32_t*>(&tmem_slot);
+
+  // After the second stage of tile i the accumulator is drained if the tile is the last one of its column tile
+  // (or of this CTA's range), or if it closes a chunk.  Writer and reader of the accumulator both use this rule.
+  auto drain_after = [&](int i, bool* last_of_acc) {
+    const int L = L0 + i, c = L / KT, kt = L - c * KT;
+    *last_of_acc = (i == ntile - 1) || (kt == KT - 1);
+    return *last_of_acc || (chunk > 0 && (kt + 1) % chunk == 0);
+  };
+
+  if (warp == 4) {
+    // ---------------------------------------------------------------- TMA producer
+    if (lane == 0) {
+      for (int q = 0; q < nsub; ++q) {
+        const int s = q % RS;
+        if (q >= RS && !mbar_wait(&raw_empty[s], ((q / RS) - 1) & 1, ctrl)) break;
+        const int L = L0 + (q >> 1), c = L / KT, kt = L - c * KT;
+        const int y = r0 + kt * 64 + (q & 1) * kTcSub;
+        unsigned char* dst = smem + s * RAW;
+        mbar_expect_tx(&raw_full[s], RAW);
+#pragma unroll
+        for (int v = 0; v < NBV; ++v) tma_load_2d(dst + v * BOX, &tmV, cv0 + v * 32, y, &raw_full[s]);
+#pragma unroll
+        for (int cb = 0; cb < NBC; ++cb)
+          tma_load_2d(dst + (NBV + cb) * BOX, &tmC, c * kTcBN + cb * 32, y, &raw_full[s]);
+      }
+    }
+  } else if (warp == 5) {
+    // ---------------------------------------------------------------- MMA issuer
+    if (lane == 0) {
+      constexpr uint32_t idesc = tc_idesc_tf32(kTcBN, B);
+      uint32_t fresh = 1;        // the next product overwrites the accumulator
+      int ndrain = 0;
+      for (int q = 0; q < nsub; ++q) {
+        const int o = q % OS;
+        if (!mbar_wait(&op_full[o], (q / OS) & 1, ctrl)) break;
+        if (fresh && ndrain > 0 && !mbar_wait(&acc_empty, (ndrain - 1) & 1, ctrl)) break;
+        tc_fence_after();
+        const uint32_t hi = smem_u32(ops + o * OPS), lo = hi + RAW;
+        const uint32_t offA = NBV * BOX;       // the W tile follows the V tile in a stage
+#pragma unroll
+        for (int ks = 0; ks < kTcSub / 8; ++ks) {
+          const uint64_t aH = tc_desc(hi + offA + ks * 1024, BOX), aL = tc_desc(lo + offA + ks * 1024, BOX);
+          const uint64_t bH = tc_desc(hi + ks * 1024, BOX), bL = tc_desc(lo + ks * 1024, BOX);
+          tc_mma_tf32(tmem, aL, bH, idesc, fresh ^ 1u);
+          tc_mma_tf32(tmem, aH, bL, idesc, 1u);
+          tc_mma_tf32(tmem, aH, bH, idesc, 1u);
+          fresh = 0;
+        }
+        tc_commit(&op_empty[o]);
+        bool last;
+        if ((q & 1) && drain_after(q >> 1, &last)) {
+          tc_commit(&acc_full);
+          fresh = 1;
+          ++ndrain;
+        }
+      }
+    }
+  } else {
+    // ---------------------------------------------------------------- operand split + accumulator drain
+    float acc[B];
+#pragma unroll
+    for (int j = 0; j < B; ++j) acc[j] = 0.f;
+    int ndrain = 0;
+    bool ok = true;
+    for (int q = 0; q < nsub && ok; ++q) {
+      const int s = q % RS, o = q % OS;
+      if (!mbar_wait(&raw_full[s], (q / RS) & 1, ctrl)) break;
+      if (q >= OS && !mbar_wait(&op_empty[o], ((q / OS) - 1) & 1, ctrl)) break;
+      const float4* src = reinterpret_cast<const float4*>(smem + s * RAW);
+      float4* dhi = reinterpret_cast<float4*>(ops + o * OPS);
+      float4* dlo = reinterpret_cast<float4*>(ops + o * OPS + RAW);
+#pragma unroll 4
+      for (int idx = tid; idx < RAW / 16; idx += 128) {
+        const float4 x = src[idx];
+        float4 h, l;
+        h.x = __uint_as_float(to_tf32(x.x));
+        h.y = __uint_as_float(to_tf32(x.y));
+        h.z = __uint_as_float(to_tf32(x.z));
+        h.w = __uint_as_float(to_tf32(x.w));
+        l.x = __uint_as_float(to_tf32(x.x - h.x));
+        l.y = __uint_as_float(to_tf32(x.y - h.y));
+        l.z = __uint_as_float(to_tf32(x.z - h.z));
+        l.w = __uint_as_float(to_tf32(x.w - h.w));
+        dhi[idx] = h;
+        dlo[idx] = l;
+      }
+      proxy_fence_async_smem();      // the planes are read by the tensor core through the async proxy
+      __syncwarp();
+      if (lane == 0) {
+        mbar_arrive(&op_full[o]);
+        mbar_arrive(&raw_empty[s]);
+      }
+      bool last;
+      if ((q & 1) && drain_after(q >> 1, &last)) {
+        if (!mbar_wait(&acc_full, ndrain & 1, ctrl)) break;
+        ++ndrain;
+        tc_fence_after();
+        const uint32_t taddr = tmem + ((uint32_t)(warp * 32) << 16);
+#pragma unroll
+        for (int jj = 0; jj < B / 16; ++jj) {
+          float v[16];
+          tmem_ld16(taddr + jj * 16, v);
+#pragma unroll
+          for (int e = 0; e < 16; ++e) acc[jj * 16 + e] += v[e];
+        }
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&acc_empty);
+        if (last) {
+          const int c = (L0 + (q >> 1)) / KT;
+          float* dst = Zpart + (size_t)(p + c) * (size_t)(B * kTcBN) + warp * 32 + lane;
+#pragma unroll
+          for (int j = 0; j < B; ++j) {
+            dst[(size_t)j * kTcBN] = acc[j];
+            acc[j] = 0.f;
+          }
+        }
+      }
+    }
+  }
+  // common exit: nothing is in flight once the last accumulator has been drained (or a wait gave up)
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 0) tmem_dealloc(tmem, B);
+}
+
+}  // namespace rrf
