@@ -378,6 +378,10 @@ def main():
                     help="no-update: A is left unchanged and B is not formed (one pass over A per block instead of "
                          "three); stops on the sampled Frobenius estimate.  Flops are counted as the in-place schedule's")
     ap.add_argument("--estimator", type=int, default=0, choices=[0, 1, 2, 3])
+    ap.add_argument("--f32-engine", default="mma", choices=["mma", "tcgen05"],
+                    help="tensor-core path of the single-precision V^T W product")
+    ap.add_argument("--tc-chunk", type=int, default=2,
+                    help="tcgen05: 64-row tiles summed in tensor memory between round-to-nearest adds (0: all)")
     ap.add_argument("--panel-ctas", type=int, default=0, help="look-ahead schedule: SMs given to the panel chain (0: library's rule)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
@@ -411,6 +415,7 @@ def main():
     if world > 1:
         dist.barrier()
     h = rrf.rrf_create(local)
+    rrf.rrf_set_f32_engine(h, 1 if args.f32_engine == "tcgen05" else 0, args.tc_chunk)
     sched = {"auto": 0, "one": rrf.RRF_FLAG_ONE_QUEUE, "two": rrf.RRF_FLAG_TWO_QUEUES}[args.schedule]
     if args.panel == "tree":
         sched |= rrf.RRF_FLAG_PANEL_TREE

@@ -11,14 +11,15 @@
 //     kernel's in the swizzle mode (and in the box height).  No transposition anywhere.
 //   * fp32 accuracy comes from the same 3xTF32 split as the mma.sync path, x = hi + lo with
 //     hi = tf32(x), lo = tf32(x - hi), D += A_lo B_hi + A_hi B_lo + A_hi B_hi.  The split is an
-//     element-wise pass by four warps from the TMA ring into a second ring of (hi, lo) planes at
-//     the same byte offsets, so the swizzle never has to be decoded.
+//     element-wise pass by eight warps from the TMA ring into a second ring of (hi, lo) planes at
+//     the same byte offsets within a box, so the swizzle never has to be decoded.
 //   * The tensor core's own accumulation does not round to nearest.  `chunk` bounds how many
-//     64-row tiles are summed inside tensor memory before the four warps add the accumulator into
+//     64-row tiles are summed inside tensor memory before those warps add the accumulator into
 //     registers with ordinary round-to-nearest adds (0: a whole accumulator stays in tensor memory).
 //
-// Warp roles: 0-3 split operands and drain the accumulator (warp w owns tensor-memory lanes
-// 32w .. 32w+31, i.e. those columns of the tile), 4 issues TMA loads, 5 issues the MMAs.
+// Warp roles: 0-7 split operands and drain the accumulator (warp w owns tensor-memory lanes
+// 32 (w % 4) ..., i.e. those columns of the tile, and half w / 4 of the B rows of Z), 8 issues TMA
+// loads, 9 issues the MMAs.
 // Every wait is bounded; on a time-out all roles fall through to the common exit, where tensor
 // memory is released.
 #pragma once
@@ -89,15 +90,32 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, float (&v)[16]) {
 
 constexpr int kTcBN = 128;     // columns of W per accumulator = rows of D = tensor-memory lanes
 constexpr int kTcSub = 32;     // rows (contraction indices) per ring stage; a 64-row tile is two stages
-constexpr int kTcThreads = 192;
+constexpr int kTcConv = 8;     // warps that split operands and drain the accumulator
+constexpr int kTcThreads = (kTcConv + 2) * 32;
 
+__device__ __forceinline__ float4 lds128(uint32_t a) {
+  float4 v;
+  asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(a));
+  return v;
+}
+__device__ __forceinline__ void sts128(uint32_t a, const float4& v) {
+  asm volatile("st.shared.v4.f32 [%0], {%1,%2,%3,%4};" ::"r"(a), "f"(v.x), "f"(v.y), "f"(v.z), "f"(v.w) : "memory");
+}
+
+// One stage of the operand ring, in boxes of 32 lines x 128 bytes:
+//   [V_hi (NBV boxes)] [V_lo (NBV)] [W_hi (NBC)] [W_lo (NBC)]
+// V_lo follows V_hi at the box stride so that one descriptor covers [V_hi | V_lo] as an operand with
+// 2B columns: per K step  D[:, 0:2B] += W_hi^T [V_hi | V_lo]  and  D[:, 0:B] += W_lo^T V_hi  - two
+// instructions instead of three, and 14 KB instead of 18 KB read from shared memory (B = 64), which
+// is what bounds the tensor core here.  Columns j and B + j of the accumulator are added when it is drained.
 template <int B, int RS, int OS>
 struct TcCfg {
   static constexpr int NBV = B / 32, NBC = kTcBN / 32;
   static constexpr int BOX = kTcSub * 128;
   static constexpr int RAW = (NBV + NBC) * BOX;       // one stage of the TMA ring
-  static constexpr int OPS = 2 * RAW;                 // one stage of the operand ring: hi plane, lo plane
+  static constexpr int OPS = 2 * RAW;                 // one stage of the operand ring
   static constexpr int SMEM = RS * RAW + OS * OPS + 1024;
+  static constexpr int COLS = 2 * B;                  // tensor-memory columns of the accumulator
 };
 
 template <int B, int RS, int OS>
@@ -107,8 +125,9 @@ __global__ void __launch_bounds__(kTcThreads, 1)
                   float* __restrict__ Zpart, int r0, int cv0, int KT, int total, int tpc, int chunk, Ctrl* ctrl) {
   if (*reinterpret_cast<volatile int*>(&ctrl->done)) return;
   using Cfg = TcCfg<B, RS, OS>;
-  constexpr int NBV = Cfg::NBV, NBC = Cfg::NBC, BOX = Cfg::BOX, RAW = Cfg::RAW, OPS = Cfg::OPS;
+  constexpr int NBV = Cfg::NBV, NBC = Cfg::NBC, BOX = Cfg::BOX, RAW = Cfg::RAW, OPS = Cfg::OPS, COLS = Cfg::COLS;
   static_assert(B == 32 || B == 64 || B == 128, "tensor-memory columns: a power of two, at least 32");
+  static_assert(BOX / 16 == kTcConv * 32, "one 16-byte chunk of a box per converter thread");
 
   extern __shared__ unsigned char smem_raw[];
   unsigned char* smem = align1024(smem_raw);
@@ -125,18 +144,18 @@ __global__ void __launch_bounds__(kTcThreads, 1)
   if (tid == 0) {
     for (int s = 0; s < RS; ++s) {
       mbar_init(&raw_full[s], 1);
-      mbar_init(&raw_empty[s], 4);
+      mbar_init(&raw_empty[s], kTcConv);
     }
     for (int s = 0; s < OS; ++s) {
-      mbar_init(&op_full[s], 4);
+      mbar_init(&op_full[s], kTcConv);
       mbar_init(&op_empty[s], 1);
     }
     mbar_init(&acc_full, 1);
-    mbar_init(&acc_empty, 4);
+    mbar_init(&acc_empty, kTcConv);
     mbar_fence_init();
   }
   __syncthreads();
-  if (warp == 0) tmem_alloc(&tmem_slot, B);
+  if (warp == 0) tmem_alloc(&tmem_slot, COLS);
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
@@ -150,7 +169,7 @@ __global__ void __launch_bounds__(kTcThreads, 1)
     return *last_of_acc || (chunk > 0 && (kt + 1) % chunk == 0);
   };
 
-  if (warp == 4) {
+  if (warp == kTcConv) {
     // ---------------------------------------------------------------- TMA producer
     if (lane == 0) {
       for (int q = 0; q < nsub; ++q) {
@@ -167,10 +186,10 @@ __global__ void __launch_bounds__(kTcThreads, 1)
           tma_load_2d(dst + (NBV + cb) * BOX, &tmC, c * kTcBN + cb * 32, y, &raw_full[s]);
       }
     }
-  } else if (warp == 5) {
+  } else if (warp == kTcConv + 1) {
     // ---------------------------------------------------------------- MMA issuer
     if (lane == 0) {
-      constexpr uint32_t idesc = tc_idesc_tf32(kTcBN, B);
+      constexpr uint32_t idesc2 = tc_idesc_tf32(kTcBN, 2 * B), idesc1 = tc_idesc_tf32(kTcBN, B);
       uint32_t fresh = 1;        // the next product overwrites the accumulator
       int ndrain = 0;
       for (int q = 0; q < nsub; ++q) {
@@ -178,15 +197,11 @@ __global__ void __launch_bounds__(kTcThreads, 1)
         if (!mbar_wait(&op_full[o], (q / OS) & 1, ctrl)) break;
         if (fresh && ndrain > 0 && !mbar_wait(&acc_empty, (ndrain - 1) & 1, ctrl)) break;
         tc_fence_after();
-        const uint32_t hi = smem_u32(ops + o * OPS), lo = hi + RAW;
-        const uint32_t offA = NBV * BOX;       // the W tile follows the V tile in a stage
+        const uint32_t vH = smem_u32(ops + o * OPS), wH = vH + 2 * NBV * BOX, wL = wH + NBC * BOX;
 #pragma unroll
         for (int ks = 0; ks < kTcSub / 8; ++ks) {
-          const uint64_t aH = tc_desc(hi + offA + ks * 1024, BOX), aL = tc_desc(lo + offA + ks * 1024, BOX);
-          const uint64_t bH = tc_desc(hi + ks * 1024, BOX), bL = tc_desc(lo + ks * 1024, BOX);
-          tc_mma_tf32(tmem, aL, bH, idesc, fresh ^ 1u);
-          tc_mma_tf32(tmem, aH, bL, idesc, 1u);
-          tc_mma_tf32(tmem, aH, bH, idesc, 1u);
+          tc_mma_tf32(tmem, tc_desc(wH + ks * 1024, BOX), tc_desc(vH + ks * 1024, BOX), idesc2, fresh ^ 1u);
+          tc_mma_tf32(tmem, tc_desc(wL + ks * 1024, BOX), tc_desc(vH + ks * 1024, BOX), idesc1, 1u);
           fresh = 0;
         }
         tc_commit(&op_empty[o]);
@@ -200,32 +215,37 @@ __global__ void __launch_bounds__(kTcThreads, 1)
     }
   } else {
     // ---------------------------------------------------------------- operand split + accumulator drain
-    float acc[B];
+    // warp w drains lanes 32 (w % 4) ... of tensor memory (the hardware's rule) and half w / 4 of the B columns
+    constexpr int HB = B / 2;
+    const int quad = warp & 3, half = warp >> 2;
+    float acc[HB];
 #pragma unroll
-    for (int j = 0; j < B; ++j) acc[j] = 0.f;
+    for (int j = 0; j < HB; ++j) acc[j] = 0.f;
     int ndrain = 0;
-    bool ok = true;
-    for (int q = 0; q < nsub && ok; ++q) {
+    const uint32_t raw0 = smem_u32(smem) + tid * 16, op0 = smem_u32(ops) + tid * 16;
+    for (int q = 0; q < nsub; ++q) {
       const int s = q % RS, o = q % OS;
       if (!mbar_wait(&raw_full[s], (q / RS) & 1, ctrl)) break;
       if (q >= OS && !mbar_wait(&op_empty[o], ((q / OS) - 1) & 1, ctrl)) break;
-      const float4* src = reinterpret_cast<const float4*>(smem + s * RAW);
-      float4* dhi = reinterpret_cast<float4*>(ops + o * OPS);
-      float4* dlo = reinterpret_cast<float4*>(ops + o * OPS + RAW);
-#pragma unroll 4
-      for (int idx = tid; idx < RAW / 16; idx += 128) {
-        const float4 x = src[idx];
+      const uint32_t src = raw0 + s * RAW, dst = op0 + o * OPS;
+      float4 x[NBV + NBC];
+#pragma unroll
+      for (int bx = 0; bx < NBV + NBC; ++bx) x[bx] = lds128(src + bx * BOX);     // box bx, this thread's chunk
+#pragma unroll
+      for (int bx = 0; bx < NBV + NBC; ++bx) {
         float4 h, l;
-        h.x = __uint_as_float(to_tf32(x.x));
-        h.y = __uint_as_float(to_tf32(x.y));
-        h.z = __uint_as_float(to_tf32(x.z));
-        h.w = __uint_as_float(to_tf32(x.w));
-        l.x = __uint_as_float(to_tf32(x.x - h.x));
-        l.y = __uint_as_float(to_tf32(x.y - h.y));
-        l.z = __uint_as_float(to_tf32(x.z - h.z));
-        l.w = __uint_as_float(to_tf32(x.w - h.w));
-        dhi[idx] = h;
-        dlo[idx] = l;
+        h.x = __uint_as_float(to_tf32(x[bx].x));
+        h.y = __uint_as_float(to_tf32(x[bx].y));
+        h.z = __uint_as_float(to_tf32(x[bx].z));
+        h.w = __uint_as_float(to_tf32(x[bx].w));
+        l.x = __uint_as_float(to_tf32(x[bx].x - h.x));
+        l.y = __uint_as_float(to_tf32(x[bx].y - h.y));
+        l.z = __uint_as_float(to_tf32(x[bx].z - h.z));
+        l.w = __uint_as_float(to_tf32(x[bx].w - h.w));
+        const int hb = bx < NBV ? bx : 2 * NBV + (bx - NBV);          // box of the hi plane in the operand stage
+        const int lb = bx < NBV ? bx + NBV : 2 * NBV + NBC + (bx - NBV);
+        sts128(dst + hb * BOX, h);
+        sts128(dst + lb * BOX, l);
       }
       proxy_fence_async_smem();      // the planes are read by the tensor core through the async proxy
       __syncwarp();
@@ -238,23 +258,24 @@ __global__ void __launch_bounds__(kTcThreads, 1)
         if (!mbar_wait(&acc_full, ndrain & 1, ctrl)) break;
         ++ndrain;
         tc_fence_after();
-        const uint32_t taddr = tmem + ((uint32_t)(warp * 32) << 16);
+        const uint32_t taddr = tmem + ((uint32_t)(quad * 32) << 16) + half * HB;
 #pragma unroll
-        for (int jj = 0; jj < B / 16; ++jj) {
-          float v[16];
+        for (int jj = 0; jj < HB / 16; ++jj) {
+          float v[16], w[16];
           tmem_ld16(taddr + jj * 16, v);
+          tmem_ld16(taddr + B + jj * 16, w);
 #pragma unroll
-          for (int e = 0; e < 16; ++e) acc[jj * 16 + e] += v[e];
+          for (int e = 0; e < 16; ++e) acc[jj * 16 + e] += v[e] + w[e];
         }
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(&acc_empty);
         if (last) {
           const int c = (L0 + (q >> 1)) / KT;
-          float* dst = Zpart + (size_t)(p + c) * (size_t)(B * kTcBN) + warp * 32 + lane;
+          float* out = Zpart + (size_t)(p + c) * (size_t)(B * kTcBN) + (size_t)(half * HB) * kTcBN + quad * 32 + lane;
 #pragma unroll
-          for (int j = 0; j < B; ++j) {
-            dst[(size_t)j * kTcBN] = acc[j];
+          for (int j = 0; j < HB; ++j) {
+            out[(size_t)j * kTcBN] = acc[j];
             acc[j] = 0.f;
           }
         }
@@ -264,7 +285,7 @@ __global__ void __launch_bounds__(kTcThreads, 1)
   // common exit: nothing is in flight once the last accumulator has been drained (or a wait gave up)
   tc_fence_before();
   __syncthreads();
-  if (warp == 0) tmem_dealloc(tmem, B);
+  if (warp == 0) tmem_dealloc(tmem, COLS);
 }
 
 }  // namespace rrf
