@@ -12,6 +12,7 @@
 
 #include "gemm_sk.cuh"
 #include "gemm_tc.cuh"
+#include "gemm_tc_upd.cuh"
 #include "panel_blk.cuh"
 
 // NVTX ranges around the phases of rrf_run (host-side enqueue order), compiled in with -DRRF_NVTX only
@@ -125,7 +126,21 @@ static VtwPlan plan_vtw(int sms, long long rows, long long ncols, int bn) {
   return p;
 }
 // stream-K plan of the fused update: tiles (row slab, column tile)
-struct UpdPlan { int NS, NC, total, tpc, P, slots; };
+// what the tcgen05 version of the fused update needs beyond the common arguments
+struct UpdTc {
+  const void* V;          // reflectors (read directly, not through a tensor map)
+  long long ldv;
+  const void* Zt;         // [npad][b], written by the T Z kernel
+  int npad;
+  const void* Om;         // OmegaT as the run sees it
+  long long ldom;
+  void* zsplit;           // [2][npad][b]: TF32 planes of Zt
+  void* osplit;           // [2][b][ldo2]: TF32 planes of the rows of OmegaT being sampled with
+  long long ldo2;
+  int chunk;
+  CUtensorMap tmZs, tmOs;
+};
+struct UpdPlan { int NS, NC, total, tpc, P, slots; const UpdTc* tc; };
 static UpdPlan plan_upd(int sms, long long rows, long long ncols, int bm, int bn, int wn) {
   UpdPlan p;
   p.NS = ceil_div(rows, bm);
@@ -134,6 +149,7 @@ static UpdPlan plan_upd(int sms, long long rows, long long ncols, int bm, int bn
   p.tpc = ceil_div(p.total, sms);
   p.P = ceil_div(p.total, p.tpc);
   p.slots = (p.P + p.NS) * wn;
+  p.tc = nullptr;
   return p;
 }
 // The panel kernel's variants: rows a lane keeps in registers, row groups, and whether the slab is
@@ -434,6 +450,8 @@ struct Ops {
   static constexpr int U_STAGES = (U_VBYTES + 3 * U_STAGE + 1024 <= 226 * 1024) ? 3 : 2;
   static constexpr int U_SMEM = U_VBYTES + U_STAGES * U_STAGE + 1024;
   static constexpr bool U_PW = false;   // the widest fp64 block needs the registers of 8 warps
+  // fused update on tcgen05: single precision, 128-row slabs and 64-column tiles (the same as above for b <= 64)
+  static constexpr bool kHasUpdTc = std::is_same<T, float>::value && B <= 64 && U_BM == kUtcBM && U_BN == kUtcBN && U_WN == 1;
   static_assert(U_SMEM + 1024 <= kMaxSmem && V_SMEM + 1024 <= kMaxSmem && S_SMEM + 1024 <= kMaxSmem, "shared memory");
 
   static cudaError_t setup() {
@@ -450,6 +468,10 @@ struct Ops {
     if constexpr (std::is_same<T, float>::value) {
       e = cudaFuncSetAttribute(vtw_tc_kernel<B, TC_RS, TC_OS>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                TcCfg<B, TC_RS, TC_OS>::SMEM);
+      if (e != cudaSuccess) return e;
+    }
+    if constexpr (kHasUpdTc) {
+      e = cudaFuncSetAttribute(upd_tc_kernel<B>, cudaFuncAttributeMaxDynamicSharedMemorySize, UtcCfg<B>::SMEM);
       if (e != cudaSuccess) return e;
     }
     e = cudaFuncSetAttribute(tz_kernel<T, B>, cudaFuncAttributeMaxDynamicSharedMemorySize, Z_SMEM);
@@ -483,6 +505,20 @@ struct Ops {
                      void* C, long long ldc, void* top, long long ldtop, int r0, int rows, int ncols, int cv0,
                      int top_rows, int j0, void* Ypart, double* norm_part, const UpdPlan& p, Ctrl* ctrl,
                      const int* samp_flag, cudaStream_t st) {
+    if constexpr (kHasUpdTc) {
+      if (p.tc != nullptr) {
+        const UpdTc& x = *p.tc;
+        split_planes_kernel<<<std::min(1024, ceil_div((long long)x.npad * B, 256)), 256, 0, st>>>(
+            (const float*)x.Zt, B, x.npad, B, (float*)x.zsplit, B, &ctrl->done);
+        if (j0 >= 0)
+          split_planes_kernel<<<std::min(1024, ceil_div((long long)ncols * B, 256)), 256, 0, st>>>(
+              (const float*)x.Om + (size_t)j0 * x.ldom, x.ldom, B, ncols, (float*)x.osplit, x.ldo2, &ctrl->done);
+        upd_tc_kernel<B><<<p.P, kUtcThreads, UtcCfg<B>::SMEM, st>>>(
+            tmC, x.tmZs, x.tmOs, (const float*)x.V, x.ldv, (float*)C, ldc, (float*)top, ldtop, r0, rows, ncols, cv0,
+            top_rows, j0 >= 0 ? 1 : 0, x.npad, (float*)Ypart, norm_part, p.NC, p.total, p.tpc, x.chunk, ctrl);
+        return;
+      }
+    }
     upd_sk_kernel<T, B, U_BM, U_BNB, U_WM, U_WN, U_STAGES, U_PW><<<p.P, (U_PW ? 9 : 8) * 32, U_SMEM, st>>>(
         tmV, tmZ, tmC, tmO, (T*)C, ldc, (T*)top, ldtop, r0, rows, ncols, cv0, top_rows, j0, (T*)Ypart, norm_part, p.NC,
         p.total, p.tpc, ctrl, samp_flag);
@@ -490,7 +526,7 @@ struct Ops {
 };
 
 struct OpTable {
-  int s_kbs, v_bn, u_bm, u_bn, u_wn;
+  int s_kbs, v_bn, u_bm, u_bn, u_wn, has_upd_tc;
   cudaError_t (*setup)();
   void (*sample)(const CUtensorMap&, const CUtensorMap&, void*, int, int, int, int, const SamplePlan&, Ctrl*,
                  const int*, double*, cudaStream_t);
@@ -502,7 +538,7 @@ struct OpTable {
 };
 template <typename T, int B>
 static OpTable make_ops() {
-  return OpTable{Ops<T, B>::S_KBS, Ops<T, B>::V_BN, Ops<T, B>::U_BM, Ops<T, B>::U_BN, Ops<T, B>::U_WN, &Ops<T, B>::setup, &Ops<T, B>::sample,
+  return OpTable{Ops<T, B>::S_KBS, Ops<T, B>::V_BN, Ops<T, B>::U_BM, Ops<T, B>::U_BN, Ops<T, B>::U_WN, Ops<T, B>::kHasUpdTc ? 1 : 0, &Ops<T, B>::setup, &Ops<T, B>::sample,
                  &Ops<T, B>::vtw,  &Ops<T, B>::tz, &Ops<T, B>::update};
 }
 static const OpTable* get_ops(int dtype, int b) {
@@ -722,9 +758,14 @@ static cudaError_t setup_all(int smem_optin, int* panel_smem_max) {
   return setup_panel_kernels(smem_optin, panel_smem_max);
 }
 
+static size_t tc_zsplit_bytes(int npad, int b) { return align_up((size_t)2 * npad * b * sizeof(float), 256); }
+static size_t tc_split_bytes(int npad, int b, long long n) {
+  return tc_zsplit_bytes(npad, b) + align_up((size_t)2 * b * align_up((size_t)n, 4) * sizeof(float), 256);
+}
+
 // ------------------------------------------------------------------ workspace of rrf_run
 struct RunLayout {
-  size_t ctrl, traces, done_after, norm_part, init_part, ypart, ypart2, zpart, zt, panel, look, csq, w, omega, total;
+  size_t ctrl, traces, done_after, norm_part, init_part, ypart, ypart2, zpart, zt, tcsplit, panel, look, csq, w, omega, total;
   int init_ctas, max_norm_parts;
   long long ldw;
 };
@@ -758,6 +799,8 @@ static bool run_layout(const rrf_params_t* p, bool need_omega, RunLayout* L) {
   L->ypart2 = off; off += align_up(ymax * esize, 256);   // the look-ahead schedule keeps two sampled panels
   L->zpart = off; off += align_up(zmax * esize, 256);
   L->zt = off; off += align_up((size_t)npad * b * esize, 256);
+  L->tcsplit = off;      // single precision: TF32 planes of Zt and of b rows of OmegaT for the tcgen05 update
+  if (ops->has_upd_tc) off += tc_split_bytes(npad, b, p->n);
   L->panel = off; off += panel_scratch_bytes(sms, b, p->m);
   L->look = off; off += look_scratch_bytes(b);
   L->csq = off; off += align_up((size_t)2 * b * ((sms + 31) / 32 * 32) * sizeof(double), 256);   // two panels in flight
@@ -1075,6 +1118,7 @@ rrf_status_t rrf_apply_workspace_bytes(int32_t dtype, int64_t m, int64_t ncols, 
   const VtwPlan vp = plan_vtw(kMaxSms, m, ncols, get_ops(dtype, b)->v_bn);
   const size_t zslots = (size_t)(kMaxSms + vp.nct) * b * vp.bn;
   *bytes = align_up((size_t)vp.npad * b * esize, 256) + align_up(zslots * esize, 256);
+  if (get_ops(dtype, b)->has_upd_tc) *bytes += tc_zsplit_bytes(vp.npad, b);
   return RRF_OK;
 }
 
@@ -1109,6 +1153,18 @@ static rrf_status_t apply_blocks(rrf_handle_t h, int dtype, long long m, int b, 
       !make_map(h, &tmV_u, dtype, dV, m, k, ldv, ops->u_bm) || !make_map(h, &tmC_u, dtype, dC, m, ncols, ldc, ops->u_bm) ||
       !make_map(h, &tmZ, dtype, Zt, vp0.npad, b, b, ops->u_bn))
     return RRF_ERR_INVALID_ARG;
+  UpdTc utc{};
+  const bool utc_on = tc && ops->has_upd_tc;
+  if (utc_on) {
+    utc.V = dV;
+    utc.ldv = ldv;
+    utc.Zt = Zt;
+    utc.npad = vp0.npad;
+    utc.zsplit = (unsigned char*)Zpart + align_up((size_t)(kMaxSms + vp0.nct) * b * vp0.bn * esize, 256);
+    utc.chunk = h->tc_chunk;
+    if (!make_map(h, &utc.tmZs, dtype, utc.zsplit, 2ull * vp0.npad, b, b, kUtcBN)) return RRF_ERR_INVALID_ARG;
+    utc.tmOs = utc.tmZs;   // not read: nothing is sampled here
+  }
   const int nblk = k / b;
   for (int q = 0; q < nblk; ++q) {
     const int l = transpose ? q : nblk - 1 - q;
@@ -1118,7 +1174,8 @@ static rrf_status_t apply_blocks(rrf_handle_t h, int dtype, long long m, int b, 
     vp.chunk = h->tc_chunk;
     ops->vtw(tmV_k, tmC_k, Zpart, r0, r0, vp, h->d_ctrl, st);
     ops->tz(Zpart, vp, (const char*)dT + (size_t)r0 * esize, ldt, transpose ? 1 : 0, Zt, &h->d_ctrl->done, st);
-    const UpdPlan up = plan_upd(h->sms, rows, ncols, ops->u_bm, ops->u_bn, ops->u_wn);
+    UpdPlan up = plan_upd(h->sms, rows, ncols, ops->u_bm, ops->u_bn, ops->u_wn);
+    if (utc_on) up.tc = &utc;
     ops->update(tmV_u, tmZ, tmC_u, tmC_u, dC, ldc, dC, ldc, r0, rows, (int)ncols, r0, 0, -1, nullptr, nullptr, up,
                 h->d_ctrl, nullptr, st);
   }
@@ -1353,6 +1410,23 @@ rrf_status_t rrf_run(rrf_handle_t h, const rrf_params_t* p, void* dA, int64_t ld
       !make_map(h, &tmW_u, p->dtype, W, m, n, ldw, ops->u_bm) ||
       !make_map(h, &tmZ, p->dtype, Zt, npad, b, b, ops->u_bn))
     return RRF_ERR_INVALID_ARG;
+  UpdTc utc{};
+  const bool utc_on = tc && ops->has_upd_tc;
+  if (utc_on) {
+    utc.V = dV;
+    utc.ldv = ldv;
+    utc.Zt = Zt;
+    utc.npad = npad;
+    utc.Om = Om;
+    utc.ldom = ldom;
+    utc.zsplit = ws + L.tcsplit;
+    utc.osplit = ws + L.tcsplit + tc_zsplit_bytes(npad, b);
+    utc.ldo2 = (long long)align_up((size_t)n, 4);
+    utc.chunk = h->tc_chunk;
+    if (!make_map(h, &utc.tmZs, p->dtype, utc.zsplit, 2ull * npad, b, b, kUtcBN) ||
+        !make_map(h, &utc.tmOs, p->dtype, utc.osplit, 2ull * b, n, utc.ldo2, b))
+      return RRF_ERR_INVALID_ARG;
+  }
 
   // profiling: one event before every kernel, tagged with (phase, block step)
   bool nvtx_open = false;
@@ -1495,7 +1569,8 @@ rrf_status_t rrf_run(rrf_handle_t h, const rrf_params_t* p, void* dA, int64_t ld
       mark(RRF_PHASE_TZ, i);
       cudaStreamWaitEvent(st, h->sync_events[2 * i + 1], 0);   // join: T_i is needed from here on
       ops->tz(Zpart, vp, Tblk(r0), p->max_rank, 1, Zt, &ctrl->done, st);
-      const UpdPlan up = plan_upd(h->sms, rows, n, ops->u_bm, ops->u_bn, ops->u_wn);
+      UpdPlan up = plan_upd(h->sms, rows, n, ops->u_bm, ops->u_bn, ops->u_wn);
+      if (utc_on) up.tc = &utc;
       const int j0 = (i + 1 < steps) ? r0 + b : -1;   // Omega rows of the next pass, if there is one
       mark(RRF_PHASE_UPDATE, i);
       ops->update(tmV_u, tmZ, i == 0 ? tmA_u : tmW_u, tmO, W, ldw, (char*)dB + (size_t)r0 * ldb * esize, ldb, r0, rows, (int)n, r0, b,
@@ -1634,7 +1709,8 @@ rrf_status_t rrf_run(rrf_handle_t h, const rrf_params_t* p, void* dA, int64_t ld
         s = next_panel();
         if (s != RRF_OK) return panel_failed(s);
       }
-      const UpdPlan up = plan_upd(gsms, rows, n, ops->u_bm, ops->u_bn, ops->u_wn);
+      UpdPlan up = plan_upd(gsms, rows, n, ops->u_bm, ops->u_bn, ops->u_wn);
+      if (utc_on) up.tc = &utc;
       const int j0 = (i + 2 < steps) ? r0 + 2 * b : -1;   // Omega rows of the pass after the next
       mark(RRF_PHASE_UPDATE, i);
       ops->update(tmV_u, tmZ, i == 0 ? tmA_u : tmW_u, tmO, W, ldw, (char*)dB + (size_t)r0 * ldb * esize, ldb, r0, rows, (int)n, r0, b,

@@ -1,0 +1,400 @@
+// Single-precision fused update of a block step (Algorithm 2 line 8, second product, with the norms
+// of line 9 and the next sample of line 7) on the fifth-generation tensor cores.
+//
+// Same tiles (row slab of 128, column tile of 64), same stream-K ranges, same output slots and the
+// same norm partials as upd_sk_kernel.  Per tile:
+//   P     = V[slab, :] Zt[tile, :]^T                  K = B      (GEMM 1)
+//   Wnew  = W[slab, tile] - P  -> global memory, sums of squares for the norms
+//   Y    += Wnew OmegaT[j0 .. j0+B, tile]^T           K = 64     (GEMM 2, only if j0 >= 0)
+// The left operand of both products sits in TENSOR MEMORY (lane = row of the slab, one column per
+// contraction index): V is written there once per slab, Wnew once per tile by the very threads that
+// compute it, each split into its two TF32 planes on the way.  The right operands are Zt and OmegaT
+// rows, which arrive by TMA already split (split_planes_kernel wrote the planes to global memory:
+// both are small and stay in L2), K-contiguous with the ordinary 128-byte swizzle.  So shared memory
+// carries only what TMA brings - W, Zt planes, OmegaT planes - and is read once by the tensor core
+// and (W) once by the epilogue: about 220 KB of shared-memory traffic per 64 KB of HBM traffic.
+//
+// 3xTF32 as everywhere: D += A_lo B_hi + A_hi B_lo + A_hi B_hi.  The accumulator of P lives for one
+// tile (K = B), that of Y for `chunk` tiles before it is added, rounded to nearest, into registers.
+//
+// Warp roles: 0-7 epilogue (warp w owns tensor-memory lanes 32 (w % 4) ... = those rows of the slab,
+// and columns 32 (w / 4) ... of the tile = one TMA box of W), 8 TMA producer, 9 MMA issuer.
+// Tensor-memory columns: [V_hi V_lo | Wnew_hi Wnew_lo | P even tile, P odd tile | Y].
+#pragma once
+
+#include "gemm_tc.cuh"
+
+namespace rrf {
+
+// dst[0][r][c] = tf32(src[r][c]), dst[1][r][c] = tf32(src[r][c] - dst[0][r][c]); dst planes have leading dimension ldd
+__global__ void split_planes_kernel(const float* __restrict__ src, long long lds, int rows, int cols,
+                                    float* __restrict__ dst, long long ldd, const int* __restrict__ done_flag) {
+  if (done_flag != nullptr && *done_flag) return;
+  const long long total = (long long)rows * cols;
+  const size_t plane = (size_t)rows * (size_t)ldd;
+  for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < total; i += (long long)gridDim.x * blockDim.x) {
+    const int r = (int)(i / cols), c = (int)(i - (long long)r * cols);
+    const float x = src[(size_t)r * lds + c];
+    const float h = __uint_as_float(to_tf32(x));
+    dst[(size_t)r * ldd + c] = h;
+    dst[plane + (size_t)r * ldd + c] = __uint_as_float(to_tf32(x - h));
+  }
+}
+
+// K-contiguous shared-memory operand with the 128-byte swizzle: rows of 128 bytes, groups of eight rows 1024 bytes apart
+__device__ __forceinline__ uint64_t tc_desc_k(uint32_t addr) {
+  return (uint64_t)((addr & 0x3FFFFu) >> 4) | ((uint64_t)1 << 16) | ((uint64_t)(1024u >> 4) << 32) | (1ull << 46) |
+         (2ull << 61);
+}
+__host__ __device__ constexpr uint32_t tc_idesc_tf32_k(int M, int N) {
+  return (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
+}
+// D (+)= A B with A in tensor memory (lane = row, column = contraction index)
+__device__ __forceinline__ void tc_mma_tf32_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::tf32 [%0], [%1], %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "r"(a_tmem), "l"(b), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+// 16 consecutive columns of this thread's tensor-memory lane <- registers
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const float (&v)[16]) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};"
+      ::"r"(taddr), "r"(__float_as_uint(v[0])), "r"(__float_as_uint(v[1])), "r"(__float_as_uint(v[2])),
+        "r"(__float_as_uint(v[3])), "r"(__float_as_uint(v[4])), "r"(__float_as_uint(v[5])), "r"(__float_as_uint(v[6])),
+        "r"(__float_as_uint(v[7])), "r"(__float_as_uint(v[8])), "r"(__float_as_uint(v[9])), "r"(__float_as_uint(v[10])),
+        "r"(__float_as_uint(v[11])), "r"(__float_as_uint(v[12])), "r"(__float_as_uint(v[13])), "r"(__float_as_uint(v[14])),
+        "r"(__float_as_uint(v[15]))
+      : "memory");
+}
+__device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+
+constexpr int kUtcBM = 128, kUtcBN = 64;
+constexpr int kUtcEpi = 8;
+constexpr int kUtcThreads = (kUtcEpi + 2) * 32;
+
+template <int B>
+struct UtcCfg {
+  static constexpr int W_BOX = kUtcBM * 128;            // 128 rows x 32 columns
+  static constexpr int W_BYTES = 2 * W_BOX;
+  static constexpr int Z_BOX = kUtcBN * 128;            // 64 rows of Zt (columns of the tile) x 32 contraction indices
+  static constexpr int KBZ = B / 32;
+  static constexpr int Z_BYTES = KBZ * 2 * Z_BOX;       // per K box: hi rows, then lo rows
+  static constexpr int O_BOX = B * 128;                 // B rows of OmegaT x 32 columns of the tile
+  static constexpr int O_BYTES = 2 * 2 * O_BOX;         // per K box (two of them): hi rows, then lo rows
+  static constexpr int STAGE = W_BYTES + Z_BYTES + O_BYTES;
+  static constexpr int STAGES = (3 * STAGE + 1024 <= 220 * 1024) ? 3 : 2;
+  static constexpr int SMEM = STAGES * STAGE + 1024;
+  static constexpr int TV = 0, TW = 2 * B, TD = TW + 2 * kUtcBN, TY = TD + 2 * kUtcBN;   // tensor-memory columns
+  static constexpr int COLS = 512;
+  static_assert(TY + B <= COLS, "tensor memory");
+};
+
+template <int B>
+__global__ void __launch_bounds__(kUtcThreads, 1)
+    upd_tc_kernel(const __grid_constant__ CUtensorMap tmC,   // C [m][ncols], box [128][32]
+                  const __grid_constant__ CUtensorMap tmZs,  // Zt planes [2 npad][B], box [64][32]
+                  const __grid_constant__ CUtensorMap tmOs,  // OmegaT planes [2 B][n], box [B][32]
+                  const float* __restrict__ V, long long ldv, float* __restrict__ C, long long ldc,
+                  float* __restrict__ top, long long ldtop, int r0, int rows, int ncols, int cv0, int top_rows,
+                  int sample, int npad, float* __restrict__ Ypart, double* __restrict__ norm_part,
+                  int NC, int total, int tpc, int chunk, Ctrl* ctrl) {
+  if (*reinterpret_cast<volatile int*>(&ctrl->done)) return;
+  using Cfg = UtcCfg<B>;
+  constexpr int S = Cfg::STAGES, STAGE = Cfg::STAGE, W_BOX = Cfg::W_BOX, W_BYTES = Cfg::W_BYTES, Z_BOX = Cfg::Z_BOX,
+                Z_BYTES = Cfg::Z_BYTES, O_BOX = Cfg::O_BOX, KBZ = Cfg::KBZ;
+  constexpr int TV = Cfg::TV, TW = Cfg::TW, TD = Cfg::TD, TY = Cfg::TY;
+  constexpr int BN = kUtcBN, BM = kUtcBM;
+  static_assert(B == 32 || B == 64, "block sizes with a 128-row slab");
+
+  extern __shared__ unsigned char smem_raw[];
+  unsigned char* smem = align1024(smem_raw);
+  __shared__ uint64_t full[S], empty[S], v_ready, d_full[2], d_empty[2], w_ready, w_empty, y_full, y_empty;
+  __shared__ uint32_t tmem_slot;
+  __shared__ double red[64];
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int p = blockIdx.x;
+  const int L0 = p * tpc;
+  const int ntile = min(total, L0 + tpc) - L0;
+  const bool do_sample = sample != 0;
+
+  if (tid == 0) {
+    for (int s = 0; s < S; ++s) {
+      mbar_init(&full[s], 1);
+      mbar_init(&empty[s], kUtcEpi + 1);
+    }
+    mbar_init(&v_ready, kUtcEpi);
+    for (int s = 0; s < 2; ++s) {
+      mbar_init(&d_full[s], 1);
+      mbar_init(&d_empty[s], kUtcEpi);
+    }
+    mbar_init(&w_ready, kUtcEpi);
+    mbar_init(&w_empty, 1);
+    mbar_init(&y_full, 1);
+    mbar_init(&y_empty, kUtcEpi);
+    mbar_fence_init();
+  }
+  __syncthreads();
+  if (warp == 0) tmem_alloc(&tmem_slot, Cfg::COLS);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = *reinterpret_cast<volatile uint32_t*>(&tmem_slot);
+
+  // The Y accumulator is drained after the tile in column c of a slab if that tile ends the slab (or this CTA's
+  // range), or closes a chunk.  Writer and reader of the accumulator both use this rule.
+  auto drain_after = [&](int i, bool* last) {
+    const int L = L0 + i, s = L / NC, c = L - s * NC;
+    *last = (i == ntile - 1) || (c == NC - 1);
+    return *last || (chunk > 0 && (c + 1) % chunk == 0);
+  };
+
+  double s_top = 0.0, s_trail = 0.0;
+
+  if (warp == kUtcEpi) {
+    // ---------------------------------------------------------------- TMA producer
+    if (lane == 0) {
+      for (int i = 0; i < ntile; ++i) {
+        const int st = i % S;
+        if (i >= S && !mbar_wait(&empty[st], ((i / S) - 1) & 1, ctrl)) break;
+        const int L = L0 + i, s = L / NC, c = L - s * NC;
+        unsigned char* sW = smem + st * STAGE;
+        unsigned char* sZ = sW + W_BYTES;
+        unsigned char* sO = sZ + Z_BYTES;
+        mbar_expect_tx(&full[st], do_sample ? STAGE : W_BYTES + Z_BYTES);
+#pragma unroll
+        for (int q = 0; q < 2; ++q) tma_load_2d(sW + q * W_BOX, &tmC, c * BN + q * 32, r0 + s * BM, &full[st]);
+#pragma unroll
+        for (int kb = 0; kb < KBZ; ++kb) {
+          tma_load_2d(sZ + kb * 2 * Z_BOX, &tmZs, kb * 32, c * BN, &full[st]);
+          tma_load_2d(sZ + kb * 2 * Z_BOX + Z_BOX, &tmZs, kb * 32, npad + c * BN, &full[st]);
+        }
+        if (do_sample) {
+#pragma unroll
+          for (int q = 0; q < 2; ++q) {
+            tma_load_2d(sO + q * 2 * O_BOX, &tmOs, c * BN + q * 32, 0, &full[st]);
+            tma_load_2d(sO + q * 2 * O_BOX + O_BOX, &tmOs, c * BN + q * 32, B, &full[st]);
+          }
+        }
+      }
+    }
+  } else if (warp == kUtcEpi + 1) {
+    // ---------------------------------------------------------------- MMA issuer
+    if (lane == 0) {
+      constexpr uint32_t idescP = tc_idesc_tf32_k(BM, BN), idescY = tc_idesc_tf32_k(BM, B);
+      uint32_t fresh_y = 1;
+      int ny = 0, cur_s = -1, nslab = 0;
+      bool ok = true;
+      // Y += Wnew(i) OmegaT^T
+      auto gemm2 = [&](int i) {
+        const int st = i % S;
+        if (!mbar_wait(&w_ready, i & 1, ctrl)) { ok = false; return; }
+        if (fresh_y && ny > 0 && !mbar_wait(&y_empty, (ny - 1) & 1, ctrl)) { ok = false; return; }
+        tc_fence_after();
+        const uint32_t sO = smem_u32(smem + st * STAGE + W_BYTES + Z_BYTES);
+#pragma unroll
+        for (int ks = 0; ks < BN / 8; ++ks) {
+          const uint32_t oh = sO + (ks / 4) * 2 * O_BOX + (ks % 4) * 32, ol = oh + O_BOX;
+          const uint32_t ah = tmem + TW + ks * 8, al = ah + BN;
+          tc_mma_tf32_ts(tmem + TY, al, tc_desc_k(oh), idescY, fresh_y ^ 1u);
+          tc_mma_tf32_ts(tmem + TY, ah, tc_desc_k(ol), idescY, 1u);
+          tc_mma_tf32_ts(tmem + TY, ah, tc_desc_k(oh), idescY, 1u);
+          fresh_y = 0;
+        }
+        tc_commit(&w_empty);
+        tc_commit(&empty[st]);
+        bool last;
+        if (drain_after(i, &last)) {
+          tc_commit(&y_full);
+          fresh_y = 1;
+          ++ny;
+        }
+      };
+      for (int i = 0; i < ntile && ok; ++i) {
+        const int st = i % S, buf = i & 1;
+        const int L = L0 + i, s = L / NC;
+        bool last;
+        // a tile after which Y is drained (and a slab change, which always follows one) must not wait behind
+        // the next tile's first product: the epilogue warps stand at that drain
+        const bool early = do_sample && i > 0 && drain_after(i - 1, &last);
+        if (early) gemm2(i - 1);
+        if (!ok) break;
+        if (!mbar_wait(&full[st], (i / S) & 1, ctrl)) break;
+        if (s != cur_s) {
+          if (!mbar_wait(&v_ready, nslab & 1, ctrl)) break;
+          ++nslab;
+          cur_s = s;
+        }
+        if (i >= 2 && !mbar_wait(&d_empty[buf], ((i >> 1) - 1) & 1, ctrl)) break;
+        tc_fence_after();
+        const uint32_t sZ = smem_u32(smem + st * STAGE + W_BYTES);
+#pragma unroll
+        for (int ks = 0; ks < B / 8; ++ks) {
+          const uint32_t zh = sZ + (ks / 4) * 2 * Z_BOX + (ks % 4) * 32, zl = zh + Z_BOX;
+          const uint32_t ah = tmem + TV + ks * 8, al = ah + B;
+          const uint32_t d = tmem + TD + buf * BN;
+          tc_mma_tf32_ts(d, al, tc_desc_k(zh), idescP, ks > 0 ? 1u : 0u);
+          tc_mma_tf32_ts(d, ah, tc_desc_k(zl), idescP, 1u);
+          tc_mma_tf32_ts(d, ah, tc_desc_k(zh), idescP, 1u);
+        }
+        tc_commit(&d_full[buf]);
+        if (!do_sample) tc_commit(&empty[st]);
+        if (do_sample && i > 0 && !early) gemm2(i - 1);
+      }
+      if (ok && do_sample && ntile > 0) gemm2(ntile - 1);
+    }
+  } else {
+    // ---------------------------------------------------------------- epilogue warps
+    constexpr int HB = B / 2;                  // this warp's columns of V and of Y
+    const int quad = warp & 3, half = warp >> 2;
+    const int r = quad * 32 + lane;            // row inside the slab = tensor-memory lane
+    const uint32_t tlane = tmem + ((uint32_t)(quad * 32) << 16);
+    float accY[HB];
+#pragma unroll
+    for (int j = 0; j < HB; ++j) accY[j] = 0.f;
+    int cur_s = -1, ny = 0;
+    float* rowp = nullptr;
+    bool is_top = false;
+    for (int i = 0; i < ntile; ++i) {
+      const int st = i % S, buf = i & 1;
+      const int L = L0 + i, s = L / NC, c = L - s * NC;
+      if (s != cur_s) {
+        // V[slab] -> tensor memory, split (every product of the previous slab that reads it is complete: the
+        // accumulator of its last tile has been drained)
+        const int lr = s * BM + r;
+        const float* vrow = V + (size_t)(r0 + lr) * ldv + cv0 + half * HB;
+#pragma unroll
+        for (int g = 0; g < HB / 16; ++g) {
+          float hi[16], lo[16];
+#pragma unroll
+          for (int e4 = 0; e4 < 4; ++e4) {
+            float4 x = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (lr < rows) x = *reinterpret_cast<const float4*>(vrow + g * 16 + e4 * 4);
+            const float xs[4] = {x.x, x.y, x.z, x.w};
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+              hi[e4 * 4 + e] = __uint_as_float(to_tf32(xs[e]));
+              lo[e4 * 4 + e] = __uint_as_float(to_tf32(xs[e] - hi[e4 * 4 + e]));
+            }
+          }
+          tmem_st16(tlane + TV + half * HB + g * 16, hi);
+          tmem_st16(tlane + TV + B + half * HB + g * 16, lo);
+        }
+        tmem_st_wait();
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&v_ready);
+        cur_s = s;
+        is_top = lr < top_rows;
+        rowp = lr >= rows ? nullptr : (is_top ? top + (size_t)lr * ldtop : C + (size_t)(r0 + lr) * ldc);
+      }
+      if (!mbar_wait(&full[st], (i / S) & 1, ctrl)) break;
+      if (!mbar_wait(&d_full[buf], (i >> 1) & 1, ctrl)) break;
+      tc_fence_after();
+      float y[32];
+      {
+        float pa[16], pb[16];
+        tmem_ld16(tlane + TD + buf * BN + half * 32, pa);
+        tmem_ld16(tlane + TD + buf * BN + half * 32 + 16, pb);
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&d_empty[buf]);
+        const uint32_t sW = smem_u32(smem + st * STAGE + half * W_BOX + r * 128);
+#pragma unroll
+        for (int c16 = 0; c16 < 8; ++c16) {
+          const float4 w = lds128(sW + (((uint32_t)c16 ^ (uint32_t)(r & 7)) << 4));
+          const float* pp = c16 < 4 ? pa + c16 * 4 : pb + (c16 - 4) * 4;
+          y[c16 * 4 + 0] = w.x - pp[0];
+          y[c16 * 4 + 1] = w.y - pp[1];
+          y[c16 * 4 + 2] = w.z - pp[2];
+          y[c16 * 4 + 3] = w.w - pp[3];
+        }
+      }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&empty[st]);      // this warp's part of the W tile is in registers
+      // ---- store, norms
+      {
+        const int col0 = c * BN + half * 32;
+        double q = 0.0;
+        if (rowp != nullptr) {
+          float* dst = rowp + col0;
+          if (col0 + 32 <= ncols && (reinterpret_cast<uintptr_t>(dst) & 15u) == 0) {
+#pragma unroll
+            for (int k = 0; k < 8; ++k)
+              *reinterpret_cast<float4*>(dst + 4 * k) = make_float4(y[4 * k], y[4 * k + 1], y[4 * k + 2], y[4 * k + 3]);
+#pragma unroll
+            for (int k = 0; k < 32; ++k) q += (double)y[k] * (double)y[k];
+          } else {
+#pragma unroll
+            for (int k = 0; k < 32; ++k)
+              if (col0 + k < ncols) {
+                dst[k] = y[k];
+                q += (double)y[k] * (double)y[k];
+              }
+          }
+        }
+        s_top += is_top ? q : 0.0;
+        s_trail += is_top ? 0.0 : q;
+      }
+      if (do_sample) {
+        // ---- Wnew -> tensor memory, split, as the left operand of the sample product
+        if (i > 0 && !mbar_wait(&w_empty, (i - 1) & 1, ctrl)) break;
+        tc_fence_after();
+#pragma unroll
+        for (int g = 0; g < 2; ++g) {
+          float hi[16], lo[16];
+#pragma unroll
+          for (int e = 0; e < 16; ++e) {
+            hi[e] = __uint_as_float(to_tf32(y[g * 16 + e]));
+            lo[e] = __uint_as_float(to_tf32(y[g * 16 + e] - hi[e]));
+          }
+          tmem_st16(tlane + TW + half * 32 + g * 16, hi);
+          tmem_st16(tlane + TW + BN + half * 32 + g * 16, lo);
+        }
+        tmem_st_wait();
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&w_ready);
+        bool last;
+        if (drain_after(i, &last)) {
+          if (!mbar_wait(&y_full, ny & 1, ctrl)) break;
+          ++ny;
+          tc_fence_after();
+#pragma unroll
+          for (int g = 0; g < HB / 16; ++g) {
+            float v[16];
+            tmem_ld16(tlane + TY + half * HB + g * 16, v);
+#pragma unroll
+            for (int e = 0; e < 16; ++e) accY[g * 16 + e] += v[e];
+          }
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(&y_empty);
+          if (last) {
+            float* out = Ypart + (size_t)(p + s) * (size_t)(BM * B) + (size_t)r * B + half * HB;
+#pragma unroll
+            for (int k = 0; k < HB / 4; ++k) {
+              *reinterpret_cast<float4*>(out + 4 * k) = make_float4(accY[4 * k], accY[4 * k + 1], accY[4 * k + 2], accY[4 * k + 3]);
+              accY[4 * k] = accY[4 * k + 1] = accY[4 * k + 2] = accY[4 * k + 3] = 0.f;
+            }
+          }
+        }
+      }
+    }
+  }
+  // per-CTA norm partials (all warps join; producer and issuer contribute zeros), then the common exit
+  const double bt = block_sum(s_top, red);
+  const double br = block_sum(s_trail, red + 32);
+  if (tid == 0 && norm_part != nullptr) {
+    norm_part[2 * p] = bt;
+    norm_part[2 * p + 1] = br;
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 0) tmem_dealloc(tmem, Cfg::COLS);
+}
+
+}  // namespace rrf
