@@ -346,9 +346,10 @@ struct PassModel {
   double rows, n;
   int b;
   bool f64;
+  bool tc;      // single precision on tcgen05
   // flop per microsecond the two GEMM kernels sustain on the whole device
-  double vtw() const { return 2.0 * rows * n * b / (f64 ? 33e6 : 45e6) + 10.0; }
-  double upd() const { return 4.0 * rows * n * b / (f64 ? 27e6 : 32e6) + 15.0; }
+  double vtw() const { return 2.0 * rows * n * b / (f64 ? 33e6 : (tc ? 85e6 : 45e6)) + 10.0; }
+  double upd() const { return 4.0 * rows * n * b / (f64 ? 27e6 : (tc ? 72e6 : 32e6)) + 15.0; }
   // fix-up + panel + T factor on `ctas` SMs, with the launch and event hand-overs of the side stream
   double panel_chain(int ctas) const {
     const double R = std::max(64.0, (rows + b) / ctas);
@@ -865,8 +866,8 @@ rrf_status_t rrf_create(rrf_handle_t* out, int device) {
   h->graph = nullptr;
   h->gexec = nullptr;
   h->graph_off = 0;
-  h->f32_engine = 0;
-  h->tc_chunk = 0;
+  h->f32_engine = 1;      // single precision runs on tcgen05 unless rrf_set_f32_engine says otherwise
+  h->tc_chunk = 2;
   std::memset(&h->profile, 0, sizeof(h->profile));
   cudaError_t e = cudaDeviceGetAttribute(&h->sms, cudaDevAttrMultiProcessorCount, device);
   if (e == cudaSuccess) e = cudaDeviceGetAttribute(&h->smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, device);
@@ -1318,7 +1319,7 @@ rrf_status_t rrf_run(rrf_handle_t h, const rrf_params_t* p, void* dA, int64_t ld
     const int fewest = panel_min_ctas(h, m, b);
     const int cap = std::min(kLookMaxCtas, h->sms / 3);
     if (fewest > 0 && fewest <= cap) {
-      const PassModel pm{h->sms, (double)m, (double)n, b, p->dtype == RRF_F64};
+      const PassModel pm{h->sms, (double)m, (double)n, b, p->dtype == RRF_F64, p->dtype == RRF_F32 && h->f32_engine == 1};
       int best = fewest;
       double best_t = std::min(pm.step_ungated(fewest), pm.step_gated(fewest));
       for (int c = fewest + 1; c <= cap; ++c) {
@@ -1361,7 +1362,7 @@ rrf_status_t rrf_run(rrf_handle_t h, const rrf_params_t* p, void* dA, int64_t ld
   } else if (p->flags & RRF_FLAG_SAMPLE_NEVER) {
     predict = 2;
   } else if (!(p->flags & RRF_FLAG_SAMPLE_ALWAYS) && !(p->flags & RRF_FLAG_FIXED_RANK)) {
-    const PassModel pm{h->sms, (double)m, (double)n, b, p->dtype == RRF_F64};
+    const PassModel pm{h->sms, (double)m, (double)n, b, p->dtype == RRF_F64, false};
     if (pm.vtw() + pm.upd() > 600.0) predict = 0;
   }
   const bool predicting = predict != 1;
@@ -1613,7 +1614,7 @@ rrf_status_t rrf_run(rrf_handle_t h, const rrf_params_t* p, void* dA, int64_t ld
     // starts as early as its inputs allow.
     auto gated = [&](int rows_i) {
       if (p->tune_gate != 0) return p->tune_gate == 2;
-      const PassModel pm{h->sms, (double)rows_i, (double)n, b, p->dtype == RRF_F64};
+      const PassModel pm{h->sms, (double)rows_i, (double)n, b, p->dtype == RRF_F64, tc};
       return pm.step_gated(look_ctas) < pm.step_ungated(look_ctas);
     };
     PanelSource src1 = src;           // panel 1: sampled from A by the sample kernel

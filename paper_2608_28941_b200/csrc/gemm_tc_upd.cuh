@@ -124,7 +124,9 @@ __global__ void __launch_bounds__(kUtcThreads, 1)
   if (tid == 0) {
     for (int s = 0; s < S; ++s) {
       mbar_init(&full[s], 1);
-      mbar_init(&empty[s], kUtcEpi + 1);
+      // a stage is free once the epilogue warps have read its W tile - which they do after the first product
+      // of the tile is complete - and, when sampling, once the second product has read its OmegaT planes
+      mbar_init(&empty[s], do_sample ? kUtcEpi + 1 : kUtcEpi);
     }
     mbar_init(&v_ready, kUtcEpi);
     for (int s = 0; s < 2; ++s) {
@@ -241,7 +243,6 @@ __global__ void __launch_bounds__(kUtcThreads, 1)
           tc_mma_tf32_ts(d, ah, tc_desc_k(zh), idescP, 1u);
         }
         tc_commit(&d_full[buf]);
-        if (!do_sample) tc_commit(&empty[st]);
         if (do_sample && i > 0 && !early) gemm2(i - 1);
       }
       if (ok && do_sample && ntile > 0) gemm2(ntile - 1);
@@ -313,8 +314,6 @@ __global__ void __launch_bounds__(kUtcThreads, 1)
           y[c16 * 4 + 3] = w.w - pp[3];
         }
       }
-      __syncwarp();
-      if (lane == 0) mbar_arrive(&empty[st]);      // this warp's part of the W tile is in registers
       // ---- store, norms
       {
         const int col0 = c * BN + half * 32;
@@ -339,6 +338,10 @@ __global__ void __launch_bounds__(kUtcThreads, 1)
         s_top += is_top ? q : 0.0;
         s_trail += is_top ? 0.0 : q;
       }
+      // Only now is the stage given back: the stores above have consumed every value loaded from the W tile, so
+      // no shared-memory read of this warp can still be in flight when TMA overwrites the stage.
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&empty[st]);
       if (do_sample) {
         // ---- Wnew -> tensor memory, split, as the left operand of the sample product
         if (i > 0 && !mbar_wait(&w_empty, (i - 1) & 1, ctrl)) break;
