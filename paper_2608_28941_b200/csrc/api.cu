@@ -128,6 +128,7 @@ static VtwPlan plan_vtw(int sms, long long rows, long long ncols, int bn) {
 // stream-K plan of the fused update: tiles (row slab, column tile)
 // what the tcgen05 version of the fused update needs beyond the common arguments
 struct UpdTc {
+  const rrf_ctx* h;       // for the tensor maps built per launch
   const void* V;          // reflectors (read directly, not through a tensor map)
   long long ldv;
   const void* Zt;         // [npad][b], written by the T Z kernel
@@ -514,9 +515,17 @@ struct Ops {
         if (j0 >= 0)
           split_planes_kernel<<<std::min(1024, ceil_div((long long)ncols * B, 256)), 256, 0, st>>>(
               (const float*)x.Om + (size_t)j0 * x.ldom, x.ldom, B, ncols, (float*)x.osplit, x.ldo2, &ctrl->done);
+        // where the updated tiles go: the working matrix, and the rows of B that this pass completes
+        CUtensorMap tmCs, tmTs;
+        if (!make_map(x.h, &tmCs, RRF_F32, C, (unsigned long long)r0 + rows, ncols, ldc, 32)) return;
+        if (top_rows > 0) {
+          if (!make_map(x.h, &tmTs, RRF_F32, top, top_rows, ncols, ldtop, 32)) return;
+        } else {
+          tmTs = tmCs;
+        }
         upd_tc_kernel<B><<<p.P, kUtcThreads, UtcCfg<B>::SMEM, st>>>(
-            tmC, x.tmZs, x.tmOs, (const float*)x.V, x.ldv, (float*)C, ldc, (float*)top, ldtop, r0, rows, ncols, cv0,
-            top_rows, j0 >= 0 ? 1 : 0, x.npad, (float*)Ypart, norm_part, p.NC, p.total, p.tpc, x.chunk, ctrl);
+            tmC, x.tmZs, x.tmOs, tmCs, tmTs, (const float*)x.V, x.ldv, r0, rows, ncols, cv0, top_rows, j0 >= 0 ? 1 : 0,
+            x.npad, (float*)Ypart, norm_part, p.NC, p.total, p.tpc, x.chunk, ctrl);
         return;
       }
     }
@@ -1157,6 +1166,7 @@ static rrf_status_t apply_blocks(rrf_handle_t h, int dtype, long long m, int b, 
   UpdTc utc{};
   const bool utc_on = tc && ops->has_upd_tc;
   if (utc_on) {
+    utc.h = h;
     utc.V = dV;
     utc.ldv = ldv;
     utc.Zt = Zt;
@@ -1414,6 +1424,7 @@ rrf_status_t rrf_run(rrf_handle_t h, const rrf_params_t* p, void* dA, int64_t ld
   UpdTc utc{};
   const bool utc_on = tc && ops->has_upd_tc;
   if (utc_on) {
+    utc.h = h;
     utc.V = dV;
     utc.ldv = ldv;
     utc.Zt = Zt;

@@ -18,11 +18,13 @@
 // tile (K = B), that of Y for `chunk` tiles before it is added, rounded to nearest, into registers.
 //
 // Warp roles: 0-7 epilogue (warp w owns tensor-memory lanes 32 (w % 4) ... = those rows of the slab,
-// and columns 32 (w / 4) ... of the tile = one TMA box of W), 8 TMA producer, 9 MMA issuer.
+// and columns 32 (w / 4) ... of the tile = one TMA box of W), 8 TMA producer of W, 9 MMA issuer,
+// 10 and 11 TMA producers of the Zt and OmegaT planes.
 // Tensor-memory columns: [V_hi V_lo | Wnew_hi Wnew_lo | P even tile, P odd tile | Y].
 #pragma once
 
 #include "gemm_tc.cuh"
+#include "panel_tsqr.cuh"
 
 namespace rrf {
 
@@ -70,11 +72,36 @@ __device__ __forceinline__ void tmem_st16(uint32_t taddr, const float (&v)[16]) 
       : "memory");
 }
 __device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+// 2-D tiled TMA store: box in shared memory -> element coordinates (x = innermost, y); rows and columns outside the
+// tensor are not written
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, uint32_t smem_src, int x, int y) {
+  asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%1, %2}], [%3];"
+               ::"l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(smem_src)
+               : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+
+// Optional cycle accounting of one CTA's waits (compiled in with -DRRF_TSQR_TRACE only)
+#ifdef RRF_TSQR_TRACE
+#define UTC_TRACE_DECL long long utc_acc[8] = {0, 0, 0, 0, 0, 0, 0, 0}; const bool utc_on = blockIdx.x == 5 && (threadIdx.x & 31) == 0
+#define UTC_T(slot, ...) { const long long utc_t0 = clock64(); __VA_ARGS__; utc_acc[slot] += clock64() - utc_t0; }
+#define UTC_DUMP(base) if (utc_on) { for (int q_ = 0; q_ < 8; ++q_) g_tsqr_trace[(base) + q_] = (unsigned long long)utc_acc[q_]; }
+#else
+#define UTC_TRACE_DECL
+#define UTC_T(slot, ...) { __VA_ARGS__; }
+#define UTC_DUMP(base)
+#endif
 
 constexpr int kUtcBM = 128, kUtcBN = 64;
 constexpr int kUtcEpi = 8;
-constexpr int kUtcThreads = (kUtcEpi + 2) * 32;
+constexpr int kUtcThreads = (kUtcEpi + 4) * 32;     // + W producer, MMA issuer, Zt producer, OmegaT producer
 
+// Shared memory is three independent TMA rings, because the three inputs of a tile are given back at
+// different times: the W tile once the epilogue warps have it in registers, the Zt planes once the
+// first product is complete, the OmegaT planes once the second is.  W comes from DRAM and gets the
+// deepest ring; the planes come from L2.
 template <int B>
 struct UtcCfg {
   static constexpr int W_BOX = kUtcBM * 128;            // 128 rows x 32 columns
@@ -84,12 +111,12 @@ struct UtcCfg {
   static constexpr int Z_BYTES = KBZ * 2 * Z_BOX;       // per K box: hi rows, then lo rows
   static constexpr int O_BOX = B * 128;                 // B rows of OmegaT x 32 columns of the tile
   static constexpr int O_BYTES = 2 * 2 * O_BOX;         // per K box (two of them): hi rows, then lo rows
-  static constexpr int STAGE = W_BYTES + Z_BYTES + O_BYTES;
-  static constexpr int STAGES = (3 * STAGE + 1024 <= 220 * 1024) ? 3 : 2;
-  static constexpr int SMEM = STAGES * STAGE + 1024;
+  static constexpr int NW = 3, NZ = (B == 64) ? 2 : 3, NO = (B == 64) ? 2 : 3;
+  static constexpr int SMEM = NW * W_BYTES + NZ * Z_BYTES + NO * O_BYTES + 1024;
   static constexpr int TV = 0, TW = 2 * B, TD = TW + 2 * kUtcBN, TY = TD + 2 * kUtcBN;   // tensor-memory columns
   static constexpr int COLS = 512;
   static_assert(TY + B <= COLS, "tensor memory");
+  static_assert(SMEM + 2048 <= 232448, "shared memory");
 };
 
 template <int B>
@@ -97,21 +124,26 @@ __global__ void __launch_bounds__(kUtcThreads, 1)
     upd_tc_kernel(const __grid_constant__ CUtensorMap tmC,   // C [m][ncols], box [128][32]
                   const __grid_constant__ CUtensorMap tmZs,  // Zt planes [2 npad][B], box [64][32]
                   const __grid_constant__ CUtensorMap tmOs,  // OmegaT planes [2 B][n], box [B][32]
-                  const float* __restrict__ V, long long ldv, float* __restrict__ C, long long ldc,
-                  float* __restrict__ top, long long ldtop, int r0, int rows, int ncols, int cv0, int top_rows,
+                  const __grid_constant__ CUtensorMap tmCs,  // C as written [r0 + rows][ncols], box [32][32]
+                  const __grid_constant__ CUtensorMap tmTs,  // rows of B being formed [top_rows][ncols], box [32][32]
+                  const float* __restrict__ V, long long ldv, int r0, int rows, int ncols, int cv0, int top_rows,
                   int sample, int npad, float* __restrict__ Ypart, double* __restrict__ norm_part,
                   int NC, int total, int tpc, int chunk, Ctrl* ctrl) {
   if (*reinterpret_cast<volatile int*>(&ctrl->done)) return;
   using Cfg = UtcCfg<B>;
-  constexpr int S = Cfg::STAGES, STAGE = Cfg::STAGE, W_BOX = Cfg::W_BOX, W_BYTES = Cfg::W_BYTES, Z_BOX = Cfg::Z_BOX,
-                Z_BYTES = Cfg::Z_BYTES, O_BOX = Cfg::O_BOX, KBZ = Cfg::KBZ;
+  constexpr int NW = Cfg::NW, NZ = Cfg::NZ, NO = Cfg::NO, W_BOX = Cfg::W_BOX, W_BYTES = Cfg::W_BYTES, Z_BOX = Cfg::Z_BOX,
+                Z_BYTES = Cfg::Z_BYTES, O_BOX = Cfg::O_BOX, O_BYTES = Cfg::O_BYTES, KBZ = Cfg::KBZ;
   constexpr int TV = Cfg::TV, TW = Cfg::TW, TD = Cfg::TD, TY = Cfg::TY;
   constexpr int BN = kUtcBN, BM = kUtcBM;
   static_assert(B == 32 || B == 64, "block sizes with a 128-row slab");
 
   extern __shared__ unsigned char smem_raw[];
   unsigned char* smem = align1024(smem_raw);
-  __shared__ uint64_t full[S], empty[S], v_ready, d_full[2], d_empty[2], w_ready, w_empty, y_full, y_empty;
+  unsigned char* ringW = smem;
+  unsigned char* ringZ = ringW + NW * W_BYTES;
+  unsigned char* ringO = ringZ + NZ * Z_BYTES;
+  __shared__ uint64_t wfull[NW], wempty[NW], zfull[NZ], zempty[NZ], ofull[NO], oempty[NO];
+  __shared__ uint64_t v_ready, d_full[2], d_empty[2], w_ready, w_empty, y_full, y_empty;
   __shared__ uint32_t tmem_slot;
   __shared__ double red[64];
 
@@ -122,11 +154,17 @@ __global__ void __launch_bounds__(kUtcThreads, 1)
   const bool do_sample = sample != 0;
 
   if (tid == 0) {
-    for (int s = 0; s < S; ++s) {
-      mbar_init(&full[s], 1);
-      // a stage is free once the epilogue warps have read its W tile - which they do after the first product
-      // of the tile is complete - and, when sampling, once the second product has read its OmegaT planes
-      mbar_init(&empty[s], do_sample ? kUtcEpi + 1 : kUtcEpi);
+    for (int s = 0; s < NW; ++s) {
+      mbar_init(&wfull[s], 1);
+      mbar_init(&wempty[s], kUtcEpi);
+    }
+    for (int s = 0; s < NZ; ++s) {
+      mbar_init(&zfull[s], 1);
+      mbar_init(&zempty[s], 1);
+    }
+    for (int s = 0; s < NO; ++s) {
+      mbar_init(&ofull[s], 1);
+      mbar_init(&oempty[s], 1);
     }
     mbar_init(&v_ready, kUtcEpi);
     for (int s = 0; s < 2; ++s) {
@@ -157,29 +195,47 @@ __global__ void __launch_bounds__(kUtcThreads, 1)
   double s_top = 0.0, s_trail = 0.0;
 
   if (warp == kUtcEpi) {
-    // ---------------------------------------------------------------- TMA producer
+    // ---------------------------------------------------------------- TMA producer: W tiles
     if (lane == 0) {
       for (int i = 0; i < ntile; ++i) {
-        const int st = i % S;
-        if (i >= S && !mbar_wait(&empty[st], ((i / S) - 1) & 1, ctrl)) break;
+        const int st = i % NW;
+        if (i >= NW && !mbar_wait(&wempty[st], ((i / NW) - 1) & 1, ctrl)) break;
         const int L = L0 + i, s = L / NC, c = L - s * NC;
-        unsigned char* sW = smem + st * STAGE;
-        unsigned char* sZ = sW + W_BYTES;
-        unsigned char* sO = sZ + Z_BYTES;
-        mbar_expect_tx(&full[st], do_sample ? STAGE : W_BYTES + Z_BYTES);
+        unsigned char* sW = ringW + st * W_BYTES;
+        mbar_expect_tx(&wfull[st], W_BYTES);
 #pragma unroll
-        for (int q = 0; q < 2; ++q) tma_load_2d(sW + q * W_BOX, &tmC, c * BN + q * 32, r0 + s * BM, &full[st]);
+        for (int q = 0; q < 2; ++q) tma_load_2d(sW + q * W_BOX, &tmC, c * BN + q * 32, r0 + s * BM, &wfull[st]);
+      }
+    }
+  } else if (warp == kUtcEpi + 2) {
+    // ---------------------------------------------------------------- TMA producer: Zt planes
+    if (lane == 0) {
+      for (int i = 0; i < ntile; ++i) {
+        const int st = i % NZ;
+        if (i >= NZ && !mbar_wait(&zempty[st], ((i / NZ) - 1) & 1, ctrl)) break;
+        const int L = L0 + i, s = L / NC, c = L - s * NC;
+        unsigned char* sZ = ringZ + st * Z_BYTES;
+        mbar_expect_tx(&zfull[st], Z_BYTES);
 #pragma unroll
         for (int kb = 0; kb < KBZ; ++kb) {
-          tma_load_2d(sZ + kb * 2 * Z_BOX, &tmZs, kb * 32, c * BN, &full[st]);
-          tma_load_2d(sZ + kb * 2 * Z_BOX + Z_BOX, &tmZs, kb * 32, npad + c * BN, &full[st]);
+          tma_load_2d(sZ + kb * 2 * Z_BOX, &tmZs, kb * 32, c * BN, &zfull[st]);
+          tma_load_2d(sZ + kb * 2 * Z_BOX + Z_BOX, &tmZs, kb * 32, npad + c * BN, &zfull[st]);
         }
-        if (do_sample) {
+      }
+    }
+  } else if (warp == kUtcEpi + 3) {
+    // ---------------------------------------------------------------- TMA producer: OmegaT planes
+    if (lane == 0 && do_sample) {
+      for (int i = 0; i < ntile; ++i) {
+        const int st = i % NO;
+        if (i >= NO && !mbar_wait(&oempty[st], ((i / NO) - 1) & 1, ctrl)) break;
+        const int L = L0 + i, s = L / NC, c = L - s * NC;
+        unsigned char* sO = ringO + st * O_BYTES;
+        mbar_expect_tx(&ofull[st], O_BYTES);
 #pragma unroll
-          for (int q = 0; q < 2; ++q) {
-            tma_load_2d(sO + q * 2 * O_BOX, &tmOs, c * BN + q * 32, 0, &full[st]);
-            tma_load_2d(sO + q * 2 * O_BOX + O_BOX, &tmOs, c * BN + q * 32, B, &full[st]);
-          }
+        for (int q = 0; q < 2; ++q) {
+          tma_load_2d(sO + q * 2 * O_BOX, &tmOs, c * BN + q * 32, 0, &ofull[st]);
+          tma_load_2d(sO + q * 2 * O_BOX + O_BOX, &tmOs, c * BN + q * 32, B, &ofull[st]);
         }
       }
     }
@@ -190,13 +246,16 @@ __global__ void __launch_bounds__(kUtcThreads, 1)
       uint32_t fresh_y = 1;
       int ny = 0, cur_s = -1, nslab = 0;
       bool ok = true;
+      UTC_TRACE_DECL;
+      const long long utc_start = clock64();
       // Y += Wnew(i) OmegaT^T
       auto gemm2 = [&](int i) {
-        const int st = i % S;
-        if (!mbar_wait(&w_ready, i & 1, ctrl)) { ok = false; return; }
-        if (fresh_y && ny > 0 && !mbar_wait(&y_empty, (ny - 1) & 1, ctrl)) { ok = false; return; }
+        const int st = i % NO;
+        UTC_T(1, if (!mbar_wait(&ofull[st], (i / NO) & 1, ctrl)) { ok = false; return; })
+        UTC_T(2, if (!mbar_wait(&w_ready, i & 1, ctrl)) { ok = false; return; })
+        UTC_T(3, if (fresh_y && ny > 0 && !mbar_wait(&y_empty, (ny - 1) & 1, ctrl)) { ok = false; return; })
         tc_fence_after();
-        const uint32_t sO = smem_u32(smem + st * STAGE + W_BYTES + Z_BYTES);
+        const uint32_t sO = smem_u32(ringO + st * O_BYTES);
 #pragma unroll
         for (int ks = 0; ks < BN / 8; ++ks) {
           const uint32_t oh = sO + (ks / 4) * 2 * O_BOX + (ks % 4) * 32, ol = oh + O_BOX;
@@ -207,7 +266,7 @@ __global__ void __launch_bounds__(kUtcThreads, 1)
           fresh_y = 0;
         }
         tc_commit(&w_empty);
-        tc_commit(&empty[st]);
+        tc_commit(&oempty[st]);
         bool last;
         if (drain_after(i, &last)) {
           tc_commit(&y_full);
@@ -216,7 +275,7 @@ __global__ void __launch_bounds__(kUtcThreads, 1)
         }
       };
       for (int i = 0; i < ntile && ok; ++i) {
-        const int st = i % S, buf = i & 1;
+        const int st = i % NZ, buf = i & 1;
         const int L = L0 + i, s = L / NC;
         bool last;
         // a tile after which Y is drained (and a slab change, which always follows one) must not wait behind
@@ -224,15 +283,15 @@ __global__ void __launch_bounds__(kUtcThreads, 1)
         const bool early = do_sample && i > 0 && drain_after(i - 1, &last);
         if (early) gemm2(i - 1);
         if (!ok) break;
-        if (!mbar_wait(&full[st], (i / S) & 1, ctrl)) break;
+        UTC_T(4, if (!mbar_wait(&zfull[st], (i / NZ) & 1, ctrl)) break;)
         if (s != cur_s) {
-          if (!mbar_wait(&v_ready, nslab & 1, ctrl)) break;
+          UTC_T(5, if (!mbar_wait(&v_ready, nslab & 1, ctrl)) break;)
           ++nslab;
           cur_s = s;
         }
-        if (i >= 2 && !mbar_wait(&d_empty[buf], ((i >> 1) - 1) & 1, ctrl)) break;
+        UTC_T(6, if (i >= 2 && !mbar_wait(&d_empty[buf], ((i >> 1) - 1) & 1, ctrl)) break;)
         tc_fence_after();
-        const uint32_t sZ = smem_u32(smem + st * STAGE + W_BYTES);
+        const uint32_t sZ = smem_u32(ringZ + st * Z_BYTES);
 #pragma unroll
         for (int ks = 0; ks < B / 8; ++ks) {
           const uint32_t zh = sZ + (ks / 4) * 2 * Z_BOX + (ks % 4) * 32, zl = zh + Z_BOX;
@@ -243,9 +302,15 @@ __global__ void __launch_bounds__(kUtcThreads, 1)
           tc_mma_tf32_ts(d, ah, tc_desc_k(zh), idescP, 1u);
         }
         tc_commit(&d_full[buf]);
+        tc_commit(&zempty[st]);
         if (do_sample && i > 0 && !early) gemm2(i - 1);
       }
       if (ok && do_sample && ntile > 0) gemm2(ntile - 1);
+#ifdef RRF_TSQR_TRACE
+      utc_acc[0] = clock64() - utc_start;
+      utc_acc[7] = ntile;
+#endif
+      UTC_DUMP(16)
     }
   } else {
     // ---------------------------------------------------------------- epilogue warps
@@ -257,11 +322,18 @@ __global__ void __launch_bounds__(kUtcThreads, 1)
 #pragma unroll
     for (int j = 0; j < HB; ++j) accY[j] = 0.f;
     int cur_s = -1, ny = 0;
-    float* rowp = nullptr;
+    UTC_TRACE_DECL;
+    const long long utc_start = clock64();
     bool is_top = false;
     for (int i = 0; i < ntile; ++i) {
-      const int st = i % S, buf = i & 1;
+      const int st = i % NW, buf = i & 1;
       const int L = L0 + i, s = L / NC, c = L - s * NC;
+      if (i > 0 && lane == 0) {
+        // the TMA store of the previous tile has read its part of the W ring by now (it was issued a whole
+        // tile ago); only then does that slot go back to the producer
+        bulk_wait_read();
+        mbar_arrive(&wempty[(i - 1) % NW]);
+      }
       if (s != cur_s) {
         // V[slab] -> tensor memory, split (every product of the previous slab that reads it is complete: the
         // accumulator of its last tile has been drained)
@@ -289,11 +361,13 @@ __global__ void __launch_bounds__(kUtcThreads, 1)
         __syncwarp();
         if (lane == 0) mbar_arrive(&v_ready);
         cur_s = s;
-        is_top = lr < top_rows;
-        rowp = lr >= rows ? nullptr : (is_top ? top + (size_t)lr * ldtop : C + (size_t)(r0 + lr) * ldc);
+        is_top = lr < top_rows;        // top_rows is a multiple of 32: the same for the whole warp
       }
-      if (!mbar_wait(&full[st], (i / S) & 1, ctrl)) break;
-      if (!mbar_wait(&d_full[buf], (i >> 1) & 1, ctrl)) break;
+      UTC_T(1, if (!mbar_wait(&wfull[st], (i / NW) & 1, ctrl)) break;)
+      UTC_T(2, if (!mbar_wait(&d_full[buf], (i >> 1) & 1, ctrl)) break;)
+#ifdef RRF_TSQR_TRACE
+      const long long utc_e0 = clock64();
+#endif
       tc_fence_after();
       float y[32];
       {
@@ -303,7 +377,7 @@ __global__ void __launch_bounds__(kUtcThreads, 1)
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(&d_empty[buf]);
-        const uint32_t sW = smem_u32(smem + st * STAGE + half * W_BOX + r * 128);
+        const uint32_t sW = smem_u32(ringW + st * W_BYTES + half * W_BOX + r * 128);
 #pragma unroll
         for (int c16 = 0; c16 < 8; ++c16) {
           const float4 w = lds128(sW + (((uint32_t)c16 ^ (uint32_t)(r & 7)) << 4));
@@ -314,37 +388,44 @@ __global__ void __launch_bounds__(kUtcThreads, 1)
           y[c16 * 4 + 3] = w.w - pp[3];
         }
       }
-      // ---- store, norms
+      // ---- Wnew goes back to where the W tile stood in shared memory (same swizzled places, so each thread
+      // overwrites exactly what it has read) and TMA stores this warp's 32 x 32 box in whole 128-byte lines;
+      // rows past the matrix and columns past its width are zero here and are not written.  Norms on the side:
+      // four single-precision partial sums of eight squares each, added in double precision.
       {
-        const int col0 = c * BN + half * 32;
-        double q = 0.0;
-        if (rowp != nullptr) {
-          float* dst = rowp + col0;
-          if (col0 + 32 <= ncols && (reinterpret_cast<uintptr_t>(dst) & 15u) == 0) {
+        const uint32_t sW = smem_u32(ringW + st * W_BYTES + half * W_BOX + r * 128);
+        float q4[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-            for (int k = 0; k < 8; ++k)
-              *reinterpret_cast<float4*>(dst + 4 * k) = make_float4(y[4 * k], y[4 * k + 1], y[4 * k + 2], y[4 * k + 3]);
+        for (int c16 = 0; c16 < 8; ++c16) {
+          sts128(sW + (((uint32_t)c16 ^ (uint32_t)(r & 7)) << 4),
+                 make_float4(y[c16 * 4], y[c16 * 4 + 1], y[c16 * 4 + 2], y[c16 * 4 + 3]));
 #pragma unroll
-            for (int k = 0; k < 32; ++k) q += (double)y[k] * (double)y[k];
-          } else {
-#pragma unroll
-            for (int k = 0; k < 32; ++k)
-              if (col0 + k < ncols) {
-                dst[k] = y[k];
-                q += (double)y[k] * (double)y[k];
-              }
-          }
+          for (int e = 0; e < 4; ++e) q4[c16 & 3] = fmaf(y[c16 * 4 + e], y[c16 * 4 + e], q4[c16 & 3]);
         }
+        proxy_fence_async_smem();
+        __syncwarp();
+        if (lane == 0) {
+          const int lr0 = s * BM + quad * 32;
+          if (lr0 < rows) {
+            const uint32_t box = smem_u32(ringW + st * W_BYTES + half * W_BOX + quad * 32 * 128);
+            if (lr0 < top_rows) tma_store_2d(&tmTs, box, c * BN + half * 32, lr0);
+            else tma_store_2d(&tmCs, box, c * BN + half * 32, r0 + lr0);
+          }
+          bulk_commit();
+        }
+        const double q = ((double)q4[0] + (double)q4[1]) + ((double)q4[2] + (double)q4[3]);
         s_top += is_top ? q : 0.0;
         s_trail += is_top ? 0.0 : q;
       }
-      // Only now is the stage given back: the stores above have consumed every value loaded from the W tile, so
-      // no shared-memory read of this warp can still be in flight when TMA overwrites the stage.
-      __syncwarp();
-      if (lane == 0) mbar_arrive(&empty[st]);
       if (do_sample) {
         // ---- Wnew -> tensor memory, split, as the left operand of the sample product
-        if (i > 0 && !mbar_wait(&w_empty, (i - 1) & 1, ctrl)) break;
+#ifdef RRF_TSQR_TRACE
+        utc_acc[5] += clock64() - utc_e0;      // P, W, store, norms
+#endif
+        UTC_T(3, if (i > 0 && !mbar_wait(&w_empty, (i - 1) & 1, ctrl)) break;)
+#ifdef RRF_TSQR_TRACE
+        const long long utc_e1 = clock64();
+#endif
         tc_fence_after();
 #pragma unroll
         for (int g = 0; g < 2; ++g) {
@@ -361,9 +442,12 @@ __global__ void __launch_bounds__(kUtcThreads, 1)
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(&w_ready);
+#ifdef RRF_TSQR_TRACE
+        utc_acc[6] += clock64() - utc_e1;      // split + store to tensor memory
+#endif
         bool last;
         if (drain_after(i, &last)) {
-          if (!mbar_wait(&y_full, ny & 1, ctrl)) break;
+          UTC_T(4, if (!mbar_wait(&y_full, ny & 1, ctrl)) break;)
           ++ny;
           tc_fence_after();
 #pragma unroll
@@ -387,6 +471,11 @@ __global__ void __launch_bounds__(kUtcThreads, 1)
         }
       }
     }
+    if (lane == 0) bulk_wait_all();      // this warp's stores are complete before the CTA may exit
+#ifdef RRF_TSQR_TRACE
+    utc_acc[0] = clock64() - utc_start;
+    if (warp == 0) { UTC_DUMP(0) }
+#endif
   }
   // per-CTA norm partials (all warps join; producer and issuer contribute zeros), then the common exit
   const double bt = block_sum(s_top, red);
