@@ -256,7 +256,27 @@ def roofline_of(pb, res, prof, steps, value_per_gpu, ms_step, ms_profiled, peaks
     peak = rrf.rrf_measure_peak(h, kind, 200.0)
     if w.dtype == "f32":
         peak /= 3.0                               # three TF32 products per fp32 product
-    if top in gemm:
+    tc = w.dtype == "f32" and getattr(pb, "f32_engine", "mma") == "tcgen05"
+    if top in gemm and tc:
+        # Single precision on tcgen05: per 64 KB of W read and written the tensor core needs about half the time
+        # HBM does, so HBM is the roof of these kernels.  Algorithmic bytes: the rows of W each launch must read
+        # (update: and write back); V, Zt and OmegaT are smaller by n / b and stay in L2.
+        hbm = peaks.get("hbm_gbs", 6650.0)
+        per_row = {"update": 2.0, "vtw": 1.0, "sample": 1.0}[top] * w.n * pb.esize
+        byts = steps * (w.m * per_row if top == "sample" else sum(r * per_row for r in mi))
+        achieved = byts / (ms * 1e-3) / 1e9
+        work = steps * sum((4.0 if top == "update" else 2.0) * r * w.n * w.b for r in mi)
+        sms = torch.cuda.get_device_properties(local).multi_processor_count
+        share = (sms - res.panel_ctas) / sms if (res.queues == 2 and top == "update") else 1.0
+        tf32 = peaks.get("bf16_tflops", 1590.0) * 0.5 / 3.0
+        rl = {"kernel": top, "bound": "hbm", "achieved": achieved, "peak": hbm, "unit": "GB/s",
+              "frac": achieved / hbm, "traffic": NCU_TRAFFIC_BYTES.get((w.name, top)),
+              "peak_source": "MEASURED_PEAKS.json (of measured)" if "hbm_gbs" in peaks else "of fallback",
+              "avg_launch_ms": ms / max(cnt, 1), "launches": cnt, "sm_share": share,
+              "tensor_tflops": work / (ms * 1e-3) / 1e12, "tensor_peak_3xtf32": tf32,
+              "tensor_peak_source": "bf16 peak x nominal TF32/bf16 ratio / 3 products per fp32 product"}
+        peak = tf32
+    elif top in gemm:
         work = steps * sum(2.0 * r * w.n * w.b for r in mi)
         if top == "update":                       # the fused kernel also samples a later panel in most passes
             work += steps * sum(2.0 * (r - w.b) * w.n * w.b for r in mi[:res.fused_samples])   # rows below B_i
@@ -378,7 +398,7 @@ def main():
                     help="no-update: A is left unchanged and B is not formed (one pass over A per block instead of "
                          "three); stops on the sampled Frobenius estimate.  Flops are counted as the in-place schedule's")
     ap.add_argument("--estimator", type=int, default=0, choices=[0, 1, 2, 3])
-    ap.add_argument("--f32-engine", default="mma", choices=["mma", "tcgen05"],
+    ap.add_argument("--f32-engine", default="tcgen05", choices=["mma", "tcgen05"],
                     help="tensor-core path of the single-precision V^T W product")
     ap.add_argument("--tc-chunk", type=int, default=2,
                     help="tcgen05: 64-row tiles summed in tensor memory between round-to-nearest adds (0: all)")
@@ -415,7 +435,7 @@ def main():
     if world > 1:
         dist.barrier()
     h = rrf.rrf_create(local)
-    rrf.rrf_set_f32_engine(h, 1 if args.f32_engine == "tcgen05" else 0, args.tc_chunk)
+    rrf.rrf_set_single_engine(h, 1 if args.f32_engine == "tcgen05" else 0, args.tc_chunk)
     sched = {"auto": 0, "one": rrf.RRF_FLAG_ONE_QUEUE, "two": rrf.RRF_FLAG_TWO_QUEUES}[args.schedule]
     if args.panel == "tree":
         sched |= rrf.RRF_FLAG_PANEL_TREE
@@ -436,6 +456,7 @@ def main():
         args.no_per_config = True
     peaks = measured_peaks()
     pb = Problem(h, w, dev, sched, estimator, args.panel_ctas)
+    pb.f32_engine = args.f32_engine
     sampler = ClockSampler(local)
     pb.step()
     barrier()
@@ -475,6 +496,7 @@ def main():
             wc = wl.CONFIGS[name]
             n_steps = 3 if name == "cfg5" else 10
             pc = Problem(h, wc, dev, sched)
+            pc.f32_engine = args.f32_engine
             r, ms, pr, msp = time_problem(pc, n_steps, 3, 1, barrier)
             v = job_tflops(method_flops(wc.m, wc.n, wc.b, r.steps), 1, ms)
             rl = roofline_of(pc, r, pr, n_steps, v, ms, msp, peaks, local)

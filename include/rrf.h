@@ -324,7 +324,7 @@ rrf_status_t rrf_fill_omega(rrf_handle_t h, int32_t dtype, uint64_t seed, int64_
                             int32_t first_vec, void* dOmegaT, int64_t ldo, void* cuda_stream);
 
 /*
- * rrf_set_f32_engine - choose the tensor-core path of the single-precision product Z = V_i^T W
+ * rrf_set_single_engine - choose the tensor-core path of the single-precision product Z = V_i^T W
  * (Algorithm 2 line 8) for every later call on this handle that computes it (rrf_run, rrf_apply_q,
  * rrf_apply_qt, rrf_form_q, rrf_subspace_transfer).  Double precision is not affected.
  *   engine 0  mma.sync m16n8k8, 3xTF32, every k-step added round-to-nearest in registers (default)
@@ -334,7 +334,7 @@ rrf_status_t rrf_fill_omega(rrf_handle_t h, int32_t dtype, uint64_t seed, int64_
  *             0 keeps a whole accumulator there.
  * Host-side setting, no device work.  Returns RRF_ERR_INVALID_ARG for other values.
  */
-rrf_status_t rrf_set_f32_engine(rrf_handle_t h, int32_t engine, int32_t chunk_tiles);
+rrf_status_t rrf_set_single_engine(rrf_handle_t h, int32_t engine, int32_t chunk_tiles);
 
 /*
  * Measurement aids (the paper reports wall times only; these have no counterpart in it).

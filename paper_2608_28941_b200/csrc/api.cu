@@ -875,7 +875,7 @@ rrf_status_t rrf_create(rrf_handle_t* out, int device) {
   h->graph = nullptr;
   h->gexec = nullptr;
   h->graph_off = 0;
-  h->f32_engine = 1;      // single precision runs on tcgen05 unless rrf_set_f32_engine says otherwise
+  h->f32_engine = 1;      // single precision runs on tcgen05 unless rrf_set_single_engine says otherwise
   h->tc_chunk = 2;
   std::memset(&h->profile, 0, sizeof(h->profile));
   cudaError_t e = cudaDeviceGetAttribute(&h->sms, cudaDevAttrMultiProcessorCount, device);
@@ -926,7 +926,7 @@ rrf_status_t rrf_last_status(rrf_handle_t h, void* cuda_stream) {
   return (rrf_status_t)c.status;
 }
 
-rrf_status_t rrf_set_f32_engine(rrf_handle_t h, int32_t engine, int32_t chunk_tiles) {
+rrf_status_t rrf_set_single_engine(rrf_handle_t h, int32_t engine, int32_t chunk_tiles) {
   if (h == nullptr || engine < 0 || engine > 1 || chunk_tiles < 0) return RRF_ERR_INVALID_ARG;
   h->f32_engine = engine;
   h->tc_chunk = chunk_tiles;

@@ -85,7 +85,7 @@ __device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wa
 
 // Optional cycle accounting of one CTA's waits (compiled in with -DRRF_TSQR_TRACE only)
 #ifdef RRF_TSQR_TRACE
-#define UTC_TRACE_DECL long long utc_acc[8] = {0, 0, 0, 0, 0, 0, 0, 0}; const bool utc_on = blockIdx.x == 5 && (threadIdx.x & 31) == 0
+#define UTC_TRACE_DECL long long utc_acc[8] = {0, 0, 0, 0, 0, 0, 0, 0}; const bool utc_on = blockIdx.x == 5 && (threadIdx.x & 31) == 0 && do_sample
 #define UTC_T(slot, ...) { const long long utc_t0 = clock64(); __VA_ARGS__; utc_acc[slot] += clock64() - utc_t0; }
 #define UTC_DUMP(base) if (utc_on) { for (int q_ = 0; q_ < 8; ++q_) g_tsqr_trace[(base) + q_] = (unsigned long long)utc_acc[q_]; }
 #else
@@ -253,9 +253,12 @@ __global__ void __launch_bounds__(kUtcThreads, 1)
         const int st = i % NO;
         UTC_T(1, if (!mbar_wait(&ofull[st], (i / NO) & 1, ctrl)) { ok = false; return; })
         UTC_T(2, if (!mbar_wait(&w_ready, i & 1, ctrl)) { ok = false; return; })
-        UTC_T(3, if (fresh_y && ny > 0 && !mbar_wait(&y_empty, (ny - 1) & 1, ctrl)) { ok = false; return; })
+        UTC_T(1, if (fresh_y && ny > 0 && !mbar_wait(&y_empty, (ny - 1) & 1, ctrl)) { ok = false; return; })
         tc_fence_after();
         const uint32_t sO = smem_u32(ringO + st * O_BYTES);
+#ifdef RRF_TSQR_TRACE
+        const long long utc_g2 = clock64();
+#endif
 #pragma unroll
         for (int ks = 0; ks < BN / 8; ++ks) {
           const uint32_t oh = sO + (ks / 4) * 2 * O_BOX + (ks % 4) * 32, ol = oh + O_BOX;
@@ -267,6 +270,9 @@ __global__ void __launch_bounds__(kUtcThreads, 1)
         }
         tc_commit(&w_empty);
         tc_commit(&oempty[st]);
+#ifdef RRF_TSQR_TRACE
+        utc_acc[3] += clock64() - utc_g2;      // issue of the second product
+#endif
         bool last;
         if (drain_after(i, &last)) {
           tc_commit(&y_full);
@@ -285,13 +291,16 @@ __global__ void __launch_bounds__(kUtcThreads, 1)
         if (!ok) break;
         UTC_T(4, if (!mbar_wait(&zfull[st], (i / NZ) & 1, ctrl)) break;)
         if (s != cur_s) {
-          UTC_T(5, if (!mbar_wait(&v_ready, nslab & 1, ctrl)) break;)
+          UTC_T(4, if (!mbar_wait(&v_ready, nslab & 1, ctrl)) break;)
           ++nslab;
           cur_s = s;
         }
         UTC_T(6, if (i >= 2 && !mbar_wait(&d_empty[buf], ((i >> 1) - 1) & 1, ctrl)) break;)
         tc_fence_after();
         const uint32_t sZ = smem_u32(ringZ + st * Z_BYTES);
+#ifdef RRF_TSQR_TRACE
+        const long long utc_g1 = clock64();
+#endif
 #pragma unroll
         for (int ks = 0; ks < B / 8; ++ks) {
           const uint32_t zh = sZ + (ks / 4) * 2 * Z_BOX + (ks % 4) * 32, zl = zh + Z_BOX;
@@ -303,6 +312,9 @@ __global__ void __launch_bounds__(kUtcThreads, 1)
         }
         tc_commit(&d_full[buf]);
         tc_commit(&zempty[st]);
+#ifdef RRF_TSQR_TRACE
+        utc_acc[5] += clock64() - utc_g1;      // issue of the first product
+#endif
         if (do_sample && i > 0 && !early) gemm2(i - 1);
       }
       if (ok && do_sample && ntile > 0) gemm2(ntile - 1);

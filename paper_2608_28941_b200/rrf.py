@@ -45,7 +45,7 @@ class rrf_profile_t(C.Structure):
     _fields_ = [("ms", C.c_double * 9), ("launches", C.c_int32 * 9), ("pad", C.c_int32)]
 
 
-EXPORTS = ["rrf_set_f32_engine", "rrf_sample_workspace_bytes", "rrf_sample_panel", "rrf_frobenius_sq", "rrf_panel_qr_blocked", "rrf_panel_qr_tree", "rrf_transfer_workspace_bytes", "rrf_subspace_transfer", "rrf_selftest_timeout", "rrf_panel_qr_static", "rrf_set_profiling", "rrf_get_profile", "rrf_measure_peak", "rrf_create", "rrf_destroy", "rrf_workspace_bytes", "rrf_run", "rrf_panel_workspace_bytes",
+EXPORTS = ["rrf_set_single_engine", "rrf_sample_workspace_bytes", "rrf_sample_panel", "rrf_frobenius_sq", "rrf_panel_qr_blocked", "rrf_panel_qr_tree", "rrf_transfer_workspace_bytes", "rrf_subspace_transfer", "rrf_selftest_timeout", "rrf_panel_qr_static", "rrf_set_profiling", "rrf_get_profile", "rrf_measure_peak", "rrf_create", "rrf_destroy", "rrf_workspace_bytes", "rrf_run", "rrf_panel_workspace_bytes",
            "rrf_panel_qr", "rrf_apply_workspace_bytes", "rrf_apply_qt", "rrf_apply_q", "rrf_form_q",
            "rrf_fill_omega", "rrf_last_status", "rrf_status_string"]
 
@@ -84,7 +84,7 @@ def load():
                                           vp, i64, vp, sz, vp]
     lib.rrf_last_status.argtypes = [vp, vp]
     lib.rrf_selftest_timeout.argtypes = [vp, C.c_double, vp]
-    lib.rrf_set_f32_engine.argtypes = [vp, i32, i32]
+    lib.rrf_set_single_engine.argtypes = [vp, i32, i32]
     lib.rrf_set_profiling.argtypes = [vp, i32]
     lib.rrf_get_profile.argtypes = [vp, C.POINTER(rrf_profile_t)]
     lib.rrf_measure_peak.argtypes = [vp, i32, C.c_double, C.POINTER(C.c_double)]
@@ -350,10 +350,10 @@ def rrf_last_status(h) -> int:
     return load().rrf_last_status(h, _stream())
 
 
-def rrf_set_f32_engine(h, engine: int, chunk_tiles: int = 0) -> None:
-    s = load().rrf_set_f32_engine(h, int(engine), int(chunk_tiles))
+def rrf_set_single_engine(h, engine: int, chunk_tiles: int = 0) -> None:
+    s = load().rrf_set_single_engine(h, int(engine), int(chunk_tiles))
     if s != 0:
-        raise RrfError(s, "rrf_set_f32_engine")
+        raise RrfError(s, "rrf_set_single_engine")
 
 
 def rrf_set_profiling(h, enable: bool) -> None:
