@@ -14,13 +14,18 @@
 // carries only what TMA brings - W, Zt planes, OmegaT planes - and is read once by the tensor core
 // and (W) once by the epilogue: about 220 KB of shared-memory traffic per 64 KB of HBM traffic.
 //
-// 3xTF32 as everywhere: D += A_lo B_hi + A_hi B_lo + A_hi B_hi.  The accumulator of P lives for one
-// tile (K = B), that of Y for `chunk` tiles before it is added, rounded to nearest, into registers.
+// 3xTF32 as everywhere, D += A_lo B_hi + A_hi B_lo + A_hi B_hi, but in two instructions per K step: the
+// hi and lo planes of the right operand lie one after the other in shared memory, so one instruction
+// with twice the columns forms A_hi [B_hi | B_lo] and a second one adds A_lo B_hi to the first half;
+// the halves are added when the accumulator is read.  (One thread issues a dependent tf32 instruction
+// every 52 to 64 clocks whether it has 64 or 128 columns - 128 is where the tensor core itself needs
+// 64 - so the wider instruction is free.)  The accumulator of P lives for one tile (K = B), that of Y
+// for `chunk` tiles before it is added, rounded to nearest, into registers.
 //
 // Warp roles: 0-7 epilogue (warp w owns tensor-memory lanes 32 (w % 4) ... = those rows of the slab,
 // and columns 32 (w / 4) ... of the tile = one TMA box of W), 8 TMA producer of W, 9 MMA issuer,
 // 10 and 11 TMA producers of the Zt and OmegaT planes.
-// Tensor-memory columns: [V_hi V_lo | Wnew_hi Wnew_lo | P even tile, P odd tile | Y].
+// Tensor-memory columns: [V_hi V_lo | Wnew_hi Wnew_lo | P, P's hi x lo part | Y, Y's hi x lo part].
 #pragma once
 
 #include "gemm_tc.cuh"
@@ -113,9 +118,10 @@ struct UtcCfg {
   static constexpr int O_BYTES = 2 * 2 * O_BOX;         // per K box (two of them): hi rows, then lo rows
   static constexpr int NW = 3, NZ = (B == 64) ? 2 : 3, NO = (B == 64) ? 2 : 3;
   static constexpr int SMEM = NW * W_BYTES + NZ * Z_BYTES + NO * O_BYTES + 1024;
-  static constexpr int TV = 0, TW = 2 * B, TD = TW + 2 * kUtcBN, TY = TD + 2 * kUtcBN;   // tensor-memory columns
+  // tensor-memory columns: [V_hi V_lo | Wnew_hi Wnew_lo | P and its hi x lo part | Y and its hi x lo part]
+  static constexpr int TV = 0, TW = 2 * B, TD = TW + 2 * kUtcBN, TY = TD + 2 * kUtcBN;
   static constexpr int COLS = 512;
-  static_assert(TY + B <= COLS, "tensor memory");
+  static_assert(TY + 2 * B <= COLS, "tensor memory");
   static_assert(SMEM + 2048 <= 232448, "shared memory");
 };
 
@@ -143,7 +149,7 @@ __global__ void __launch_bounds__(kUtcThreads, 1)
   unsigned char* ringZ = ringW + NW * W_BYTES;
   unsigned char* ringO = ringZ + NZ * Z_BYTES;
   __shared__ uint64_t wfull[NW], wempty[NW], zfull[NZ], zempty[NZ], ofull[NO], oempty[NO];
-  __shared__ uint64_t v_ready, d_full[2], d_empty[2], w_ready, w_empty, y_full, y_empty;
+  __shared__ uint64_t v_ready, d_full, d_empty, w_ready, w_empty, y_full, y_empty;
   __shared__ uint32_t tmem_slot;
   __shared__ double red[64];
 
@@ -167,10 +173,8 @@ __global__ void __launch_bounds__(kUtcThreads, 1)
       mbar_init(&oempty[s], 1);
     }
     mbar_init(&v_ready, kUtcEpi);
-    for (int s = 0; s < 2; ++s) {
-      mbar_init(&d_full[s], 1);
-      mbar_init(&d_empty[s], kUtcEpi);
-    }
+    mbar_init(&d_full, 1);
+    mbar_init(&d_empty, kUtcEpi);
     mbar_init(&w_ready, kUtcEpi);
     mbar_init(&w_empty, 1);
     mbar_init(&y_full, 1);
@@ -242,7 +246,8 @@ __global__ void __launch_bounds__(kUtcThreads, 1)
   } else if (warp == kUtcEpi + 1) {
     // ---------------------------------------------------------------- MMA issuer
     if (lane == 0) {
-      constexpr uint32_t idescP = tc_idesc_tf32_k(BM, BN), idescY = tc_idesc_tf32_k(BM, B);
+      constexpr uint32_t idescP2 = tc_idesc_tf32_k(BM, 2 * BN), idescP1 = tc_idesc_tf32_k(BM, BN);
+      constexpr uint32_t idescY2 = tc_idesc_tf32_k(BM, 2 * B), idescY1 = tc_idesc_tf32_k(BM, B);
       uint32_t fresh_y = 1;
       int ny = 0, cur_s = -1, nslab = 0;
       bool ok = true;
@@ -261,11 +266,10 @@ __global__ void __launch_bounds__(kUtcThreads, 1)
 #endif
 #pragma unroll
         for (int ks = 0; ks < BN / 8; ++ks) {
-          const uint32_t oh = sO + (ks / 4) * 2 * O_BOX + (ks % 4) * 32, ol = oh + O_BOX;
+          const uint64_t oh = tc_desc_k(sO + (ks / 4) * 2 * O_BOX + (ks % 4) * 32);   // hi rows, lo rows right behind
           const uint32_t ah = tmem + TW + ks * 8, al = ah + BN;
-          tc_mma_tf32_ts(tmem + TY, al, tc_desc_k(oh), idescY, fresh_y ^ 1u);
-          tc_mma_tf32_ts(tmem + TY, ah, tc_desc_k(ol), idescY, 1u);
-          tc_mma_tf32_ts(tmem + TY, ah, tc_desc_k(oh), idescY, 1u);
+          tc_mma_tf32_ts(tmem + TY, ah, oh, idescY2, fresh_y ^ 1u);
+          tc_mma_tf32_ts(tmem + TY, al, oh, idescY1, 1u);
           fresh_y = 0;
         }
         tc_commit(&w_empty);
@@ -281,7 +285,7 @@ __global__ void __launch_bounds__(kUtcThreads, 1)
         }
       };
       for (int i = 0; i < ntile && ok; ++i) {
-        const int st = i % NZ, buf = i & 1;
+        const int st = i % NZ;
         const int L = L0 + i, s = L / NC;
         bool last;
         // a tile after which Y is drained (and a slab change, which always follows one) must not wait behind
@@ -295,7 +299,7 @@ __global__ void __launch_bounds__(kUtcThreads, 1)
           ++nslab;
           cur_s = s;
         }
-        UTC_T(6, if (i >= 2 && !mbar_wait(&d_empty[buf], ((i >> 1) - 1) & 1, ctrl)) break;)
+        UTC_T(6, if (i >= 1 && !mbar_wait(&d_empty, (i - 1) & 1, ctrl)) break;)
         tc_fence_after();
         const uint32_t sZ = smem_u32(ringZ + st * Z_BYTES);
 #ifdef RRF_TSQR_TRACE
@@ -303,14 +307,12 @@ __global__ void __launch_bounds__(kUtcThreads, 1)
 #endif
 #pragma unroll
         for (int ks = 0; ks < B / 8; ++ks) {
-          const uint32_t zh = sZ + (ks / 4) * 2 * Z_BOX + (ks % 4) * 32, zl = zh + Z_BOX;
+          const uint64_t zh = tc_desc_k(sZ + (ks / 4) * 2 * Z_BOX + (ks % 4) * 32);   // hi rows, lo rows right behind
           const uint32_t ah = tmem + TV + ks * 8, al = ah + B;
-          const uint32_t d = tmem + TD + buf * BN;
-          tc_mma_tf32_ts(d, al, tc_desc_k(zh), idescP, ks > 0 ? 1u : 0u);
-          tc_mma_tf32_ts(d, ah, tc_desc_k(zl), idescP, 1u);
-          tc_mma_tf32_ts(d, ah, tc_desc_k(zh), idescP, 1u);
+          tc_mma_tf32_ts(tmem + TD, ah, zh, idescP2, ks > 0 ? 1u : 0u);
+          tc_mma_tf32_ts(tmem + TD, al, zh, idescP1, 1u);
         }
-        tc_commit(&d_full[buf]);
+        tc_commit(&d_full);
         tc_commit(&zempty[st]);
 #ifdef RRF_TSQR_TRACE
         utc_acc[5] += clock64() - utc_g1;      // issue of the first product
@@ -338,7 +340,7 @@ __global__ void __launch_bounds__(kUtcThreads, 1)
     const long long utc_start = clock64();
     bool is_top = false;
     for (int i = 0; i < ntile; ++i) {
-      const int st = i % NW, buf = i & 1;
+      const int st = i % NW;
       const int L = L0 + i, s = L / NC, c = L - s * NC;
       if (i > 0 && lane == 0) {
         // the TMA store of the previous tile has read its part of the W ring by now (it was issued a whole
@@ -376,7 +378,7 @@ __global__ void __launch_bounds__(kUtcThreads, 1)
         is_top = lr < top_rows;        // top_rows is a multiple of 32: the same for the whole warp
       }
       UTC_T(1, if (!mbar_wait(&wfull[st], (i / NW) & 1, ctrl)) break;)
-      UTC_T(2, if (!mbar_wait(&d_full[buf], (i >> 1) & 1, ctrl)) break;)
+      UTC_T(2, if (!mbar_wait(&d_full, i & 1, ctrl)) break;)
 #ifdef RRF_TSQR_TRACE
       const long long utc_e0 = clock64();
 #endif
@@ -384,11 +386,19 @@ __global__ void __launch_bounds__(kUtcThreads, 1)
       float y[32];
       {
         float pa[16], pb[16];
-        tmem_ld16(tlane + TD + buf * BN + half * 32, pa);
-        tmem_ld16(tlane + TD + buf * BN + half * 32 + 16, pb);
+        {
+          float qa[16], qb[16];                 // the hi x lo part of P
+          tmem_ld16x4(tlane + TD + half * 32, tlane + TD + half * 32 + 16, tlane + TD + BN + half * 32,
+                      tlane + TD + BN + half * 32 + 16, pa, pb, qa, qb);
+#pragma unroll
+          for (int e = 0; e < 16; ++e) {
+            pa[e] += qa[e];
+            pb[e] += qb[e];
+          }
+        }
         tc_fence_before();
         __syncwarp();
-        if (lane == 0) mbar_arrive(&d_empty[buf]);
+        if (lane == 0) mbar_arrive(&d_empty);
         const uint32_t sW = smem_u32(ringW + st * W_BYTES + half * W_BOX + r * 128);
 #pragma unroll
         for (int c16 = 0; c16 < 8; ++c16) {
@@ -464,10 +474,11 @@ __global__ void __launch_bounds__(kUtcThreads, 1)
           tc_fence_after();
 #pragma unroll
           for (int g = 0; g < HB / 16; ++g) {
-            float v[16];
+            float v[16], w2[16];
             tmem_ld16(tlane + TY + half * HB + g * 16, v);
+            tmem_ld16(tlane + TY + B + half * HB + g * 16, w2);      // the hi x lo part
 #pragma unroll
-            for (int e = 0; e < 16; ++e) accY[g * 16 + e] += v[e];
+            for (int e = 0; e < 16; ++e) accY[g * 16 + e] += v[e] + w2[e];
           }
           tc_fence_before();
           __syncwarp();
