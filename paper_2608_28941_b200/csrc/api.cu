@@ -525,7 +525,7 @@ struct Ops {
         }
         upd_tc_kernel<B><<<p.P, kUtcThreads, UtcCfg<B>::SMEM, st>>>(
             tmC, x.tmZs, x.tmOs, tmCs, tmTs, (const float*)x.V, x.ldv, r0, rows, ncols, cv0, top_rows, j0 >= 0 ? 1 : 0,
-            x.npad, (float*)Ypart, norm_part, p.NC, p.total, p.tpc, x.chunk, ctrl);
+            x.npad, (float*)Ypart, norm_part, p.NC, p.total, p.tpc, x.chunk * kUtcYChunkFactor, ctrl);
         return;
       }
     }

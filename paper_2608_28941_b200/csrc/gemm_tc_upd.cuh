@@ -101,6 +101,10 @@ __device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wa
 
 constexpr int kUtcBM = 128, kUtcBN = 64;
 constexpr int kUtcEpi = 8;
+// The sampled panel Y is summed in tensor memory over this many times more 64-element pieces of its contraction
+// index than Z is (the chunk length of rrf_set_single_engine): an error in Y moves the sample, not the accuracy
+// of the factorisation, and every drain of Y stalls both the issuer and the epilogue warps for one product.
+constexpr int kUtcYChunkFactor = 8;
 constexpr int kUtcThreads = (kUtcEpi + 4) * 32;     // + W producer, MMA issuer, Zt producer, OmegaT producer
 
 // Shared memory is three independent TMA rings, because the three inputs of a tile are given back at

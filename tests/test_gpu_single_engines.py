@@ -131,6 +131,8 @@ def test_last_pass_without_a_sample_at_full_width(h):
                         flags=rrf.RRF_FLAG_ONE_QUEUE | rrf.RRF_FLAG_INPLACE)
         out[engine] = (g.k, Ac, g.B[:g.k].clone())
     assert out[MMA][0] == out[TC][0] == 128
-    scale = dA.abs().max().item()
-    assert (out[MMA][1][128:] - out[TC][1][128:]).abs().max().item() <= 2e-5 * scale
-    assert (out[MMA][2] - out[TC][2]).abs().max().item() <= 2e-5 * scale
+    # the bar of the parity tests (1e-4 of the largest entry of B); a tile computed from a stage that was
+    # overwritten under it is off by the size of the entries themselves
+    scale = out[MMA][2].abs().max().item()
+    assert (out[MMA][1][128:] - out[TC][1][128:]).abs().max().item() <= 1e-4 * scale
+    assert (out[MMA][2] - out[TC][2]).abs().max().item() <= 1e-4 * scale
