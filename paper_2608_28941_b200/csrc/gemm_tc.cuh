@@ -115,6 +115,11 @@ __device__ __forceinline__ void tmem_ld16x4(uint32_t t0, uint32_t t1, uint32_t t
   }
 }
 
+// x rounded to TF32 (nearest, ties away from zero - what cvt.rna.tf32.f32 returns) with two integer
+// instructions, which issue at the full rate where the conversion instruction does not.  A NaN may come out as a
+// signed zero; the kernels below use the planes only as tensor-core operands and keep x itself for everything else.
+__device__ __forceinline__ float tf32_rn(float x) { return __uint_as_float((__float_as_uint(x) + 0x1000u) & 0xFFFFE000u); }
+
 constexpr int kTcBN = 128;     // columns of W per accumulator = rows of D = tensor-memory lanes
 constexpr int kTcSub = 32;     // rows (contraction indices) per ring stage; a 64-row tile is two stages
 constexpr int kTcConv = 8;     // warps that split operands and drain the accumulator
@@ -261,14 +266,14 @@ __global__ void __launch_bounds__(kTcThreads, 1)
 #pragma unroll
       for (int bx = 0; bx < NBV + NBC; ++bx) {
         float4 h, l;
-        h.x = __uint_as_float(to_tf32(x[bx].x));
-        h.y = __uint_as_float(to_tf32(x[bx].y));
-        h.z = __uint_as_float(to_tf32(x[bx].z));
-        h.w = __uint_as_float(to_tf32(x[bx].w));
-        l.x = __uint_as_float(to_tf32(x[bx].x - h.x));
-        l.y = __uint_as_float(to_tf32(x[bx].y - h.y));
-        l.z = __uint_as_float(to_tf32(x[bx].z - h.z));
-        l.w = __uint_as_float(to_tf32(x[bx].w - h.w));
+        h.x = tf32_rn(x[bx].x);
+        h.y = tf32_rn(x[bx].y);
+        h.z = tf32_rn(x[bx].z);
+        h.w = tf32_rn(x[bx].w);
+        l.x = tf32_rn(x[bx].x - h.x);
+        l.y = tf32_rn(x[bx].y - h.y);
+        l.z = tf32_rn(x[bx].z - h.z);
+        l.w = tf32_rn(x[bx].w - h.w);
         const int hb = bx < NBV ? bx : 2 * NBV + (bx - NBV);          // box of the hi plane in the operand stage
         const int lb = bx < NBV ? bx + NBV : 2 * NBV + NBC + (bx - NBV);
         sts128(dst + hb * BOX, h);

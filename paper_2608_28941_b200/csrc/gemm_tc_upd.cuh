@@ -42,9 +42,9 @@ __global__ void split_planes_kernel(const float* __restrict__ src, long long lds
   for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < total; i += (long long)gridDim.x * blockDim.x) {
     const int r = (int)(i / cols), c = (int)(i - (long long)r * cols);
     const float x = src[(size_t)r * lds + c];
-    const float h = __uint_as_float(to_tf32(x));
+    const float h = tf32_rn(x);
     dst[(size_t)r * ldd + c] = h;
-    dst[plane + (size_t)r * ldd + c] = __uint_as_float(to_tf32(x - h));
+    dst[plane + (size_t)r * ldd + c] = tf32_rn(x - h);
   }
 }
 
@@ -367,8 +367,8 @@ __global__ void __launch_bounds__(kUtcThreads, 1)
             const float xs[4] = {x.x, x.y, x.z, x.w};
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
-              hi[e4 * 4 + e] = __uint_as_float(to_tf32(xs[e]));
-              lo[e4 * 4 + e] = __uint_as_float(to_tf32(xs[e] - hi[e4 * 4 + e]));
+              hi[e4 * 4 + e] = tf32_rn(xs[e]);
+              lo[e4 * 4 + e] = tf32_rn(xs[e] - hi[e4 * 4 + e]);
             }
           }
           tmem_st16(tlane + TV + half * HB + g * 16, hi);
@@ -458,8 +458,8 @@ __global__ void __launch_bounds__(kUtcThreads, 1)
           float hi[16], lo[16];
 #pragma unroll
           for (int e = 0; e < 16; ++e) {
-            hi[e] = __uint_as_float(to_tf32(y[g * 16 + e]));
-            lo[e] = __uint_as_float(to_tf32(y[g * 16 + e] - hi[e]));
+            hi[e] = tf32_rn(y[g * 16 + e]);
+            lo[e] = tf32_rn(y[g * 16 + e] - hi[e]);
           }
           tmem_st16(tlane + TW + half * 32 + g * 16, hi);
           tmem_st16(tlane + TW + BN + half * 32 + g * 16, lo);
