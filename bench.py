@@ -30,7 +30,10 @@ import numpy as np  # noqa: E402
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel of the default
 # workload, from the ncu capture summarised in profiles/kernels_cfg2_4096x4096_b64.md (captured on a
 # 4096 x 4096 case and scaled to the bench's average launch by the elements processed).
-NCU_TRAFFIC_BYTES = {("cfg2", "update"): 1.07e9, ("cfg2", "vtw"): 136.3e6 * 3.875}
+NCU_TRAFFIC_BYTES = {("cfg2", "update"): 1.07e9, ("cfg2", "vtw"): 136.3e6 * 3.875,
+                     # tcgen05 kernels, block step 0 (profiles/kernels_cfg4_4096x11008_fp32_b64_tcgen05.md); of the update's
+                     # 180 MB of writes 59 MB were still in L2 when the launch ended
+                     ("cfg4", "update"): 185.9e6 + 121.1e6, ("cfg4", "vtw"): 178.6e6 + 5.6e6}
 
 NOMINAL_FP64_OVER_BF16 = 37.0 / 2250.0   # HGX B200 dense figures: FP64 tensor 37 TF, bf16 2250 TF
 
