@@ -72,6 +72,7 @@ struct rrf_ctx {
   std::vector<unsigned char> gcand;      // arguments of the last directly enqueued call
   std::vector<std::pair<int, int>> gmarks;
   int graph_off;                         // set when a capture failed: enqueue directly from then on
+  int cluster_ok;                        // a 16-CTA cluster of the panel kernel can be resident on this device
   int f32_engine;                        // single-precision V^T W: 0 = mma.sync 3xTF32, 1 = tcgen05 3xTF32
   int tc_chunk;                          // tcgen05: 64-row tiles summed in tensor memory between round-to-nearest adds
 };
@@ -170,12 +171,51 @@ static const void* panel_variant(int q) {
     default: return (const void*)panel_kernel<T, 7, 1, false>;
   }
 }
-struct PanelPlan { int G, R, Rp, variant; size_t smem; };
+template <typename T>
+static const void* panel_variant_cl(int q) {     // the same shapes as one thread-block cluster (padded ones only)
+  switch (q) {
+    case 0: return (const void*)panel_kernel<T, 2, 1, true, true>;
+    case 1: return (const void*)panel_kernel<T, 4, 1, true, true>;
+    case 2: return (const void*)panel_kernel<T, 7, 1, true, true>;
+    case 3: return (const void*)panel_kernel<T, 5, 2, true, true>;
+    default: return (const void*)panel_kernel<T, 8, 2, true, true>;
+  }
+}
+constexpr int kPanelVariantsCl = 5;
+constexpr int kClusterMaxRows = 128;
+struct PanelPlan { int G, R, Rp, variant; size_t smem; bool cl; };
 // ctas == 0: the panel is spread over every SM (short slabs, short passes).  ctas > 0: the panel is
 // confined to that many CTAs so that the other SMs stay free for the GEMM kernels of the look-ahead
 // schedule; `fix` adds the b rows above the panel and the shared memory of the late reflector
 // application.
+// The panel as ONE thread-block cluster (sums through distributed shared memory): possible when at most
+// kClusterMax slabs hold it.  The grid is a power of two so that every cluster size is one the hardware takes;
+// CTAs past the last row hold no rows and only take part in the exchanges.
+static bool plan_panel_cl(const rrf_ctx* h, long long rows, int b, PanelPlan* p, bool fix) {
+  if (!h->cluster_ok || (fix && b > 64)) return false;
+  const long long ext = rows + (fix ? b : 0);
+  const int R = std::max(64, ceil_div(ext, kClusterMax));
+  // With slabs taller than this the longer pass over a slab costs more than the cheaper exchange saves
+  // (measured: 4096 x 64 takes 279 us as one cluster of 16 against 260 us on 148 CTAs; 1024 x 16 falls from 64 to 54)
+  if (R > kClusterMaxRows) return false;
+  int G = 1;
+  while (G < ceil_div(ext, R)) G *= 2;
+  if (G > kClusterMax) return false;
+  const size_t extra = (size_t)panel_extra_doubles(b) + (fix ? panel_fix_doubles(b) : 0) + panel_cluster_doubles(b);
+  for (int q = 0; q < kPanelVariantsCl; ++q) {
+    if (R > kVariantRows[q]) continue;
+    p->R = R;
+    p->G = G;
+    p->Rp = kVariantRows[q] + 1;
+    p->variant = q;
+    p->cl = true;
+    p->smem = ((size_t)b * p->Rp + extra) * sizeof(double);
+    if (p->smem <= (size_t)h->panel_smem_max) return true;
+  }
+  return false;
+}
 static bool plan_panel(const rrf_ctx* h, long long rows, int b, PanelPlan* p, int ctas = 0, bool fix = false) {
+  p->cl = false;
   if (fix && b > 64) return false;
   const long long ext = rows + (fix ? b : 0);
   // tall slabs keep the grid, and with it the all-to-all read of the partial sums, small
@@ -588,6 +628,7 @@ struct PanelOpts {
   unsigned* bar_used = nullptr;    // out: what this launch adds to the counter
   cudaStream_t st_t = nullptr;     // side stream for the T factor, with its fork / join events
   cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
+  bool no_cluster = false;         // keep the per-column kernel on a cooperative grid even where one cluster would hold the panel
   bool tree = false;               // b <= 64: use the tree kernel (no grid barrier per column)
   bool blocked = false;            // use the blocked kernel (micro-panels of eight columns, panel_blk.cuh) if it fits
   bool global_slab = false;        // blocked kernel: keep the slabs in global memory
@@ -661,16 +702,34 @@ static rrf_status_t launch_panel(rrf_ctx* h, int dtype, const void* Y, PanelSour
     e = cudaLaunchCooperativeKernel(fn, dim3(bp.G), dim3(kPanelThreads), args, smem, st);
   } else {
     PanelPlan pp;
-    if (!plan_panel(h, rows, b, &pp, o.ctas, o.fix.enabled != 0)) return RRF_ERR_WORKSPACE;
+    const bool as_cluster = !o.no_cluster && !o.blocked && plan_panel_cl(h, rows, b, &pp, o.fix.enabled != 0);
+    if (!as_cluster && !plan_panel(h, rows, b, &pp, o.ctas, o.fix.enabled != 0)) return RRF_ERR_WORKSPACE;
     int R = pp.R, Rp = pp.Rp;
     void* args[] = {&Y,   &src, &alt, &fused_flag, &rows_i, &b,    &R,    &Rp,        &V,   &ldv,      &P,
                     &piv, &gram, &tau, &bar,       &ctrl,   &done_flag, &fix, &bar_base, &Tmerged, &ldt, &csq};
     if (o.merge_t) pp.smem = std::max(pp.smem, tsmem);
-    if (o.bar_used != nullptr) *o.bar_used = (unsigned)(b + (o.fix.enabled ? 2 : 0)) * (unsigned)pp.G;
+    if (o.bar_used != nullptr) *o.bar_used = as_cluster ? 0u : (unsigned)(b + (o.fix.enabled ? 2 : 0)) * (unsigned)pp.G;
     if (o.g_out != nullptr) *o.g_out = pp.G;
     mark(RRF_PHASE_PANEL, step);
-    const void* fn = dtype == RRF_F64 ? panel_variant<double>(pp.variant) : panel_variant<float>(pp.variant);
-    e = cudaLaunchCooperativeKernel(fn, dim3(pp.G), dim3(kPanelThreads), args, pp.smem, st);
+    if (as_cluster) {
+      const void* fn = dtype == RRF_F64 ? panel_variant_cl<double>(pp.variant) : panel_variant_cl<float>(pp.variant);
+      cudaLaunchConfig_t cfg = {};
+      cfg.gridDim = dim3(pp.G);
+      cfg.blockDim = dim3(kPanelThreads);
+      cfg.dynamicSmemBytes = pp.smem;
+      cfg.stream = st;
+      cudaLaunchAttribute at[1];
+      at[0].id = cudaLaunchAttributeClusterDimension;
+      at[0].val.clusterDim.x = pp.G;
+      at[0].val.clusterDim.y = 1;
+      at[0].val.clusterDim.z = 1;
+      cfg.attrs = at;
+      cfg.numAttrs = 1;
+      e = cudaLaunchKernelExC(&cfg, fn, args);
+    } else {
+      const void* fn = dtype == RRF_F64 ? panel_variant<double>(pp.variant) : panel_variant<float>(pp.variant);
+      e = cudaLaunchCooperativeKernel(fn, dim3(pp.G), dim3(kPanelThreads), args, pp.smem, st);
+    }
   }
   if (e == cudaSuccess && !o.merge_t) {
     cudaStream_t tt = st;
@@ -696,12 +755,16 @@ static rrf_status_t launch_panel(rrf_ctx* h, int dtype, const void* Y, PanelSour
 }
 
 // attributes of the panel and T-factor kernels; reports the dynamic shared memory a panel may use
-static cudaError_t setup_panel_kernels(int smem_optin, int* panel_smem_max) {
+static cudaError_t setup_panel_kernels(int smem_optin, int* panel_smem_max, int* cluster_ok) {
   cudaError_t e;
-  const void* pk[2 * kPanelVariants];
+  const void* pk[2 * kPanelVariants + 2 * kPanelVariantsCl];
   for (int q = 0; q < kPanelVariants; ++q) {
     pk[q] = panel_variant<double>(q);
     pk[kPanelVariants + q] = panel_variant<float>(q);
+  }
+  for (int q = 0; q < kPanelVariantsCl; ++q) {
+    pk[2 * kPanelVariants + q] = panel_variant_cl<double>(q);
+    pk[2 * kPanelVariants + kPanelVariantsCl + q] = panel_variant_cl<float>(q);
   }
   size_t stat = 0;
   for (const void* f : pk) {
@@ -714,6 +777,32 @@ static cudaError_t setup_panel_kernels(int smem_optin, int* panel_smem_max) {
   for (const void* f : pk) {
     e = cudaFuncSetAttribute(f, cudaFuncAttributeMaxDynamicSharedMemorySize, *panel_smem_max);
     if (e != cudaSuccess) return e;
+  }
+  // clusters of up to kClusterMax CTAs (above the portable 8): allowed per kernel, and checked once for residency
+  *cluster_ok = 1;
+  for (int q = 0; q < 2 * kPanelVariantsCl; ++q) {
+    if (cudaFuncSetAttribute(pk[2 * kPanelVariants + q], cudaFuncAttributeNonPortableClusterSizeAllowed, 1) != cudaSuccess) {
+      cudaGetLastError();
+      *cluster_ok = 0;
+    }
+  }
+  if (*cluster_ok) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(kClusterMax);
+    cfg.blockDim = dim3(kPanelThreads);
+    cfg.dynamicSmemBytes = *panel_smem_max;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeClusterDimension;
+    at[0].val.clusterDim.x = kClusterMax;
+    at[0].val.clusterDim.y = 1;
+    at[0].val.clusterDim.z = 1;
+    cfg.attrs = at;
+    cfg.numAttrs = 1;
+    int nclusters = 0;
+    if (cudaOccupancyMaxActiveClusters(&nclusters, pk[2 * kPanelVariants + kPanelVariantsCl - 1], &cfg) != cudaSuccess || nclusters < 1) {
+      cudaGetLastError();
+      *cluster_ok = 0;
+    }
   }
   const int tmax = (128 * 129 + 64 * 65) * 8;
   e = cudaFuncSetAttribute(tfactor_kernel<double>, cudaFuncAttributeMaxDynamicSharedMemorySize, tmax);
@@ -755,7 +844,7 @@ static cudaError_t setup_blk_kernels(int smem_optin, int* blk_smem_max) {
   return cudaSuccess;
 }
 
-static cudaError_t setup_all(int smem_optin, int* panel_smem_max) {
+static cudaError_t setup_all(int smem_optin, int* panel_smem_max, int* cluster_ok) {
   cudaError_t e;
   for (int b : {16, 32, 64, 128}) {
     e = get_ops(RRF_F64, b)->setup();
@@ -765,7 +854,7 @@ static cudaError_t setup_all(int smem_optin, int* panel_smem_max) {
     e = get_ops(RRF_F32, b)->setup();
     if (e != cudaSuccess) return e;
   }
-  return setup_panel_kernels(smem_optin, panel_smem_max);
+  return setup_panel_kernels(smem_optin, panel_smem_max, cluster_ok);
 }
 
 static size_t tc_zsplit_bytes(int npad, int b) { return align_up((size_t)2 * npad * b * sizeof(float), 256); }
@@ -886,7 +975,7 @@ rrf_status_t rrf_create(rrf_handle_t* out, int device) {
   if (e == cudaSuccess && (fn == nullptr || q != cudaDriverEntryPointSuccess)) e = cudaErrorUnknown;
   if (e == cudaSuccess && h->sms > kMaxSms) e = cudaErrorInvalidConfiguration;
   h->encode = reinterpret_cast<EncodeTiledFn>(fn);
-  if (e == cudaSuccess) e = setup_all(h->smem_optin, &h->panel_smem_max);
+  if (e == cudaSuccess) e = setup_all(h->smem_optin, &h->panel_smem_max, &h->cluster_ok);
   if (e == cudaSuccess) e = setup_tree_kernels(h->smem_optin, &h->tsqr_smem_max);
   if (e == cudaSuccess) e = setup_blk_kernels(h->smem_optin, &h->blk_smem_max);
   if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&h->aux, cudaStreamNonBlocking);
@@ -1905,7 +1994,8 @@ static cudaError_t static_setup(int dev, StaticDevice* sd) {
   if (e != cudaSuccess) return e;
   e = cudaDeviceGetAttribute(&smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
   if (e != cudaSuccess) return e;
-  e = setup_panel_kernels(smem_optin, &sd->panel_smem_max);
+  int cluster_unused = 0;
+  e = setup_panel_kernels(smem_optin, &sd->panel_smem_max, &cluster_unused);
   if (e != cudaSuccess) return e;
   sd->ptr = static_cast<unsigned char*>(ptr);
   return cudaSuccess;

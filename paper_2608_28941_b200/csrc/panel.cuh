@@ -39,6 +39,73 @@ __device__ __forceinline__ bool grid_barrier(unsigned* ctr, unsigned target, Ctr
   return ok_s != 0;
 }
 
+// ---------------------------------------------------------------- thread-block cluster exchange
+// A panel that fits the shared memory of at most 16 CTAs is factored by ONE cluster: the per-column sums
+// travel through distributed shared memory (every CTA writes its partials straight into every peer's
+// shared memory) and the barrier is an mbarrier per CTA on which every peer arrives - about 0.7 to 1 us per
+// column against the 2.4 us of an all-to-all exchange through L2.
+constexpr int kClusterMax = 16;
+__host__ __device__ constexpr int panel_cluster_doubles(int b) { return 2 * kClusterMax * b + 2 * b; }
+
+__device__ __forceinline__ uint32_t cl_map(uint32_t addr, uint32_t rank) {   // the same address in CTA `rank` of the cluster
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ void cl_st(uint32_t addr, double v) {
+  asm volatile("st.shared::cluster.f64 [%0], %1;" ::"r"(addr), "d"(v) : "memory");
+}
+__device__ __forceinline__ void cl_st(uint32_t addr, int v) {
+  asm volatile("st.shared::cluster.b32 [%0], %1;" ::"r"(addr), "r"(v) : "memory");
+}
+__device__ __forceinline__ void cl_arrive(uint32_t bar_addr) {
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(bar_addr) : "memory");
+}
+__device__ __forceinline__ uint32_t cl_try_wait(uint64_t* bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(smem_u32(bar)), "r"(parity)
+      : "memory");
+  return ok;
+}
+// the hardware barrier of the cluster (unbounded: used once, before any data-dependent exit)
+__device__ __forceinline__ void cl_hw_sync() {
+  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// Barrier over the G CTAs of the cluster: every CTA arrives on every peer's mbarrier and waits, bounded, on its
+// own.  Everything this CTA stored before it - into peers' shared memory, or (with `global_too`) into global
+// memory - is visible to the peers behind it.  `nx` counts the barriers passed (the phase parity).
+__device__ __forceinline__ bool cluster_barrier(uint64_t* cbar, unsigned& nx, int G, bool global_too, Ctrl* ctrl) {
+  __shared__ int cl_ok_s;
+  __syncthreads();
+  if ((int)threadIdx.x < G) {
+    if (global_too) __threadfence();
+    cl_arrive(cl_map(smem_u32(cbar), threadIdx.x));
+  }
+  if (threadIdx.x == 0) {
+    int ok = 1;
+    if (!cl_try_wait(cbar, nx & 1u)) {
+      const long long t0 = clock64();
+      while (!cl_try_wait(cbar, nx & 1u)) {
+        if (clock64() - t0 > kWaitLimitClocks) {
+          atomicExch(&ctrl->status, (int)RRF_ERR_TIMEOUT);
+          atomicExch(&ctrl->done, 1);
+          ok = 0;
+          break;
+        }
+      }
+    }
+    cl_ok_s = ok;
+  }
+  ++nx;
+  __syncthreads();
+  return cl_ok_s != 0;
+}
+
 // Sums four per-lane values over the warp with 6 adds and 6 shuffles instead of 20: after the
 // exchanges with lanes ^16 and ^8 every lane carries one of the four sums (number 2*bit4 + bit3 of
 // its lane index), which three more butterfly steps complete.  Fixed order, so reproducible.
@@ -199,7 +266,9 @@ __device__ __forceinline__ void tfactor_block(const double* __restrict__ gram, c
 // slab is allocated at that full height and zero filled below its last row, which removes every
 // per-element bounds test from the pass; PAD = false keeps the tests (for the one shape whose slab only
 // fits unpadded).
-template <typename T, int QMAX, int RH, bool PAD = true>
+// CL: the grid is one thread-block cluster of at most kClusterMax CTAs; sums and pivot rows are exchanged through
+// distributed shared memory and the barriers are cluster_barrier (P, piv and the barrier counter are not used).
+template <typename T, int QMAX, int RH, bool PAD = true, bool CL = false>
 __global__ void __launch_bounds__(kPanelThreads)
     panel_kernel(const T* __restrict__ Y, PanelSource src_fused, PanelSource src_alt, const int* __restrict__ fused_flag,
                  int rows, int b, int R, int Rp,
@@ -212,7 +281,27 @@ __global__ void __launch_bounds__(kPanelThreads)
                  unsigned bar_base,                 // value of the barrier counter when this launch starts
                  T* __restrict__ Tout, long long ldt,     // non-NULL: CTA 0 also builds the T factor at the end
                  double* __restrict__ csq) {              // non-NULL: [b][Gp] per-CTA sums of squares of the panel's columns
-  if (*reinterpret_cast<const volatile int*>(done_flag) || *reinterpret_cast<const volatile int*>(&ctrl->status) < 0) return;
+  __shared__ uint64_t cbar;      // cluster mode: this CTA's barrier, on which every CTA of the cluster arrives
+  __shared__ int go_s;
+  unsigned nx = 0;               // cluster barriers passed
+  if (CL) {
+    // The decision to run must be the same in every CTA of the cluster (a CTA that left would never arrive at
+    // its peers' barriers): rank 0 reads the flags and tells everyone, under the hardware barrier of the cluster.
+    if (threadIdx.x == 0) {
+      mbar_init(&cbar, gridDim.x);
+      mbar_fence_init();
+    }
+    cl_hw_sync();                // every CTA of the cluster runs and has its barrier initialised
+    if (blockIdx.x == 0 && threadIdx.x < gridDim.x) {
+      const int go = !(*reinterpret_cast<const volatile int*>(done_flag) ||
+                       *reinterpret_cast<const volatile int*>(&ctrl->status) < 0);
+      cl_st(cl_map(smem_u32(&go_s), threadIdx.x), go);
+    }
+    cl_hw_sync();
+    if (!go_s) return;
+  } else {
+    if (*reinterpret_cast<const volatile int*>(done_flag) || *reinterpret_cast<const volatile int*>(&ctrl->status) < 0) return;
+  }
   // the panel's entries were sampled by the fused update, or - where the predictor had skipped that - by
   // the separate sample kernel, in its layout
   const bool use_alt = fused_flag != nullptr && *fused_flag == 0;
@@ -223,6 +312,9 @@ __global__ void __launch_bounds__(kPanelThreads)
   double* p_s = w_s + b;                  // [2][b]: per row group, then (first b) the grid-wide sums
   double* pr_s = p_s + 2 * b;             // [b]
   double* sc_s = pr_s + b;                // [4]: tau_j, 1/(alpha - beta)
+  // cluster mode: partial sums [2][kClusterMax][b] and pivot rows [2][b] written by the peers, behind everything else
+  double* px_s = sc_s + 4 + (fix.enabled ? panel_fix_doubles(b) : 0);
+  double* prx_s = px_s + 2 * kClusterMax * b;
 
   constexpr int NT = kPanelThreads, NW = NT / 32;
   constexpr int NWC = NW / RH;            // warps that share the columns within one row group
@@ -328,7 +420,9 @@ __global__ void __launch_bounds__(kPanelThreads)
         }
       }
     }
-    if (!grid_barrier(bar, bar_base + (++nbar) * (unsigned)G, ctrl)) return;
+    if (CL) {
+      if (!cluster_barrier(&cbar, nx, G, true, ctrl)) return;
+    } else if (!grid_barrier(bar, bar_base + (++nbar) * (unsigned)G, ctrl)) return;
     // Phase 2: CTA c owns columns c, c + G, ... of G = sum of the partials (in CTA order) and of
     // M = Tp^T G, column by column: M[k][c2] = sum_{l <= k} Tp[l][k] G[l][c2].
     {
@@ -366,7 +460,9 @@ __global__ void __launch_bounds__(kPanelThreads)
         }
       }
     }
-    if (!grid_barrier(bar, bar_base + (++nbar) * (unsigned)G, ctrl)) return;
+    if (CL) {
+      if (!cluster_barrier(&cbar, nx, G, true, ctrl)) return;
+    } else if (!grid_barrier(bar, bar_base + (++nbar) * (unsigned)G, ctrl)) return;
     // Phase 3: S -= Vp[slab] M.  A task is a 16-row x 8-column tile of a chunk.
     {
       const int PV = b + 4, PM = b + 8;
@@ -479,6 +575,31 @@ __global__ void __launch_bounds__(kPanelThreads)
       }
     }
     __syncthreads();
+    if (CL) {
+      // this CTA's b partial sums, and from the CTA that holds it the pivot row, into every peer's shared memory
+      // (two buffers: a peer may be one column ahead, never two)
+      const int pb = j & 1;
+      for (int idx = tid; idx < G * b; idx += NT) {
+        const int q = idx >> lb, c = idx & (b - 1);
+        double v = p_s[c];
+#pragma unroll
+        for (int h = 1; h < RH; ++h) v += p_s[h * b + c];
+        cl_st(cl_map(smem_u32(px_s + ((size_t)pb * kClusterMax + cta) * b + c), q), v);
+      }
+      if (pr >= gr0 && pr < gr0 + nloc)
+        for (int idx = tid; idx < G * b; idx += NT) {
+          const int q = idx >> lb, c = idx & (b - 1);
+          cl_st(cl_map(smem_u32(prx_s + pb * b + c), q), S[(size_t)c * Rp + (pr - gr0)]);
+        }
+      if (!cluster_barrier(&cbar, nx, G, false, ctrl)) return;
+      if (tid < b) {
+        double v = 0.0;
+        for (int q = 0; q < G; ++q) v += px_s[((size_t)pb * kClusterMax + q) * b + tid];     // CTA order: reproducible
+        p_s[tid] = v;
+        pr_s[tid] = prx_s[pb * b + tid];
+      }
+      __syncthreads();
+    } else {
     double* Pj = P + (size_t)(j & 1) * b * Gp;
     for (int c = tid; c < b; c += NT) {
       double v = p_s[c];
@@ -520,6 +641,7 @@ __global__ void __launch_bounds__(kPanelThreads)
       }
       if (tid < b) pr_s[tid] = prv;
       __syncthreads();
+    }
     }
     // The reflector's scalars are computed once (square root and divisions are long FP64 sequences
     // and the SM has few FP64 lanes) and shared: tau, 1/(alpha - beta), and whether there is
