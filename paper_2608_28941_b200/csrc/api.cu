@@ -557,11 +557,15 @@ struct Ops {
               (const float*)x.Om + (size_t)j0 * x.ldom, x.ldom, B, ncols, (float*)x.osplit, x.ldo2, &ctrl->done);
         // where the updated tiles go: the working matrix, and the rows of B that this pass completes
         CUtensorMap tmCs, tmTs;
-        if (!make_map(x.h, &tmCs, RRF_F32, C, (unsigned long long)r0 + rows, ncols, ldc, 32)) return;
-        if (top_rows > 0) {
-          if (!make_map(x.h, &tmTs, RRF_F32, top, top_rows, ncols, ldtop, 32)) return;
-        } else {
-          tmTs = tmCs;
+        bool maps_ok = make_map(x.h, &tmCs, RRF_F32, C, (unsigned long long)r0 + rows, ncols, ldc, 32);
+        if (maps_ok && top_rows > 0) maps_ok = make_map(x.h, &tmTs, RRF_F32, top, top_rows, ncols, ldtop, 32);
+        if (top_rows <= 0) tmTs = tmCs;
+        if (!maps_ok) {
+          // cannot happen for arguments that passed the entry checks (aligned bases, leading dimensions of whole
+          // 16 bytes); if it does, the run ends with an error status instead of an update that never ran
+          static const int kErr[2] = {1, (int)RRF_ERR_CUDA};     // Ctrl::done, Ctrl::status
+          cudaMemcpyAsync(ctrl, kErr, sizeof(kErr), cudaMemcpyHostToDevice, st);
+          return;
         }
         upd_tc_kernel<B><<<p.P, kUtcThreads, UtcCfg<B>::SMEM, st>>>(
             tmC, x.tmZs, x.tmOs, tmCs, tmTs, (const float*)x.V, x.ldv, r0, rows, ncols, cv0, top_rows, j0 >= 0 ? 1 : 0,
