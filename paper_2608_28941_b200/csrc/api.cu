@@ -178,10 +178,12 @@ static const void* panel_variant_cl(int q) {     // the same shapes as one threa
     case 1: return (const void*)panel_kernel<T, 4, 1, true, true>;
     case 2: return (const void*)panel_kernel<T, 7, 1, true, true>;
     case 3: return (const void*)panel_kernel<T, 5, 2, true, true>;
-    default: return (const void*)panel_kernel<T, 8, 2, true, true>;
+    case 4: return (const void*)panel_kernel<T, 8, 2, true, true>;
+    default: return (const void*)panel_kernel<T, 8, 1, true, true, true>;   // slab in registers during the column loop
   }
 }
-constexpr int kPanelVariantsCl = 5;
+constexpr int kPanelVariantsCl = 6;
+constexpr int kPanelVariantReg = 5;
 constexpr int kClusterMaxRows = 128;
 struct PanelPlan { int G, R, Rp, variant; size_t smem; bool cl; };
 // ctas == 0: the panel is spread over every SM (short slabs, short passes).  ctas > 0: the panel is
@@ -197,12 +199,24 @@ static bool plan_panel_cl(const rrf_ctx* h, long long rows, int b, PanelPlan* p,
   const int R = std::max(64, ceil_div(ext, kClusterMax));
   // With slabs taller than this the longer pass over a slab costs more than the cheaper exchange saves
   // (measured: 4096 x 64 takes 279 us as one cluster of 16 against 260 us on 148 CTAs; 1024 x 16 falls from 64 to 54)
+  // With the register-resident column loop (b <= 64) a 4096 x 64 panel takes 232 us on its own, but inside a run, where
+  // 16 CTAs also sum the partial panels and store V, the 4096-row passes of config 4 take 284 us against 261 us.
   if (R > kClusterMaxRows) return false;
+  const bool reg = b <= 64;
   int G = 1;
   while (G < ceil_div(ext, R)) G *= 2;
   if (G > kClusterMax) return false;
   const size_t extra = (size_t)panel_extra_doubles(b) + (fix ? panel_fix_doubles(b) : 0) + panel_cluster_doubles(b);
-  for (int q = 0; q < kPanelVariantsCl; ++q) {
+  if (reg) {
+    p->R = R;
+    p->G = G;
+    p->Rp = kRegRows + 1;
+    p->variant = kPanelVariantReg;
+    p->cl = true;
+    p->smem = ((size_t)b * p->Rp + extra) * sizeof(double);
+    return p->smem <= (size_t)h->panel_smem_max;
+  }
+  for (int q = 0; q < kPanelVariantReg; ++q) {
     if (R > kVariantRows[q]) continue;
     p->R = R;
     p->G = G;
@@ -2047,6 +2061,9 @@ extern "C" rrf_status_t rrf_panel_qr_static(int32_t dtype, int64_t rows, int32_t
 }
 
 #ifdef RRF_TSQR_TRACE
+extern "C" int rrf_debug_trace_panel(unsigned long long* out) {
+  return (int)cudaMemcpyFromSymbol(out, rrf::g_pcl_trace, sizeof(unsigned long long) * 16);
+}
 extern "C" int rrf_debug_trace(unsigned long long* out) {
   return (int)cudaMemcpyFromSymbol(out, rrf::g_tsqr_trace, sizeof(unsigned long long) * 64);
 }

@@ -45,7 +45,14 @@ __device__ __forceinline__ bool grid_barrier(unsigned* ctr, unsigned target, Ctr
 // shared memory) and the barrier is an mbarrier per CTA on which every peer arrives - about 0.7 to 1 us per
 // column against the 2.4 us of an all-to-all exchange through L2.
 constexpr int kClusterMax = 16;
-__host__ __device__ constexpr int panel_cluster_doubles(int b) { return 2 * kClusterMax * b + 2 * b; }
+#ifdef RRF_TSQR_TRACE
+__device__ unsigned long long g_pcl_trace[16];
+#define PCL_STAMP(k) if (j == 8 && blockIdx.x == 0 && threadIdx.x == 0) g_pcl_trace[k] = (unsigned long long)clock64()
+#else
+#define PCL_STAMP(k)
+#endif
+constexpr int kRegRows = 256;       // rows of a slab in the register-resident column loop
+__host__ __device__ constexpr int panel_cluster_doubles(int b) { return 2 * kClusterMax * b + 2 * b + 2 * kRegRows + b; }
 
 __device__ __forceinline__ uint32_t cl_map(uint32_t addr, uint32_t rank) {   // the same address in CTA `rank` of the cluster
   uint32_t r;
@@ -268,7 +275,12 @@ __device__ __forceinline__ void tfactor_block(const double* __restrict__ gram, c
 // fits unpadded).
 // CL: the grid is one thread-block cluster of at most kClusterMax CTAs; sums and pivot rows are exchanged through
 // distributed shared memory and the barriers are cluster_barrier (P, piv and the barrier counter are not used).
-template <typename T, int QMAX, int RH, bool PAD = true, bool CL = false>
+// REG (with CL, b <= 64, slabs of at most 256 rows): during the column loop the slab lives in REGISTERS - lane l of
+// warp w keeps rows l, l + 32, ..., l + 224 of columns 4w ... 4w + 3 - so a column costs each thread 32 fused
+// multiply-adds and a warp reduction instead of a pass over the slab in shared memory (which is what makes a slab
+// of 256 rows, i.e. a 4096-row panel on 16 CTAs, worth its while).  Column j and the finished v_{j-1} go round
+// through two 256-element arrays in shared memory.
+template <typename T, int QMAX, int RH, bool PAD = true, bool CL = false, bool REG = false>
 __global__ void __launch_bounds__(kPanelThreads)
     panel_kernel(const T* __restrict__ Y, PanelSource src_fused, PanelSource src_alt, const int* __restrict__ fused_flag,
                  int rows, int b, int R, int Rp,
@@ -315,6 +327,9 @@ __global__ void __launch_bounds__(kPanelThreads)
   // cluster mode: partial sums [2][kClusterMax][b] and pivot rows [2][b] written by the peers, behind everything else
   double* px_s = sc_s + 4 + (fix.enabled ? panel_fix_doubles(b) : 0);
   double* prx_s = px_s + 2 * kClusterMax * b;
+  double* ycol_s = prx_s + 2 * b;         // [kRegRows] column j below its pivot (register-resident loop)
+  double* vcol_s = ycol_s + kRegRows;     // [kRegRows] v_{j-1}
+  double* prow_s = vcol_s + kRegRows;     // [b] this CTA's entries of the pivot row
 
   constexpr int NT = kPanelThreads, NW = NT / 32;
   constexpr int NWC = NW / RH;            // warps that share the columns within one row group
@@ -511,6 +526,140 @@ __global__ void __launch_bounds__(kPanelThreads)
   }
 
   double tau_prev = 0.0;
+  if constexpr (CL && REG) {
+    static_assert(QMAX == 8 && RH == 1 && PAD, "the register tile is 8 rows x 4 columns per thread");
+    const bool has = warp < (b >> 2);                  // warps that hold columns
+    const int c0 = warp * 4;
+    double x[8][4];
+#pragma unroll
+    for (int q = 0; q < 8; ++q)
+#pragma unroll
+      for (int u = 0; u < 4; ++u) x[q][u] = has ? S[(size_t)(c0 + u) * Rp + lane + 32 * q] : 0.0;
+    for (int j = 0; j < b; ++j) {
+      const int pr = row0 + j;
+      const int ow = j >> 2, uj = j & 3;               // warp and tile column that hold column j
+      PCL_STAMP(0);
+      // pending reflector H_{j-1} on this thread's columns j and later (v_{j-1} is zero above its pivot)
+      if (has && j > 0 && tau_prev != 0.0 && c0 + 3 >= j) {
+        double v[8];
+#pragma unroll
+        for (int q = 0; q < 8; ++q) v[q] = vcol_s[lane + 32 * q];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          if (c0 + u >= j) {
+            const double f = tau_prev * w_s[c0 + u];
+#pragma unroll
+            for (int q = 0; q < 8; ++q) x[q][u] -= f * v[q];
+          }
+        }
+      }
+      // column j below its pivot, and this CTA's entries of the pivot row, for everyone
+      if (warp == ow) {
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+          const int r = lane + 32 * q;
+          double yv = 0.0;
+#pragma unroll
+          for (int u = 0; u < 4; ++u) yv = (u == uj) ? x[q][u] : yv;
+          ycol_s[r] = (gr0 + r > pr) ? yv : 0.0;
+        }
+      }
+      if (has && pr >= gr0 && pr < gr0 + nloc && ((pr - gr0) & 31) == lane) {
+        const int qp = (pr - gr0) >> 5;
+#pragma unroll
+        for (int q = 0; q < 8; ++q)
+          if (q == qp) {
+#pragma unroll
+            for (int u = 0; u < 4; ++u) prow_s[c0 + u] = x[q][u];
+          }
+      }
+      __syncthreads();
+      PCL_STAMP(1);
+      if (has) {
+        double y[8], acc[4] = {0.0, 0.0, 0.0, 0.0};
+#pragma unroll
+        for (int q = 0; q < 8; ++q) y[q] = ycol_s[lane + 32 * q];
+#pragma unroll
+        for (int q = 0; q < 8; ++q)
+#pragma unroll
+          for (int u = 0; u < 4; ++u) acc[u] += y[q] * x[q][u];
+        const double tot = warp_sum4(acc, lane);
+        const int u = ((lane >> 4) << 1) | ((lane >> 3) & 1);
+        if ((lane & 7) == 0) p_s[c0 + u] = tot;
+      }
+      __syncthreads();
+      PCL_STAMP(2);
+      {
+        const int pb = j & 1;
+        for (int idx = tid; idx < G * b; idx += NT) {
+          const int q = idx >> lb, c = idx & (b - 1);
+          cl_st(cl_map(smem_u32(px_s + ((size_t)pb * kClusterMax + cta) * b + c), q), p_s[c]);
+        }
+        if (pr >= gr0 && pr < gr0 + nloc)
+          for (int idx = tid; idx < G * b; idx += NT) {
+            const int q = idx >> lb, c = idx & (b - 1);
+            cl_st(cl_map(smem_u32(prx_s + pb * b + c), q), prow_s[c]);
+          }
+        PCL_STAMP(3);
+        if (!cluster_barrier(&cbar, nx, G, false, ctrl)) return;
+        PCL_STAMP(4);
+        if (tid < b) {
+          double v = 0.0;
+          for (int q = 0; q < G; ++q) v += px_s[((size_t)pb * kClusterMax + q) * b + tid];     // CTA order: reproducible
+          p_s[tid] = v;
+          pr_s[tid] = prx_s[pb * b + tid];
+        }
+        __syncthreads();
+      }
+      PCL_STAMP(5);
+      if (warp == 0) {
+        const double alpha = pr_s[j], s2 = p_s[j];
+        double tau = 0.0, rdenom = 0.0;
+        if (s2 != 0.0) {
+          const double beta = -copysign(sqrt(alpha * alpha + s2), alpha);
+          tau = (beta - alpha) / beta;
+          rdenom = 1.0 / (alpha - beta);
+        }
+        if (lane == 0) {
+          sc_s[0] = tau;
+          sc_s[1] = rdenom;
+          if (cta == 0) tau_out[j] = tau;
+        }
+      }
+      __syncthreads();
+      PCL_STAMP(6);
+      const double tau = sc_s[0], rdenom = sc_s[1];     // rdenom == 0 marks H_j = I
+      if (tid < b && tid != j) {
+        const double wv = pr_s[tid] + p_s[tid] * rdenom;
+        w_s[tid] = wv;
+        if (cta == 0 && tid < j) gram[(size_t)j * b + tid] = wv;
+      }
+      // column j becomes v_j (unit lower trapezoidal, explicit ones and zeros), and goes round as v_{j-1}
+      if (warp == ow) {
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+          const int r = lane + 32 * q, grow = gr0 + r;
+          double xv = 0.0;
+#pragma unroll
+          for (int u = 0; u < 4; ++u) xv = (u == uj) ? x[q][u] : xv;
+          const double vv = grow > pr ? xv * rdenom : ((grow == pr && r < nloc) ? 1.0 : 0.0);
+#pragma unroll
+          for (int u = 0; u < 4; ++u) x[q][u] = (u == uj) ? vv : x[q][u];
+          vcol_s[r] = vv;
+        }
+      }
+      tau_prev = tau;
+      __syncthreads();
+      PCL_STAMP(7);
+    }
+    if (has) {
+#pragma unroll
+      for (int q = 0; q < 8; ++q)
+#pragma unroll
+        for (int u = 0; u < 4; ++u) S[(size_t)(c0 + u) * Rp + lane + 32 * q] = x[q][u];
+    }
+    __syncthreads();
+  } else
   for (int j = 0; j < b; ++j) {
     const int pr = row0 + j;                           // slab-numbering row of the pivot
     double* Sj = S + (size_t)j * Rp;
