@@ -52,8 +52,19 @@ __device__ unsigned long long g_pcl_trace[16];
 #define PCL_STAMP(k)
 #endif
 constexpr int kRegRows = 256;       // rows of a slab in the register-resident column loop
-__host__ __device__ constexpr int panel_cluster_doubles(int b) { return 2 * kClusterMax * b + 2 * b + 2 * kRegRows + b; }
+// px [2][kClusterMax][2b], prx [2][b], ycol/vcol [kRegRows] each, prow [b], send buffers [2][2b]
+__host__ __device__ constexpr int panel_cluster_doubles(int b) {
+  return 2 * kClusterMax * 2 * b + 2 * b + 2 * kRegRows + b + 4 * b;
+}
+// One bulk copy from this CTA's shared memory into a peer's, which also counts its bytes on the peer's mbarrier:
+// data and signal in one message.
+__device__ __forceinline__ void cl_bulk_send(uint32_t dst_cluster, uint32_t src_cta, uint32_t bytes, uint32_t bar_cluster) {
+  asm volatile("cp.async.bulk.shared::cluster.shared::cta.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+               ::"r"(dst_cluster), "r"(src_cta), "r"(bytes), "r"(bar_cluster)
+               : "memory");
+}
 
+__device__ __forceinline__ void proxy_fence_smem_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 __device__ __forceinline__ uint32_t cl_map(uint32_t addr, uint32_t rank) {   // the same address in CTA `rank` of the cluster
   uint32_t r;
   asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
@@ -294,6 +305,7 @@ __global__ void __launch_bounds__(kPanelThreads)
                  T* __restrict__ Tout, long long ldt,     // non-NULL: CTA 0 also builds the T factor at the end
                  double* __restrict__ csq) {              // non-NULL: [b][Gp] per-CTA sums of squares of the panel's columns
   __shared__ uint64_t cbar;      // cluster mode: this CTA's barrier, on which every CTA of the cluster arrives
+  __shared__ uint64_t xbar[2];   // ... and the two on which the per-column messages of the peers are counted
   __shared__ int go_s;
   unsigned nx = 0;               // cluster barriers passed
   if (CL) {
@@ -301,6 +313,8 @@ __global__ void __launch_bounds__(kPanelThreads)
     // its peers' barriers): rank 0 reads the flags and tells everyone, under the hardware barrier of the cluster.
     if (threadIdx.x == 0) {
       mbar_init(&cbar, gridDim.x);
+      mbar_init(&xbar[0], 1);
+      mbar_init(&xbar[1], 1);
       mbar_fence_init();
     }
     cl_hw_sync();                // every CTA of the cluster runs and has its barrier initialised
@@ -326,10 +340,11 @@ __global__ void __launch_bounds__(kPanelThreads)
   double* sc_s = pr_s + b;                // [4]: tau_j, 1/(alpha - beta)
   // cluster mode: partial sums [2][kClusterMax][b] and pivot rows [2][b] written by the peers, behind everything else
   double* px_s = sc_s + 4 + (fix.enabled ? panel_fix_doubles(b) : 0);
-  double* prx_s = px_s + 2 * kClusterMax * b;
+  double* prx_s = px_s + 2 * kClusterMax * 2 * b;
   double* ycol_s = prx_s + 2 * b;         // [kRegRows] column j below its pivot (register-resident loop)
   double* vcol_s = ycol_s + kRegRows;     // [kRegRows] v_{j-1}
   double* prow_s = vcol_s + kRegRows;     // [b] this CTA's entries of the pivot row
+  double* snd_s = prow_s + b;             // [2][2b] what this CTA sends per column: its partial sums, its pivot-row entries
 
   constexpr int NT = kPanelThreads, NW = NT / 32;
   constexpr int NWC = NW / RH;            // warps that share the columns within one row group
@@ -590,24 +605,48 @@ __global__ void __launch_bounds__(kPanelThreads)
       __syncthreads();
       PCL_STAMP(2);
       {
+        // One message per peer: this CTA's b partial sums and its entries of the pivot row (zeros unless it holds
+        // that row), 16 b bytes, copied into the peer's shared memory by cp.async.bulk, which also counts the bytes
+        // on the peer's barrier.  Two buffers and two barriers alternate: a peer is at most one column ahead.
         const int pb = j & 1;
-        for (int idx = tid; idx < G * b; idx += NT) {
-          const int q = idx >> lb, c = idx & (b - 1);
-          cl_st(cl_map(smem_u32(px_s + ((size_t)pb * kClusterMax + cta) * b + c), q), p_s[c]);
+        double* snd = snd_s + pb * 2 * b;
+        const bool mine = pr >= gr0 && pr < gr0 + nloc;
+        if (tid < b) {
+          snd[tid] = p_s[tid];
+          snd[b + tid] = mine ? prow_s[tid] : 0.0;
         }
-        if (pr >= gr0 && pr < gr0 + nloc)
-          for (int idx = tid; idx < G * b; idx += NT) {
-            const int q = idx >> lb, c = idx & (b - 1);
-            cl_st(cl_map(smem_u32(prx_s + pb * b + c), q), prow_s[c]);
-          }
+        proxy_fence_smem_async();
+        __syncthreads();
+        const uint32_t bytes = 2u * (uint32_t)b * 8u;
+        if (tid == 0) mbar_expect_tx(&xbar[pb], (uint32_t)G * bytes);
+        if (tid < G)
+          cl_bulk_send(cl_map(smem_u32(px_s + ((size_t)pb * kClusterMax + cta) * 2 * b), tid), smem_u32(snd), bytes,
+                       cl_map(smem_u32(&xbar[pb]), tid));
         PCL_STAMP(3);
-        if (!cluster_barrier(&cbar, nx, G, false, ctrl)) return;
+        if (tid == 0) {
+          int ok = 1;
+          const uint32_t par = (uint32_t)(j >> 1) & 1u;
+          if (!cl_try_wait(&xbar[pb], par)) {
+            const long long t0 = clock64();
+            while (!cl_try_wait(&xbar[pb], par)) {
+              if (clock64() - t0 > kWaitLimitClocks) {
+                atomicExch(&ctrl->status, (int)RRF_ERR_TIMEOUT);
+                atomicExch(&ctrl->done, 1);
+                ok = 0;
+                break;
+              }
+            }
+          }
+          go_s = ok;
+        }
+        __syncthreads();
+        if (!go_s) return;
         PCL_STAMP(4);
         if (tid < b) {
           double v = 0.0;
-          for (int q = 0; q < G; ++q) v += px_s[((size_t)pb * kClusterMax + q) * b + tid];     // CTA order: reproducible
+          for (int q = 0; q < G; ++q) v += px_s[((size_t)pb * kClusterMax + q) * 2 * b + tid];     // CTA order: reproducible
           p_s[tid] = v;
-          pr_s[tid] = prx_s[pb * b + tid];
+          pr_s[tid] = px_s[((size_t)pb * kClusterMax + pr / R) * 2 * b + b + tid];   // from the CTA that holds row pr
         }
         __syncthreads();
       }
@@ -733,7 +772,7 @@ __global__ void __launch_bounds__(kPanelThreads)
         double v = p_s[c];
 #pragma unroll
         for (int h = 1; h < RH; ++h) v += p_s[h * b + c];
-        cl_st(cl_map(smem_u32(px_s + ((size_t)pb * kClusterMax + cta) * b + c), q), v);
+        cl_st(cl_map(smem_u32(px_s + ((size_t)pb * kClusterMax + cta) * 2 * b + c), q), v);
       }
       if (pr >= gr0 && pr < gr0 + nloc)
         for (int idx = tid; idx < G * b; idx += NT) {
@@ -743,7 +782,7 @@ __global__ void __launch_bounds__(kPanelThreads)
       if (!cluster_barrier(&cbar, nx, G, false, ctrl)) return;
       if (tid < b) {
         double v = 0.0;
-        for (int q = 0; q < G; ++q) v += px_s[((size_t)pb * kClusterMax + q) * b + tid];     // CTA order: reproducible
+        for (int q = 0; q < G; ++q) v += px_s[((size_t)pb * kClusterMax + q) * 2 * b + tid];     // CTA order: reproducible
         p_s[tid] = v;
         pr_s[tid] = prx_s[pb * b + tid];
       }
