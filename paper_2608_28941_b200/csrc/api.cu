@@ -996,7 +996,12 @@ rrf_status_t rrf_create(rrf_handle_t* out, int device) {
   if (e == cudaSuccess) e = setup_all(h->smem_optin, &h->panel_smem_max, &h->cluster_ok);
   if (e == cudaSuccess) e = setup_tree_kernels(h->smem_optin, &h->tsqr_smem_max);
   if (e == cudaSuccess) e = setup_blk_kernels(h->smem_optin, &h->blk_smem_max);
-  if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&h->aux, cudaStreamNonBlocking);
+  // The side stream carries the panel chain of the look-ahead schedule, the critical path wherever that schedule is
+  // chosen: its kernels (a whole thread-block cluster where the panel is short) are placed ahead of GEMM CTAs that
+  // wait at the same moment.
+  int prio_lo = 0, prio_hi = 0;
+  if (e == cudaSuccess) e = cudaDeviceGetStreamPriorityRange(&prio_lo, &prio_hi);
+  if (e == cudaSuccess) e = cudaStreamCreateWithPriority(&h->aux, cudaStreamNonBlocking, prio_hi);
   if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&h->cap, cudaStreamNonBlocking);
   if (e == cudaSuccess) e = cudaMalloc(&h->d_ctrl, sizeof(Ctrl));
   if (e == cudaSuccess) e = cudaMemset(h->d_ctrl, 0, sizeof(Ctrl));
