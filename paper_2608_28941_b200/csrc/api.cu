@@ -2066,6 +2066,9 @@ extern "C" rrf_status_t rrf_panel_qr_static(int32_t dtype, int64_t rows, int32_t
 }
 
 #ifdef RRF_TSQR_TRACE
+extern "C" int rrf_debug_trace_vtw(unsigned long long* out) {
+  return (int)cudaMemcpyFromSymbol(out, rrf::g_vtc_trace, sizeof(unsigned long long) * 16);
+}
 extern "C" int rrf_debug_trace_panel(unsigned long long* out) {
   return (int)cudaMemcpyFromSymbol(out, rrf::g_pcl_trace, sizeof(unsigned long long) * 16);
 }

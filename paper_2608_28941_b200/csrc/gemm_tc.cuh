@@ -120,6 +120,17 @@ __device__ __forceinline__ void tmem_ld16x4(uint32_t t0, uint32_t t1, uint32_t t
 // signed zero; the kernels below use the planes only as tensor-core operands and keep x itself for everything else.
 __device__ __forceinline__ float tf32_rn(float x) { return __uint_as_float((__float_as_uint(x) + 0x1000u) & 0xFFFFE000u); }
 
+#ifdef RRF_TSQR_TRACE
+__device__ unsigned long long g_vtc_trace[16];
+#define VTC_DECL long long vtc_acc[8] = {0, 0, 0, 0, 0, 0, 0, 0}; const bool vtc_on = blockIdx.x == 5 && (threadIdx.x & 31) == 0
+#define VTC_T(slot, ...) { const long long vtc_t0 = clock64(); __VA_ARGS__; vtc_acc[slot] += clock64() - vtc_t0; }
+#define VTC_DUMP(base) if (vtc_on) { for (int q_ = 0; q_ < 8; ++q_) g_vtc_trace[(base) + q_] = (unsigned long long)vtc_acc[q_]; }
+#else
+#define VTC_DECL
+#define VTC_T(slot, ...) { __VA_ARGS__; }
+#define VTC_DUMP(base)
+#endif
+
 constexpr int kTcBN = 128;     // columns of W per accumulator = rows of D = tensor-memory lanes
 constexpr int kTcSub = 32;     // rows (contraction indices) per ring stage; a 64-row tile is two stages
 constexpr int kTcConv = 8;     // warps that split operands and drain the accumulator
@@ -224,10 +235,12 @@ __global__ void __launch_bounds__(kTcThreads, 1)
       constexpr uint32_t idesc2 = tc_idesc_tf32(kTcBN, 2 * B), idesc1 = tc_idesc_tf32(kTcBN, B);
       uint32_t fresh = 1;        // the next product overwrites the accumulator
       int ndrain = 0;
+      VTC_DECL;
+      const long long vtc_s = clock64();
       for (int q = 0; q < nsub; ++q) {
         const int o = q % OS;
-        if (!mbar_wait(&op_full[o], (q / OS) & 1, ctrl)) break;
-        if (fresh && ndrain > 0 && !mbar_wait(&acc_empty, (ndrain - 1) & 1, ctrl)) break;
+        VTC_T(1, if (!mbar_wait(&op_full[o], (q / OS) & 1, ctrl)) break;)
+        VTC_T(2, if (fresh && ndrain > 0 && !mbar_wait(&acc_empty, (ndrain - 1) & 1, ctrl)) break;)
         tc_fence_after();
         const uint32_t vH = smem_u32(ops + o * OPS), wH = vH + 2 * NBV * BOX, wL = wH + NBC * BOX;
 #pragma unroll
@@ -244,6 +257,11 @@ __global__ void __launch_bounds__(kTcThreads, 1)
           ++ndrain;
         }
       }
+#ifdef RRF_TSQR_TRACE
+      vtc_acc[0] = clock64() - vtc_s;
+      vtc_acc[7] = nsub;
+#endif
+      VTC_DUMP(8)
     }
   } else {
     // ---------------------------------------------------------------- operand split + accumulator drain
@@ -255,10 +273,15 @@ __global__ void __launch_bounds__(kTcThreads, 1)
     for (int j = 0; j < HB; ++j) acc[j] = 0.f;
     int ndrain = 0;
     const uint32_t raw0 = smem_u32(smem) + tid * 16, op0 = smem_u32(ops) + tid * 16;
+    VTC_DECL;
+    const long long vtc_s = clock64();
     for (int q = 0; q < nsub; ++q) {
       const int s = q % RS, o = q % OS;
-      if (!mbar_wait(&raw_full[s], (q / RS) & 1, ctrl)) break;
-      if (q >= OS && !mbar_wait(&op_empty[o], ((q / OS) - 1) & 1, ctrl)) break;
+      VTC_T(1, if (!mbar_wait(&raw_full[s], (q / RS) & 1, ctrl)) break;)
+      VTC_T(2, if (q >= OS && !mbar_wait(&op_empty[o], ((q / OS) - 1) & 1, ctrl)) break;)
+#ifdef RRF_TSQR_TRACE
+      const long long vtc_c0 = clock64();
+#endif
       const uint32_t src = raw0 + s * RAW, dst = op0 + o * OPS;
       float4 x[NBV + NBC];
 #pragma unroll
@@ -285,10 +308,16 @@ __global__ void __launch_bounds__(kTcThreads, 1)
         mbar_arrive(&op_full[o]);
         mbar_arrive(&raw_empty[s]);
       }
+#ifdef RRF_TSQR_TRACE
+      vtc_acc[4] += clock64() - vtc_c0;      // split of one stage
+#endif
       bool last;
       if ((q & 1) && drain_after(q >> 1, &last)) {
-        if (!mbar_wait(&acc_full, ndrain & 1, ctrl)) break;
+        VTC_T(3, if (!mbar_wait(&acc_full, ndrain & 1, ctrl)) break;)
         ++ndrain;
+#ifdef RRF_TSQR_TRACE
+        const long long vtc_d0 = clock64();
+#endif
         tc_fence_after();
         const uint32_t taddr = tmem + ((uint32_t)(quad * 32) << 16) + half * HB;
 #pragma unroll
@@ -311,8 +340,15 @@ __global__ void __launch_bounds__(kTcThreads, 1)
             acc[j] = 0.f;
           }
         }
+#ifdef RRF_TSQR_TRACE
+        vtc_acc[5] += clock64() - vtc_d0;    // drain
+#endif
       }
     }
+#ifdef RRF_TSQR_TRACE
+    vtc_acc[0] = clock64() - vtc_s;
+    if (warp == 0) { VTC_DUMP(0) }
+#endif
   }
   // common exit: nothing is in flight once the last accumulator has been drained (or a wait gave up)
   tc_fence_before();
