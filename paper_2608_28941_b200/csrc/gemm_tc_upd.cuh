@@ -4,7 +4,8 @@
 // Same tiles (row slab of 128, column tile of 64), same stream-K ranges, same output slots and the
 // same norm partials as upd_sk_kernel.  Per tile:
 //   P     = V[slab, :] Zt[tile, :]^T                  K = B      (GEMM 1)
-//   Wnew  = W[slab, tile] - P  -> global memory, sums of squares for the norms
+//   Wnew  = W[slab, tile] - P  -> back into the W tile's place in shared memory and from there to global memory
+//                                 by a TMA store (whole 128-byte lines); sums of squares for the norms
 //   Y    += Wnew OmegaT[j0 .. j0+B, tile]^T           K = 64     (GEMM 2, only if j0 >= 0)
 // The left operand of both products sits in TENSOR MEMORY (lane = row of the slab, one column per
 // contraction index): V is written there once per slab, Wnew once per tile by the very threads that
