@@ -207,6 +207,59 @@ __device__ __forceinline__ double panel_entry(const T* __restrict__ Y, const Pan
   return s;
 }
 
+// The same sums for a whole slab, S[c][r] (pitch Rp) = entry (gr0 + r - row0, c), with the loads of eight entries
+// in flight per thread: the terms of one entry are a dependent chain of global loads (up to a dozen partial
+// panels), and a CTA that holds a tall slab has dozens of entries per thread.  Same order of additions as
+// panel_entry, so the same bits.
+template <typename T>
+__device__ __forceinline__ void panel_load_slab(const T* __restrict__ Y, const PanelSource& src, double* __restrict__ S, int Rp,
+                                                int nloc, int b, int lb, int gr0, int row0, int tid, int nthr) {
+  constexpr int E = 8;
+  const int total = nloc * b;
+  const size_t tstride = src.slots ? (size_t)src.bm * b : (size_t)src.seg_stride;
+  for (int base = tid; base < total; base += E * nthr) {
+    const T* ptr[E];
+    int cnt[E];
+    double v[E];
+    int maxcnt = 0;
+#pragma unroll
+    for (int e = 0; e < E; ++e) {
+      const int idx = base + e * nthr;
+      const int r = idx >> lb, c = idx & (b - 1);
+      cnt[e] = 0;
+      ptr[e] = Y;
+      if (idx < total) {
+        const int lr = gr0 + r - row0 + src.row_off;
+        if (src.slots) {
+          const int sl = lr / src.bm, rl = lr - sl * src.bm;
+          const int p_lo = (sl * src.nc) / src.tpc, p_hi = ((sl + 1) * src.nc - 1) / src.tpc;
+          cnt[e] = (p_hi - p_lo + 1) * src.wn;
+          ptr[e] = Y + (size_t)(p_lo + sl) * src.wn * tstride + (size_t)rl * b + c;
+        } else {
+          cnt[e] = src.nseg;
+          ptr[e] = Y + (size_t)lr * src.ldy + c;
+        }
+      }
+      maxcnt = max(maxcnt, cnt[e]);
+    }
+#pragma unroll
+    for (int e = 0; e < E; ++e) {
+      const double first = cnt[e] > 0 ? (double)ptr[e][0] : 0.0;
+      v[e] = src.slots ? 0.0 + first : first;      // as panel_entry: a lone -0.0 of a stacked panel keeps its sign
+    }
+    for (int t = 1; t < maxcnt; ++t) {
+#pragma unroll
+      for (int e = 0; e < E; ++e)
+        if (t < cnt[e]) v[e] += (double)ptr[e][(size_t)t * tstride];
+    }
+#pragma unroll
+    for (int e = 0; e < E; ++e) {
+      const int idx = base + e * nthr;
+      if (idx < total) S[(size_t)(idx & (b - 1)) * Rp + (idx >> lb)] = v[e];
+    }
+  }
+}
+
 // Compact-WY factor T from the Gram rows and tau, by recursive doubling (see tfactor_kernel below).
 // The block-level body: every thread of one CTA calls it; `tsm` holds b*(b+1) + (b/2)*(b/2+1) doubles.
 template <typename T>
@@ -364,10 +417,7 @@ __global__ void __launch_bounds__(kPanelThreads)
   unsigned nbar = 0;                      // grid barriers passed so far
 
   // load the slab: sum the partial panels in their fixed order
-  for (int idx = tid; idx < nloc * b; idx += NT) {
-    const int r = idx >> lb, c = idx & (b - 1);
-    S[(size_t)c * Rp + r] = panel_entry(Y, src, gr0 + r - row0, c, b);
-  }
+  panel_load_slab<T>(Y, src, S, Rp, nloc, b, lb, gr0, row0, tid, NT);
   if (PAD) {
     const int npad = RS - nloc;
     for (int idx = tid; idx < npad * b; idx += NT) {
