@@ -201,8 +201,8 @@ static bool plan_panel_cl(const rrf_ctx* h, long long rows, int b, PanelPlan* p,
   // (measured: 4096 x 64 takes 279 us as one cluster of 16 against 260 us on 148 CTAs; 1024 x 16 falls from 64 to 54)
   // With the register-resident column loop (b <= 64) a 4096 x 64 panel takes 232 us on its own, but inside a run, where
   // 16 CTAs also sum the partial panels and store V, the 4096-row passes of config 4 take 284 us against 261 us.
-  if (R > kClusterMaxRows) return false;
-  const bool reg = b <= 64;
+  const bool reg = b <= 64 && R <= kRegRows;
+  if (!reg && R > kClusterMaxRows) return false;
   int G = 1;
   while (G < ceil_div(ext, R)) G *= 2;
   if (G > kClusterMax) return false;
@@ -402,12 +402,15 @@ struct PassModel {
   int b;
   bool f64;
   bool tc;      // single precision on tcgen05
+  bool cl;      // the confined panel runs as one thread-block cluster with its slab in registers
   // flop per microsecond the two GEMM kernels sustain on the whole device
-  double vtw() const { return 2.0 * rows * n * b / (f64 ? 33e6 : (tc ? 85e6 : 45e6)) + 10.0; }
-  double upd() const { return 4.0 * rows * n * b / (f64 ? 27e6 : (tc ? 72e6 : 32e6)) + 15.0; }
+  double vtw() const { return 2.0 * rows * n * b / (f64 ? 33e6 : (tc ? 75e6 : 45e6)) + 10.0; }
+  double upd() const { return 4.0 * rows * n * b / (f64 ? 27e6 : (tc ? 100e6 : 32e6)) + 15.0; }
   // fix-up + panel + T factor on `ctas` SMs, with the launch and event hand-overs of the side stream
   double panel_chain(int ctas) const {
     const double R = std::max(64.0, (rows + b) / ctas);
+    if (cl)     // one cluster, slab in registers: 4096 x 64 takes 232 us, 4096 x 32 107 us, 1024 x 16 55 us on their own
+      return (b * (3700.0 + 42.0 * b) + 40000.0 + 0.07 * R * b * b) / 1965.0 + 20.0;
     const double cycles = b * (7000.0 + 0.14 * R * b) + 20000.0 + 0.07 * R * b * b;
     return cycles / 1965.0 + 0.3 * b + (f64 ? 45.0 : 85.0);
   }
@@ -1426,6 +1429,8 @@ rrf_status_t rrf_run(rrf_handle_t h, const rrf_params_t* p, void* dA, int64_t ld
   const bool tree = (p->flags & RRF_FLAG_PANEL_TREE) != 0 && b <= kTsqrMaxB;
   const bool blocked = (p->flags & RRF_FLAG_PANEL_BLOCKED) != 0;
   int look_ctas = 0;
+  bool look_cl = false;
+  PanelPlan pcl_probe, pcl_probe0;
   if (blocked && !tree) {
     // opt-in blocked panel kernel: under look-ahead (only if asked for) the panel is confined to a few SMs, its
     // slabs in global memory when shared memory does not hold them
@@ -1437,11 +1442,29 @@ rrf_status_t rrf_run(rrf_handle_t h, const rrf_params_t* p, void* dA, int64_t ld
     const int lim = p->tune_panel_ctas > 0 ? std::min(cap, (int)p->tune_panel_ctas) : cap;
     if ((p->flags & RRF_FLAG_TWO_QUEUES) && steps_total >= 2 && plan_tree(h, m, b, lim, true, &tl)) look_ctas = tl.ctas;
     if (look_ctas == 0 && !plan_tree(h, m, b, 0, false, &tl)) return fail(RRF_ERR_WORKSPACE);
+  } else if (!(p->flags & RRF_FLAG_ONE_QUEUE) && !unchanged && steps_total >= 2 && plan_panel_cl(h, m - b, b, &pcl_probe, true) &&
+             plan_panel_cl(h, m, b, &pcl_probe0, false)) {
+    // every panel of the chain fits one thread-block cluster (the first as it is, the later ones with the b rows
+    // of the fix-up): the chain takes only that many SMs
+    const PassModel pm{h->sms, (double)m, (double)n, b, p->dtype == RRF_F64, p->dtype == RRF_F32 && h->f32_engine == 1, true};
+    const double t = std::min(pm.step_ungated(kClusterMax), pm.step_gated(kClusterMax));
+    if ((p->flags & RRF_FLAG_TWO_QUEUES) || t < pm.step_serial()) {
+      // A cluster needs its SMs inside one GPC, and where the GEMM kernels' CTAs land cannot be chosen: with exactly
+      // the cluster's SMs kept free the panel often waits for a GEMM kernel to drain.  Where the panel chain is the
+      // critical path the GEMM kernels therefore leave 44 SMs free (measured on 4096 x 11008 fp32: 2.61 ms against
+      // 2.69 with 16, 2.67 with 20, 2.72 with 32); where the GEMMs are, they get every SM the cluster does not
+      // take (4096 x 4096 fp64, b = 32: 2.51 ms with 16 against 2.88 with 44).
+      const int gcl = std::max(pcl_probe.G, pcl_probe0.G);
+      const bool chain_critical = pm.panel_chain(gcl) > (pm.vtw() + pm.upd()) * pm.scale(gcl);
+      const int keep = chain_critical ? std::max(gcl, std::min(44, h->sms / 3)) : gcl;
+      look_ctas = p->tune_panel_ctas > 0 ? std::max(gcl, std::min((int)p->tune_panel_ctas, h->sms / 3)) : keep;
+      look_cl = true;
+    }
   } else if (!(p->flags & RRF_FLAG_ONE_QUEUE) && !unchanged && steps_total >= 2) {
     const int fewest = panel_min_ctas(h, m, b);
     const int cap = std::min(kLookMaxCtas, h->sms / 3);
     if (fewest > 0 && fewest <= cap) {
-      const PassModel pm{h->sms, (double)m, (double)n, b, p->dtype == RRF_F64, p->dtype == RRF_F32 && h->f32_engine == 1};
+      const PassModel pm{h->sms, (double)m, (double)n, b, p->dtype == RRF_F64, p->dtype == RRF_F32 && h->f32_engine == 1, false};
       int best = fewest;
       double best_t = std::min(pm.step_ungated(fewest), pm.step_gated(fewest));
       for (int c = fewest + 1; c <= cap; ++c) {
@@ -1484,7 +1507,7 @@ rrf_status_t rrf_run(rrf_handle_t h, const rrf_params_t* p, void* dA, int64_t ld
   } else if (p->flags & RRF_FLAG_SAMPLE_NEVER) {
     predict = 2;
   } else if (!(p->flags & RRF_FLAG_SAMPLE_ALWAYS) && !(p->flags & RRF_FLAG_FIXED_RANK)) {
-    const PassModel pm{h->sms, (double)m, (double)n, b, p->dtype == RRF_F64, false};
+    const PassModel pm{h->sms, (double)m, (double)n, b, p->dtype == RRF_F64, false, false};
     if (pm.vtw() + pm.upd() > 600.0) predict = 0;
   }
   const bool predicting = predict != 1;
@@ -1737,7 +1760,7 @@ rrf_status_t rrf_run(rrf_handle_t h, const rrf_params_t* p, void* dA, int64_t ld
     // starts as early as its inputs allow.
     auto gated = [&](int rows_i) {
       if (p->tune_gate != 0) return p->tune_gate == 2;
-      const PassModel pm{h->sms, (double)rows_i, (double)n, b, p->dtype == RRF_F64, tc};
+      const PassModel pm{h->sms, (double)rows_i, (double)n, b, p->dtype == RRF_F64, tc, look_cl};
       return pm.step_gated(look_ctas) < pm.step_ungated(look_ctas);
     };
     PanelSource src1 = src;           // panel 1: sampled from A by the sample kernel
