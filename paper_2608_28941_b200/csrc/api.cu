@@ -1760,6 +1760,7 @@ rrf_status_t rrf_run(rrf_handle_t h, const rrf_params_t* p, void* dA, int64_t ld
     // starts as early as its inputs allow.
     auto gated = [&](int rows_i) {
       if (p->tune_gate != 0) return p->tune_gate == 2;
+      if (look_cl) return false;       // a cluster takes so few SMs that holding it back never pays (measured)
       const PassModel pm{h->sms, (double)rows_i, (double)n, b, p->dtype == RRF_F64, tc, look_cl};
       return pm.step_gated(look_ctas) < pm.step_ungated(look_ctas);
     };
