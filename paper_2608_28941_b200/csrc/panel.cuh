@@ -693,9 +693,14 @@ __global__ void __launch_bounds__(kPanelThreads)
         if (!go_s) return;
         PCL_STAMP(4);
         if (tid < b) {
-          double v = 0.0;
-          for (int q = 0; q < G; ++q) v += px_s[((size_t)pb * kClusterMax + q) * 2 * b + tid];     // CTA order: reproducible
-          p_s[tid] = v;
+          // four interleaved partial sums (CTAs q = 0, 4, 8, 12; 1, 5, ...; ...), then their sum: a fixed order
+          double v4[4] = {0.0, 0.0, 0.0, 0.0};
+          for (int q = 0; q < G; q += 4) {
+#pragma unroll
+            for (int e = 0; e < 4; ++e)
+              if (q + e < G) v4[e] += px_s[((size_t)pb * kClusterMax + q + e) * 2 * b + tid];
+          }
+          p_s[tid] = (v4[0] + v4[1]) + (v4[2] + v4[3]);
           pr_s[tid] = px_s[((size_t)pb * kClusterMax + pr / R) * 2 * b + b + tid];   // from the CTA that holds row pr
         }
         __syncthreads();
