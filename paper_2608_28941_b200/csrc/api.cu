@@ -662,7 +662,9 @@ static rrf_status_t launch_panel(rrf_ctx* h, int dtype, const void* Y, PanelSour
                                  long long rows, int b, void* V, long long ldv, void* Tout, long long ldt,
                                  const PanelScratch& ps, Ctrl* ctrl, const int* done_flag, cudaStream_t st,
                                  Mark mark = Mark(), int step = 0, const PanelOpts& o = PanelOpts()) {
-  if (b <= kTsqrMaxB && o.tree && ps.ts.Rbuf != nullptr) {
+  // (a square panel goes to the per-column kernel: its last column has nothing below the pivot, for which the
+  // Householder convention is H = I, tau = 0, while the reconstruction from a tree always reflects, tau = 2)
+  if (b <= kTsqrMaxB && o.tree && ps.ts.Rbuf != nullptr && rows > b) {
     // tree kernel: factorisation, T factor and all, in one cooperative launch
     TreePlan tp;
     if (!plan_tree(h, rows, b, o.ctas, o.fix.enabled != 0, &tp)) return RRF_ERR_WORKSPACE;

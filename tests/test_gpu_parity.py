@@ -135,7 +135,11 @@ def check_run(h, w, g, o, A, Om, q_envelope=True, estimator="direct"):
 @pytest.mark.parametrize("rows,b,dtype", [(200, 16, "f64"), (1024, 16, "f64"), (4096, 32, "f64"),
                                           (8192, 64, "f64"), (5001, 64, "f64"), (300, 128, "f64"),
                                           (20000, 128, "f64"), (4096, 64, "f32"), (777, 32, "f32"),
-                                          (60000, 32, "f64"), (45000, 64, "f64")])      # slabs of 512 / 320 rows
+                                          (60000, 32, "f64"), (45000, 64, "f64"),       # slabs of 512 / 320 rows
+                                          # one thread-block cluster: 1, 2, 16 CTAs; its largest panel, one row more
+                                          # (cooperative grid again); b = 128 keeps the shared-memory loop
+                                          (64, 64, "f64"), (100, 32, "f64"), (4096, 64, "f64"), (4097, 64, "f64"),
+                                          (4095, 16, "f64"), (2048, 128, "f64"), (2049, 128, "f64"), (3000, 64, "f32")])
 @pytest.mark.parametrize("algo", ALGOS)
 def test_panel_qr_matches_oracle(h, rows, b, dtype, algo):
     tree, blocked = algo == "tree", algo == "blocked"
