@@ -72,6 +72,8 @@ struct rrf_ctx {
   std::vector<unsigned char> gcand;      // arguments of the last directly enqueued call
   std::vector<std::pair<int, int>> gmarks;
   int graph_off;                         // set when a capture failed: enqueue directly from then on
+  int cand_steps;                        // block steps the last directly enqueued call ran, -1 if it did not end by its own rule
+  int gsteps;                            // block steps the instantiated graph holds (it may hold fewer than max_rank / b)
   int cluster_ok;                        // a 16-CTA cluster of the panel kernel can be resident on this device
   int f32_engine;                        // single-precision V^T W: 0 = mma.sync 3xTF32, 1 = tcgen05 3xTF32
   int tc_chunk;                          // tcgen05: 64-row tiles summed in tensor memory between round-to-nearest adds
@@ -987,6 +989,8 @@ rrf_status_t rrf_create(rrf_handle_t* out, int device) {
   h->graph = nullptr;
   h->gexec = nullptr;
   h->graph_off = 0;
+  h->cand_steps = -1;
+  h->gsteps = 0;
   h->f32_engine = 1;      // single precision runs on tcgen05 unless rrf_set_single_engine says otherwise
   h->tc_chunk = 2;
   std::memset(&h->profile, 0, sizeof(h->profile));
@@ -1490,6 +1494,11 @@ rrf_status_t rrf_run(rrf_handle_t h, const rrf_params_t* p, void* dA, int64_t ld
   unsigned char* ws = (unsigned char*)d_workspace;
   Ctrl* ctrl = reinterpret_cast<Ctrl*>(ws + L.ctrl);
   const int steps = p->max_rank / b;
+  // Block steps the launch sequence holds.  A graph captured for a call that repeats the previous one holds only as
+  // many as that one needed (plus one): the passes after the stop, whose kernels start and return, are then not
+  // launched at all.  Should the data have changed so that the loop is still open at the end, the call is run again
+  // in full (which is why an in-place run, whose input is gone by then, always holds every pass).
+  int steps_run = steps;
   double* tr_sub = reinterpret_cast<double*>(ws + L.traces);
   double* tr_dir = tr_sub + steps;
   double* tr_est = tr_dir + steps;                   // [steps + 1]
@@ -1641,7 +1650,7 @@ rrf_status_t rrf_run(rrf_handle_t h, const rrf_params_t* p, void* dA, int64_t ld
       return RRF_ERR_INVALID_ARG;
     unsigned bar_next = 0, bar_used = 0;
     const int sum_grid = (int)std::min<long long>((m * b + 255) / 256, (long long)h->sms * 8);
-    for (int i = 0; i < steps; ++i) {
+    for (int i = 0; i < steps_run; ++i) {
       const int r0 = i * b, rows = (int)(m - r0);
       if (i > 0) {
         mark(RRF_PHASE_SAMPLE, i);
@@ -1690,7 +1699,7 @@ rrf_status_t rrf_run(rrf_handle_t h, const rrf_params_t* p, void* dA, int64_t ld
     // of the fused update of pass i.
     PanelSource alt{};             // the upcoming panel as the separate sample kernel would leave it
     const int* fused_flag = nullptr;
-    for (int i = 0; i < steps; ++i) {
+    for (int i = 0; i < steps_run; ++i) {
       const int r0 = i * b, rows = (int)(m - r0);
       PanelOpts po;
       po.st_t = h->aux;
@@ -1797,7 +1806,7 @@ rrf_status_t rrf_run(rrf_handle_t h, const rrf_params_t* p, void* dA, int64_t ld
     }
     UpdPlan up_prev{};
     PanelSource alt_prev{};        // the panel of pass i+1 as the separate sample kernel would leave it
-    for (int i = 0; i < steps; ++i) {
+    for (int i = 0; i < steps_run; ++i) {
       const int r0 = i * b, rows = (int)(m - r0);
       const bool gate = gated(rows);
       auto next_panel = [&]() -> rrf_status_t {
@@ -1838,7 +1847,7 @@ rrf_status_t rrf_run(rrf_handle_t h, const rrf_params_t* p, void* dA, int64_t ld
         }
         return ls;
       };
-      if (i + 1 < steps && !gate) {
+      if (i + 1 < steps_run && !gate) {
         s = next_panel();
         if (s != RRF_OK) return panel_failed(s);
       }
@@ -1854,7 +1863,7 @@ rrf_status_t rrf_run(rrf_handle_t h, const rrf_params_t* p, void* dA, int64_t ld
       ops->vtw(tmV_k, i == 0 ? tmA_k : tmW_k, Zpart, r0, r0, vp, ctrl, st);
       mark(RRF_PHASE_TZ, i);
       ops->tz(Zpart, vp, Tblk(r0), p->max_rank, 1, Zt, &ctrl->done, st);
-      if (i + 1 < steps && gate) {
+      if (i + 1 < steps_run && gate) {
         cudaEventRecord(evZ(i), st);
         s = next_panel();
         if (s != RRF_OK) return panel_failed(s);
@@ -1911,6 +1920,7 @@ rrf_status_t rrf_run(rrf_handle_t h, const rrf_params_t* p, void* dA, int64_t ld
   if (graphs_ok && h->gexec != nullptr && key == h->gkey) {
     marks = h->gmarks;
     nev = marks.size();
+    steps_run = h->gsteps;
     launched = cudaGraphLaunch(h->gexec, user_st) == cudaSuccess;
     if (!launched) h->graph_off = 1;
   } else if (graphs_ok && key == h->gcand) {
@@ -1921,6 +1931,7 @@ rrf_status_t rrf_run(rrf_handle_t h, const rrf_params_t* p, void* dA, int64_t ld
     h->gkey.clear();
     st = h->cap;
     capturing = true;
+    if (!inplace && h->cand_steps > 0) steps_run = std::min(steps, h->cand_steps + 1);
     rrf_status_t cs = RRF_ERR_CUDA;
     if (cudaStreamBeginCapture(st, cudaStreamCaptureModeRelaxed) == cudaSuccess) {
       cs = enqueue();
@@ -1931,12 +1942,14 @@ rrf_status_t rrf_run(rrf_handle_t h, const rrf_params_t* p, void* dA, int64_t ld
         h->graph = g;
         h->gkey = key;
         h->gmarks = marks;
+        h->gsteps = steps_run;
         launched = cudaGraphLaunch(h->gexec, user_st) == cudaSuccess;
       } else if (g != nullptr) {
         cudaGraphDestroy(g);
       }
     }
     if (!launched) {               // capture is not available here: enqueue directly from now on
+      steps_run = steps;
       cudaGetLastError();
       if (h->gexec != nullptr) cudaGraphExecDestroy(h->gexec);
       if (h->graph != nullptr) cudaGraphDestroy(h->graph);
@@ -1949,9 +1962,11 @@ rrf_status_t rrf_run(rrf_handle_t h, const rrf_params_t* p, void* dA, int64_t ld
     capturing = false;
     st = user_st;
   }
+  const bool direct = !launched;
   if (!launched) {
     marks.clear();
     nev = 0;
+    steps_run = steps;
     s = enqueue();
     if (s != RRF_OK) return fail(s);
     h->gcand = key;
@@ -1961,11 +1976,29 @@ rrf_status_t rrf_run(rrf_handle_t h, const rrf_params_t* p, void* dA, int64_t ld
   Ctrl hc;
   if (e == cudaSuccess) e = cudaMemcpyAsync(&hc, ctrl, sizeof(Ctrl), cudaMemcpyDeviceToHost, st);
   if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+  if (e == cudaSuccess && !direct && steps_run < steps && !hc.done && hc.status >= 0) {
+    // the graph held fewer passes than this input needs: drop it and run the call in full
+    if (h->gexec != nullptr) cudaGraphExecDestroy(h->gexec);
+    if (h->graph != nullptr) cudaGraphDestroy(h->graph);
+    h->gexec = nullptr;
+    h->graph = nullptr;
+    h->gkey.clear();
+    h->gcand.clear();
+    marks.clear();
+    nev = 0;
+    steps_run = steps;
+    s = enqueue();
+    if (s != RRF_OK) return fail(s);
+    e = cudaGetLastError();
+    if (e == cudaSuccess) e = cudaMemcpyAsync(&hc, ctrl, sizeof(Ctrl), cudaMemcpyDeviceToHost, st);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+  }
   if (e != cudaSuccess) {
     h->last_cuda = (int)e;
     out->cuda_error = (int)e;
     return fail(RRF_ERR_CUDA);
   }
+  if (direct) h->cand_steps = (hc.done && hc.status >= 0) ? hc.steps : -1;
   if (h->profiling && nev > 1) {
     std::memset(&h->profile, 0, sizeof(h->profile));
     for (size_t q = 0; q + 1 < nev; ++q) {
@@ -1989,12 +2022,15 @@ rrf_status_t rrf_run(rrf_handle_t h, const rrf_params_t* p, void* dA, int64_t ld
     const int lag = look_ctas > 0 ? 2 : 1;
     // without the predictor every executed pass that has a later panel to sample samples it
     out->fused_samples = predicting ? hc.fused_samples : std::min(hc.steps, std::max(0, steps - lag));
+    const int sl = steps_run;      // passes whose kernels were launched
     if (unchanged)
-      out->kernel_launches = (dOmegaT == nullptr ? 1 : 0) + 1 + 4 * steps + 3 * steps * (steps - 1) / 2;
+      out->kernel_launches = (dOmegaT == nullptr ? 1 : 0) + 1 + 4 * sl + 3 * sl * (sl - 1) / 2;
     else
-    out->kernel_launches = (sampled ? steps : 0) + 1 + (dOmegaT == nullptr ? 1 : 0) + 1 + ((look_ctas > 0 && steps > 1) ? 1 : 0) +
-                           ((look_ctas > 0 || tree) ? 5 : 6) * steps +   // look-ahead, tree kernel: the panel kernel builds T itself
-                           (predicting ? std::max(0, steps - lag) : 0);
+    out->kernel_launches = (sampled ? sl : 0) + 1 + (dOmegaT == nullptr ? 1 : 0) + 1 + ((look_ctas > 0 && steps > 1) ? 1 : 0) +
+                           ((look_ctas > 0 || tree) ? 5 : 6) * sl +   // look-ahead, tree kernel: the panel kernel builds T itself
+                           (predicting ? std::max(0, std::min(sl, steps - lag)) : 0) +
+                           ((p->dtype == RRF_F32 && h->f32_engine == 1 && get_ops(p->dtype, b)->has_upd_tc)   // TF32 planes of Zt, OmegaT's rows
+                                ? sl + std::max(0, std::min(sl, steps - lag)) : 0);
   }
   out->extra_samples = hc.extra_samples;
   out->panel_ctas = look_ctas;

@@ -679,3 +679,50 @@ def test_column_sharded_driver_as_a_single_rank(h, name, kw):
     Q = Q.cpu().numpy().astype(np.float64)
     assert np.linalg.norm(Q.T @ Q - np.eye(g.k)) <= tl["orth"]
     assert relmax(Q @ g.B[:g.k].cpu().numpy().astype(np.float64), orc.form_q(o.V, o.T, w.b) @ o.B) <= 10 * tl["rel"]
+
+
+@pytest.mark.parametrize("sched", [rrf.RRF_FLAG_ONE_QUEUE, rrf.RRF_FLAG_TWO_QUEUES], ids=["one-queue", "two-queues"])
+@pytest.mark.parametrize("dtype", ["f64", "f32"])
+def test_replayed_graph_that_holds_fewer_passes_than_the_new_input_needs(h, sched, dtype):
+    """A graph captured for a repeated call holds only the passes that call needed.  The same buffers then get an
+    input of higher rank: the replay ends with the loop still open, and the call must be run again in full and give
+    the oracle's answer for the NEW input (and the old answer again when the old input comes back)."""
+    m, n, b, max_rank = 900, 700, 32, 256
+    tol = 1e-6 if dtype == "f64" else 1e-3
+    npdt = np.float64 if dtype == "f64" else np.float32
+    rng = np.random.default_rng(5)
+
+    def lowrank(r):
+        return (rng.standard_normal((m, r)) @ rng.standard_normal((r, n)) / np.sqrt(r)).astype(npdt)
+
+    A_small, A_big = lowrank(40), lowrank(150)
+    Om = rng.standard_normal((n, max_rank)).astype(npdt)
+    dA = torch.empty((m, n), dtype=torch.float64 if dtype == "f64" else torch.float32, device="cuda")
+    dOmT = torch.from_numpy(np.ascontiguousarray(Om.T)).cuda()
+    V = torch.empty((m, max_rank), dtype=dA.dtype, device="cuda")
+    T = torch.empty((b, max_rank), dtype=dA.dtype, device="cuda")
+    B = torch.empty((max_rank, n), dtype=dA.dtype, device="cuda")
+    need = rrf.rrf_workspace_bytes(rrf.make_params(rrf.RRF_F64 if dtype == "f64" else rrf.RRF_F32, m, n, b, tol, max_rank))
+    ws = torch.empty(need, dtype=torch.uint8, device="cuda")
+
+    def run():
+        return rrf.rrf_run(h, dA, b, tol, max_rank, omegaT=dOmT, flags=sched, V=V, T=T, B=B, workspace=ws)
+
+    def check(A):
+        o = orc.rrf(A.astype(np.float64), Om.astype(np.float64), b, tol, max_rank)
+        g = run()
+        assert (g.k, g.steps, g.status) == (o.k, o.steps, o.status), (g.k, o.k)
+        Bg = g.B[:g.k].cpu().numpy().astype(np.float64)
+        assert relmax(Bg, o.B) <= TOL[dtype]["rel"]
+        return g.k
+
+    dA.copy_(torch.from_numpy(A_small))
+    k_small = check(A_small)           # enqueued directly
+    assert check(A_small) == k_small   # captured, holding k_small / b + 1 passes
+    assert check(A_small) == k_small   # replayed
+    dA.copy_(torch.from_numpy(A_big))
+    k_big = check(A_big)               # replayed, found too short, run in full
+    assert k_big > k_small + b
+    assert check(A_big) == k_big       # captured anew
+    dA.copy_(torch.from_numpy(A_small))
+    assert check(A_small) == k_small   # the longer graph serves the shorter input
