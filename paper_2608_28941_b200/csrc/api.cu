@@ -502,7 +502,7 @@ struct Ops {
   static_assert(TcCfg<TC_B, TC_RS, TC_OS>::SMEM + 1024 <= kMaxSmem, "shared memory");
   // fused update: slab height 128 (64 for the widest block), two 128-byte column groups per tile
   static constexpr int U_BM = (B >= 128) ? 64 : 128;
-  static constexpr int U_BNB = 2;
+  static constexpr int U_BNB = (sizeof(T) == 8 && B == 32) ? 4 : 2;
   static constexpr int U_WM = U_BM / 16, U_WN = 8 / U_WM;
   static constexpr int U_BN = U_BNB * KE;
   static constexpr int U_KB = B / KE;
