@@ -144,7 +144,8 @@ struct UpdTc {
   int chunk;
   CUtensorMap tmZs, tmOs;
 };
-struct UpdPlan { int NS, NC, total, tpc, P, slots; const UpdTc* tc; };
+// p0, Lb: this launch's CTAs are numbers p0 ... of the pass and start at tile Lb (a pass split over two launches)
+struct UpdPlan { int NS, NC, total, tpc, P, slots; const UpdTc* tc; int p0, Lb; };
 static UpdPlan plan_upd(int sms, long long rows, long long ncols, int bm, int bn, int wn) {
   UpdPlan p;
   p.NS = ceil_div(rows, bm);
@@ -154,6 +155,8 @@ static UpdPlan plan_upd(int sms, long long rows, long long ncols, int bm, int bn
   p.P = ceil_div(p.total, p.tpc);
   p.slots = (p.P + p.NS) * wn;
   p.tc = nullptr;
+  p.p0 = 0;
+  p.Lb = 0;
   return p;
 }
 // The panel kernel's variants: rows a lane keeps in registers, row groups, and whether the slab is
@@ -594,7 +597,7 @@ struct Ops {
     }
     upd_sk_kernel<T, B, U_BM, U_BNB, U_WM, U_WN, U_STAGES, U_PW><<<p.P, (U_PW ? 9 : 8) * 32, U_SMEM, st>>>(
         tmV, tmZ, tmC, tmO, (T*)C, ldc, (T*)top, ldtop, r0, rows, ncols, cv0, top_rows, j0, (T*)Ypart, norm_part, p.NC,
-        p.total, p.tpc, ctrl, samp_flag);
+        p.total, p.tpc, ctrl, samp_flag, p.p0, p.Lb);
   }
 };
 
@@ -1608,7 +1611,7 @@ rrf_status_t rrf_run(rrf_handle_t h, const rrf_params_t* p, void* dA, int64_t ld
     return RRF_ERR_CUDA;
 
   // fork/join events for the side stream, created once and kept in the handle
-  while (h->sync_events.size() < (size_t)3 * steps + 2) {
+  while (h->sync_events.size() < (size_t)4 * steps + 2) {
     cudaEvent_t ev;
     if (cudaEventCreateWithFlags(&ev, cudaEventDisableTiming) != cudaSuccess) return RRF_ERR_CUDA;
     h->sync_events.push_back(ev);
@@ -1766,6 +1769,7 @@ rrf_status_t rrf_run(rrf_handle_t h, const rrf_params_t* p, void* dA, int64_t ld
     auto evP = [&](int i) { return h->sync_events[3 * i]; };
     auto evU = [&](int i) { return h->sync_events[3 * i + 1]; };
     auto evZ = [&](int i) { return h->sync_events[3 * i + 2]; };
+    auto evH = [&](int i) { return h->sync_events[3 * steps + 2 + i]; };
     // Where the update alone outlasts the next panel, the panel is held back until V^T W and T Z of
     // the pass are done, and V^T W gets every SM; otherwise the panel chain is the critical path and
     // starts as early as its inputs allow.
@@ -1805,6 +1809,7 @@ rrf_status_t rrf_run(rrf_handle_t h, const rrf_params_t* p, void* dA, int64_t ld
       cudaEventRecord(evS2, st);
     }
     UpdPlan up_prev{};
+    int pv_t1 = 0, pv_p1 = 0, pv_tpc2 = 0;   // how the update of the previous pass was split over two launches
     PanelSource alt_prev{};        // the panel of pass i+1 as the separate sample kernel would leave it
     for (int i = 0; i < steps_run; ++i) {
       const int r0 = i * b, rows = (int)(m - r0);
@@ -1820,6 +1825,9 @@ rrf_status_t rrf_run(rrf_handle_t h, const rrf_params_t* p, void* dA, int64_t ld
           sn.nc = up_prev.NC;
           sn.tpc = up_prev.tpc;
           sn.wn = ops->u_wn;
+          sn.t1 = pv_t1;
+          sn.p1 = pv_p1;
+          sn.tpc2 = pv_tpc2;
         }
         PanelOpts pn = po;
         pn.bar_base = bar_next;
@@ -1871,9 +1879,50 @@ rrf_status_t rrf_run(rrf_handle_t h, const rrf_params_t* p, void* dA, int64_t ld
       UpdPlan up = plan_upd(gsms, rows, n, ops->u_bm, ops->u_bn, ops->u_wn);
       if (utc_on) up.tc = &utc;
       const int j0 = (i + 2 < steps) ? r0 + 2 * b : -1;   // Omega rows of the pass after the next
+      // Gated passes: the panel kernel, started together with the update, is done long before it, and its SMs
+      // would idle.  The last tiles of the pass are therefore left to a second launch of the update kernel that
+      // follows the panel kernel on ITS stream and so runs on the SMs it leaves: `look_ctas` CTAs with as many
+      // tiles as they can do in the time the first launch still needs (by the schedule model, with a wide margin).
+      int t1 = 0, tpc2 = 0;
+      if (gate && !look_cl && !utc_on && i + 1 < steps_run && !h->profiling) {
+        const PassModel pm{h->sms, (double)rows, (double)n, b, p->dtype == RRF_F64, tc, false};
+        const double t_upd = pm.upd() * pm.scale(look_ctas), t_pan = pm.panel_chain(look_ctas);
+        if (t_pan < 0.9 * t_upd) {
+          const double t_all = ((double)gsms * t_upd + (double)look_ctas * t_pan) / h->sms;   // both launches end together
+          // 0.35 of what the model allows: measured on 8192 x 8192, b = 64 (8.685 ms without the second launch):
+          // 8.654 / 8.607 / 8.653 / 8.94 / 9.28 ms with 0.2 / 0.4 / 0.6 / 0.8 / 1.0 of it
+          const double share = 0.35 * (double)look_ctas * (t_all - t_pan) / ((double)gsms * t_upd);
+          const int tiles_h = (int)(share * up.total);
+          if (tiles_h >= 4 * look_ctas) {
+            tpc2 = ceil_div(tiles_h, look_ctas);
+            t1 = up.total - tpc2 * look_ctas;
+          }
+        }
+      }
       mark(RRF_PHASE_UPDATE, i);
-      ops->update(tmV_u, tmZ, i == 0 ? tmA_u : tmW_u, tmO, W, ldw, (char*)dB + (size_t)r0 * ldb * esize, ldb, r0, rows, (int)n, r0, b,
-                  j0, Ybuf[i & 1], norm_part, up, ctrl, samp + i, st);
+      if (t1 > 0) {
+        UpdPlan um = up, uh = up;
+        um.total = t1;
+        um.tpc = ceil_div(t1, gsms);
+        um.P = ceil_div(t1, um.tpc);
+        uh.p0 = um.P;
+        uh.Lb = t1;
+        uh.tpc = tpc2;
+        uh.P = ceil_div(up.total - t1, tpc2);
+        ops->update(tmV_u, tmZ, i == 0 ? tmA_u : tmW_u, tmO, W, ldw, (char*)dB + (size_t)r0 * ldb * esize, ldb, r0, rows, (int)n,
+                    r0, b, j0, Ybuf[i & 1], norm_part, um, ctrl, samp + i, st);
+        // behind the panel kernel of pass i+1 on the side stream (which has waited for T Z of this pass)
+        ops->update(tmV_u, tmZ, i == 0 ? tmA_u : tmW_u, tmO, W, ldw, (char*)dB + (size_t)r0 * ldb * esize, ldb, r0, rows, (int)n,
+                    r0, b, j0, Ybuf[i & 1], norm_part, uh, ctrl, samp + i, h->aux);
+        cudaEventRecord(evH(i), h->aux);
+        cudaStreamWaitEvent(st, evH(i), 0);
+        up.tpc = um.tpc;          // what the loader of the sampled panel needs to find the partial results
+        up.P = um.P + uh.P;
+      } else {
+        ops->update(tmV_u, tmZ, i == 0 ? tmA_u : tmW_u, tmO, W, ldw, (char*)dB + (size_t)r0 * ldb * esize, ldb, r0, rows, (int)n, r0, b,
+                    j0, Ybuf[i & 1], norm_part, up, ctrl, samp + i, st);
+      }
+      const int up_t1 = t1, up_p1 = t1 > 0 ? ceil_div(t1, up.tpc) : 0, up_tpc2 = tpc2;
       mark(RRF_PHASE_STOP, i);
       stop_kernel<<<1, 256, 0, st>>>(norm_part, up.P, b, p->max_rank, p->estimator, fixed ? 1 : 0, tr_sub, tr_dir, ctrl,
                                      done_after, 0, predicting ? samp : nullptr, predict);
@@ -1890,6 +1939,9 @@ rrf_status_t rrf_run(rrf_handle_t h, const rrf_params_t* p, void* dA, int64_t ld
       }
       cudaEventRecord(evU(i), st);
       up_prev = up;
+      pv_t1 = up_t1;
+      pv_p1 = up_p1;
+      pv_tpc2 = up_tpc2;
     }
   }
   mark(RRF_PHASE_SKIPPED, steps);   // closing event

@@ -201,7 +201,8 @@ __global__ void __launch_bounds__((WM * WN + (PW ? 1 : 0)) * 32, 1)
                   int r0, int rows, int ncols, int cv0, int top_rows, int j0,
                   T* __restrict__ Ypart, double* __restrict__ norm_part,
                   int NC, int total, int tpc, Ctrl* ctrl,
-                  const int* __restrict__ samp_flag) {   // non-NULL: sample only if *samp_flag != 0
+                  const int* __restrict__ samp_flag,     // non-NULL: sample only if *samp_flag != 0
+                  int p0, int Lb) {                      // this launch is CTAs p0 ... of the pass and starts at tile Lb
   if (*reinterpret_cast<volatile int*>(&ctrl->done)) return;
   constexpr int KE = Elem<T>::KE, NV = Elem<T>::NV, KS = Elem<T>::KS;
   constexpr int U = KE / 8;            // n-tiles per 128-byte column group
@@ -225,9 +226,11 @@ __global__ void __launch_bounds__((WM * WN + (PW ? 1 : 0)) * 32, 1)
   __shared__ double red[64];
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
-  const int p = blockIdx.x;
-  const int L0 = p * tpc;
-  const int ntile = min(total, L0 + tpc) - L0;
+  // A pass may be split over two launches (the second one, on the SMs a finished panel kernel has left, takes the
+  // tiles from Lb on): CTA numbers, which name the partial-result slots, run on from the first launch's.
+  const int p = p0 + blockIdx.x;
+  const int L0 = Lb + blockIdx.x * tpc;
+  const int ntile = max(0, min(total, L0 + tpc) - L0);
   // the widest block size and single precision keep the host's decision (those instantiations are at
   // the register limit and lose 3-4 % with the extra test)
   constexpr bool kPredicted = B < 128 && sizeof(T) == 8;

@@ -169,7 +169,12 @@ struct PanelSource {
   int ldy;                 // stacked: leading dimension
   int row_off;             // panel row 0 is row `row_off` of the producer's row numbering
   int bm, nc, tpc, wn;     // slots: slab height, tiles per slab, tiles per CTA, warp columns
+  int t1, p1, tpc2;        // slots: tiles from t1 on belong to CTAs p1, p1 + 1, ... at tpc2 tiles each (t1 <= 0: none)
 };
+// CTA (= slot) that computed tile L of a pass
+__device__ __forceinline__ int slot_cta(const PanelSource& src, int L) {
+  return (src.t1 > 0 && L >= src.t1) ? src.p1 + (L - src.t1) / src.tpc2 : L / src.tpc;
+}
 
 // Look-ahead schedule (Section "Implementation", the two-queue variant): the panel was sampled from
 // the matrix BEFORE the previous block's reflectors were applied, P = W_old * Omega, so the kernel
@@ -199,7 +204,7 @@ __device__ __forceinline__ double panel_entry(const T* __restrict__ Y, const Pan
   } else {
     const int lr = r + src.row_off;
     const int sl = lr / src.bm, rl = lr - sl * src.bm;
-    const int p_lo = (sl * src.nc) / src.tpc, p_hi = ((sl + 1) * src.nc - 1) / src.tpc;
+    const int p_lo = slot_cta(src, sl * src.nc), p_hi = slot_cta(src, (sl + 1) * src.nc - 1);
     for (int p = p_lo; p <= p_hi; ++p)
       for (int w = 0; w < src.wn; ++w)
         s += (double)Y[((size_t)(p + sl) * src.wn + w) * (size_t)(src.bm * b) + (size_t)rl * b + c];
@@ -232,7 +237,7 @@ __device__ __forceinline__ void panel_load_slab(const T* __restrict__ Y, const P
         const int lr = gr0 + r - row0 + src.row_off;
         if (src.slots) {
           const int sl = lr / src.bm, rl = lr - sl * src.bm;
-          const int p_lo = (sl * src.nc) / src.tpc, p_hi = ((sl + 1) * src.nc - 1) / src.tpc;
+          const int p_lo = slot_cta(src, sl * src.nc), p_hi = slot_cta(src, (sl + 1) * src.nc - 1);
           cnt[e] = (p_hi - p_lo + 1) * src.wn;
           ptr[e] = Y + (size_t)(p_lo + sl) * src.wn * tstride + (size_t)rl * b + c;
         } else {
