@@ -228,9 +228,10 @@ __global__ void __launch_bounds__((WM * WN + (PW ? 1 : 0)) * 32, 1)
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
   // A pass may be split over two launches (the second one, on the SMs a finished panel kernel has left, takes the
   // tiles from Lb on): CTA numbers, which name the partial-result slots, run on from the first launch's.
-  const int p = p0 + blockIdx.x;
-  const int L0 = Lb + blockIdx.x * tpc;
-  const int ntile = max(0, min(total, L0 + tpc) - L0);
+  // (the widest block is never split: its instantiation has no register to spare)
+  const int p = (B >= 128 ? 0 : p0) + blockIdx.x;
+  const int L0 = (B >= 128 ? 0 : Lb) + blockIdx.x * tpc;
+  const int ntile = B >= 128 ? min(total, L0 + tpc) - L0 : max(0, min(total, L0 + tpc) - L0);
   // the widest block size and single precision keep the host's decision (those instantiations are at
   // the register limit and lose 3-4 % with the extra test)
   constexpr bool kPredicted = B < 128 && sizeof(T) == 8;
