@@ -136,3 +136,25 @@ def test_last_pass_without_a_sample_at_full_width(h):
     scale = out[MMA][2].abs().max().item()
     assert (out[MMA][1][128:] - out[TC][1][128:]).abs().max().item() <= 1e-4 * scale
     assert (out[MMA][2] - out[TC][2]).abs().max().item() <= 1e-4 * scale
+
+
+def test_single_precision_runs_are_bitwise_reproducible(h):
+    """Every reduction of the tcgen05 kernels and of the cluster panel kernel has a fixed order, and no result may
+    depend on which CTA or message arrives first: two hundred runs on both schedules give the same bits."""
+    rng = np.random.default_rng(3)
+    m, n, b, max_rank = 2304, 3136, 64, 384
+    A = (rng.standard_normal((m, 200)) @ rng.standard_normal((200, n)) / 14.0 + 1e-3 * rng.standard_normal((m, n))).astype(np.float32)
+    dA = torch.from_numpy(A).cuda()
+    dOmT = torch.from_numpy(rng.standard_normal((max_rank, n)).astype(np.float32)).cuda()
+    rrf.rrf_set_single_engine(h, TC, 2)
+    for flags in (rrf.RRF_FLAG_ONE_QUEUE, rrf.RRF_FLAG_TWO_QUEUES):
+        ref = None
+        for _ in range(200):
+            g = rrf.rrf_run(h, dA, b, 1e-3, max_rank, omegaT=dOmT, flags=flags)
+            cur = (g.k, g.status, g.V[:, :g.k].clone(), g.T[:, :g.k].clone(), g.B[:g.k].clone(), tuple(g.E_dir_trace[:g.steps]))
+            if ref is None:
+                ref = cur
+                assert g.k >= 2 * b
+            else:
+                assert cur[0] == ref[0] and cur[1] == ref[1] and cur[5] == ref[5]
+                assert torch.equal(cur[2], ref[2]) and torch.equal(cur[3], ref[3]) and torch.equal(cur[4], ref[4])
