@@ -13,6 +13,7 @@
 #include "gemm_sk.cuh"
 #include "gemm_tc.cuh"
 #include "gemm_tc_upd.cuh"
+#include "gemm_tc_vtw.cuh"
 #include "panel_blk.cuh"
 
 // NVTX ranges around the phases of rrf_run (host-side enqueue order), compiled in with -DRRF_NVTX only
@@ -499,9 +500,9 @@ struct Ops {
   static constexpr int V_STAGE = kVtwBK * (B + V_BN) * (int)sizeof(T);
   static constexpr int V_STAGES = (3 * V_STAGE + 1024 > 200 * 1024) ? 2 : (4 * V_STAGE + 1024 > 200 * 1024 ? 3 : 4);
   static constexpr int V_SMEM = V_STAGES * V_STAGE + 1024;
-  // vtw on tcgen05 (single precision only): stages of the TMA ring and of the (hi, lo) operand ring
   static constexpr int TC_B = (B == 16) ? 32 : B;
-  static constexpr int TC_RS = (B >= 128) ? 3 : 4, TC_OS = (B == 32) ? 3 : 2;
+  // vtw on tcgen05 (single precision only), W tile in tensor memory: stages of the TMA ring and of V's plane ring
+  static constexpr int TC_RS = (B >= 128) ? 5 : 6, TC_OS = 2;
   static_assert(TcCfg<TC_B, TC_RS, TC_OS>::SMEM + 1024 <= kMaxSmem, "shared memory");
   // fused update: slab height 128 (64 for the widest block), two 128-byte column groups per tile
   static constexpr int U_BM = (B >= 128) ? 64 : 128;
@@ -2180,9 +2181,6 @@ extern "C" rrf_status_t rrf_panel_qr_static(int32_t dtype, int64_t rows, int32_t
 }
 
 #ifdef RRF_TSQR_TRACE
-extern "C" int rrf_debug_trace_vtw(unsigned long long* out) {
-  return (int)cudaMemcpyFromSymbol(out, rrf::g_vtc_trace, sizeof(unsigned long long) * 16);
-}
 extern "C" int rrf_debug_trace_panel(unsigned long long* out) {
   return (int)cudaMemcpyFromSymbol(out, rrf::g_pcl_trace, sizeof(unsigned long long) * 16);
 }
