@@ -33,7 +33,7 @@ import numpy as np  # noqa: E402
 NCU_TRAFFIC_BYTES = {("cfg2", "update"): 1.07e9, ("cfg2", "vtw"): 136.3e6 * 3.875,
                      # tcgen05 kernels, block step 0 (profiles/kernels_cfg4_4096x11008_fp32_b64_tcgen05.md); of the update's
                      # 180 MB of writes 59 MB were still in L2 when the launch ended
-                     ("cfg4", "update"): 185.9e6 + 121.1e6, ("cfg4", "vtw"): 178.6e6 + 5.6e6}
+                     ("cfg4", "update"): 185.4e6 + 120.9e6, ("cfg4", "vtw"): 178.6e6 + 6.4e6}
 
 NOMINAL_FP64_OVER_BF16 = 37.0 / 2250.0   # HGX B200 dense figures: FP64 tensor 37 TF, bf16 2250 TF
 
