@@ -1,4 +1,4 @@
-// tcgen05 building blocks of the single-precision kernels (gemm_tc_vtw2.cuh, gemm_tc_upd.cuh): tensor-memory
+// tcgen05 building blocks of the single-precision kernels (gemm_tc_vtw.cuh, gemm_tc_upd.cuh): tensor-memory
 // allocation, loads and waits, commit, shared-memory operand descriptors, instruction descriptors, TF32 rounding.
 //
 // fp32 accuracy comes from the 3xTF32 split, x = hi + lo with hi = tf32(x), lo = tf32(x - hi),
