@@ -177,6 +177,40 @@ rrf_status_t rrf_run(rrf_handle_t h, const rrf_params_t* p,
                      double* h_E_sub_trace, double* h_E_dir_trace, double* h_E_est_trace);
 
 /*
+ * Column-major view of Algorithm 2 (the LAPACK / MAGMA storage of the paper's Section "Implementation").
+ *
+ * rrf_run_colmajor takes and returns every matrix stored column by column:
+ *   dA      m x n, lda >= m, read-only (RRF_FLAG_INPLACE is rejected);
+ *   dOmega  n x max_rank, ldo >= n (16-byte aligned, ldo a multiple of 16 bytes): column block i is Omega_i.
+ *           This is the same memory as rrf_run's dOmegaT.  NULL: drawn from p->seed;
+ *   dV      m x max_rank, ldv >= m; columns >= k unspecified;
+ *   dT      b x max_rank, leading dimension b: T_i in columns i*b ...;
+ *   dB      max_rank x n, ldb >= max_rank: the leading k x n block is B = Q^T A (may be NULL with RRF_FLAG_NO_UPDATE).
+ * No alignment is asked of dA, dV, dT, dB.  The call transposes A into a row-major working copy in the workspace
+ * (rrf_colmajor_workspace_bytes: rrf_run's workspace plus m*n + m*max_rank + b*max_rank elements), runs rrf_run
+ * on it in place with the same parameters, schedule and result fields, and transposes the k computed columns of
+ * V and T and the k rows of B into the caller's arrays; it costs one extra read and write of A and of the results.
+ * It synchronises the stream before it returns.  Values are those of rrf_run on the same matrices.
+ *
+ * rrf_transpose: dDst (cols x rows, ldd >= rows) = dSrc^T for dSrc rows x cols (lds >= cols), both row-major, not
+ * in place - equivalently a change between row- and column-major storage of one matrix.  It is what a caller with
+ * column-major data puts around rrf_apply_qt, rrf_apply_q, rrf_form_q and rrf_subspace_transfer, which are row-major
+ * only.  Does not synchronise the stream.
+ */
+rrf_status_t rrf_colmajor_workspace_bytes(const rrf_params_t* p, size_t* bytes);
+rrf_status_t rrf_run_colmajor(rrf_handle_t h, const rrf_params_t* p,
+                              const void* dA, int64_t lda,
+                              const void* dOmega, int64_t ldo,
+                              void* dV, int64_t ldv,
+                              void* dT,
+                              void* dB, int64_t ldb,
+                              void* d_workspace, size_t workspace_bytes,
+                              void* cuda_stream, rrf_result_t* out,
+                              double* h_E_sub_trace, double* h_E_dir_trace, double* h_E_est_trace);
+rrf_status_t rrf_transpose(rrf_handle_t h, int32_t dtype, int64_t rows, int64_t cols, const void* dSrc, int64_t lds,
+                           void* dDst, int64_t ldd, void* cuda_stream);
+
+/*
  * rrf_panel_qr - Algorithm 2 line 7 on its own (LAPACK geqrt semantics): Householder QR of a
  * tall device panel Y (rows x b, ldy >= b) into V (rows x b, ldv >= b, unit lower trapezoidal,
  * explicit ones and zeros) and the compact-WY factor T (b x b, ldt >= b, upper triangular) with

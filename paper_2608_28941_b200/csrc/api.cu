@@ -2097,6 +2097,122 @@ rrf_status_t rrf_run(rrf_handle_t h, const rrf_params_t* p, void* dA, int64_t ld
   return (rrf_status_t)hc.status;
 }
 
+// ------------------------------------------------------------------------------------------
+// Column-major view (the LAPACK / MAGMA convention of the paper's setting).  A column-major matrix is its
+// transpose stored row by row, so the entry points below transpose on the way in and on the way out and run
+// the row-major path in between, on a working copy that the update overwrites anyway.
+// ------------------------------------------------------------------------------------------
+static cudaError_t launch_transpose(const rrf_ctx* h, int dtype, long long rows, long long cols, const void* src,
+                                    long long lds, void* dst, long long ldd, cudaStream_t st) {
+  if (rows == 0 || cols == 0) return cudaSuccess;
+  const long long tiles = ((rows + 31) / 32) * ((cols + 31) / 32);
+  const int grid = (int)std::min<long long>(tiles, (long long)h->sms * 16);
+  if (dtype == RRF_F64)
+    transpose_kernel<double><<<grid, 256, 0, st>>>((const double*)src, lds, rows, cols, (double*)dst, ldd);
+  else
+    transpose_kernel<float><<<grid, 256, 0, st>>>((const float*)src, lds, rows, cols, (float*)dst, ldd);
+  return cudaGetLastError();
+}
+
+rrf_status_t rrf_transpose(rrf_handle_t h, int32_t dtype, int64_t rows, int64_t cols, const void* dSrc, int64_t lds,
+                           void* dDst, int64_t ldd, void* cuda_stream) {
+  if (h == nullptr || (dtype != RRF_F64 && dtype != RRF_F32) || rows < 0 || cols < 0 || lds < cols || ldd < rows)
+    return RRF_ERR_INVALID_ARG;
+  if (rows > 0 && cols > 0 && (dSrc == nullptr || dDst == nullptr || dSrc == dDst)) return RRF_ERR_INVALID_ARG;
+  const cudaError_t e = launch_transpose(h, dtype, rows, cols, dSrc, lds, dDst, ldd, (cudaStream_t)cuda_stream);
+  if (e != cudaSuccess) {
+    h->last_cuda = (int)e;
+    return RRF_ERR_CUDA;
+  }
+  return RRF_OK;
+}
+
+struct ColMajorLayout {
+  rrf_params_t q;          // the row-major run in the middle
+  size_t inner, at, v, t, total;
+  long long ldat;
+};
+static rrf_status_t colmajor_layout(const rrf_params_t* p, ColMajorLayout* L) {
+  const rrf_status_t s = check_params(p);
+  if (s != RRF_OK) return s;
+  if (p->flags & RRF_FLAG_INPLACE) return RRF_ERR_INVALID_ARG;   // the input is read-only here
+  L->q = *p;
+  if (!(p->flags & RRF_FLAG_NO_UPDATE)) L->q.flags |= RRF_FLAG_INPLACE;   // the transposed copy is the working matrix
+  const rrf_status_t s2 = check_params(&L->q);
+  if (s2 != RRF_OK) return s2;
+  const size_t esize = p->dtype == RRF_F64 ? 8 : 4;
+  const long long pad = 16 / (long long)esize;
+  L->ldat = (p->n + pad - 1) / pad * pad;
+  RunLayout R;
+  run_layout(&L->q, true, &R);
+  size_t off = align_up(R.total, 256);
+  L->inner = off;
+  L->at = off;
+  off += align_up((size_t)p->m * (size_t)L->ldat * esize, 256);
+  L->v = off;
+  off += align_up((size_t)p->m * (size_t)p->max_rank * esize, 256);
+  L->t = off;
+  off += align_up((size_t)p->b * (size_t)p->max_rank * esize, 256);
+  L->total = off;
+  return RRF_OK;
+}
+
+rrf_status_t rrf_colmajor_workspace_bytes(const rrf_params_t* p, size_t* bytes) {
+  if (bytes == nullptr) return RRF_ERR_INVALID_ARG;
+  ColMajorLayout L;
+  const rrf_status_t s = colmajor_layout(p, &L);
+  if (s != RRF_OK) return s;
+  *bytes = L.total;
+  return RRF_OK;
+}
+
+rrf_status_t rrf_run_colmajor(rrf_handle_t h, const rrf_params_t* p, const void* dA, int64_t lda, const void* dOmega,
+                              int64_t ldo, void* dV, int64_t ldv, void* dT, void* dB, int64_t ldb, void* d_workspace,
+                              size_t workspace_bytes, void* cuda_stream, rrf_result_t* out, double* h_E_sub_trace,
+                              double* h_E_dir_trace, double* h_E_est_trace) {
+  if (out == nullptr) return RRF_ERR_INVALID_ARG;
+  std::memset(out, 0, sizeof(*out));
+  auto fail = [&](rrf_status_t s) {
+    out->status = s;
+    return s;
+  };
+  if (h == nullptr) return fail(RRF_ERR_INVALID_ARG);
+  ColMajorLayout L;
+  const rrf_status_t s = colmajor_layout(p, &L);
+  if (s != RRF_OK) return fail(s);
+  const bool unchanged = (p->flags & RRF_FLAG_NO_UPDATE) != 0;
+  if (dA == nullptr || dV == nullptr || dT == nullptr || (dB == nullptr && !unchanged) || d_workspace == nullptr)
+    return fail(RRF_ERR_INVALID_ARG);
+  if (lda < p->m || ldv < p->m || (dB != nullptr && ldb < p->max_rank)) return fail(RRF_ERR_INVALID_ARG);
+  if (reinterpret_cast<uintptr_t>(d_workspace) & 255u) return fail(RRF_ERR_INVALID_ARG);
+  if (workspace_bytes < L.total) return fail(RRF_ERR_WORKSPACE);
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  unsigned char* ws = (unsigned char*)d_workspace;
+  void* At = ws + L.at;
+  void* Vr = ws + L.v;
+  void* Tr = ws + L.t;
+  auto cuda_fail = [&](cudaError_t e) {
+    h->last_cuda = (int)e;
+    out->cuda_error = (int)e;
+    return fail(RRF_ERR_CUDA);
+  };
+  // column-major m x n with leading dimension lda = row-major n x m with the same leading dimension
+  cudaError_t e = launch_transpose(h, p->dtype, p->n, p->m, dA, lda, At, L.ldat, st);
+  if (e != cudaSuccess) return cuda_fail(e);
+  const rrf_status_t r = rrf_run(h, &L.q, At, L.ldat, dOmega, ldo, Vr, p->max_rank, Tr, unchanged ? nullptr : At, L.ldat,
+                                 ws, L.inner, cuda_stream, out, h_E_sub_trace, h_E_dir_trace, h_E_est_trace);
+  if (r < 0) return r;
+  const int k = out->k;
+  e = launch_transpose(h, p->dtype, p->m, k, Vr, p->max_rank, dV, ldv, st);
+  // T_i goes to columns i b ... of a column-major b x max_rank array with leading dimension b
+  if (e == cudaSuccess) e = launch_transpose(h, p->dtype, p->b, k, Tr, p->max_rank, dT, p->b, st);
+  if (e == cudaSuccess && !unchanged) e = launch_transpose(h, p->dtype, k, p->n, At, L.ldat, dB, ldb, st);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+  if (e != cudaSuccess) return cuda_fail(e);
+  out->kernel_launches += 1 + (k > 0 ? (unchanged ? 2 : 3) : 0);
+  return r;
+}
+
 }  // extern "C"
 
 // ------------------------------------------------------------------------------------------

@@ -45,7 +45,7 @@ class rrf_profile_t(C.Structure):
     _fields_ = [("ms", C.c_double * 9), ("launches", C.c_int32 * 9), ("pad", C.c_int32)]
 
 
-EXPORTS = ["rrf_set_single_engine", "rrf_sample_workspace_bytes", "rrf_sample_panel", "rrf_frobenius_sq", "rrf_panel_qr_blocked", "rrf_panel_qr_tree", "rrf_transfer_workspace_bytes", "rrf_subspace_transfer", "rrf_selftest_timeout", "rrf_panel_qr_static", "rrf_set_profiling", "rrf_get_profile", "rrf_measure_peak", "rrf_create", "rrf_destroy", "rrf_workspace_bytes", "rrf_run", "rrf_panel_workspace_bytes",
+EXPORTS = ["rrf_run_colmajor", "rrf_colmajor_workspace_bytes", "rrf_transpose", "rrf_set_single_engine", "rrf_sample_workspace_bytes", "rrf_sample_panel", "rrf_frobenius_sq", "rrf_panel_qr_blocked", "rrf_panel_qr_tree", "rrf_transfer_workspace_bytes", "rrf_subspace_transfer", "rrf_selftest_timeout", "rrf_panel_qr_static", "rrf_set_profiling", "rrf_get_profile", "rrf_measure_peak", "rrf_create", "rrf_destroy", "rrf_workspace_bytes", "rrf_run", "rrf_panel_workspace_bytes",
            "rrf_panel_qr", "rrf_apply_workspace_bytes", "rrf_apply_qt", "rrf_apply_q", "rrf_form_q",
            "rrf_fill_omega", "rrf_last_status", "rrf_status_string"]
 
@@ -66,6 +66,9 @@ def load():
     lib.rrf_run.argtypes = [vp, C.POINTER(rrf_params_t), vp, i64, vp, i64, vp, i64, vp, vp, i64, vp, sz, vp,
                             C.POINTER(rrf_result_t), C.POINTER(C.c_double), C.POINTER(C.c_double),
                             C.POINTER(C.c_double)]
+    lib.rrf_run_colmajor.argtypes = lib.rrf_run.argtypes
+    lib.rrf_colmajor_workspace_bytes.argtypes = [C.POINTER(rrf_params_t), C.POINTER(sz)]
+    lib.rrf_transpose.argtypes = [vp, i32, i64, i64, vp, i64, vp, i64, vp]
     lib.rrf_panel_workspace_bytes.argtypes = [i32, i64, i32, C.POINTER(sz)]
     lib.rrf_panel_qr.argtypes = [vp, i32, i64, i32, vp, i64, vp, i64, vp, i64, vp, sz, vp]
     lib.rrf_panel_qr_tree.argtypes = [vp, i32, i64, i32, vp, i64, vp, i64, vp, i64, vp, sz, vp]
@@ -220,6 +223,61 @@ def rrf_run(h, A: torch.Tensor, b: int, tol: float, max_rank: int, omegaT: torch
     return RunResult(res.status, res.k, res.steps, res.normA2, res.sigma2, res.E_sub, res.E_dir,
                      list(tr_sub)[:res.steps], list(tr_dir)[:res.steps], V, T, B, res.queues, res.panel_ctas,
                      res.fused_samples, res.extra_samples, res.kernel_launches, list(tr_est)[:res.n_est])
+
+
+def _colmajor(t: torch.Tensor, name: str) -> int:
+    """Leading dimension of a 2-D column-major tensor (first stride 1)."""
+    if t.dim() != 2 or t.stride(0) != 1 or not t.is_cuda:
+        raise ValueError(f"{name} must be a 2-D CUDA tensor with unit stride along its columns")
+    return t.stride(1) if t.shape[1] > 1 else max(t.shape[0], t.stride(1))
+
+
+def rrf_run_colmajor(h, A: torch.Tensor, b: int, tol: float, max_rank: int, omega: torch.Tensor | None = None,
+                     relative: bool = True, estimator: int = 0, flags: int = 0, seed: int = 0,
+                     check: bool = True) -> RunResult:
+    """Algorithm 2 on column-major storage.  `A` (m x n) and `omega` (n x max_rank) are tensors whose FIRST stride
+    is 1 (e.g. `X.t()` of a contiguous X); V (m x max_rank), T (b x max_rank) and B (max_rank x n) come back as
+    such tensors too."""
+    lib = load()
+    m, n = A.shape
+    dt = _dtype_code(A)
+    p = make_params(dt, m, n, b, tol, max_rank, relative, estimator, flags, seed)
+    need = C.c_size_t()
+    s = lib.rrf_colmajor_workspace_bytes(C.byref(p), C.byref(need))
+    if s != RRF_OK:
+        raise RrfError(s, "rrf_colmajor_workspace_bytes")
+    dev = A.device
+    V = torch.empty((max_rank, m), dtype=A.dtype, device=dev).t()
+    T = torch.empty((max_rank, b), dtype=A.dtype, device=dev).t()
+    B = None if flags & RRF_FLAG_NO_UPDATE else torch.empty((n, max_rank), dtype=A.dtype, device=dev).t()
+    workspace = torch.empty(need.value, dtype=torch.uint8, device=dev)
+    res = rrf_result_t()
+    steps = max_rank // b
+    tr_sub = (C.c_double * steps)()
+    tr_dir = (C.c_double * steps)()
+    tr_est = (C.c_double * (steps + 1))()
+    om_ptr, ldo = (None, 0) if omega is None else (C.c_void_p(omega.data_ptr()), _colmajor(omega, "omega"))
+    s = lib.rrf_run_colmajor(h, C.byref(p), C.c_void_p(A.data_ptr()), _colmajor(A, "A"), om_ptr, ldo,
+                             C.c_void_p(V.data_ptr()), _colmajor(V, "V"), C.c_void_p(T.data_ptr()),
+                             None if B is None else C.c_void_p(B.data_ptr()), 0 if B is None else _colmajor(B, "B"),
+                             C.c_void_p(workspace.data_ptr()), workspace.numel(), _stream(), C.byref(res),
+                             tr_sub, tr_dir, tr_est)
+    if check and s < 0:
+        raise RrfError(s, "rrf_run_colmajor")
+    return RunResult(res.status, res.k, res.steps, res.normA2, res.sigma2, res.E_sub, res.E_dir,
+                     list(tr_sub)[:res.steps], list(tr_dir)[:res.steps], V, T, B, res.queues, res.panel_ctas,
+                     res.fused_samples, res.extra_samples, res.kernel_launches, list(tr_est)[:res.n_est])
+
+
+def rrf_transpose(h, src: torch.Tensor) -> torch.Tensor:
+    """A new row-major tensor holding src^T (src row-major)."""
+    rows, cols = src.shape
+    dst = _empty(cols, rows, src.dtype, src.device)
+    s = load().rrf_transpose(h, _dtype_code(src), rows, cols, C.c_void_p(src.data_ptr()), _rowmajor(src, "src"),
+                             C.c_void_p(dst.data_ptr()), _rowmajor(dst, "dst"), _stream())
+    if s != RRF_OK:
+        raise RrfError(s, "rrf_transpose")
+    return dst
 
 
 def rrf_panel_qr(h, Y: torch.Tensor, tree: bool = False, blocked: bool = False):
