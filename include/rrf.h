@@ -165,6 +165,15 @@ rrf_status_t rrf_workspace_bytes(const rrf_params_t* p, size_t* bytes);
  * A call whose arguments (parameters, pointers, leading dimensions, workspace) repeat those of
  * the previous call on this handle is captured into a CUDA graph and replayed on later repeats;
  * the buffers' CONTENTS may change freely between calls.  RRF_FLAG_NO_GRAPH disables this.
+ *
+ * Resuming.  A run made with RRF_FLAG_INPLACE that ended with RRF_MAX_RANK_REACHED at k0 = out->k leaves the
+ * residual in rows k0.. of dA, and the blocks still to come are Algorithm 2 on that residual.  To carry on up to a
+ * larger cap K call rrf_run again with m - k0 rows, max_rank = K - k0, the absolute tolerance
+ * tol = sqrt(out->sigma2) (tol_is_relative = 0), RRF_FLAG_INPLACE, and every pointer moved on:
+ * dA and dB to row k0, dV to row k0 and column k0 of an m x K array whose rows above k0 are zero in the new
+ * columns, dOmegaT to its row k0 (or rrf_fill_omega with first_vec = k0), dT to a b x (K - k0) array.  The second
+ * call's k, steps and traces continue the first one's; its normA2 is the residual's.  (The Python binding's
+ * rrf_resume does exactly this.)
  */
 rrf_status_t rrf_run(rrf_handle_t h, const rrf_params_t* p,
                      void* dA, int64_t lda,

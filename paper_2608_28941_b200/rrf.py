@@ -225,6 +225,35 @@ def rrf_run(h, A: torch.Tensor, b: int, tol: float, max_rank: int, omegaT: torch
                      res.fused_samples, res.extra_samples, res.kernel_launches, list(tr_est)[:res.n_est])
 
 
+def rrf_resume(h, W: torch.Tensor, prev: RunResult, b: int, max_rank: int, omegaT: torch.Tensor | None = None,
+               seed: int = 0, flags: int = 0) -> RunResult:
+    """Carry on a run that ended at its rank cap (status RRF_MAX_RANK_REACHED) up to the larger cap `max_rank`.
+
+    `W` is the matrix the earlier run worked on IN PLACE (RRF_FLAG_INPLACE): its rows [:prev.k] hold B, the rest is
+    the residual.  The blocks still to come are Algorithm 2 on that residual W[prev.k:, :] with the absolute
+    tolerance of the first run, so this is one more rrf_run call on offset pointers: V and B continue below and to
+    the right of what exists, the sample vectors continue at number prev.k (`omegaT`, max_rank x n, or the built-in
+    generator from `seed`).  Returns the merged result (V: m x max_rank, T: b x max_rank, B: rows of W)."""
+    k0 = prev.k
+    m, n = W.shape
+    if prev.status != RRF_MAX_RANK_REACHED or max_rank <= k0 or max_rank % b or k0 % b:
+        raise ValueError("rrf_resume continues a run that stopped at its cap, up to a larger cap that is a multiple of b")
+    V = _empty(m, max_rank, W.dtype, W.device)
+    V[:, :k0] = prev.V[:, :k0]
+    V[:k0, k0:].zero_()                      # the new blocks' reflectors start at row k0
+    if omegaT is None:
+        om = rrf_fill_omega(h, n, max_rank - k0, seed, dtype=W.dtype, first_vec=k0, device=W.device)
+    else:
+        om = omegaT[k0:max_rank]
+    r = rrf_run(h, W[k0:], b, float(prev.sigma2) ** 0.5, max_rank - k0, omegaT=om, relative=False,
+                flags=flags | RRF_FLAG_INPLACE, V=V[k0:, k0:], B=W[k0:max_rank])
+    T = torch.cat([prev.T[:, :k0], r.T], dim=1)
+    return RunResult(r.status, k0 + r.k, prev.steps + r.steps, prev.normA2, prev.sigma2, r.E_sub, r.E_dir,
+                     prev.E_sub_trace + r.E_sub_trace, prev.E_dir_trace + r.E_dir_trace, V, T, W[:max_rank], r.queues,
+                     r.panel_ctas, prev.fused_samples + r.fused_samples, prev.extra_samples + r.extra_samples,
+                     prev.kernel_launches + r.kernel_launches, [])
+
+
 def _colmajor(t: torch.Tensor, name: str) -> int:
     """Leading dimension of a 2-D column-major tensor (first stride 1)."""
     if t.dim() != 2 or t.stride(0) != 1 or not t.is_cuda:
