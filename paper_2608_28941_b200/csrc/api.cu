@@ -2105,7 +2105,8 @@ rrf_status_t rrf_run(rrf_handle_t h, const rrf_params_t* p, void* dA, int64_t ld
 static cudaError_t launch_transpose(const rrf_ctx* h, int dtype, long long rows, long long cols, const void* src,
                                     long long lds, void* dst, long long ldd, cudaStream_t st) {
   if (rows == 0 || cols == 0) return cudaSuccess;
-  const long long tiles = ((rows + 31) / 32) * ((cols + 31) / 32);
+  const long long d = dtype == RRF_F64 ? 32 : 64;      // the kernel's tile side
+  const long long tiles = ((rows + d - 1) / d) * ((cols + d - 1) / d);
   const int grid = (int)std::min<long long>(tiles, (long long)h->sms * 16);
   if (dtype == RRF_F64)
     transpose_kernel<double><<<grid, 256, 0, st>>>((const double*)src, lds, rows, cols, (double*)dst, ldd);

@@ -1228,21 +1228,23 @@ __global__ void __launch_bounds__(256) frob2_final_kernel(const double* __restri
 }
 
 // dst (cols x rows, leading dimension ldd) = src^T for a rows x cols matrix src (leading dimension lds), both stored
-// row by row: 32 x 32 tiles pass through shared memory so that reads and writes are both along rows.  This is all
-// the column-major entry points need: a column-major matrix is its transpose stored row by row.
+// row by row: square tiles of 256 bytes a side (32 doubles, 64 floats) pass through shared memory so that reads and
+// writes are both along rows.  This is all the column-major entry points need: a column-major matrix is its
+// transpose stored row by row.
 template <typename T>
 __global__ void __launch_bounds__(256)
     transpose_kernel(const T* __restrict__ src, long long lds, long long rows, long long cols, T* __restrict__ dst,
                      long long ldd) {
-  __shared__ T tile[32][33];
-  const long long tiles_c = (cols + 31) / 32, tiles = tiles_c * ((rows + 31) / 32);
-  const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
+  constexpr int D = 256 / (int)sizeof(T), RS = 256 / D;      // tile side; tile rows covered by one sweep of the block
+  __shared__ T tile[D][D + 1];
+  const long long tiles_c = (cols + D - 1) / D, tiles = tiles_c * ((rows + D - 1) / D);
+  const int tx = threadIdx.x % D, ty = threadIdx.x / D;
   for (long long t = blockIdx.x; t < tiles; t += gridDim.x) {
-    const long long r0 = (t / tiles_c) * 32, c0 = (t % tiles_c) * 32;
-    for (int i = ty; i < 32; i += 8)
+    const long long r0 = (t / tiles_c) * D, c0 = (t % tiles_c) * D;
+    for (int i = ty; i < D; i += RS)
       if (r0 + i < rows && c0 + tx < cols) tile[i][tx] = src[(r0 + i) * lds + c0 + tx];
     __syncthreads();
-    for (int i = ty; i < 32; i += 8)
+    for (int i = ty; i < D; i += RS)
       if (c0 + i < cols && r0 + tx < rows) dst[(c0 + i) * ldd + r0 + tx] = tile[tx][i];
     __syncthreads();
   }
