@@ -13,7 +13,7 @@ torch.distributed (NCCL over NVLink on GPUs) for the two all-reduces.  The loop 
 once per block (the reduced scalars have to be read anyway).  With `group=None` and no initialised process group
 it runs as a single rank.  V, T, k and the traces come out identical on every rank; B is the rank's column block.
 
-No TMA multicast or peer pointer is involved: remote data arrives through the all-reduce into this GPU's memory.
+No kernel reads another GPU's memory: remote data arrives through the all-reduce into this GPU's own memory.
 """
 from __future__ import annotations
 
