@@ -1,6 +1,6 @@
 """Seeded random sweep of shapes, block sizes, schedules and sampling modes against the oracle.
 
-Sixty small problems (ragged sizes, ranks from 1 to full, tolerances over eight decades, both precisions, both
+Four hundred small problems (ragged sizes, ranks from 1 to full, tolerances over eight decades, both precisions, both
 estimators, fixed-rank mode, one and two queues, every sampling mode).  Compared: k (unless the oracle's own
 stopping quantity sits within 1e-6 / 1e-2 of the threshold, where either answer is right), Q^T Q, and B and Q B
 block by block.  Block i is sampled from a residual of relative size sqrt(E_{i-1}/E_0) (E_{i-2} under the
@@ -8,7 +8,9 @@ look-ahead schedule, which samples one update early) that carries rounding noise
 rows of B are held to the plain bar times that amplification.  Which blocks are instead sampled from pure rounding
 noise is decided from the INPUT: the generated rank is known, and a block that starts at or beyond it (or whose
 residual, by the oracle's own trace, is within a factor 1e4 / 1e2 of the rounding floor) has no unique B or Q; for
-those the test checks what is unique: the residual norm and the orthogonality."""
+those the test checks what is unique: the residual norm and the orthogonality.  Inside a block, rows at or beyond
+the generated rank are not compared, and rows are compared up to sign from the first reflector whose pivot lies
+within the rounding noise of its sampled panel (the Householder sign rule is discontinuous there)."""
 import numpy as np
 import pytest
 import torch
@@ -32,7 +34,7 @@ def _pad(x, mult):
     return buf[:, :c]
 
 
-@pytest.mark.parametrize("seed", range(60))
+@pytest.mark.parametrize("seed", range(400))
 def test_random_problem(seed):
     rng = np.random.default_rng(9000 + seed)
     h = rrf.rrf_create(0)
@@ -83,6 +85,7 @@ def test_random_problem(seed):
         scaleB = np.max(np.abs(o.B[:k]))
         floor = (1e4 if dt == "f64" else 1e2) * max(m, n) * u
         unique = 0
+        signs_fixed = True
         for i in range(k // b):
             lag = 2 if (g.queues == 2 and i >= 2) else 1       # look-ahead: sampled one update earlier
             rel_res = np.sqrt(max(E[i], 0.0) / o.normA2)
@@ -90,7 +93,25 @@ def test_random_problem(seed):
                 break                                          # from here on the blocks are sampled from noise
             amp = np.sqrt(o.normA2 / max(E[i], 1e-300)) * np.sqrt(max(E[max(i - lag + 1, 0)], 0.0) / max(E[i], 1e-300))
             blk = slice(i * b, (i + 1) * b)
-            eB = np.max(np.abs(B[blk] - o.B[blk])) / scaleB
+            # Inside a block: rows at or beyond the generated rank are reflectors of rounding noise (nothing to
+            # compare), and the SIGN of a row is the sign of its reflector's pivot alpha_j (beta = -sign(alpha)
+            # ||x||).  The panel's triangular factor is R_i = B_i Omega_i, r_jj = beta_j, alpha_j = beta_j (1 -
+            # tau_j); a pivot within the rounding noise of the sampled panel, 64 u max|r_jj|, has no sign the
+            # input determines, and the other choice is an equally valid factorisation that also moves the
+            # pivots after it - so from the first such row on, rows are compared up to sign.
+            rows_i = min(b, rank - i * b)
+            Ti = o.T[:, blk]
+            rdiag = np.einsum("jn,nj->j", o.B[blk], Om64[:, blk])
+            alpha = rdiag * (1.0 - np.diag(Ti))
+            noise = 64 * u * np.max(np.abs(rdiag))
+            eB = 0.0
+            for j in range(rows_i):
+                if abs(alpha[j]) <= noise:
+                    signs_fixed = False
+                dj = np.max(np.abs(B[i * b + j] - o.B[i * b + j]))
+                if not signs_fixed:
+                    dj = min(dj, np.max(np.abs(B[i * b + j] + o.B[i * b + j])))
+                eB = max(eB, dj / scaleB)
             assert eB <= bar * max(1.0, amp), (i, eB, amp)
             unique = i + 1
         ku = unique * b
