@@ -201,12 +201,13 @@ class Problem:
         self.T = torch.empty((w.b, w.max_rank), dtype=self.tdt, device=dev)
         self.B = torch.empty((w.max_rank, w.n), dtype=self.tdt, device=dev)
 
-    def step(self, A=None, omegaT="resident", flags=0):
+    def step(self, A=None, omegaT="resident", flags=0, out=None):
         from paper_2608_28941_b200 import rrf
         w = self.w
         om = self.OmT if isinstance(omegaT, str) else omegaT
-        return rrf.rrf_run(self.h, self.A if A is None else A, w.b, w.tol, w.max_rank, omegaT=om, V=self.V, T=self.T,
-                           B=self.B, workspace=self.ws, flags=self.sched | flags, seed=w.seed, estimator=self.estimator, panel_ctas=self.panel_ctas)
+        V, T, B = (self.V, self.T, self.B) if out is None else out
+        return rrf.rrf_run(self.h, self.A if A is None else A, w.b, w.tol, w.max_rank, omegaT=om, V=V, T=T,
+                           B=B, workspace=self.ws, flags=self.sched | flags, seed=w.seed, estimator=self.estimator, panel_ctas=self.panel_ctas)
 
 
 def time_problem(pb, steps, warmup, world, barrier):
@@ -323,11 +324,15 @@ def e2e_of(pb, res, steps, world, barrier, flops):
     B_h = torch.empty((w.max_rank, w.n), dtype=pb.tdt).pin_memory()
     V_h = torch.empty((w.m, w.max_rank), dtype=pb.tdt).pin_memory()
     T_h = torch.empty((w.b, w.max_rank), dtype=pb.tdt).pin_memory()
-    # Two device input buffers: the input of step s+1 travels on a copy stream while step s computes and its
-    # results go back, as a caller that streams problems through the library would do.
+    # Two device input buffers and two sets of output buffers: the input of step s+1 travels on a copy stream and
+    # the results of step s-1 go back on another one while step s computes, as a caller that streams problems
+    # through the library would do (the link carries both directions at once).
     A_d = [torch.empty_like(pb.A), torch.empty_like(pb.A)]
+    outs = [(pb.V, pb.T, pb.B), (torch.empty_like(pb.V), torch.empty_like(pb.T), torch.empty_like(pb.B))]
     arrived = [torch.cuda.Event(), torch.cuda.Event()]
+    returned = [torch.cuda.Event(), torch.cuda.Event()]
     copy_stream = torch.cuda.Stream()
+    back_stream = torch.cuda.Stream()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
 
     # the pinned host-to-device rate on its own, to tell the link from the loop
@@ -353,18 +358,24 @@ def e2e_of(pb, res, steps, world, barrier, flops):
             if s + 1 < nsteps:
                 send(1 - slot)                 # the previous user of that slot has finished: rrf_run synchronises
             torch.cuda.current_stream().wait_event(arrived[slot])
-            r = pb.step(A=A_d[slot], omegaT=None, flags=rrf.RRF_FLAG_NO_GRAPH)   # the inputs alternate: nothing to replay
-            # B's rows are contiguous; V and T go back whole (a strided copy of their first k columns runs
-            # at 2 GB/s, the whole buffers at the link's rate)
-            B_h[:r.k].copy_(pb.B[:r.k], non_blocking=True)
-            V_h.copy_(pb.V, non_blocking=True)
-            T_h.copy_(pb.T, non_blocking=True)
+            if s >= 2:
+                torch.cuda.current_stream().wait_event(returned[slot])   # this set's results of step s-2 are on the host
+            V_d, T_d, B_d = outs[slot]
+            r = pb.step(A=A_d[slot], omegaT=None, flags=rrf.RRF_FLAG_NO_GRAPH, out=outs[slot])   # the inputs alternate: nothing to replay
+            # rrf_run has synchronised: the results are complete.  B's rows are contiguous; V and T go back whole (a
+            # strided copy of their first k columns runs at 2 GB/s, the whole buffers at the link's rate)
+            with torch.cuda.stream(back_stream):
+                B_h[:r.k].copy_(B_d[:r.k], non_blocking=True)
+                V_h.copy_(V_d, non_blocking=True)
+                T_h.copy_(T_d, non_blocking=True)
+                returned[slot].record(back_stream)
+        torch.cuda.current_stream().wait_stream(back_stream)     # the timed region ends when the last results are back
         torch.cuda.current_stream().synchronize()
         return r
 
     loop(2)
     barrier()
-    n_e2e = max(2, min(steps, 6))
+    n_e2e = max(2, min(steps, 12))
     e0.record()
     r = loop(n_e2e)
     e1.record()
@@ -376,8 +387,8 @@ def e2e_of(pb, res, steps, world, barrier, flops):
             "d2h_bytes_per_step": int((r.k * w.n + w.m * w.max_rank + w.b * w.max_rank) * pb.esize),
             "k": r.k, "omega": "drawn on the device from the seed (rrf_fill_omega), not copied",
             "pinned_h2d_gbs_alone": h2d_gbs,
-            "pipelined": "the input of step s+1 is copied on a second stream while step s computes; %d steps timed, "
-                         "first copy not overlapped" % n_e2e}
+            "pipelined": "the input of step s+1 is copied in on a second stream and the results of step s-1 out on a "
+                         "third while step s computes; %d steps timed, first copy in and last copy out not overlapped" % n_e2e}
 
 
 def main():
